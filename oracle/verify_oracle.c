@@ -1,0 +1,425 @@
+/*
+ * TEST INFRASTRUCTURE -- NOT PART OF THE PRODUCT PATH.
+ *
+ * Plain, slow, fp64 CPU statement of the two draft-verification procedures of
+ * "Block Verification Accelerates Speculative Decoding" (arXiv 2403.10444):
+ *
+ *   - Token Verification  (Algorithm 1, residual distribution Eq. "pres-token")
+ *   - Block Verification  (Algorithm 2, prefix recursion Eq. "def_as",
+ *                          residual distribution Eq. "pres-block",
+ *                          acceptance weights Eq. "pacc_block")
+ *
+ * It follows the algorithms step by step in the paper's order and notation,
+ * with no blocking, fusion or reordering.  It shares no code with the CUDA
+ * library, and only tests, the smoke check and the benchmark's CPU-baseline
+ * leg may call it.
+ *
+ * Pins (see tests/test_oracle_*.py): the paper's two-token worked example
+ * (expected accepted lengths 10/9 and 11/9), brute-force enumeration of every
+ * drafted block showing the output law equals the target model's (Theorem 1 /
+ * Eq. "output_block_distribution"), Lemma 3 (Pr(tau >= i | X^i) = p_i), the
+ * expected-length ordering of Theorem 2, the gamma = 1 coincidence of the two
+ * procedures, scipy's logsumexp for the normalisers, and explicit cumulative
+ * sums for the sampler.
+ *
+ * Notation (0-based storage rows, 1-based tokens):
+ *   P_r = softmax(target_logits[b, r, :] / T),  r = 0..gamma    (M_b(. | c, X^r))
+ *   Q_r = softmax(draft_logits [b, r, :] / T),  r = 0..gamma-1  (M_s(. | c, X^r))
+ *   X_i = draft_tokens[b, i-1],  eta_i = uniforms[b, i-1],  i = 1..gamma
+ *   uniforms[b, gamma]   drives the residual sample (tau < gamma)
+ *   uniforms[b, gamma+1] drives the target sample   (tau == gamma)
+ *
+ * Readings taken where the paper is silent (each is listed in the design doc):
+ *   - temperature divides both models' logits before the softmax;
+ *   - a position is selectable only if its acceptance weight is > 0, and
+ *     h_i := 0 when S_i = 0 (the 0/0 case of Eq. "pacc_block");
+ *   - sampling is inverse-CDF in vocabulary-index order with a strict
+ *     comparison: Y = min{k : C_k > u * W}; if rounding leaves none, the last
+ *     k with positive weight;
+ *   - a residual whose total mass is exactly 0 (P_tau == Q_tau bit for bit, a
+ *     probability-zero event) falls back to sampling P_tau with the same uniform;
+ *   - NaN / +inf logits in a row that is used, an all -inf row, a drafted token
+ *     outside [0, V) or one whose draft logit is -inf are per-sequence domain
+ *     errors: out_len = -1 and out_tokens = -1.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F64 = 2 };
+enum { ORACLE_TOKEN_VERIFY = 0, ORACLE_BLOCK_VERIFY = 1 };
+
+/* One logit, widened exactly to double. */
+static double logit_at(const void *base, int dtype, size_t idx)
+{
+    if (dtype == ORACLE_F32)
+        return (double)((const float *)base)[idx];
+    if (dtype == ORACLE_BF16) {
+        uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+    return ((const double *)base)[idx];
+}
+
+/* log sum_x exp(z_x / T) over one row; returns 0, or 1 on a domain error. */
+static int row_lse(const void *base, int dtype, size_t off, int V, double T,
+                   double *lse_out)
+{
+    double m = -INFINITY;
+    for (int x = 0; x < V; ++x) {
+        double z = logit_at(base, dtype, off + (size_t)x) / T;
+        if (isnan(z) || z == INFINITY)
+            return 1;
+        if (z > m)
+            m = z;
+    }
+    if (!isfinite(m))
+        return 1; /* every logit is -inf */
+    double s = 0.0;
+    for (int x = 0; x < V; ++x)
+        s += exp(logit_at(base, dtype, off + (size_t)x) / T - m);
+    *lse_out = m + log(s);
+    return 0;
+}
+
+/* softmax probability of token x in a row whose log-normaliser is lse */
+static double prob_at(const void *base, int dtype, size_t off, int x, double T,
+                      double lse)
+{
+    return exp(logit_at(base, dtype, off + (size_t)x) / T - lse);
+}
+
+/*
+ * Unnormalised sampling weight of token x at one position:
+ *   max(p * P(x) - Q(x), 0)   (Eq. "pres-block"; p = 1 gives Eq. "pres-token"),
+ * or P(x) itself when there is no draft row (the target sample at tau = gamma).
+ */
+static double weight_at(const void *tgt, size_t toff, double lse_t,
+                        const void *drf, size_t doff, double lse_d, int have_draft,
+                        int dtype, int x, double T, double p)
+{
+    double P = prob_at(tgt, dtype, toff, x, T, lse_t);
+    if (!have_draft)
+        return P;
+    double Q = prob_at(drf, dtype, doff, x, T, lse_d);
+    double w = p * P - Q;
+    return w > 0.0 ? w : 0.0;
+}
+
+/*
+ * Inverse-CDF sample in vocabulary-index order.  W = sum of weights and the
+ * running sums C_k are plain sequential fp64 sums.  Returns the token;
+ * *margin receives min(u - C_{k-1}/W, C_k/W - u), the distance (in probability)
+ * of u from the nearest edge of the chosen token's CDF cell.
+ */
+static int sample_index_order(const void *tgt, size_t toff, double lse_t,
+                              const void *drf, size_t doff, double lse_d,
+                              int have_draft, int dtype, int V, double T, double p,
+                              double u, double *W_out, double *margin)
+{
+    double W = 0.0;
+    for (int x = 0; x < V; ++x)
+        W += weight_at(tgt, toff, lse_t, drf, doff, lse_d, have_draft, dtype, x, T, p);
+    *W_out = W;
+    if (!(W > 0.0)) {
+        /* empty residual: sample the target row itself (reading, see header) */
+        have_draft = 0;
+        W = 0.0;
+        for (int x = 0; x < V; ++x)
+            W += weight_at(tgt, toff, lse_t, drf, doff, lse_d, 0, dtype, x, T, p);
+    }
+    double t = u * W, C = 0.0;
+    int last_pos = -1;
+    for (int x = 0; x < V; ++x) {
+        double w = weight_at(tgt, toff, lse_t, drf, doff, lse_d, have_draft, dtype, x, T, p);
+        double Cprev = C;
+        C += w;
+        if (w > 0.0)
+            last_pos = x;
+        if (C > t) {
+            double lo = u - Cprev / W, hi = C / W - u;
+            *margin = lo < hi ? lo : hi;
+            return x;
+        }
+    }
+    *margin = 0.0; /* u*W fell beyond the last running sum by rounding */
+    return last_pos;
+}
+
+/* Everything one sequence needs; rows are addressed by element offsets. */
+typedef struct {
+    const void *tgt, *drf;
+    const int32_t *X;   /* gamma drafted tokens */
+    const float *u;     /* gamma + 2 uniforms   */
+    int gamma, V, dtype;
+    double T;
+    size_t toff, doff;  /* offset of row 0 of this sequence in tgt / drf */
+} seq_t;
+
+typedef struct {
+    double *p, *S, *h, *lse_t, *lse_d; /* per-sequence slices, may be NULL */
+    double *margin_eta, *margin_smp;   /* one value each, may be NULL      */
+} diag_t;
+
+static void diag_fill_nan(const diag_t *d, int gamma)
+{
+    for (int i = 0; i <= gamma; ++i) {
+        if (d->p) d->p[i] = NAN;
+        if (d->h) d->h[i] = NAN;
+        if (d->lse_t) d->lse_t[i] = NAN;
+        if (i < gamma && d->S) d->S[i] = NAN;
+        if (i < gamma && d->lse_d) d->lse_d[i] = NAN;
+    }
+    if (d->margin_eta) *d->margin_eta = NAN;
+    if (d->margin_smp) *d->margin_smp = NAN;
+}
+
+static void emit(const seq_t *s, int tau, int Y, int32_t *out_tokens, int32_t *out_len)
+{
+    for (int i = 0; i <= s->gamma; ++i)
+        out_tokens[i] = -1;
+    if (tau < 0) { /* domain error */
+        *out_len = -1;
+        return;
+    }
+    for (int i = 0; i < tau; ++i)
+        out_tokens[i] = s->X[i];
+    out_tokens[tau] = Y;
+    *out_len = tau + 1; /* "Return X^tau, Y" */
+}
+
+/*
+ * ln of the ratio M_b(X_i | c, X^{i-1}) / M_s(X_i | c, X^{i-1})  (Algorithm 1
+ * "Set h_i", Algorithm 2 "Set p_i"): both distributions are the ones
+ * conditioned on X^{i-1}, i.e. storage row i-1.  Returns 1 on a domain error.
+ */
+static int log_ratio(const seq_t *s, int i, double lse_t, double lse_d, double *lr)
+{
+    int x = s->X[i - 1];
+    if (x < 0 || x >= s->V)
+        return 1;
+    size_t V = (size_t)s->V;
+    double zq = logit_at(s->drf, s->dtype, s->doff + (size_t)(i - 1) * V + (size_t)x);
+    double zp = logit_at(s->tgt, s->dtype, s->toff + (size_t)(i - 1) * V + (size_t)x);
+    if (zq == -INFINITY)
+        return 1; /* a token the draft model cannot have produced */
+    *lr = (zp / s->T - lse_t) - (zq / s->T - lse_d);
+    return 0;
+}
+
+/* ---------------- Algorithm 1: Token Verification ---------------- */
+static void token_verify_one(const seq_t *s, const diag_t *d,
+                             int32_t *out_tokens, int32_t *out_len)
+{
+    const int g = s->gamma;
+    const size_t V = (size_t)s->V;
+    double lse_t = 0.0, lse_d = 0.0, m_eta = INFINITY;
+    diag_fill_nan(d, g);
+
+    int tau = 0;
+    for (int i = 1; i <= g; ++i) {
+        /* the distributions conditioned on X^{i-1} */
+        if (row_lse(s->tgt, s->dtype, s->toff + (size_t)(i - 1) * V, s->V, s->T, &lse_t) ||
+            row_lse(s->drf, s->dtype, s->doff + (size_t)(i - 1) * V, s->V, s->T, &lse_d)) {
+            emit(s, -1, -1, out_tokens, out_len);
+            return;
+        }
+        if (d->lse_t) d->lse_t[i - 1] = lse_t;
+        if (d->lse_d) d->lse_d[i - 1] = lse_d;
+        double lr;
+        if (log_ratio(s, i, lse_t, lse_d, &lr)) {
+            emit(s, -1, -1, out_tokens, out_len);
+            return;
+        }
+        double ratio = exp(lr);
+        double h = ratio < 1.0 ? ratio : 1.0;       /* h_i^token = min(ratio, 1) */
+        if (d->h) d->h[i] = h;
+        double eta = (double)s->u[i - 1];
+        double gap = fabs(eta - h);
+        if (gap < m_eta) m_eta = gap;
+        if (h > 0.0 && eta <= h)
+            tau = i;
+        else
+            break;
+    }
+    if (d->h) d->h[0] = 1.0;
+
+    /* the distributions conditioned on X^tau */
+    if (row_lse(s->tgt, s->dtype, s->toff + (size_t)tau * V, s->V, s->T, &lse_t)) {
+        emit(s, -1, -1, out_tokens, out_len);
+        return;
+    }
+    if (d->lse_t) d->lse_t[tau] = lse_t;
+    int have_draft = tau < g;
+    if (have_draft) {
+        if (row_lse(s->drf, s->dtype, s->doff + (size_t)tau * V, s->V, s->T, &lse_d)) {
+            emit(s, -1, -1, out_tokens, out_len);
+            return;
+        }
+        if (d->lse_d) d->lse_d[tau] = lse_d;
+    }
+    double u = (double)s->u[have_draft ? g : g + 1];
+    double W, m_smp;
+    int Y = sample_index_order(s->tgt, s->toff + (size_t)tau * V, lse_t,
+                               s->drf, s->doff + (size_t)tau * V, lse_d,
+                               have_draft, s->dtype, s->V, s->T, 1.0, u, &W, &m_smp);
+    if (have_draft && d->S) d->S[tau] = W; /* residual mass sum_x max(P - Q, 0) */
+    if (d->margin_eta) *d->margin_eta = m_eta;
+    if (d->margin_smp) *d->margin_smp = m_smp;
+    emit(s, tau, Y, out_tokens, out_len);
+}
+
+/* ---------------- Algorithm 2: Block Verification ---------------- */
+static void block_verify_one(const seq_t *s, const diag_t *d,
+                             int32_t *out_tokens, int32_t *out_len)
+{
+    const int g = s->gamma;
+    const size_t V = (size_t)s->V;
+    diag_fill_nan(d, g);
+
+    double *lse_t = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *lse_d = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *p = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *S = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *h = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    int bad = 0;
+
+    /* the conditional distributions along the sample path */
+    for (int r = 0; r <= g && !bad; ++r) {
+        bad |= row_lse(s->tgt, s->dtype, s->toff + (size_t)r * V, s->V, s->T, &lse_t[r]);
+        if (r < g)
+            bad |= row_lse(s->drf, s->dtype, s->doff + (size_t)r * V, s->V, s->T, &lse_d[r]);
+    }
+
+    /* p_0 = 1;  p_i = min{ p_{i-1} * M_b(X_i|c,X^{i-1}) / M_s(X_i|c,X^{i-1}), 1 } */
+    p[0] = 1.0;
+    for (int i = 1; i <= g && !bad; ++i) {
+        double lr;
+        if (log_ratio(s, i, lse_t[i - 1], lse_d[i - 1], &lr)) {
+            bad = 1;
+            break;
+        }
+        double v = p[i - 1] * exp(lr);
+        p[i] = v < 1.0 ? v : 1.0;
+    }
+    if (bad) {
+        emit(s, -1, -1, out_tokens, out_len);
+        goto done;
+    }
+
+    /* S_i = sum_x max{ p_i * M_b(x|c,X^i) - M_s(x|c,X^i), 0 },  i = 0..gamma-1 */
+    for (int i = 0; i < g; ++i) {
+        double acc = 0.0;
+        for (int x = 0; x < s->V; ++x)
+            acc += weight_at(s->tgt, s->toff + (size_t)i * V, lse_t[i],
+                             s->drf, s->doff + (size_t)i * V, lse_d[i], 1,
+                             s->dtype, x, s->T, p[i]);
+        S[i] = acc;
+    }
+
+    /* h_gamma = p_gamma;  h_i = S_i / (S_i + 1 - p_i) for i < gamma */
+    h[0] = 1.0; /* tau = 0 is what remains when nothing is selected */
+    for (int i = 1; i < g; ++i)
+        h[i] = S[i] > 0.0 ? S[i] / (S[i] + 1.0 - p[i]) : 0.0;
+    h[g] = p[g];
+
+    /* tau = the largest i with eta_i <= h_i (every i is tried: "continue") */
+    int tau = 0;
+    double m_eta = INFINITY;
+    for (int i = 1; i <= g; ++i) {
+        double eta = (double)s->u[i - 1];
+        if (h[i] > 0.0 && eta <= h[i])
+            tau = i;
+    }
+    /* comparisons at i >= tau decide the outcome; those below tau do not */
+    for (int i = (tau > 0 ? tau : 1); i <= g; ++i) {
+        double gap = fabs((double)s->u[i - 1] - h[i]);
+        if (gap < m_eta) m_eta = gap;
+    }
+
+    {
+        int have_draft = tau < g;
+        double u = (double)s->u[have_draft ? g : g + 1];
+        double W, m_smp;
+        int Y = sample_index_order(s->tgt, s->toff + (size_t)tau * V, lse_t[tau],
+                                   s->drf, s->doff + (size_t)tau * V, lse_d[tau],
+                                   have_draft, s->dtype, s->V, s->T, p[tau], u, &W, &m_smp);
+        if (d->margin_eta) *d->margin_eta = m_eta;
+        if (d->margin_smp) *d->margin_smp = m_smp;
+        emit(s, tau, Y, out_tokens, out_len);
+    }
+    for (int i = 0; i <= g; ++i) {
+        if (d->p) d->p[i] = p[i];
+        if (d->h) d->h[i] = h[i];
+        if (d->lse_t) d->lse_t[i] = lse_t[i];
+        if (i < g && d->S) d->S[i] = S[i];
+        if (i < g && d->lse_d) d->lse_d[i] = lse_d[i];
+    }
+done:
+    free(lse_t); free(lse_d); free(p); free(S); free(h);
+}
+
+/*
+ * Batch entry.  All pointers are host pointers.
+ *   algo: 0 = Token Verification, 1 = Block Verification
+ *   target [B, gamma+1, V], draft [B, gamma, V] in dtype (0 f32, 1 bf16 bits, 2 f64)
+ *   tokens [B, gamma] int32, uniforms [B, gamma+2] f32
+ *   out_tokens [B, gamma+1], out_len [B]
+ *   diagnostics (each may be NULL): p [B,gamma+1], S [B,gamma], h [B,gamma+1],
+ *   lse_t [B,gamma+1], lse_d [B,gamma], margin_eta [B], margin_smp [B].
+ *   Values an algorithm never forms are NaN (Token Verification forms h_i up to
+ *   the first rejection, S only at tau, and no p).
+ * Sequences are independent; the loop over b may run on several threads.
+ * Returns 0, or 1 for an invalid argument.
+ */
+int oracle_verify(int algo, const void *target, const void *draft,
+                  const int32_t *tokens, const float *uniforms,
+                  int B, int gamma, int V, int dtype, double temperature,
+                  int32_t *out_tokens, int32_t *out_len,
+                  double *p, double *S, double *h, double *lse_t, double *lse_d,
+                  double *margin_eta, double *margin_smp)
+{
+    if (!target || !draft || !tokens || !uniforms || !out_tokens || !out_len)
+        return 1;
+    if (B < 0 || gamma < 1 || V < 1 || !(temperature > 0.0) || !isfinite(temperature))
+        return 1;
+    if (dtype < 0 || dtype > 2 || (algo != 0 && algo != 1))
+        return 1;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int b = 0; b < B; ++b) {
+        seq_t s;
+        s.tgt = target; s.drf = draft;
+        s.X = tokens + (size_t)b * (size_t)gamma;
+        s.u = uniforms + (size_t)b * (size_t)(gamma + 2);
+        s.gamma = gamma; s.V = V; s.dtype = dtype; s.T = temperature;
+        s.toff = (size_t)b * (size_t)(gamma + 1) * (size_t)V;
+        s.doff = (size_t)b * (size_t)gamma * (size_t)V;
+        diag_t d;
+        d.p = p ? p + (size_t)b * (size_t)(gamma + 1) : NULL;
+        d.S = S ? S + (size_t)b * (size_t)gamma : NULL;
+        d.h = h ? h + (size_t)b * (size_t)(gamma + 1) : NULL;
+        d.lse_t = lse_t ? lse_t + (size_t)b * (size_t)(gamma + 1) : NULL;
+        d.lse_d = lse_d ? lse_d + (size_t)b * (size_t)gamma : NULL;
+        d.margin_eta = margin_eta ? margin_eta + b : NULL;
+        d.margin_smp = margin_smp ? margin_smp + b : NULL;
+        int32_t *ot = out_tokens + (size_t)b * (size_t)(gamma + 1);
+        if (algo == ORACLE_BLOCK_VERIFY)
+            block_verify_one(&s, &d, ot, out_len + b);
+        else
+            token_verify_one(&s, &d, ot, out_len + b);
+    }
+    return 0;
+}
+
+/* Number of threads the batch loop uses (1 when built without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_threads(void) { return omp_get_max_threads(); }
+#else
+int oracle_threads(void) { return 1; }
+#endif
