@@ -1,0 +1,142 @@
+/*
+ * bv.h -- C ABI of the batched draft-verification step of speculative decoding
+ * ("Block Verification Accelerates Speculative Decoding", arXiv 2403.10444)
+ * for NVIDIA B200 (sm_100a).
+ *
+ * One call verifies B independent drafted blocks of gamma tokens each.
+ *
+ * Notation (0-based storage rows, 1-based tokens), T = temperature:
+ *   P_r = softmax(target_logits[b, r, :] / T), r = 0..gamma    -- M_b(. | c, X^r)
+ *   Q_r = softmax(draft_logits [b, r, :] / T), r = 0..gamma-1  -- M_s(. | c, X^r)
+ *   X_i = draft_tokens[b, i-1], i = 1..gamma, drawn from Q_{i-1}
+ *   eta_i = uniforms[b, i-1], i = 1..gamma      (acceptance tests)
+ *   uniforms[b, gamma]    drives the residual sample (tau < gamma)
+ *   uniforms[b, gamma+1]  drives the target sample   (tau = gamma)
+ *
+ * Layout: every tensor is dense, row-major, contiguous.  dtype selects the
+ * logit storage type; all arithmetic is fp32 per element with fp64 combination
+ * of partial sums and an fp64 scalar recursion.
+ *
+ * Sampling is inverse-CDF in vocabulary-index order with weights w_x >= 0,
+ * W = sum w, C_k = sum_{x<=k} w_x:  Y = min{k : C_k > u * W}.
+ *
+ * Ownership: the caller owns every buffer; inputs are never written.  The
+ * device entry points enqueue work on `stream` and return without
+ * synchronising; buffers must stay valid until that work has completed.
+ *
+ * Errors: every entry point returns BV_OK (0) or a negative bv_status; nothing
+ * is launched when an argument is rejected.  Data faults are per sequence: a
+ * NaN or +inf logit in a row the algorithm reads, a row of all -inf, a drafted
+ * token outside [0, V) or whose draft logit is -inf give out_len[b] = -1 and
+ * out_tokens[b, :] = -1; other sequences are unaffected.
+ */
+#ifndef BV_H_
+#define BV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum bv_status {
+    BV_OK = 0,
+    BV_ERR_INVALID_ARG = -1,  /* null pointer, B < 0, gamma < 1, V < 1, T <= 0 or not finite,
+                                 unknown dtype, pointer not aligned to its element size */
+    BV_ERR_UNSUPPORTED = -2,  /* gamma > BV_MAX_GAMMA, or no sm_100 device              */
+    BV_ERR_CUDA = -3,         /* a CUDA runtime call failed; see bv_last_cuda_error()   */
+    BV_ERR_TIMEOUT = -4       /* a bounded device-side wait gave up (reported by the
+                                 host-buffer entry points, which synchronise)           */
+} bv_status;
+
+enum { BV_DTYPE_F32 = 0, BV_DTYPE_BF16 = 1 };
+enum { BV_MAX_GAMMA = 64 };
+
+/*
+ * Block Verification: Algorithm 2 with Eq. "def_as" (p_0 = 1,
+ * p_i = min(p_{i-1} P_{i-1}(X_i)/Q_{i-1}(X_i), 1)), Eq. "pacc_block"
+ * (S_i = sum_x max(p_i P_i(x) - Q_i(x), 0); h_gamma = p_gamma,
+ * h_i = S_i / (S_i + 1 - p_i), taken as 0 when S_i = 0), tau = the largest i
+ * with h_i > 0 and eta_i <= h_i (0 if none), and Y drawn from Eq. "pres-block"
+ * at position tau, or from P_gamma when tau = gamma.
+ *
+ * All pointers are DEVICE pointers.
+ *   target_logits [B, gamma+1, V]  dtype      draft_logits [B, gamma, V]  dtype
+ *   draft_tokens  [B, gamma]  int32           uniforms     [B, gamma+2]  float in [0,1)
+ *   out_tokens    [B, gamma+1] int32: X_1..X_tau, Y, then -1
+ *   out_len       [B] int32: tau + 1, or -1 for a sequence with a data fault
+ *   stream        a cudaStream_t (NULL = the default stream)
+ * Rows whose byte length is a multiple of 16 with 16-byte aligned bases use the
+ * 128-bit path; any other V >= 1 is served by an element-wise path.
+ */
+int bv_verify(const void* target_logits, const void* draft_logits,
+              const int32_t* draft_tokens, const float* uniforms,
+              int B, int gamma, int V, int dtype, float temperature,
+              int32_t* out_tokens, int32_t* out_len, void* stream);
+
+/*
+ * Token Verification: Algorithm 1 with Eq. "accept_probability"
+ * (h_i = min(P_{i-1}(X_i)/Q_{i-1}(X_i), 1)); tau = length of the initial run of
+ * i with h_i > 0 and eta_i <= h_i; Y from Eq. "pres-token" at position tau, or
+ * from P_gamma when tau = gamma.  Only rows 0..tau are read.  Arguments as for
+ * bv_verify.
+ */
+int tv_verify(const void* target_logits, const void* draft_logits,
+              const int32_t* draft_tokens, const float* uniforms,
+              int B, int gamma, int V, int dtype, float temperature,
+              int32_t* out_tokens, int32_t* out_len, void* stream);
+
+/*
+ * The same two procedures, also writing their intermediates (device pointers,
+ * float, any of which may be NULL):
+ *   out_p     [B, gamma+1]  p_0..p_gamma                (Eq. "def_as"; NaN for tv)
+ *   out_S     [B, gamma]    S_0..S_{gamma-1}            (tv: only S_tau, NaN elsewhere)
+ *   out_h     [B, gamma+1]  h_0 := 1, h_1..h_gamma      (tv: up to the first rejection)
+ *   out_lse_t [B, gamma+1]  ln sum_x exp(target/T) per row (NaN for rows not read)
+ *   out_lse_d [B, gamma]    ln sum_x exp(draft/T)  per row
+ */
+int bv_verify_ex(const void* target_logits, const void* draft_logits,
+                 const int32_t* draft_tokens, const float* uniforms,
+                 int B, int gamma, int V, int dtype, float temperature,
+                 int32_t* out_tokens, int32_t* out_len,
+                 float* out_p, float* out_S, float* out_h,
+                 float* out_lse_t, float* out_lse_d, void* stream);
+int tv_verify_ex(const void* target_logits, const void* draft_logits,
+                 const int32_t* draft_tokens, const float* uniforms,
+                 int B, int gamma, int V, int dtype, float temperature,
+                 int32_t* out_tokens, int32_t* out_len,
+                 float* out_p, float* out_S, float* out_h,
+                 float* out_lse_t, float* out_lse_d, void* stream);
+
+/*
+ * Host-buffer forms of Algorithm 2 / Algorithm 1: every pointer is a HOST
+ * pointer (pinned memory makes the copies asynchronous).  The call copies the
+ * inputs to device staging buffers owned by the library (grown on demand, kept
+ * until bv_release()), runs the device path on the current device, copies
+ * out_tokens and out_len back, and returns after they have landed.
+ */
+int bv_verify_host(const void* target_logits, const void* draft_logits,
+                   const int32_t* draft_tokens, const float* uniforms,
+                   int B, int gamma, int V, int dtype, float temperature,
+                   int32_t* out_tokens, int32_t* out_len);
+int tv_verify_host(const void* target_logits, const void* draft_logits,
+                   const int32_t* draft_tokens, const float* uniforms,
+                   int B, int gamma, int V, int dtype, float temperature,
+                   int32_t* out_tokens, int32_t* out_len);
+
+/* Frees the library's cached device buffers on the current device. */
+int bv_release(void);
+
+/* Number of kernel launches the last device-path call on this thread enqueued. */
+int bv_last_launch_count(void);
+/* cudaError_t value of the last failing runtime call on this thread (0 if none). */
+int bv_last_cuda_error(void);
+/* Static description of a bv_status value. */
+const char* bv_status_string(int status);
+/* Library version: major * 10000 + minor * 100 + patch. */
+int bv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BV_H_ */

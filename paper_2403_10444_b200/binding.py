@@ -1,0 +1,195 @@
+"""ctypes binding of libbv_b200.so: argument marshalling only.
+
+Every step of the verification path runs inside the CUDA library; nothing here
+computes.  There is no CPU fallback: if the library is missing, or an entry
+point reports an error, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libbv_b200.so")
+
+DTYPE_F32 = 0
+DTYPE_BF16 = 1
+
+# every symbol include/bv.h declares
+EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
+           "tv_verify_host", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
+           "bv_status_string", "bv_version"]
+
+
+class BVError(RuntimeError):
+    """An entry point of libbv_b200.so returned a non-zero status."""
+
+    def __init__(self, status: int, text: str):
+        super().__init__("libbv_b200: %s (status %d)" % (text, status))
+        self.status = status
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Load libbv_b200.so (built by ``python -m paper_2403_10444_b200.build``)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _LIB_PATH
+    if not os.path.exists(p):
+        raise RuntimeError(
+            "CUDA library %s is missing: build it with `python -m paper_2403_10444_b200.build` "
+            "(there is no CPU fallback)" % p)
+    lib = ctypes.CDLL(p)
+    vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    base = [vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp]
+    for name in ("bv_verify", "tv_verify"):
+        getattr(lib, name).argtypes = base + [vp]
+    for name in ("bv_verify_ex", "tv_verify_ex"):
+        getattr(lib, name).argtypes = base + [vp, vp, vp, vp, vp, vp]
+    for name in ("bv_verify_host", "tv_verify_host"):
+        getattr(lib, name).argtypes = base
+    for name in EXPORTS:
+        getattr(lib, name).restype = ci
+    lib.bv_status_string.restype = ctypes.c_char_p
+    lib.bv_status_string.argtypes = [ci]
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def bv_status_string(status: int) -> str:
+    return load_library().bv_status_string(int(status)).decode()
+
+
+def bv_version() -> int:
+    return int(load_library().bv_version())
+
+
+def bv_last_launch_count() -> int:
+    return int(load_library().bv_last_launch_count())
+
+
+def bv_release() -> None:
+    _check(load_library().bv_release())
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        lib = load_library()
+        text = lib.bv_status_string(int(status)).decode()
+        if status == -3:
+            text += " (cudaError %d)" % lib.bv_last_cuda_error()
+        raise BVError(status, text)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    raise TypeError("logits must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _shapes(target, draft, tokens, uniforms, want_cuda: bool):
+    if target.dim() != 3 or draft.dim() != 3:
+        raise ValueError("target_logits must be [B, gamma+1, V] and draft_logits [B, gamma, V]")
+    B, g1, V = target.shape
+    gamma = g1 - 1
+    if tuple(draft.shape) != (B, gamma, V):
+        raise ValueError("draft_logits must be [B, gamma, V]")
+    if tuple(tokens.shape) != (B, gamma) or tokens.dtype != torch.int32:
+        raise ValueError("draft_tokens must be int32 [B, gamma]")
+    if tuple(uniforms.shape) != (B, gamma + 2) or uniforms.dtype != torch.float32:
+        raise ValueError("uniforms must be float32 [B, gamma+2]")
+    if target.dtype != draft.dtype:
+        raise TypeError("target and draft logits must share a dtype")
+    for t in (target, draft, tokens, uniforms):
+        if not t.is_contiguous():
+            raise ValueError("all tensors must be contiguous")
+        if t.is_cuda != want_cuda:
+            raise ValueError("expected %s tensors" % ("CUDA" if want_cuda else "host"))
+    return B, gamma, V
+
+
+def _device_call(name: str, target, draft, tokens, uniforms, temperature, diagnostics: bool,
+                 stream: Optional[torch.cuda.Stream]):
+    lib = load_library()
+    B, gamma, V = _shapes(target, draft, tokens, uniforms, True)
+    dev = target.device
+    out_tokens = torch.empty((B, gamma + 1), dtype=torch.int32, device=dev)
+    out_len = torch.empty((B,), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        s = stream if stream is not None else torch.cuda.current_stream(dev)
+        args = [target.data_ptr(), draft.data_ptr(), tokens.data_ptr(), uniforms.data_ptr(),
+                B, gamma, V, _dtype_code(target), float(temperature),
+                out_tokens.data_ptr(), out_len.data_ptr()]
+        if diagnostics:
+            f = lambda *shape: torch.empty(shape, dtype=torch.float32, device=dev)
+            diag = dict(p=f(B, gamma + 1), S=f(B, gamma), h=f(B, gamma + 1),
+                        lse_t=f(B, gamma + 1), lse_d=f(B, gamma))
+            args += [diag[k].data_ptr() for k in ("p", "S", "h", "lse_t", "lse_d")]
+        _check(getattr(lib, name)(*args, s.cuda_stream))
+    if diagnostics:
+        return out_tokens, out_len, diag
+    return out_tokens, out_len
+
+
+def bv_verify(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+              stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Block Verification (Algorithm 2) on CUDA tensors; returns (out_tokens, out_len)."""
+    return _device_call("bv_verify", target_logits, draft_logits, draft_tokens, uniforms,
+                        temperature, False, stream)
+
+
+def tv_verify(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+              stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Token Verification (Algorithm 1) on CUDA tensors; returns (out_tokens, out_len)."""
+    return _device_call("tv_verify", target_logits, draft_logits, draft_tokens, uniforms,
+                        temperature, False, stream)
+
+
+def bv_verify_ex(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                 stream=None):
+    """bv_verify plus its intermediates: returns (out_tokens, out_len, dict(p, S, h, lse_t, lse_d))."""
+    return _device_call("bv_verify_ex", target_logits, draft_logits, draft_tokens, uniforms,
+                        temperature, True, stream)
+
+
+def tv_verify_ex(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                 stream=None):
+    """tv_verify plus its intermediates (NaN where Algorithm 1 forms none)."""
+    return _device_call("tv_verify_ex", target_logits, draft_logits, draft_tokens, uniforms,
+                        temperature, True, stream)
+
+
+def _host_call(name: str, target, draft, tokens, uniforms, temperature, out_tokens, out_len):
+    lib = load_library()
+    B, gamma, V = _shapes(target, draft, tokens, uniforms, False)
+    if out_tokens is None:
+        out_tokens = torch.empty((B, gamma + 1), dtype=torch.int32).pin_memory()
+    if out_len is None:
+        out_len = torch.empty((B,), dtype=torch.int32).pin_memory()
+    _check(getattr(lib, name)(target.data_ptr(), draft.data_ptr(), tokens.data_ptr(),
+                              uniforms.data_ptr(), B, gamma, V, _dtype_code(target),
+                              float(temperature), out_tokens.data_ptr(), out_len.data_ptr()))
+    return out_tokens, out_len
+
+
+def bv_verify_host(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                   out_tokens=None, out_len=None):
+    """Block Verification on HOST tensors (pinned for speed): copies in, runs, copies out."""
+    return _host_call("bv_verify_host", target_logits, draft_logits, draft_tokens, uniforms,
+                      temperature, out_tokens, out_len)
+
+
+def tv_verify_host(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                   out_tokens=None, out_len=None):
+    """Token Verification on HOST tensors (pinned for speed): copies in, runs, copies out."""
+    return _host_call("tv_verify_host", target_logits, draft_logits, draft_tokens, uniforms,
+                      temperature, out_tokens, out_len)

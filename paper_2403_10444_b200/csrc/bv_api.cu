@@ -1,0 +1,260 @@
+// C-ABI layer: argument checks, per-device workspace, launch-shape selection and
+// the host-buffer entry points.  Declarations and contracts are in include/bv.h.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+#include <mutex>
+
+#include "../../include/bv.h"
+#include "bv_launch.h"
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr int kTicketSlots = 64;  // concurrent calls on one device each need their own slot
+
+struct DeviceState {
+    bool ready = false;
+    int sm_count = 0;
+    int cc_major = 0;
+    unsigned int* tickets = nullptr;  // [kTicketSlots][2], zero when idle
+    unsigned long long calls = 0;
+    int max_clusters[2][2][2][bv::kMaxCluster + 1] = {};  // [algo][dtype][vec][cluster], 0 = not asked yet
+    // staging for the host-buffer entry points
+    void* stage = nullptr;
+    size_t stage_bytes = 0;
+    cudaStream_t stream = nullptr;
+};
+
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mu;
+
+thread_local int t_last_launches = 0;
+thread_local int t_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e) {
+    t_last_cuda_error = static_cast<int>(e);
+    cudaGetLastError();
+    return BV_ERR_CUDA;
+}
+
+// Per-device set-up on first use: device attributes and the ticket slots.
+int device_state(DeviceState** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return BV_ERR_UNSUPPORTED;
+    DeviceState& d = g_dev[dev];
+    if (!d.ready) {
+        if ((e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return cuda_fail(e);
+        if ((e = cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
+            return cuda_fail(e);
+        if (d.cc_major < 10) return BV_ERR_UNSUPPORTED;
+        if ((e = cudaMalloc(&d.tickets, sizeof(unsigned int) * 2 * kTicketSlots)) != cudaSuccess)
+            return cuda_fail(e);
+        if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned int) * 2 * kTicketSlots)) != cudaSuccess)
+            return cuda_fail(e);
+        d.ready = true;
+    }
+    *out = &d;
+    return BV_OK;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_args(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+               int V, int dtype, float T, const int32_t* ot, const int32_t* ol) {
+    if (!tgt || !drf || !tok || !uni || !ot || !ol) return BV_ERR_INVALID_ARG;
+    if (B < 0 || gamma < 1 || V < 1) return BV_ERR_INVALID_ARG;
+    if (!(T > 0.f) || !std::isfinite(T)) return BV_ERR_INVALID_ARG;
+    if (dtype != BV_DTYPE_F32 && dtype != BV_DTYPE_BF16) return BV_ERR_INVALID_ARG;
+    const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
+    if (!aligned(tgt, esz) || !aligned(drf, esz) || !aligned(tok, 4) || !aligned(uni, 4) ||
+        !aligned(ot, 4) || !aligned(ol, 4))
+        return BV_ERR_INVALID_ARG;
+    if (gamma > BV_MAX_GAMMA) return BV_ERR_UNSUPPORTED;
+    return BV_OK;
+}
+
+// Cluster width for the streaming kernel: wide enough that a CTA's slice of a row
+// is at most 64 KB, widened further while the batch alone cannot fill the SMs.
+int pick_cluster(const DeviceState& d, int B, size_t row_bytes) {
+    if (const char* env = std::getenv("BV_CLUSTER")) {
+        int c = std::atoi(env);
+        if (c == 1 || c == 2 || c == 4 || c == 8) return c;
+    }
+    int c = 1;
+    while (c < bv::kMaxCluster && row_bytes / c > (64u << 10)) c *= 2;
+    while (c < bv::kMaxCluster && static_cast<long long>(B) * c < d.sm_count && row_bytes / (2 * c) >= (8u << 10))
+        c *= 2;
+    return c;
+}
+
+int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
+               int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p, float* out_S,
+               float* out_h, float* out_lse_t, float* out_lse_d, cudaStream_t stream) {
+    t_last_launches = 0;
+    int rc = check_args(tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
+    if (rc != BV_OK) return rc;
+    if (B == 0) return BV_OK;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState* d = nullptr;
+    if ((rc = device_state(&d)) != BV_OK) return rc;
+
+    const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
+    const size_t row_bytes = static_cast<size_t>(V) * esz;
+    const bool vec = (row_bytes % 16 == 0) && aligned(tgt, 16) && aligned(drf, 16);
+    int cluster = pick_cluster(*d, B, row_bytes);
+    int& cached = d->max_clusters[algo][dtype][vec ? 1 : 0][cluster];
+    if (cached == 0) {
+        cached = bv::stream_max_clusters(algo, dtype, vec, cluster);
+        if (cached <= 0) cached = -1;
+    }
+    if (cached < 0) return BV_ERR_UNSUPPORTED;
+    const int nclusters = B < cached ? B : cached;
+
+    bv::Params prm{};
+    prm.tgt = tgt; prm.drf = drf; prm.tok = tok; prm.uni = uni;
+    prm.B = B; prm.gamma = gamma; prm.V = V;
+    const double kd = 1.4426950408889634073599246810019 / static_cast<double>(T);
+    prm.kd = kd;
+    prm.kf = static_cast<float>(kd);
+    prm.out_tokens = ot; prm.out_len = ol;
+    prm.out_p = out_p; prm.out_S = out_S; prm.out_h = out_h;
+    prm.out_lse_t = out_lse_t; prm.out_lse_d = out_lse_d;
+    prm.ticket = d->tickets + 2 * (d->calls++ % kTicketSlots);
+    prm.nclusters = nclusters;
+
+    cudaError_t e = bv::launch_stream(prm, algo, dtype, vec, cluster, nclusters, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    t_last_launches = 1;
+    return BV_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
+             int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol) {
+    int rc = check_args(tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
+    if (rc != BV_OK) return rc;
+    if (B == 0) return BV_OK;
+    const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
+    const size_t n_t = static_cast<size_t>(B) * (gamma + 1) * V * esz;
+    const size_t n_d = static_cast<size_t>(B) * gamma * V * esz;
+    const size_t n_tok = static_cast<size_t>(B) * gamma * 4, n_uni = static_cast<size_t>(B) * (gamma + 2) * 4;
+    const size_t n_ot = static_cast<size_t>(B) * (gamma + 1) * 4, n_ol = static_cast<size_t>(B) * 4;
+    const size_t o_t = 0, o_d = align_up(o_t + n_t, 256), o_tok = align_up(o_d + n_d, 256);
+    const size_t o_uni = align_up(o_tok + n_tok, 256), o_ot = align_up(o_uni + n_uni, 256);
+    const size_t o_ol = align_up(o_ot + n_ot, 256), total = align_up(o_ol + n_ol, 256);
+
+    char* base = nullptr;
+    cudaStream_t s = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        DeviceState* d = nullptr;
+        if ((rc = device_state(&d)) != BV_OK) return rc;
+        cudaError_t e;
+        if (!d->stream && (e = cudaStreamCreateWithFlags(&d->stream, cudaStreamNonBlocking)) != cudaSuccess)
+            return cuda_fail(e);
+        if (d->stage_bytes < total) {
+            if (d->stage) cudaFree(d->stage);
+            d->stage = nullptr;
+            d->stage_bytes = 0;
+            if ((e = cudaMalloc(&d->stage, total)) != cudaSuccess) return cuda_fail(e);
+            d->stage_bytes = total;
+        }
+        base = static_cast<char*>(d->stage);
+        s = d->stream;
+    }
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(base + o_t, tgt, n_t, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(base + o_d, drf, n_d, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(base + o_tok, tok, n_tok, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(base + o_uni, uni, n_uni, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+    rc = run_device(algo, base + o_t, base + o_d, reinterpret_cast<const int32_t*>(base + o_tok),
+                    reinterpret_cast<const float*>(base + o_uni), B, gamma, V, dtype, T,
+                    reinterpret_cast<int32_t*>(base + o_ot), reinterpret_cast<int32_t*>(base + o_ol),
+                    nullptr, nullptr, nullptr, nullptr, nullptr, s);
+    if (rc != BV_OK) return rc;
+    if ((e = cudaMemcpyAsync(ot, base + o_ot, n_ot, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(ol, base + o_ol, n_ol, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
+    return BV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int bv_verify(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+              int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, nullptr, nullptr,
+                      nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int tv_verify(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+              int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
+    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, nullptr, nullptr,
+                      nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int bv_verify_ex(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+                 int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p, float* out_S,
+                 float* out_h, float* out_lse_t, float* out_lse_d, void* stream) {
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, out_p, out_S,
+                      out_h, out_lse_t, out_lse_d, static_cast<cudaStream_t>(stream));
+}
+
+int tv_verify_ex(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+                 int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p, float* out_S,
+                 float* out_h, float* out_lse_t, float* out_lse_d, void* stream) {
+    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, out_p, out_S,
+                      out_h, out_lse_t, out_lse_d, static_cast<cudaStream_t>(stream));
+}
+
+int bv_verify_host(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
+                   int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol) {
+    return run_host(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
+}
+
+int tv_verify_host(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
+                   int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol) {
+    return run_host(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
+}
+
+int bv_release(void) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return BV_ERR_UNSUPPORTED;
+    DeviceState& d = g_dev[dev];
+    if ((e = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(e);
+    if (d.stage) cudaFree(d.stage);
+    if (d.tickets) cudaFree(d.tickets);
+    if (d.stream) cudaStreamDestroy(d.stream);
+    d = DeviceState{};
+    return BV_OK;
+}
+
+int bv_last_launch_count(void) { return t_last_launches; }
+int bv_last_cuda_error(void) { return t_last_cuda_error; }
+
+const char* bv_status_string(int status) {
+    switch (status) {
+        case BV_OK: return "ok";
+        case BV_ERR_INVALID_ARG: return "invalid argument";
+        case BV_ERR_UNSUPPORTED: return "unsupported shape or device";
+        case BV_ERR_CUDA: return "CUDA runtime error";
+        case BV_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+int bv_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,151 @@
+// Device-side building blocks shared by the verification kernels: parameter
+// block, 128-bit streaming loads, bf16 widening, (max, sum-exp) reductions.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bv {
+
+constexpr int kMaxGamma = 64;     // longest drafted block the kernels accept
+constexpr int kMaxCluster = 8;    // portable thread-block cluster limit
+
+enum : int { kF32 = 0, kBF16 = 1 };
+enum : int { kTokenVerify = 0, kBlockVerify = 1 };
+
+struct Params {
+    const void* tgt;          // [B, gamma+1, V]
+    const void* drf;          // [B, gamma,   V]
+    const int32_t* tok;       // [B, gamma]
+    const float* uni;         // [B, gamma+2]
+    int B, gamma, V;
+    float kf;                 // log2(e) / T, rounded to float (per-element scale)
+    double kd;                // log2(e) / T in double (scalar recursion)
+    int32_t* out_tokens;      // [B, gamma+1]
+    int32_t* out_len;         // [B]
+    float* out_p;             // optional diagnostics, may be null
+    float* out_S;
+    float* out_h;
+    float* out_lse_t;
+    float* out_lse_d;
+    unsigned int* ticket;     // [2]: next sequence index, clusters that have finished
+    int nclusters;            // clusters in the grid
+};
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// One "unit" of a logit row: EPV consecutive elements widened to float.
+// VEC = true reads 16 bytes at once and needs 16-byte aligned rows.
+template <int DT, bool VEC> struct Unit;
+
+template <> struct Unit<kF32, true> {
+    static constexpr int EPV = 4;
+    static __device__ __forceinline__ void load(const void* row, int i, float (&v)[4]) {
+        uint4 r = ld_stream_v4(reinterpret_cast<const uint4*>(row) + i);
+        v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y);
+        v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+    }
+};
+template <> struct Unit<kBF16, true> {
+    static constexpr int EPV = 8;
+    static __device__ __forceinline__ void load(const void* row, int i, float (&v)[8]) {
+        uint4 r = ld_stream_v4(reinterpret_cast<const uint4*>(row) + i);
+        v[0] = __uint_as_float(r.x << 16); v[1] = __uint_as_float(r.x & 0xffff0000u);
+        v[2] = __uint_as_float(r.y << 16); v[3] = __uint_as_float(r.y & 0xffff0000u);
+        v[4] = __uint_as_float(r.z << 16); v[5] = __uint_as_float(r.z & 0xffff0000u);
+        v[6] = __uint_as_float(r.w << 16); v[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+};
+template <> struct Unit<kF32, false> {
+    static constexpr int EPV = 1;
+    static __device__ __forceinline__ void load(const void* row, int i, float (&v)[1]) {
+        v[0] = __ldg(reinterpret_cast<const float*>(row) + i);
+    }
+};
+template <> struct Unit<kBF16, false> {
+    static constexpr int EPV = 1;
+    static __device__ __forceinline__ void load(const void* row, int i, float (&v)[1]) {
+        unsigned short h = __ldg(reinterpret_cast<const unsigned short*>(row) + i);
+        v[0] = __uint_as_float(static_cast<uint32_t>(h) << 16);
+    }
+};
+
+template <int DT> __device__ __forceinline__ double load_logit(const void* row, int x) {
+    float v[1];
+    Unit<DT, false>::load(row, x, v);
+    return static_cast<double>(v[0]);
+}
+
+// 2^d for an integer-valued d <= 0 (or -inf): an exact power of two, 0 below 2^-126.
+__device__ __forceinline__ float pow2_nonpos(float d) {
+    int n = (d < -126.f) ? -127 : static_cast<int>(d);
+    return __int_as_float((n + 127) << 23);
+}
+
+// Running sum of 2^{z*k - M} over the elements a thread has seen, where the
+// reference M is an INTEGER (the rounded scaled maximum so far).  An integer
+// reference is exact in fp32, so z*k - M costs one fused multiply-add with a
+// single rounding, and changing the reference rescales by an exact power of two.
+// A NaN element makes s NaN; M = +inf is caught when the row is combined.
+struct MaxSum {
+    float M, s;
+    __device__ __forceinline__ void init() { M = -INFINITY; s = 0.f; }
+    template <int N> __device__ __forceinline__ void add(const float (&v)[N], float kf) {
+        float vm = v[0];
+#pragma unroll
+        for (int e = 1; e < N; ++e) vm = fmaxf(vm, v[e]);
+        const float y = rintf(vm * kf);
+        if (y > M) { s = (s != s) ? s : s * pow2_nonpos(M - y); M = y; }
+        if (M > -INFINITY) {
+            const float nM = -M;
+#pragma unroll
+            for (int e = 0; e < N; ++e) s += ex2(fmaf(v[e], kf, nM));
+        } else {
+#pragma unroll
+            for (int e = 0; e < N; ++e) if (v[e] != v[e]) s = v[e];
+        }
+    }
+};
+
+// Combine the lanes of a warp: afterwards every lane holds the warp's (M, s).
+__device__ __forceinline__ void warp_combine(float& M, float& s) {
+    float Mw = M;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) Mw = fmaxf(Mw, __shfl_xor_sync(0xffffffffu, Mw, off));
+    s = (s != s) ? s : s * pow2_nonpos(M - Mw);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    M = Mw;
+}
+
+__device__ __forceinline__ double shfl_xor_d(double v, int off) {
+    int lo = __double2loint(v), hi = __double2hiint(v);
+    lo = __shfl_xor_sync(0xffffffffu, lo, off);
+    hi = __shfl_xor_sync(0xffffffffu, hi, off);
+    return __hiloint2double(hi, lo);
+}
+__device__ __forceinline__ double shfl_up_d(double v, int off) {
+    int lo = __double2loint(v), hi = __double2hiint(v);
+    lo = __shfl_up_sync(0xffffffffu, lo, off);
+    hi = __shfl_up_sync(0xffffffffu, hi, off);
+    return __hiloint2double(hi, lo);
+}
+__device__ __forceinline__ double shfl_d(double v, int src) {
+    int lo = __double2loint(v), hi = __double2hiint(v);
+    lo = __shfl_sync(0xffffffffu, lo, src);
+    hi = __shfl_sync(0xffffffffu, hi, src);
+    return __hiloint2double(hi, lo);
+}
+
+}  // namespace bv

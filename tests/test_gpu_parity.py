@@ -1,0 +1,163 @@
+"""GPU parity: the CUDA library against the CPU oracle on the same seeded bits,
+element by element, through the C-ABI (via the ctypes binding)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2403_10444_b200 import workloads as wl
+from parity import run_oracle, run_cuda, compare, assert_parity
+
+pytestmark = pytest.mark.gpu
+
+ALGOS = [oracle.BLOCK_VERIFY, oracle.TOKEN_VERIFY]
+
+
+def parity_case(inp, algo, check_diag=True):
+    ref = run_oracle(algo, inp)
+    ot, ol, diag = run_cuda(algo, inp)
+    rep = compare(algo, ref, ot, ol, diag)
+    print(rep)
+    assert_parity(rep, check_diag)
+    return rep
+
+
+def random_inputs(B, gamma, V, dtype, seed, T=1.0, sigma_t=2.0, sigma_d=1.0):
+    w = wl.Workload("t", B, gamma, V, dtype, T, seed, sigma_t, 0.0, 0, 0.0, sigma_d)
+    return wl.make_inputs(w, "cpu")
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("name", ["c1", "c2"])
+def test_small_configs(name, algo):
+    parity_case(wl.make_inputs(wl.CONFIGS[name], "cpu"), algo)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("name", ["c3", "c4"])
+def test_full_size_configs(name, algo):
+    # generated on the GPU (fast), the same bits copied to the oracle
+    inp = wl.make_inputs(wl.CONFIGS[name], "cuda")
+    parity_case(inp, algo)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 2, 3, 8, 17, 1000, 1027, 4104, 20000])
+def test_ragged_vocabularies(V, dtype, algo):
+    # V = 1..17 and odd V take the element-wise path; multiples of 16 bytes the 128-bit path
+    for gamma, B in ((1, 5), (2, 37), (5, 9)):
+        parity_case(random_inputs(B, gamma, V, dtype, seed=V * 7 + gamma), algo)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+def test_every_cluster_width(cluster, algo, monkeypatch):
+    monkeypatch.setenv("BV_CLUSTER", str(cluster))
+    parity_case(random_inputs(19, 4, 24000, "bf16", seed=cluster, T=0.8), algo)
+    parity_case(random_inputs(7, 3, 5000, "f32", seed=cluster + 10), algo)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_more_sequences_than_resident_clusters(algo):
+    parity_case(random_inputs(700, 3, 512, "f32", seed=3), algo)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("gamma", [1, 16, 64])
+def test_block_lengths(gamma, algo):
+    parity_case(random_inputs(6, gamma, 2048, "bf16", seed=gamma, sigma_d=0.3), algo)
+
+
+@pytest.mark.parametrize("T", [0.2, 0.6, 1.0, 2.5])
+def test_temperatures(T):
+    for algo in ALGOS:
+        parity_case(random_inputs(12, 4, 8192, "f32", seed=5, T=T), algo)
+
+
+def test_gamma1_block_equals_token_bitwise():
+    inp = random_inputs(300, 1, 777, "f32", seed=21)
+    a = run_cuda(oracle.BLOCK_VERIFY, inp, diagnostics=False)
+    b = run_cuda(oracle.TOKEN_VERIFY, inp, diagnostics=False)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_draft_equals_target():
+    inp = random_inputs(16, 6, 4096, "bf16", seed=22)
+    inp["draft_logits"] = inp["target_logits"][:, :6].clone()
+    for algo in ALGOS:
+        ot, ol, diag = run_cuda(algo, inp)
+        assert torch.all(ol == 7)
+        assert torch.equal(ot[:, :6].cpu(), inp["draft_tokens"])
+        parity_case(inp, algo)
+    _, _, diag = run_cuda(oracle.BLOCK_VERIFY, inp)
+    assert torch.all(diag["S"] == 0) and torch.all(diag["p"] == 1)
+
+
+def test_masked_logits_and_domain_errors():
+    inp = random_inputs(8, 3, 640, "f32", seed=23)
+    t, d, tok = inp["target_logits"], inp["draft_logits"], inp["draft_tokens"]
+    # top-k style masking: legal
+    t[0, :, 100:] = -float("inf")
+    d[0, :, 200:] = -float("inf")
+    q = torch.softmax(d[0], dim=-1)
+    tok[0] = torch.multinomial(q, 1).squeeze(1).to(torch.int32)
+    t[1, 0, 3] = float("nan")
+    tok[2, 1] = 640
+    d[3, 0, tok[3, 0]] = -float("inf")
+    t[4, 1, :] = -float("inf")
+    t[5, 2, 7] = float("inf")
+    tok[6, 0] = -1
+    ref = run_oracle(oracle.BLOCK_VERIFY, inp)
+    ot, ol, _ = run_cuda(oracle.BLOCK_VERIFY, inp)
+    assert list(ol.cpu().numpy()[[1, 2, 3, 4, 5, 6]]) == [-1] * 6
+    assert torch.all(ot[[1, 2, 3, 4, 5, 6]] == -1)
+    assert np.array_equal(ol.cpu().numpy(), ref.out_len)
+    assert np.array_equal(ot.cpu().numpy(), ref.out_tokens)
+    # Algorithm 1 reads rows 0..tau only: same inputs, compare with its oracle
+    ref = run_oracle(oracle.TOKEN_VERIFY, inp)
+    ot, ol, _ = run_cuda(oracle.TOKEN_VERIFY, inp)
+    assert np.array_equal(ol.cpu().numpy(), ref.out_len)
+    assert np.array_equal(ot.cpu().numpy(), ref.out_tokens)
+
+
+def test_deterministic_bits():
+    inp = wl.make_inputs(wl.scaled(wl.CONFIGS["c3"], B=8), "cuda")
+    a = run_cuda(oracle.BLOCK_VERIFY, inp)
+    b = run_cuda(oracle.BLOCK_VERIFY, inp)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    for k in a[2]:
+        assert torch.equal(a[2][k].view(torch.int32), b[2][k].view(torch.int32))
+
+
+@pytest.mark.parametrize("cell", [(1, 2, 0.1), (16, 16, 1.0), (64, 4, 3.0), (512, 2, 1.0)])
+def test_sweep_cells(cell):
+    inp = wl.make_inputs(wl.sweep_cell(*cell), "cuda")
+    for algo in ALGOS:
+        parity_case(inp, algo)
+
+
+def test_host_buffer_entry_matches_device_entry():
+    import paper_2403_10444_b200 as bv
+    inp = random_inputs(33, 4, 3000, "bf16", seed=31)
+    pinned = {k: (v.pin_memory() if torch.is_tensor(v) else v) for k, v in inp.items()}
+    for host_fn, algo in ((bv.bv_verify_host, oracle.BLOCK_VERIFY), (bv.tv_verify_host, oracle.TOKEN_VERIFY)):
+        ot, ol = host_fn(pinned["target_logits"], pinned["draft_logits"], pinned["draft_tokens"],
+                         pinned["uniforms"], pinned["temperature"])
+        dt, dl = run_cuda(algo, inp, diagnostics=False)
+        assert torch.equal(ot, dt.cpu()) and torch.equal(ol, dl.cpu())
+
+
+def test_launch_count_and_nonblocking_stream():
+    import paper_2403_10444_b200 as bv
+    inp = {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in random_inputs(5, 2, 1024, "f32", 1).items()}
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        ot, ol = bv.bv_verify(inp["target_logits"], inp["draft_logits"], inp["draft_tokens"],
+                              inp["uniforms"], 1.0, stream=s)
+    s.synchronize()
+    assert bv.bv_last_launch_count() == 1
+    ref = run_oracle(oracle.BLOCK_VERIFY, inp)
+    assert np.array_equal(ol.cpu().numpy(), ref.out_len)
