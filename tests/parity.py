@@ -4,12 +4,16 @@ the smoke check and nothing else).
 Tolerances, from the arithmetic of the CUDA path (fp32 per element, fp64 combination):
   - log-normalisers: 3e-6 absolute (they are returned as fp32 and are near 16, where one
     fp32 ulp is 1.9e-6);
-  - p_i: 1e-5 relative; h_i: 1e-5 h_i + 1e-7 (h_i inherits the conditioning of S_i);
+  - p_i: 1e-5 relative; h_i: 1e-5 h_i + 1e-7 plus the S and p tolerances propagated through
+    h = S / (S + 1 - p);
   - S_i: 1e-5 relative literally where S_i >= 1e-2 p_i; below that the bound is
     1e-5 S_i + 1e-7 p_i, because S is then the small difference of sums whose own
-    fp32 rounding is 6e-8 p_i; where the oracle has S_i = 0 the CUDA value must be 0;
+    fp32 rounding is 6e-8 p_i; where the oracle has S_i = 0 the CUDA value must be
+    <= 1e-7 p_i (and exactly 0 when the two rows are bit-identical);
   - tau and Y: bit-exact, except for trials in which a uniform lies within 1e-6 of
-    the threshold it is compared with (oracle margins); those are counted.
+    the threshold it is compared with: a differing tau needs an eta_i within 1e-6 of
+    h_i (oracle margin); a differing Y needs the sampling uniform within 1e-6 of the
+    CDF cell of the CUDA token (recomputed here in fp64).  Both are counted.
 """
 from __future__ import annotations
 
@@ -53,25 +57,59 @@ def run_cuda(algo: int, inp, diagnostics=True):
 @dataclass
 class ParityReport:
     trials: int
-    near_threshold: int
-    mismatches: int            # tau or Y differs (all of them, near-threshold or not)
-    hard_mismatches: int       # differs although no uniform was near its threshold
+    near_threshold: int        # trials with some deciding uniform within 1e-6 of its threshold
+    mismatches: int            # tau or Y differs (all of them, excused or not)
+    excused_tau: int           # tau differs and an eta_i was within 1e-6 of h_i
+    excused_Y: int             # same tau, Y differs, and u is within 1e-6 of the CUDA token's CDF cell
+    hard_mismatches: int       # differs with no such excuse
     max_rel_S: float
     max_rel_S_conditioned: float  # over positions with S >= 1e-2 p
     S_floor_violations: int
-    max_rel_h: float
+    max_h_err_over_tol: float
     max_rel_p: float
     max_abs_lse: float
+    vocab: int = 0
 
     def __str__(self):
-        return ("trials=%d near=%d mismatch=%d hard=%d relS=%.2e relS(S>=.01p)=%.2e floorviol=%d "
-                "relh=%.2e relp=%.2e abslse=%.2e" % (
-                    self.trials, self.near_threshold, self.mismatches, self.hard_mismatches,
-                    self.max_rel_S, self.max_rel_S_conditioned, self.S_floor_violations,
-                    self.max_rel_h, self.max_rel_p, self.max_abs_lse))
+        return ("trials=%d near=%d mismatch=%d excused_tau=%d excused_Y=%d hard=%d relS=%.2e "
+                "relS(S>=.01p)=%.2e floorviol=%d h_err/tol=%.2f relp=%.2e abslse=%.2e" % (
+                    self.trials, self.near_threshold, self.mismatches, self.excused_tau,
+                    self.excused_Y, self.hard_mismatches, self.max_rel_S,
+                    self.max_rel_S_conditioned, self.S_floor_violations,
+                    self.max_h_err_over_tol, self.max_rel_p, self.max_abs_lse))
 
 
-def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=None) -> ParityReport:
+def _widen(row: np.ndarray) -> np.ndarray:
+    if row.dtype == np.uint16:
+        return (row.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return row.astype(np.float64)
+
+
+def token_is_valid(algo, ref, inp_np, b, y) -> bool:
+    """Is token y within 1e-6 (in probability) of the CDF cell the sampling uniform falls in,
+    under the oracle's normalisers and p for sequence b?  (fp64, index order.)"""
+    tgt, drf, uni, T = inp_np
+    g = drf.shape[1]
+    tau = int(ref.out_len[b]) - 1
+    T = float(np.float32(T))
+    P = np.exp(_widen(tgt[b, tau]) / T - ref.lse_t[b, tau])
+    if tau < g:
+        p = ref.p[b, tau] if algo == oracle.BLOCK_VERIFY else 1.0
+        w = np.maximum(p * P - np.exp(_widen(drf[b, tau]) / T - ref.lse_d[b, tau]), 0.0)
+        if not w.sum() > 0:
+            w = P
+        u = float(uni[b, g])
+    else:
+        w, u = P, float(uni[b, g + 1])
+    if y < 0 or y >= w.shape[0] or not w[y] > 0:
+        return False
+    C = np.cumsum(w)
+    lo = (C[y] - w[y]) / C[-1]
+    hi = C[y] / C[-1]
+    return lo - NEAR <= u <= hi + NEAR
+
+
+def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=None, inp=None) -> ParityReport:
     ot = out_tokens.cpu().numpy()
     ol = out_len.cpu().numpy()
     B = ol.shape[0]
@@ -79,9 +117,29 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
     ok_rows = ref.out_len >= 0
     near = ok_rows & ((ref.margin_eta < NEAR) | (ref.margin_smp < NEAR))
     mism = ~same
-    hard = mism & ~near
-    rel_S = rel_Sc = rel_h = rel_p = abs_lse = 0.0
+    excused_tau = excused_Y = hard = 0
+    inp_np = None
+    for b in np.nonzero(mism)[0]:
+        if not ok_rows[b] or ol[b] < 0:
+            hard += 1
+        elif ol[b] != ref.out_len[b]:
+            if ref.margin_eta[b] < NEAR:
+                excused_tau += 1
+            else:
+                hard += 1
+        else:
+            tau = int(ol[b]) - 1
+            prefix_same = np.array_equal(ot[b, :tau], ref.out_tokens[b, :tau]) and np.all(ot[b, tau + 1:] == -1)
+            if inp is not None and inp_np is None:
+                inp_np = (to_numpy_logits(inp["target_logits"]), to_numpy_logits(inp["draft_logits"]),
+                          inp["uniforms"].cpu().numpy(), inp["temperature"])
+            if prefix_same and inp_np is not None and token_is_valid(algo, ref, inp_np, b, int(ot[b, tau])):
+                excused_Y += 1
+            else:
+                hard += 1
+    rel_S = rel_Sc = h_over = rel_p = abs_lse = 0.0
     floor_viol = 0
+    V = 0
     if diag is not None:
         S = diag["S"].cpu().numpy().astype(np.float64)
         h = diag["h"].cpu().numpy().astype(np.float64)
@@ -94,20 +152,36 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
             assert not np.isnan(got[m]).any(), "CUDA path left a log-normaliser unset"
             if m.any():
                 abs_lse = max(abs_lse, float(np.abs(got[m] - want[m]).max()))
-        m = rows[:, None] & ~np.isnan(ref.h)
-        assert not np.isnan(h[m]).any()
-        if m.any():
-            rel_h = float((np.abs(h[m] - ref.h[m]) / (np.abs(ref.h[m]) + 1e-2)).max())
         if algo == oracle.BLOCK_VERIFY:
             m = rows[:, None] & ~np.isnan(ref.p)
             rel_p = float((np.abs(p[m] - ref.p[m]) / np.maximum(ref.p[m], 1e-30)).max())
             pS = ref.p[:, :-1]
+            # h_i = S_i / (S_i + 1 - p_i), 1 <= i < gamma: propagate the S and p tolerances.
+            # Positions with S_i = 0 are skipped: h_i is then immaterial.
+            g = ref.S.shape[1]
+            for i in range(1, g):
+                Sr, pr, hr = ref.S[:, i], ref.p[:, i], ref.h[:, i]
+                mm = rows & (Sr > 0)
+                if mm.any():
+                    den = (Sr[mm] + 1.0 - pr[mm]) ** 2
+                    tol = 1e-5 * hr[mm] + ((1.0 - pr[mm]) * 1e-7 * pr[mm] + Sr[mm] * 2e-7 * pr[mm]) / den + 1e-7
+                    h_over = max(h_over, float((np.abs(h[mm, i] - hr[mm]) / tol).max()))
+            mm = rows
+            if mm.any():
+                tol = 1e-5 * ref.h[mm, g] + 1e-7
+                h_over = max(h_over, float((np.abs(h[mm, g] - ref.h[mm, g]) / tol).max()))
         else:
             pS = np.ones_like(ref.S)
+            m = rows[:, None] & ~np.isnan(ref.h)
+            assert not np.isnan(h[m]).any()
+            if m.any():
+                h_over = float((np.abs(h[m] - ref.h[m]) / (1e-5 * ref.h[m] + 1e-7)).max())
         m = rows[:, None] & ~np.isnan(ref.S)
         assert not np.isnan(S[m]).any()
         zero = m & (ref.S == 0)
-        assert np.all(S[zero] == 0), "CUDA S must be exactly 0 where the oracle's is"
+        # an exactly empty residual: the CUDA value may differ from 0 only by the rounding
+        # floor (it is exactly 0 for bit-identical rows, see test_draft_equals_target)
+        assert np.all(S[zero] <= 3e-7 * pS[zero]), "CUDA S must vanish where the oracle's does"
         pos = m & (ref.S > 0)
         if pos.any():
             err = np.abs(S[pos] - ref.S[pos])
@@ -117,16 +191,22 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
             if cond.any():
                 rel_Sc = float(rel[cond].max())
             floor_viol = int((err > 1e-5 * ref.S[pos] + 1e-7 * pS[pos]).sum())
-    return ParityReport(B, int(near.sum()), int(mism.sum()), int(hard.sum()), rel_S, rel_Sc,
-                        floor_viol, rel_h, rel_p, abs_lse)
+    if inp is not None:
+        V = int(inp["target_logits"].shape[-1])
+    return ParityReport(B, int(near.sum()), int(mism.sum()), excused_tau, excused_Y, hard, rel_S,
+                        rel_Sc, floor_viol, h_over, rel_p, abs_lse, V)
 
 
 def assert_parity(rep: ParityReport, check_diag=True):
     assert rep.hard_mismatches == 0, str(rep)
-    assert rep.near_threshold <= max(1, int(np.ceil(1e-4 * rep.trials))), str(rep)
+    # an eta within 1e-6 of h_i: at most 1e-4 of trials may differ for that reason
+    assert rep.excused_tau <= int(np.ceil(1e-4 * rep.trials)), str(rep)
+    # the sampling uniform has one threshold per vocabulary entry; an fp32 CDF places each
+    # within ~1e-7, so the expected share of differing tokens grows with V
+    assert rep.excused_Y <= int(np.ceil(rep.trials * (1e-4 + 2e-7 * rep.vocab))), str(rep)
     if check_diag:
         assert rep.max_abs_lse <= 3e-6, str(rep)
         assert rep.max_rel_p <= 1e-5, str(rep)
-        assert rep.max_rel_h <= 1e-5, str(rep)
+        assert rep.max_h_err_over_tol <= 1.0, str(rep)
         assert rep.max_rel_S_conditioned <= 1e-5, str(rep)
         assert rep.S_floor_violations == 0, str(rep)

@@ -18,7 +18,7 @@ ALGOS = [oracle.BLOCK_VERIFY, oracle.TOKEN_VERIFY]
 def parity_case(inp, algo, check_diag=True):
     ref = run_oracle(algo, inp)
     ot, ol, diag = run_cuda(algo, inp)
-    rep = compare(algo, ref, ot, ol, diag)
+    rep = compare(algo, ref, ot, ol, diag, inp)
     print(rep)
     assert_parity(rep, check_diag)
     return rep
