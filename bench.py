@@ -1,0 +1,291 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-verification hot path.
+
+A "step" is one Block Verification call (every stage: normalisers, drafted-token
+probabilities, prefix recursion, residual masses, acceptance weights, selection
+of tau, residual sample) over one batch of synthetic logits.  The default
+workload is B=256, gamma=8, V=256000, bf16 (2.2 GB of logits, far larger than
+L2, so nothing is served from cache between steps).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload c1|c2|c3|c4] [--algo block|token]
+
+Prints one JSON line.  With N > 1 (launched by torch.distributed.run) every rank
+verifies its own batch of the same shape (weak scaling, no collective on the
+data path); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2403_10444_b200 import workloads as wl  # noqa: E402
+
+METRIC = "verifications/s (B*gamma logit rows)"
+UNIT = "verifications/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        return rank, world, local, dist
+    return 0, 1, 0, None
+
+
+def time_oracle(w, algo_name: str, budget_s: float = 20.0):
+    """The CPU oracle, as it stands, on a bounded sample of the workload."""
+    import numpy as np
+    import oracle
+    algo = oracle.BLOCK_VERIFY if algo_name == "block" else oracle.TOKEN_VERIFY
+    cores = oracle.threads()
+    # one sequence first to size the sample for about budget_s of work
+    probe = wl.make_inputs(wl.scaled(w, B=max(1, min(w.B, cores))), "cpu")
+
+    def run(inp):
+        t = inp["target_logits"]; d = inp["draft_logits"]
+        if t.dtype == torch.bfloat16:
+            t = t.view(torch.int16).numpy().view(np.uint16); d = d.view(torch.int16).numpy().view(np.uint16)
+        else:
+            t = t.numpy(); d = d.numpy()
+        t0 = time.perf_counter()
+        oracle.verify(algo, t, d, inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), inp["temperature"])
+        return time.perf_counter() - t0
+
+    t_probe = run(probe)
+    per_seq = t_probe / probe["draft_tokens"].shape[0]
+    n = int(max(1, min(w.B, budget_s / max(per_seq, 1e-9))))
+    n = max(min(n, w.B), min(w.B, cores))
+    sample = wl.make_inputs(wl.scaled(w, B=n), "cpu")
+    dt = run(sample)
+    return {"value": n * w.gamma / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "first %d of %d sequences of workload %s (%s verify), %.2f s" % (n, w.B, w.name, algo_name, dt),
+            "seconds": dt, "sequences": n}
+
+
+def reference_arm(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warmup = args.steps, args.warmup
+    budget = max(2.0, min(20.0, 120.0 / max(1, steps + warmup)))
+    times, last = [], None
+    for i in range(warmup + steps):
+        last = time_oracle(w, args.algo, budget_s=budget)
+        if i >= warmup:
+            times.append(last["seconds"])
+    n = last["sequences"]
+    ms = 1e3 * sum(times) / len(times)
+    value = n * w.gamma / (ms * 1e-3)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "gamma": w.gamma, "V": w.V, "storage": w.dtype,
+                       "algo": args.algo, "step": "%d sequences per step (bounded sample)" % n},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
+                             "sample": last["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--algo", default="block", choices=["block", "token"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = wl.CONFIGS[args.workload]
+
+    if args.impl == "reference":
+        reference_arm(args, w)
+        return
+
+    import paper_2403_10444_b200 as bv
+    bv.load_library()  # fails loudly if the CUDA library was not built
+    rank, world, local, dist = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    # weak scaling: every rank draws its own batch of the same shape
+    inp = wl.make_inputs(wl.scaled(w, seed=w.seed + 1000 * rank), dev)
+    fn = bv.bv_verify if args.algo == "block" else bv.tv_verify
+    a = (inp["target_logits"], inp["draft_logits"], inp["draft_tokens"], inp["uniforms"], inp["temperature"])
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        fn(*a)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    launches = 0
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(args.steps):
+        evs[i][0].record()
+        out = fn(*a)
+        evs[i][1].record()
+        launches += bv.bv_last_launch_count()
+    stop.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = start.elapsed_time(stop)
+    kernel_ms = [e0.elapsed_time(e1) for e0, e1 in evs]
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * w.B * w.gamma / (ms_per_step * 1e-3)
+
+    # ---- end to end: host buffers through the C-ABI host entry, copies inside the timed region ----
+    host = {k: (v.cpu().pin_memory() if torch.is_tensor(v) else v) for k, v in inp.items()}
+    hfn = bv.bv_verify_host if args.algo == "block" else bv.tv_verify_host
+    ha = (host["target_logits"], host["draft_logits"], host["draft_tokens"], host["uniforms"], host["temperature"])
+    ot = torch.empty((w.B, w.gamma + 1), dtype=torch.int32).pin_memory()
+    ol = torch.empty((w.B,), dtype=torch.int32).pin_memory()
+    hfn(*ha, out_tokens=ot, out_len=ol)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        hfn(*ha, out_tokens=ot, out_len=ol)
+    e2e_s = (time.perf_counter() - t0) / args.e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    h2d = sum(host[k].numel() * host[k].element_size()
+              for k in ("target_logits", "draft_logits", "draft_tokens", "uniforms"))
+    d2h = ot.numel() * 4 + ol.numel() * 4
+    assert torch.equal(ot, out[0].cpu()) and torch.equal(ol, out[1].cpu()), "host and device entry points disagree"
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peak()
+    k_ms = statistics.mean(kernel_ms)
+    achieved = w.logit_bytes / (k_ms * 1e-3) / 1e9
+    mean_len = float(out[1].float().mean().item())
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "gamma": w.gamma, "V": w.V, "storage": w.dtype,
+                   "temperature": w.temperature, "algo": args.algo, "parallelism": "batch-sharded x%d" % world,
+                   "l2": "inputs (%.2f GB per step) exceed L2" % (w.logit_bytes / 1e9),
+                   "mean_emitted_len": mean_len},
+        "clocks": clocks,
+        "e2e": {"value": world * w.B * w.gamma / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": TRAFFIC_BYTES.get((args.workload, args.algo)),
+                     "peak_source": peak_src, "kernel": "verify_stream_kernel", "kernel_ms": k_ms,
+                     "algorithmic_bytes": w.logit_bytes, "frac_of_8TBps": achieved / 8000.0},
+        "sequences_per_s": world * w.B / (ms_per_step * 1e-3),
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = {k: v for k, v in time_oracle(w, args.algo).items() if k not in ("seconds", "sequences")}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/; None until a capture of the current kernel exists.
+TRAFFIC_BYTES = {}
+
+
+if __name__ == "__main__":
+    main()
