@@ -172,9 +172,12 @@ def main():
     ap.add_argument("--algo", default="block", choices=["block", "token"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = wl.CONFIGS[args.workload]
+    if args.batch > 0:
+        w = wl.scaled(w, B=args.batch, name="%s_B%d" % (w.name, args.batch))
 
     if args.impl == "reference":
         reference_arm(args, w)
@@ -228,6 +231,18 @@ def main():
     value = world * w.B * w.gamma / (ms_per_step * 1e-3)
 
     # ---- end to end: host buffers through the C-ABI host entry, copies inside the timed region ----
+    e2e = None
+    if args.e2e_steps > 0:
+        e2e = end_to_end(args, w, inp, out, bv, barrier, dist, dev, world)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches, out, dist)
+
+
+def end_to_end(args, w, inp, out, bv, barrier, dist, dev, world):
     host = {k: (v.cpu().pin_memory() if torch.is_tensor(v) else v) for k, v in inp.items()}
     hfn = bv.bv_verify_host if args.algo == "block" else bv.tv_verify_host
     ha = (host["target_logits"], host["draft_logits"], host["draft_tokens"], host["uniforms"], host["temperature"])
@@ -247,12 +262,11 @@ def main():
               for k in ("target_logits", "draft_logits", "draft_tokens", "uniforms"))
     d2h = ot.numel() * 4 + ol.numel() * 4
     assert torch.equal(ot, out[0].cpu()) and torch.equal(ol, out[1].cpu()), "host and device entry points disagree"
+    return {"value": world * w.B * w.gamma / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps}
 
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
 
+def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches, out, dist):
     peak, peak_src = measured_peak()
     k_ms = statistics.mean(kernel_ms)
     achieved = w.logit_bytes / (k_ms * 1e-3) / 1e9
@@ -266,12 +280,11 @@ def main():
                    "l2": "inputs (%.2f GB per step) exceed L2" % (w.logit_bytes / 1e9),
                    "mean_emitted_len": mean_len},
         "clocks": clocks,
-        "e2e": {"value": world * w.B * w.gamma / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps},
+        "e2e": e2e,
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": TRAFFIC_BYTES.get((args.workload, args.algo)),
-                     "peak_source": peak_src, "kernel": "verify_stream_kernel", "kernel_ms": k_ms,
+                     "peak_source": peak_src, "kernel": "verify_resident_kernel" if args.algo == "block" else "verify_stream_kernel", "kernel_ms": k_ms,
                      "algorithmic_bytes": w.logit_bytes, "frac_of_8TBps": achieved / 8000.0},
         "sequences_per_s": world * w.B / (ms_per_step * 1e-3),
     }

@@ -22,6 +22,7 @@ struct DeviceState {
     unsigned int* tickets = nullptr;  // [kTicketSlots][2], zero when idle
     unsigned long long calls = 0;
     int max_clusters[2][2][2][bv::kMaxCluster + 1] = {};  // [algo][dtype][vec][cluster], 0 = not asked yet
+    int res_clusters[2][9][bv::kMaxCluster + 1] = {};     // resident kernel: [dtype][nk][cluster]
     // staging for the host-buffer entry points
     void* stage = nullptr;
     size_t stage_bytes = 0;
@@ -108,14 +109,6 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
     const size_t row_bytes = static_cast<size_t>(V) * esz;
     const bool vec = (row_bytes % 16 == 0) && aligned(tgt, 16) && aligned(drf, 16);
-    int cluster = pick_cluster(*d, B, row_bytes);
-    int& cached = d->max_clusters[algo][dtype][vec ? 1 : 0][cluster];
-    if (cached == 0) {
-        cached = bv::stream_max_clusters(algo, dtype, vec, cluster);
-        if (cached <= 0) cached = -1;
-    }
-    if (cached < 0) return BV_ERR_UNSUPPORTED;
-    const int nclusters = B < cached ? B : cached;
 
     bv::Params prm{};
     prm.tgt = tgt; prm.drf = drf; prm.tok = tok; prm.uni = uni;
@@ -126,6 +119,49 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     prm.out_tokens = ot; prm.out_len = ol;
     prm.out_p = out_p; prm.out_S = out_S; prm.out_h = out_h;
     prm.out_lse_t = out_lse_t; prm.out_lse_d = out_lse_d;
+
+    // Block Verification on 16-byte rows: the kernel that keeps each row pair on chip,
+    // when some cluster width lets a thread hold its share (at most 8 vectors per row).
+    if (algo == bv::kBlockVerify && vec && !std::getenv("BV_FORCE_STREAM")) {
+        const long long units = static_cast<long long>(row_bytes / 16);
+        int best_c = 0, best_nk = 0, best_n = 0;
+        long long best_sms = -1;
+        const char* ec = std::getenv("BV_RES_CLUSTER");
+        for (int c = bv::kMaxCluster; c >= 1; c /= 2) {
+            if (ec && std::atoi(ec) != c) continue;
+            const long long per_warp = ((units + c - 1) / c + 15) / 16;
+            int nk = 0;
+            for (int cand : {2, 4, 8}) if (per_warp <= 32LL * cand) { nk = cand; break; }
+            if (!nk) continue;
+            int& cached = d->res_clusters[dtype][nk][c];
+            if (cached == 0) {
+                cached = bv::resident_max_clusters(dtype, nk, c);
+                if (cached <= 0) cached = -1;
+            }
+            if (cached < 0) continue;
+            const int n = B < cached ? B : cached;
+            const long long sms = static_cast<long long>(n) * c;
+            if (sms >= best_sms) { best_sms = sms; best_c = c; best_nk = nk; best_n = n; }
+        }
+        if (best_c) {
+            prm.ticket = nullptr;
+            prm.nclusters = best_n;
+            cudaError_t e = bv::launch_resident(prm, dtype, best_nk, best_c, best_n, stream);
+            if (e != cudaSuccess) return cuda_fail(e);
+            t_last_launches = 1;
+            return BV_OK;
+        }
+    }
+
+    int cluster = pick_cluster(*d, B, row_bytes);
+    int& cached = d->max_clusters[algo][dtype][vec ? 1 : 0][cluster];
+    if (cached == 0) {
+        cached = bv::stream_max_clusters(algo, dtype, vec, cluster);
+        if (cached <= 0) cached = -1;
+    }
+    if (cached < 0) return BV_ERR_UNSUPPORTED;
+    const int nclusters = B < cached ? B : cached;
+
     prm.ticket = d->tickets + 2 * (d->calls++ % kTicketSlots);
     prm.nclusters = nclusters;
 

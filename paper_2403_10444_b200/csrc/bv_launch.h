@@ -15,4 +15,11 @@ int stream_max_clusters(int algo, int dtype, bool vec, int cluster);
 cudaError_t launch_stream(const Params& prm, int algo, int dtype, bool vec, int cluster,
                           int nclusters, cudaStream_t stream);
 
+// Resident kernel (Block Verification only, 128-bit path): a thread holds up to `nk`
+// vectors per row, nk in {2, 4, 8}.
+int resident_vectors_per_cta(int nk);
+int resident_max_clusters(int dtype, int nk, int cluster);
+cudaError_t launch_resident(const Params& prm, int dtype, int nk, int cluster, int nclusters,
+                            cudaStream_t stream);
+
 }  // namespace bv
