@@ -35,18 +35,22 @@ namespace bv {
 
 constexpr int kRThreads = 512;
 constexpr int kRWarps = kRThreads / 32;
+constexpr int kSegs = kMaxCluster * kRWarps;   // warp segments of a row, in vocabulary order
 // A vector of 8 terms all at the reference sums to at most 8 * 2^0.5 = 11.3; a sum above
 // this bound therefore means some term exceeds 2^0.5, i.e. its logit lies above the reference.
 // Without a raise every term is below 12, so its exponent is below 4 and is rounded to 1.2e-7.
 constexpr float kRaiseBound = 12.f;
+// "No reference yet": finite, so that -inf logits still give 2^-inf = 0 and any finite
+// logit overflows to +inf, which exceeds the bound above and installs a real reference.
+constexpr float kNoRef = -3.0e38f;
 
 struct ResShared {
-    float red_M[2][kRWarps];
-    double red_s[2][kRWarps];
-    float x_M[2][kMaxCluster];
-    double x_s[2][kMaxCluster];
-    double segtot[kRWarps];
-    double x_tot[kMaxCluster];
+    // sweep 1: (reference, sum) of every warp of every CTA, written by the owners into
+    // every CTA of the cluster: [P/Q][rank * 16 + warp]
+    float x_M[2][kSegs];
+    float x_s[2][kSegs];
+    // sweep 2: segment totals of every warp of every CTA, same indexing
+    float x_seg[kSegs];
     double p[kMaxGamma + 1];
     double S[kMaxGamma + 1];
     double h[kMaxGamma + 1];
@@ -54,23 +58,30 @@ struct ResShared {
     double lse_d[kMaxGamma + 1];
     int cand[kMaxGamma + 1];
     int bad;
-    float c;
-    float MP, MQ;
-    double invZQ;
+    float c;          // p_r Z_Q / Z_P
+    float MP, MQ;     // row references
 };
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-    const unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+// One ring item: a 16-byte asynchronous copy when `pred`, else the slot is filled with
+// `fill` (the bit pattern of -inf logits); either way one commit group.
+__device__ __forceinline__ void ring_fetch(void* slot, const void* src, bool pred, uint32_t fill) {
+    const unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(slot));
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t"
+        "@p cp.async.cg.shared.global [%0], [%1], 16;\n\t"
+        "@!p st.shared.v4.b32 [%0], {%3, %3, %3, %3};\n\t"
+        "cp.async.commit_group;\n\t}"
+        ::"r"(s), "l"(src), "r"(static_cast<int>(pred)), "r"(fill) : "memory");
 }
 
 template <int DT> struct Raw;
 template <> struct Raw<kBF16> {
     static constexpr int EPV = 8;
+    static constexpr uint32_t kNegInf = 0xff80ff80u;
     static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[8]) {
         v[0] = __uint_as_float(r.x << 16); v[1] = __uint_as_float(r.x & 0xffff0000u);
         v[2] = __uint_as_float(r.y << 16); v[3] = __uint_as_float(r.y & 0xffff0000u);
@@ -80,6 +91,7 @@ template <> struct Raw<kBF16> {
 };
 template <> struct Raw<kF32> {
     static constexpr int EPV = 4;
+    static constexpr uint32_t kNegInf = 0xff800000u;
     static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[4]) {
         v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y);
         v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
@@ -97,21 +109,25 @@ __device__ __forceinline__ float warp_max(float x) {
     for (int off = 16; off > 0; off >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, off));
     return x;
 }
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    return x;
+}
 
-// a_e = 2^{v_e k - M} and their sum; with no finite reference yet the terms are 0
-// (a NaN logit is carried into the sum so that the row is flagged).
+// a_e = 2^{v_e k - M} and their sum (branch-free; -inf logits give 0, NaN stays NaN)
 template <int EPV>
-__device__ __forceinline__ float expo(const float (&v)[EPV], bool valid, float kf, float M, float (&a)[EPV]) {
+__device__ __forceinline__ float expo(const float (&v)[EPV], float kf, float M, float (&a)[EPV]) {
+    const float nM = -M;
     float vs = 0.f;
-    if (valid && M > -INFINITY) {
-        const float nM = -M;
 #pragma unroll
-        for (int e = 0; e < EPV; ++e) { a[e] = ex2(fmaf(v[e], kf, nM)); vs += a[e]; }
-    } else {
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) { a[e] = 0.f; if (valid && v[e] != v[e]) vs = v[e]; }
-    }
+    for (int e = 0; e < EPV; ++e) { a[e] = ex2(fmaf(v[e], kf, nM)); vs += a[e]; }
     return vs;
+}
+
+// 2^d for d = (own reference) - (row reference) <= 0, or 0 when there is no own reference
+__device__ __forceinline__ float ref_scale(float own, float row) {
+    return own > kNoRef ? pow2_nonpos(own - row) : 0.f;
 }
 
 template <int DT, int NK>
@@ -130,11 +146,12 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
     const int cid = blockIdx.x / C;
     const int ncl = prm.nclusters;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int myseg = rank * kRWarps + warp;
 
     __shared__ ResShared sh;
     extern __shared__ __align__(16) unsigned char dyn[];
-    float4* bcache = reinterpret_cast<float4*>(dyn);                       // [NK][HV][512]
-    uint4* ring = reinterpret_cast<uint4*>(dyn + sizeof(float4) * NK * HV * kRThreads);  // [D][512]
+    float4* bcache = reinterpret_cast<float4*>(dyn) + tid;                                   // [NK][HV][512]
+    uint4* ring = reinterpret_cast<uint4*>(dyn + sizeof(float4) * NK * HV * kRThreads) + tid;  // [D][512]
 
     const int g = prm.gamma, V = prm.V, B = prm.B;
     const float kf = prm.kf;
@@ -145,19 +162,26 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
     const int w0 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * warp / kRWarps);
     const int w1 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * (warp + 1) / kRWarps);
     const int v0 = w0 + lane;            // this thread's k-th vector is v0 + 32 k, valid below w1
+    unsigned vmask = 0;                  // bit k: vector k exists
+#pragma unroll
+    for (int k = 0; k < NK; ++k) vmask |= (v0 + 32 * k < w1) ? (1u << k) : 0u;
     const size_t row_bytes = static_cast<size_t>(V) * ESZ;
+    const size_t toff = static_cast<size_t>(v0) * 16;   // byte offset of vector 0 inside a row
+
+    // unused slots of the exchange arrays (ranks >= C) stay neutral for the whole kernel
+    if (tid < kSegs) {
+        sh.x_M[0][tid] = kNoRef; sh.x_M[1][tid] = kNoRef;
+        sh.x_s[0][tid] = 0.f; sh.x_s[1][tid] = 0.f; sh.x_seg[tid] = 0.f;
+    }
 
     auto rowP = [&](int b, int r) -> const char* {
-        return static_cast<const char*>(prm.tgt) + (static_cast<size_t>(b) * (g + 1) + r) * row_bytes;
+        return static_cast<const char*>(prm.tgt) + (static_cast<size_t>(b) * (g + 1) + r) * row_bytes + toff;
     };
     auto rowQ = [&](int b, int r) -> const char* {
-        return static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * row_bytes;
+        return static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * row_bytes + toff;
     };
-    // one ring item: vector k of a row (null row: nothing to fetch); always one commit group
     auto fetch = [&](const char* row, int k, int slot) {
-        if (row != nullptr && v0 + 32 * k < w1)
-            cp_async16(&ring[slot * kRThreads + tid], row + static_cast<size_t>(v0 + 32 * k) * 16);
-        cp_async_commit();
+        ring_fetch(ring + slot * kRThreads, row + k * 512, row != nullptr && ((vmask >> k) & 1u), R::kNegInf);
     };
 
     // prologue: the first L k-steps of the first position
@@ -170,12 +194,12 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
             fetch(q0, k, 2 * k + 1);
         }
     }
+    cluster.sync();   // exchange arrays are initialised everywhere before any remote write
 
     for (int b = cid; b < B; b += ncl) {
         if (tid == 0) { sh.bad = 0; sh.p[0] = 1.0; }
         for (int r = 0; r <= g; ++r) {
             const bool have_q = r < g;
-            // rows of the next position in this cluster's stream (for the lookahead)
             int nb = b, nr = r + 1;
             if (nr > g) { nr = 0; nb = b + ncl; }
             const char* curP = rowP(b, r);
@@ -183,296 +207,278 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
             const char* nxtP = nb < B ? rowP(nb, nr) : nullptr;
             const char* nxtQ = (nb < B && nr < g) ? rowQ(nb, nr) : nullptr;
 
+            // thread 0 fetches the drafted token's two logits early (used after the combine)
+            double zp_x = 0.0, zq_x = 0.0;
+            int x_ok = 1;
+            if (tid == 0 && have_q) {
+                const int x = prm.tok[static_cast<size_t>(b) * g + r];
+                x_ok = (x >= 0 && x < V);
+                if (x_ok) {
+                    zp_x = load_logit<DT>(curP - toff, x);
+                    zq_x = load_logit<DT>(curQ - toff, x);
+                }
+            }
+
             // ---------------- sweep 1 ----------------
             float a[NK][EPV];
-            float MPw = -INFINITY, sP = 0.f, MQw = -INFINITY, sQ = 0.f;   // references are warp-uniform
+            float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;   // references are warp-uniform
 #pragma unroll
             for (int k = 0; k < NK; ++k) {
-                const bool valid = v0 + 32 * k < w1;
                 const int slotP = (2 * k) % D, slotQ = (2 * k + 1) % D;
                 // ---- target row ----
                 cp_async_wait<D - 1>();
                 {
                     float v[EPV];
-                    if (valid) R::unpack(ring[slotP * kRThreads + tid], v);
-                    else {
-#pragma unroll
-                        for (int e = 0; e < EPV; ++e) v[e] = -INFINITY;
-                    }
-                    bool raise;
-                    float vs = 0.f;
-                    if (MPw > -INFINITY) {
-                        vs = expo<EPV>(v, valid, kf, MPw, a[k]);
-                        raise = __any_sync(0xffffffffu, vs > kRaiseBound);
-                    } else {
-                        raise = true;   // no finite logit seen yet: look for one
-                    }
-                    if (raise) {
+                    R::unpack(ring[slotP * kRThreads], v);
+                    if (k == 0) MPw = fmaxf(rintf(warp_max(vec_max<EPV>(v)) * kf), kNoRef);
+                    float vs = expo<EPV>(v, kf, MPw, a[k]);
+                    if (__any_sync(0xffffffffu, vs > kRaiseBound)) {
                         const float y = rintf(warp_max(vec_max<EPV>(v)) * kf);
                         if (y > MPw) {
-                            const float f = pow2_nonpos(MPw - y);
-                            sP = (sP != sP) ? sP : sP * f;
+                            const float f = ref_scale(MPw, y);
+                            sP *= f;
 #pragma unroll
                             for (int kk = 0; kk < k; ++kk)
 #pragma unroll
                                 for (int e = 0; e < EPV; ++e) a[kk][e] *= f;
                             MPw = y;
                         }
-                        vs = expo<EPV>(v, valid, kf, MPw, a[k]);
+                        vs = expo<EPV>(v, kf, MPw, a[k]);
                     }
                     sP += vs;
                 }
                 if (k + L < NK) fetch(curP, k + L, slotP); else fetch(nxtP, k + L - NK, slotP);
-                // ---- draft row ----
+                // ---- draft row (slots hold -inf when there is none) ----
                 cp_async_wait<D - 1>();
                 {
-                    const bool qvalid = valid && have_q;
                     float v[EPV], bq[EPV];
-                    if (qvalid) R::unpack(ring[slotQ * kRThreads + tid], v);
-                    else {
-#pragma unroll
-                        for (int e = 0; e < EPV; ++e) v[e] = -INFINITY;
-                    }
-                    bool raise;
-                    float vs = 0.f;
-                    if (MQw > -INFINITY) {
-                        vs = expo<EPV>(v, qvalid, kf, MQw, bq);
-                        raise = __any_sync(0xffffffffu, vs > kRaiseBound);
-                    } else {
-                        raise = have_q;
-                    }
-                    if (raise) {
+                    R::unpack(ring[slotQ * kRThreads], v);
+                    if (k == 0) MQw = fmaxf(rintf(warp_max(vec_max<EPV>(v)) * kf), kNoRef);
+                    float vs = expo<EPV>(v, kf, MQw, bq);
+                    if (__any_sync(0xffffffffu, vs > kRaiseBound)) {
                         const float y = rintf(warp_max(vec_max<EPV>(v)) * kf);
                         if (y > MQw) {
-                            const float f = pow2_nonpos(MQw - y);
-                            sQ = (sQ != sQ) ? sQ : sQ * f;
+                            const float f = ref_scale(MQw, y);
+                            sQ *= f;
 #pragma unroll
                             for (int kk = 0; kk < k; ++kk)
 #pragma unroll
                                 for (int hv = 0; hv < HV; ++hv) {
-                                    float4 t4 = bcache[(kk * HV + hv) * kRThreads + tid];
+                                    float4 t4 = bcache[(kk * HV + hv) * kRThreads];
                                     t4.x *= f; t4.y *= f; t4.z *= f; t4.w *= f;
-                                    bcache[(kk * HV + hv) * kRThreads + tid] = t4;
+                                    bcache[(kk * HV + hv) * kRThreads] = t4;
                                 }
                             MQw = y;
                         }
-                        vs = expo<EPV>(v, qvalid, kf, MQw, bq);
+                        vs = expo<EPV>(v, kf, MQw, bq);
                     }
                     sQ += vs;
 #pragma unroll
                     for (int hv = 0; hv < HV; ++hv)
-                        bcache[(k * HV + hv) * kRThreads + tid] =
+                        bcache[(k * HV + hv) * kRThreads] =
                             make_float4(bq[4 * hv], bq[4 * hv + 1], bq[4 * hv + 2], bq[4 * hv + 3]);
                 }
                 if (k + L < NK) fetch(curQ, k + L, slotQ); else fetch(nxtQ, k + L - NK, slotQ);
             }
 
-            // ---------------- combine: warp -> CTA -> cluster ----------------
-            float sPw = sP, sQw = sQ;
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                sPw += __shfl_xor_sync(0xffffffffu, sPw, off);
-                sQw += __shfl_xor_sync(0xffffffffu, sQw, off);
-            }
-            if (lane == 0) {
-                sh.red_M[0][warp] = MPw; sh.red_s[0][warp] = static_cast<double>(sPw);
-                sh.red_M[1][warp] = MQw; sh.red_s[1][warp] = static_cast<double>(sQw);
-            }
-            __syncthreads();
-            if (warp == 0) {
-#pragma unroll
-                for (int row = 0; row < 2; ++row) {
-                    float M = lane < kRWarps ? sh.red_M[row][lane] : -INFINITY;
-                    double s = lane < kRWarps ? sh.red_s[row][lane] : 0.0;
-                    float Mc = M;
-#pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) Mc = fmaxf(Mc, __shfl_xor_sync(0xffffffffu, Mc, off));
-                    s = (s != s) ? s : s * static_cast<double>(pow2_nonpos(M - Mc));
-#pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) s += shfl_xor_d(s, off);
-                    if (lane < C) {
-                        *cluster.map_shared_rank(&sh.x_M[row][rank], lane) = Mc;
-                        *cluster.map_shared_rank(&sh.x_s[row][rank], lane) = s;
-                    }
-                }
+            // ---------------- publish this warp's partials to every CTA ----------------
+            sP = warp_sum(sP);
+            sQ = warp_sum(sQ);
+            if (lane < C) {
+                ResShared* peer = cluster.map_shared_rank(&sh, lane);
+                peer->x_M[0][myseg] = MPw; peer->x_s[0][myseg] = sP;
+                peer->x_M[1][myseg] = MQw; peer->x_s[1][myseg] = sQ;
             }
             cluster.sync();
 
-            // ---------------- scalars ----------------
+            // ---------------- row normalisers and the scale of sweep 2 (warp 0) ----------------
+            double ZP = 0.0, ZQ = 0.0;     // meaningful in thread 0
+            float MPr = 0.f, MQr = 0.f;
             if (warp == 0) {
-                const int row = (lane >> 3) & 1, rk = lane & 7;
-                const bool live = lane < 16 && rk < C;
-                float M = live ? sh.x_M[row][rk] : -INFINITY;
-                double s = live ? sh.x_s[row][rk] : 0.0;
-                float Mr = M;
+                float m[2];
+                double z[2];
 #pragma unroll
-                for (int off = 4; off > 0; off >>= 1) Mr = fmaxf(Mr, __shfl_xor_sync(0xffffffffu, Mr, off));
-                s = (s != s) ? s : s * static_cast<double>(pow2_nonpos(M - Mr));
+                for (int row = 0; row < 2; ++row) {
+                    const float4 M4 = reinterpret_cast<const float4*>(sh.x_M[row])[lane];
+                    const float4 s4 = reinterpret_cast<const float4*>(sh.x_s[row])[lane];
+                    const float Mr = warp_max(fmaxf(fmaxf(M4.x, M4.y), fmaxf(M4.z, M4.w)));
+                    double s = static_cast<double>(s4.x) * ref_scale(M4.x, Mr) +
+                               static_cast<double>(s4.y) * ref_scale(M4.y, Mr) +
+                               static_cast<double>(s4.z) * ref_scale(M4.z, Mr) +
+                               static_cast<double>(s4.w) * ref_scale(M4.w, Mr);
 #pragma unroll
-                for (int off = 4; off > 0; off >>= 1) s += shfl_xor_d(s, off);
-                const float MQ = __shfl_sync(0xffffffffu, Mr, 8);
-                const double ZQ = shfl_d(s, 8);
+                    for (int off = 16; off > 0; off >>= 1) s += shfl_xor_d(s, off);
+                    m[row] = Mr; z[row] = s;
+                }
+                MPr = m[0]; MQr = m[1]; ZP = z[0]; ZQ = z[1];
                 if (lane == 0) {
-                    const float MP = Mr;
-                    const double ZP = s;
-                    const double ln2 = 0.693147180559945309417232;
-                    int bad = sh.bad;
-                    if (!(fabsf(MP) < INFINITY) || !(ZP < INFINITY)) bad = 1;   // also catches NaN
-                    if (have_q && (!(fabsf(MQ) < INFINITY) || !(ZQ < INFINITY))) bad = 1;
-                    const double lse2P = static_cast<double>(MP) + log2(ZP);
-                    const double lse2Q = static_cast<double>(MQ) + log2(ZQ);
-                    sh.lse_t[r] = lse2P * ln2;
-                    if (have_q) sh.lse_d[r] = lse2Q * ln2;
-                    const double p_r = sh.p[r];
-                    if (have_q) {
-                        double ratio = 0.0;
-                        const int x = prm.tok[static_cast<size_t>(b) * g + r];
-                        if (x < 0 || x >= V) {
-                            bad = 1;
-                        } else {
-                            const double zq = load_logit<DT>(curQ, x), zp = load_logit<DT>(curP, x);
-                            if (zq == -INFINITY) bad = 1;
-                            else ratio = exp2((zp * kd - lse2P) - (zq * kd - lse2Q));
-                        }
-                        sh.p[r + 1] = fmin(p_r * ratio, 1.0);
-                    }
-                    sh.bad = bad;
-                    sh.c = have_q ? static_cast<float>(p_r * ZQ / ZP) : 1.f;
-                    sh.MP = MP;
-                    sh.MQ = MQ;
-                    sh.invZQ = have_q ? 1.0 / ZQ : 1.0 / ZP;
+                    sh.c = have_q ? static_cast<float>(sh.p[r] * ZQ / ZP) : 1.f;
+                    sh.MP = MPr;
+                    sh.MQ = MQr;
                     if (rank == 0) sh.cand[r] = -1;
                 }
             }
             __syncthreads();
 
+            // thread 0, overlapped with sweep 2: data checks and p_{r+1} = min(p_r ratio, 1)
+            double invZ = 0.0;
+            if (tid == 0) {
+                int bad = sh.bad;
+                // the row's maximum is finite iff its reference is; Z is NaN / inf iff the row
+                // holds a NaN / the sum overflowed
+                if (!(MPr > kNoRef && MPr < INFINITY) || !(ZP < INFINITY)) bad = 1;
+                if (have_q && (!(MQr > kNoRef && MQr < INFINITY) || !(ZQ < INFINITY))) bad = 1;
+                if (have_q) {
+                    double ratio = 0.0;
+                    if (!x_ok || zq_x == -INFINITY) bad = 1;
+                    else ratio = exp2((zp_x - zq_x) * kd - static_cast<double>(MPr - MQr)) * (ZQ / ZP);
+                    sh.p[r + 1] = fmin(sh.p[r] * ratio, 1.0);
+                }
+                sh.bad = bad;
+                invZ = have_q ? 1.0 / ZQ : 1.0 / ZP;
+                if (prm.out_lse_t) {
+                    const double ln2 = 0.693147180559945309417232;
+                    sh.lse_t[r] = (static_cast<double>(MPr) + log2(ZP)) * ln2;
+                    if (have_q) sh.lse_d[r] = (static_cast<double>(MQr) + log2(ZQ)) * ln2;
+                }
+            }
+
             // ---------------- sweep 2 + candidate ----------------
-            const float c = sh.c;
-            const float cPt = c * pow2_nonpos(MPw - sh.MP);     // exact rescale to the row reference
-            const float cQt = pow2_nonpos(MQw - sh.MQ);
+            const float cPw = ref_scale(MPw, sh.MP);      // exact rescale to the row references
+            const float cQw = ref_scale(MQw, sh.MQ);
             bool use_q = have_q;
             for (int attempt = 0; attempt < 2; ++attempt) {
-                const float cp = use_q ? cPt : pow2_nonpos(MPw - sh.MP);
+                const float cp = use_q ? sh.c * cPw : cPw;
+                const float cq = use_q ? cQw : 0.f;
                 float acc = 0.f;
 #pragma unroll
                 for (int k = 0; k < NK; ++k) {
                     float bq[EPV];
 #pragma unroll
                     for (int hv = 0; hv < HV; ++hv) {
-                        const float4 f = bcache[(k * HV + hv) * kRThreads + tid];
+                        const float4 f = bcache[(k * HV + hv) * kRThreads];
                         bq[4 * hv] = f.x; bq[4 * hv + 1] = f.y; bq[4 * hv + 2] = f.z; bq[4 * hv + 3] = f.w;
                     }
                     float v = 0.f;
 #pragma unroll
-                    for (int e = 0; e < EPV; ++e) {
-                        const float q = use_q ? cQt * bq[e] : 0.f;
-                        v += fmaxf(fmaf(cp, a[k][e], -q), 0.f);
-                    }
+                    for (int e = 0; e < EPV; ++e) v += fmaxf(fmaf(cp, a[k][e], -(cq * bq[e])), 0.f);
                     acc += v;
                 }
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-                if (lane == 0) sh.segtot[warp] = static_cast<double>(acc);
-                __syncthreads();
-                if (warp == 0) {
-                    double v = lane < kRWarps ? sh.segtot[lane] : 0.0;
-#pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) v += shfl_xor_d(v, off);
-                    if (lane < C) *cluster.map_shared_rank(&sh.x_tot[rank], lane) = v;
-                }
+                acc = warp_sum(acc);
+                if (lane < C) cluster.map_shared_rank(&sh, lane)->x_seg[myseg] = acc;
                 cluster.sync();
 
-                double total = 0.0;
-                for (int k = 0; k < C; ++k) total += sh.x_tot[k];
-                if (attempt == 0 && use_q && tid == 0) sh.S[r] = total * sh.invZQ;
-                const bool empty = !(total > 0.0);
+                // every warp locates u * total among the 128 segment totals (index order)
+                const float4 t4 = reinterpret_cast<const float4*>(sh.x_seg)[lane];
+                const float l1 = t4.x, l2 = l1 + t4.y, l3 = l2 + t4.z, l4 = l3 + t4.w;
+                float inc = l4;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const float o = __shfl_up_sync(0xffffffffu, inc, off);
+                    if (lane >= off) inc += o;
+                }
+                const float total = __shfl_sync(0xffffffffu, inc, 31);
+                if (attempt == 0 && use_q && tid == 0) {
+                    // S_r in double from the same 128 partials
+                    double sd = static_cast<double>(t4.x) + static_cast<double>(t4.y) +
+                                static_cast<double>(t4.z) + static_cast<double>(t4.w);
+                    (void)sd;
+                }
+                if (attempt == 0 && use_q && warp == 0) {
+                    double sd = (static_cast<double>(t4.x) + static_cast<double>(t4.y)) +
+                                (static_cast<double>(t4.z) + static_cast<double>(t4.w));
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
+                    if (lane == 0) sh.S[r] = sd * invZ;
+                }
+                const bool empty = !(total > 0.f);
                 if (empty && use_q && attempt == 0 && r == 0) {
                     use_q = false;   // empty residual at position 0: sample P_0 with the same uniform
-                    cluster.sync();
+                    cluster.sync();  // everyone has read x_seg before it is rewritten
                     continue;
                 }
                 if (!empty) {
                     const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
-                    const double t = static_cast<double>(uf) * total;
-                    int sel = -1, lastnz = -1;
-                    double run = 0.0, sel_before = 0.0, nz_before = 0.0;
-                    for (int k = 0; k < C; ++k) {
-                        const double v = sh.x_tot[k];
-                        if (v > 0.0) { lastnz = k; nz_before = run; }
-                        if (sel < 0 && run + v > t) { sel = k; sel_before = run; }
-                        run += v;
+                    const float t = uf * total;
+                    const float exc = inc - l4;
+                    // first segment whose inclusive prefix exceeds t, else the last non-empty one
+                    const unsigned hit = __ballot_sync(0xffffffffu, inc > t);
+                    const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
+                    int sel_seg = -1;
+                    float sel_before = 0.f;
+                    if (hit) {
+                        const int src = __ffs(hit) - 1;
+                        int e = 3; float bef = exc + l3;
+                        if (exc + l1 > t) { e = 0; bef = exc; }
+                        else if (exc + l2 > t) { e = 1; bef = exc + l1; }
+                        else if (exc + l3 > t) { e = 2; bef = exc + l2; }
+                        sel_seg = __shfl_sync(0xffffffffu, 4 * lane + e, src);
+                        sel_before = __shfl_sync(0xffffffffu, bef, src);
+                    } else if (nz) {
+                        const int src = 31 - __clz(nz);
+                        int e = 0; float bef = exc;
+                        if (t4.w > 0.f) { e = 3; bef = exc + l3; }
+                        else if (t4.z > 0.f) { e = 2; bef = exc + l2; }
+                        else if (t4.y > 0.f) { e = 1; bef = exc + l1; }
+                        sel_seg = __shfl_sync(0xffffffffu, 4 * lane + e, src);
+                        sel_before = __shfl_sync(0xffffffffu, bef, src);
                     }
-                    if (sel < 0) { sel = lastnz; sel_before = nz_before; }
-                    if (sel == rank) {
-                        const double tc = t - sel_before;
-                        int wsel = -1, wlast = -1;
-                        double wrun = 0.0, wsel_before = 0.0, wnz_before = 0.0;
-                        for (int k = 0; k < kRWarps; ++k) {
-                            const double v = sh.segtot[k];
-                            if (v > 0.0) { wlast = k; wnz_before = wrun; }
-                            if (wsel < 0 && wrun + v > tc) { wsel = k; wsel_before = wrun; }
-                            wrun += v;
-                        }
-                        if (wsel < 0) { wsel = wlast; wsel_before = wnz_before; }
-                        if (warp == wsel) {
-                            // rescan this warp's cached terms in index order
-                            const double tw = tc - wsel_before;
-                            double runw = 0.0;
-                            int found = -1, last_pos = -1;
+                    if (sel_seg == myseg) {
+                        // rescan this warp's cached terms in index order
+                        const float tw = t - sel_before;
+                        float runw = 0.f;
+                        int found = -1, last_pos = -1;
 #pragma unroll
-                            for (int k = 0; k < NK; ++k) {
-                                if (found < 0) {
-                                    float tt[EPV];
-                                    float ls = 0.f;
-#pragma unroll
-                                    for (int hv = 0; hv < HV; ++hv) {
-                                        const float4 f = bcache[(k * HV + hv) * kRThreads + tid];
-                                        tt[4 * hv] = f.x; tt[4 * hv + 1] = f.y; tt[4 * hv + 2] = f.z; tt[4 * hv + 3] = f.w;
-                                    }
-                                    const int i = v0 + 32 * k;
-#pragma unroll
-                                    for (int e = 0; e < EPV; ++e) {
-                                        const float q = use_q ? cQt * tt[e] : 0.f;
-                                        tt[e] = fmaxf(fmaf(cp, a[k][e], -q), 0.f);
-                                        ls += tt[e];
-                                        if (tt[e] > 0.f) last_pos = i * EPV + e;
-                                    }
-                                    double inc = static_cast<double>(ls);
-#pragma unroll
-                                    for (int off = 1; off < 32; off <<= 1) {
-                                        const double o = shfl_up_d(inc, off);
-                                        if (lane >= off) inc += o;
-                                    }
-                                    const bool hit = runw + inc > tw;
-                                    const unsigned bal = __ballot_sync(0xffffffffu, hit);
-                                    if (bal) {
-                                        const int src = __ffs(bal) - 1;
-                                        int f = -1;
-                                        if (lane == src) {
-                                            double cum = runw + inc - static_cast<double>(ls);
-                                            int lp = -1;
-#pragma unroll
-                                            for (int e = 0; e < EPV; ++e) {
-                                                cum += static_cast<double>(tt[e]);
-                                                if (tt[e] > 0.f) lp = i * EPV + e;
-                                                if (f < 0 && cum > tw && tt[e] > 0.f) f = i * EPV + e;
-                                            }
-                                            if (f < 0) f = lp;
-                                        }
-                                        f = __shfl_sync(0xffffffffu, f, src);
-                                        if (f >= 0) found = f;
-                                    }
-                                    runw += shfl_d(inc, 31);
-                                }
-                            }
+                        for (int k = 0; k < NK; ++k) {
                             if (found < 0) {
+                                float tt[EPV];
 #pragma unroll
-                                for (int off = 16; off > 0; off >>= 1)
-                                    last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, off));
-                                found = last_pos;
+                                for (int hv = 0; hv < HV; ++hv) {
+                                    const float4 f = bcache[(k * HV + hv) * kRThreads];
+                                    tt[4 * hv] = f.x; tt[4 * hv + 1] = f.y; tt[4 * hv + 2] = f.z; tt[4 * hv + 3] = f.w;
+                                }
+                                const int i = v0 + 32 * k;
+                                float ls = 0.f;
+#pragma unroll
+                                for (int e = 0; e < EPV; ++e) {
+                                    tt[e] = fmaxf(fmaf(cp, a[k][e], -(cq * tt[e])), 0.f);
+                                    ls += tt[e];
+                                    if (tt[e] > 0.f) last_pos = i * EPV + e;
+                                }
+                                float incw = ls;
+#pragma unroll
+                                for (int off = 1; off < 32; off <<= 1) {
+                                    const float o = __shfl_up_sync(0xffffffffu, incw, off);
+                                    if (lane >= off) incw += o;
+                                }
+                                const unsigned bal = __ballot_sync(0xffffffffu, runw + incw > tw);
+                                if (bal) {
+                                    const int src = __ffs(bal) - 1;
+                                    int f = -1;
+                                    if (lane == src) {
+                                        float cum = runw + incw - ls;
+                                        int lp = -1;
+#pragma unroll
+                                        for (int e = 0; e < EPV; ++e) {
+                                            cum += tt[e];
+                                            if (tt[e] > 0.f) lp = i * EPV + e;
+                                            if (f < 0 && cum > tw && tt[e] > 0.f) f = i * EPV + e;
+                                        }
+                                        if (f < 0) f = lp;
+                                    }
+                                    f = __shfl_sync(0xffffffffu, f, src);
+                                    if (f >= 0) found = f;
+                                }
+                                runw += __shfl_sync(0xffffffffu, incw, 31);
                             }
-                            if (lane == 0) *cluster.map_shared_rank(&sh.cand[r], 0) = found;
                         }
+                        if (found < 0) {
+#pragma unroll
+                            for (int off = 16; off > 0; off >>= 1)
+                                last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, off));
+                            found = last_pos;
+                        }
+                        if (lane == 0) *cluster.map_shared_rank(&sh.cand[r], 0) = found;
                     }
                 }
                 break;
@@ -515,6 +521,7 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
         }
     }
     cp_async_wait<0>();
+    cluster.sync();   // no CTA exits while a peer may still write into its shared memory
 }
 
 // ---------------------------------------------------------------------------
