@@ -54,9 +54,10 @@ int device_state(DeviceState** out) {
         if ((e = cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
             return cuda_fail(e);
         if (d.cc_major < 10) return BV_ERR_UNSUPPORTED;
-        if ((e = cudaMalloc(&d.tickets, sizeof(unsigned int) * 2 * kTicketSlots)) != cudaSuccess)
+        // ticket slots, then one status word that a kernel sets if a bounded wait gives up
+        if ((e = cudaMalloc(&d.tickets, sizeof(unsigned int) * (2 * kTicketSlots + 1))) != cudaSuccess)
             return cuda_fail(e);
-        if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned int) * 2 * kTicketSlots)) != cudaSuccess)
+        if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned int) * (2 * kTicketSlots + 1))) != cudaSuccess)
             return cuda_fail(e);
         d.ready = true;
     }
@@ -119,6 +120,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     prm.out_tokens = ot; prm.out_len = ol;
     prm.out_p = out_p; prm.out_S = out_S; prm.out_h = out_h;
     prm.out_lse_t = out_lse_t; prm.out_lse_d = out_lse_d;
+    prm.status = reinterpret_cast<int*>(d->tickets + 2 * kTicketSlots);
 
     // Block Verification on 16-byte rows: the kernel that keeps each row pair on chip,
     // when some cluster width lets a thread hold its share (at most 8 vectors per row).
@@ -189,6 +191,7 @@ int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, con
 
     char* base = nullptr;
     cudaStream_t s = nullptr;
+    int* status_word = nullptr;
     {
         std::lock_guard<std::mutex> lock(g_mu);
         DeviceState* d = nullptr;
@@ -205,6 +208,7 @@ int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, con
         }
         base = static_cast<char*>(d->stage);
         s = d->stream;
+        status_word = reinterpret_cast<int*>(d->tickets + 2 * kTicketSlots);
     }
     cudaError_t e;
     if ((e = cudaMemcpyAsync(base + o_t, tgt, n_t, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
@@ -218,8 +222,11 @@ int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, con
     if (rc != BV_OK) return rc;
     if ((e = cudaMemcpyAsync(ot, base + o_ot, n_ot, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaMemcpyAsync(ol, base + o_ol, n_ol, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    int status = 0;
+    if ((e = cudaMemcpyAsync(&status, status_word, sizeof(int), cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+        return cuda_fail(e);
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
-    return BV_OK;
+    return status ? BV_ERR_TIMEOUT : BV_OK;
 }
 
 }  // namespace

@@ -29,6 +29,7 @@ struct Params {
     float* out_lse_t;
     float* out_lse_d;
     unsigned int* ticket;     // [2]: next sequence index, clusters that have finished
+    int* status;              // set to 1 if a bounded device-side wait gave up
     int nclusters;            // clusters in the grid
 };
 

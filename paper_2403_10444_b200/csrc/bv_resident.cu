@@ -45,12 +45,13 @@ constexpr float kRaiseBound = 12.f;
 constexpr float kNoRef = -3.0e38f;
 
 struct ResShared {
-    // sweep 1: (reference, sum) of every warp of every CTA, written by the owners into
-    // every CTA of the cluster: [P/Q][rank * 16 + warp]
-    float x_M[2][kSegs];
-    float x_s[2][kSegs];
+    // sweep 1: {reference P, sum P, reference Q, sum Q} of every warp of every CTA, sent by
+    // the owners to every CTA of the cluster; index rank * 16 + warp
+    float4 x_ms[kSegs];
     // sweep 2: segment totals of every warp of every CTA, same indexing
     float x_seg[kSegs];
+    // transaction barriers that count the bytes of the two exchanges and of the candidates
+    unsigned long long bar_ms, bar_seg, bar_cand;
     double p[kMaxGamma + 1];
     double S[kMaxGamma + 1];
     double h[kMaxGamma + 1];
@@ -76,6 +77,51 @@ __device__ __forceinline__ void ring_fetch(void* slot, const void* src, bool pre
         "@!p st.shared.v4.b32 [%0], {%3, %3, %3, %3};\n\t"
         "cp.async.commit_group;\n\t}"
         ::"r"(s), "l"(src), "r"(static_cast<int>(pred)), "r"(fill) : "memory");
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+// address of the same shared-memory location in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, int rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Wait for the phase with the given parity.  The wait is bounded: after about a second it
+// gives up, records the fact in *status and returns, so a protocol error cannot hang the GPU.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return;
+        // give up after about a second, or at once if another wait has already given up
+        if (clock64() - t0 > 2000000000LL || (status && *reinterpret_cast<volatile int*>(status))) {
+            if (status) atomicExch(status, 1);
+            return;
+        }
+    }
+}
+// 16 or 4 bytes into another CTA's shared memory; the bytes are counted by that CTA's barrier
+__device__ __forceinline__ void send_v4(uint32_t raddr, uint32_t rbar, float a, float b, float c, float d) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(raddr), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)),
+                   "r"(__float_as_uint(d)), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void send_b32(uint32_t raddr, uint32_t rbar, uint32_t v) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(raddr), "r"(v), "r"(rbar) : "memory");
 }
 
 template <int DT> struct Raw;
@@ -119,10 +165,11 @@ __device__ __forceinline__ float warp_sum(float x) {
 template <int EPV>
 __device__ __forceinline__ float expo(const float (&v)[EPV], float kf, float M, float (&a)[EPV]) {
     const float nM = -M;
-    float vs = 0.f;
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) { a[e] = ex2(fmaf(v[e], kf, nM)); vs += a[e]; }
-    return vs;
+    for (int e = 0; e < EPV; ++e) a[e] = ex2(fmaf(v[e], kf, nM));
+    float s0 = a[0] + a[1], s1 = a[2] + a[3];
+    if (EPV == 8) { s0 += a[4] + a[5]; s1 += a[6] + a[7]; }
+    return s0 + s1;
 }
 
 // 2^d for d = (own reference) - (row reference) <= 0, or 0 when there is no own reference
@@ -170,9 +217,26 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
 
     // unused slots of the exchange arrays (ranks >= C) stay neutral for the whole kernel
     if (tid < kSegs) {
-        sh.x_M[0][tid] = kNoRef; sh.x_M[1][tid] = kNoRef;
-        sh.x_s[0][tid] = 0.f; sh.x_s[1][tid] = 0.f; sh.x_seg[tid] = 0.f;
+        sh.x_ms[tid] = make_float4(kNoRef, 0.f, kNoRef, 0.f);
+        sh.x_seg[tid] = 0.f;
     }
+    if (tid == 0) {
+        mbar_init(smem_u32(&sh.bar_ms), 1);
+        mbar_init(smem_u32(&sh.bar_seg), 1);
+        mbar_init(smem_u32(&sh.bar_cand), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // where this warp's messages go: lane l < C addresses CTA l of the cluster
+    const int peer = lane < C ? lane : 0;
+    const uint32_t r_ms = map_to_rank(smem_u32(&sh.x_ms[myseg]), peer);
+    const uint32_t r_seg = map_to_rank(smem_u32(&sh.x_seg[myseg]), peer);
+    const uint32_t r_bar_ms = map_to_rank(smem_u32(&sh.bar_ms), peer);
+    const uint32_t r_bar_seg = map_to_rank(smem_u32(&sh.bar_seg), peer);
+    const uint32_t r_bar_cand = map_to_rank(smem_u32(&sh.bar_cand), 0);
+    const uint32_t bytes_ms = static_cast<uint32_t>(C) * kRWarps * 16u;
+    const uint32_t bytes_seg = static_cast<uint32_t>(C) * kRWarps * 4u;
+    uint32_t ph_ms = 0, ph_seg = 0, ph_cand = 0;     // phase parities of the three barriers
+    int* const status = prm.status;
 
     auto rowP = [&](int b, int r) -> const char* {
         return static_cast<const char*>(prm.tgt) + (static_cast<size_t>(b) * (g + 1) + r) * row_bytes + toff;
@@ -194,10 +258,13 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
             fetch(q0, k, 2 * k + 1);
         }
     }
-    cluster.sync();   // exchange arrays are initialised everywhere before any remote write
+    cluster.sync();   // barriers and exchange arrays are ready everywhere before any message
 
     for (int b = cid; b < B; b += ncl) {
-        if (tid == 0) { sh.bad = 0; sh.p[0] = 1.0; }
+        if (tid == 0) {
+            sh.bad = 0; sh.p[0] = 1.0;
+            if (rank == 0) mbar_arrive_expect(smem_u32(&sh.bar_cand), 4u * static_cast<uint32_t>(g + 1));
+        }
         for (int r = 0; r <= g; ++r) {
             const bool have_q = r < g;
             int nb = b, nr = r + 1;
@@ -207,6 +274,10 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
             const char* nxtP = nb < B ? rowP(nb, nr) : nullptr;
             const char* nxtQ = (nb < B && nr < g) ? rowQ(nb, nr) : nullptr;
 
+            if (tid == 0) {
+                mbar_arrive_expect(smem_u32(&sh.bar_ms), bytes_ms);
+                mbar_arrive_expect(smem_u32(&sh.bar_seg), bytes_seg);
+            }
             // thread 0 fetches the drafted token's two logits early (used after the combine)
             double zp_x = 0.0, zq_x = 0.0;
             int x_ok = 1;
@@ -225,99 +296,84 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
 #pragma unroll
             for (int k = 0; k < NK; ++k) {
                 const int slotP = (2 * k) % D, slotQ = (2 * k + 1) % D;
-                // ---- target row ----
-                cp_async_wait<D - 1>();
-                {
-                    float v[EPV];
-                    R::unpack(ring[slotP * kRThreads], v);
-                    if (k == 0) MPw = fmaxf(rintf(warp_max(vec_max<EPV>(v)) * kf), kNoRef);
-                    float vs = expo<EPV>(v, kf, MPw, a[k]);
-                    if (__any_sync(0xffffffffu, vs > kRaiseBound)) {
-                        const float y = rintf(warp_max(vec_max<EPV>(v)) * kf);
-                        if (y > MPw) {
-                            const float f = ref_scale(MPw, y);
-                            sP *= f;
-#pragma unroll
-                            for (int kk = 0; kk < k; ++kk)
-#pragma unroll
-                                for (int e = 0; e < EPV; ++e) a[kk][e] *= f;
-                            MPw = y;
-                        }
-                        vs = expo<EPV>(v, kf, MPw, a[k]);
-                    }
-                    sP += vs;
+                cp_async_wait<D - 2>();          // vectors k of both rows have landed
+                float vp[EPV], vq[EPV], bq[EPV];
+                R::unpack(ring[slotP * kRThreads], vp);
+                R::unpack(ring[slotQ * kRThreads], vq);   // -inf pattern when there is no draft row
+                if (k == 0) {
+                    MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
+                    MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vq)) * kf), kNoRef);
                 }
-                if (k + L < NK) fetch(curP, k + L, slotP); else fetch(nxtP, k + L - NK, slotP);
-                // ---- draft row (slots hold -inf when there is none) ----
-                cp_async_wait<D - 1>();
-                {
-                    float v[EPV], bq[EPV];
-                    R::unpack(ring[slotQ * kRThreads], v);
-                    if (k == 0) MQw = fmaxf(rintf(warp_max(vec_max<EPV>(v)) * kf), kNoRef);
-                    float vs = expo<EPV>(v, kf, MQw, bq);
-                    if (__any_sync(0xffffffffu, vs > kRaiseBound)) {
-                        const float y = rintf(warp_max(vec_max<EPV>(v)) * kf);
-                        if (y > MQw) {
-                            const float f = ref_scale(MQw, y);
-                            sQ *= f;
+                float vsP = expo<EPV>(vp, kf, MPw, a[k]);
+                float vsQ = expo<EPV>(vq, kf, MQw, bq);
+                if (__any_sync(0xffffffffu, vsP > kRaiseBound)) {
+                    const float y = rintf(warp_max(vec_max<EPV>(vp)) * kf);
+                    if (y > MPw) {
+                        const float f = ref_scale(MPw, y);
+                        sP *= f;
 #pragma unroll
-                            for (int kk = 0; kk < k; ++kk)
+                        for (int kk = 0; kk < k; ++kk)
 #pragma unroll
-                                for (int hv = 0; hv < HV; ++hv) {
-                                    float4 t4 = bcache[(kk * HV + hv) * kRThreads];
-                                    t4.x *= f; t4.y *= f; t4.z *= f; t4.w *= f;
-                                    bcache[(kk * HV + hv) * kRThreads] = t4;
-                                }
-                            MQw = y;
-                        }
-                        vs = expo<EPV>(v, kf, MQw, bq);
+                            for (int e = 0; e < EPV; ++e) a[kk][e] *= f;
+                        MPw = y;
                     }
-                    sQ += vs;
-#pragma unroll
-                    for (int hv = 0; hv < HV; ++hv)
-                        bcache[(k * HV + hv) * kRThreads] =
-                            make_float4(bq[4 * hv], bq[4 * hv + 1], bq[4 * hv + 2], bq[4 * hv + 3]);
+                    vsP = expo<EPV>(vp, kf, MPw, a[k]);
                 }
-                if (k + L < NK) fetch(curQ, k + L, slotQ); else fetch(nxtQ, k + L - NK, slotQ);
+                if (__any_sync(0xffffffffu, vsQ > kRaiseBound)) {
+                    const float y = rintf(warp_max(vec_max<EPV>(vq)) * kf);
+                    if (y > MQw) {
+                        const float f = ref_scale(MQw, y);
+                        sQ *= f;
+#pragma unroll
+                        for (int kk = 0; kk < k; ++kk)
+#pragma unroll
+                            for (int hv = 0; hv < HV; ++hv) {
+                                float4 t4 = bcache[(kk * HV + hv) * kRThreads];
+                                t4.x *= f; t4.y *= f; t4.z *= f; t4.w *= f;
+                                bcache[(kk * HV + hv) * kRThreads] = t4;
+                            }
+                        MQw = y;
+                    }
+                    vsQ = expo<EPV>(vq, kf, MQw, bq);
+                }
+                sP += vsP;
+                sQ += vsQ;
+#pragma unroll
+                for (int hv = 0; hv < HV; ++hv)
+                    bcache[(k * HV + hv) * kRThreads] =
+                        make_float4(bq[4 * hv], bq[4 * hv + 1], bq[4 * hv + 2], bq[4 * hv + 3]);
+                if (k + L < NK) { fetch(curP, k + L, slotP); fetch(curQ, k + L, slotQ); }
+                else            { fetch(nxtP, k + L - NK, slotP); fetch(nxtQ, k + L - NK, slotQ); }
             }
 
             // ---------------- publish this warp's partials to every CTA ----------------
             sP = warp_sum(sP);
             sQ = warp_sum(sQ);
-            if (lane < C) {
-                ResShared* peer = cluster.map_shared_rank(&sh, lane);
-                peer->x_M[0][myseg] = MPw; peer->x_s[0][myseg] = sP;
-                peer->x_M[1][myseg] = MQw; peer->x_s[1][myseg] = sQ;
-            }
-            cluster.sync();
+            if (lane < C) send_v4(r_ms, r_bar_ms, MPw, sP, MQw, sQ);
 
             // ---------------- row normalisers and the scale of sweep 2 (warp 0) ----------------
             double ZP = 0.0, ZQ = 0.0;     // meaningful in thread 0
             float MPr = 0.f, MQr = 0.f;
             if (warp == 0) {
-                float m[2];
-                double z[2];
+                mbar_wait(smem_u32(&sh.bar_ms), ph_ms, status);
+                // lane l combines segments 4l .. 4l+3
+                const float4 e0 = sh.x_ms[4 * lane], e1 = sh.x_ms[4 * lane + 1];
+                const float4 e2 = sh.x_ms[4 * lane + 2], e3 = sh.x_ms[4 * lane + 3];
+                MPr = warp_max(fmaxf(fmaxf(e0.x, e1.x), fmaxf(e2.x, e3.x)));
+                MQr = warp_max(fmaxf(fmaxf(e0.z, e1.z), fmaxf(e2.z, e3.z)));
+                ZP = static_cast<double>(e0.y) * ref_scale(e0.x, MPr) + static_cast<double>(e1.y) * ref_scale(e1.x, MPr) +
+                     static_cast<double>(e2.y) * ref_scale(e2.x, MPr) + static_cast<double>(e3.y) * ref_scale(e3.x, MPr);
+                ZQ = static_cast<double>(e0.w) * ref_scale(e0.z, MQr) + static_cast<double>(e1.w) * ref_scale(e1.z, MQr) +
+                     static_cast<double>(e2.w) * ref_scale(e2.z, MQr) + static_cast<double>(e3.w) * ref_scale(e3.z, MQr);
 #pragma unroll
-                for (int row = 0; row < 2; ++row) {
-                    const float4 M4 = reinterpret_cast<const float4*>(sh.x_M[row])[lane];
-                    const float4 s4 = reinterpret_cast<const float4*>(sh.x_s[row])[lane];
-                    const float Mr = warp_max(fmaxf(fmaxf(M4.x, M4.y), fmaxf(M4.z, M4.w)));
-                    double s = static_cast<double>(s4.x) * ref_scale(M4.x, Mr) +
-                               static_cast<double>(s4.y) * ref_scale(M4.y, Mr) +
-                               static_cast<double>(s4.z) * ref_scale(M4.z, Mr) +
-                               static_cast<double>(s4.w) * ref_scale(M4.w, Mr);
-#pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) s += shfl_xor_d(s, off);
-                    m[row] = Mr; z[row] = s;
-                }
-                MPr = m[0]; MQr = m[1]; ZP = z[0]; ZQ = z[1];
+                for (int off = 16; off > 0; off >>= 1) { ZP += shfl_xor_d(ZP, off); ZQ += shfl_xor_d(ZQ, off); }
                 if (lane == 0) {
                     sh.c = have_q ? static_cast<float>(sh.p[r] * ZQ / ZP) : 1.f;
                     sh.MP = MPr;
                     sh.MQ = MQr;
-                    if (rank == 0) sh.cand[r] = -1;
                 }
             }
+            ph_ms ^= 1u;
             __syncthreads();
 
             // thread 0, overlapped with sweep 2: data checks and p_{r+1} = min(p_r ratio, 1)
@@ -351,22 +407,26 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
                 const float cp = use_q ? sh.c * cPw : cPw;
                 const float cq = use_q ? cQw : 0.f;
                 float acc = 0.f;
+                float vsum[NK];      // this thread's residual mass per vector, kept for the rescan
 #pragma unroll
                 for (int k = 0; k < NK; ++k) {
-                    float bq[EPV];
+                    float bq[EPV], tt[EPV];
 #pragma unroll
                     for (int hv = 0; hv < HV; ++hv) {
                         const float4 f = bcache[(k * HV + hv) * kRThreads];
                         bq[4 * hv] = f.x; bq[4 * hv + 1] = f.y; bq[4 * hv + 2] = f.z; bq[4 * hv + 3] = f.w;
                     }
-                    float v = 0.f;
 #pragma unroll
-                    for (int e = 0; e < EPV; ++e) v += fmaxf(fmaf(cp, a[k][e], -(cq * bq[e])), 0.f);
-                    acc += v;
+                    for (int e = 0; e < EPV; ++e) tt[e] = fmaxf(fmaf(cp, a[k][e], -(cq * bq[e])), 0.f);
+                    float s0 = tt[0] + tt[1], s1 = tt[2] + tt[3];
+                    if (EPV == 8) { s0 += tt[4] + tt[5]; s1 += tt[6] + tt[7]; }
+                    vsum[k] = s0 + s1;
+                    acc += vsum[k];
                 }
                 acc = warp_sum(acc);
-                if (lane < C) cluster.map_shared_rank(&sh, lane)->x_seg[myseg] = acc;
-                cluster.sync();
+                if (lane < C) send_b32(r_seg, r_bar_seg, __float_as_uint(acc));
+                mbar_wait(smem_u32(&sh.bar_seg), ph_seg, status);
+                ph_seg ^= 1u;
 
                 // every warp locates u * total among the 128 segment totals (index order)
                 const float4 t4 = reinterpret_cast<const float4*>(sh.x_seg)[lane];
@@ -378,12 +438,6 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
                     if (lane >= off) inc += o;
                 }
                 const float total = __shfl_sync(0xffffffffu, inc, 31);
-                if (attempt == 0 && use_q && tid == 0) {
-                    // S_r in double from the same 128 partials
-                    double sd = static_cast<double>(t4.x) + static_cast<double>(t4.y) +
-                                static_cast<double>(t4.z) + static_cast<double>(t4.w);
-                    (void)sd;
-                }
                 if (attempt == 0 && use_q && warp == 0) {
                     double sd = (static_cast<double>(t4.x) + static_cast<double>(t4.y)) +
                                 (static_cast<double>(t4.z) + static_cast<double>(t4.w));
@@ -394,100 +448,110 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
                 const bool empty = !(total > 0.f);
                 if (empty && use_q && attempt == 0 && r == 0) {
                     use_q = false;   // empty residual at position 0: sample P_0 with the same uniform
-                    cluster.sync();  // everyone has read x_seg before it is rewritten
+                    cluster.sync();  // every warp of every CTA has read x_seg before it is rewritten
+                    if (tid == 0) mbar_arrive_expect(smem_u32(&sh.bar_seg), bytes_seg);
                     continue;
                 }
                 if (!empty) {
                     const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
                     const float t = uf * total;
-                    const float exc = inc - l4;
-                    // first segment whose inclusive prefix exceeds t, else the last non-empty one
-                    const unsigned hit = __ballot_sync(0xffffffffu, inc > t);
+                    // exclusive prefix of this lane; p1..p4 = inclusive prefixes of its four segments
+                    float exc = __shfl_up_sync(0xffffffffu, inc, 1);
+                    if (lane == 0) exc = 0.f;
+                    const float p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+                    // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
+                    const bool h1 = p1 > t && t4.x > 0.f, h2 = p2 > t && t4.y > 0.f;
+                    const bool h3 = p3 > t && t4.z > 0.f, h4 = p4 > t && t4.w > 0.f;
+                    const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
                     const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
                     int sel_seg = -1;
                     float sel_before = 0.f;
                     if (hit) {
                         const int src = __ffs(hit) - 1;
                         int e = 3; float bef = exc + l3;
-                        if (exc + l1 > t) { e = 0; bef = exc; }
-                        else if (exc + l2 > t) { e = 1; bef = exc + l1; }
-                        else if (exc + l3 > t) { e = 2; bef = exc + l2; }
+                        if (h1) { e = 0; bef = exc; }
+                        else if (h2) { e = 1; bef = p1; }
+                        else if (h3) { e = 2; bef = p2; }
                         sel_seg = __shfl_sync(0xffffffffu, 4 * lane + e, src);
                         sel_before = __shfl_sync(0xffffffffu, bef, src);
                     } else if (nz) {
                         const int src = 31 - __clz(nz);
                         int e = 0; float bef = exc;
-                        if (t4.w > 0.f) { e = 3; bef = exc + l3; }
-                        else if (t4.z > 0.f) { e = 2; bef = exc + l2; }
-                        else if (t4.y > 0.f) { e = 1; bef = exc + l1; }
+                        if (t4.w > 0.f) { e = 3; bef = p3; }
+                        else if (t4.z > 0.f) { e = 2; bef = p2; }
+                        else if (t4.y > 0.f) { e = 1; bef = p1; }
                         sel_seg = __shfl_sync(0xffffffffu, 4 * lane + e, src);
                         sel_before = __shfl_sync(0xffffffffu, bef, src);
                     }
                     if (sel_seg == myseg) {
-                        // rescan this warp's cached terms in index order
+                        // This warp holds u * S_r.  Its segment is ordered vector-major: step k covers
+                        // 32 consecutive vectors, one per lane.  Row totals of the NK steps first,
+                        // then a lane scan inside the one step that crosses the target.
                         const float tw = t - sel_before;
-                        float runw = 0.f;
-                        int found = -1, last_pos = -1;
+                        float rowtot[NK];
+#pragma unroll
+                        for (int k = 0; k < NK; ++k) rowtot[k] = warp_sum(vsum[k]);
+                        int ks = -1, klast = -1;
+                        float before = 0.f, ks_before = 0.f, klast_before = 0.f;
 #pragma unroll
                         for (int k = 0; k < NK; ++k) {
-                            if (found < 0) {
-                                float tt[EPV];
+                            if (rowtot[k] > 0.f) { klast = k; klast_before = before; }
+                            if (ks < 0 && rowtot[k] > 0.f && before + rowtot[k] > tw) { ks = k; ks_before = before; }
+                            before += rowtot[k];
+                        }
+                        if (ks < 0) { ks = klast; ks_before = klast_before; }
+                        int found = -1;
 #pragma unroll
-                                for (int hv = 0; hv < HV; ++hv) {
-                                    const float4 f = bcache[(k * HV + hv) * kRThreads];
-                                    tt[4 * hv] = f.x; tt[4 * hv + 1] = f.y; tt[4 * hv + 2] = f.z; tt[4 * hv + 3] = f.w;
-                                }
-                                const int i = v0 + 32 * k;
-                                float ls = 0.f;
-#pragma unroll
-                                for (int e = 0; e < EPV; ++e) {
-                                    tt[e] = fmaxf(fmaf(cp, a[k][e], -(cq * tt[e])), 0.f);
-                                    ls += tt[e];
-                                    if (tt[e] > 0.f) last_pos = i * EPV + e;
-                                }
+                        for (int k = 0; k < NK; ++k) {
+                            if (k == ks) {       // warp-uniform
+                                const float tk = tw - ks_before;
+                                const float ls = vsum[k];
                                 float incw = ls;
 #pragma unroll
                                 for (int off = 1; off < 32; off <<= 1) {
                                     const float o = __shfl_up_sync(0xffffffffu, incw, off);
                                     if (lane >= off) incw += o;
                                 }
-                                const unsigned bal = __ballot_sync(0xffffffffu, runw + incw > tw);
-                                if (bal) {
-                                    const int src = __ffs(bal) - 1;
-                                    int f = -1;
-                                    if (lane == src) {
-                                        float cum = runw + incw - ls;
-                                        int lp = -1;
+                                const unsigned bal = __ballot_sync(0xffffffffu, incw > tk && ls > 0.f);
+                                const unsigned nzl = __ballot_sync(0xffffffffu, ls > 0.f);
+                                const int src = bal ? __ffs(bal) - 1 : 31 - __clz(nzl);
+                                int f = -1;
+                                if (lane == src) {
+                                    float bq[EPV];
 #pragma unroll
-                                        for (int e = 0; e < EPV; ++e) {
-                                            cum += tt[e];
-                                            if (tt[e] > 0.f) lp = i * EPV + e;
-                                            if (f < 0 && cum > tw && tt[e] > 0.f) f = i * EPV + e;
-                                        }
-                                        if (f < 0) f = lp;
+                                    for (int hv = 0; hv < HV; ++hv) {
+                                        const float4 f4 = bcache[(k * HV + hv) * kRThreads];
+                                        bq[4 * hv] = f4.x; bq[4 * hv + 1] = f4.y; bq[4 * hv + 2] = f4.z; bq[4 * hv + 3] = f4.w;
                                     }
-                                    f = __shfl_sync(0xffffffffu, f, src);
-                                    if (f >= 0) found = f;
+                                    float cum = incw - ls;
+                                    int lp = -1;
+                                    const int i = v0 + 32 * k;
+#pragma unroll
+                                    for (int e = 0; e < EPV; ++e) {
+                                        const float te = fmaxf(fmaf(cp, a[k][e], -(cq * bq[e])), 0.f);
+                                        cum += te;
+                                        if (te > 0.f) lp = i * EPV + e;
+                                        if (f < 0 && cum > tk && te > 0.f) f = i * EPV + e;
+                                    }
+                                    if (f < 0) f = lp;
                                 }
-                                runw += __shfl_sync(0xffffffffu, incw, 31);
+                                found = __shfl_sync(0xffffffffu, f, src);
                             }
                         }
-                        if (found < 0) {
-#pragma unroll
-                            for (int off = 16; off > 0; off >>= 1)
-                                last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, off));
-                            found = last_pos;
-                        }
-                        if (lane == 0) *cluster.map_shared_rank(&sh.cand[r], 0) = found;
+                        if (lane == 0)
+                            send_b32(map_to_rank(smem_u32(&sh.cand[r]), 0), r_bar_cand, static_cast<uint32_t>(found));
                     }
+                } else if (myseg == 0 && lane == 0) {
+                    // no candidate at this position: rank 0 is still owed its 4 bytes
+                    send_b32(map_to_rank(smem_u32(&sh.cand[r]), 0), r_bar_cand, 0xffffffffu);
                 }
                 break;
             }
         }
 
         // ---------------- end of the block: h, tau, emit (rank 0) ----------------
-        cluster.sync();   // every candidate has landed in rank 0's shared memory
         if (rank == 0 && tid == 0) {
+            mbar_wait(smem_u32(&sh.bar_cand), ph_cand, status);   // all gamma+1 candidates have landed
             int32_t* ot = prm.out_tokens + static_cast<size_t>(b) * (g + 1);
             const int32_t* X = prm.tok + static_cast<size_t>(b) * g;
             const float* u = prm.uni + static_cast<size_t>(b) * (g + 2);
@@ -519,6 +583,7 @@ __global__ void __launch_bounds__(kRThreads, 1) verify_resident_kernel(const Par
                 if (i < g && prm.out_lse_d) prm.out_lse_d[o0] = static_cast<float>(sh.lse_d[i]);
             }
         }
+        ph_cand ^= 1u;
     }
     cp_async_wait<0>();
     cluster.sync();   // no CTA exits while a peer may still write into its shared memory
