@@ -23,6 +23,7 @@ struct DeviceState {
     unsigned long long calls = 0;
     int max_clusters[2][2][2][bv::kMaxCluster + 1] = {};  // [algo][dtype][vec][cluster], 0 = not asked yet
     int res_clusters[2][9][bv::kMaxCluster + 1] = {};     // resident kernel: [dtype][nk][cluster]
+    int clu_clusters[2][2][bv::kMaxCluster + 1] = {};     // cluster kernel: [algo][dtype][cluster]
     // staging for the host-buffer entry points
     void* stage = nullptr;
     size_t stage_bytes = 0;
@@ -124,7 +125,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
 
     // Block Verification on 16-byte rows: the kernel that keeps each row pair on chip,
     // when some cluster width lets a thread hold its share (at most 8 vectors per row).
-    if (algo == bv::kBlockVerify && vec && !std::getenv("BV_FORCE_STREAM")) {
+    if (algo == bv::kBlockVerify && vec && std::getenv("BV_RESIDENT")) {
         const long long units = static_cast<long long>(row_bytes / 16);
         int best_c = 0, best_nk = 0, best_n = 0;
         long long best_sms = -1;
@@ -156,6 +157,26 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     }
 
     int cluster = pick_cluster(*d, B, row_bytes);
+    if (vec && !std::getenv("BV_FORCE_STREAM")) {
+        int& cc = d->clu_clusters[algo][dtype][cluster];
+        if (cc == 0) {
+            cc = bv::cluster_max_clusters(algo, dtype, cluster);
+            if (cc <= 0) cc = -1;
+        }
+        if (cc > 0) {
+            int n = B < cc ? B : cc;
+            if (const char* env = std::getenv("BV_MAX_CLUSTERS")) {
+                const int cap = std::atoi(env);
+                if (cap > 0 && cap < n) n = cap;
+            }
+            prm.ticket = d->tickets + 2 * (d->calls++ % kTicketSlots);
+            prm.nclusters = n;
+            cudaError_t e = bv::launch_cluster(prm, algo, dtype, cluster, n, stream);
+            if (e != cudaSuccess) return cuda_fail(e);
+            t_last_launches = 1;
+            return BV_OK;
+        }
+    }
     int& cached = d->max_clusters[algo][dtype][vec ? 1 : 0][cluster];
     if (cached == 0) {
         cached = bv::stream_max_clusters(algo, dtype, vec, cluster);

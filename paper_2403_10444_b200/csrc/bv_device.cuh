@@ -149,4 +149,100 @@ __device__ __forceinline__ double shfl_d(double v, int src) {
     return __hiloint2double(hi, lo);
 }
 
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+// address of the same shared-memory location in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, int rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Wait for the phase with the given parity.  The wait is bounded: after about a second it
+// gives up, records the fact in *status and returns, so a protocol error cannot hang the GPU.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return;
+        // give up after about a second, or at once if another wait has already given up
+        if (clock64() - t0 > 2000000000LL || (status && *reinterpret_cast<volatile int*>(status))) {
+            if (status) atomicExch(status, 1);
+            return;
+        }
+    }
+}
+// 16 or 4 bytes into another CTA's shared memory; the bytes are counted by that CTA's barrier
+__device__ __forceinline__ void send_v4(uint32_t raddr, uint32_t rbar, float a, float b, float c, float d) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(raddr), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)),
+                   "r"(__float_as_uint(d)), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void send_b32(uint32_t raddr, uint32_t rbar, uint32_t v) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(raddr), "r"(v), "r"(rbar) : "memory");
+}
+
+template <int DT> struct Raw;
+template <> struct Raw<kBF16> {
+    static constexpr int EPV = 8;
+    static constexpr uint32_t kNegInf = 0xff80ff80u;
+    static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[8]) {
+        v[0] = __uint_as_float(r.x << 16); v[1] = __uint_as_float(r.x & 0xffff0000u);
+        v[2] = __uint_as_float(r.y << 16); v[3] = __uint_as_float(r.y & 0xffff0000u);
+        v[4] = __uint_as_float(r.z << 16); v[5] = __uint_as_float(r.z & 0xffff0000u);
+        v[6] = __uint_as_float(r.w << 16); v[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+};
+template <> struct Raw<kF32> {
+    static constexpr int EPV = 4;
+    static constexpr uint32_t kNegInf = 0xff800000u;
+    static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[4]) {
+        v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y);
+        v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+    }
+};
+
+template <int EPV> __device__ __forceinline__ float vec_max(const float (&v)[EPV]) {
+    float vm = v[0];
+#pragma unroll
+    for (int e = 1; e < EPV; ++e) vm = fmaxf(vm, v[e]);
+    return vm;
+}
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, off));
+    return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    return x;
+}
+
+
+// "No reference yet": finite, so that -inf logits still give 2^-inf = 0 and any finite
+// logit overflows to +inf, which exceeds the raise bound and installs a real reference.
+constexpr float kNoRef = -3.0e38f;
+// A vector of 8 terms all at the reference sums to at most 8 * 2^0.5 = 11.3; a sum above
+// this bound therefore means some term exceeds 2^0.5, i.e. its logit lies above the reference.
+// Without a raise every term is below 12, so its exponent is below 4 and is rounded to 1.2e-7.
+constexpr float kRaiseBound = 12.f;
+
+// 2^d for d = (own reference) - (row reference) <= 0, or 0 when there is no own reference
+__device__ __forceinline__ float ref_scale(float own, float row) {
+    return own > kNoRef ? pow2_nonpos(own - row) : 0.f;
+}
+
 }  // namespace bv

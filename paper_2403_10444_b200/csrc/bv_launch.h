@@ -15,6 +15,11 @@ int stream_max_clusters(int algo, int dtype, bool vec, int cluster);
 cudaError_t launch_stream(const Params& prm, int algo, int dtype, bool vec, int cluster,
                           int nclusters, cudaStream_t stream);
 
+// Cluster kernel for 16-byte aligned rows (both algorithms): several clusters per SM,
+// rows re-read from L2 for the residual sweep.
+int cluster_max_clusters(int algo, int dtype, int cluster);
+cudaError_t launch_cluster(const Params& prm, int algo, int dtype, int cluster, int nclusters, cudaStream_t stream);
+
 // Resident kernel (Block Verification only, 128-bit path): a thread holds up to `nk`
 // vectors per row, nk in {2, 4, 8}.
 int resident_vectors_per_cta(int nk);
