@@ -164,20 +164,22 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
 __device__ __forceinline__ void mbar_arrive_expect(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Wait for the phase with the given parity.  The wait is bounded: after about a second it
-// gives up, records the fact in *status and returns, so a protocol error cannot hang the GPU.
+// Wait for the phase with the given parity.  Each attempt lets the hardware suspend the
+// thread for up to about 2 us; the number of attempts is bounded (a few seconds in all),
+// after which the wait gives up, records the fact in *status and returns, so that a
+// protocol error cannot hang the GPU.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* status) {
-    const long long t0 = clock64();
-    for (;;) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return;
-        // give up after about a second, or at once if another wait has already given up
-        if (clock64() - t0 > 2000000000LL || (status && *reinterpret_cast<volatile int*>(status))) {
+    for (uint32_t spins = 0; !mbar_try_wait(bar, parity, 2000u); ++spins) {
+        if (spins > (1u << 20)) {
             if (status) atomicExch(status, 1);
             return;
         }
