@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstdlib>
+#include <cstring>
 #include <mutex>
 
 #include "../../include/bv.h"
@@ -24,6 +25,12 @@ struct DeviceState {
     int max_clusters[2][2][2][bv::kMaxCluster + 1] = {};  // [algo][dtype][vec][cluster], 0 = not asked yet
     int res_clusters[2][9][bv::kMaxCluster + 1] = {};     // resident kernel: [dtype][nk][cluster]
     int clu_clusters[2][2][bv::kMaxCluster + 1] = {};     // cluster kernel: [algo][dtype][cluster]
+    // scratch of the flow kernel: a small ring, so that calls in flight on different streams
+    // do not share counters (more than kFlowSlots overlapping calls on one device would)
+    void* flow_ws[4] = {};
+    size_t flow_bytes[4] = {};
+    unsigned long long flow_calls = 0;
+    int flow_ctas_per_sm[2] = {};
     // staging for the host-buffer entry points
     void* stage = nullptr;
     size_t stage_bytes = 0;
@@ -125,7 +132,57 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
 
     // Block Verification on 16-byte rows: the kernel that keeps each row pair on chip,
     // when some cluster width lets a thread hold its share (at most 8 vectors per row).
-    if (algo == bv::kBlockVerify && vec && std::getenv("BV_RESIDENT")) {
+    const char* force = std::getenv("BV_KERNEL");   // "flow", "cluster", "resident", "stream": experiments and tests
+    const bool want = force != nullptr;
+    auto forced = [&](const char* name) { return want && std::strcmp(force, name) == 0; };
+
+    // Block Verification on 16-byte rows: the flow of independent work items
+    if (algo == bv::kBlockVerify && vec && (!want || forced("flow"))) {
+        const long long units = static_cast<long long>(row_bytes / 16);
+        int nch = static_cast<int>(units / 1024);
+        nch = nch < 1 ? 1 : (nch > 8 ? 8 : nch);
+        if (const char* env = std::getenv("BV_FLOW_CHUNKS")) {
+            const int v = std::atoi(env);
+            if (v >= 1 && v <= 8) nch = v;
+        }
+        int& per_sm = d->flow_ctas_per_sm[dtype];
+        if (per_sm == 0) {
+            per_sm = bv::flow_max_ctas_per_sm(dtype);
+            if (per_sm <= 0) per_sm = -1;
+        }
+        if (per_sm > 0) {
+            size_t zero_bytes = 0;
+            const size_t need = bv::flow_scratch_bytes(B, gamma, nch, &zero_bytes);
+            const int slot = static_cast<int>(d->flow_calls++ % 4);
+            if (d->flow_bytes[slot] < need) {
+                if (d->flow_ws[slot]) cudaFree(d->flow_ws[slot]);
+                d->flow_ws[slot] = nullptr;
+                d->flow_bytes[slot] = 0;
+                cudaError_t e = cudaMalloc(&d->flow_ws[slot], need);
+                if (e != cudaSuccess) return cuda_fail(e);
+                d->flow_bytes[slot] = need;
+            }
+            bv::FlowScratch fl;
+            bv::flow_scratch_layout(d->flow_ws[slot], B, gamma, nch, &fl);
+            cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
+            if (e != cudaSuccess) return cuda_fail(e);
+            long long items = static_cast<long long>(B) * (gamma + 1) * nch;
+            long long nctas = static_cast<long long>(d->sm_count) * per_sm;
+            if (const char* env = std::getenv("BV_FLOW_CTAS")) {
+                const long long v = std::atoll(env);
+                if (v >= 1 && v < nctas) nctas = v;
+            }
+            if (nctas > items) nctas = items;
+            prm.ticket = nullptr;
+            prm.nclusters = 0;
+            e = bv::launch_flow(prm, fl, dtype, static_cast<int>(nctas), stream);
+            if (e != cudaSuccess) return cuda_fail(e);
+            t_last_launches = 1;
+            return BV_OK;
+        }
+    }
+
+    if (algo == bv::kBlockVerify && vec && forced("resident")) {
         const long long units = static_cast<long long>(row_bytes / 16);
         int best_c = 0, best_nk = 0, best_n = 0;
         long long best_sms = -1;
@@ -157,7 +214,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     }
 
     int cluster = pick_cluster(*d, B, row_bytes);
-    if (vec && !std::getenv("BV_FORCE_STREAM")) {
+    if (vec && !forced("stream")) {
         int& cc = d->clu_clusters[algo][dtype][cluster];
         if (cc == 0) {
             cc = bv::cluster_max_clusters(algo, dtype, cluster);
@@ -300,6 +357,7 @@ int bv_release(void) {
     if ((e = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(e);
     if (d.stage) cudaFree(d.stage);
     if (d.tickets) cudaFree(d.tickets);
+    for (void* w : d.flow_ws) if (w) cudaFree(w);
     if (d.stream) cudaStreamDestroy(d.stream);
     d = DeviceState{};
     return BV_OK;

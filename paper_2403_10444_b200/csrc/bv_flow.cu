@@ -1,0 +1,578 @@
+// Block Verification (Algorithm 2) as a dependency-driven flow of independent work items.
+//
+// A row pair (P_r, Q_r) of one drafted block is cut into NCH chunks.  Persistent CTAs
+// pull items from two sources:
+//
+//   sweep-1 item (b, r, chunk)  streams the chunk of both rows from HBM and leaves the
+//       chunk's {reference, sum 2^{z k - M}} pair for each row in scratch.  The CTA that
+//       completes a row combines the chunks into the row normalisers and, holding the
+//       block's lock, advances the prefix recursion p_{r+1} = min(p_r P_r(X)/Q_r(X), 1)
+//       (Eq. "def_as") over every row that is complete, releasing their sweep-2 items.
+//   sweep-2 item (b, r, chunk)  re-reads the chunk (an L2 hit: it was streamed moments
+//       ago, and released items are taken before new sweep-1 items) and leaves
+//       sum max(p_r P_r(x) - Q_r(x), 0) per warp segment (Eq. "pacc_block").  The CTA
+//       that completes a position adds the segments to S_r, locates u * S_r, rescans that
+//       one segment in index order for the candidate Y_r (Eq. "pres-block"), and the CTA
+//       that completes the block forms h_i, selects tau and emits X^tau, Y_tau.
+//
+// No CTA ever waits for another one while it holds work that others need: sweep-1 items
+// have no prerequisites, the lock is only held over a few scalar operations, and a CTA
+// polls (bounded) only when nothing is left to start.  So CTAs need not be co-resident.
+#include "bv_device.cuh"
+#include "bv_launch.h"
+
+namespace bv {
+
+constexpr int kFThreads = 512;
+constexpr int kFWarps = kFThreads / 32;
+
+struct FlowShared {
+    float red_M[2][kFWarps];
+    float red_s[2][kFWarps];
+    int kind, item, last;       // what this CTA does next; whether it completed a row / position
+    float c, MP, MQ;            // sweep 2: p_r Z_Q / Z_P and the row references
+};
+
+enum : int { kExit = 0, kSweep1 = 1, kSweep2 = 2 };
+// counters, one per 128-byte line: next sweep-1 item; released-but-untaken sweep-2 items
+// (a semaphore); slots taken from / reserved in the ready list
+enum : int { kNext = 0, kAvail = 32, kHead = 64, kTail = 96, kCounterWords = 128 };
+
+__device__ __forceinline__ unsigned ld_volatile(const unsigned* p) {
+    return *reinterpret_cast<const volatile unsigned*>(p);
+}
+
+// ---- per-vector arithmetic (same formulation as the cluster kernel) ----
+template <int EPV> __device__ __forceinline__ float f_exp_sum(const float (&v)[EPV], float kf, float nM) {
+    float a[EPV];
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) a[e] = ex2(fmaf(v[e], kf, nM));
+    float s0 = a[0] + a[1], s1 = a[2] + a[3];
+    if (EPV == 8) { s0 += a[4] + a[5]; s1 += a[6] + a[7]; }
+    return s0 + s1;
+}
+template <int EPV> __device__ __forceinline__ void f_accumulate(const float (&v)[EPV], float kf, float& M, float& s) {
+    float vs = f_exp_sum<EPV>(v, kf, -M);
+    if (__any_sync(0xffffffffu, vs > kRaiseBound)) {      // some logit lies above the reference
+        const float y = rintf(warp_max(vec_max<EPV>(v)) * kf);
+        if (y > M) { s *= ref_scale(M, y); M = y; }
+        vs = f_exp_sum<EPV>(v, kf, -M);
+    }
+    s += vs;
+}
+template <int EPV>
+__device__ __forceinline__ float f_pair_sum(const float (&vp)[EPV], const float (&vq)[EPV], float kf, float cp,
+                                            float cq, float nMP, float nMQ, float (&t)[EPV]) {
+#pragma unroll
+    for (int e = 0; e < EPV; ++e) {
+        const float a = ex2(fmaf(vp[e], kf, nMP));
+        const float q = ex2(fmaf(vq[e], kf, nMQ));
+        t[e] = fmaxf(fmaf(cp, a, -(cq * q)), 0.f);
+    }
+    float s0 = t[0] + t[1], s1 = t[2] + t[3];
+    if (EPV == 8) { s0 += t[4] + t[5]; s1 += t[6] + t[7]; }
+    return s0 + s1;
+}
+template <int DT> __device__ __forceinline__ void f_load(const char* row, int i, float (&v)[Raw<DT>::EPV]) {
+    Raw<DT>::unpack(ld_stream_v4(row + static_cast<size_t>(i) * 16), v);
+}
+template <int DT>
+__device__ __forceinline__ void f_load_tail(const char* row, int i, int end, float (&v)[Raw<DT>::EPV]) {
+    if (row != nullptr && i < end) {
+        f_load<DT>(row, i, v);
+    } else {
+#pragma unroll
+        for (int e = 0; e < Raw<DT>::EPV; ++e) v[e] = -INFINITY;
+    }
+}
+
+// scratch written by other CTAs is always read through L2
+__device__ __forceinline__ RowZ load_rowz(const RowZ* p) {
+    RowZ z;
+    z.MP = __ldcg(&p->MP); z.ZP = __ldcg(&p->ZP); z.MQ = __ldcg(&p->MQ); z.ZQ = __ldcg(&p->ZQ);
+    return z;
+}
+
+struct FlowCtx {
+    int g, V, B, nch, units;
+    size_t row_bytes;
+    float kf;
+    double kd;
+};
+
+__device__ __forceinline__ void chunk_range(const FlowCtx& cx, int ch, int warp, int& w0, int& w1) {
+    const int u0 = static_cast<int>(static_cast<long long>(cx.units) * ch / cx.nch);
+    const int u1 = static_cast<int>(static_cast<long long>(cx.units) * (ch + 1) / cx.nch);
+    w0 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * warp / kFWarps);
+    w1 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * (warp + 1) / kFWarps);
+}
+
+// One warp walks segment [w0, w1) of a row pair in index order and returns the first element
+// whose running residual mass exceeds tw (else the last element with positive mass, else -1).
+template <int DT>
+__device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int lane, float kf, float cp, float cq,
+                        float nMP, float nMQ, float tw) {
+    constexpr int EPV = Raw<DT>::EPV;
+    float run = 0.f;
+    int found = -1, last_pos = -1;
+    for (int base = w0; base < w1 && found < 0; base += 32) {
+        const int i = base + lane;
+        float vp[EPV], vq[EPV], tt[EPV];
+        f_load_tail<DT>(rowP, i, w1, vp);
+        f_load_tail<DT>(rowQ, i, w1, vq);
+        const float ls = f_pair_sum<EPV>(vp, vq, kf, cp, cq, nMP, nMQ, tt);
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) if (tt[e] > 0.f) last_pos = i * EPV + e;
+        float incw = ls;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float o = __shfl_up_sync(0xffffffffu, incw, off);
+            if (lane >= off) incw += o;
+        }
+        const unsigned bal = __ballot_sync(0xffffffffu, run + incw > tw && ls > 0.f);
+        if (bal) {
+            const int src = __ffs(bal) - 1;
+            int f = -1;
+            if (lane == src) {
+                float cum = run + incw - ls;
+                int lp = -1;
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) {
+                    cum += tt[e];
+                    if (tt[e] > 0.f) lp = i * EPV + e;
+                    if (f < 0 && cum > tw && tt[e] > 0.f) f = i * EPV + e;
+                }
+                if (f < 0) f = lp;
+            }
+            found = __shfl_sync(0xffffffffu, f, src);
+        }
+        run += __shfl_sync(0xffffffffu, incw, 31);
+    }
+    if (found < 0) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, off));
+        found = last_pos;
+    }
+    return found;
+}
+
+// ---- the end of a block (one thread): Eq. "pacc_block", selection of tau, output ----
+__device__ void f_finalize_block(const Params& prm, const FlowScratch& fl, int b) {
+    const int g = prm.gamma;
+    int32_t* ot = prm.out_tokens + static_cast<size_t>(b) * (g + 1);
+    const int32_t* X = prm.tok + static_cast<size_t>(b) * g;
+    const float* u = prm.uni + static_cast<size_t>(b) * (g + 2);
+    const double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
+    const double* S = fl.S + static_cast<size_t>(b) * (g + 1);
+    const int* cand = fl.cand + static_cast<size_t>(b) * (g + 1);
+    const bool bad = ld_volatile(&fl.bad[b]) != 0;
+    int tau = -1;
+    if (!bad) {
+        tau = 0;
+        // h_gamma = p_gamma; h_i = S_i / (S_i + 1 - p_i); tau = max{i : eta_i <= h_i}
+        for (int i = g; i >= 1; --i) {
+            const double pi = __ldcg(&p[i]);
+            double h = pi;
+            if (i < g) { const double Si = __ldcg(&S[i]); h = Si > 0.0 ? Si / (Si + 1.0 - pi) : 0.0; }
+            if (h > 0.0 && static_cast<double>(u[i - 1]) <= h) { tau = i; break; }
+        }
+    }
+    for (int i = 0; i <= g; ++i) ot[i] = -1;
+    if (tau >= 0) {
+        for (int i = 0; i < tau; ++i) ot[i] = X[i];
+        ot[tau] = __ldcg(&cand[tau]);
+        prm.out_len[b] = tau + 1;
+    } else {
+        prm.out_len[b] = -1;
+    }
+    if (prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d) {
+        const double ln2 = 0.693147180559945309417232;
+        for (int i = 0; i <= g; ++i) {
+            const size_t o1 = static_cast<size_t>(b) * (g + 1) + i, o0 = static_cast<size_t>(b) * g + i;
+            const double pi = __ldcg(&p[i]);
+            const double Si = i < g ? __ldcg(&S[i]) : 0.0;
+            double h = (i == 0) ? 1.0 : (i == g ? pi : (Si > 0.0 ? Si / (Si + 1.0 - pi) : 0.0));
+            const RowZ z = load_rowz(&fl.rowZ[static_cast<size_t>(b) * (g + 1) + i]);
+            if (prm.out_p) prm.out_p[o1] = static_cast<float>(pi);
+            if (prm.out_h) prm.out_h[o1] = static_cast<float>(h);
+            if (prm.out_lse_t) prm.out_lse_t[o1] = static_cast<float>((static_cast<double>(z.MP) + log2(z.ZP)) * ln2);
+            if (i < g && prm.out_S) prm.out_S[o0] = static_cast<float>(Si);
+            if (i < g && prm.out_lse_d) prm.out_lse_d[o0] = static_cast<float>((static_cast<double>(z.MQ) + log2(z.ZQ)) * ln2);
+        }
+    }
+}
+
+// ---- a row is complete: normalisers, then the recursion over every complete row ----
+template <int DT>
+__device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int r) {
+    const int g = cx.g;
+    const size_t rowi = static_cast<size_t>(b) * (g + 1) + r;
+    // combine the chunks (fp64): row reference = max of the chunk references
+    double MP = kNoRef, MQ = kNoRef;
+    for (int ch = 0; ch < cx.nch; ++ch) {
+        const RowZ z = load_rowz(&fl.part[rowi * cx.nch + ch]);
+        MP = fmax(MP, z.MP); MQ = fmax(MQ, z.MQ);
+    }
+    double ZP = 0.0, ZQ = 0.0;
+    for (int ch = 0; ch < cx.nch; ++ch) {
+        const RowZ z = load_rowz(&fl.part[rowi * cx.nch + ch]);
+        ZP += z.ZP * static_cast<double>(ref_scale(static_cast<float>(z.MP), static_cast<float>(MP)));
+        ZQ += z.ZQ * static_cast<double>(ref_scale(static_cast<float>(z.MQ), static_cast<float>(MQ)));
+    }
+    RowZ out; out.MP = MP; out.ZP = ZP; out.MQ = MQ; out.ZQ = ZQ;
+    fl.rowZ[rowi] = out;
+    const bool have_q = r < g;
+    // the row's maximum is finite iff its reference is; Z is NaN / inf iff the row holds a NaN / overflowed
+    if (!(MP > kNoRef && MP < INFINITY) || !(ZP < INFINITY)) atomicOr(&fl.bad[b], 1u);
+    if (have_q && (!(MQ > kNoRef && MQ < INFINITY) || !(ZQ < INFINITY))) atomicOr(&fl.bad[b], 1u);
+    __threadfence();
+    atomicExch(&fl.row_done[rowi], 1u);
+
+    // advance the block's recursion while the next row is complete (short critical section)
+    unsigned spins = 0;
+    while (atomicCAS(&fl.lock[b], 0u, 1u) != 0u) {
+        __nanosleep(100);
+        if (++spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return; }
+    }
+    __threadfence();
+    unsigned c = ld_volatile(&fl.chain[b]);
+    double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
+    while (c <= static_cast<unsigned>(g) && ld_volatile(&fl.row_done[static_cast<size_t>(b) * (g + 1) + c]) != 0u) {
+        __threadfence();
+        const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
+        const RowZ z = load_rowz(&fl.rowZ[ci]);
+        const double p_c = (c == 0) ? 1.0 : __ldcg(&p[c]);
+        if (c == 0) p[0] = 1.0;
+        float cs = 1.f;
+        if (c < static_cast<unsigned>(g)) {
+            // ratio = P_c(X_{c+1}) / Q_c(X_{c+1}) from the two logits of the drafted token
+            double ratio = 0.0;
+            const int x = prm.tok[static_cast<size_t>(b) * g + c];
+            if (x < 0 || x >= cx.V) {
+                atomicOr(&fl.bad[b], 1u);
+            } else {
+                const char* rowP = static_cast<const char*>(prm.tgt) + ci * cx.row_bytes;
+                const char* rowQ = static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + c) * cx.row_bytes;
+                const double zq = load_logit<DT>(rowQ, x), zp = load_logit<DT>(rowP, x);
+                if (zq == -INFINITY) atomicOr(&fl.bad[b], 1u);
+                else ratio = exp2((zp - zq) * cx.kd - (z.MP - z.MQ)) * (z.ZQ / z.ZP);
+            }
+            p[c + 1] = fmin(p_c * ratio, 1.0);
+            cs = static_cast<float>(p_c * z.ZQ / z.ZP);
+        }
+        fl.cscale[ci] = cs;
+        __threadfence();
+        // release the row's sweep-2 items
+        const unsigned t = atomicAdd(&fl.counters[kTail], static_cast<unsigned>(cx.nch));
+        for (int ch = 0; ch < cx.nch; ++ch)
+            atomicExch(&fl.ready[t + ch], static_cast<unsigned>(ci * cx.nch + ch) + 1u);
+        __threadfence();
+        atomicAdd(&fl.counters[kAvail], static_cast<unsigned>(cx.nch));
+        ++c;
+        *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
+    }
+    __threadfence();
+    atomicExch(&fl.lock[b], 0u);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params prm, const FlowScratch fl) {
+    using R = Raw<DT>;
+    constexpr int EPV = R::EPV;
+    constexpr size_t ESZ = (DT == kF32) ? 4 : 2;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ FlowShared sh;
+
+    FlowCtx cx;
+    cx.g = prm.gamma; cx.V = prm.V; cx.B = prm.B; cx.nch = fl.nch; cx.units = prm.V / EPV;
+    cx.row_bytes = static_cast<size_t>(prm.V) * ESZ; cx.kf = prm.kf; cx.kd = prm.kd;
+    const int g = cx.g;
+    const float kf = cx.kf;
+    const unsigned total_items = static_cast<unsigned>(cx.B) * (g + 1) * cx.nch;   // of either kind
+    bool s1_left = true;
+
+    for (;;) {
+        // ---------------- pick the next item (thread 0) ----------------
+        if (tid == 0) {
+            int kind = kExit, item = 0;
+            unsigned idle = 0;
+            for (;;) {
+                // a released sweep-2 item first: take one unit of the semaphore, then a slot
+                bool got = false;
+                if (static_cast<int>(ld_volatile(&fl.counters[kAvail])) > 0) {
+                    if (static_cast<int>(atomicSub(&fl.counters[kAvail], 1u)) > 0) got = true;
+                    else atomicAdd(&fl.counters[kAvail], 1u);       // lost the race: give it back
+                }
+                if (got) {
+                    const unsigned h = atomicAdd(&fl.counters[kHead], 1u);
+                    unsigned v, spins = 0;
+                    while ((v = ld_volatile(&fl.ready[h])) == 0u) {   // its writer is a few stores away
+                        if (++spins > (1u << 24)) { if (prm.status) atomicExch(prm.status, 1); break; }
+                    }
+                    if (v != 0u) { kind = kSweep2; item = static_cast<int>(v - 1u); }
+                    break;
+                }
+                if (s1_left) {
+                    const unsigned idx = atomicAdd(&fl.counters[kNext], 1u);
+                    if (idx < total_items) { kind = kSweep1; item = static_cast<int>(idx); break; }
+                    s1_left = false;
+                }
+                if (ld_volatile(&fl.counters[kHead]) >= total_items) break;   // every sweep-2 item is taken: done
+                __nanosleep(256);
+                if (++idle > (1u << 23)) { if (prm.status) atomicExch(prm.status, 1); break; }
+            }
+            sh.kind = kind; sh.item = item; sh.last = 0;
+            if (kind == kSweep2) {
+                __threadfence();
+                const int ri = item / cx.nch;
+                const RowZ z = load_rowz(&fl.rowZ[ri]);
+                sh.c = __ldcg(&fl.cscale[ri]);
+                sh.MP = static_cast<float>(z.MP);
+                sh.MQ = static_cast<float>(z.MQ);
+            }
+        }
+        __syncthreads();
+        const int kind = sh.kind, item = sh.item;
+        if (kind == kExit) break;
+        const int ch = item % cx.nch, ri = item / cx.nch, r = ri % (g + 1), b = ri / (g + 1);
+        const bool have_q = r < g;
+        const char* rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
+        const char* rowQ = have_q ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
+                                  : nullptr;
+        int w0, w1;
+        chunk_range(cx, ch, warp, w0, w1);
+        const int wfull = w0 + ((w1 - w0) & ~31);
+
+        if (kind == kSweep1) {
+            // ---------------- sweep 1 over this chunk ----------------
+            float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
+            int base = w0;
+            if (w0 < w1) {   // references from the first vector of every lane
+                float vp[EPV], vq[EPV];
+                f_load_tail<DT>(rowP, base + lane, w1, vp);
+                f_load_tail<DT>(rowQ, base + lane, w1, vq);
+                MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
+                f_accumulate<EPV>(vp, kf, MPw, sP);
+                if (have_q) {
+                    MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vq)) * kf), kNoRef);
+                    f_accumulate<EPV>(vq, kf, MQw, sQ);
+                }
+                base += 32;
+            }
+            if (have_q) {
+                for (; base + 64 <= wfull; base += 64) {      // two steps in which every lane has a vector
+                    float vp0[EPV], vq0[EPV], vp1[EPV], vq1[EPV];
+                    f_load<DT>(rowP, base + lane, vp0); f_load<DT>(rowQ, base + lane, vq0);
+                    f_load<DT>(rowP, base + 32 + lane, vp1); f_load<DT>(rowQ, base + 32 + lane, vq1);
+                    f_accumulate<EPV>(vp0, kf, MPw, sP); f_accumulate<EPV>(vq0, kf, MQw, sQ);
+                    f_accumulate<EPV>(vp1, kf, MPw, sP); f_accumulate<EPV>(vq1, kf, MQw, sQ);
+                }
+                for (; base < w1; base += 32) {
+                    float vp[EPV], vq[EPV];
+                    f_load_tail<DT>(rowP, base + lane, w1, vp); f_load_tail<DT>(rowQ, base + lane, w1, vq);
+                    f_accumulate<EPV>(vp, kf, MPw, sP); f_accumulate<EPV>(vq, kf, MQw, sQ);
+                }
+            } else {
+                for (; base < w1; base += 32) {
+                    float vp[EPV];
+                    f_load_tail<DT>(rowP, base + lane, w1, vp);
+                    f_accumulate<EPV>(vp, kf, MPw, sP);
+                }
+            }
+            sP = warp_sum(sP);
+            sQ = warp_sum(sQ);
+            if (lane == 0) {
+                sh.red_M[0][warp] = MPw; sh.red_s[0][warp] = sP;
+                sh.red_M[1][warp] = MQw; sh.red_s[1][warp] = sQ;
+            }
+            __syncthreads();
+            if (warp == 0) {
+                // combine the 16 warps of this chunk in fp64
+                const float mP = lane < kFWarps ? sh.red_M[0][lane] : kNoRef;
+                const float mQ = lane < kFWarps ? sh.red_M[1][lane] : kNoRef;
+                const float MPc = warp_max(mP), MQc = warp_max(mQ);
+                double zP = lane < kFWarps ? static_cast<double>(sh.red_s[0][lane]) * ref_scale(mP, MPc) : 0.0;
+                double zQ = lane < kFWarps ? static_cast<double>(sh.red_s[1][lane]) * ref_scale(mQ, MQc) : 0.0;
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) { zP += shfl_xor_d(zP, off); zQ += shfl_xor_d(zQ, off); }
+                if (lane == 0) {
+                    RowZ z; z.MP = MPc; z.ZP = zP; z.MQ = MQc; z.ZQ = zQ;
+                    fl.part[item] = z;
+                    __threadfence();
+                    if (atomicAdd(&fl.row_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u) {
+                        __threadfence();
+                        f_row_complete<DT>(prm, fl, cx, b, r);
+                    }
+                }
+            }
+        } else {
+            // ---------------- sweep 2 over this chunk ----------------
+            const float cp = have_q ? sh.c : 1.f, cq = have_q ? 1.f : 0.f;
+            const float nMP = -sh.MP, nMQ = -sh.MQ;
+            float acc = 0.f;
+            int base = w0;
+            for (; base + 64 <= wfull; base += 64) {
+                float vp0[EPV], vq0[EPV], vp1[EPV], vq1[EPV], t0[EPV], t1[EPV];
+                f_load<DT>(rowP, base + lane, vp0); f_load<DT>(rowP, base + 32 + lane, vp1);
+                f_load_tail<DT>(rowQ, base + lane, w1, vq0); f_load_tail<DT>(rowQ, base + 32 + lane, w1, vq1);
+                acc += f_pair_sum<EPV>(vp0, vq0, kf, cp, cq, nMP, nMQ, t0);
+                acc += f_pair_sum<EPV>(vp1, vq1, kf, cp, cq, nMP, nMQ, t1);
+            }
+            for (; base < w1; base += 32) {
+                float vp[EPV], vq[EPV], t[EPV];
+                f_load_tail<DT>(rowP, base + lane, w1, vp);
+                f_load_tail<DT>(rowQ, base + lane, w1, vq);
+                acc += f_pair_sum<EPV>(vp, vq, kf, cp, cq, nMP, nMQ, t);
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) fl.seg_tot[static_cast<size_t>(ri) * (cx.nch * kFWarps) + ch * kFWarps + warp] = acc;
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) {
+                __threadfence();
+                sh.last = atomicAdd(&fl.s2_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u;
+            }
+            __syncthreads();
+            if (sh.last && warp == 0) {
+                // ---------------- the position is complete: S_r and the candidate Y_r ----------------
+                __threadfence();
+                const int nseg = cx.nch * kFWarps;
+                const float* segs = fl.seg_tot + static_cast<size_t>(ri) * nseg;
+                float w[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) w[j] = (4 * lane + j < nseg) ? __ldcg(&segs[4 * lane + j]) : 0.f;
+                double sd = (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
+                            (static_cast<double>(w[2]) + static_cast<double>(w[3]));
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
+                const RowZ z = load_rowz(&fl.rowZ[ri]);
+                if (lane == 0 && have_q) fl.S[ri] = sd / z.ZQ;
+                const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
+                float inc = l4;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const float o = __shfl_up_sync(0xffffffffu, inc, off);
+                    if (lane >= off) inc += o;
+                }
+                const float total = __shfl_sync(0xffffffffu, inc, 31);
+                const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
+                int found = -1;
+                if (total > 0.f) {
+                    const float t = uf * total;
+                    float exc = __shfl_up_sync(0xffffffffu, inc, 1);
+                    if (lane == 0) exc = 0.f;
+                    const float p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+                    // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
+                    const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
+                    const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
+                    const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
+                    const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
+                    int e = 3; float bef = p3; int src;
+                    if (hit) {
+                        src = __ffs(hit) - 1;
+                        if (h1) { e = 0; bef = exc; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
+                    } else {
+                        src = 31 - __clz(nz);
+                        e = 0; bef = exc;
+                        if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
+                        else if (w[1] > 0.f) { e = 1; bef = p1; }
+                    }
+                    const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
+                    const float before = __shfl_sync(0xffffffffu, bef, src);
+                    int s0, s1;
+                    chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1);
+                    found = f_rescan<DT>(rowP, rowQ, s0, s1, lane, kf, cp, cq, nMP, nMQ, t - before);
+                } else if (have_q && r == 0 && total == 0.f) {
+                    // empty residual at position 0 (P_0 and Q_0 coincide): sample P_0 with the same uniform.
+                    // Two plain passes over the whole row by this warp: rare, so speed does not matter.
+                    float tot = 0.f;
+                    for (int base2 = 0; base2 < cx.units; base2 += 32) {
+                        float vp[EPV], vq[EPV], t2[EPV];
+                        f_load_tail<DT>(rowP, base2 + lane, cx.units, vp);
+                        f_load_tail<DT>(nullptr, 0, 0, vq);
+                        tot += f_pair_sum<EPV>(vp, vq, kf, 1.f, 0.f, nMP, nMQ, t2);
+                    }
+                    tot = warp_sum(tot);
+                    found = f_rescan<DT>(rowP, nullptr, 0, cx.units, lane, kf, 1.f, 0.f, nMP, nMQ, uf * tot);
+                }
+                if (lane == 0) {
+                    fl.cand[ri] = found;
+                    __threadfence();
+                    if (atomicAdd(&fl.cand_cnt[b], 1u) == static_cast<unsigned>(g)) {
+                        __threadfence();
+                        f_finalize_block(prm, fl, b);
+                    }
+                }
+            }
+        }
+        __syncthreads();   // shared scratch is reused by the next item
+    }
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+
+size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes) {
+    const size_t rows = static_cast<size_t>(B) * (gamma + 1);
+    size_t z = 0;
+    z += up256(kCounterWords * sizeof(unsigned));   // counters
+    z += 3 * up256(rows * sizeof(unsigned));        // row_cnt, row_done, s2_cnt
+    z += 4 * up256(static_cast<size_t>(B) * sizeof(unsigned));   // cand_cnt, chain, lock, bad
+    z += up256(rows * nch * sizeof(unsigned));      // ready
+    if (zero_bytes) *zero_bytes = z;
+    size_t n = z;
+    n += up256(rows * nch * sizeof(RowZ));          // part
+    n += up256(rows * sizeof(RowZ));                // rowZ
+    n += up256(static_cast<size_t>(B) * (gamma + 2) * sizeof(double));   // pchain
+    n += up256(rows * sizeof(float));               // cscale
+    n += up256(rows * nch * kFWarps * sizeof(float));   // seg_tot
+    n += up256(rows * sizeof(double));              // S
+    n += up256(rows * sizeof(int));                 // cand
+    return n;
+}
+
+void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl) {
+    const size_t rows = static_cast<size_t>(B) * (gamma + 1);
+    char* p = static_cast<char*>(base);
+    auto take = [&](size_t bytes) { char* q = p; p += up256(bytes); return q; };
+    fl->counters = reinterpret_cast<unsigned*>(take(kCounterWords * sizeof(unsigned)));
+    fl->row_cnt = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
+    fl->row_done = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
+    fl->s2_cnt = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
+    fl->cand_cnt = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
+    fl->chain = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
+    fl->lock = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
+    fl->bad = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
+    fl->ready = reinterpret_cast<unsigned*>(take(rows * nch * sizeof(unsigned)));
+    fl->part = reinterpret_cast<RowZ*>(take(rows * nch * sizeof(RowZ)));
+    fl->rowZ = reinterpret_cast<RowZ*>(take(rows * sizeof(RowZ)));
+    fl->pchain = reinterpret_cast<double*>(take(static_cast<size_t>(B) * (gamma + 2) * sizeof(double)));
+    fl->cscale = reinterpret_cast<float*>(take(rows * sizeof(float)));
+    fl->seg_tot = reinterpret_cast<float*>(take(rows * nch * kFWarps * sizeof(float)));
+    fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
+    fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
+    fl->nch = nch;
+}
+
+using FKernelFn = void (*)(const Params, const FlowScratch);
+static FKernelFn pick_flow(int dtype) {
+    return dtype == kF32 ? verify_flow_kernel<kF32> : verify_flow_kernel<kBF16>;
+}
+
+int flow_max_ctas_per_sm(int dtype) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_flow(dtype), kFThreads, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
+cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream) {
+    pick_flow(dtype)<<<nctas, kFThreads, 0, stream>>>(prm, fl);
+    return cudaGetLastError();
+}
+
+}  // namespace bv

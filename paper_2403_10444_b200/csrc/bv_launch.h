@@ -20,6 +20,34 @@ cudaError_t launch_stream(const Params& prm, int algo, int dtype, bool vec, int 
 int cluster_max_clusters(int algo, int dtype, int cluster);
 cudaError_t launch_cluster(const Params& prm, int algo, int dtype, int cluster, int nclusters, cudaStream_t stream);
 
+// Flow kernel (Block Verification, 128-bit path): independent work items with dependency
+// counters in a scratch area of flow_scratch_bytes(); its first *zero_bytes must be zero
+// when the kernel starts.
+struct RowZ { double MP, ZP, MQ, ZQ; };   // row (or chunk) references and sums of 2^{z k - M}
+struct FlowScratch {
+    unsigned* counters;   // next sweep-1 item, semaphore of released items, ready head, ready tail
+    unsigned* row_cnt;    // [B (gamma+1)] sweep-1 chunks finished per row
+    unsigned* row_done;   // [B (gamma+1)] row normalisers published
+    unsigned* s2_cnt;     // [B (gamma+1)] sweep-2 chunks finished per position
+    unsigned* cand_cnt;   // [B] positions with a candidate
+    unsigned* chain;      // [B] rows folded into the recursion
+    unsigned* lock;       // [B]
+    unsigned* bad;        // [B] data fault seen
+    unsigned* ready;      // [B (gamma+1) nch] released sweep-2 items (+1; 0 = not written yet)
+    RowZ* part;           // [B (gamma+1) nch]
+    RowZ* rowZ;           // [B (gamma+1)]
+    double* pchain;       // [B (gamma+2)]
+    float* cscale;        // [B (gamma+1)] p_r Z_Q / Z_P
+    float* seg_tot;       // [B (gamma+1) nch 16]
+    double* S;            // [B (gamma+1)]
+    int* cand;            // [B (gamma+1)]
+    int nch;
+};
+size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes);
+void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl);
+int flow_max_ctas_per_sm(int dtype);
+cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream);
+
 // Resident kernel (Block Verification only, 128-bit path): a thread holds up to `nk`
 // vectors per row, nk in {2, 4, 8}.
 int resident_vectors_per_cta(int nk);
