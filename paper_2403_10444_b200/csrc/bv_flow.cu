@@ -275,6 +275,9 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
     atomicExch(&fl.lock[b], 0u);
 }
 
+constexpr int kFDepth = 8;     // ring slots per thread: four (P, Q) steps of lookahead
+constexpr int kFAhead = kFDepth / 2;
+
 template <int DT>
 __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params prm, const FlowScratch fl) {
     using R = Raw<DT>;
@@ -282,6 +285,10 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
     constexpr size_t ESZ = (DT == kF32) ? 4 : 2;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ FlowShared sh;
+    // Each thread streams its own vectors through a private ring of 16-byte slots filled by
+    // cp.async, so loads run kFAhead steps ahead of the arithmetic without costing registers.
+    extern __shared__ __align__(16) unsigned char dyn[];
+    uint4* ring = reinterpret_cast<uint4*>(dyn) + tid;      // slot s of this thread: ring[s * kFThreads]
 
     FlowCtx cx;
     cx.g = prm.gamma; cx.V = prm.V; cx.B = prm.B; cx.nch = fl.nch; cx.units = prm.V / EPV;
@@ -341,43 +348,35 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
                                   : nullptr;
         int w0, w1;
         chunk_range(cx, ch, warp, w0, w1);
-        const int wfull = w0 + ((w1 - w0) & ~31);
+
+        const int nsteps = (w1 - w0 + 31) >> 5;             // warp-uniform; lanes past w1 see -inf logits
+        const char* srcP = rowP + static_cast<size_t>(w0 + lane) * 16;
+        const char* srcQ = have_q ? rowQ + static_cast<size_t>(w0 + lane) * 16 : nullptr;
+        auto fetch_step = [&](int k, int slot) {
+            const bool ok = k < nsteps && (w0 + lane + 32 * k) < w1;
+            ring_fetch(ring + slot * kFThreads, srcP + static_cast<size_t>(k) * 512, ok, R::kNegInf);
+            ring_fetch(ring + (slot + 1) * kFThreads, srcQ + static_cast<size_t>(k) * 512, ok && have_q, R::kNegInf);
+        };
+#pragma unroll
+        for (int k = 0; k < kFAhead; ++k) fetch_step(k, 2 * k);
 
         if (kind == kSweep1) {
             // ---------------- sweep 1 over this chunk ----------------
             float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
-            int base = w0;
-            if (w0 < w1) {   // references from the first vector of every lane
+            int slot = 0;
+            for (int k = 0; k < nsteps; ++k) {
+                cp_async_wait<kFDepth - 2>();            // step k of both rows has landed
                 float vp[EPV], vq[EPV];
-                f_load_tail<DT>(rowP, base + lane, w1, vp);
-                f_load_tail<DT>(rowQ, base + lane, w1, vq);
-                MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
-                f_accumulate<EPV>(vp, kf, MPw, sP);
-                if (have_q) {
+                R::unpack(ring[slot * kFThreads], vp);
+                R::unpack(ring[(slot + 1) * kFThreads], vq);
+                if (k == 0) {                            // references from the first vector of every lane
+                    MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
                     MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vq)) * kf), kNoRef);
-                    f_accumulate<EPV>(vq, kf, MQw, sQ);
                 }
-                base += 32;
-            }
-            if (have_q) {
-                for (; base + 64 <= wfull; base += 64) {      // two steps in which every lane has a vector
-                    float vp0[EPV], vq0[EPV], vp1[EPV], vq1[EPV];
-                    f_load<DT>(rowP, base + lane, vp0); f_load<DT>(rowQ, base + lane, vq0);
-                    f_load<DT>(rowP, base + 32 + lane, vp1); f_load<DT>(rowQ, base + 32 + lane, vq1);
-                    f_accumulate<EPV>(vp0, kf, MPw, sP); f_accumulate<EPV>(vq0, kf, MQw, sQ);
-                    f_accumulate<EPV>(vp1, kf, MPw, sP); f_accumulate<EPV>(vq1, kf, MQw, sQ);
-                }
-                for (; base < w1; base += 32) {
-                    float vp[EPV], vq[EPV];
-                    f_load_tail<DT>(rowP, base + lane, w1, vp); f_load_tail<DT>(rowQ, base + lane, w1, vq);
-                    f_accumulate<EPV>(vp, kf, MPw, sP); f_accumulate<EPV>(vq, kf, MQw, sQ);
-                }
-            } else {
-                for (; base < w1; base += 32) {
-                    float vp[EPV];
-                    f_load_tail<DT>(rowP, base + lane, w1, vp);
-                    f_accumulate<EPV>(vp, kf, MPw, sP);
-                }
+                f_accumulate<EPV>(vp, kf, MPw, sP);
+                if (have_q) f_accumulate<EPV>(vq, kf, MQw, sQ);
+                fetch_step(k + kFAhead, slot);
+                slot = (slot + 2) & (kFDepth - 1);
             }
             sP = warp_sum(sP);
             sQ = warp_sum(sQ);
@@ -410,19 +409,15 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
             const float cp = have_q ? sh.c : 1.f, cq = have_q ? 1.f : 0.f;
             const float nMP = -sh.MP, nMQ = -sh.MQ;
             float acc = 0.f;
-            int base = w0;
-            for (; base + 64 <= wfull; base += 64) {
-                float vp0[EPV], vq0[EPV], vp1[EPV], vq1[EPV], t0[EPV], t1[EPV];
-                f_load<DT>(rowP, base + lane, vp0); f_load<DT>(rowP, base + 32 + lane, vp1);
-                f_load_tail<DT>(rowQ, base + lane, w1, vq0); f_load_tail<DT>(rowQ, base + 32 + lane, w1, vq1);
-                acc += f_pair_sum<EPV>(vp0, vq0, kf, cp, cq, nMP, nMQ, t0);
-                acc += f_pair_sum<EPV>(vp1, vq1, kf, cp, cq, nMP, nMQ, t1);
-            }
-            for (; base < w1; base += 32) {
+            int slot = 0;
+            for (int k = 0; k < nsteps; ++k) {
+                cp_async_wait<kFDepth - 2>();
                 float vp[EPV], vq[EPV], t[EPV];
-                f_load_tail<DT>(rowP, base + lane, w1, vp);
-                f_load_tail<DT>(rowQ, base + lane, w1, vq);
+                R::unpack(ring[slot * kFThreads], vp);
+                R::unpack(ring[(slot + 1) * kFThreads], vq);
                 acc += f_pair_sum<EPV>(vp, vq, kf, cp, cq, nMP, nMQ, t);
+                fetch_step(k + kFAhead, slot);
+                slot = (slot + 2) & (kFDepth - 1);
             }
             acc = warp_sum(acc);
             if (lane == 0) fl.seg_tot[static_cast<size_t>(ri) * (cx.nch * kFWarps) + ch * kFWarps + warp] = acc;
@@ -505,6 +500,7 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
                 }
             }
         }
+        cp_async_wait<0>();
         __syncthreads();   // shared scratch is reused by the next item
     }
 }
@@ -561,9 +557,16 @@ static FKernelFn pick_flow(int dtype) {
     return dtype == kF32 ? verify_flow_kernel<kF32> : verify_flow_kernel<kBF16>;
 }
 
+static constexpr size_t kFlowSmem = sizeof(uint4) * kFDepth * kFThreads;
+
 int flow_max_ctas_per_sm(int dtype) {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_flow(dtype), kFThreads, 0) != cudaSuccess) {
+    if (cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_flow(dtype)),
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kFlowSmem)) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_flow(dtype), kFThreads, kFlowSmem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -571,7 +574,7 @@ int flow_max_ctas_per_sm(int dtype) {
 }
 
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream) {
-    pick_flow(dtype)<<<nctas, kFThreads, 0, stream>>>(prm, fl);
+    pick_flow(dtype)<<<nctas, kFThreads, kFlowSmem, stream>>>(prm, fl);
     return cudaGetLastError();
 }
 

@@ -55,22 +55,6 @@ struct ResShared {
     float MP, MQ;     // row references
 };
 
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-// One ring item: a 16-byte asynchronous copy when `pred`, else the slot is filled with
-// `fill` (the bit pattern of -inf logits); either way one commit group.
-__device__ __forceinline__ void ring_fetch(void* slot, const void* src, bool pred, uint32_t fill) {
-    const unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(slot));
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t"
-        "@p cp.async.cg.shared.global [%0], [%1], 16;\n\t"
-        "@!p st.shared.v4.b32 [%0], {%3, %3, %3, %3};\n\t"
-        "cp.async.commit_group;\n\t}"
-        ::"r"(s), "l"(src), "r"(static_cast<int>(pred)), "r"(fill) : "memory");
-}
-
 // a_e = 2^{v_e k - M} and their sum (branch-free; -inf logits give 0, NaN stays NaN)
 template <int EPV>
 __device__ __forceinline__ float expo(const float (&v)[EPV], float kf, float M, float (&a)[EPV]) {
