@@ -45,12 +45,15 @@ typedef enum bv_status {
                                  unknown dtype, pointer not aligned to its element size */
     BV_ERR_UNSUPPORTED = -2,  /* gamma > BV_MAX_GAMMA, or no sm_100 device              */
     BV_ERR_CUDA = -3,         /* a CUDA runtime call failed; see bv_last_cuda_error()   */
-    BV_ERR_TIMEOUT = -4       /* a bounded device-side wait gave up (reported by the
+    BV_ERR_TIMEOUT = -4,      /* a bounded device-side wait gave up (reported by the
                                  host-buffer entry points, which synchronise)           */
+    BV_ERR_TOO_LARGE = -5     /* bv_verify_noalloc: B, gamma, V need more scratch than
+                                 BV_NOALLOC_SCRATCH_BYTES                               */
 } bv_status;
 
 enum { BV_DTYPE_F32 = 0, BV_DTYPE_BF16 = 1 };
 enum { BV_MAX_GAMMA = 64 };
+enum { BV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024 };
 
 /*
  * Block Verification: Algorithm 2 with Eq. "def_as" (p_0 = 1,
@@ -123,6 +126,34 @@ int tv_verify_host(const void* target_logits, const void* draft_logits,
                    const int32_t* draft_tokens, const float* uniforms,
                    int B, int gamma, int V, int dtype, float temperature,
                    int32_t* out_tokens, int32_t* out_len);
+
+/*
+ * Block Verification without any allocation.  (The paper has no counterpart: this entry
+ * point exists for the way the library is embedded, not for the method.)
+ *
+ * For callers that cannot let a library call cudaMalloc when they call it: servers whose
+ * memory pool owns the whole device, code that may run under stream capture, processes
+ * with allocator hooks.  Same arguments, outputs and arithmetic as bv_verify(), DEVICE
+ * pointers, asynchronous on `stream`; it never calls cudaMalloc, cudaFree or any routine
+ * that allocates.  Its scratch is a fixed array of BV_NOALLOC_SCRATCH_BYTES (4 MiB) inside
+ * the library image, present on every GPU that loads the library until the process exits.
+ *
+ * Limits and rules that bv_verify() does not have:
+ *   - the scratch needed grows with B (gamma+1), about 0.9 KB per logit row pair at large V
+ *     (B = 256, gamma = 8, V = 256000 needs 2.0 MiB); a problem that needs more than the
+ *     array returns BV_ERR_TOO_LARGE and launches nothing;
+ *   - rows must be whole 16-byte vectors on 16-byte aligned bases (V a multiple of 8 for
+ *     bf16, of 4 for fp32), else BV_ERR_UNSUPPORTED;
+ *   - the first call on each device looks the array's device address up and queries the
+ *     device; make that first call before any stream capture begins;
+ *   - every call on a device uses the same array, which keeps the previous call's contents
+ *     (the entry point clears the part that must start at zero, on `stream`).  Two calls
+ *     that overlap on the GPU, on different streams, race on it: order them yourself.
+ */
+int bv_verify_noalloc(const void* target_logits, const void* draft_logits,
+                      const int32_t* draft_tokens, const float* uniforms,
+                      int B, int gamma, int V, int dtype, float temperature,
+                      int32_t* out_tokens, int32_t* out_len, void* stream);
 
 /* Frees the library's cached device buffers on the current device. */
 int bv_release(void);

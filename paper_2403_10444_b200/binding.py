@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -48,7 +48,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib = ctypes.CDLL(p)
     vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
     base = [vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp]
-    for name in ("bv_verify", "tv_verify"):
+    for name in ("bv_verify", "tv_verify", "bv_verify_noalloc"):
         getattr(lib, name).argtypes = base + [vp]
     for name in ("bv_verify_ex", "tv_verify_ex"):
         getattr(lib, name).argtypes = base + [vp, vp, vp, vp, vp, vp]
@@ -166,6 +166,31 @@ def tv_verify_ex(target_logits, draft_logits, draft_tokens, uniforms, temperatur
     """tv_verify plus its intermediates (NaN where Algorithm 1 forms none)."""
     return _device_call("tv_verify_ex", target_logits, draft_logits, draft_tokens, uniforms,
                         temperature, True, stream)
+
+
+def bv_verify_noalloc(target_logits, draft_logits, draft_tokens, uniforms, out_tokens, out_len,
+                      temperature: float = 1.0, stream=None) -> None:
+    """Block Verification through the entry point that allocates nothing.
+
+    For embedders that cannot let the library allocate device memory when they call it
+    (a memory pool that owns the device, possible stream capture, allocator hooks).  The
+    caller supplies the outputs: ``out_tokens`` int32 [B, gamma+1] and ``out_len`` int32 [B],
+    CUDA tensors; this wrapper creates no tensor either.  Raises BVError(status -5) when the
+    problem needs more than the library's fixed 4 MiB scratch array.
+    """
+    lib = load_library()
+    B, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms, True)
+    if tuple(out_tokens.shape) != (B, gamma + 1) or out_tokens.dtype != torch.int32 or not out_tokens.is_cuda:
+        raise ValueError("out_tokens must be a CUDA int32 tensor [B, gamma+1]")
+    if tuple(out_len.shape) != (B,) or out_len.dtype != torch.int32 or not out_len.is_cuda:
+        raise ValueError("out_len must be a CUDA int32 tensor [B]")
+    dev = target_logits.device
+    with torch.cuda.device(dev):
+        s = stream if stream is not None else torch.cuda.current_stream(dev)
+        _check(lib.bv_verify_noalloc(target_logits.data_ptr(), draft_logits.data_ptr(),
+                                     draft_tokens.data_ptr(), uniforms.data_ptr(), B, gamma, V,
+                                     _dtype_code(target_logits), float(temperature),
+                                     out_tokens.data_ptr(), out_len.data_ptr(), s.cuda_stream))
 
 
 def _host_call(name: str, target, draft, tokens, uniforms, temperature, out_tokens, out_len):

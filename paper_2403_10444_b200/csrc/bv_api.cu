@@ -373,6 +373,7 @@ const char* bv_status_string(int status) {
         case BV_ERR_UNSUPPORTED: return "unsupported shape or device";
         case BV_ERR_CUDA: return "CUDA runtime error";
         case BV_ERR_TIMEOUT: return "device-side wait timed out";
+        case BV_ERR_TOO_LARGE: return "problem needs more scratch than the no-allocation entry point has";
         default: return "unknown status";
     }
 }

@@ -1,0 +1,114 @@
+// Block Verification for callers that must not allocate device memory.
+//
+// Some hosts of this library run where cudaMalloc is off limits at call time: inside a
+// serving loop whose memory pool owns every byte of the device and treats a foreign
+// allocation as a leak or an out-of-memory risk, inside code that may be under stream
+// capture (where an allocation is an error), or in a process whose allocator hooks forbid
+// it.  bv_verify() keeps its scratch in buffers it allocates on demand, so it does not
+// suit them.  bv_verify_noalloc() runs the same flow kernel with its scratch in a
+// fixed array that is part of the library image: nothing is allocated, ever, at the price
+// of a hard size limit and of one array shared by every call on a device.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <mutex>
+
+#include "../../include/bv.h"
+#include "bv_launch.h"
+
+namespace {
+
+// Every GPU that loads the library holds this array until the process exits.
+constexpr size_t kScratchBytes = static_cast<size_t>(BV_NOALLOC_SCRATCH_BYTES);
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
+
+constexpr int kMaxDevices = 64;
+struct NoAllocDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;   // device address of g_noalloc_scratch on this device
+    int sm_count = 0;
+    int ctas_per_sm[2] = {};
+};
+NoAllocDevice g_na[kMaxDevices];
+std::mutex g_na_mu;
+
+bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace
+
+extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
+                                 int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
+    if (!tgt || !drf || !tok || !uni || !ot || !ol) return BV_ERR_INVALID_ARG;
+    if (B < 0 || gamma < 1 || V < 1) return BV_ERR_INVALID_ARG;
+    if (!(T > 0.f) || !std::isfinite(T)) return BV_ERR_INVALID_ARG;
+    if (dtype != BV_DTYPE_F32 && dtype != BV_DTYPE_BF16) return BV_ERR_INVALID_ARG;
+    if (gamma > BV_MAX_GAMMA) return BV_ERR_UNSUPPORTED;
+    const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
+    const size_t row_bytes = static_cast<size_t>(V) * esz;
+    // only the 128-bit path exists here: rows of whole 16-byte vectors on 16-byte aligned bases
+    if (row_bytes % 16 != 0 || !aligned_to(tgt, 16) || !aligned_to(drf, 16)) return BV_ERR_UNSUPPORTED;
+    if (!aligned_to(tok, 4) || !aligned_to(uni, 4) || !aligned_to(ot, 4) || !aligned_to(ol, 4))
+        return BV_ERR_INVALID_ARG;
+    if (B == 0) return BV_OK;
+
+    // same chunking rule as bv_verify, so both entry points take identical arithmetic paths
+    const long long units = static_cast<long long>(row_bytes / 16);
+    int nch = static_cast<int>(units / 1024);
+    nch = nch < 1 ? 1 : (nch > 8 ? 8 : nch);
+    size_t zero_bytes = 0;
+    const size_t need = bv::flow_scratch_bytes(B, gamma, nch, &zero_bytes) + 256;   // + the status word
+    if (need > kScratchBytes) return BV_ERR_TOO_LARGE;
+
+    std::lock_guard<std::mutex> lock(g_na_mu);
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BV_ERR_CUDA;
+    NoAllocDevice& d = g_na[dev];
+    if (!d.ready) {
+        // Set-up, once per device with that device current.  In host code the array's name only
+        // stands for the symbol; the address a kernel can use comes from the runtime.
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return BV_ERR_CUDA;
+        }
+        int major = 0;
+        if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return BV_ERR_CUDA;
+        }
+        if (major < 10) return BV_ERR_UNSUPPORTED;
+        d.scratch = static_cast<unsigned char*>(p);
+        d.ready = true;
+    }
+    int& per_sm = d.ctas_per_sm[dtype];
+    if (per_sm == 0) {
+        per_sm = bv::flow_max_ctas_per_sm(dtype);
+        if (per_sm <= 0) per_sm = -1;
+    }
+    if (per_sm < 0) return BV_ERR_UNSUPPORTED;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The array keeps what the previous call left: counters, locks and the ready list must
+    // start at zero, and so does the status word at the very end of the used part.
+    if (cudaMemsetAsync(d.scratch, 0, zero_bytes, s) != cudaSuccess) { cudaGetLastError(); return BV_ERR_CUDA; }
+    unsigned char* status_word = d.scratch + (need - 256);
+    if (cudaMemsetAsync(status_word, 0, 256, s) != cudaSuccess) { cudaGetLastError(); return BV_ERR_CUDA; }
+
+    bv::FlowScratch fl;
+    bv::flow_scratch_layout(d.scratch, B, gamma, nch, &fl);
+    bv::Params prm{};
+    prm.tgt = tgt; prm.drf = drf; prm.tok = tok; prm.uni = uni;
+    prm.B = B; prm.gamma = gamma; prm.V = V;
+    const double kd = 1.4426950408889634073599246810019 / static_cast<double>(T);
+    prm.kd = kd;
+    prm.kf = static_cast<float>(kd);
+    prm.out_tokens = ot; prm.out_len = ol;
+    prm.status = reinterpret_cast<int*>(status_word);
+    long long items = static_cast<long long>(B) * (gamma + 1) * nch;
+    long long nctas = static_cast<long long>(d.sm_count) * per_sm;
+    if (nctas > items) nctas = items;
+    if (bv::launch_flow(prm, fl, dtype, static_cast<int>(nctas), s) != cudaSuccess) return BV_ERR_CUDA;
+    return BV_OK;
+}
