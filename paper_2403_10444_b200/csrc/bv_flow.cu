@@ -42,14 +42,29 @@ __device__ __forceinline__ unsigned ld_volatile(const unsigned* p) {
     return *reinterpret_cast<const volatile unsigned*>(p);
 }
 
-// ---- per-vector arithmetic (same formulation as the cluster kernel) ----
+// ---- per-vector arithmetic; multiply-adds and additions are issued two lanes at a time
+// (fma.rn.f32x2 / add.rn.f32x2), which halves their share of the instruction stream ----
+__device__ __forceinline__ float2 f2(float x, float y) { return make_float2(x, y); }
+
+// a_e = 2^{v_e k - M}
+template <int EPV> __device__ __forceinline__ void f_exps(const float (&v)[EPV], float kf, float nM, float (&a)[EPV]) {
+    const float2 kk = f2(kf, kf), mm = f2(nM, nM);
+#pragma unroll
+    for (int e = 0; e < EPV; e += 2) {
+        const float2 x = __ffma2_rn(f2(v[e], v[e + 1]), kk, mm);
+        a[e] = ex2(x.x);
+        a[e + 1] = ex2(x.y);
+    }
+}
+template <int EPV> __device__ __forceinline__ float f_sum(const float (&a)[EPV]) {
+    float2 s = __fadd2_rn(f2(a[0], a[1]), f2(a[2], a[3]));
+    if (EPV == 8) s = __fadd2_rn(s, __fadd2_rn(f2(a[4], a[5]), f2(a[6], a[7])));
+    return s.x + s.y;
+}
 template <int EPV> __device__ __forceinline__ float f_exp_sum(const float (&v)[EPV], float kf, float nM) {
     float a[EPV];
-#pragma unroll
-    for (int e = 0; e < EPV; ++e) a[e] = ex2(fmaf(v[e], kf, nM));
-    float s0 = a[0] + a[1], s1 = a[2] + a[3];
-    if (EPV == 8) { s0 += a[4] + a[5]; s1 += a[6] + a[7]; }
-    return s0 + s1;
+    f_exps<EPV>(v, kf, nM, a);
+    return f_sum<EPV>(a);
 }
 template <int EPV> __device__ __forceinline__ void f_accumulate(const float (&v)[EPV], float kf, float& M, float& s) {
     float vs = f_exp_sum<EPV>(v, kf, -M);
@@ -60,18 +75,27 @@ template <int EPV> __device__ __forceinline__ void f_accumulate(const float (&v)
     }
     s += vs;
 }
-template <int EPV>
+// residual terms t_e = max(cp 2^{zP k - MP} - 2^{zQ k - MQ}, 0) and their sum; HAVEQ = false: t_e = cp 2^{zP k - MP}
+template <int EPV, bool HAVEQ>
 __device__ __forceinline__ float f_pair_sum(const float (&vp)[EPV], const float (&vq)[EPV], float kf, float cp,
-                                            float cq, float nMP, float nMQ, float (&t)[EPV]) {
+                                            float nMP, float nMQ, float (&t)[EPV]) {
+    float a[EPV], q[EPV];
+    f_exps<EPV>(vp, kf, nMP, a);
+    if (HAVEQ) f_exps<EPV>(vq, kf, nMQ, q);
+    const float2 cc = f2(cp, cp);
 #pragma unroll
-    for (int e = 0; e < EPV; ++e) {
-        const float a = ex2(fmaf(vp[e], kf, nMP));
-        const float q = ex2(fmaf(vq[e], kf, nMQ));
-        t[e] = fmaxf(fmaf(cp, a, -(cq * q)), 0.f);
+    for (int e = 0; e < EPV; e += 2) {
+        if (HAVEQ) {
+            const float2 d = __ffma2_rn(cc, f2(a[e], a[e + 1]), f2(-q[e], -q[e + 1]));
+            t[e] = fmaxf(d.x, 0.f);
+            t[e + 1] = fmaxf(d.y, 0.f);
+        } else {
+            const float2 d = __fmul2_rn(cc, f2(a[e], a[e + 1]));
+            t[e] = d.x;
+            t[e + 1] = d.y;
+        }
     }
-    float s0 = t[0] + t[1], s1 = t[2] + t[3];
-    if (EPV == 8) { s0 += t[4] + t[5]; s1 += t[6] + t[7]; }
-    return s0 + s1;
+    return f_sum<EPV>(t);
 }
 template <int DT> __device__ __forceinline__ void f_load(const char* row, int i, float (&v)[Raw<DT>::EPV]) {
     Raw<DT>::unpack(ld_stream_v4(row + static_cast<size_t>(i) * 16), v);
@@ -110,7 +134,7 @@ __device__ __forceinline__ void chunk_range(const FlowCtx& cx, int ch, int warp,
 // One warp walks segment [w0, w1) of a row pair in index order and returns the first element
 // whose running residual mass exceeds tw (else the last element with positive mass, else -1).
 template <int DT>
-__device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int lane, float kf, float cp, float cq,
+__device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int lane, float kf, float cp,
                         float nMP, float nMQ, float tw) {
     constexpr int EPV = Raw<DT>::EPV;
     float run = 0.f;
@@ -120,7 +144,8 @@ __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int 
         float vp[EPV], vq[EPV], tt[EPV];
         f_load_tail<DT>(rowP, i, w1, vp);
         f_load_tail<DT>(rowQ, i, w1, vq);
-        const float ls = f_pair_sum<EPV>(vp, vq, kf, cp, cq, nMP, nMQ, tt);
+        const float ls = rowQ ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, tt)
+                              : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, tt);
 #pragma unroll
         for (int e = 0; e < EPV; ++e) if (tt[e] > 0.f) last_pos = i * EPV + e;
         float incw = ls;
@@ -406,7 +431,7 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
             }
         } else {
             // ---------------- sweep 2 over this chunk ----------------
-            const float cp = have_q ? sh.c : 1.f, cq = have_q ? 1.f : 0.f;
+            const float cp = have_q ? sh.c : 1.f;
             const float nMP = -sh.MP, nMQ = -sh.MQ;
             float acc = 0.f;
             int slot = 0;
@@ -415,7 +440,8 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
                 float vp[EPV], vq[EPV], t[EPV];
                 R::unpack(ring[slot * kFThreads], vp);
                 R::unpack(ring[(slot + 1) * kFThreads], vq);
-                acc += f_pair_sum<EPV>(vp, vq, kf, cp, cq, nMP, nMQ, t);
+                acc += have_q ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, t)
+                              : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, t);
                 fetch_step(k + kFAhead, slot);
                 slot = (slot + 2) & (kFDepth - 1);
             }
@@ -476,7 +502,7 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
                     const float before = __shfl_sync(0xffffffffu, bef, src);
                     int s0, s1;
                     chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1);
-                    found = f_rescan<DT>(rowP, rowQ, s0, s1, lane, kf, cp, cq, nMP, nMQ, t - before);
+                    found = f_rescan<DT>(rowP, rowQ, s0, s1, lane, kf, cp, nMP, nMQ, t - before);
                 } else if (have_q && r == 0 && total == 0.f) {
                     // empty residual at position 0 (P_0 and Q_0 coincide): sample P_0 with the same uniform.
                     // Two plain passes over the whole row by this warp: rare, so speed does not matter.
@@ -485,10 +511,10 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
                         float vp[EPV], vq[EPV], t2[EPV];
                         f_load_tail<DT>(rowP, base2 + lane, cx.units, vp);
                         f_load_tail<DT>(nullptr, 0, 0, vq);
-                        tot += f_pair_sum<EPV>(vp, vq, kf, 1.f, 0.f, nMP, nMQ, t2);
+                        tot += f_pair_sum<EPV, false>(vp, vq, kf, 1.f, nMP, nMQ, t2);
                     }
                     tot = warp_sum(tot);
-                    found = f_rescan<DT>(rowP, nullptr, 0, cx.units, lane, kf, 1.f, 0.f, nMP, nMQ, uf * tot);
+                    found = f_rescan<DT>(rowP, nullptr, 0, cx.units, lane, kf, 1.f, nMP, nMQ, uf * tot);
                 }
                 if (lane == 0) {
                     fl.cand[ri] = found;
