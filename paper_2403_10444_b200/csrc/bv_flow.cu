@@ -30,6 +30,8 @@ struct FlowShared {
     float red_M[2][kFWarps];
     float red_s[2][kFWarps];
     int kind, item, last;       // what this CTA does next; whether it completed a row / position
+    int sel, found;             // sampling: segment that holds the target, token found
+    float target;               // sampling: target mass inside that segment
     float c, MP, MQ;            // sweep 2: p_r Z_Q / Z_P and the row references
 };
 
@@ -250,53 +252,59 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
     // the row's maximum is finite iff its reference is; Z is NaN / inf iff the row holds a NaN / overflowed
     if (!(MP > kNoRef && MP < INFINITY) || !(ZP < INFINITY)) atomicOr(&fl.bad[b], 1u);
     if (have_q && (!(MQ > kNoRef && MQ < INFINITY) || !(ZQ < INFINITY))) atomicOr(&fl.bad[b], 1u);
+    // everything the recursion needs from this row, computed before the lock is taken:
+    // ratio = P_r(X_{r+1}) / Q_r(X_{r+1}) from the two logits of the drafted token, and Z_Q / Z_P
+    if (have_q) {
+        double ratio = 0.0;
+        const int x = prm.tok[static_cast<size_t>(b) * g + r];
+        if (x < 0 || x >= cx.V) {
+            atomicOr(&fl.bad[b], 1u);
+        } else {
+            const char* rowP = static_cast<const char*>(prm.tgt) + rowi * cx.row_bytes;
+            const char* rowQ = static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes;
+            const double zq = load_logit<DT>(rowQ, x), zp = load_logit<DT>(rowP, x);
+            if (zq == -INFINITY) atomicOr(&fl.bad[b], 1u);
+            else ratio = exp2((zp - zq) * cx.kd - (MP - MQ)) * (ZQ / ZP);
+        }
+        fl.ratio[rowi] = ratio;
+        fl.zratio[rowi] = ZQ / ZP;
+    }
     __threadfence();
     atomicExch(&fl.row_done[rowi], 1u);
 
-    // advance the block's recursion while the next row is complete (short critical section)
-    unsigned spins = 0;
-    while (atomicCAS(&fl.lock[b], 0u, 1u) != 0u) {
-        __nanosleep(100);
-        if (++spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return; }
+    // Fold every complete row, in order, into p_{c+1} = min(p_c ratio_c, 1) and release its
+    // sweep-2 items.  The critical section is a few loads and stores per row.
+    double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
+    for (unsigned spins = 0;; ++spins) {
+        if (atomicCAS(&fl.lock[b], 0u, 1u) == 0u) break;
+        // the holder may have looked at this row before it was marked: wait for it to let go,
+        // unless the recursion has already moved past this row
+        if (ld_volatile(&fl.chain[b]) > static_cast<unsigned>(r)) return;
+        __nanosleep(32);
+        if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return; }
     }
     __threadfence();
     unsigned c = ld_volatile(&fl.chain[b]);
-    double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
+    unsigned pushed = 0;
     while (c <= static_cast<unsigned>(g) && ld_volatile(&fl.row_done[static_cast<size_t>(b) * (g + 1) + c]) != 0u) {
-        __threadfence();
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
-        const RowZ z = load_rowz(&fl.rowZ[ci]);
         const double p_c = (c == 0) ? 1.0 : __ldcg(&p[c]);
         if (c == 0) p[0] = 1.0;
         float cs = 1.f;
         if (c < static_cast<unsigned>(g)) {
-            // ratio = P_c(X_{c+1}) / Q_c(X_{c+1}) from the two logits of the drafted token
-            double ratio = 0.0;
-            const int x = prm.tok[static_cast<size_t>(b) * g + c];
-            if (x < 0 || x >= cx.V) {
-                atomicOr(&fl.bad[b], 1u);
-            } else {
-                const char* rowP = static_cast<const char*>(prm.tgt) + ci * cx.row_bytes;
-                const char* rowQ = static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + c) * cx.row_bytes;
-                const double zq = load_logit<DT>(rowQ, x), zp = load_logit<DT>(rowP, x);
-                if (zq == -INFINITY) atomicOr(&fl.bad[b], 1u);
-                else ratio = exp2((zp - zq) * cx.kd - (z.MP - z.MQ)) * (z.ZQ / z.ZP);
-            }
-            p[c + 1] = fmin(p_c * ratio, 1.0);
-            cs = static_cast<float>(p_c * z.ZQ / z.ZP);
+            p[c + 1] = fmin(p_c * __ldcg(&fl.ratio[ci]), 1.0);
+            cs = static_cast<float>(p_c * __ldcg(&fl.zratio[ci]));
         }
         fl.cscale[ci] = cs;
-        __threadfence();
-        // release the row's sweep-2 items
         const unsigned t = atomicAdd(&fl.counters[kTail], static_cast<unsigned>(cx.nch));
         for (int ch = 0; ch < cx.nch; ++ch)
-            atomicExch(&fl.ready[t + ch], static_cast<unsigned>(ci * cx.nch + ch) + 1u);
-        __threadfence();
-        atomicAdd(&fl.counters[kAvail], static_cast<unsigned>(cx.nch));
+            *reinterpret_cast<volatile unsigned*>(&fl.ready[t + ch]) = static_cast<unsigned>(ci * cx.nch + ch) + 1u;
+        pushed += static_cast<unsigned>(cx.nch);
         ++c;
-        *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
     }
-    __threadfence();
+    *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
+    __threadfence();                       // p, cscale and the ready entries are visible ...
+    if (pushed) atomicAdd(&fl.counters[kAvail], pushed);   // ... before the items can be taken
     atomicExch(&fl.lock[b], 0u);
 }
 
@@ -454,58 +462,98 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
                 sh.last = atomicAdd(&fl.s2_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u;
             }
             __syncthreads();
-            if (sh.last && warp == 0) {
+            if (sh.last) {
                 // ---------------- the position is complete: S_r and the candidate Y_r ----------------
                 __threadfence();
-                const int nseg = cx.nch * kFWarps;
-                const float* segs = fl.seg_tot + static_cast<size_t>(ri) * nseg;
-                float w[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) w[j] = (4 * lane + j < nseg) ? __ldcg(&segs[4 * lane + j]) : 0.f;
-                double sd = (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
-                            (static_cast<double>(w[2]) + static_cast<double>(w[3]));
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
-                const RowZ z = load_rowz(&fl.rowZ[ri]);
-                if (lane == 0 && have_q) fl.S[ri] = sd / z.ZQ;
-                const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
-                float inc = l4;
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const float o = __shfl_up_sync(0xffffffffu, inc, off);
-                    if (lane >= off) inc += o;
-                }
-                const float total = __shfl_sync(0xffffffffu, inc, 31);
                 const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
-                int found = -1;
-                if (total > 0.f) {
-                    const float t = uf * total;
-                    float exc = __shfl_up_sync(0xffffffffu, inc, 1);
-                    if (lane == 0) exc = 0.f;
-                    const float p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
-                    // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
-                    const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
-                    const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
-                    const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
-                    const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
-                    int e = 3; float bef = p3; int src;
-                    if (hit) {
-                        src = __ffs(hit) - 1;
-                        if (h1) { e = 0; bef = exc; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
-                    } else {
-                        src = 31 - __clz(nz);
-                        e = 0; bef = exc;
-                        if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
-                        else if (w[1] > 0.f) { e = 1; bef = p1; }
+                if (warp == 0) {
+                    const int nseg = cx.nch * kFWarps;
+                    const float* segs = fl.seg_tot + static_cast<size_t>(ri) * nseg;
+                    float w[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) w[j] = (4 * lane + j < nseg) ? __ldcg(&segs[4 * lane + j]) : 0.f;
+                    double sd = (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
+                                (static_cast<double>(w[2]) + static_cast<double>(w[3]));
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
+                    if (lane == 0 && have_q) fl.S[ri] = sd / __ldcg(&fl.rowZ[ri].ZQ);
+                    const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
+                    float inc = l4;
+#pragma unroll
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const float o = __shfl_up_sync(0xffffffffu, inc, off);
+                        if (lane >= off) inc += o;
                     }
-                    const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
-                    const float before = __shfl_sync(0xffffffffu, bef, src);
+                    const float total = __shfl_sync(0xffffffffu, inc, 31);
+                    int sel = -1;
+                    float before = 0.f;
+                    if (total > 0.f) {
+                        const float t = uf * total;
+                        float exc = __shfl_up_sync(0xffffffffu, inc, 1);
+                        if (lane == 0) exc = 0.f;
+                        const float p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+                        // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
+                        const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
+                        const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
+                        const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
+                        const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
+                        int e = 3; float bef = p3; int src;
+                        if (hit) {
+                            src = __ffs(hit) - 1;
+                            if (h1) { e = 0; bef = exc; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
+                        } else {
+                            src = 31 - __clz(nz);
+                            e = 0; bef = exc;
+                            if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
+                            else if (w[1] > 0.f) { e = 1; bef = p1; }
+                        }
+                        sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
+                        before = t - __shfl_sync(0xffffffffu, bef, src);    // target inside the segment
+                    } else if (have_q && r == 0 && total == 0.f) {
+                        sel = -2;   // empty residual at position 0: handled below
+                    }
+                    if (lane == 0) { sh.sel = sel; sh.target = before; sh.found = -1; }
+                }
+                __syncthreads();
+                const int sel = sh.sel;
+                if (sel >= 0) {
+                    // the segment that holds the target, cut into one piece per warp: piece totals,
+                    // then only the piece that holds the target is walked element by element
                     int s0, s1;
                     chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1);
-                    found = f_rescan<DT>(rowP, rowQ, s0, s1, lane, kf, cp, nMP, nMQ, t - before);
-                } else if (have_q && r == 0 && total == 0.f) {
-                    // empty residual at position 0 (P_0 and Q_0 coincide): sample P_0 with the same uniform.
-                    // Two plain passes over the whole row by this warp: rare, so speed does not matter.
+                    const int q0 = s0 + static_cast<int>(static_cast<long long>(s1 - s0) * warp / kFWarps);
+                    const int q1 = s0 + static_cast<int>(static_cast<long long>(s1 - s0) * (warp + 1) / kFWarps);
+                    float sub = 0.f;
+                    for (int base2 = q0; base2 < q1; base2 += 32) {
+                        float vp[EPV], vq[EPV], t2[EPV];
+                        f_load_tail<DT>(rowP, base2 + lane, q1, vp);
+                        f_load_tail<DT>(rowQ, base2 + lane, q1, vq);
+                        sub += have_q ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, t2)
+                                      : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, t2);
+                    }
+                    sub = warp_sum(sub);
+                    if (lane == 0) sh.red_s[0][warp] = sub;
+                    __syncthreads();
+                    const float mine = lane < kFWarps ? sh.red_s[0][lane] : 0.f;
+                    float incp = mine;
+#pragma unroll
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const float o = __shfl_up_sync(0xffffffffu, incp, off);
+                        if (lane >= off) incp += o;
+                    }
+                    const float tgt = sh.target;
+                    const unsigned hitp = __ballot_sync(0xffffffffu, incp > tgt && mine > 0.f);
+                    const unsigned nzp = __ballot_sync(0xffffffffu, mine > 0.f);
+                    const int piece = hitp ? __ffs(hitp) - 1 : (nzp ? 31 - __clz(nzp) : -1);
+                    if (piece == warp) {
+                        const float befp = __shfl_sync(0xffffffffu, incp - mine, piece);
+                        const int y = f_rescan<DT>(rowP, rowQ, q0, q1, lane, kf, cp, nMP, nMQ, tgt - befp);
+                        if (lane == 0) sh.found = y;
+                    }
+                    __syncthreads();
+                } else if (sel == -2 && warp == 0) {
+                    // sample P_0 with the same uniform: two plain passes over the whole row by one
+                    // warp (rare: P_0 and Q_0 coincide bit for bit), so speed does not matter
                     float tot = 0.f;
                     for (int base2 = 0; base2 < cx.units; base2 += 32) {
                         float vp[EPV], vq[EPV], t2[EPV];
@@ -514,10 +562,12 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
                         tot += f_pair_sum<EPV, false>(vp, vq, kf, 1.f, nMP, nMQ, t2);
                     }
                     tot = warp_sum(tot);
-                    found = f_rescan<DT>(rowP, nullptr, 0, cx.units, lane, kf, 1.f, nMP, nMQ, uf * tot);
+                    const int y = f_rescan<DT>(rowP, nullptr, 0, cx.units, lane, kf, 1.f, nMP, nMQ, uf * tot);
+                    if (lane == 0) sh.found = y;
                 }
-                if (lane == 0) {
-                    fl.cand[ri] = found;
+                if (sel == -2) __syncthreads();
+                if (tid == 0) {
+                    fl.cand[ri] = sh.found;
                     __threadfence();
                     if (atomicAdd(&fl.cand_cnt[b], 1u) == static_cast<unsigned>(g)) {
                         __threadfence();
@@ -549,6 +599,7 @@ size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes) {
     n += up256(rows * sizeof(RowZ));                // rowZ
     n += up256(static_cast<size_t>(B) * (gamma + 2) * sizeof(double));   // pchain
     n += up256(rows * sizeof(float));               // cscale
+    n += 2 * up256(rows * sizeof(double));          // ratio, zratio
     n += up256(rows * nch * kFWarps * sizeof(float));   // seg_tot
     n += up256(rows * sizeof(double));              // S
     n += up256(rows * sizeof(int));                 // cand
@@ -572,6 +623,8 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl)
     fl->rowZ = reinterpret_cast<RowZ*>(take(rows * sizeof(RowZ)));
     fl->pchain = reinterpret_cast<double*>(take(static_cast<size_t>(B) * (gamma + 2) * sizeof(double)));
     fl->cscale = reinterpret_cast<float*>(take(rows * sizeof(float)));
+    fl->ratio = reinterpret_cast<double*>(take(rows * sizeof(double)));
+    fl->zratio = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->seg_tot = reinterpret_cast<float*>(take(rows * nch * kFWarps * sizeof(float)));
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));

@@ -38,6 +38,8 @@ struct FlowScratch {
     RowZ* rowZ;           // [B (gamma+1)]
     double* pchain;       // [B (gamma+2)]
     float* cscale;        // [B (gamma+1)] p_r Z_Q / Z_P
+    double* ratio;        // [B (gamma+1)] P_r(X_{r+1}) / Q_r(X_{r+1})
+    double* zratio;       // [B (gamma+1)] Z_Q / Z_P
     float* seg_tot;       // [B (gamma+1) nch 16]
     double* S;            // [B (gamma+1)]
     int* cand;            // [B (gamma+1)]
