@@ -138,19 +138,18 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
 
     // Block Verification on 16-byte rows: the flow of independent work items
     if (algo == bv::kBlockVerify && vec && (!want || forced("flow"))) {
-        const long long units = static_cast<long long>(row_bytes / 16);
-        int nch = static_cast<int>(units / 1024);
-        nch = nch < 1 ? 1 : (nch > 8 ? 8 : nch);
-        if (const char* env = std::getenv("BV_FLOW_CHUNKS")) {
-            const int v = std::atoi(env);
-            if (v >= 1 && v <= 8) nch = v;
-        }
         int& per_sm = d->flow_ctas_per_sm[dtype];
         if (per_sm == 0) {
             per_sm = bv::flow_max_ctas_per_sm(dtype);
             if (per_sm <= 0) per_sm = -1;
         }
         if (per_sm > 0) {
+            const long long units = static_cast<long long>(row_bytes / 16);
+            int nch = bv::flow_pick_chunks(units, B, gamma, static_cast<long long>(d->sm_count) * per_sm);
+            if (const char* env = std::getenv("BV_FLOW_CHUNKS")) {
+                const int v = std::atoi(env);
+                if (v >= 1 && v <= 8) nch = v;
+            }
             size_t zero_bytes = 0;
             const size_t need = bv::flow_scratch_bytes(B, gamma, nch, &zero_bytes);
             const int slot = static_cast<int>(d->flow_calls++ % 4);

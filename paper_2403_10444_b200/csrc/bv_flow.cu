@@ -631,6 +631,18 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl)
     fl->nch = nch;
 }
 
+// Chunks per row.  An item should be large next to what it costs to hand it out (about
+// 16000 vectors, 256 KB, per row), yet there should be a few items per CTA to balance the
+// load, as long as a chunk keeps at least 2048 vectors.
+int flow_pick_chunks(long long units, int B, int gamma, long long nctas) {
+    long long nch = (units + 8000) / 16000;
+    if (nch < 1) nch = 1;
+    if (nch > 8) nch = 8;
+    const long long rows = static_cast<long long>(B) * (gamma + 1);
+    while (nch < 8 && rows * nch < 4 * nctas && units / (nch + 1) >= 2048) ++nch;
+    return static_cast<int>(nch);
+}
+
 using FKernelFn = void (*)(const Params, const FlowScratch);
 static FKernelFn pick_flow(int dtype) {
     return dtype == kF32 ? verify_flow_kernel<kF32> : verify_flow_kernel<kBF16>;

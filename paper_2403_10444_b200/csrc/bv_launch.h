@@ -48,6 +48,7 @@ struct FlowScratch {
 size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes);
 void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl);
 int flow_max_ctas_per_sm(int dtype);
+int flow_pick_chunks(long long units, int B, int gamma, long long nctas);
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream);
 
 // Resident kernel (Block Verification only, 128-bit path): a thread holds up to `nk`

@@ -52,14 +52,6 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
         return BV_ERR_INVALID_ARG;
     if (B == 0) return BV_OK;
 
-    // same chunking rule as bv_verify, so both entry points take identical arithmetic paths
-    const long long units = static_cast<long long>(row_bytes / 16);
-    int nch = static_cast<int>(units / 1024);
-    nch = nch < 1 ? 1 : (nch > 8 ? 8 : nch);
-    size_t zero_bytes = 0;
-    const size_t need = bv::flow_scratch_bytes(B, gamma, nch, &zero_bytes) + 256;   // + the status word
-    if (need > kScratchBytes) return BV_ERR_TOO_LARGE;
-
     std::lock_guard<std::mutex> lock(g_na_mu);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BV_ERR_CUDA;
@@ -88,6 +80,13 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
         if (per_sm <= 0) per_sm = -1;
     }
     if (per_sm < 0) return BV_ERR_UNSUPPORTED;
+
+    // same chunking rule as bv_verify, so both entry points take identical arithmetic paths
+    const long long units = static_cast<long long>(row_bytes / 16);
+    const int nch = bv::flow_pick_chunks(units, B, gamma, static_cast<long long>(d.sm_count) * per_sm);
+    size_t zero_bytes = 0;
+    const size_t need = bv::flow_scratch_bytes(B, gamma, nch, &zero_bytes) + 256;   // + the status word
+    if (need > kScratchBytes) return BV_ERR_TOO_LARGE;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // The array keeps what the previous call left: counters, locks and the ready list must
