@@ -251,6 +251,17 @@ __device__ __forceinline__ void ring_fetch(void* slot, const void* src, bool pre
 }
 
 
+// 16-byte asynchronous copy and 16-byte load with the shared-memory address given as a
+// 32-bit shared-space address (saves the generic-to-shared conversion in inner loops)
+__device__ __forceinline__ void cp_async16_s(uint32_t saddr, const void* gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr) : "memory");
+    return v;
+}
+
 // "No reference yet": finite, so that -inf logits still give 2^-inf = 0 and any finite
 // logit overflows to +inf, which exceeds the raise bound and installs a real reference.
 constexpr float kNoRef = -3.0e38f;

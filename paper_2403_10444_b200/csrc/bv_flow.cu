@@ -84,13 +84,14 @@ __device__ __forceinline__ float f_pair_sum(const float (&vp)[EPV], const float 
     float a[EPV], q[EPV];
     f_exps<EPV>(vp, kf, nMP, a);
     if (HAVEQ) f_exps<EPV>(vq, kf, nMQ, q);
-    const float2 cc = f2(cp, cp);
+    const float2 cc = f2(cp, cp), ncc = f2(-cp, -cp);
 #pragma unroll
     for (int e = 0; e < EPV; e += 2) {
         if (HAVEQ) {
-            const float2 d = __ffma2_rn(cc, f2(a[e], a[e + 1]), f2(-q[e], -q[e + 1]));
-            t[e] = fmaxf(d.x, 0.f);
-            t[e + 1] = fmaxf(d.y, 0.f);
+            // q - cp a in one packed multiply-add; the sign flips for free inside the max
+            const float2 d = __ffma2_rn(ncc, f2(a[e], a[e + 1]), f2(q[e], q[e + 1]));
+            t[e] = fmaxf(-d.x, 0.f);
+            t[e + 1] = fmaxf(-d.y, 0.f);
         } else {
             const float2 d = __fmul2_rn(cc, f2(a[e], a[e + 1]));
             t[e] = d.x;
@@ -321,7 +322,6 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
     // Each thread streams its own vectors through a private ring of 16-byte slots filled by
     // cp.async, so loads run kFAhead steps ahead of the arithmetic without costing registers.
     extern __shared__ __align__(16) unsigned char dyn[];
-    uint4* ring = reinterpret_cast<uint4*>(dyn) + tid;      // slot s of this thread: ring[s * kFThreads]
 
     FlowCtx cx;
     cx.g = prm.gamma; cx.V = prm.V; cx.B = prm.B; cx.nch = fl.nch; cx.units = prm.V / EPV;
@@ -382,34 +382,54 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
         int w0, w1;
         chunk_range(cx, ch, warp, w0, w1);
 
-        const int nsteps = (w1 - w0 + 31) >> 5;             // warp-uniform; lanes past w1 see -inf logits
-        const char* srcP = rowP + static_cast<size_t>(w0 + lane) * 16;
-        const char* srcQ = have_q ? rowQ + static_cast<size_t>(w0 + lane) * 16 : nullptr;
-        auto fetch_step = [&](int k, int slot) {
-            const bool ok = k < nsteps && (w0 + lane + 32 * k) < w1;
-            ring_fetch(ring + slot * kFThreads, srcP + static_cast<size_t>(k) * 512, ok, R::kNegInf);
-            ring_fetch(ring + (slot + 1) * kFThreads, srcQ + static_cast<size_t>(k) * 512, ok && have_q, R::kNegInf);
+        // This warp's segment: nfull steps in which every lane has a vector (streamed through the
+        // ring) and at most one partial step (loaded directly; lanes past the end see -inf logits).
+        const int nv = w1 - w0, nfull = nv >> 5;
+        constexpr uint32_t kSlot = kFThreads * 16;           // bytes between consecutive ring slots
+        const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;
+        const char* gP = rowP + static_cast<size_t>(w0 + lane) * 16;
+        const char* gQ = have_q ? rowQ + static_cast<size_t>(w0 + lane) * 16 : gP;
+        auto fetch_step = [&](int k, int j) {                // step k goes to slots 2j, 2j+1 (j = k & 3)
+            if (k < nfull) {
+                cp_async16_s(sb + (2 * j) * kSlot, gP + static_cast<size_t>(k) * 512);
+                if (have_q) cp_async16_s(sb + (2 * j + 1) * kSlot, gQ + static_cast<size_t>(k) * 512);
+            }
+            cp_async_commit();
         };
 #pragma unroll
-        for (int k = 0; k < kFAhead; ++k) fetch_step(k, 2 * k);
+        for (int j = 0; j < kFAhead; ++j) fetch_step(j, j);
+        const int itail = w0 + 32 * nfull + lane;            // this lane's vector in the partial step
 
         if (kind == kSweep1) {
             // ---------------- sweep 1 over this chunk ----------------
             float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
-            int slot = 0;
-            for (int k = 0; k < nsteps; ++k) {
-                cp_async_wait<kFDepth - 2>();            // step k of both rows has landed
-                float vp[EPV], vq[EPV];
-                R::unpack(ring[slot * kFThreads], vp);
-                R::unpack(ring[(slot + 1) * kFThreads], vq);
-                if (k == 0) {                            // references from the first vector of every lane
+            auto step1 = [&](const float (&vp)[EPV], const float (&vq)[EPV], bool first) {
+                if (first) {                                 // references from the first vector of every lane
                     MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
-                    MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vq)) * kf), kNoRef);
+                    if (have_q) MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vq)) * kf), kNoRef);
                 }
                 f_accumulate<EPV>(vp, kf, MPw, sP);
                 if (have_q) f_accumulate<EPV>(vq, kf, MQw, sQ);
-                fetch_step(k + kFAhead, slot);
-                slot = (slot + 2) & (kFDepth - 1);
+            };
+            for (int kb = 0; kb < nfull; kb += kFAhead) {
+#pragma unroll
+                for (int j = 0; j < kFAhead; ++j) {
+                    const int k = kb + j;
+                    if (k < nfull) {
+                        cp_async_wait<kFAhead - 1>();        // step k of both rows has landed
+                        float vp[EPV], vq[EPV];
+                        R::unpack(lds128(sb + (2 * j) * kSlot), vp);
+                        if (have_q) R::unpack(lds128(sb + (2 * j + 1) * kSlot), vq);
+                        step1(vp, vq, k == 0);
+                        fetch_step(k + kFAhead, j);
+                    }
+                }
+            }
+            if (nv & 31) {
+                float vp[EPV], vq[EPV];
+                f_load_tail<DT>(rowP, itail, w1, vp);
+                f_load_tail<DT>(rowQ, itail, w1, vq);
+                step1(vp, vq, nfull == 0);
             }
             sP = warp_sum(sP);
             sQ = warp_sum(sQ);
@@ -442,16 +462,30 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
             const float cp = have_q ? sh.c : 1.f;
             const float nMP = -sh.MP, nMQ = -sh.MQ;
             float acc = 0.f;
-            int slot = 0;
-            for (int k = 0; k < nsteps; ++k) {
-                cp_async_wait<kFDepth - 2>();
+            for (int kb = 0; kb < nfull; kb += kFAhead) {
+#pragma unroll
+                for (int j = 0; j < kFAhead; ++j) {
+                    const int k = kb + j;
+                    if (k < nfull) {
+                        cp_async_wait<kFAhead - 1>();
+                        float vp[EPV], vq[EPV], t[EPV];
+                        R::unpack(lds128(sb + (2 * j) * kSlot), vp);
+                        if (have_q) {
+                            R::unpack(lds128(sb + (2 * j + 1) * kSlot), vq);
+                            acc += f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, t);
+                        } else {
+                            acc += f_pair_sum<EPV, false>(vp, vp, kf, cp, nMP, nMQ, t);
+                        }
+                        fetch_step(k + kFAhead, j);
+                    }
+                }
+            }
+            if (nv & 31) {
                 float vp[EPV], vq[EPV], t[EPV];
-                R::unpack(ring[slot * kFThreads], vp);
-                R::unpack(ring[(slot + 1) * kFThreads], vq);
+                f_load_tail<DT>(rowP, itail, w1, vp);
+                f_load_tail<DT>(rowQ, itail, w1, vq);
                 acc += have_q ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, t)
                               : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, t);
-                fetch_step(k + kFAhead, slot);
-                slot = (slot + 2) & (kFDepth - 1);
             }
             acc = warp_sum(acc);
             if (lane == 0) fl.seg_tot[static_cast<size_t>(ri) * (cx.nch * kFWarps) + ch * kFWarps + warp] = acc;
