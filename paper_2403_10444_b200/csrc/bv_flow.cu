@@ -26,19 +26,8 @@ namespace bv {
 constexpr int kFThreads = 512;
 constexpr int kFWarps = kFThreads / 32;
 
-struct FlowShared {
-    float red_M[2][kFWarps];
-    float red_s[2][kFWarps];
-    int kind, item, last;       // what this CTA does next; whether it completed a row / position
-    int sel, found;             // sampling: segment that holds the target, token found
-    float target;               // sampling: target mass inside that segment
-    float c, MP, MQ;            // sweep 2: p_r Z_Q / Z_P and the row references
-};
-
 enum : int { kExit = 0, kSweep1 = 1, kSweep2 = 2 };
-// counters, one per 128-byte line: next sweep-1 item; released-but-untaken sweep-2 items
-// (a semaphore); slots taken from / reserved in the ready list
-enum : int { kNext = 0, kAvail = 32, kHead = 64, kTail = 96, kCounterWords = 128 };
+constexpr int kCounterWords = 32;   // [0]: the ticket counter
 
 __device__ __forceinline__ unsigned ld_volatile(const unsigned* p) {
     return *reinterpret_cast<const volatile unsigned*>(p);
@@ -286,7 +275,6 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
     }
     __threadfence();
     unsigned c = ld_volatile(&fl.chain[b]);
-    unsigned pushed = 0;
     while (c <= static_cast<unsigned>(g) && ld_volatile(&fl.row_done[static_cast<size_t>(b) * (g + 1) + c]) != 0u) {
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
         const double p_c = (c == 0) ? 1.0 : __ldcg(&p[c]);
@@ -297,30 +285,167 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
             cs = static_cast<float>(p_c * __ldcg(&fl.zratio[ci]));
         }
         fl.cscale[ci] = cs;
-        const unsigned t = atomicAdd(&fl.counters[kTail], static_cast<unsigned>(cx.nch));
-        for (int ch = 0; ch < cx.nch; ++ch)
-            *reinterpret_cast<volatile unsigned*>(&fl.ready[t + ch]) = static_cast<unsigned>(ci * cx.nch + ch) + 1u;
-        pushed += static_cast<unsigned>(cx.nch);
+        __threadfence();                       // p, cscale are visible ...
+        atomicExch(&fl.rel[ci], 1u);           // ... before the row's sweep-2 items may start
         ++c;
     }
     *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
-    __threadfence();                       // p, cscale and the ready entries are visible ...
-    if (pushed) atomicAdd(&fl.counters[kAvail], pushed);   // ... before the items can be taken
+    __threadfence();
     atomicExch(&fl.lock[b], 0u);
 }
 
-constexpr int kFDepth = 8;     // ring slots per thread: four (P, Q) steps of lookahead
+constexpr int kFDepth = 8;     // ring slots per worker thread: four (P, Q) steps of lookahead
 constexpr int kFAhead = kFDepth / 2;
+constexpr int kFDesc = 3;      // items in flight per CTA: one being swept, two queued behind it
+constexpr int kFAllThreads = kFThreads + 32;   // 16 worker warps + 1 service warp
+
+// One work item as the service warp hands it to the workers.
+struct FlowDesc {
+    int kind;                   // kExit, kSweep1, kSweep2
+    int ri, ch;                 // row index b (gamma+1) + r, chunk
+    int have_q;
+    const char* rowP;
+    const char* rowQ;
+    float cp, nMP, nMQ;         // sweep 2: p_r Z_Q / Z_P and minus the row references
+};
+
+struct FlowShared {
+    FlowDesc desc[kFDesc];
+    unsigned long long full[kFDesc];    // the service warp has filled desc[i]
+    unsigned long long done[kFDesc];    // all 16 worker warps have left their partials of desc[i]
+    float part_M[kFDesc][2][kFWarps];   // sweep 1: references of P and Q per worker warp
+    float part_s[kFDesc][2][kFWarps];   // sweep 1: sums; sweep 2: [0] holds the residual totals
+};
+
+// Items are handed out in one fixed order by a single ticket counter: step n carries the
+// sweep-1 chunks of row n and then the sweep-2 chunks of row n - lag.  Everything an item
+// waits for therefore has a smaller ticket, so whoever holds it is already running.
+struct FlowOrder { int rows, nch, lag; unsigned total; };
+
+__device__ __forceinline__ bool f_decode(const FlowOrder& od, unsigned t, int& kind, int& ri, int& ch) {
+    const int step = static_cast<int>(t / (2u * od.nch)), w = static_cast<int>(t % (2u * od.nch));
+    if (w < od.nch) { kind = kSweep1; ri = step; ch = w; }
+    else            { kind = kSweep2; ri = step - od.lag; ch = w - od.nch; }
+    return ri >= 0 && ri < od.rows;
+}
+
+// ---- service warp: what follows the sweep of one item ----
+template <int DT>
+__device__ void f_after_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int slot,
+                               int ri, int ch, int lane) {
+    // combine the 16 worker warps of this chunk in fp64
+    const float mP = lane < kFWarps ? sh.part_M[slot][0][lane] : kNoRef;
+    const float mQ = lane < kFWarps ? sh.part_M[slot][1][lane] : kNoRef;
+    const float MPc = warp_max(mP), MQc = warp_max(mQ);
+    double zP = lane < kFWarps ? static_cast<double>(sh.part_s[slot][0][lane]) * ref_scale(mP, MPc) : 0.0;
+    double zQ = lane < kFWarps ? static_cast<double>(sh.part_s[slot][1][lane]) * ref_scale(mQ, MQc) : 0.0;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) { zP += shfl_xor_d(zP, off); zQ += shfl_xor_d(zQ, off); }
+    if (lane == 0) {
+        RowZ z; z.MP = MPc; z.ZP = zP; z.MQ = MQc; z.ZQ = zQ;
+        fl.part[static_cast<size_t>(ri) * cx.nch + ch] = z;
+        __threadfence();
+        if (atomicAdd(&fl.row_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u) {
+            __threadfence();
+            f_row_complete<DT>(prm, fl, cx, ri / (cx.g + 1), ri % (cx.g + 1));
+        }
+    }
+    __syncwarp();
+}
 
 template <int DT>
-__global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params prm, const FlowScratch fl) {
+__device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int slot,
+                               const FlowDesc& d, int lane) {
+    constexpr int EPV = Raw<DT>::EPV;
+    const int g = cx.g, ri = d.ri, r = ri % (g + 1), b = ri / (g + 1);
+    const int nseg = cx.nch * kFWarps;
+    float* segs = fl.seg_tot + static_cast<size_t>(ri) * nseg;
+    if (lane < kFWarps) segs[d.ch * kFWarps + lane] = sh.part_s[slot][0][lane];
+    __threadfence();
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) last = atomicAdd(&fl.s2_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u;
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+
+    // ---------------- the position is complete: S_r and the candidate Y_r ----------------
+    __threadfence();
+    const bool have_q = d.have_q != 0;
+    const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
+    float w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w[j] = (4 * lane + j < nseg) ? __ldcg(&segs[4 * lane + j]) : 0.f;
+    double sd = (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
+                (static_cast<double>(w[2]) + static_cast<double>(w[3]));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
+    if (lane == 0 && have_q) fl.S[ri] = sd / __ldcg(&fl.rowZ[ri].ZQ);
+    const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
+    float inc = l4;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float o = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += o;
+    }
+    const float total = __shfl_sync(0xffffffffu, inc, 31);
+    int found = -1;
+    if (total > 0.f) {
+        const float t = uf * total;
+        float exc = __shfl_up_sync(0xffffffffu, inc, 1);
+        if (lane == 0) exc = 0.f;
+        const float p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+        // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
+        const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
+        const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
+        const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
+        const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
+        int e = 3; float bef = p3; int src;
+        if (hit) {
+            src = __ffs(hit) - 1;
+            if (h1) { e = 0; bef = exc; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
+        } else {
+            src = 31 - __clz(nz);
+            e = 0; bef = exc;
+            if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
+            else if (w[1] > 0.f) { e = 1; bef = p1; }
+        }
+        const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
+        const float before = __shfl_sync(0xffffffffu, bef, src);
+        int s0, s1;
+        chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1);
+        found = f_rescan<DT>(d.rowP, d.rowQ, s0, s1, lane, cx.kf, d.cp, d.nMP, d.nMQ, t - before);
+    } else if (have_q && r == 0 && total == 0.f) {
+        // empty residual at position 0 (P_0 and Q_0 coincide bit for bit): sample P_0 with the same
+        // uniform.  Two plain passes over the whole row by this warp: rare, so speed does not matter.
+        float tot = 0.f;
+        for (int base2 = 0; base2 < cx.units; base2 += 32) {
+            float vp[EPV], t2[EPV];
+            f_load_tail<DT>(d.rowP, base2 + lane, cx.units, vp);
+            tot += f_pair_sum<EPV, false>(vp, vp, cx.kf, 1.f, d.nMP, d.nMQ, t2);
+        }
+        tot = warp_sum(tot);
+        found = f_rescan<DT>(d.rowP, nullptr, 0, cx.units, lane, cx.kf, 1.f, d.nMP, d.nMQ, uf * tot);
+    }
+    if (lane == 0) {
+        fl.cand[ri] = found;
+        __threadfence();
+        if (atomicAdd(&fl.cand_cnt[b], 1u) == static_cast<unsigned>(g)) {
+            __threadfence();
+            f_finalize_block(prm, fl, b);
+        }
+    }
+    __syncwarp();
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Params prm, const FlowScratch fl) {
     using R = Raw<DT>;
     constexpr int EPV = R::EPV;
     constexpr size_t ESZ = (DT == kF32) ? 4 : 2;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ FlowShared sh;
-    // Each thread streams its own vectors through a private ring of 16-byte slots filled by
-    // cp.async, so loads run kFAhead steps ahead of the arithmetic without costing registers.
+    // Each worker thread streams its own vectors through a private ring of 16-byte slots filled
+    // by cp.async, so loads run kFAhead steps ahead of the arithmetic without costing registers.
     extern __shared__ __align__(16) unsigned char dyn[];
 
     FlowCtx cx;
@@ -328,65 +453,112 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
     cx.row_bytes = static_cast<size_t>(prm.V) * ESZ; cx.kf = prm.kf; cx.kd = prm.kd;
     const int g = cx.g;
     const float kf = cx.kf;
-    const unsigned total_items = static_cast<unsigned>(cx.B) * (g + 1) * cx.nch;   // of either kind
-    bool s1_left = true;
+    FlowOrder od;
+    od.rows = cx.B * (g + 1); od.nch = cx.nch; od.lag = fl.lag;
+    od.total = static_cast<unsigned>(od.rows + od.lag) * 2u * static_cast<unsigned>(od.nch);
 
-    for (;;) {
-        // ---------------- pick the next item (thread 0) ----------------
-        if (tid == 0) {
-            int kind = kExit, item = 0;
-            unsigned idle = 0;
-            for (;;) {
-                // a released sweep-2 item first: take one unit of the semaphore, then a slot
-                bool got = false;
-                if (static_cast<int>(ld_volatile(&fl.counters[kAvail])) > 0) {
-                    if (static_cast<int>(atomicSub(&fl.counters[kAvail], 1u)) > 0) got = true;
-                    else atomicAdd(&fl.counters[kAvail], 1u);       // lost the race: give it back
-                }
-                if (got) {
-                    const unsigned h = atomicAdd(&fl.counters[kHead], 1u);
-                    unsigned v, spins = 0;
-                    while ((v = ld_volatile(&fl.ready[h])) == 0u) {   // its writer is a few stores away
-                        if (++spins > (1u << 24)) { if (prm.status) atomicExch(prm.status, 1); break; }
-                    }
-                    if (v != 0u) { kind = kSweep2; item = static_cast<int>(v - 1u); }
-                    break;
-                }
-                if (s1_left) {
-                    const unsigned idx = atomicAdd(&fl.counters[kNext], 1u);
-                    if (idx < total_items) { kind = kSweep1; item = static_cast<int>(idx); break; }
-                    s1_left = false;
-                }
-                if (ld_volatile(&fl.counters[kHead]) >= total_items) break;   // every sweep-2 item is taken: done
-                __nanosleep(256);
-                if (++idle > (1u << 23)) { if (prm.status) atomicExch(prm.status, 1); break; }
-            }
-            sh.kind = kind; sh.item = item; sh.last = 0;
-            if (kind == kSweep2) {
-                __threadfence();
-                const int ri = item / cx.nch;
-                const RowZ z = load_rowz(&fl.rowZ[ri]);
-                sh.c = __ldcg(&fl.cscale[ri]);
-                sh.MP = static_cast<float>(z.MP);
-                sh.MQ = static_cast<float>(z.MQ);
-            }
+    if (tid == 0) {
+        for (int i = 0; i < kFDesc; ++i) {
+            mbar_init(smem_u32(&sh.full[i]), 1);
+            mbar_init(smem_u32(&sh.done[i]), kFWarps);
         }
-        __syncthreads();
-        const int kind = sh.kind, item = sh.item;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kFWarps) {
+        // =============================== service warp ===============================
+        // takes tickets, waits for what a sweep-2 item needs, hands descriptors to the workers,
+        // and does everything that follows a sweep, so that the workers never stop streaming
+        // a ticket decoded into a descriptor; never blocks
+        auto take = [&](FlowDesc& d) {
+            for (;;) {
+                unsigned t = 0;
+                if (lane == 0) t = atomicAdd(&fl.counters[0], 1u);
+                t = __shfl_sync(0xffffffffu, t, 0);
+                if (t >= od.total) { d.kind = kExit; return; }
+                int kind, ri, ch;
+                if (!f_decode(od, t, kind, ri, ch)) continue;
+                const int r = ri % (g + 1), b = ri / (g + 1);
+                d.kind = kind; d.ri = ri; d.ch = ch; d.have_q = r < g;
+                d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
+                d.rowQ = r < g ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
+                               : nullptr;
+                d.cp = 1.f; d.nMP = 0.f; d.nMQ = 0.f;
+                return;
+            }
+        };
+        // A sweep-2 item may start once its row has been folded into the recursion.  That is done
+        // by whoever completes the row, possibly this very warp a few items from now, which is why
+        // the warp never blocks here: it goes on with its own finished items and asks again.
+        auto ready = [&](FlowDesc& d) -> bool {
+            if (d.kind != kSweep2) return true;
+            unsigned rel = 0;
+            if (lane == 0) rel = ld_volatile(&fl.rel[d.ri]);
+            if (__shfl_sync(0xffffffffu, rel, 0) == 0u) return false;
+            __threadfence();
+            if (d.have_q) d.cp = __ldcg(&fl.cscale[d.ri]);
+            d.nMP = -static_cast<float>(__ldcg(&fl.rowZ[d.ri].MP));
+            d.nMQ = -static_cast<float>(__ldcg(&fl.rowZ[d.ri].MQ));
+            return true;
+        };
+        FlowDesc nd;
+        bool have_nd = false;
+        int q = 0, n = 0, qexit = -1;     // items published / post-processed; index of the exit descriptor
+        unsigned idle = 0;
+        for (;;) {
+            // 1. publish what can be published (a slot is free once its previous item is post-processed)
+            while (qexit < 0 && q - n < kFDesc) {
+                if (!have_nd) { take(nd); have_nd = true; }
+                if (!ready(nd)) break;
+                if (lane == 0) { sh.desc[q % kFDesc] = nd; mbar_arrive(smem_u32(&sh.full[q % kFDesc])); }
+                __syncwarp();
+                if (nd.kind == kExit) qexit = q;
+                ++q;
+                have_nd = false;
+            }
+            // 2. the oldest item in flight: wait for the workers, then do what follows its sweep
+            const int in_flight_end = qexit >= 0 ? qexit : q;
+            if (n < in_flight_end) {
+                const int slot = n % kFDesc;
+                const FlowDesc d = sh.desc[slot];
+                mbar_wait(smem_u32(&sh.done[slot]), static_cast<uint32_t>(n / kFDesc) & 1u, prm.status);
+                if (d.kind == kSweep1) f_after_sweep1<DT>(prm, fl, cx, sh, slot, d.ri, d.ch, lane);
+                else                   f_after_sweep2<DT>(prm, fl, cx, sh, slot, d, lane);
+                ++n;
+                idle = 0;
+                continue;
+            }
+            if (qexit >= 0) break;
+            // 3. nothing in flight and the next item waits for a row that another CTA completes
+            __nanosleep(128);
+            if (++idle > (1u << 23)) { if (prm.status) atomicExch(prm.status, 1); break; }
+        }
+        if (qexit < 0) {      // gave up: release the workers
+            if (lane == 0) { sh.desc[q % kFDesc].kind = kExit; mbar_arrive(smem_u32(&sh.full[q % kFDesc])); }
+        }
+        return;
+    }
+
+    // =============================== worker warps ===============================
+    constexpr uint32_t kSlot = kFThreads * 16;               // bytes between consecutive ring slots
+    const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;
+    for (int n = 0;; ++n) {
+        const int slot = n % kFDesc;
+        const uint32_t parity = static_cast<uint32_t>(n / kFDesc) & 1u;
+        mbar_wait(smem_u32(&sh.full[slot]), parity, prm.status);
+        const int kind = sh.desc[slot].kind;
         if (kind == kExit) break;
-        const int ch = item % cx.nch, ri = item / cx.nch, r = ri % (g + 1), b = ri / (g + 1);
-        const bool have_q = r < g;
-        const char* rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
-        const char* rowQ = have_q ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
-                                  : nullptr;
+        const int ch = sh.desc[slot].ch;
+        const bool have_q = sh.desc[slot].have_q != 0;
+        const char* rowP = sh.desc[slot].rowP;
+        const char* rowQ = sh.desc[slot].rowQ;
         int w0, w1;
         chunk_range(cx, ch, warp, w0, w1);
 
         // This warp's segment: nfull steps in which every lane has a vector (streamed through the
         // ring) and at most one partial step (loaded directly; lanes past the end see -inf logits).
         const int nv = w1 - w0, nfull = nv >> 5;
-        constexpr uint32_t kSlot = kFThreads * 16;           // bytes between consecutive ring slots
-        const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;
         const char* gP = rowP + static_cast<size_t>(w0 + lane) * 16;
         const char* gQ = have_q ? rowQ + static_cast<size_t>(w0 + lane) * 16 : gP;
         auto fetch_step = [&](int k, int j) {                // step k goes to slots 2j, 2j+1 (j = k & 3)
@@ -401,7 +573,7 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
         const int itail = w0 + 32 * nfull + lane;            // this lane's vector in the partial step
 
         if (kind == kSweep1) {
-            // ---------------- sweep 1 over this chunk ----------------
+            // ---------------- sweep 1 over this warp's segment ----------------
             float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
             auto step1 = [&](const float (&vp)[EPV], const float (&vq)[EPV], bool first) {
                 if (first) {                                 // references from the first vector of every lane
@@ -434,33 +606,12 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
             sP = warp_sum(sP);
             sQ = warp_sum(sQ);
             if (lane == 0) {
-                sh.red_M[0][warp] = MPw; sh.red_s[0][warp] = sP;
-                sh.red_M[1][warp] = MQw; sh.red_s[1][warp] = sQ;
-            }
-            __syncthreads();
-            if (warp == 0) {
-                // combine the 16 warps of this chunk in fp64
-                const float mP = lane < kFWarps ? sh.red_M[0][lane] : kNoRef;
-                const float mQ = lane < kFWarps ? sh.red_M[1][lane] : kNoRef;
-                const float MPc = warp_max(mP), MQc = warp_max(mQ);
-                double zP = lane < kFWarps ? static_cast<double>(sh.red_s[0][lane]) * ref_scale(mP, MPc) : 0.0;
-                double zQ = lane < kFWarps ? static_cast<double>(sh.red_s[1][lane]) * ref_scale(mQ, MQc) : 0.0;
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) { zP += shfl_xor_d(zP, off); zQ += shfl_xor_d(zQ, off); }
-                if (lane == 0) {
-                    RowZ z; z.MP = MPc; z.ZP = zP; z.MQ = MQc; z.ZQ = zQ;
-                    fl.part[item] = z;
-                    __threadfence();
-                    if (atomicAdd(&fl.row_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u) {
-                        __threadfence();
-                        f_row_complete<DT>(prm, fl, cx, b, r);
-                    }
-                }
+                sh.part_M[slot][0][warp] = MPw; sh.part_s[slot][0][warp] = sP;
+                sh.part_M[slot][1][warp] = MQw; sh.part_s[slot][1][warp] = sQ;
             }
         } else {
-            // ---------------- sweep 2 over this chunk ----------------
-            const float cp = have_q ? sh.c : 1.f;
-            const float nMP = -sh.MP, nMQ = -sh.MQ;
+            // ---------------- sweep 2 over this warp's segment ----------------
+            const float cp = sh.desc[slot].cp, nMP = sh.desc[slot].nMP, nMQ = sh.desc[slot].nMQ;
             float acc = 0.f;
             for (int kb = 0; kb < nfull; kb += kFAhead) {
 #pragma unroll
@@ -488,130 +639,11 @@ __global__ void __launch_bounds__(kFThreads, 2) verify_flow_kernel(const Params 
                               : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, t);
             }
             acc = warp_sum(acc);
-            if (lane == 0) fl.seg_tot[static_cast<size_t>(ri) * (cx.nch * kFWarps) + ch * kFWarps + warp] = acc;
-            __threadfence();
-            __syncthreads();
-            if (tid == 0) {
-                __threadfence();
-                sh.last = atomicAdd(&fl.s2_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u;
-            }
-            __syncthreads();
-            if (sh.last) {
-                // ---------------- the position is complete: S_r and the candidate Y_r ----------------
-                __threadfence();
-                const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
-                if (warp == 0) {
-                    const int nseg = cx.nch * kFWarps;
-                    const float* segs = fl.seg_tot + static_cast<size_t>(ri) * nseg;
-                    float w[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) w[j] = (4 * lane + j < nseg) ? __ldcg(&segs[4 * lane + j]) : 0.f;
-                    double sd = (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
-                                (static_cast<double>(w[2]) + static_cast<double>(w[3]));
-#pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
-                    if (lane == 0 && have_q) fl.S[ri] = sd / __ldcg(&fl.rowZ[ri].ZQ);
-                    const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
-                    float inc = l4;
-#pragma unroll
-                    for (int off = 1; off < 32; off <<= 1) {
-                        const float o = __shfl_up_sync(0xffffffffu, inc, off);
-                        if (lane >= off) inc += o;
-                    }
-                    const float total = __shfl_sync(0xffffffffu, inc, 31);
-                    int sel = -1;
-                    float before = 0.f;
-                    if (total > 0.f) {
-                        const float t = uf * total;
-                        float exc = __shfl_up_sync(0xffffffffu, inc, 1);
-                        if (lane == 0) exc = 0.f;
-                        const float p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
-                        // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
-                        const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
-                        const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
-                        const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
-                        const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
-                        int e = 3; float bef = p3; int src;
-                        if (hit) {
-                            src = __ffs(hit) - 1;
-                            if (h1) { e = 0; bef = exc; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
-                        } else {
-                            src = 31 - __clz(nz);
-                            e = 0; bef = exc;
-                            if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
-                            else if (w[1] > 0.f) { e = 1; bef = p1; }
-                        }
-                        sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
-                        before = t - __shfl_sync(0xffffffffu, bef, src);    // target inside the segment
-                    } else if (have_q && r == 0 && total == 0.f) {
-                        sel = -2;   // empty residual at position 0: handled below
-                    }
-                    if (lane == 0) { sh.sel = sel; sh.target = before; sh.found = -1; }
-                }
-                __syncthreads();
-                const int sel = sh.sel;
-                if (sel >= 0) {
-                    // the segment that holds the target, cut into one piece per warp: piece totals,
-                    // then only the piece that holds the target is walked element by element
-                    int s0, s1;
-                    chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1);
-                    const int q0 = s0 + static_cast<int>(static_cast<long long>(s1 - s0) * warp / kFWarps);
-                    const int q1 = s0 + static_cast<int>(static_cast<long long>(s1 - s0) * (warp + 1) / kFWarps);
-                    float sub = 0.f;
-                    for (int base2 = q0; base2 < q1; base2 += 32) {
-                        float vp[EPV], vq[EPV], t2[EPV];
-                        f_load_tail<DT>(rowP, base2 + lane, q1, vp);
-                        f_load_tail<DT>(rowQ, base2 + lane, q1, vq);
-                        sub += have_q ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, t2)
-                                      : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, t2);
-                    }
-                    sub = warp_sum(sub);
-                    if (lane == 0) sh.red_s[0][warp] = sub;
-                    __syncthreads();
-                    const float mine = lane < kFWarps ? sh.red_s[0][lane] : 0.f;
-                    float incp = mine;
-#pragma unroll
-                    for (int off = 1; off < 32; off <<= 1) {
-                        const float o = __shfl_up_sync(0xffffffffu, incp, off);
-                        if (lane >= off) incp += o;
-                    }
-                    const float tgt = sh.target;
-                    const unsigned hitp = __ballot_sync(0xffffffffu, incp > tgt && mine > 0.f);
-                    const unsigned nzp = __ballot_sync(0xffffffffu, mine > 0.f);
-                    const int piece = hitp ? __ffs(hitp) - 1 : (nzp ? 31 - __clz(nzp) : -1);
-                    if (piece == warp) {
-                        const float befp = __shfl_sync(0xffffffffu, incp - mine, piece);
-                        const int y = f_rescan<DT>(rowP, rowQ, q0, q1, lane, kf, cp, nMP, nMQ, tgt - befp);
-                        if (lane == 0) sh.found = y;
-                    }
-                    __syncthreads();
-                } else if (sel == -2 && warp == 0) {
-                    // sample P_0 with the same uniform: two plain passes over the whole row by one
-                    // warp (rare: P_0 and Q_0 coincide bit for bit), so speed does not matter
-                    float tot = 0.f;
-                    for (int base2 = 0; base2 < cx.units; base2 += 32) {
-                        float vp[EPV], vq[EPV], t2[EPV];
-                        f_load_tail<DT>(rowP, base2 + lane, cx.units, vp);
-                        f_load_tail<DT>(nullptr, 0, 0, vq);
-                        tot += f_pair_sum<EPV, false>(vp, vq, kf, 1.f, nMP, nMQ, t2);
-                    }
-                    tot = warp_sum(tot);
-                    const int y = f_rescan<DT>(rowP, nullptr, 0, cx.units, lane, kf, 1.f, nMP, nMQ, uf * tot);
-                    if (lane == 0) sh.found = y;
-                }
-                if (sel == -2) __syncthreads();
-                if (tid == 0) {
-                    fl.cand[ri] = sh.found;
-                    __threadfence();
-                    if (atomicAdd(&fl.cand_cnt[b], 1u) == static_cast<unsigned>(g)) {
-                        __threadfence();
-                        f_finalize_block(prm, fl, b);
-                    }
-                }
-            }
+            if (lane == 0) sh.part_s[slot][0][warp] = acc;
         }
         cp_async_wait<0>();
-        __syncthreads();   // shared scratch is reused by the next item
+        if (lane == 0) mbar_arrive(smem_u32(&sh.done[slot]));   // releases this warp's partials and the descriptor
+        __syncwarp();
     }
 }
 
@@ -626,7 +658,7 @@ size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes) {
     z += up256(kCounterWords * sizeof(unsigned));   // counters
     z += 3 * up256(rows * sizeof(unsigned));        // row_cnt, row_done, s2_cnt
     z += 4 * up256(static_cast<size_t>(B) * sizeof(unsigned));   // cand_cnt, chain, lock, bad
-    z += up256(rows * nch * sizeof(unsigned));      // ready
+    z += up256(rows * sizeof(unsigned));            // rel
     if (zero_bytes) *zero_bytes = z;
     size_t n = z;
     n += up256(rows * nch * sizeof(RowZ));          // part
@@ -652,7 +684,7 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl)
     fl->chain = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->lock = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->bad = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
-    fl->ready = reinterpret_cast<unsigned*>(take(rows * nch * sizeof(unsigned)));
+    fl->rel = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->part = reinterpret_cast<RowZ*>(take(rows * nch * sizeof(RowZ)));
     fl->rowZ = reinterpret_cast<RowZ*>(take(rows * sizeof(RowZ)));
     fl->pchain = reinterpret_cast<double*>(take(static_cast<size_t>(B) * (gamma + 2) * sizeof(double)));
@@ -663,6 +695,7 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl)
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
     fl->nch = nch;
+    fl->lag = 0;
 }
 
 // Chunks per row.  An item should be large next to what it costs to hand it out (about
@@ -684,6 +717,8 @@ static FKernelFn pick_flow(int dtype) {
 
 static constexpr size_t kFlowSmem = sizeof(uint4) * kFDepth * kFThreads;
 
+int flow_threads() { return kFAllThreads; }
+
 int flow_max_ctas_per_sm(int dtype) {
     int n = 0;
     if (cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_flow(dtype)),
@@ -691,15 +726,22 @@ int flow_max_ctas_per_sm(int dtype) {
         cudaGetLastError();
         return 0;
     }
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_flow(dtype), kFThreads, kFlowSmem) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_flow(dtype), kFAllThreads, kFlowSmem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
     return n;
 }
 
-cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream) {
-    pick_flow(dtype)<<<nctas, kFThreads, kFlowSmem, stream>>>(prm, fl);
+cudaError_t launch_flow(const Params& prm, const FlowScratch& fl_in, int dtype, int nctas, cudaStream_t stream) {
+    FlowScratch fl = fl_in;
+    if (fl.lag <= 0) {
+        // sweep-2 items trail by about the rows that are in flight at once (every CTA holds up
+        // to kFDesc items, half of them sweep-1), so that they rarely have to wait and the rows
+        // they re-read are still in L2
+        fl.lag = (nctas * kFDesc) / (2 * fl.nch) + 2;
+    }
+    pick_flow(dtype)<<<nctas, kFAllThreads, kFlowSmem, stream>>>(prm, fl);
     return cudaGetLastError();
 }
 

@@ -25,7 +25,7 @@ cudaError_t launch_cluster(const Params& prm, int algo, int dtype, int cluster, 
 // when the kernel starts.
 struct RowZ { double MP, ZP, MQ, ZQ; };   // row (or chunk) references and sums of 2^{z k - M}
 struct FlowScratch {
-    unsigned* counters;   // next sweep-1 item, semaphore of released items, ready head, ready tail
+    unsigned* counters;   // [0]: ticket counter of the item order
     unsigned* row_cnt;    // [B (gamma+1)] sweep-1 chunks finished per row
     unsigned* row_done;   // [B (gamma+1)] row normalisers published
     unsigned* s2_cnt;     // [B (gamma+1)] sweep-2 chunks finished per position
@@ -33,7 +33,7 @@ struct FlowScratch {
     unsigned* chain;      // [B] rows folded into the recursion
     unsigned* lock;       // [B]
     unsigned* bad;        // [B] data fault seen
-    unsigned* ready;      // [B (gamma+1) nch] released sweep-2 items (+1; 0 = not written yet)
+    unsigned* rel;        // [B (gamma+1)] row folded into the recursion: its sweep-2 items may run
     RowZ* part;           // [B (gamma+1) nch]
     RowZ* rowZ;           // [B (gamma+1)]
     double* pchain;       // [B (gamma+2)]
@@ -43,7 +43,8 @@ struct FlowScratch {
     float* seg_tot;       // [B (gamma+1) nch 16]
     double* S;            // [B (gamma+1)]
     int* cand;            // [B (gamma+1)]
-    int nch;
+    int nch;              // chunks per row
+    int lag;              // rows by which sweep-2 items trail sweep-1 items in the item order
 };
 size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes);
 void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl);
