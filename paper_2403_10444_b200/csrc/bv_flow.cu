@@ -309,8 +309,11 @@ struct FlowDesc {
     float cp, nMP, nMQ;         // sweep 2: p_r Z_Q / Z_P and minus the row references
 };
 
+constexpr int kFDefer = 8;     // sweep-2 items a CTA may set aside while their row is not folded yet
+
 struct FlowShared {
     FlowDesc desc[kFDesc];
+    FlowDesc defer[kFDefer];
     unsigned long long full[kFDesc];    // the service warp has filled desc[i]
     unsigned long long done[kFDesc];    // all 16 worker warps have left their partials of desc[i]
     float part_M[kFDesc][2][kFWarps];   // sweep 1: references of P and Q per worker warp
@@ -489,33 +492,67 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             }
         };
         // A sweep-2 item may start once its row has been folded into the recursion.  That is done
-        // by whoever completes the row, possibly this very warp a few items from now, which is why
-        // the warp never blocks here: it goes on with its own finished items and asks again.
-        auto ready = [&](FlowDesc& d) -> bool {
-            if (d.kind != kSweep2) return true;
-            unsigned rel = 0;
-            if (lane == 0) rel = ld_volatile(&fl.rel[d.ri]);
-            if (__shfl_sync(0xffffffffu, rel, 0) == 0u) return false;
+        // by whoever completes the row, possibly this very warp a few items from now, so the warp
+        // never blocks on it: an item that is not ready is set aside, later tickets go first, and
+        // the items set aside are asked about again on every round (all of them with one load each,
+        // side by side in the lanes).
+        auto fill_scalars = [&](FlowDesc& d) {
             __threadfence();
             if (d.have_q) d.cp = __ldcg(&fl.cscale[d.ri]);
             d.nMP = -static_cast<float>(__ldcg(&fl.rowZ[d.ri].MP));
             d.nMQ = -static_cast<float>(__ldcg(&fl.rowZ[d.ri].MQ));
-            return true;
         };
-        FlowDesc nd;
-        bool have_nd = false;
+        auto publish = [&](const FlowDesc& d, int q) {
+            if (lane == 0) { sh.desc[q % kFDesc] = d; mbar_arrive(smem_u32(&sh.full[q % kFDesc])); }
+            __syncwarp();
+        };
         int q = 0, n = 0, qexit = -1;     // items published / post-processed; index of the exit descriptor
+        int ndef = 0;                     // items set aside
+        bool exhausted = false;           // the ticket counter has run past the last item
         unsigned idle = 0;
         for (;;) {
             // 1. publish what can be published (a slot is free once its previous item is post-processed)
             while (qexit < 0 && q - n < kFDesc) {
-                if (!have_nd) { take(nd); have_nd = true; }
-                if (!ready(nd)) break;
-                if (lane == 0) { sh.desc[q % kFDesc] = nd; mbar_arrive(smem_u32(&sh.full[q % kFDesc])); }
-                __syncwarp();
-                if (nd.kind == kExit) qexit = q;
-                ++q;
-                have_nd = false;
+                // (a) the oldest item set aside whose row has been folded meanwhile
+                unsigned rel = 0;
+                if (lane < ndef) rel = ld_volatile(&fl.rel[sh.defer[lane].ri]);
+                const unsigned okmask = __ballot_sync(0xffffffffu, rel != 0u);
+                if (okmask) {
+                    const int i = __ffs(okmask) - 1;
+                    FlowDesc d = sh.defer[i];
+                    fill_scalars(d);
+                    __syncwarp();
+                    if (lane == 0) for (int j = i; j + 1 < ndef; ++j) sh.defer[j] = sh.defer[j + 1];
+                    --ndef;
+                    __syncwarp();
+                    publish(d, q);
+                    ++q;
+                    continue;
+                }
+                // (b) a new ticket
+                if (exhausted) {
+                    if (ndef == 0) { FlowDesc d; d.kind = kExit; publish(d, q); qexit = q; ++q; }
+                    break;
+                }
+                if (ndef == kFDefer) break;      // enough set aside: wait for one of them
+                FlowDesc d;
+                take(d);
+                if (d.kind == kExit) { exhausted = true; continue; }
+                bool ok = true;
+                if (d.kind == kSweep2) {
+                    unsigned r1 = 0;
+                    if (lane == 0) r1 = ld_volatile(&fl.rel[d.ri]);
+                    ok = __shfl_sync(0xffffffffu, r1, 0) != 0u;
+                }
+                if (ok) {
+                    if (d.kind == kSweep2) fill_scalars(d);
+                    publish(d, q);
+                    ++q;
+                } else {
+                    if (lane == 0) sh.defer[ndef] = d;
+                    ++ndef;
+                    __syncwarp();
+                }
             }
             // 2. the oldest item in flight: wait for the workers, then do what follows its sweep
             const int in_flight_end = qexit >= 0 ? qexit : q;
@@ -535,7 +572,8 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             if (++idle > (1u << 23)) { if (prm.status) atomicExch(prm.status, 1); break; }
         }
         if (qexit < 0) {      // gave up: release the workers
-            if (lane == 0) { sh.desc[q % kFDesc].kind = kExit; mbar_arrive(smem_u32(&sh.full[q % kFDesc])); }
+            FlowDesc d; d.kind = kExit;
+            publish(d, q);
         }
         return;
     }
