@@ -259,6 +259,15 @@ __device__ __forceinline__ void ring_fetch(void* slot, const void* src, bool pre
 __device__ __forceinline__ void cp_async16_s(uint32_t saddr, const void* gmem) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(gmem) : "memory");
 }
+// One ring item given by shared-space address: a 16-byte asynchronous copy when `pred`,
+// else the slot is filled with `fill` (the bit pattern of -inf logits).  No commit.
+__device__ __forceinline__ void ring_fetch_s(uint32_t saddr, const void* src, bool pred, uint32_t fill) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t"
+        "@p cp.async.cg.shared.global [%0], [%1], 16;\n\t"
+        "@!p st.shared.v4.b32 [%0], {%3, %3, %3, %3};\n\t}"
+        ::"r"(saddr), "l"(src), "r"(static_cast<int>(pred)), "r"(fill) : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t saddr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr) : "memory");

@@ -440,6 +440,81 @@ __device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const F
     __syncwarp();
 }
 
+// ---- worker warps: one warp's segment of one item ----
+// The segment's vectors go through the thread's private ring, kFAhead steps ahead of the
+// arithmetic.  A step is one vector per lane of each row; the last step may be partial, and
+// lanes past the end then find -inf logits in their slots.
+template <int DT, bool HAVEQ, int KIND>
+__device__ __forceinline__ void f_sweep_segment(uint32_t sb, const char* rowP, const char* rowQ, int w0, int w1,
+                                                int lane, float kf, float cp, float nMP, float nMQ,
+                                                float& oMP, float& osP, float& oMQ, float& osQ) {
+    using R = Raw<DT>;
+    constexpr int EPV = R::EPV;
+    constexpr uint32_t kSlot = kFThreads * 16;               // bytes between consecutive ring slots
+    const int nv = w1 - w0;
+    const int nsteps = (nv + 31) >> 5;
+    const int nlast = nv - 32 * (nsteps - 1);                // lanes that take part in the last step
+    const char* gP = rowP + static_cast<size_t>(w0 + lane) * 16;
+    const char* gQ = HAVEQ ? rowQ + static_cast<size_t>(w0 + lane) * 16 : gP;
+    auto fetch_step = [&](int k, int j) {                    // step k goes to slots 2j, 2j+1 (j = k & 3)
+        if (k < nsteps) {
+            const bool ok = (k + 1 < nsteps) || lane < nlast;
+            ring_fetch_s(sb + (2 * j) * kSlot, gP + static_cast<size_t>(k) * 512, ok, R::kNegInf);
+            if (HAVEQ) ring_fetch_s(sb + (2 * j + 1) * kSlot, gQ + static_cast<size_t>(k) * 512, ok, R::kNegInf);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int j = 0; j < kFAhead; ++j) fetch_step(j, j);
+
+    float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f, acc = 0.f;
+    for (int kb = 0; kb < nsteps; kb += kFAhead) {
+#pragma unroll
+        for (int j = 0; j < kFAhead; ++j) {
+            const int k = kb + j;
+            if (k < nsteps) {
+                cp_async_wait<kFAhead - 1>();                // step k of both rows has landed
+                float vp[EPV], vq[EPV];
+                R::unpack(lds128(sb + (2 * j) * kSlot), vp);
+                if (HAVEQ) R::unpack(lds128(sb + (2 * j + 1) * kSlot), vq);
+                if (KIND == kSweep1) {
+                    if (j == 0 && kb == 0) {                 // references from the first vector of every lane
+                        MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
+                        if (HAVEQ) MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vq)) * kf), kNoRef);
+                    }
+                    float vsP = f_exp_sum<EPV>(vp, kf, -MPw);
+                    float vsQ = HAVEQ ? f_exp_sum<EPV>(vq, kf, -MQw) : 0.f;
+                    if (__any_sync(0xffffffffu, fmaxf(vsP, vsQ) > kRaiseBound)) {   // a logit above a reference
+                        if (__any_sync(0xffffffffu, vsP > kRaiseBound)) {
+                            const float y = rintf(warp_max(vec_max<EPV>(vp)) * kf);
+                            if (y > MPw) { sP *= ref_scale(MPw, y); MPw = y; }
+                            vsP = f_exp_sum<EPV>(vp, kf, -MPw);
+                        }
+                        if (HAVEQ && __any_sync(0xffffffffu, vsQ > kRaiseBound)) {
+                            const float y = rintf(warp_max(vec_max<EPV>(vq)) * kf);
+                            if (y > MQw) { sQ *= ref_scale(MQw, y); MQw = y; }
+                            vsQ = f_exp_sum<EPV>(vq, kf, -MQw);
+                        }
+                    }
+                    sP += vsP;
+                    sQ += vsQ;
+                } else {
+                    float t[EPV];
+                    acc += f_pair_sum<EPV, HAVEQ>(vp, vq, kf, cp, nMP, nMQ, t);
+                }
+                fetch_step(k + kFAhead, j);
+            }
+        }
+    }
+    cp_async_wait<0>();
+    if (KIND == kSweep1) {
+        oMP = MPw; osP = warp_sum(sP);
+        oMQ = MQw; osQ = HAVEQ ? warp_sum(sQ) : 0.f;
+    } else {
+        osP = warp_sum(acc);
+    }
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Params prm, const FlowScratch fl) {
     using R = Raw<DT>;
@@ -579,107 +654,32 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     }
 
     // =============================== worker warps ===============================
-    constexpr uint32_t kSlot = kFThreads * 16;               // bytes between consecutive ring slots
-    const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;
+    const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;   // this thread's ring slot 0
     for (int n = 0;; ++n) {
         const int slot = n % kFDesc;
         const uint32_t parity = static_cast<uint32_t>(n / kFDesc) & 1u;
         mbar_wait(smem_u32(&sh.full[slot]), parity, prm.status);
         const int kind = sh.desc[slot].kind;
         if (kind == kExit) break;
-        const int ch = sh.desc[slot].ch;
         const bool have_q = sh.desc[slot].have_q != 0;
         const char* rowP = sh.desc[slot].rowP;
         const char* rowQ = sh.desc[slot].rowQ;
         int w0, w1;
-        chunk_range(cx, ch, warp, w0, w1);
-
-        // This warp's segment: nfull steps in which every lane has a vector (streamed through the
-        // ring) and at most one partial step (loaded directly; lanes past the end see -inf logits).
-        const int nv = w1 - w0, nfull = nv >> 5;
-        const char* gP = rowP + static_cast<size_t>(w0 + lane) * 16;
-        const char* gQ = have_q ? rowQ + static_cast<size_t>(w0 + lane) * 16 : gP;
-        auto fetch_step = [&](int k, int j) {                // step k goes to slots 2j, 2j+1 (j = k & 3)
-            if (k < nfull) {
-                cp_async16_s(sb + (2 * j) * kSlot, gP + static_cast<size_t>(k) * 512);
-                if (have_q) cp_async16_s(sb + (2 * j + 1) * kSlot, gQ + static_cast<size_t>(k) * 512);
-            }
-            cp_async_commit();
-        };
-#pragma unroll
-        for (int j = 0; j < kFAhead; ++j) fetch_step(j, j);
-        const int itail = w0 + 32 * nfull + lane;            // this lane's vector in the partial step
-
+        chunk_range(cx, sh.desc[slot].ch, warp, w0, w1);
+        float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
         if (kind == kSweep1) {
-            // ---------------- sweep 1 over this warp's segment ----------------
-            float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
-            auto step1 = [&](const float (&vp)[EPV], const float (&vq)[EPV], bool first) {
-                if (first) {                                 // references from the first vector of every lane
-                    MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
-                    if (have_q) MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vq)) * kf), kNoRef);
-                }
-                f_accumulate<EPV>(vp, kf, MPw, sP);
-                if (have_q) f_accumulate<EPV>(vq, kf, MQw, sQ);
-            };
-            for (int kb = 0; kb < nfull; kb += kFAhead) {
-#pragma unroll
-                for (int j = 0; j < kFAhead; ++j) {
-                    const int k = kb + j;
-                    if (k < nfull) {
-                        cp_async_wait<kFAhead - 1>();        // step k of both rows has landed
-                        float vp[EPV], vq[EPV];
-                        R::unpack(lds128(sb + (2 * j) * kSlot), vp);
-                        if (have_q) R::unpack(lds128(sb + (2 * j + 1) * kSlot), vq);
-                        step1(vp, vq, k == 0);
-                        fetch_step(k + kFAhead, j);
-                    }
-                }
-            }
-            if (nv & 31) {
-                float vp[EPV], vq[EPV];
-                f_load_tail<DT>(rowP, itail, w1, vp);
-                f_load_tail<DT>(rowQ, itail, w1, vq);
-                step1(vp, vq, nfull == 0);
-            }
-            sP = warp_sum(sP);
-            sQ = warp_sum(sQ);
+            if (have_q) f_sweep_segment<DT, true, kSweep1>(sb, rowP, rowQ, w0, w1, lane, kf, 1.f, 0.f, 0.f, MPw, sP, MQw, sQ);
+            else        f_sweep_segment<DT, false, kSweep1>(sb, rowP, rowQ, w0, w1, lane, kf, 1.f, 0.f, 0.f, MPw, sP, MQw, sQ);
             if (lane == 0) {
                 sh.part_M[slot][0][warp] = MPw; sh.part_s[slot][0][warp] = sP;
                 sh.part_M[slot][1][warp] = MQw; sh.part_s[slot][1][warp] = sQ;
             }
         } else {
-            // ---------------- sweep 2 over this warp's segment ----------------
             const float cp = sh.desc[slot].cp, nMP = sh.desc[slot].nMP, nMQ = sh.desc[slot].nMQ;
-            float acc = 0.f;
-            for (int kb = 0; kb < nfull; kb += kFAhead) {
-#pragma unroll
-                for (int j = 0; j < kFAhead; ++j) {
-                    const int k = kb + j;
-                    if (k < nfull) {
-                        cp_async_wait<kFAhead - 1>();
-                        float vp[EPV], vq[EPV], t[EPV];
-                        R::unpack(lds128(sb + (2 * j) * kSlot), vp);
-                        if (have_q) {
-                            R::unpack(lds128(sb + (2 * j + 1) * kSlot), vq);
-                            acc += f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, t);
-                        } else {
-                            acc += f_pair_sum<EPV, false>(vp, vp, kf, cp, nMP, nMQ, t);
-                        }
-                        fetch_step(k + kFAhead, j);
-                    }
-                }
-            }
-            if (nv & 31) {
-                float vp[EPV], vq[EPV], t[EPV];
-                f_load_tail<DT>(rowP, itail, w1, vp);
-                f_load_tail<DT>(rowQ, itail, w1, vq);
-                acc += have_q ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, t)
-                              : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, t);
-            }
-            acc = warp_sum(acc);
-            if (lane == 0) sh.part_s[slot][0][warp] = acc;
+            if (have_q) f_sweep_segment<DT, true, kSweep2>(sb, rowP, rowQ, w0, w1, lane, kf, cp, nMP, nMQ, MPw, sP, MQw, sQ);
+            else        f_sweep_segment<DT, false, kSweep2>(sb, rowP, rowQ, w0, w1, lane, kf, cp, nMP, nMQ, MPw, sP, MQw, sQ);
+            if (lane == 0) sh.part_s[slot][0][warp] = sP;
         }
-        cp_async_wait<0>();
         if (lane == 0) mbar_arrive(smem_u32(&sh.done[slot]));   // releases this warp's partials and the descriptor
         __syncwarp();
     }
