@@ -163,10 +163,6 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             }
             bv::FlowScratch fl;
             bv::flow_scratch_layout(d->flow_ws[slot], B, gamma, nch, &fl);
-            if (const char* env = std::getenv("BV_FLOW_LAG")) {
-                const int v = std::atoi(env);
-                if (v >= 1) fl.lag = v;
-            }
             cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
             if (e != cudaSuccess) return cuda_fail(e);
             long long items = static_cast<long long>(B) * (gamma + 1) * nch;

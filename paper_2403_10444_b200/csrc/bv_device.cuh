@@ -268,6 +268,26 @@ __device__ __forceinline__ void ring_fetch_s(uint32_t saddr, const void* src, bo
         "@!p st.shared.v4.b32 [%0], {%3, %3, %3, %3};\n\t}"
         ::"r"(saddr), "l"(src), "r"(static_cast<int>(pred)), "r"(fill) : "memory");
 }
+// L2 eviction-priority policies: rows streamed by the first sweep should outlive the traffic
+// that passes before their second sweep; rows read by the second sweep are dead afterwards.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+// ring item with an L2 policy (see ring_fetch_s)
+__device__ __forceinline__ void ring_fetch_hint(uint32_t saddr, const void* src, bool pred, uint32_t fill, uint64_t pol) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t"
+        "@p cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %4;\n\t"
+        "@!p st.shared.v4.b32 [%0], {%3, %3, %3, %3};\n\t}"
+        ::"r"(saddr), "l"(src), "r"(static_cast<int>(pred)), "r"(fill), "l"(pol) : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t saddr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr) : "memory");

@@ -309,7 +309,7 @@ struct FlowDesc {
     float cp, nMP, nMQ;         // sweep 2: p_r Z_Q / Z_P and minus the row references
 };
 
-constexpr int kFDefer = 8;     // sweep-2 items a CTA may set aside while their row is not folded yet
+constexpr int kFDefer = 8;     // chunks a CTA may hold between their first and their second sweep
 
 struct FlowShared {
     FlowDesc desc[kFDesc];
@@ -320,18 +320,10 @@ struct FlowShared {
     float part_s[kFDesc][2][kFWarps];   // sweep 1: sums; sweep 2: [0] holds the residual totals
 };
 
-// Items are handed out in one fixed order by a single ticket counter: step n carries the
-// sweep-1 chunks of row n and then the sweep-2 chunks of row n - lag.  Everything an item
-// waits for therefore has a smaller ticket, so whoever holds it is already running.
-struct FlowOrder { int rows, nch, lag; unsigned total; };
-
-__device__ __forceinline__ bool f_decode(const FlowOrder& od, unsigned t, int& kind, int& ri, int& ch) {
-    const int step = static_cast<int>(t / (2u * od.nch)), w = static_cast<int>(t % (2u * od.nch));
-    if (w < od.nch) { kind = kSweep1; ri = step; ch = w; }
-    else            { kind = kSweep2; ri = step - od.lag; ch = w - od.nch; }
-    return ri >= 0 && ri < od.rows;
-}
-
+// Sweep-1 items are handed out in row order by a single ticket counter.  A CTA keeps the chunks
+// it has swept in a short list and runs the second sweep of each of them itself, as soon as the
+// chunk's row has been folded into the recursion: the re-read follows the first read as closely
+// as the dependency allows, so the rows are still in L2.
 // ---- service warp: what follows the sweep of one item ----
 template <int DT>
 __device__ void f_after_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int slot,
@@ -456,11 +448,13 @@ __device__ __forceinline__ void f_sweep_segment(uint32_t sb, const char* rowP, c
     const int nlast = nv - 32 * (nsteps - 1);                // lanes that take part in the last step
     const char* gP = rowP + static_cast<size_t>(w0 + lane) * 16;
     const char* gQ = HAVEQ ? rowQ + static_cast<size_t>(w0 + lane) * 16 : gP;
+    // sweep 1 asks L2 to keep the rows (they are read again soon); sweep 2 marks them as done with
+    const uint64_t pol = KIND == kSweep1 ? l2_policy_evict_last() : l2_policy_evict_first();
     auto fetch_step = [&](int k, int j) {                    // step k goes to slots 2j, 2j+1 (j = k & 3)
         if (k < nsteps) {
             const bool ok = (k + 1 < nsteps) || lane < nlast;
-            ring_fetch_s(sb + (2 * j) * kSlot, gP + static_cast<size_t>(k) * 512, ok, R::kNegInf);
-            if (HAVEQ) ring_fetch_s(sb + (2 * j + 1) * kSlot, gQ + static_cast<size_t>(k) * 512, ok, R::kNegInf);
+            ring_fetch_hint(sb + (2 * j) * kSlot, gP + static_cast<size_t>(k) * 512, ok, R::kNegInf, pol);
+            if (HAVEQ) ring_fetch_hint(sb + (2 * j + 1) * kSlot, gQ + static_cast<size_t>(k) * 512, ok, R::kNegInf, pol);
         }
         cp_async_commit();
     };
@@ -531,9 +525,6 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     cx.row_bytes = static_cast<size_t>(prm.V) * ESZ; cx.kf = prm.kf; cx.kd = prm.kd;
     const int g = cx.g;
     const float kf = cx.kf;
-    FlowOrder od;
-    od.rows = cx.B * (g + 1); od.nch = cx.nch; od.lag = fl.lag;
-    od.total = static_cast<unsigned>(od.rows + od.lag) * 2u * static_cast<unsigned>(od.nch);
 
     if (tid == 0) {
         for (int i = 0; i < kFDesc; ++i) {
@@ -548,29 +539,25 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         // =============================== service warp ===============================
         // takes tickets, waits for what a sweep-2 item needs, hands descriptors to the workers,
         // and does everything that follows a sweep, so that the workers never stop streaming
-        // a ticket decoded into a descriptor; never blocks
+        const unsigned total_s1 = static_cast<unsigned>(cx.B) * (g + 1) * cx.nch;
+        // the next sweep-1 item, or kExit when all have been handed out; never blocks
         auto take = [&](FlowDesc& d) {
-            for (;;) {
-                unsigned t = 0;
-                if (lane == 0) t = atomicAdd(&fl.counters[0], 1u);
-                t = __shfl_sync(0xffffffffu, t, 0);
-                if (t >= od.total) { d.kind = kExit; return; }
-                int kind, ri, ch;
-                if (!f_decode(od, t, kind, ri, ch)) continue;
-                const int r = ri % (g + 1), b = ri / (g + 1);
-                d.kind = kind; d.ri = ri; d.ch = ch; d.have_q = r < g;
-                d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
-                d.rowQ = r < g ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
-                               : nullptr;
-                d.cp = 1.f; d.nMP = 0.f; d.nMQ = 0.f;
-                return;
-            }
+            unsigned t = 0;
+            if (lane == 0) t = atomicAdd(&fl.counters[0], 1u);
+            t = __shfl_sync(0xffffffffu, t, 0);
+            if (t >= total_s1) { d.kind = kExit; return; }
+            const int ri = static_cast<int>(t / cx.nch), ch = static_cast<int>(t % cx.nch);
+            const int r = ri % (g + 1), b = ri / (g + 1);
+            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = r < g;
+            d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
+            d.rowQ = r < g ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
+                           : nullptr;
+            d.cp = 1.f; d.nMP = 0.f; d.nMQ = 0.f;
         };
-        // A sweep-2 item may start once its row has been folded into the recursion.  That is done
-        // by whoever completes the row, possibly this very warp a few items from now, so the warp
-        // never blocks on it: an item that is not ready is set aside, later tickets go first, and
-        // the items set aside are asked about again on every round (all of them with one load each,
-        // side by side in the lanes).
+        // A chunk's second sweep may start once its row has been folded into the recursion.  That
+        // is done by whoever completes the row, possibly this very warp a few items from now, so
+        // the warp never blocks on it: it keeps a list of its swept chunks and asks about all of
+        // them on every round (one load each, side by side in the lanes).
         auto fill_scalars = [&](FlowDesc& d) {
             __threadfence();
             if (d.have_q) d.cp = __ldcg(&fl.cscale[d.ri]);
@@ -582,13 +569,14 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             __syncwarp();
         };
         int q = 0, n = 0, qexit = -1;     // items published / post-processed; index of the exit descriptor
-        int ndef = 0;                     // items set aside
+        int ndef = 0;                     // chunks swept once, waiting for their second sweep
+        int s1_flying = 0;                // sweep-1 items published and not yet post-processed
         bool exhausted = false;           // the ticket counter has run past the last item
         unsigned idle = 0;
         for (;;) {
             // 1. publish what can be published (a slot is free once its previous item is post-processed)
             while (qexit < 0 && q - n < kFDesc) {
-                // (a) the oldest item set aside whose row has been folded meanwhile
+                // (a) second sweep of the oldest waiting chunk whose row has been folded
                 unsigned rel = 0;
                 if (lane < ndef) rel = ld_volatile(&fl.rel[sh.defer[lane].ri]);
                 const unsigned okmask = __ballot_sync(0xffffffffu, rel != 0u);
@@ -604,30 +592,18 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                     ++q;
                     continue;
                 }
-                // (b) a new ticket
+                // (b) a new sweep-1 item, unless the list could overflow when those in flight finish
                 if (exhausted) {
-                    if (ndef == 0) { FlowDesc d; d.kind = kExit; publish(d, q); qexit = q; ++q; }
+                    if (ndef == 0 && s1_flying == 0) { FlowDesc d; d.kind = kExit; publish(d, q); qexit = q; ++q; }
                     break;
                 }
-                if (ndef == kFDefer) break;      // enough set aside: wait for one of them
+                if (ndef + s1_flying >= kFDefer) break;
                 FlowDesc d;
                 take(d);
                 if (d.kind == kExit) { exhausted = true; continue; }
-                bool ok = true;
-                if (d.kind == kSweep2) {
-                    unsigned r1 = 0;
-                    if (lane == 0) r1 = ld_volatile(&fl.rel[d.ri]);
-                    ok = __shfl_sync(0xffffffffu, r1, 0) != 0u;
-                }
-                if (ok) {
-                    if (d.kind == kSweep2) fill_scalars(d);
-                    publish(d, q);
-                    ++q;
-                } else {
-                    if (lane == 0) sh.defer[ndef] = d;
-                    ++ndef;
-                    __syncwarp();
-                }
+                publish(d, q);
+                ++q;
+                ++s1_flying;
             }
             // 2. the oldest item in flight: wait for the workers, then do what follows its sweep
             const int in_flight_end = qexit >= 0 ? qexit : q;
@@ -635,8 +611,15 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 const int slot = n % kFDesc;
                 const FlowDesc d = sh.desc[slot];
                 mbar_wait(smem_u32(&sh.done[slot]), static_cast<uint32_t>(n / kFDesc) & 1u, prm.status);
-                if (d.kind == kSweep1) f_after_sweep1<DT>(prm, fl, cx, sh, slot, d.ri, d.ch, lane);
-                else                   f_after_sweep2<DT>(prm, fl, cx, sh, slot, d, lane);
+                if (d.kind == kSweep1) {
+                    f_after_sweep1<DT>(prm, fl, cx, sh, slot, d.ri, d.ch, lane);
+                    if (lane == 0) { sh.defer[ndef] = d; sh.defer[ndef].kind = kSweep2; }   // its second sweep is ours
+                    ++ndef;
+                    --s1_flying;
+                    __syncwarp();
+                } else {
+                    f_after_sweep2<DT>(prm, fl, cx, sh, slot, d, lane);
+                }
                 ++n;
                 idle = 0;
                 continue;
@@ -733,7 +716,6 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl)
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
     fl->nch = nch;
-    fl->lag = 0;
 }
 
 // Chunks per row.  An item should be large next to what it costs to hand it out (about
@@ -772,13 +754,7 @@ int flow_max_ctas_per_sm(int dtype) {
 }
 
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl_in, int dtype, int nctas, cudaStream_t stream) {
-    FlowScratch fl = fl_in;
-    if (fl.lag <= 0) {
-        // sweep-2 items trail by about the rows that are in flight at once (every CTA holds up
-        // to kFDesc items, half of them sweep-1), so that they rarely have to wait and the rows
-        // they re-read are still in L2
-        fl.lag = (nctas * kFDesc) / (2 * fl.nch) + 2;
-    }
+    const FlowScratch& fl = fl_in;
     pick_flow(dtype)<<<nctas, kFAllThreads, kFlowSmem, stream>>>(prm, fl);
     return cudaGetLastError();
 }

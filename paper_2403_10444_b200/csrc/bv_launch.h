@@ -25,7 +25,7 @@ cudaError_t launch_cluster(const Params& prm, int algo, int dtype, int cluster, 
 // when the kernel starts.
 struct RowZ { double MP, ZP, MQ, ZQ; };   // row (or chunk) references and sums of 2^{z k - M}
 struct FlowScratch {
-    unsigned* counters;   // [0]: ticket counter of the item order
+    unsigned* counters;   // [0]: ticket counter of the sweep-1 items
     unsigned* row_cnt;    // [B (gamma+1)] sweep-1 chunks finished per row
     unsigned* row_done;   // [B (gamma+1)] row normalisers published
     unsigned* s2_cnt;     // [B (gamma+1)] sweep-2 chunks finished per position
@@ -44,7 +44,6 @@ struct FlowScratch {
     double* S;            // [B (gamma+1)]
     int* cand;            // [B (gamma+1)]
     int nch;              // chunks per row
-    int lag;              // rows by which sweep-2 items trail sweep-1 items in the item order
 };
 size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes);
 void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl);
