@@ -31,6 +31,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 from paper_2403_10444_b200 import workloads as wl  # noqa: E402
+from paper_2403_10444_b200 import sharding  # noqa: E402
 
 METRIC = "verifications/s (B*gamma logit rows)"
 UNIT = "verifications/s"
@@ -223,12 +224,9 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     total_ms = start.elapsed_time(stop)
     kernel_ms = [e0.elapsed_time(e1) for e0, e1 in evs]
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = sharding.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * w.B * w.gamma / (ms_per_step * 1e-3)
+    value = sharding.whole_job_rate(w.B * w.gamma, ms_per_step)
 
     # ---- end to end: host buffers through the C-ABI host entry, copies inside the timed region ----
     e2e = None
@@ -254,10 +252,7 @@ def end_to_end(args, w, inp, out, bv, barrier, dist, dev, world):
     for _ in range(args.e2e_steps):
         hfn(*ha, out_tokens=ot, out_len=ol)
     e2e_s = (time.perf_counter() - t0) / args.e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = sharding.max_over_ranks(e2e_s, dev)
     h2d = sum(host[k].numel() * host[k].element_size()
               for k in ("target_logits", "draft_logits", "draft_tokens", "uniforms"))
     d2h = ot.numel() * 4 + ol.numel() * 4
@@ -269,8 +264,20 @@ def end_to_end(args, w, inp, out, bv, barrier, dist, dev, world):
 def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches, out, dist):
     peak, peak_src = measured_peak()
     k_ms = statistics.mean(kernel_ms)
-    achieved = w.logit_bytes / (k_ms * 1e-3) / 1e9
     mean_len = float(out[1].float().mean().item())
+    esz = 4 if w.dtype == "f32" else 2
+    if args.algo == "block":
+        # Algorithm 2 needs every row: B (2 gamma + 1) V elements
+        algo_bytes = w.logit_bytes
+        kernel = "verify_flow_kernel"
+    else:
+        # Algorithm 1 stops at the first rejection: a sequence that emits n tokens needs the row
+        # pairs 0 .. min(n, gamma) - 1 and, when all gamma tokens were accepted, target row gamma
+        n = out[1].long().clamp(min=0)
+        rows = 2 * n.clamp(max=w.gamma) + (n == w.gamma + 1).long()
+        algo_bytes = int(rows.sum().item()) * w.V * esz
+        kernel = "verify_cluster_kernel"
+    achieved = algo_bytes / (k_ms * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -283,9 +290,9 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
         "e2e": e2e,
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": TRAFFIC_BYTES.get((args.workload, args.algo)),
-                     "peak_source": peak_src, "kernel": "verify_resident_kernel" if args.algo == "block" else "verify_stream_kernel", "kernel_ms": k_ms,
-                     "algorithmic_bytes": w.logit_bytes, "frac_of_8TBps": achieved / 8000.0},
+                     "frac": achieved / peak, "traffic": TRAFFIC_BYTES.get((w.name, args.algo, kernel)),
+                     "peak_source": peak_src, "kernel": kernel, "kernel_ms": k_ms,
+                     "algorithmic_bytes": algo_bytes, "frac_of_8TBps": achieved / 8000.0},
         "sequences_per_s": world * w.B / (ms_per_step * 1e-3),
     }
     if not args.no_cpu_baseline and world == 1:
@@ -296,8 +303,11 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/; None until a capture of the current kernel exists.
-TRAFFIC_BYTES = {}
+# captures summarised under profiles/ (a B=128 capture scaled by the batch: the traffic grows in
+# proportion to B); None for a workload or kernel with no capture.
+TRAFFIC_BYTES = {
+    ("c4", "block", "verify_flow_kernel"): 4360644096,
+}
 
 
 if __name__ == "__main__":
