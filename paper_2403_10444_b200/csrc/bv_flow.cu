@@ -18,103 +18,12 @@
 // No CTA ever waits for another one while it holds work that others need: sweep-1 items
 // have no prerequisites, the lock is only held over a few scalar operations, and a CTA
 // polls (bounded) only when nothing is left to start.  So CTAs need not be co-resident.
-#include "bv_device.cuh"
-#include "bv_launch.h"
+#include "bv_flow_common.cuh"
 
 namespace bv {
 
 constexpr int kFThreads = 512;
 constexpr int kFWarps = kFThreads / 32;
-
-enum : int { kExit = 0, kSweep1 = 1, kSweep2 = 2 };
-constexpr int kCounterWords = 32;   // [0]: the ticket counter
-
-__device__ __forceinline__ unsigned ld_volatile(const unsigned* p) {
-    return *reinterpret_cast<const volatile unsigned*>(p);
-}
-
-// ---- per-vector arithmetic; multiply-adds and additions are issued two lanes at a time
-// (fma.rn.f32x2 / add.rn.f32x2), which halves their share of the instruction stream ----
-__device__ __forceinline__ float2 f2(float x, float y) { return make_float2(x, y); }
-
-// a_e = 2^{v_e k - M}
-template <int EPV> __device__ __forceinline__ void f_exps(const float (&v)[EPV], float kf, float nM, float (&a)[EPV]) {
-    const float2 kk = f2(kf, kf), mm = f2(nM, nM);
-#pragma unroll
-    for (int e = 0; e < EPV; e += 2) {
-        const float2 x = __ffma2_rn(f2(v[e], v[e + 1]), kk, mm);
-        a[e] = ex2(x.x);
-        a[e + 1] = ex2(x.y);
-    }
-}
-template <int EPV> __device__ __forceinline__ float f_sum(const float (&a)[EPV]) {
-    float2 s = __fadd2_rn(f2(a[0], a[1]), f2(a[2], a[3]));
-    if (EPV == 8) s = __fadd2_rn(s, __fadd2_rn(f2(a[4], a[5]), f2(a[6], a[7])));
-    return s.x + s.y;
-}
-template <int EPV> __device__ __forceinline__ float f_exp_sum(const float (&v)[EPV], float kf, float nM) {
-    float a[EPV];
-    f_exps<EPV>(v, kf, nM, a);
-    return f_sum<EPV>(a);
-}
-template <int EPV> __device__ __forceinline__ void f_accumulate(const float (&v)[EPV], float kf, float& M, float& s) {
-    float vs = f_exp_sum<EPV>(v, kf, -M);
-    if (__any_sync(0xffffffffu, vs > kRaiseBound)) {      // some logit lies above the reference
-        const float y = rintf(warp_max(vec_max<EPV>(v)) * kf);
-        if (y > M) { s *= ref_scale(M, y); M = y; }
-        vs = f_exp_sum<EPV>(v, kf, -M);
-    }
-    s += vs;
-}
-// residual terms t_e = max(cp 2^{zP k - MP} - 2^{zQ k - MQ}, 0) and their sum; HAVEQ = false: t_e = cp 2^{zP k - MP}
-template <int EPV, bool HAVEQ>
-__device__ __forceinline__ float f_pair_sum(const float (&vp)[EPV], const float (&vq)[EPV], float kf, float cp,
-                                            float nMP, float nMQ, float (&t)[EPV]) {
-    float a[EPV], q[EPV];
-    f_exps<EPV>(vp, kf, nMP, a);
-    if (HAVEQ) f_exps<EPV>(vq, kf, nMQ, q);
-    const float2 cc = f2(cp, cp), ncc = f2(-cp, -cp);
-#pragma unroll
-    for (int e = 0; e < EPV; e += 2) {
-        if (HAVEQ) {
-            // q - cp a in one packed multiply-add; the sign flips for free inside the max
-            const float2 d = __ffma2_rn(ncc, f2(a[e], a[e + 1]), f2(q[e], q[e + 1]));
-            t[e] = fmaxf(-d.x, 0.f);
-            t[e + 1] = fmaxf(-d.y, 0.f);
-        } else {
-            const float2 d = __fmul2_rn(cc, f2(a[e], a[e + 1]));
-            t[e] = d.x;
-            t[e + 1] = d.y;
-        }
-    }
-    return f_sum<EPV>(t);
-}
-template <int DT> __device__ __forceinline__ void f_load(const char* row, int i, float (&v)[Raw<DT>::EPV]) {
-    Raw<DT>::unpack(ld_stream_v4(row + static_cast<size_t>(i) * 16), v);
-}
-template <int DT>
-__device__ __forceinline__ void f_load_tail(const char* row, int i, int end, float (&v)[Raw<DT>::EPV]) {
-    if (row != nullptr && i < end) {
-        f_load<DT>(row, i, v);
-    } else {
-#pragma unroll
-        for (int e = 0; e < Raw<DT>::EPV; ++e) v[e] = -INFINITY;
-    }
-}
-
-// scratch written by other CTAs is always read through L2
-__device__ __forceinline__ RowZ load_rowz(const RowZ* p) {
-    RowZ z;
-    z.MP = __ldcg(&p->MP); z.ZP = __ldcg(&p->ZP); z.MQ = __ldcg(&p->MQ); z.ZQ = __ldcg(&p->ZQ);
-    return z;
-}
-
-struct FlowCtx {
-    int g, V, B, nch, units;
-    size_t row_bytes;
-    float kf;
-    double kd;
-};
 
 __device__ __forceinline__ void chunk_range(const FlowCtx& cx, int ch, int warp, int& w0, int& w1) {
     const int u0 = static_cast<int>(static_cast<long long>(cx.units) * ch / cx.nch);
@@ -123,176 +32,6 @@ __device__ __forceinline__ void chunk_range(const FlowCtx& cx, int ch, int warp,
     w1 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * (warp + 1) / kFWarps);
 }
 
-// One warp walks segment [w0, w1) of a row pair in index order and returns the first element
-// whose running residual mass exceeds tw (else the last element with positive mass, else -1).
-template <int DT>
-__device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int lane, float kf, float cp,
-                        float nMP, float nMQ, float tw) {
-    constexpr int EPV = Raw<DT>::EPV;
-    float run = 0.f;
-    int found = -1, last_pos = -1;
-    for (int base = w0; base < w1 && found < 0; base += 32) {
-        const int i = base + lane;
-        float vp[EPV], vq[EPV], tt[EPV];
-        f_load_tail<DT>(rowP, i, w1, vp);
-        f_load_tail<DT>(rowQ, i, w1, vq);
-        const float ls = rowQ ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, tt)
-                              : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, tt);
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) if (tt[e] > 0.f) last_pos = i * EPV + e;
-        float incw = ls;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const float o = __shfl_up_sync(0xffffffffu, incw, off);
-            if (lane >= off) incw += o;
-        }
-        const unsigned bal = __ballot_sync(0xffffffffu, run + incw > tw && ls > 0.f);
-        if (bal) {
-            const int src = __ffs(bal) - 1;
-            int f = -1;
-            if (lane == src) {
-                float cum = run + incw - ls;
-                int lp = -1;
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) {
-                    cum += tt[e];
-                    if (tt[e] > 0.f) lp = i * EPV + e;
-                    if (f < 0 && cum > tw && tt[e] > 0.f) f = i * EPV + e;
-                }
-                if (f < 0) f = lp;
-            }
-            found = __shfl_sync(0xffffffffu, f, src);
-        }
-        run += __shfl_sync(0xffffffffu, incw, 31);
-    }
-    if (found < 0) {
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, off));
-        found = last_pos;
-    }
-    return found;
-}
-
-// ---- the end of a block (one thread): Eq. "pacc_block", selection of tau, output ----
-__device__ void f_finalize_block(const Params& prm, const FlowScratch& fl, int b) {
-    const int g = prm.gamma;
-    int32_t* ot = prm.out_tokens + static_cast<size_t>(b) * (g + 1);
-    const int32_t* X = prm.tok + static_cast<size_t>(b) * g;
-    const float* u = prm.uni + static_cast<size_t>(b) * (g + 2);
-    const double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
-    const double* S = fl.S + static_cast<size_t>(b) * (g + 1);
-    const int* cand = fl.cand + static_cast<size_t>(b) * (g + 1);
-    const bool bad = ld_volatile(&fl.bad[b]) != 0;
-    int tau = -1;
-    if (!bad) {
-        tau = 0;
-        // h_gamma = p_gamma; h_i = S_i / (S_i + 1 - p_i); tau = max{i : eta_i <= h_i}
-        for (int i = g; i >= 1; --i) {
-            const double pi = __ldcg(&p[i]);
-            double h = pi;
-            if (i < g) { const double Si = __ldcg(&S[i]); h = Si > 0.0 ? Si / (Si + 1.0 - pi) : 0.0; }
-            if (h > 0.0 && static_cast<double>(u[i - 1]) <= h) { tau = i; break; }
-        }
-    }
-    for (int i = 0; i <= g; ++i) ot[i] = -1;
-    if (tau >= 0) {
-        for (int i = 0; i < tau; ++i) ot[i] = X[i];
-        ot[tau] = __ldcg(&cand[tau]);
-        prm.out_len[b] = tau + 1;
-    } else {
-        prm.out_len[b] = -1;
-    }
-    if (prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d) {
-        const double ln2 = 0.693147180559945309417232;
-        for (int i = 0; i <= g; ++i) {
-            const size_t o1 = static_cast<size_t>(b) * (g + 1) + i, o0 = static_cast<size_t>(b) * g + i;
-            const double pi = __ldcg(&p[i]);
-            const double Si = i < g ? __ldcg(&S[i]) : 0.0;
-            double h = (i == 0) ? 1.0 : (i == g ? pi : (Si > 0.0 ? Si / (Si + 1.0 - pi) : 0.0));
-            const RowZ z = load_rowz(&fl.rowZ[static_cast<size_t>(b) * (g + 1) + i]);
-            if (prm.out_p) prm.out_p[o1] = static_cast<float>(pi);
-            if (prm.out_h) prm.out_h[o1] = static_cast<float>(h);
-            if (prm.out_lse_t) prm.out_lse_t[o1] = static_cast<float>((static_cast<double>(z.MP) + log2(z.ZP)) * ln2);
-            if (i < g && prm.out_S) prm.out_S[o0] = static_cast<float>(Si);
-            if (i < g && prm.out_lse_d) prm.out_lse_d[o0] = static_cast<float>((static_cast<double>(z.MQ) + log2(z.ZQ)) * ln2);
-        }
-    }
-}
-
-// ---- a row is complete: normalisers, then the recursion over every complete row ----
-template <int DT>
-__device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int r) {
-    const int g = cx.g;
-    const size_t rowi = static_cast<size_t>(b) * (g + 1) + r;
-    // combine the chunks (fp64): row reference = max of the chunk references
-    double MP = kNoRef, MQ = kNoRef;
-    for (int ch = 0; ch < cx.nch; ++ch) {
-        const RowZ z = load_rowz(&fl.part[rowi * cx.nch + ch]);
-        MP = fmax(MP, z.MP); MQ = fmax(MQ, z.MQ);
-    }
-    double ZP = 0.0, ZQ = 0.0;
-    for (int ch = 0; ch < cx.nch; ++ch) {
-        const RowZ z = load_rowz(&fl.part[rowi * cx.nch + ch]);
-        ZP += z.ZP * static_cast<double>(ref_scale(static_cast<float>(z.MP), static_cast<float>(MP)));
-        ZQ += z.ZQ * static_cast<double>(ref_scale(static_cast<float>(z.MQ), static_cast<float>(MQ)));
-    }
-    RowZ out; out.MP = MP; out.ZP = ZP; out.MQ = MQ; out.ZQ = ZQ;
-    fl.rowZ[rowi] = out;
-    const bool have_q = r < g;
-    // the row's maximum is finite iff its reference is; Z is NaN / inf iff the row holds a NaN / overflowed
-    if (!(MP > kNoRef && MP < INFINITY) || !(ZP < INFINITY)) atomicOr(&fl.bad[b], 1u);
-    if (have_q && (!(MQ > kNoRef && MQ < INFINITY) || !(ZQ < INFINITY))) atomicOr(&fl.bad[b], 1u);
-    // everything the recursion needs from this row, computed before the lock is taken:
-    // ratio = P_r(X_{r+1}) / Q_r(X_{r+1}) from the two logits of the drafted token, and Z_Q / Z_P
-    if (have_q) {
-        double ratio = 0.0;
-        const int x = prm.tok[static_cast<size_t>(b) * g + r];
-        if (x < 0 || x >= cx.V) {
-            atomicOr(&fl.bad[b], 1u);
-        } else {
-            const char* rowP = static_cast<const char*>(prm.tgt) + rowi * cx.row_bytes;
-            const char* rowQ = static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes;
-            const double zq = load_logit<DT>(rowQ, x), zp = load_logit<DT>(rowP, x);
-            if (zq == -INFINITY) atomicOr(&fl.bad[b], 1u);
-            else ratio = exp2((zp - zq) * cx.kd - (MP - MQ)) * (ZQ / ZP);
-        }
-        fl.ratio[rowi] = ratio;
-        fl.zratio[rowi] = ZQ / ZP;
-    }
-    __threadfence();
-    atomicExch(&fl.row_done[rowi], 1u);
-
-    // Fold every complete row, in order, into p_{c+1} = min(p_c ratio_c, 1) and release its
-    // sweep-2 items.  The critical section is a few loads and stores per row.
-    double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
-    for (unsigned spins = 0;; ++spins) {
-        if (atomicCAS(&fl.lock[b], 0u, 1u) == 0u) break;
-        // the holder may have looked at this row before it was marked: wait for it to let go,
-        // unless the recursion has already moved past this row
-        if (ld_volatile(&fl.chain[b]) > static_cast<unsigned>(r)) return;
-        __nanosleep(32);
-        if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return; }
-    }
-    __threadfence();
-    unsigned c = ld_volatile(&fl.chain[b]);
-    while (c <= static_cast<unsigned>(g) && ld_volatile(&fl.row_done[static_cast<size_t>(b) * (g + 1) + c]) != 0u) {
-        const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
-        const double p_c = (c == 0) ? 1.0 : __ldcg(&p[c]);
-        if (c == 0) p[0] = 1.0;
-        float cs = 1.f;
-        if (c < static_cast<unsigned>(g)) {
-            p[c + 1] = fmin(p_c * __ldcg(&fl.ratio[ci]), 1.0);
-            cs = static_cast<float>(p_c * __ldcg(&fl.zratio[ci]));
-        }
-        fl.cscale[ci] = cs;
-        __threadfence();                       // p, cscale are visible ...
-        atomicExch(&fl.rel[ci], 1u);           // ... before the row's sweep-2 items may start
-        ++c;
-    }
-    *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
-    __threadfence();
-    atomicExch(&fl.lock[b], 0u);
-}
 
 constexpr int kFDepth = 8;     // ring slots per worker thread: four (P, Q) steps of lookahead
 constexpr int kFAhead = kFDepth / 2;
@@ -351,8 +90,7 @@ __device__ void f_after_sweep1(const Params& prm, const FlowScratch& fl, const F
 template <int DT>
 __device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int slot,
                                const FlowDesc& d, int lane) {
-    constexpr int EPV = Raw<DT>::EPV;
-    const int g = cx.g, ri = d.ri, r = ri % (g + 1), b = ri / (g + 1);
+    const int ri = d.ri;
     const int nseg = cx.nch * kFWarps;
     float* segs = fl.seg_tot + static_cast<size_t>(ri) * nseg;
     if (lane < kFWarps) segs[d.ch * kFWarps + lane] = sh.part_s[slot][0][lane];
@@ -363,73 +101,8 @@ __device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const F
     last = __shfl_sync(0xffffffffu, last, 0);
     if (!last) return;
 
-    // ---------------- the position is complete: S_r and the candidate Y_r ----------------
-    __threadfence();
-    const bool have_q = d.have_q != 0;
-    const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
-    float w[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) w[j] = (4 * lane + j < nseg) ? __ldcg(&segs[4 * lane + j]) : 0.f;
-    double sd = (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
-                (static_cast<double>(w[2]) + static_cast<double>(w[3]));
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
-    if (lane == 0 && have_q) fl.S[ri] = sd / __ldcg(&fl.rowZ[ri].ZQ);
-    const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
-    float inc = l4;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const float o = __shfl_up_sync(0xffffffffu, inc, off);
-        if (lane >= off) inc += o;
-    }
-    const float total = __shfl_sync(0xffffffffu, inc, 31);
-    int found = -1;
-    if (total > 0.f) {
-        const float t = uf * total;
-        float exc = __shfl_up_sync(0xffffffffu, inc, 1);
-        if (lane == 0) exc = 0.f;
-        const float p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
-        // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
-        const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
-        const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
-        const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
-        const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
-        int e = 3; float bef = p3; int src;
-        if (hit) {
-            src = __ffs(hit) - 1;
-            if (h1) { e = 0; bef = exc; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
-        } else {
-            src = 31 - __clz(nz);
-            e = 0; bef = exc;
-            if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
-            else if (w[1] > 0.f) { e = 1; bef = p1; }
-        }
-        const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
-        const float before = __shfl_sync(0xffffffffu, bef, src);
-        int s0, s1;
-        chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1);
-        found = f_rescan<DT>(d.rowP, d.rowQ, s0, s1, lane, cx.kf, d.cp, d.nMP, d.nMQ, t - before);
-    } else if (have_q && r == 0 && total == 0.f) {
-        // empty residual at position 0 (P_0 and Q_0 coincide bit for bit): sample P_0 with the same
-        // uniform.  Two plain passes over the whole row by this warp: rare, so speed does not matter.
-        float tot = 0.f;
-        for (int base2 = 0; base2 < cx.units; base2 += 32) {
-            float vp[EPV], t2[EPV];
-            f_load_tail<DT>(d.rowP, base2 + lane, cx.units, vp);
-            tot += f_pair_sum<EPV, false>(vp, vp, cx.kf, 1.f, d.nMP, d.nMQ, t2);
-        }
-        tot = warp_sum(tot);
-        found = f_rescan<DT>(d.rowP, nullptr, 0, cx.units, lane, cx.kf, 1.f, d.nMP, d.nMQ, uf * tot);
-    }
-    if (lane == 0) {
-        fl.cand[ri] = found;
-        __threadfence();
-        if (atomicAdd(&fl.cand_cnt[b], 1u) == static_cast<unsigned>(g)) {
-            __threadfence();
-            f_finalize_block(prm, fl, b);
-        }
-    }
-    __syncwarp();
+    f_position_complete<DT>(prm, fl, cx, ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, nseg, segs, lane,
+                            [&](int sel, int& s0, int& s1) { chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1); });
 }
 
 // ---- worker warps: one warp's segment of one item ----
@@ -575,7 +248,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         unsigned idle = 0;
         for (;;) {
             // 1. publish what can be published (a slot is free once its previous item is post-processed)
-            while (qexit < 0 && q - n < kFDesc) {
+            while (qexit < 0 && q - n < fl.depth) {
                 // (a) second sweep of the oldest waiting chunk whose row has been folded
                 unsigned rel = 0;
                 if (lane < ndef) rel = ld_volatile(&fl.rel[sh.defer[lane].ri]);
@@ -674,6 +347,10 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
 static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
 size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes) {
+    return flow_scratch_bytes_segs(B, gamma, nch, nch * kFWarps, zero_bytes);
+}
+
+size_t flow_scratch_bytes_segs(int B, int gamma, int nch, int segs, size_t* zero_bytes) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
     size_t z = 0;
     z += up256(kCounterWords * sizeof(unsigned));   // counters
@@ -687,13 +364,17 @@ size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes) {
     n += up256(static_cast<size_t>(B) * (gamma + 2) * sizeof(double));   // pchain
     n += up256(rows * sizeof(float));               // cscale
     n += 2 * up256(rows * sizeof(double));          // ratio, zratio
-    n += up256(rows * nch * kFWarps * sizeof(float));   // seg_tot
+    n += up256(rows * segs * sizeof(float));        // seg_tot
     n += up256(rows * sizeof(double));              // S
     n += up256(rows * sizeof(int));                 // cand
     return n;
 }
 
 void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl) {
+    flow_scratch_layout_segs(base, B, gamma, nch, nch * kFWarps, fl);
+}
+
+void flow_scratch_layout_segs(void* base, int B, int gamma, int nch, int segs, FlowScratch* fl) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
     char* p = static_cast<char*>(base);
     auto take = [&](size_t bytes) { char* q = p; p += up256(bytes); return q; };
@@ -712,10 +393,12 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl)
     fl->cscale = reinterpret_cast<float*>(take(rows * sizeof(float)));
     fl->ratio = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->zratio = reinterpret_cast<double*>(take(rows * sizeof(double)));
-    fl->seg_tot = reinterpret_cast<float*>(take(rows * nch * kFWarps * sizeof(float)));
+    fl->seg_tot = reinterpret_cast<float*>(take(rows * segs * sizeof(float)));
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
     fl->nch = nch;
+    fl->depth = kFDesc;
+    fl->segs = segs;
 }
 
 // Chunks per row.  An item should be large next to what it costs to hand it out (about

@@ -43,13 +43,26 @@ struct FlowScratch {
     float* seg_tot;       // [B (gamma+1) nch 16]
     double* S;            // [B (gamma+1)]
     int* cand;            // [B (gamma+1)]
-    int nch;              // chunks per row
+    int nch;              // chunks per row (1 .. kFlowMaxChunks)
+    int depth;            // flow kernel: descriptors a CTA may have published and not yet post-processed (2 or 3)
+    int segs;             // residual totals kept per row
 };
+constexpr int kFlowMaxChunks = 32;
 size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes);
 void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl);
 int flow_max_ctas_per_sm(int dtype);
 int flow_pick_chunks(long long units, int B, int gamma, long long nctas);
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream);
+
+// Group kernel (Block Verification, 128-bit path): same scratch with nch = CTAs per group and
+// `segs` residual totals per row.  Cooperative launch of G * NG CTAs.
+size_t flow_scratch_bytes_segs(int B, int gamma, int nch, int segs, size_t* zero_bytes);
+void flow_scratch_layout_segs(void* base, int B, int gamma, int nch, int segs, FlowScratch* fl);
+int group_share_vectors();
+int group_segments_per_share();
+int group_max_lag();
+int group_max_ctas_per_sm(int dtype);
+cudaError_t launch_group(const Params& prm, const FlowScratch& fl, int dtype, int G, int NG, int L, cudaStream_t stream);
 
 // Resident kernel (Block Verification only, 128-bit path): a thread holds up to `nk`
 // vectors per row, nk in {2, 4, 8}.
