@@ -169,7 +169,13 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
         }
         bv::FlowScratch fl;
         bv::flow_scratch_layout_segs(d->flow_ws[slot], B, gamma, static_cast<int>(G), segs, &fl);
-        cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
+        // the counters and, right behind them, the per-CTA row statistics (their words say
+        // "not written yet" by being zero)
+        const size_t part_bytes = (static_cast<size_t>(B) * (gamma + 1) * G * sizeof(bv::RowZ) + 255) / 256 * 256;
+        cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes + part_bytes, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+        // likewise the residual totals
+        e = cudaMemsetAsync(fl.seg_tot, 0, static_cast<size_t>(B) * (gamma + 1) * segs * sizeof(float), stream);
         if (e != cudaSuccess) return cuda_fail(e);
         prm.ticket = nullptr;
         prm.nclusters = 0;

@@ -188,6 +188,25 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* st
         }
     }
 }
+// The same wait without a suspend-time hint: the thread polls and resumes as soon as the phase
+// completes (a hinted wait was seen to resume late).  Bounded like mbar_wait.
+__device__ __forceinline__ bool mbar_try_wait_now(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_wait_now(uint32_t bar, uint32_t parity, int* status) {
+    for (uint32_t spins = 0; !mbar_try_wait_now(bar, parity); ++spins) {
+        if (spins > (1u << 24)) {
+            if (status) atomicExch(status, 1);
+            return;
+        }
+    }
+}
 // 16 or 4 bytes into another CTA's shared memory; the bytes are counted by that CTA's barrier
 __device__ __forceinline__ void send_v4(uint32_t raddr, uint32_t rbar, float a, float b, float c, float d) {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"

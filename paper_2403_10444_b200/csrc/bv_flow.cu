@@ -101,7 +101,7 @@ __device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const F
     last = __shfl_sync(0xffffffffu, last, 0);
     if (!last) return;
 
-    f_position_complete<DT>(prm, fl, cx, ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, nseg, segs, lane,
+    f_position_complete<DT, false>(prm, fl, cx, ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, nseg, segs, lane,
                             [&](int sel, int& s0, int& s1) { chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1); });
 }
 
@@ -255,12 +255,14 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 const unsigned okmask = __ballot_sync(0xffffffffu, rel != 0u);
                 if (okmask) {
                     const int i = __ffs(okmask) - 1;
+                    const bool wanted = __shfl_sync(0xffffffffu, rel, i) == kRelSweep;
                     FlowDesc d = sh.defer[i];
-                    fill_scalars(d);
+                    if (wanted) fill_scalars(d);
                     __syncwarp();
                     if (lane == 0) for (int j = i; j + 1 < ndef; ++j) sh.defer[j] = sh.defer[j + 1];
                     --ndef;
                     __syncwarp();
+                    if (!wanted) continue;          // nothing depends on this position: no second sweep
                     publish(d, q);
                     ++q;
                     continue;
@@ -283,7 +285,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             if (n < in_flight_end) {
                 const int slot = n % kFDesc;
                 const FlowDesc d = sh.desc[slot];
-                mbar_wait(smem_u32(&sh.done[slot]), static_cast<uint32_t>(n / kFDesc) & 1u, prm.status);
+                mbar_wait_now(smem_u32(&sh.done[slot]), static_cast<uint32_t>(n / kFDesc) & 1u, prm.status);
                 if (d.kind == kSweep1) {
                     f_after_sweep1<DT>(prm, fl, cx, sh, slot, d.ri, d.ch, lane);
                     if (lane == 0) { sh.defer[ndef] = d; sh.defer[ndef].kind = kSweep2; }   // its second sweep is ours
@@ -314,7 +316,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     for (int n = 0;; ++n) {
         const int slot = n % kFDesc;
         const uint32_t parity = static_cast<uint32_t>(n / kFDesc) & 1u;
-        mbar_wait(smem_u32(&sh.full[slot]), parity, prm.status);
+        mbar_wait_now(smem_u32(&sh.full[slot]), parity, prm.status);
         const int kind = sh.desc[slot].kind;
         if (kind == kExit) break;
         const bool have_q = sh.desc[slot].have_q != 0;

@@ -13,6 +13,8 @@ namespace bv {
 
 enum : int { kExit = 0, kSweep1 = 1, kSweep2 = 2 };
 constexpr int kCounterWords = 32;   // [0]: the ticket counter
+// rel[row]: 0 = not folded yet, then whether the row's second sweep is wanted
+enum : unsigned { kRelSweep = 1u, kRelSkip = 2u };
 
 __device__ __forceinline__ unsigned ld_volatile(const unsigned* p) {
     return *reinterpret_cast<const volatile unsigned*>(p);
@@ -242,6 +244,8 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
         if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return; }
     }
     __threadfence();
+    const bool all_positions = prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
+    unsigned nskip = 0;
     unsigned c = ld_volatile(&fl.chain[b]);
     while (c <= static_cast<unsigned>(g) && ld_volatile(&fl.row_done[static_cast<size_t>(b) * (g + 1) + c]) != 0u) {
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
@@ -253,13 +257,32 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
             cs = static_cast<float>(p_c * __ldcg(&fl.zratio[ci]));
         }
         fl.cscale[ci] = cs;
+        // Does anything depend on this position's second sweep?  S_c <= p_c (the residual mass of
+        // Eq. "pacc_block" is at most p_c sum_x P_c(x)), hence h_c <= p_c: a position whose
+        // uniform lies above p_c can never be the selected one, and nobody will ask for its S_c or
+        // its candidate.  Position gamma is selected iff eta_gamma <= h_gamma = p_gamma, and only then
+        // is the sample from P_gamma drawn.  Position 0 is what remains when no other is selected.
+        // (The margin keeps a uniform within rounding of p_c on the long path; with diagnostic
+        // outputs every position is computed.)
+        bool need = all_positions || c == 0;
+        if (!need) need = static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + c - 1]) <= p_c * (1.0 + 1e-6);
+        if (!need) {
+            if (c < static_cast<unsigned>(g)) fl.S[ci] = 0.0;
+            fl.cand[ci] = -1;
+            ++nskip;
+        }
         __threadfence();                       // p, cscale are visible ...
-        atomicExch(&fl.rel[ci], 1u);           // ... before the row's sweep-2 items may start
+        atomicExch(&fl.rel[ci], need ? kRelSweep : kRelSkip);   // ... before the row's sweep-2 items may start
         ++c;
     }
     *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
     __threadfence();
     atomicExch(&fl.lock[b], 0u);
+    // skipped positions count as complete; the last position to complete finishes the block
+    if (nskip > 0 && atomicAdd(&fl.cand_cnt[b], nskip) + nskip == static_cast<unsigned>(g) + 1u) {
+        __threadfence();
+        f_finalize_block(prm, fl, b);
+    }
 }
 
 
@@ -286,7 +309,12 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
 // ---- a position is complete (one warp): S_r from the segment totals, and the candidate Y_r.
 // `segs` holds the nseg totals of the row's segments in index order; range(s, v0, v1) gives the
 // vectors [v0, v1) of segment s. ----
-template <int DT, class RangeFn>
+// a segment total as stored: plain, or (ENC) with its lowest mantissa bit set to mark it written
+template <bool ENC> __device__ __forceinline__ float f_seg(const float* p) {
+    const float v = __ldcg(p);
+    return ENC ? __uint_as_float(__float_as_uint(v) & ~1u) : v;
+}
+template <int DT, bool ENC, class RangeFn>
 __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, bool have_q,
                                     const char* rowP, const char* rowQ, float cp, float nMP, float nMQ,
                                     int nseg, const float* segs, int lane, RangeFn range) {
@@ -306,7 +334,7 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int i = 128 * grp + 4 * lane + j;
-            w[j] = i < nseg ? __ldcg(&segs[i]) : 0.f;
+            w[j] = i < nseg ? f_seg<ENC>(&segs[i]) : 0.f;
         }
         sd += (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
               (static_cast<double>(w[2]) + static_cast<double>(w[3]));
@@ -332,7 +360,7 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int i = 128 * grp + 4 * lane + j;
-                w[j] = i < nseg ? __ldcg(&segs[i]) : 0.f;
+                w[j] = i < nseg ? f_seg<ENC>(&segs[i]) : 0.f;
             }
             const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
             float inc = l4;

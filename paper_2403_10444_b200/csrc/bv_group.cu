@@ -88,14 +88,29 @@ __device__ __forceinline__ unsigned g_ld_acquire(const unsigned* p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-// counter += 1, ordered after this thread's earlier writes; nothing comes back
-__device__ __forceinline__ void g_red_release(unsigned* p) {
-    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+// counter += 1; nothing comes back and nothing is ordered: a hint for whoever polls
+__device__ __forceinline__ void g_red_relaxed(unsigned* p) {
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
 }
 // warp-wide integer reference of one vector per lane: round(max * k)
 template <int EPV> __device__ __forceinline__ float g_ref(const float (&v)[EPV], float kf) {
     const int m = __reduce_max_sync(0xffffffffu, __float2int_rn(vec_max<EPV>(v) * kf));
     return m == INT_MIN ? kNoRef : static_cast<float>(m);
+}
+
+// Sum of the 32 floats at p as a balanced tree (the same shape as a warp shuffle reduction), read
+// in an order that starts at a different element in every lane so that the lanes of a warp, each
+// summing its own 32, never meet in a shared-memory bank.  fp32 with short dependency chains: the
+// fp64 pipe is far too slow for a 32-long chain per step.
+__device__ __forceinline__ float g_sum32(const float* p, int lane) {
+    float a[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = p[(i + lane) & 31];
+#pragma unroll
+    for (int j = 1; j < 4; ++j)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] += p[(8 * j + i + lane) & 31];
+    return ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
 }
 
 // A ring position that advances one slot at a time: slot index and how often it has been used.
@@ -107,19 +122,104 @@ struct GRing {
     __device__ __forceinline__ uint32_t prev_parity() const { return (use & 1u) ^ 1u; }   // the use before
 };
 
-// Row statistics from the G pairs in scratch (whole warp; all lanes return the same values).
+// A CTA's {M_P, Z_P, M_Q, Z_Q} of one row lives in scratch as four 8-byte words that each say
+// whether they have been written: the scratch starts at zero and every word is stored with its
+// lowest mantissa bit set (a change of 2^-52 in Z, none in the integer M once the bit is cleared
+// again).  A reader therefore needs no flag, no counter and no second trip to L2.
+__device__ __forceinline__ double g_enc(double v) {
+    return __longlong_as_double(__double_as_longlong(v) | 1ll);
+}
+struct GPart {
+    unsigned long long w[4];
+    __device__ __forceinline__ bool complete() const { return w[0] != 0ull && w[1] != 0ull && w[2] != 0ull && w[3] != 0ull; }
+    __device__ __forceinline__ double get(int i) const { return __longlong_as_double(static_cast<long long>(w[i] & ~1ull)); }
+};
+__device__ __forceinline__ GPart g_load_part(const RowZ* p) {
+    const unsigned long long* q = reinterpret_cast<const unsigned long long*>(p);
+    GPart r;
+    r.w[0] = __ldcg(q); r.w[1] = __ldcg(q + 1); r.w[2] = __ldcg(q + 2); r.w[3] = __ldcg(q + 3);
+    return r;
+}
+__device__ __forceinline__ RowZ g_load_rowz(const RowZ* p) {
+    const GPart t = g_load_part(p);
+    RowZ z; z.MP = t.get(0); z.ZP = t.get(1); z.MQ = t.get(2); z.ZQ = t.get(3);
+    return z;
+}
+
+// A reference as a saturating integer (INT_MIN: no reference), and back.
+__device__ __forceinline__ int g_ref_int(double M) { return M > kNoRef ? __double2int_rn(M) : INT_MIN; }
+__device__ __forceinline__ float g_ref_float(int m) { return m == INT_MIN ? kNoRef : static_cast<float>(m); }
+// z 2^{own - row} for integer references own <= row (0 without a reference of its own): exact
+__device__ __forceinline__ double g_scale_down(double z, int own, int row) {
+    if (own == INT_MIN) return 0.0;
+    const long long d = static_cast<long long>(own) - row;          // <= 0
+    if (d < -1000) return 0.0;
+    return z * __longlong_as_double((1023ll + d) << 52);
+}
+// 1 / x to fp64 accuracy from the fp32 reciprocal and two Newton steps (x > 0, finite)
+__device__ __forceinline__ double g_recip(double x) {
+    double y = static_cast<double>(__frcp_rn(static_cast<float>(x)));
+    y = y * (2.0 - x * y);
+    return y * (2.0 - x * y);
+}
+// 2^x in a handful of fp64 multiply-adds: 2^round(x) by the exponent field, 2^f, |f| <= 1/2, by
+// its Taylor series in f ln 2 to degree 10 (relative error below 1e-13).  x = -inf gives 0; a NaN
+// or a value beyond the exponent range is left to exp2.
+__device__ __forceinline__ double g_exp2(double x) {
+    if (!(x > -1000.0 && x < 1000.0)) return exp2(x);
+    const double xi = rint(x);
+    const double t = (x - xi) * 0.693147180559945309417232;
+    double y = 1.0 / 3628800.0;
+    y = fma(y, t, 1.0 / 362880.0);
+    y = fma(y, t, 1.0 / 40320.0);
+    y = fma(y, t, 1.0 / 5040.0);
+    y = fma(y, t, 1.0 / 720.0);
+    y = fma(y, t, 1.0 / 120.0);
+    y = fma(y, t, 1.0 / 24.0);
+    y = fma(y, t, 1.0 / 6.0);
+    y = fma(y, t, 0.5);
+    y = fma(y, t, 1.0);
+    y = fma(y, t, 1.0);
+    return y * __longlong_as_double((1023ll + static_cast<long long>(xi)) << 52);
+}
+
+// Row statistics from two parts per lane that are already in registers (G <= 64); whole warp,
+// all lanes return the same values.
+__device__ __forceinline__ void g_combine2(const GPart& a, const GPart& b, bool has_a, bool has_b,
+                                           double& MP, double& ZP, double& MQ, double& ZQ) {
+    MP = kNoRef; MQ = kNoRef;
+    if (has_a) { MP = fmax(MP, a.get(0)); MQ = fmax(MQ, a.get(2)); }
+    if (has_b) { MP = fmax(MP, b.get(0)); MQ = fmax(MQ, b.get(2)); }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) { MP = fmax(MP, shfl_xor_d(MP, off)); MQ = fmax(MQ, shfl_xor_d(MQ, off)); }
+    ZP = 0.0; ZQ = 0.0;
+    const float fMP = static_cast<float>(MP), fMQ = static_cast<float>(MQ);
+    if (has_a) {
+        ZP += a.get(1) * static_cast<double>(ref_scale(static_cast<float>(a.get(0)), fMP));
+        ZQ += a.get(3) * static_cast<double>(ref_scale(static_cast<float>(a.get(2)), fMQ));
+    }
+    if (has_b) {
+        ZP += b.get(1) * static_cast<double>(ref_scale(static_cast<float>(b.get(0)), fMP));
+        ZQ += b.get(3) * static_cast<double>(ref_scale(static_cast<float>(b.get(2)), fMQ));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) { ZP += shfl_xor_d(ZP, off); ZQ += shfl_xor_d(ZQ, off); }
+}
+
+// Row statistics from the G pairs in scratch, all known to be there (whole warp; all lanes return
+// the same values; same order of operations as g_combine2 for G <= 64).
 __device__ __forceinline__ void g_combine(const FlowScratch& fl, size_t rowi, int G, int lane,
                                           double& MP, double& ZP, double& MQ, double& ZQ) {
     MP = kNoRef; MQ = kNoRef;
     for (int ch = lane; ch < G; ch += 32) {
-        const RowZ z = load_rowz(&fl.part[rowi * G + ch]);
+        const RowZ z = g_load_rowz(&fl.part[rowi * G + ch]);
         MP = fmax(MP, z.MP); MQ = fmax(MQ, z.MQ);
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) { MP = fmax(MP, shfl_xor_d(MP, off)); MQ = fmax(MQ, shfl_xor_d(MQ, off)); }
     ZP = 0.0; ZQ = 0.0;
     for (int ch = lane; ch < G; ch += 32) {
-        const RowZ z = load_rowz(&fl.part[rowi * G + ch]);
+        const RowZ z = g_load_rowz(&fl.part[rowi * G + ch]);
         ZP += z.ZP * static_cast<double>(ref_scale(static_cast<float>(z.MP), static_cast<float>(MP)));
         ZQ += z.ZQ * static_cast<double>(ref_scale(static_cast<float>(z.MQ), static_cast<float>(MQ)));
     }
@@ -213,42 +313,114 @@ verify_group_kernel(const Params prm, const FlowScratch fl, const GroupGeom geo)
 
     if (warp == kGRel) {
         // =============================== release warp ===============================
-        // Row after row: wait until all G pairs of the row are in scratch, combine them, advance the
-        // recursion and hand the scalars of the row's second sweep to the consumers.
+        // Row after row: as soon as all G pairs of the row are in scratch, combine them, advance the
+        // recursion and hand the scalars of the row's second sweep to the consumers.  The warp
+        // shares its scheduler with seven consumer warps and sits on the path between the two
+        // sweeps, so it is kept short and never waits for a load it could have issued earlier:
+        // the next row's pairs are requested before this row's are looked at (two register sets
+        // that swap roles), references are integers reduced warp-wide, 2^x and 1/x take a few fp64
+        // multiply-adds, and the drafted tokens' logits of a block are fetched a block ahead
+        // (lane r keeps row r's).
         GRing slot;
-        int q = 0, r = 0;
-        double p = 1.0;
-        double zp = 0.0, zq = 0.0;
-        bool tok_ok = false;
-        if (lane == 0) g_token_logits<DT>(prm, cx, grp, 0, zp, zq, tok_ok);
-        for (int n = 0; n < N; ++n) {
-            const int b = grp + q * NG;
-            const size_t rowi = static_cast<size_t>(b) * (g + 1) + r;
-            for (unsigned spins = 0; g_ld_acquire(&fl.row_cnt[rowi]) != static_cast<unsigned>(G); ++spins) {
-                if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return; }
-            }
-            double MP, ZP, MQ, ZQ;
-            g_combine(fl, rowi, G, lane, MP, ZP, MQ, ZQ);
-            float cs = 1.f;
-            if (lane == 0) {
-                if (r == 0) p = 1.0;
-                if (r < g) {
-                    cs = static_cast<float>(p * (ZQ / ZP));
-                    const double ratio = tok_ok ? exp2((zp - zq) * cx.kd - (MP - MQ)) * (ZQ / ZP) : 0.0;
-                    p = fmin(p * ratio, 1.0);
+        struct TokenLogits { float zp[2], zq[2]; };       // NaN in zq: no valid token
+        auto token_logits = [&](int b, TokenLogits& d) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int r = lane + 32 * t;
+                d.zp[t] = 0.f; d.zq[t] = NAN;
+                if (r < g && b < cx.B) {
+                    const int x = prm.tok[static_cast<size_t>(b) * g + r];
+                    if (x >= 0 && x < cx.V) {
+                        d.zq[t] = static_cast<float>(load_logit<DT>(static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes, x));
+                        d.zp[t] = static_cast<float>(load_logit<DT>(static_cast<const char*>(prm.tgt) + (static_cast<size_t>(b) * (g + 1) + r) * cx.row_bytes, x));
+                    }
                 }
-                // the next row's token logits: on their way while the consumers are being served
-                const int rn = r == g ? 0 : r + 1, bn = r == g ? b + NG : b;
-                if (n + 1 < N && rn < g) g_token_logits<DT>(prm, cx, bn, rn, zp, zq, tok_ok);
             }
-            if (slot.use > 0 && !g_wait(smem_u32(&sh.done2[slot.idx]), slot.prev_parity(), prm.status)) return;
+        };
+        TokenLogits dcur, dnxt;
+        token_logits(grp, dcur);
+        token_logits(grp + NG, dnxt);
+        int n = 0, q = 0, r = 0;
+        double p = 1.0;
+        const bool fast = G <= 64, la = lane < G, lb = lane + 32 < G;
+        auto row_of = [&](int qq, int rr) { return static_cast<size_t>(grp + qq * NG) * (g + 1) + rr; };
+        auto load_set = [&](size_t row, GPart& xa, GPart& xb) {
+            if (la) xa = g_load_part(&fl.part[row * G + lane]);
+            if (lb) xb = g_load_part(&fl.part[row * G + lane + 32]);
+        };
+        // row n from the set (xa, xb), which has been requested already; the set (ya, yb) is
+        // requested for row n + 1 on the way.  False: gave up waiting.
+        auto step = [&](GPart& xa, GPart& xb, GPart& ya, GPart& yb) -> bool {
+            const size_t row0 = row_of(q, r);
+            int iMP = INT_MIN, iMQ = INT_MIN;
+            double ZP = 0.0, ZQ = 0.0;
+            if (fast) {
+                if (n + 1 < N) load_set(r == g ? row_of(q + 1, 0) : row0 + 1, ya, yb);
+                for (unsigned idle = 0; !__all_sync(0xffffffffu, (!la || xa.complete()) && (!lb || xb.complete())); ++idle) {
+                    if (idle > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
+                    load_set(row0, xa, xb);
+                }
+                if (la) { iMP = g_ref_int(xa.get(0)); iMQ = g_ref_int(xa.get(2)); }
+                if (lb) { iMP = max(iMP, g_ref_int(xb.get(0))); iMQ = max(iMQ, g_ref_int(xb.get(2))); }
+                iMP = __reduce_max_sync(0xffffffffu, iMP);
+                iMQ = __reduce_max_sync(0xffffffffu, iMQ);
+                if (la) { ZP += g_scale_down(xa.get(1), g_ref_int(xa.get(0)), iMP); ZQ += g_scale_down(xa.get(3), g_ref_int(xa.get(2)), iMQ); }
+                if (lb) { ZP += g_scale_down(xb.get(1), g_ref_int(xb.get(0)), iMP); ZQ += g_scale_down(xb.get(3), g_ref_int(xb.get(2)), iMQ); }
+            } else {
+                for (unsigned idle = 0;; ++idle) {
+                    bool ok = true;
+                    iMP = INT_MIN; iMQ = INT_MIN;
+                    for (int ch = lane; ch < G; ch += 32) {
+                        const GPart t = g_load_part(&fl.part[row0 * G + ch]);
+                        ok = ok && t.complete();
+                        iMP = max(iMP, g_ref_int(t.get(0)));
+                        iMQ = max(iMQ, g_ref_int(t.get(2)));
+                    }
+                    if (__all_sync(0xffffffffu, ok)) break;
+                    if (idle > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
+                }
+                iMP = __reduce_max_sync(0xffffffffu, iMP);
+                iMQ = __reduce_max_sync(0xffffffffu, iMQ);
+                for (int ch = lane; ch < G; ch += 32) {
+                    const GPart t = g_load_part(&fl.part[row0 * G + ch]);
+                    ZP += g_scale_down(t.get(1), g_ref_int(t.get(0)), iMP);
+                    ZQ += g_scale_down(t.get(3), g_ref_int(t.get(2)), iMQ);
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) { ZP += shfl_xor_d(ZP, off); ZQ += shfl_xor_d(ZQ, off); }
+            // ---- the recursion (Eq. "def_as") and the scale of the row's second sweep ----
+            float cs = 1.f;
+            if (r == 0) p = 1.0;
+            if (r < g) {
+                const float zpx = __shfl_sync(0xffffffffu, r < 32 ? dcur.zp[0] : dcur.zp[1], r & 31);
+                const float zqx = __shfl_sync(0xffffffffu, r < 32 ? dcur.zq[0] : dcur.zq[1], r & 31);
+                const double zr = ZQ * g_recip(ZP);
+                cs = static_cast<float>(p * zr);
+                const bool tok_ok = zqx == zqx && zqx != -INFINITY;
+                const double e = (static_cast<double>(zpx) - static_cast<double>(zqx)) * cx.kd - static_cast<double>(iMP - iMQ);
+                p = fmin(p * (tok_ok ? g_exp2(e) * zr : 0.0), 1.0);
+            }
+            if (slot.use > 0 && !g_wait(smem_u32(&sh.done2[slot.idx]), slot.prev_parity(), prm.status)) return false;
             if (lane == 0) {
-                sh.meta2[slot.idx] = make_float4(cs, -static_cast<float>(MP), -static_cast<float>(MQ), 0.f);
+                sh.meta2[slot.idx] = make_float4(cs, -g_ref_float(iMP), -g_ref_float(iMQ), 0.f);
                 mbar_arrive(smem_u32(&sh.s2ready[slot.idx]));
             }
             __syncwarp();
             slot.next(kGR);
-            if (++r > g) { r = 0; ++q; }
+            ++n;
+            if (++r > g) {
+                r = 0; ++q;
+                dcur = dnxt;
+                token_logits(grp + (q + 1) * NG, dnxt);
+            }
+            return true;
+        };
+        GPart A0, A1, B0, B1;
+        if (fast) load_set(row_of(0, 0), A0, A1);
+        while (n < N) {
+            if (!step(A0, A1, B0, B1)) return;
+            if (n < N && !step(B0, B1, A0, A1)) return;
         }
         return;
     }
@@ -267,12 +439,8 @@ verify_group_kernel(const Params prm, const FlowScratch fl, const GroupGeom geo)
                 double zP = 0.0, zQ = 0.0;
                 float mP = kNoRef, mQ = kNoRef;
                 if (lane < kGWarps) {
-#pragma unroll 8
-                    for (int i = 0; i < 32; ++i) {
-                        const int k = (i + lane) & 31;
-                        zP += static_cast<double>(lp[k]);
-                        zQ += static_cast<double>(lp[kGShareVecs + k]);
-                    }
+                    zP = static_cast<double>(g_sum32(lp, lane));
+                    zQ = static_cast<double>(g_sum32(lp + kGShareVecs, lane));
                     mP = sh.wref[s1.idx][0][lane]; mQ = sh.wref[s1.idx][1][lane];
                 }
                 __syncwarp();
@@ -283,9 +451,8 @@ verify_group_kernel(const Params prm, const FlowScratch fl, const GroupGeom geo)
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) { zP += shfl_xor_d(zP, off); zQ += shfl_xor_d(zQ, off); }
                 if (lane == 0) {
-                    RowZ z; z.MP = MPc; z.ZP = zP; z.MQ = MQc; z.ZQ = zQ;
-                    fl.part[rowi * G + j] = z;
-                    g_red_release(&fl.row_cnt[rowi]);
+                    RowZ z; z.MP = g_enc(MPc); z.ZP = g_enc(zP); z.MQ = g_enc(MQc); z.ZQ = g_enc(zQ);
+                    fl.part[rowi * G + j] = z;          // four self-validating words: no fence, no counter
                 }
                 s1.next(kGR);
                 if (++r1 > g) { r1 = 0; ++q1; }
@@ -294,17 +461,16 @@ verify_group_kernel(const Params prm, const FlowScratch fl, const GroupGeom geo)
                 if (!g_wait(smem_u32(&sh.done2[s2.idx]), s2.parity(), prm.status)) return;
                 const size_t rowi = static_cast<size_t>(grp + q2 * NG) * (g + 1) + r2;
                 const float* lp = part2 + static_cast<size_t>(s2.idx) * kGShareVecs + lane * 32;
-                double t = 0.0;
-                if (lane < kGWarps) {
-#pragma unroll 8
-                    for (int i = 0; i < 32; ++i) t += static_cast<double>(lp[(i + lane) & 31]);
-                }
+                float t = 0.f;
+                if (lane < kGWarps) t = g_sum32(lp, lane);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&sh.free2[s2.idx]));
                 if (lane < kGWarps) {
                     // a segment is one consumer warp's 32 vectors: contiguous in the row
-                    fl.seg_tot[rowi * nseg + j * kGWarps + lane] = static_cast<float>(t);
-                    g_red_release(&fl.s2_cnt[rowi]);
+                    // (the total says "written" by its lowest mantissa bit; the counter is only a hint)
+                    fl.seg_tot[rowi * nseg + j * kGWarps + lane] =
+                        __uint_as_float(__float_as_uint(t) | 1u);
+                    g_red_relaxed(&fl.s2_cnt[rowi]);
                 }
                 s2.next(kGR);
                 if (++r2 > g) { r2 = 0; ++q2; }
@@ -329,10 +495,18 @@ verify_group_kernel(const Params prm, const FlowScratch fl, const GroupGeom geo)
             while (pos_r <= g) {
                 const size_t row_f = static_cast<size_t>(b) * (g + 1) + min(fold_r, g);
                 const size_t row_p = static_cast<size_t>(b) * (g + 1) + pos_r;
-                const unsigned c1 = fold_r <= g ? g_ld_acquire(&fl.row_cnt[row_f]) : 0u;
-                const unsigned c2 = pos_r < fold_r ? g_ld_acquire(&fl.s2_cnt[row_p]) : 0u;
+                bool parts_in = fold_r <= g;
+                if (fold_r <= g)
+                    for (int ch = lane; ch < G; ch += 32) parts_in = parts_in && g_load_part(&fl.part[row_f * G + ch]).complete();
+                parts_in = __all_sync(0xffffffffu, parts_in);
+                bool segs_in = pos_r < fold_r && ld_volatile(&fl.s2_cnt[row_p]) == all_segs;
+                if (segs_in) {
+                    const float* sg = fl.seg_tot + row_p * nseg;
+                    for (int i = lane; i < nseg; i += 32) segs_in = segs_in && __float_as_uint(__ldcg(&sg[i])) != 0u;
+                }
+                segs_in = __all_sync(0xffffffffu, segs_in);
                 bool did = false;
-                if (fold_r <= g && c1 == static_cast<unsigned>(G)) {
+                if (parts_in) {
                     const int r = fold_r;
                     double MP, ZP, MQ, ZQ;
                     g_combine(fl, row_f, G, lane, MP, ZP, MQ, ZQ);
@@ -359,7 +533,7 @@ verify_group_kernel(const Params prm, const FlowScratch fl, const GroupGeom geo)
                     ++fold_r;
                     did = true;
                 }
-                if (pos_r < fold_r && c2 == all_segs) {
+                if (segs_in) {
                     const int r = pos_r;
                     const bool have_q = r < g;
                     const char* rowP = static_cast<const char*>(prm.tgt) + row_p * cx.row_bytes;
@@ -369,7 +543,7 @@ verify_group_kernel(const Params prm, const FlowScratch fl, const GroupGeom geo)
                     const float nMP = -static_cast<float>(__ldcg(&fl.rowZ[row_p].MP));
                     const float nMQ = -static_cast<float>(__ldcg(&fl.rowZ[row_p].MQ));
                     const int units = cx.units;
-                    f_position_complete<DT>(prm, fl, cx, static_cast<int>(row_p), have_q, rowP, rowQ, cs, nMP, nMQ, nseg,
+                    f_position_complete<DT, true>(prm, fl, cx, static_cast<int>(row_p), have_q, rowP, rowQ, cs, nMP, nMQ, nseg,
                                             fl.seg_tot + row_p * nseg, lane, [units](int sel, int& s0, int& s1) {
                                                 s0 = min(sel * 32, units);
                                                 s1 = min(sel * 32 + 32, units);
