@@ -31,7 +31,6 @@ struct DeviceState {
     size_t flow_bytes[4] = {};
     unsigned long long flow_calls = 0;
     int flow_ctas_per_sm[2] = {};
-    int group_ctas_per_sm[2] = {};
     // staging for the host-buffer entry points
     void* stage = nullptr;
     size_t stage_bytes = 0;
@@ -137,54 +136,6 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     const bool want = force != nullptr;
     auto forced = [&](const char* name) { return want && std::strcmp(force, name) == 0; };
 
-    // Block Verification on 16-byte rows, every logit read once: groups of CTAs that keep their
-    // shares of a row in shared memory between the two sweeps (BV_KERNEL=group)
-    if (algo == bv::kBlockVerify && vec && forced("group")) {
-        int& per_sm = d->group_ctas_per_sm[dtype];
-        if (per_sm == 0) {
-            per_sm = bv::group_max_ctas_per_sm(dtype);
-            if (per_sm <= 0) per_sm = -1;
-        }
-        const long long units = static_cast<long long>(row_bytes / 16);
-        const long long G = (units + bv::group_share_vectors() - 1) / bv::group_share_vectors();
-        long long NG = per_sm > 0 ? static_cast<long long>(d->sm_count) * per_sm / G : 0;
-        if (NG > B) NG = B;
-        if (NG < 1) return BV_ERR_UNSUPPORTED;
-        int L = bv::group_max_lag() - 1;
-        if (const char* env = std::getenv("BV_GROUP_LAG")) {
-            const int v = std::atoi(env);
-            if (v >= 1 && v <= bv::group_max_lag()) L = v;
-        }
-        const int segs = static_cast<int>(G) * bv::group_segments_per_share();
-        size_t zero_bytes = 0;
-        const size_t need = bv::flow_scratch_bytes_segs(B, gamma, static_cast<int>(G), segs, &zero_bytes);
-        const int slot = static_cast<int>(d->flow_calls++ % 4);
-        if (d->flow_bytes[slot] < need) {
-            if (d->flow_ws[slot]) cudaFree(d->flow_ws[slot]);
-            d->flow_ws[slot] = nullptr;
-            d->flow_bytes[slot] = 0;
-            cudaError_t e = cudaMalloc(&d->flow_ws[slot], need);
-            if (e != cudaSuccess) return cuda_fail(e);
-            d->flow_bytes[slot] = need;
-        }
-        bv::FlowScratch fl;
-        bv::flow_scratch_layout_segs(d->flow_ws[slot], B, gamma, static_cast<int>(G), segs, &fl);
-        // the counters and, right behind them, the per-CTA row statistics (their words say
-        // "not written yet" by being zero)
-        const size_t part_bytes = (static_cast<size_t>(B) * (gamma + 1) * G * sizeof(bv::RowZ) + 255) / 256 * 256;
-        cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes + part_bytes, stream);
-        if (e != cudaSuccess) return cuda_fail(e);
-        // likewise the residual totals
-        e = cudaMemsetAsync(fl.seg_tot, 0, static_cast<size_t>(B) * (gamma + 1) * segs * sizeof(float), stream);
-        if (e != cudaSuccess) return cuda_fail(e);
-        prm.ticket = nullptr;
-        prm.nclusters = 0;
-        e = bv::launch_group(prm, fl, dtype, static_cast<int>(G), static_cast<int>(NG), L, stream);
-        if (e != cudaSuccess) return cuda_fail(e);
-        t_last_launches = 1;
-        return BV_OK;
-    }
-
     // Block Verification on 16-byte rows: the flow of independent work items
     if (algo == bv::kBlockVerify && vec && (!want || forced("flow"))) {
         int& per_sm = d->flow_ctas_per_sm[dtype];
@@ -214,7 +165,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             bv::flow_scratch_layout(d->flow_ws[slot], B, gamma, nch, &fl);
             if (const char* env = std::getenv("BV_FLOW_DEPTH")) {
                 const int v = std::atoi(env);
-                if (v >= 2 && v <= fl.depth) fl.depth = v;
+                if (v >= 2 && v <= 3) fl.depth = v;
             }
             cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
             if (e != cudaSuccess) return cuda_fail(e);

@@ -101,7 +101,7 @@ __device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const F
     last = __shfl_sync(0xffffffffu, last, 0);
     if (!last) return;
 
-    f_position_complete<DT, false>(prm, fl, cx, ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, nseg, segs, lane,
+    f_position_complete<DT>(prm, fl, cx, ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, nseg, segs, lane,
                             [&](int sel, int& s0, int& s1) { chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1); });
 }
 
@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 // (a) second sweep of the oldest waiting chunk whose row has been folded
                 unsigned rel = 0;
                 if (lane < ndef) rel = ld_volatile(&fl.rel[sh.defer[lane].ri]);
-                const unsigned okmask = __ballot_sync(0xffffffffu, rel != 0u);
+                const unsigned okmask = __ballot_sync(0xffffffffu, rel == kRelSweep || rel == kRelSkip);
                 if (okmask) {
                     const int i = __ffs(okmask) - 1;
                     const bool wanted = __shfl_sync(0xffffffffu, rel, i) == kRelSweep;
@@ -399,7 +399,7 @@ void flow_scratch_layout_segs(void* base, int B, int gamma, int nch, int segs, F
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
     fl->nch = nch;
-    fl->depth = kFDesc;
+    fl->depth = 2;      // one item being swept, one queued: the service warp reacts sooner to released rows
     fl->segs = segs;
 }
 

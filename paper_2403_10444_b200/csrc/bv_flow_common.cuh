@@ -1,5 +1,5 @@
 // Pieces shared by the kernels that run Block Verification (Algorithm 2) as a flow of work
-// items (bv_flow.cu, bv_group.cu): per-vector arithmetic, the rescan that turns a sampled mass
+// items (bv_flow.cu and the entry point without allocations): per-vector arithmetic, the rescan that turns a sampled mass
 // into a token, the end of a row (normalisers, prefix recursion of Eq. "def_as"), the end of a
 // position (S_r of Eq. "pacc_block" and the candidate of Eq. "pres-block") and the end of a
 // block (h_i, tau, output).
@@ -14,7 +14,7 @@ namespace bv {
 enum : int { kExit = 0, kSweep1 = 1, kSweep2 = 2 };
 constexpr int kCounterWords = 32;   // [0]: the ticket counter
 // rel[row]: 0 = not folded yet, then whether the row's second sweep is wanted
-enum : unsigned { kRelSweep = 1u, kRelSkip = 2u };
+enum : unsigned { kRelSweep = 1u, kRelSkip = 2u, kRelHold = 3u };   // hold: wanted only if every higher candidate is rejected
 
 __device__ __forceinline__ unsigned ld_volatile(const unsigned* p) {
     return *reinterpret_cast<const volatile unsigned*>(p);
@@ -199,6 +199,50 @@ static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl
     }
 }
 
+// ---- which positions get a second sweep (one thread each) ----
+// Is position i the selected one, given p_i and (for 0 < i < gamma) S_i?  Position 0 is what
+// remains when no other is selected.  (Eq. "pacc_block": h_gamma = p_gamma, h_i = S_i / (S_i + 1 - p_i).)
+static __device__ bool f_position_selected(const Params& prm, const FlowScratch& fl, int b, int i) {
+    const int g = prm.gamma;
+    if (i == 0) return true;
+    const double pi = __ldcg(&fl.pchain[static_cast<size_t>(b) * (g + 2) + i]);
+    double h = pi;
+    if (i < g) {
+        const double Si = __ldcg(&fl.S[static_cast<size_t>(b) * (g + 1) + i]);
+        h = Si > 0.0 ? Si / (Si + 1.0 - pi) : 0.0;
+    }
+    return h > 0.0 && static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + i - 1]) <= h;
+}
+// The selected position is the highest candidate that passes its test, so the candidates are
+// swept from the top, one at a time: start the highest one on hold below `below`.
+static __device__ void f_release_next(const FlowScratch& fl, int b, int g, int below) {
+    for (int c = below - 1; c >= 0; --c) {
+        const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
+        if (ld_volatile(&fl.rel[ci]) == kRelHold) { atomicExch(&fl.rel[ci], kRelSweep); return; }
+    }
+}
+// Position i has just been completed (S_i and its candidate token are in scratch): either it is
+// the selected one, and no lower position is wanted, or the next lower candidate is started.
+// Returns the number of positions that are complete through this call (itself included).
+static __device__ unsigned f_after_position(const Params& prm, const FlowScratch& fl, int b, int i) {
+    const int g = prm.gamma;
+    unsigned done = 1;
+    if (f_position_selected(prm, fl, b, i)) {
+        for (int c = i - 1; c >= 0; --c) {
+            const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
+            if (ld_volatile(&fl.rel[ci]) != kRelHold) continue;
+            if (c < g) fl.S[ci] = 0.0;
+            fl.cand[ci] = -1;
+            __threadfence();
+            atomicExch(&fl.rel[ci], kRelSkip);
+            ++done;
+        }
+    } else {
+        f_release_next(fl, b, g, i);
+    }
+    return done;
+}
+
 // ---- a row is complete (one thread): its normalisers are published, then the recursion
 // advances over every complete row of the block ----
 template <int DT>
@@ -246,6 +290,7 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
     __threadfence();
     const bool all_positions = prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
     unsigned nskip = 0;
+    bool folded = false;
     unsigned c = ld_volatile(&fl.chain[b]);
     while (c <= static_cast<unsigned>(g) && ld_volatile(&fl.row_done[static_cast<size_t>(b) * (g + 1) + c]) != 0u) {
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
@@ -272,9 +317,13 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
             ++nskip;
         }
         __threadfence();                       // p, cscale are visible ...
-        atomicExch(&fl.rel[ci], need ? kRelSweep : kRelSkip);   // ... before the row's sweep-2 items may start
+        // ... before the row's sweep-2 items may start.  Candidates wait (on hold) until the whole
+        // block is folded and every higher candidate has been rejected.
+        atomicExch(&fl.rel[ci], need ? (all_positions ? kRelSweep : kRelHold) : kRelSkip);
         ++c;
+        folded = true;
     }
+    if (folded && c == static_cast<unsigned>(g) + 1u && !all_positions) f_release_next(fl, b, g, g + 1);
     *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
     __threadfence();
     atomicExch(&fl.lock[b], 0u);
@@ -309,12 +358,7 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
 // ---- a position is complete (one warp): S_r from the segment totals, and the candidate Y_r.
 // `segs` holds the nseg totals of the row's segments in index order; range(s, v0, v1) gives the
 // vectors [v0, v1) of segment s. ----
-// a segment total as stored: plain, or (ENC) with its lowest mantissa bit set to mark it written
-template <bool ENC> __device__ __forceinline__ float f_seg(const float* p) {
-    const float v = __ldcg(p);
-    return ENC ? __uint_as_float(__float_as_uint(v) & ~1u) : v;
-}
-template <int DT, bool ENC, class RangeFn>
+template <int DT, class RangeFn>
 __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, bool have_q,
                                     const char* rowP, const char* rowQ, float cp, float nMP, float nMQ,
                                     int nseg, const float* segs, int lane, RangeFn range) {
@@ -334,7 +378,7 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int i = 128 * grp + 4 * lane + j;
-            w[j] = i < nseg ? f_seg<ENC>(&segs[i]) : 0.f;
+            w[j] = i < nseg ? __ldcg(&segs[i]) : 0.f;
         }
         sd += (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
               (static_cast<double>(w[2]) + static_cast<double>(w[3]));
@@ -360,7 +404,7 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int i = 128 * grp + 4 * lane + j;
-                w[j] = i < nseg ? f_seg<ENC>(&segs[i]) : 0.f;
+                w[j] = i < nseg ? __ldcg(&segs[i]) : 0.f;
             }
             const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
             float inc = l4;
@@ -413,7 +457,9 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
     if (lane == 0) {
         fl.cand[ri] = found;
         __threadfence();
-        if (atomicAdd(&fl.cand_cnt[b], 1u) == static_cast<unsigned>(g)) {
+        const bool all_positions = prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
+        const unsigned done = all_positions ? 1u : f_after_position(prm, fl, b, r);
+        if (atomicAdd(&fl.cand_cnt[b], done) + done == static_cast<unsigned>(g) + 1u) {
             __threadfence();
             f_finalize_block(prm, fl, b);
         }

@@ -54,15 +54,9 @@ int flow_max_ctas_per_sm(int dtype);
 int flow_pick_chunks(long long units, int B, int gamma, long long nctas);
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream);
 
-// Group kernel (Block Verification, 128-bit path): same scratch with nch = CTAs per group and
-// `segs` residual totals per row.  Cooperative launch of G * NG CTAs.
+// The same scratch with any number of residual totals per row.
 size_t flow_scratch_bytes_segs(int B, int gamma, int nch, int segs, size_t* zero_bytes);
 void flow_scratch_layout_segs(void* base, int B, int gamma, int nch, int segs, FlowScratch* fl);
-int group_share_vectors();
-int group_segments_per_share();
-int group_max_lag();
-int group_max_ctas_per_sm(int dtype);
-cudaError_t launch_group(const Params& prm, const FlowScratch& fl, int dtype, int G, int NG, int L, cudaStream_t stream);
 
 // Resident kernel (Block Verification only, 128-bit path): a thread holds up to `nk`
 // vectors per row, nk in {2, 4, 8}.

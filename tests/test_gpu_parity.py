@@ -61,7 +61,7 @@ def test_every_cluster_width(cluster, algo, monkeypatch):
     parity_case(random_inputs(7, 3, 5000, "f32", seed=cluster + 10), algo)
 
 
-@pytest.mark.parametrize("kernel", ["flow", "group", "cluster", "resident", "stream"])
+@pytest.mark.parametrize("kernel", ["flow", "cluster", "resident", "stream"])
 def test_every_block_verification_kernel(kernel, monkeypatch):
     # the library has several kernels for Algorithm 2; each must match the oracle
     monkeypatch.setenv("BV_KERNEL", kernel)
