@@ -151,7 +151,12 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
                 if (v >= 1 && v <= bv::kFlowMaxChunks) nch = v;
             }
             size_t zero_bytes = 0;
-            const size_t need = bv::flow_scratch_bytes(B, gamma, nch, &zero_bytes);
+            int np = bv::flow_pick_pieces(units);
+            if (const char* env = std::getenv("BV_FLOW_PIECES")) {
+                const int v = std::atoi(env);
+                if (v >= 1 && v <= bv::kFlowMaxChunks) np = v;
+            }
+            const size_t need = bv::flow_scratch_bytes(B, gamma, nch, np, &zero_bytes);
             const int slot = static_cast<int>(d->flow_calls++ % 4);
             if (d->flow_bytes[slot] < need) {
                 if (d->flow_ws[slot]) cudaFree(d->flow_ws[slot]);
@@ -162,7 +167,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
                 d->flow_bytes[slot] = need;
             }
             bv::FlowScratch fl;
-            bv::flow_scratch_layout(d->flow_ws[slot], B, gamma, nch, &fl);
+            bv::flow_scratch_layout(d->flow_ws[slot], B, gamma, nch, np, &fl);
             if (const char* env = std::getenv("BV_FLOW_DEPTH")) {
                 const int v = std::atoi(env);
                 if (v >= 2 && v <= 3) fl.depth = v;

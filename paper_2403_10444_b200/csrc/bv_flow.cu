@@ -25,9 +25,10 @@ namespace bv {
 constexpr int kFThreads = 512;
 constexpr int kFWarps = kFThreads / 32;
 
-__device__ __forceinline__ void chunk_range(const FlowCtx& cx, int ch, int warp, int& w0, int& w1) {
-    const int u0 = static_cast<int>(static_cast<long long>(cx.units) * ch / cx.nch);
-    const int u1 = static_cast<int>(static_cast<long long>(cx.units) * (ch + 1) / cx.nch);
+// vectors [w0, w1) of a row that worker `warp` takes of part `ch` out of `nparts`
+__device__ __forceinline__ void chunk_range(const FlowCtx& cx, int nparts, int ch, int warp, int& w0, int& w1) {
+    const int u0 = static_cast<int>(static_cast<long long>(cx.units) * ch / nparts);
+    const int u1 = static_cast<int>(static_cast<long long>(cx.units) * (ch + 1) / nparts);
     w0 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * warp / kFWarps);
     w1 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * (warp + 1) / kFWarps);
 }
@@ -48,11 +49,9 @@ struct FlowDesc {
     float cp, nMP, nMQ;         // sweep 2: p_r Z_Q / Z_P and minus the row references
 };
 
-constexpr int kFDefer = 8;     // chunks a CTA may hold between their first and their second sweep
 
 struct FlowShared {
     FlowDesc desc[kFDesc];
-    FlowDesc defer[kFDefer];
     unsigned long long full[kFDesc];    // the service warp has filled desc[i]
     unsigned long long done[kFDesc];    // all 16 worker warps have left their partials of desc[i]
     float part_M[kFDesc][2][kFWarps];   // sweep 1: references of P and Q per worker warp
@@ -91,18 +90,19 @@ template <int DT>
 __device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int slot,
                                const FlowDesc& d, int lane) {
     const int ri = d.ri;
-    const int nseg = cx.nch * kFWarps;
+    const int np = fl.np;
+    const int nseg = np * kFWarps;
     float* segs = fl.seg_tot + static_cast<size_t>(ri) * nseg;
     if (lane < kFWarps) segs[d.ch * kFWarps + lane] = sh.part_s[slot][0][lane];
     __threadfence();
     __syncwarp();
     int last = 0;
-    if (lane == 0) last = atomicAdd(&fl.s2_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u;
+    if (lane == 0) last = atomicAdd(&fl.s2_cnt[ri], 1u) == static_cast<unsigned>(np) - 1u;
     last = __shfl_sync(0xffffffffu, last, 0);
     if (!last) return;
 
     f_position_complete<DT>(prm, fl, cx, ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, nseg, segs, lane,
-                            [&](int sel, int& s0, int& s1) { chunk_range(cx, sel / kFWarps, sel % kFWarps, s0, s1); });
+                            [&](int sel, int& s0, int& s1) { chunk_range(cx, np, sel / kFWarps, sel % kFWarps, s0, s1); });
 }
 
 // ---- worker warps: one warp's segment of one item ----
@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         // the next sweep-1 item, or kExit when all have been handed out; never blocks
         auto take = [&](FlowDesc& d) {
             unsigned t = 0;
-            if (lane == 0) t = atomicAdd(&fl.counters[0], 1u);
+            if (lane == 0) t = atomicAdd(&fl.counters[kCtrTicket], 1u);
             t = __shfl_sync(0xffffffffu, t, 0);
             if (t >= total_s1) { d.kind = kExit; return; }
             const int ri = static_cast<int>(t / cx.nch), ch = static_cast<int>(t % cx.nch);
@@ -227,58 +227,70 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                            : nullptr;
             d.cp = 1.f; d.nMP = 0.f; d.nMQ = 0.f;
         };
-        // A chunk's second sweep may start once its row has been folded into the recursion.  That
-        // is done by whoever completes the row, possibly this very warp a few items from now, so
-        // the warp never blocks on it: it keeps a list of its swept chunks and asks about all of
-        // them on every round (one load each, side by side in the lanes).
-        auto fill_scalars = [&](FlowDesc& d) {
+        // Rows whose second sweep has been started stand in a queue, each cut into np pieces.  A
+        // piece is claimed by a ticket from the queue's head counter, drawn only while the head is
+        // seen behind the tail; a ticket that still runs ahead of the tail (several CTAs drew at
+        // once) is kept until its row arrives.  -1: no piece right now.
+        int held = -1;                    // (lane 0) a ticket drawn and not yet used
+        auto take_piece = [&]() -> int {
+            int t = -1;
+            if (lane == 0) {
+                unsigned avail = ld_volatile(&fl.counters[kCtrQueued]) * static_cast<unsigned>(fl.np);
+                if (held < 0 && ld_volatile(&fl.counters[kCtrPieces]) < avail)
+                    held = static_cast<int>(atomicAdd(&fl.counters[kCtrPieces], 1u));
+                if (held >= 0 && static_cast<unsigned>(held) < avail) { t = held; held = -1; }
+            }
+            return __shfl_sync(0xffffffffu, t, 0);
+        };
+        auto piece_desc = [&](int t, FlowDesc& d) -> bool {
+            unsigned e = 0;
+            for (unsigned spins = 0; (e = ld_volatile(&fl.s2q[t / fl.np])) == 0u; ++spins)   // the entry follows the tail at once
+                if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
+            const int ri = static_cast<int>(e - 1u);
+            const int r = ri % (g + 1), b = ri / (g + 1);
+            d.kind = kSweep2; d.ri = ri; d.ch = t % fl.np; d.have_q = r < g;
+            d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
+            d.rowQ = r < g ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
+                           : nullptr;
+            d.cp = 1.f;
             __threadfence();
-            if (d.have_q) d.cp = __ldcg(&fl.cscale[d.ri]);
-            d.nMP = -static_cast<float>(__ldcg(&fl.rowZ[d.ri].MP));
-            d.nMQ = -static_cast<float>(__ldcg(&fl.rowZ[d.ri].MQ));
+            if (d.have_q) d.cp = __ldcg(&fl.cscale[ri]);
+            d.nMP = -static_cast<float>(__ldcg(&fl.rowZ[ri].MP));
+            d.nMQ = -static_cast<float>(__ldcg(&fl.rowZ[ri].MQ));
+            return true;
         };
         auto publish = [&](const FlowDesc& d, int q) {
             if (lane == 0) { sh.desc[q % kFDesc] = d; mbar_arrive(smem_u32(&sh.full[q % kFDesc])); }
             __syncwarp();
         };
         int q = 0, n = 0, qexit = -1;     // items published / post-processed; index of the exit descriptor
-        int ndef = 0;                     // chunks swept once, waiting for their second sweep
-        int s1_flying = 0;                // sweep-1 items published and not yet post-processed
         bool exhausted = false;           // the ticket counter has run past the last item
         unsigned idle = 0;
         for (;;) {
             // 1. publish what can be published (a slot is free once its previous item is post-processed)
             while (qexit < 0 && q - n < fl.depth) {
-                // (a) second sweep of the oldest waiting chunk whose row has been folded
-                unsigned rel = 0;
-                if (lane < ndef) rel = ld_volatile(&fl.rel[sh.defer[lane].ri]);
-                const unsigned okmask = __ballot_sync(0xffffffffu, rel == kRelSweep || rel == kRelSkip);
-                if (okmask) {
-                    const int i = __ffs(okmask) - 1;
-                    const bool wanted = __shfl_sync(0xffffffffu, rel, i) == kRelSweep;
-                    FlowDesc d = sh.defer[i];
-                    if (wanted) fill_scalars(d);
-                    __syncwarp();
-                    if (lane == 0) for (int j = i; j + 1 < ndef; ++j) sh.defer[j] = sh.defer[j + 1];
-                    --ndef;
-                    __syncwarp();
-                    if (!wanted) continue;          // nothing depends on this position: no second sweep
+                FlowDesc d;
+                // (a) a piece of a row that waits for its second sweep: they are few and others wait for them
+                const int t = take_piece();
+                if (t >= 0) {
+                    if (!piece_desc(t, d)) { exhausted = true; break; }
                     publish(d, q);
                     ++q;
                     continue;
                 }
-                // (b) a new sweep-1 item, unless the list could overflow when those in flight finish
-                if (exhausted) {
-                    if (ndef == 0 && s1_flying == 0) { FlowDesc d; d.kind = kExit; publish(d, q); qexit = q; ++q; }
-                    break;
+                // (b) a new sweep-1 item
+                if (!exhausted) {
+                    take(d);
+                    if (d.kind == kExit) { exhausted = true; continue; }
+                    publish(d, q);
+                    ++q;
+                    continue;
                 }
-                if (ndef + s1_flying >= kFDefer) break;
-                FlowDesc d;
-                take(d);
-                if (d.kind == kExit) { exhausted = true; continue; }
-                publish(d, q);
-                ++q;
-                ++s1_flying;
+                // (c) nothing to start: leave once every block is finished
+                if (q == n && ld_volatile(&fl.counters[kCtrBlocks]) >= static_cast<unsigned>(cx.B)) {
+                    d.kind = kExit; publish(d, q); qexit = q; ++q;
+                }
+                break;
             }
             // 2. the oldest item in flight: wait for the workers, then do what follows its sweep
             const int in_flight_end = qexit >= 0 ? qexit : q;
@@ -288,10 +300,6 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 mbar_wait_now(smem_u32(&sh.done[slot]), static_cast<uint32_t>(n / kFDesc) & 1u, prm.status);
                 if (d.kind == kSweep1) {
                     f_after_sweep1<DT>(prm, fl, cx, sh, slot, d.ri, d.ch, lane);
-                    if (lane == 0) { sh.defer[ndef] = d; sh.defer[ndef].kind = kSweep2; }   // its second sweep is ours
-                    ++ndef;
-                    --s1_flying;
-                    __syncwarp();
                 } else {
                     f_after_sweep2<DT>(prm, fl, cx, sh, slot, d, lane);
                 }
@@ -301,8 +309,9 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             }
             if (qexit >= 0) break;
             // 3. nothing in flight and the next item waits for a row that another CTA completes
-            __nanosleep(128);
-            if (++idle > (1u << 23)) { if (prm.status) atomicExch(prm.status, 1); break; }
+            // (all idle CTAs look at the same counters: wait long enough not to crowd those who work)
+            __nanosleep(idle < 4 ? 500 : 2000);
+            if (++idle > (1u << 21)) { if (prm.status) atomicExch(prm.status, 1); break; }
         }
         if (qexit < 0) {      // gave up: release the workers
             FlowDesc d; d.kind = kExit;
@@ -323,7 +332,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         const char* rowP = sh.desc[slot].rowP;
         const char* rowQ = sh.desc[slot].rowQ;
         int w0, w1;
-        chunk_range(cx, sh.desc[slot].ch, warp, w0, w1);
+        chunk_range(cx, kind == kSweep1 ? cx.nch : fl.np, sh.desc[slot].ch, warp, w0, w1);
         float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
         if (kind == kSweep1) {
             if (have_q) f_sweep_segment<DT, true, kSweep1>(sb, rowP, rowQ, w0, w1, lane, kf, 1.f, 0.f, 0.f, MPw, sP, MQw, sQ);
@@ -348,17 +357,14 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
 // ---------------------------------------------------------------------------
 static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
-size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes) {
-    return flow_scratch_bytes_segs(B, gamma, nch, nch * kFWarps, zero_bytes);
-}
-
-size_t flow_scratch_bytes_segs(int B, int gamma, int nch, int segs, size_t* zero_bytes) {
+size_t flow_scratch_bytes(int B, int gamma, int nch, int np, size_t* zero_bytes) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
+    const size_t segs = static_cast<size_t>(np) * kFWarps;
     size_t z = 0;
     z += up256(kCounterWords * sizeof(unsigned));   // counters
     z += 3 * up256(rows * sizeof(unsigned));        // row_cnt, row_done, s2_cnt
     z += 4 * up256(static_cast<size_t>(B) * sizeof(unsigned));   // cand_cnt, chain, lock, bad
-    z += up256(rows * sizeof(unsigned));            // rel
+    z += 2 * up256(rows * sizeof(unsigned));        // rel, s2q
     if (zero_bytes) *zero_bytes = z;
     size_t n = z;
     n += up256(rows * nch * sizeof(RowZ));          // part
@@ -372,12 +378,9 @@ size_t flow_scratch_bytes_segs(int B, int gamma, int nch, int segs, size_t* zero
     return n;
 }
 
-void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl) {
-    flow_scratch_layout_segs(base, B, gamma, nch, nch * kFWarps, fl);
-}
-
-void flow_scratch_layout_segs(void* base, int B, int gamma, int nch, int segs, FlowScratch* fl) {
+void flow_scratch_layout(void* base, int B, int gamma, int nch, int np, FlowScratch* fl) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
+    const size_t segs = static_cast<size_t>(np) * kFWarps;
     char* p = static_cast<char*>(base);
     auto take = [&](size_t bytes) { char* q = p; p += up256(bytes); return q; };
     fl->counters = reinterpret_cast<unsigned*>(take(kCounterWords * sizeof(unsigned)));
@@ -389,6 +392,7 @@ void flow_scratch_layout_segs(void* base, int B, int gamma, int nch, int segs, F
     fl->lock = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->bad = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->rel = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
+    fl->s2q = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->part = reinterpret_cast<RowZ*>(take(rows * nch * sizeof(RowZ)));
     fl->rowZ = reinterpret_cast<RowZ*>(take(rows * sizeof(RowZ)));
     fl->pchain = reinterpret_cast<double*>(take(static_cast<size_t>(B) * (gamma + 2) * sizeof(double)));
@@ -399,8 +403,20 @@ void flow_scratch_layout_segs(void* base, int B, int gamma, int nch, int segs, F
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
     fl->nch = nch;
+    fl->np = np;
     fl->depth = 2;      // one item being swept, one queued: the service warp reacts sooner to released rows
-    fl->segs = segs;
+    fl->segs = static_cast<int>(segs);
+}
+
+// Pieces per row in the second sweep.  Only the few rows that may hold the selected position are
+// swept again, and the candidates of a block are swept one after the other, so their rows are cut
+// finer than in the first sweep: more CTAs share a row and the chain of a block gets shorter.  A
+// piece keeps at least 2048 vectors.
+int flow_pick_pieces(long long units) {
+    long long np = units / 4000;
+    if (np < 1) np = 1;
+    if (np > 8) np = 8;
+    return static_cast<int>(np);
 }
 
 // Chunks per row.  An item should be large next to what it costs to hand it out (about

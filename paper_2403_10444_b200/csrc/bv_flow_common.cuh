@@ -12,7 +12,11 @@ namespace bv {
 
 
 enum : int { kExit = 0, kSweep1 = 1, kSweep2 = 2 };
-constexpr int kCounterWords = 32;   // [0]: the ticket counter
+// Global counters, one per 128-byte line so that polling one does not slow the others down:
+// the sweep-1 ticket counter, rows queued for their second sweep, pieces of queued rows handed
+// out, blocks finished.
+constexpr int kCounterWords = 128;
+enum : int { kCtrTicket = 0, kCtrQueued = 32, kCtrPieces = 64, kCtrBlocks = 96 };
 // rel[row]: 0 = not folded yet, then whether the row's second sweep is wanted
 enum : unsigned { kRelSweep = 1u, kRelSkip = 2u, kRelHold = 3u };   // hold: wanted only if every higher candidate is rejected
 
@@ -197,6 +201,8 @@ static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl
             if (i < g && prm.out_lse_d) prm.out_lse_d[o0] = static_cast<float>((static_cast<double>(z.MQ) + log2(z.ZQ)) * ln2);
         }
     }
+    __threadfence();
+    atomicAdd(&fl.counters[kCtrBlocks], 1u);      // (CTAs leave when every block is finished)
 }
 
 // ---- which positions get a second sweep (one thread each) ----
@@ -215,10 +221,18 @@ static __device__ bool f_position_selected(const Params& prm, const FlowScratch&
 }
 // The selected position is the highest candidate that passes its test, so the candidates are
 // swept from the top, one at a time: start the highest one on hold below `below`.
+static __device__ void f_start_second_sweep(const FlowScratch& fl, size_t ci) {
+    atomicExch(&fl.rel[ci], kRelSweep);
+    // the row joins the queue from which every CTA draws pieces; the entry itself says when it is
+    // written (the queue starts at zero), so the order of the two stores does not matter
+    __threadfence();
+    const unsigned slot = atomicAdd(&fl.counters[kCtrQueued], 1u);
+    atomicExch(&fl.s2q[slot], static_cast<unsigned>(ci) + 1u);
+}
 static __device__ void f_release_next(const FlowScratch& fl, int b, int g, int below) {
     for (int c = below - 1; c >= 0; --c) {
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
-        if (ld_volatile(&fl.rel[ci]) == kRelHold) { atomicExch(&fl.rel[ci], kRelSweep); return; }
+        if (ld_volatile(&fl.rel[ci]) == kRelHold) { f_start_second_sweep(fl, ci); return; }
     }
 }
 // Position i has just been completed (S_i and its candidate token are in scratch): either it is
@@ -319,7 +333,8 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
         __threadfence();                       // p, cscale are visible ...
         // ... before the row's sweep-2 items may start.  Candidates wait (on hold) until the whole
         // block is folded and every higher candidate has been rejected.
-        atomicExch(&fl.rel[ci], need ? (all_positions ? kRelSweep : kRelHold) : kRelSkip);
+        if (need && all_positions) f_start_second_sweep(fl, ci);
+        else atomicExch(&fl.rel[ci], need ? kRelHold : kRelSkip);
         ++c;
         folded = true;
     }

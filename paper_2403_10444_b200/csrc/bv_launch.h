@@ -25,7 +25,8 @@ cudaError_t launch_cluster(const Params& prm, int algo, int dtype, int cluster, 
 // when the kernel starts.
 struct RowZ { double MP, ZP, MQ, ZQ; };   // row (or chunk) references and sums of 2^{z k - M}
 struct FlowScratch {
-    unsigned* counters;   // [0]: ticket counter of the sweep-1 items
+    unsigned* counters;   // ticket counter of the sweep-1 items, rows queued for their second sweep, pieces of
+                          // queued rows handed out, blocks finished (one 128-byte line each)
     unsigned* row_cnt;    // [B (gamma+1)] sweep-1 chunks finished per row
     unsigned* row_done;   // [B (gamma+1)] row normalisers published
     unsigned* s2_cnt;     // [B (gamma+1)] sweep-2 chunks finished per position
@@ -33,30 +34,30 @@ struct FlowScratch {
     unsigned* chain;      // [B] rows folded into the recursion
     unsigned* lock;       // [B]
     unsigned* bad;        // [B] data fault seen
-    unsigned* rel;        // [B (gamma+1)] row folded into the recursion: its sweep-2 items may run
+    unsigned* rel;        // [B (gamma+1)] row folded into the recursion, and what becomes of its second sweep
+    unsigned* s2q;        // [B (gamma+1)] queue of rows whose second sweep has been started (row index + 1)
     RowZ* part;           // [B (gamma+1) nch]
     RowZ* rowZ;           // [B (gamma+1)]
     double* pchain;       // [B (gamma+2)]
     float* cscale;        // [B (gamma+1)] p_r Z_Q / Z_P
     double* ratio;        // [B (gamma+1)] P_r(X_{r+1}) / Q_r(X_{r+1})
     double* zratio;       // [B (gamma+1)] Z_Q / Z_P
-    float* seg_tot;       // [B (gamma+1) nch 16]
+    float* seg_tot;       // [B (gamma+1) segs]
     double* S;            // [B (gamma+1)]
     int* cand;            // [B (gamma+1)]
-    int nch;              // chunks per row (1 .. kFlowMaxChunks)
+    int nch;              // chunks per row in the first sweep (1 .. kFlowMaxChunks)
+    int np;               // pieces per row in the second sweep (1 .. kFlowMaxChunks)
     int depth;            // flow kernel: descriptors a CTA may have published and not yet post-processed (2 or 3)
     int segs;             // residual totals kept per row
 };
 constexpr int kFlowMaxChunks = 32;
-size_t flow_scratch_bytes(int B, int gamma, int nch, size_t* zero_bytes);
-void flow_scratch_layout(void* base, int B, int gamma, int nch, FlowScratch* fl);
+size_t flow_scratch_bytes(int B, int gamma, int nch, int np, size_t* zero_bytes);
+void flow_scratch_layout(void* base, int B, int gamma, int nch, int np, FlowScratch* fl);
+int flow_pick_pieces(long long units);
 int flow_max_ctas_per_sm(int dtype);
 int flow_pick_chunks(long long units, int B, int gamma, long long nctas);
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream);
 
-// The same scratch with any number of residual totals per row.
-size_t flow_scratch_bytes_segs(int B, int gamma, int nch, int segs, size_t* zero_bytes);
-void flow_scratch_layout_segs(void* base, int B, int gamma, int nch, int segs, FlowScratch* fl);
 
 // Resident kernel (Block Verification only, 128-bit path): a thread holds up to `nk`
 // vectors per row, nk in {2, 4, 8}.

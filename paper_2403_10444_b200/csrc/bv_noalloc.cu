@@ -85,7 +85,8 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     const long long units = static_cast<long long>(row_bytes / 16);
     const int nch = bv::flow_pick_chunks(units, B, gamma, static_cast<long long>(d.sm_count) * per_sm);
     size_t zero_bytes = 0;
-    const size_t need = bv::flow_scratch_bytes(B, gamma, nch, &zero_bytes) + 256;   // + the status word
+    const int np = bv::flow_pick_pieces(units);
+    const size_t need = bv::flow_scratch_bytes(B, gamma, nch, np, &zero_bytes) + 256;   // + the status word
     if (need > kScratchBytes) return BV_ERR_TOO_LARGE;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -96,7 +97,7 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     if (cudaMemsetAsync(status_word, 0, 256, s) != cudaSuccess) { cudaGetLastError(); return BV_ERR_CUDA; }
 
     bv::FlowScratch fl;
-    bv::flow_scratch_layout(d.scratch, B, gamma, nch, &fl);
+    bv::flow_scratch_layout(d.scratch, B, gamma, nch, np, &fl);
     bv::Params prm{};
     prm.tgt = tgt; prm.drf = drf; prm.tok = tok; prm.uni = uni;
     prm.B = B; prm.gamma = gamma; prm.V = V;
