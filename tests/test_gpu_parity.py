@@ -21,6 +21,13 @@ def parity_case(inp, algo, check_diag=True):
     rep = compare(algo, ref, ot, ol, diag, inp)
     print(rep)
     assert_parity(rep, check_diag)
+    # the entry points without diagnostic outputs are the ones a server calls (and the bench times);
+    # for Algorithm 2 they leave out the second sweep of positions that cannot be selected, so
+    # their tokens are checked against the oracle on their own
+    ot2, ol2 = run_cuda(algo, inp, diagnostics=False)[:2]
+    rep2 = compare(algo, ref, ot2, ol2, None, inp)
+    print(rep2)
+    assert_parity(rep2, False)
     return rep
 
 
@@ -179,3 +186,16 @@ def test_launch_count_and_nonblocking_stream():
     assert bv.bv_last_launch_count() == 1
     ref = run_oracle(oracle.BLOCK_VERIFY, inp)
     assert np.array_equal(ol.cpu().numpy(), ref.out_len)
+
+
+@pytest.mark.parametrize("sigma_d", [0.05, 0.5, 2.0])
+def test_skipped_second_sweeps_change_nothing(sigma_d):
+    # Without diagnostic outputs Algorithm 2's second sweep runs only for positions with
+    # eta_i <= p_i (h_i <= p_i always), from the top down, until one is selected.  The emitted
+    # tokens must be bit for bit those of the call that computes every position, at every
+    # acceptance level: nearly all positions wanted (small noise) or nearly none (large).
+    for seed in range(3):
+        inp = random_inputs(48, 6, 12000, "bf16", seed=100 + seed, T=0.9, sigma_d=sigma_d)
+        full = run_cuda(oracle.BLOCK_VERIFY, inp, diagnostics=True)
+        fast = run_cuda(oracle.BLOCK_VERIFY, inp, diagnostics=False)
+        assert torch.equal(full[0], fast[0]) and torch.equal(full[1], fast[1])
