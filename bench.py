@@ -302,11 +302,11 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (a B=128 capture scaled by the batch: the traffic grows in
-# proportion to B); None for a workload or kernel with no capture.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the one-pass
+# ncu capture of this command at full size that profiles/ summarises; None for a workload or
+# kernel with no capture.
 TRAFFIC_BYTES = {
-    ("c4", "block", "verify_flow_kernel"): 4360644096,
+    ("c4", "block", "verify_flow_kernel"): 2579547648,
 }
 
 

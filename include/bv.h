@@ -71,6 +71,11 @@ enum { BV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024 };
  *   stream        a cudaStream_t (NULL = the default stream)
  * Rows whose byte length is a multiple of 16 with 16-byte aligned bases use the
  * 128-bit path; any other V >= 1 is served by an element-wise path.
+ * Since S_i <= p_i, h_i <= p_i: on the 128-bit path S_i is evaluated only for
+ * positions with eta_i <= p_i, from the highest down to the first one that passes
+ * eta_i <= h_i; tau and Y are those of the full evaluation (bv_verify_ex does the
+ * full evaluation).  The cost of a call therefore depends on how many drafted
+ * tokens are accepted.
  */
 int bv_verify(const void* target_logits, const void* draft_logits,
               const int32_t* draft_tokens, const float* uniforms,
@@ -139,8 +144,8 @@ int tv_verify_host(const void* target_logits, const void* draft_logits,
  * the library image, present on every GPU that loads the library until the process exits.
  *
  * Limits and rules that bv_verify() does not have:
- *   - the scratch needed grows with B (gamma+1), about 0.9 KB per logit row pair at large V
- *     (B = 256, gamma = 8, V = 256000 needs 2.0 MiB); a problem that needs more than the
+ *   - the scratch needed grows with B (gamma+1), about 0.7 KB per logit row pair at large V
+ *     (B = 256, gamma = 8, V = 256000 needs 1.5 MiB); a problem that needs more than the
  *     array returns BV_ERR_TOO_LARGE and launches nothing;
  *   - rows must be whole 16-byte vectors on 16-byte aligned bases (V a multiple of 8 for
  *     bf16, of 4 for fp32), else BV_ERR_UNSUPPORTED;
