@@ -122,7 +122,8 @@ __device__ __forceinline__ void f_sweep_segment(uint32_t sb, const char* rowP, c
     const char* gP = rowP + static_cast<size_t>(w0 + lane) * 16;
     const char* gQ = HAVEQ ? rowQ + static_cast<size_t>(w0 + lane) * 16 : gP;
     // sweep 1 asks L2 to keep the rows (they are read again soon); sweep 2 marks them as done with
-    const uint64_t pol = KIND == kSweep1 ? l2_policy_evict_last() : l2_policy_evict_first();
+    // no row is needed again soon (the few second sweeps come long after the first): stream past L2
+    const uint64_t pol = l2_policy_evict_first();
     auto fetch_step = [&](int k, int j) {                    // step k goes to slots 2j, 2j+1 (j = k & 3)
         if (k < nsteps) {
             const bool ok = (k + 1 < nsteps) || lane < nlast;
