@@ -213,16 +213,18 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         // =============================== service warp ===============================
         // takes tickets, waits for what a sweep-2 item needs, hands descriptors to the workers,
         // and does everything that follows a sweep, so that the workers never stop streaming
-        const unsigned total_s1 = static_cast<unsigned>(cx.B) * (g + 1) * cx.nch;
+        // tickets cover the rows that every block needs: target and draft rows 0 .. gamma-1
+        const unsigned total_s1 = static_cast<unsigned>(cx.B) * g * cx.nch;
         // the next sweep-1 item, or kExit when all have been handed out; never blocks
         auto take = [&](FlowDesc& d) {
             unsigned t = 0;
             if (lane == 0) t = atomicAdd(&fl.counters[kCtrTicket], 1u);
             t = __shfl_sync(0xffffffffu, t, 0);
             if (t >= total_s1) { d.kind = kExit; return; }
-            const int ri = static_cast<int>(t / cx.nch), ch = static_cast<int>(t % cx.nch);
-            const int r = ri % (g + 1), b = ri / (g + 1);
-            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = r < g;
+            const int ch = static_cast<int>(t % cx.nch);
+            const int r = static_cast<int>(t / cx.nch) % g, b = static_cast<int>(t / cx.nch) / g;
+            const int ri = b * (g + 1) + r;
+            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = 1;
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
             d.rowQ = r < g ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
                            : nullptr;
@@ -232,16 +234,31 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         // piece is claimed by a ticket from the queue's head counter, drawn only while the head is
         // seen behind the tail; a ticket that still runs ahead of the tail (several CTAs drew at
         // once) is kept until its row arrives.  -1: no piece right now.
-        int held = -1;                    // (lane 0) a ticket drawn and not yet used
-        auto take_piece = [&]() -> int {
+        int held = -1, held_late = -1;    // (lane 0) tickets drawn and not yet used
+        auto claim = [&](int queued, int taken, int per_row, int& hold) -> int {
             int t = -1;
             if (lane == 0) {
-                unsigned avail = ld_volatile(&fl.counters[kCtrQueued]) * static_cast<unsigned>(fl.np);
-                if (held < 0 && ld_volatile(&fl.counters[kCtrPieces]) < avail)
-                    held = static_cast<int>(atomicAdd(&fl.counters[kCtrPieces], 1u));
-                if (held >= 0 && static_cast<unsigned>(held) < avail) { t = held; held = -1; }
+                const unsigned avail = ld_volatile(&fl.counters[queued]) * static_cast<unsigned>(per_row);
+                if (hold < 0 && ld_volatile(&fl.counters[taken]) < avail)
+                    hold = static_cast<int>(atomicAdd(&fl.counters[taken], 1u));
+                if (hold >= 0 && static_cast<unsigned>(hold) < avail) { t = hold; hold = -1; }
             }
             return __shfl_sync(0xffffffffu, t, 0);
+        };
+        auto take_piece = [&]() -> int { return claim(kCtrQueued, kCtrPieces, fl.np, held); };
+        // likewise the chunks of last target rows whose first sweep has been asked for
+        auto late_desc = [&](FlowDesc& d) -> bool {
+            const int t = claim(kCtrLateQueued, kCtrLateChunks, cx.nch, held_late);
+            if (t < 0) return false;
+            unsigned e = 0;
+            for (unsigned spins = 0; (e = ld_volatile(&fl.lq[t / cx.nch])) == 0u; ++spins)
+                if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
+            const int ri = static_cast<int>(e - 1u);
+            d.kind = kSweep1; d.ri = ri; d.ch = t % cx.nch; d.have_q = 0;
+            d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
+            d.rowQ = nullptr;
+            d.cp = 1.f; d.nMP = 0.f; d.nMQ = 0.f;
+            return true;
         };
         auto piece_desc = [&](int t, FlowDesc& d) -> bool {
             unsigned e = 0;
@@ -279,7 +296,13 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                     ++q;
                     continue;
                 }
-                // (b) a new sweep-1 item
+                // (b) a chunk of a last target row that turned out to be wanted
+                if (late_desc(d)) {
+                    publish(d, q);
+                    ++q;
+                    continue;
+                }
+                // (c) a new sweep-1 item
                 if (!exhausted) {
                     take(d);
                     if (d.kind == kExit) { exhausted = true; continue; }
@@ -287,7 +310,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                     ++q;
                     continue;
                 }
-                // (c) nothing to start: leave once every block is finished
+                // (d) nothing to start: leave once every block is finished
                 if (q == n && ld_volatile(&fl.counters[kCtrBlocks]) >= static_cast<unsigned>(cx.B)) {
                     d.kind = kExit; publish(d, q); qexit = q; ++q;
                 }
@@ -366,6 +389,7 @@ size_t flow_scratch_bytes(int B, int gamma, int nch, int np, size_t* zero_bytes)
     z += 3 * up256(rows * sizeof(unsigned));        // row_cnt, row_done, s2_cnt
     z += 4 * up256(static_cast<size_t>(B) * sizeof(unsigned));   // cand_cnt, chain, lock, bad
     z += 2 * up256(rows * sizeof(unsigned));        // rel, s2q
+    z += up256(static_cast<size_t>(B) * sizeof(unsigned));       // lq
     if (zero_bytes) *zero_bytes = z;
     size_t n = z;
     n += up256(rows * nch * sizeof(RowZ));          // part
@@ -394,6 +418,7 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, int np, FlowScra
     fl->bad = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->rel = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->s2q = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
+    fl->lq = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->part = reinterpret_cast<RowZ*>(take(rows * nch * sizeof(RowZ)));
     fl->rowZ = reinterpret_cast<RowZ*>(take(rows * sizeof(RowZ)));
     fl->pchain = reinterpret_cast<double*>(take(static_cast<size_t>(B) * (gamma + 2) * sizeof(double)));

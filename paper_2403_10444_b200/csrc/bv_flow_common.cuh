@@ -14,11 +14,12 @@ namespace bv {
 enum : int { kExit = 0, kSweep1 = 1, kSweep2 = 2 };
 // Global counters, one per 128-byte line so that polling one does not slow the others down:
 // the sweep-1 ticket counter, rows queued for their second sweep, pieces of queued rows handed
-// out, blocks finished.
-constexpr int kCounterWords = 128;
-enum : int { kCtrTicket = 0, kCtrQueued = 32, kCtrPieces = 64, kCtrBlocks = 96 };
+// out, blocks finished, last target rows queued for their first sweep, chunks of those handed out.
+constexpr int kCounterWords = 192;
+enum : int { kCtrTicket = 0, kCtrQueued = 32, kCtrPieces = 64, kCtrBlocks = 96, kCtrLateQueued = 128, kCtrLateChunks = 160 };
 // rel[row]: 0 = not folded yet, then whether the row's second sweep is wanted
-enum : unsigned { kRelSweep = 1u, kRelSkip = 2u, kRelHold = 3u };   // hold: wanted only if every higher candidate is rejected
+enum : unsigned { kRelSweep = 1u, kRelSkip = 2u, kRelHold = 3u, kRelLate = 4u };   // hold: wanted only if every higher
+// candidate is rejected; late: the last target row, whose first sweep has only now been asked for
 
 __device__ __forceinline__ unsigned ld_volatile(const unsigned* p) {
     return *reinterpret_cast<const volatile unsigned*>(p);
@@ -306,8 +307,30 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
     unsigned nskip = 0;
     bool folded = false;
     unsigned c = ld_volatile(&fl.chain[b]);
-    while (c <= static_cast<unsigned>(g) && ld_volatile(&fl.row_done[static_cast<size_t>(b) * (g + 1) + c]) != 0u) {
+    while (c <= static_cast<unsigned>(g)) {
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
+        if (ld_volatile(&fl.row_done[ci]) == 0u) {
+            // The last target row is read only on demand: P_gamma matters only if position gamma is
+            // the selected one, i.e. if eta_gamma <= p_gamma, which is known at this point.  Its first
+            // sweep is asked for now (the row joins a queue of its own), or the position is closed.
+            if (c == static_cast<unsigned>(g) && ld_volatile(&fl.rel[ci]) == 0u) {
+                const double p_g = __ldcg(&p[g]);
+                if (all_positions || static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + g - 1]) <= p_g * (1.0 + 1e-6)) {
+                    atomicExch(&fl.rel[ci], kRelLate);
+                    const unsigned slot = atomicAdd(&fl.counters[kCtrLateQueued], 1u);
+                    atomicExch(&fl.lq[slot], static_cast<unsigned>(ci) + 1u);
+                } else {
+                    fl.cand[ci] = -1;
+                    ++nskip;
+                    __threadfence();
+                    atomicExch(&fl.rel[ci], kRelSkip);
+                    ++c;
+                    folded = true;
+                    continue;
+                }
+            }
+            break;
+        }
         const double p_c = (c == 0) ? 1.0 : __ldcg(&p[c]);
         if (c == 0) p[0] = 1.0;
         float cs = 1.f;

@@ -36,6 +36,7 @@ struct FlowScratch {
     unsigned* bad;        // [B] data fault seen
     unsigned* rel;        // [B (gamma+1)] row folded into the recursion, and what becomes of its second sweep
     unsigned* s2q;        // [B (gamma+1)] queue of rows whose second sweep has been started (row index + 1)
+    unsigned* lq;         // [B] queue of last target rows whose first sweep has been asked for (row index + 1)
     RowZ* part;           // [B (gamma+1) nch]
     RowZ* rowZ;           // [B (gamma+1)]
     double* pchain;       // [B (gamma+2)]
