@@ -430,7 +430,7 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, int np, FlowScra
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
     fl->nch = nch;
     fl->np = np;
-    fl->depth = 2;      // one item being swept, one queued: the service warp reacts sooner to released rows
+    fl->depth = kFDesc;
     fl->segs = static_cast<int>(segs);
 }
 
