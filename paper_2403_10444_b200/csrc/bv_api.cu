@@ -100,6 +100,9 @@ int pick_cluster(const DeviceState& d, int B, size_t row_bytes) {
     while (c < bv::kMaxCluster && row_bytes / c > (64u << 10)) c *= 2;
     while (c < bv::kMaxCluster && static_cast<long long>(B) * c < d.sm_count && row_bytes / (2 * c) >= (8u << 10))
         c *= 2;
+    // With several sequences per cluster to go through, narrower clusters (more sequences at a time,
+    // cheaper exchanges) win: measured 0.43 against 0.57 ms at B = 256, gamma = 8, V = 152064.
+    if (c == 8 && static_cast<long long>(B) * c >= 8LL * d.sm_count) c = 4;
     return c;
 }
 
