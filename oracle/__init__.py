@@ -53,6 +53,8 @@ def _load():
         lib.oracle_verify.argtypes = [ip, vp, vp, vp, vp, ip, ip, ip, ip, ctypes.c_double,
                                       vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_threads.restype = ctypes.c_int
+        lib.oracle_sample_rows.restype = ctypes.c_int
+        lib.oracle_sample_rows.argtypes = [vp, vp, ip, ip, ip, ctypes.c_double, vp, vp, vp]
         _lib = lib
     return _lib
 
@@ -120,3 +122,26 @@ def block_verify(*a, **k) -> OracleResult:
 
 def token_verify(*a, **k) -> OracleResult:
     return verify(TOKEN_VERIFY, *a, **k)
+
+
+def sample_rows(logits: np.ndarray, uniforms: np.ndarray, temperature: float = 1.0):
+    """The drafting step of Algorithm 3 on rows of logits [rows, V] (float32, float64 or uint16
+    bf16 bits) with one float32 uniform per row: returns (tokens int32 [rows], lse f64 [rows],
+    margin f64 [rows]); see ``oracle_sample_rows`` in verify_oracle.c."""
+    lib = _load()
+    logits = np.ascontiguousarray(logits)
+    if logits.dtype not in _DTYPE_CODE or logits.ndim != 2:
+        raise TypeError("logits must be [rows, V] float32, float64 or uint16 (bf16 bits)")
+    rows, V = logits.shape
+    uniforms = np.ascontiguousarray(uniforms, dtype=np.float32)
+    if uniforms.shape != (rows,):
+        raise ValueError("uniforms must be [rows]")
+    tok = np.empty((rows,), np.int32)
+    lse = np.empty((rows,))
+    margin = np.empty((rows,))
+    ptr = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    rc = lib.oracle_sample_rows(ptr(logits), ptr(uniforms), rows, V, _DTYPE_CODE[logits.dtype],
+                                float(np.float32(temperature)), ptr(tok), ptr(lse), ptr(margin))
+    if rc != 0:
+        raise ValueError("oracle_sample_rows rejected its arguments")
+    return tok, lse, margin

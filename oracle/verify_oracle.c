@@ -416,6 +416,43 @@ int oracle_verify(int algo, const void *target, const void *draft,
     return 0;
 }
 
+/*
+ * The drafting step of Algorithm 3 ("Sample X_1..X_gamma ~ M_s ... keep the conditional
+ * probabilities at each step") for rows of logits: for every row r,
+ *   M_s(x) = softmax(logits[r, :] / T)(x),
+ *   tokens[r] = inverse-CDF sample in vocabulary-index order with uniforms[r]
+ *               (the same convention as the verification samples),
+ *   lse[r]    = ln sum_x exp(logits[r, x] / T)   (what the verification needs of the row).
+ * A row with a NaN or +inf logit, or with no finite logit, gives tokens[r] = -1, lse[r] = NaN.
+ * margin[r] (may be NULL): distance in probability of the uniform from its CDF cell's edges.
+ * Returns 0, or 1 for an invalid argument.
+ */
+int oracle_sample_rows(const void *logits, const float *uniforms, int rows, int V, int dtype,
+                       double temperature, int32_t *tokens, double *lse, double *margin)
+{
+    if (!logits || !uniforms || !tokens || rows < 0 || V < 1)
+        return 1;
+    if (!(temperature > 0.0) || !isfinite(temperature) || dtype < 0 || dtype > 2)
+        return 1;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int r = 0; r < rows; ++r) {
+        size_t off = (size_t)r * (size_t)V;
+        double l, W, m = NAN;
+        if (row_lse(logits, dtype, off, V, temperature, &l)) {
+            tokens[r] = -1;
+            l = NAN;
+        } else {
+            tokens[r] = sample_index_order(logits, off, l, NULL, 0, 0.0, 0, dtype, V, temperature,
+                                           1.0, (double)uniforms[r], &W, &m);
+        }
+        if (lse) lse[r] = l;
+        if (margin) margin[r] = m;
+    }
+    return 0;
+}
+
 /* Number of threads the batch loop uses (1 when built without OpenMP). */
 #ifdef _OPENMP
 #include <omp.h>

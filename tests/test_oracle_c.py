@@ -312,3 +312,52 @@ def test_domain_errors_are_per_sequence():
     assert r.out_len[0] >= 1 and r.out_len[5] >= 1
     with pytest.raises(ValueError):
         oracle.block_verify(t, d, tok, uni, temperature=0.0)
+
+
+# ---------------- the drafting step of Algorithm 3 (oracle_sample_rows) ----------------
+def test_draft_sampler_frequencies_are_the_softmax():
+    # a mid-point grid of n uniforms integrates the sampler exactly up to 1/n per token:
+    # Pr(X = x) must be softmax(z / T)(x), written out here with numpy
+    rng = np.random.default_rng(5)
+    V, n, T = 7, 4000, 0.7
+    z = rng.normal(size=V) * 2
+    z[3] = -np.inf                                   # a token of probability zero
+    p = np.exp(z / np.float32(T) - np.max(z / np.float32(T)))
+    p /= p.sum()
+    u = midgrid(n)
+    tok, lse, _ = oracle.sample_rows(np.tile(z, (n, 1)), u, T)
+    freq = np.bincount(tok, minlength=V) / n
+    assert np.all(np.abs(freq - p) <= 1.0 / n + 1e-12)
+    assert freq[3] == 0
+    assert np.allclose(lse, logsumexp(z / np.float32(T)), rtol=1e-14)
+    # index order: the token is non-decreasing in the uniform, u = 0 gives the first token
+    assert np.all(np.diff(tok) >= 0) and tok[0] == 0
+
+
+def test_draft_sampler_matches_searchsorted_and_storage_types():
+    rng = np.random.default_rng(6)
+    rows, V = 64, 1000
+    z32 = (rng.normal(size=(rows, V)) * 3).astype(np.float32)
+    u = rng.random(rows, dtype=np.float32)
+    tok, lse, margin = oracle.sample_rows(z32, u, 1.0)
+    for r in range(rows):
+        w = np.exp(z32[r].astype(np.float64) - lse[r])
+        C = np.cumsum(w)
+        k = int(np.searchsorted(C, float(u[r]) * C[-1], side="right"))
+        if margin[r] > 1e-12:
+            assert tok[r] == min(k, V - 1)
+    # bf16 bits and float64 holding the same values give the same tokens
+    bits = (z32.view(np.uint32) >> 16).astype(np.uint16)
+    widened = (bits.astype(np.uint32) << 16).view(np.float32)
+    t16, l16, _ = oracle.sample_rows(bits, u, 1.0)
+    t64, l64, _ = oracle.sample_rows(widened.astype(np.float64), u, 1.0)
+    assert np.array_equal(t16, t64) and np.array_equal(l16, l64)
+
+
+def test_draft_sampler_domain_errors():
+    z = np.zeros((3, 5), np.float32)
+    z[0, 2] = np.nan
+    z[1, :] = -np.inf
+    tok, lse, _ = oracle.sample_rows(z, np.full(3, 0.5, np.float32), 1.0)
+    assert tok[0] == -1 and tok[1] == -1 and tok[2] == 2
+    assert np.isnan(lse[0]) and np.isnan(lse[1]) and abs(lse[2] - np.log(5)) < 1e-15
