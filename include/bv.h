@@ -160,6 +160,21 @@ int bv_verify_noalloc(const void* target_logits, const void* draft_logits,
                       int B, int gamma, int V, int dtype, float temperature,
                       int32_t* out_tokens, int32_t* out_len, void* stream);
 
+/*
+ * The drafting step of Algorithm 3 ("Sample X_1, ..., X_gamma ~ M_s using autoregressive sampling,
+ * keep the conditional probabilities at each step") for `rows` rows of draft logits [rows, V]:
+ *   out_tokens[r] ~ softmax(logits[r, :] / temperature), drawn by inverse CDF in vocabulary-index
+ *                   order with uniforms[r] in [0, 1): min{k : C_k > u W} over the running sums C_k of
+ *                   the weights, the convention of the verification samples;
+ *   out_lse[r]    = ln sum_x exp(logits[r, x] / temperature)  (float; may be NULL).
+ * DEVICE pointers, asynchronous on `stream`, no allocation.  A row with a NaN or +inf logit, or
+ * with no finite logit, gives out_tokens[r] = -1 and out_lse[r] = NaN.  Rows must be whole 16-byte
+ * vectors on a 16-byte aligned base (V a multiple of 8 for bf16, of 4 for fp32), else
+ * BV_ERR_UNSUPPORTED.  Each logit is read from HBM once.
+ */
+int bv_sample_draft(const void* logits, const float* uniforms, int rows, int V, int dtype,
+                    float temperature, int32_t* out_tokens, float* out_lse, void* stream);
+
 /* Frees the library's cached device buffers on the current device. */
 int bv_release(void);
 

@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_verify_noalloc", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_sample_draft", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -54,6 +54,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
         getattr(lib, name).argtypes = base + [vp, vp, vp, vp, vp, vp]
     for name in ("bv_verify_host", "tv_verify_host"):
         getattr(lib, name).argtypes = base
+    lib.bv_sample_draft.argtypes = [vp, vp, ci, ci, ci, cf, vp, vp, vp]
     for name in EXPORTS:
         getattr(lib, name).restype = ci
     lib.bv_status_string.restype = ctypes.c_char_p
@@ -218,3 +219,24 @@ def tv_verify_host(target_logits, draft_logits, draft_tokens, uniforms, temperat
     """Token Verification on HOST tensors (pinned for speed): copies in, runs, copies out."""
     return _host_call("tv_verify_host", target_logits, draft_logits, draft_tokens, uniforms,
                       temperature, out_tokens, out_len)
+
+
+def bv_sample_draft(logits, uniforms, temperature: float = 1.0, want_lse: bool = True, stream=None):
+    """The drafting step of Algorithm 3 on CUDA tensors: logits [rows, V] (float32 or bfloat16),
+    uniforms [rows] float32.  Returns (tokens int32 [rows], lse float32 [rows] or None)."""
+    if not (logits.is_cuda and uniforms.is_cuda):
+        raise ValueError("bv_sample_draft takes CUDA tensors")
+    if logits.dim() != 2 or not logits.is_contiguous():
+        raise ValueError("logits must be a contiguous [rows, V] tensor")
+    rows, V = logits.shape
+    if uniforms.shape != (rows,) or uniforms.dtype != torch.float32 or not uniforms.is_contiguous():
+        raise ValueError("uniforms must be a contiguous float32 tensor of [rows]")
+    lib = load_library()
+    tokens = torch.empty((rows,), dtype=torch.int32, device=logits.device)
+    lse = torch.empty((rows,), dtype=torch.float32, device=logits.device) if want_lse else None
+    st = stream if stream is not None else torch.cuda.current_stream(logits.device)
+    with torch.cuda.device(logits.device):
+        _check(lib.bv_sample_draft(logits.data_ptr(), uniforms.data_ptr(), rows, V, _dtype_code(logits),
+                                   float(temperature), tokens.data_ptr(), lse.data_ptr() if want_lse else None,
+                                   st.cuda_stream))
+    return tokens, lse

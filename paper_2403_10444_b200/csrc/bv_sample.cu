@@ -1,0 +1,151 @@
+// The drafting step of Algorithm 3 for rows of logits: one token per row drawn from
+// softmax(logits / T) by inverse CDF in vocabulary-index order with a supplied uniform, and the
+// row's log-normaliser (what the verification needs of a draft row besides the logits).
+//
+// Persistent CTAs take rows round-robin.  Every warp streams its contiguous sixteenth of the row
+// once, in eight sub-segments, and leaves each sub-segment's {integer reference, sum 2^{z k - M}}
+// in shared memory; warp 0 combines the 128 pairs (fp64 for the normaliser, fp32 prefix sums for
+// the sampler), finds the sub-segment that holds u * Z and rescans that one - a few KB still in
+// L2 - in index order for the token.  Each logit is read from HBM once.
+#include <cmath>
+#include <cstdint>
+
+#include "bv_flow_common.cuh"
+
+#include "../../include/bv.h"
+
+namespace bv {
+
+constexpr int kSThreads = 512;
+constexpr int kSWarps = kSThreads / 32;
+constexpr int kSSub = 8;                          // sub-segments per warp
+constexpr int kSSegs = kSWarps * kSSub;           // 128: four per lane of warp 0
+
+// vectors [a0, a1) of sub-segment `sub` of warp `warp` in a row of `units` vectors
+__device__ __forceinline__ void s_range(int units, int warp, int sub, int& a0, int& a1) {
+    const int u0 = static_cast<int>(static_cast<long long>(units) * warp / kSWarps);
+    const int u1 = static_cast<int>(static_cast<long long>(units) * (warp + 1) / kSWarps);
+    a0 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * sub / kSSub);
+    a1 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * (sub + 1) / kSSub);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kSThreads, 2)
+sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float kf, int32_t* tokens, float* lse) {
+    using R = Raw<DT>;
+    constexpr int EPV = R::EPV;
+    constexpr size_t ESZ = (DT == kF32) ? 4 : 2;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int units = V / EPV;
+    const size_t row_bytes = static_cast<size_t>(V) * ESZ;
+    __shared__ float sM[kSSegs], sS[kSSegs];
+
+    for (int r = blockIdx.x; r < rows; r += gridDim.x) {
+        const char* row = logits + static_cast<size_t>(r) * row_bytes;
+        // ---- one pass over the warp's part of the row ----
+        for (int sub = 0; sub < kSSub; ++sub) {
+            int a0, a1;
+            s_range(units, warp, sub, a0, a1);
+            float M = kNoRef, s = 0.f;
+            for (int base = a0; base < a1; base += 128) {
+                float v[4][EPV];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) f_load_tail<DT>(row, base + 32 * j + lane, a1, v[j]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (base + 32 * j < a1) f_accumulate<EPV>(v[j], kf, M, s);
+            }
+            s = warp_sum(s);
+            if (lane == 0) { sM[warp * kSSub + sub] = M; sS[warp * kSSub + sub] = s; }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // ---- normaliser (fp64) and the sampled sub-segment (fp32 prefix sums, index order) ----
+            float m[4], w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { m[j] = sM[4 * lane + j]; w[j] = sS[4 * lane + j]; }
+            const float Mrow = warp_max(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) w[j] *= ref_scale(m[j], Mrow);
+            double Z = (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
+                       (static_cast<double>(w[2]) + static_cast<double>(w[3]));
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) Z += shfl_xor_d(Z, off);
+            const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
+            float inc = l4;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float o = __shfl_up_sync(0xffffffffu, inc, off);
+                if (lane >= off) inc += o;
+            }
+            const float total = __shfl_sync(0xffffffffu, inc, 31);
+            // a row with a NaN or +inf logit has a NaN / infinite sum or reference; one without a finite logit has none
+            const bool ok = Mrow > kNoRef && Mrow < INFINITY && Z > 0.0 && Z < INFINITY && total > 0.f && total < INFINITY;
+            int found = -1;
+            if (ok) {
+                const float t = uni[r] * total;
+                float exc = __shfl_up_sync(0xffffffffu, inc, 1);
+                if (lane == 0) exc = 0.f;
+                const float p0 = exc, p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+                // first non-empty sub-segment whose inclusive prefix exceeds t, else the last non-empty one
+                const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
+                const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
+                const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
+                const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
+                int e = 3; float bef = p3; int src;
+                if (hit) {
+                    src = __ffs(hit) - 1;
+                    if (h1) { e = 0; bef = p0; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
+                } else {
+                    src = 31 - __clz(nz);
+                    e = 0; bef = p0;
+                    if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
+                    else if (w[1] > 0.f) { e = 1; bef = p1; }
+                }
+                const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
+                const float before = __shfl_sync(0xffffffffu, bef, src);
+                int a0, a1;
+                s_range(units, sel / kSSub, sel % kSSub, a0, a1);
+                found = f_rescan<DT>(row, nullptr, a0, a1, lane, kf, 1.f, -Mrow, 0.f, t - before);
+            }
+            if (lane == 0) {
+                tokens[r] = found;
+                if (lse) lse[r] = found >= 0 ? static_cast<float>((static_cast<double>(Mrow) + log2(Z)) * 0.693147180559945309417232)
+                                             : __int_as_float(0x7fc00000);
+            }
+        }
+        __syncthreads();      // the pairs are overwritten by the next row
+    }
+}
+
+}  // namespace bv
+
+namespace {
+thread_local int t_sample_cuda_error = 0;
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) % 16) == 0; }
+}  // namespace
+
+extern "C" int bv_sample_draft(const void* logits, const float* uniforms, int rows, int V, int dtype,
+                               float temperature, int32_t* out_tokens, float* out_lse, void* stream) {
+    if (!logits || !uniforms || !out_tokens) return BV_ERR_INVALID_ARG;
+    if (rows < 0 || V < 1) return BV_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !std::isfinite(temperature)) return BV_ERR_INVALID_ARG;
+    if (dtype != BV_DTYPE_F32 && dtype != BV_DTYPE_BF16) return BV_ERR_INVALID_ARG;
+    const size_t row_bytes = static_cast<size_t>(V) * (dtype == BV_DTYPE_F32 ? 4 : 2);
+    if (row_bytes % 16 != 0 || !aligned16(logits)) return BV_ERR_UNSUPPORTED;
+    if (rows == 0) return BV_OK;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) { t_sample_cuda_error = static_cast<int>(e); return BV_ERR_CUDA; }
+    const int grid = rows < 2 * sms ? rows : 2 * sms;
+    const float kf = static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == BV_DTYPE_F32)
+        bv::sample_rows_kernel<bv::kF32><<<grid, bv::kSThreads, 0, st>>>(static_cast<const char*>(logits), uniforms, rows, V, kf, out_tokens, out_lse);
+    else
+        bv::sample_rows_kernel<bv::kBF16><<<grid, bv::kSThreads, 0, st>>>(static_cast<const char*>(logits), uniforms, rows, V, kf, out_tokens, out_lse);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { t_sample_cuda_error = static_cast<int>(e); return BV_ERR_CUDA; }
+    return BV_OK;
+}
