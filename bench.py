@@ -124,7 +124,12 @@ def time_oracle(w, algo_name: str, budget_s: float = 20.0):
         else:
             t = t.numpy(); d = d.numpy()
         t0 = time.perf_counter()
-        oracle.verify(algo, t, d, inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), inp["temperature"])
+        if algo_name == "sample":
+            g = inp["draft_tokens"].shape[1]
+            oracle.sample_rows(d.reshape(-1, d.shape[-1]), inp["uniforms"].numpy()[:, :g].reshape(-1).copy(),
+                               inp["temperature"])
+        else:
+            oracle.verify(algo, t, d, inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), inp["temperature"])
         return time.perf_counter() - t0
 
     t_probe = run(probe)
@@ -134,7 +139,8 @@ def time_oracle(w, algo_name: str, budget_s: float = 20.0):
     sample = wl.make_inputs(wl.scaled(w, B=n), "cpu")
     dt = run(sample)
     return {"value": n * w.gamma / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "first %d of %d sequences of workload %s (%s verify), %.2f s" % (n, w.B, w.name, algo_name, dt),
+            "sample": "first %d of %d sequences of workload %s (%s), %.2f s" % (
+                n, w.B, w.name, "drafting step" if algo_name == "sample" else algo_name + " verify", dt),
             "seconds": dt, "sequences": n}
 
 
@@ -170,7 +176,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(wl.CONFIGS))
-    ap.add_argument("--algo", default="block", choices=["block", "token"])
+    ap.add_argument("--algo", default="block", choices=["block", "token", "sample"],
+                    help="block / token verification, or the drafting step (sampling the draft rows)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
@@ -196,6 +203,12 @@ def main():
     inp = wl.make_inputs(wl.scaled(w, seed=w.seed + 1000 * rank), dev)
     fn = bv.bv_verify if args.algo == "block" else bv.tv_verify
     a = (inp["target_logits"], inp["draft_logits"], inp["draft_tokens"], inp["uniforms"], inp["temperature"])
+    if args.algo == "sample":
+        # the drafting step on the same draft rows: B gamma rows of V logits, one uniform each
+        rows2d = inp["draft_logits"].view(w.B * w.gamma, w.V)
+        u_rows = inp["uniforms"][:, : w.gamma].contiguous().view(-1)
+        fn = lambda *_: bv.bv_sample_draft(rows2d, u_rows, inp["temperature"])
+        args.e2e_steps = 0          # (no host-buffer form of this entry point)
 
     def barrier():
         if dist is not None:
@@ -218,7 +231,7 @@ def main():
         evs[i][0].record()
         out = fn(*a)
         evs[i][1].record()
-        launches += bv.bv_last_launch_count()
+        launches += 1 if args.algo == "sample" else bv.bv_last_launch_count()
     stop.record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
@@ -264,9 +277,12 @@ def end_to_end(args, w, inp, out, bv, barrier, dist, dev, world):
 def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches, out, dist):
     peak, peak_src = measured_peak()
     k_ms = statistics.mean(kernel_ms)
-    mean_len = float(out[1].float().mean().item())
+    mean_len = float(out[1].float().mean().item()) if args.algo != "sample" else None
     esz = 4 if w.dtype == "f32" else 2
-    if args.algo == "block":
+    if args.algo == "sample":
+        algo_bytes = w.B * w.gamma * w.V * esz
+        kernel = "sample_rows_kernel"
+    elif args.algo == "block":
         # Algorithm 2 needs every row: B (2 gamma + 1) V elements
         algo_bytes = w.logit_bytes
         kernel = "verify_flow_kernel"

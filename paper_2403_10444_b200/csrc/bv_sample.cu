@@ -2,9 +2,9 @@
 // softmax(logits / T) by inverse CDF in vocabulary-index order with a supplied uniform, and the
 // row's log-normaliser (what the verification needs of a draft row besides the logits).
 //
-// Persistent CTAs take rows round-robin.  Every warp streams its contiguous sixteenth of the row
-// once, in eight sub-segments, and leaves each sub-segment's {integer reference, sum 2^{z k - M}}
-// in shared memory; warp 0 combines the 128 pairs (fp64 for the normaliser, fp32 prefix sums for
+// Persistent CTAs take rows round-robin.  Each of 16 warps streams its contiguous sixteenth of the
+// row once, in eight sub-segments, and leaves each sub-segment's {integer reference, sum 2^{z k - M}}
+// in shared memory; a seventeenth warp, one row behind, combines the 128 pairs (fp64 for the normaliser, fp32 prefix sums for
 // the sampler), finds the sub-segment that holds u * Z and rescans that one - a few KB still in
 // L2 - in index order for the token.  Each logit is read from HBM once.
 #include <cmath>
@@ -16,10 +16,12 @@
 
 namespace bv {
 
-constexpr int kSThreads = 512;
+constexpr int kSThreads = 512;                    // streaming threads; one more warp draws the samples
 constexpr int kSWarps = kSThreads / 32;
+constexpr int kSAllThreads = kSThreads + 32;
 constexpr int kSSub = 8;                          // sub-segments per warp
 constexpr int kSSegs = kSWarps * kSSub;           // 128: four per lane of warp 0
+constexpr int kSInFlight = 8;                     // 16-byte loads a thread has in flight
 
 // vectors [a0, a1) of sub-segment `sub` of warp `warp` in a row of `units` vectors
 __device__ __forceinline__ void s_range(int units, int warp, int sub, int& a0, int& a1) {
@@ -30,7 +32,7 @@ __device__ __forceinline__ void s_range(int units, int warp, int sub, int& a0, i
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kSThreads, 2)
+__global__ void __launch_bounds__(kSAllThreads, 2)
 sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float kf, int32_t* tokens, float* lse) {
     using R = Raw<DT>;
     constexpr int EPV = R::EPV;
@@ -38,28 +40,48 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int units = V / EPV;
     const size_t row_bytes = static_cast<size_t>(V) * ESZ;
-    __shared__ float sM[kSSegs], sS[kSSegs];
+    __shared__ float sM2[2][kSSegs], sS2[2][kSSegs];
 
-    for (int r = blockIdx.x; r < rows; r += gridDim.x) {
+    // Iteration `it`: the streaming warps sweep the CTA's it-th row while the sampling warp draws
+    // the token of the row before from the pairs that were left for it; one barrier per row.
+    const int nmine = rows > static_cast<int>(blockIdx.x) ? (rows - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
+    for (int it = 0; it <= nmine; ++it) {
+        if (warp < kSWarps && it < nmine) {
+        const int r = blockIdx.x + it * gridDim.x;
+        float* sM = sM2[it & 1];
+        float* sS = sS2[it & 1];
         const char* row = logits + static_cast<size_t>(r) * row_bytes;
         // ---- one pass over the warp's part of the row ----
         for (int sub = 0; sub < kSSub; ++sub) {
             int a0, a1;
             s_range(units, warp, sub, a0, a1);
             float M = kNoRef, s = 0.f;
-            for (int base = a0; base < a1; base += 128) {
-                float v[4][EPV];
+            const uint4 ninf = make_uint4(R::kNegInf, R::kNegInf, R::kNegInf, R::kNegInf);
+            for (int base = a0; base < a1; base += 32 * kSInFlight) {
+                uint4 raw[kSInFlight];                // all loads of the round are issued before any is used
 #pragma unroll
-                for (int j = 0; j < 4; ++j) f_load_tail<DT>(row, base + 32 * j + lane, a1, v[j]);
+                for (int j = 0; j < kSInFlight; ++j) {
+                    const int i = base + 32 * j + lane;
+                    raw[j] = i < a1 ? ld_stream_v4(row + static_cast<size_t>(i) * 16) : ninf;
+                }
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (base + 32 * j < a1) f_accumulate<EPV>(v[j], kf, M, s);
+                for (int j = 0; j < kSInFlight; ++j) {
+                    if (base + 32 * j < a1) {
+                        float v[EPV];
+                        R::unpack(raw[j], v);
+                        f_accumulate<EPV>(v, kf, M, s);
+                    }
+                }
             }
             s = warp_sum(s);
             if (lane == 0) { sM[warp * kSSub + sub] = M; sS[warp * kSSub + sub] = s; }
         }
-        __syncthreads();
-        if (warp == 0) {
+        }
+        if (warp == kSWarps && it >= 1) {
+            const int r = blockIdx.x + (it - 1) * gridDim.x;
+            const float* sM = sM2[(it - 1) & 1];
+            const float* sS = sS2[(it - 1) & 1];
+            const char* row = logits + static_cast<size_t>(r) * row_bytes;
             // ---- normaliser (fp64) and the sampled sub-segment (fp32 prefix sums, index order) ----
             float m[4], w[4];
 #pragma unroll
@@ -114,7 +136,7 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
                                              : __int_as_float(0x7fc00000);
             }
         }
-        __syncthreads();      // the pairs are overwritten by the next row
+        __syncthreads();      // row `it` is swept, the token of row `it - 1` is drawn
     }
 }
 
@@ -142,9 +164,9 @@ extern "C" int bv_sample_draft(const void* logits, const float* uniforms, int ro
     const float kf = static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (dtype == BV_DTYPE_F32)
-        bv::sample_rows_kernel<bv::kF32><<<grid, bv::kSThreads, 0, st>>>(static_cast<const char*>(logits), uniforms, rows, V, kf, out_tokens, out_lse);
+        bv::sample_rows_kernel<bv::kF32><<<grid, bv::kSAllThreads, 0, st>>>(static_cast<const char*>(logits), uniforms, rows, V, kf, out_tokens, out_lse);
     else
-        bv::sample_rows_kernel<bv::kBF16><<<grid, bv::kSThreads, 0, st>>>(static_cast<const char*>(logits), uniforms, rows, V, kf, out_tokens, out_lse);
+        bv::sample_rows_kernel<bv::kBF16><<<grid, bv::kSAllThreads, 0, st>>>(static_cast<const char*>(logits), uniforms, rows, V, kf, out_tokens, out_lse);
     e = cudaGetLastError();
     if (e != cudaSuccess) { t_sample_cuda_error = static_cast<int>(e); return BV_ERR_CUDA; }
     return BV_OK;
