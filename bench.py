@@ -323,6 +323,7 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
 # kernel with no capture.
 TRAFFIC_BYTES = {
     ("c4", "block", "verify_flow_kernel"): 2447101952,
+    ("c4", "sample", "sample_rows_kernel"): 1054102784,
 }
 
 
