@@ -4,9 +4,9 @@
 //
 // Persistent CTAs take rows round-robin.  Each of 16 warps streams its contiguous sixteenth of the
 // row once, in eight sub-segments, and leaves each sub-segment's {integer reference, sum 2^{z k - M}}
-// in shared memory; a seventeenth warp, one row behind, combines the 128 pairs (fp64 for the normaliser, fp32 prefix sums for
-// the sampler), finds the sub-segment that holds u * Z and rescans that one - a few KB still in
-// L2 - in index order for the token.  Each logit is read from HBM once.
+// in shared memory; a seventeenth warp, one row behind, combines the 128 pairs (fp64 for the
+// normaliser, fp32 prefix sums for the sampler), finds the sub-segment that holds u * Z and rescans
+// that one - a few KB still in L2 - in index order for the token.  Each logit is read from HBM once.
 #include <cmath>
 #include <cstdint>
 
