@@ -62,6 +62,68 @@ struct FlowShared {
 // it has swept in a short list and runs the second sweep of each of them itself, as soon as the
 // chunk's row has been folded into the recursion: the re-read follows the first read as closely
 // as the dependency allows, so the rows are still in L2.
+// ---- service warp: Y ~ P_gamma from the first sweep of the last target row ----
+// The sample needs the row's normaliser and a second look at one segment only: the segment
+// {reference, sum} pairs of all chunks are in scratch, so u * Z is located among their prefix sums
+// (fp32, index order) and that one segment is rescanned.  No second sweep of the row.
+template <int DT>
+__device__ void f_draw_from_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, int lane) {
+    const int g = cx.g, b = ri / (g + 1);
+    const int nseg = cx.nch * kFWarps;                       // <= 128: four per lane
+    const float* pairs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
+    float m[4], w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int i = 4 * lane + j;
+        m[j] = i < nseg ? __ldcg(&pairs[2 * i]) : kNoRef;
+        w[j] = i < nseg ? __ldcg(&pairs[2 * i + 1]) : 0.f;
+    }
+    const float Mrow = warp_max(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])));
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w[j] *= ref_scale(m[j], Mrow);
+    const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
+    float inc = l4;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float o = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += o;
+    }
+    const float total = __shfl_sync(0xffffffffu, inc, 31);
+    int found = -1;
+    if (Mrow > kNoRef && Mrow < INFINITY && total > 0.f && total < INFINITY) {
+        const float t = prm.uni[static_cast<size_t>(b) * (g + 2) + g + 1] * total;
+        float exc = __shfl_up_sync(0xffffffffu, inc, 1);
+        if (lane == 0) exc = 0.f;
+        const float p0 = exc, p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+        // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
+        const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
+        const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
+        const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
+        const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
+        int e = 3; float bef = p3; int src;
+        if (hit) {
+            src = __ffs(hit) - 1;
+            if (h1) { e = 0; bef = p0; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
+        } else {
+            src = 31 - __clz(nz);
+            e = 0; bef = p0;
+            if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
+            else if (w[1] > 0.f) { e = 1; bef = p1; }
+        }
+        const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
+        const float before = __shfl_sync(0xffffffffu, bef, src);
+        int s0, s1;
+        chunk_range(cx, cx.nch, sel / kFWarps, sel % kFWarps, s0, s1);
+        const char* rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
+        found = f_rescan<DT>(rowP, nullptr, s0, s1, lane, cx.kf, 1.f, -Mrow, 0.f, t - before);
+    }
+    if (lane == 0) {
+        fl.cand[ri] = found;
+        __threadfence();
+    }
+    __syncwarp();
+}
+
 // ---- service warp: what follows the sweep of one item ----
 template <int DT>
 __device__ void f_after_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int slot,
@@ -74,15 +136,27 @@ __device__ void f_after_sweep1(const Params& prm, const FlowScratch& fl, const F
     double zQ = lane < kFWarps ? static_cast<double>(sh.part_s[slot][1][lane]) * ref_scale(mQ, MQc) : 0.0;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) { zP += shfl_xor_d(zP, off); zQ += shfl_xor_d(zQ, off); }
+    // A last target row is swept for one purpose only: the sample from P_gamma.  Its warps' pairs
+    // {reference, sum} are kept, so that the token can be drawn from this one sweep (below).
+    const bool draw = ri % (cx.g + 1) == cx.g && f_draws_in_sweep1(prm, cx.nch);
+    if (draw) {
+        float* pairs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs + static_cast<size_t>(ch) * kFWarps * 2;
+        if (lane < kFWarps) { pairs[2 * lane] = mP; pairs[2 * lane + 1] = sh.part_s[slot][0][lane]; }
+        __threadfence();
+        __syncwarp();
+    }
+    int last = 0;
     if (lane == 0) {
         RowZ z; z.MP = MPc; z.ZP = zP; z.MQ = MQc; z.ZQ = zQ;
         fl.part[static_cast<size_t>(ri) * cx.nch + ch] = z;
         __threadfence();
-        if (atomicAdd(&fl.row_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u) {
-            __threadfence();
-            f_row_complete<DT>(prm, fl, cx, ri / (cx.g + 1), ri % (cx.g + 1));
-        }
+        last = atomicAdd(&fl.row_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u;
     }
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+    __threadfence();
+    if (draw) f_draw_from_sweep1<DT>(prm, fl, cx, ri, lane);
+    if (lane == 0) f_row_complete<DT>(prm, fl, cx, ri / (cx.g + 1), ri % (cx.g + 1));
     __syncwarp();
 }
 
@@ -92,7 +166,7 @@ __device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const F
     const int ri = d.ri;
     const int np = fl.np;
     const int nseg = np * kFWarps;
-    float* segs = fl.seg_tot + static_cast<size_t>(ri) * nseg;
+    float* segs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
     if (lane < kFWarps) segs[d.ch * kFWarps + lane] = sh.part_s[slot][0][lane];
     __threadfence();
     __syncwarp();
@@ -380,10 +454,16 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
 // host side
 // ---------------------------------------------------------------------------
 static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+// floats of seg_tot per row: the sweep-2 totals (np pieces of kFWarps segments) or, for a last
+// target row, the sweep-1 {reference, sum} pairs (nch chunks of kFWarps segments)
+static size_t flow_seg_stride(int nch, int np) {
+    const size_t a = static_cast<size_t>(np) * kFWarps, b = static_cast<size_t>(nch) * kFWarps * 2;
+    return a > b ? a : b;
+}
 
 size_t flow_scratch_bytes(int B, int gamma, int nch, int np, size_t* zero_bytes) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
-    const size_t segs = static_cast<size_t>(np) * kFWarps;
+    const size_t segs = flow_seg_stride(nch, np);
     size_t z = 0;
     z += up256(kCounterWords * sizeof(unsigned));   // counters
     z += 3 * up256(rows * sizeof(unsigned));        // row_cnt, row_done, s2_cnt
@@ -405,7 +485,7 @@ size_t flow_scratch_bytes(int B, int gamma, int nch, int np, size_t* zero_bytes)
 
 void flow_scratch_layout(void* base, int B, int gamma, int nch, int np, FlowScratch* fl) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
-    const size_t segs = static_cast<size_t>(np) * kFWarps;
+    const size_t segs = flow_seg_stride(nch, np);
     char* p = static_cast<char*>(base);
     auto take = [&](size_t bytes) { char* q = p; p += up256(bytes); return q; };
     fl->counters = reinterpret_cast<unsigned*>(take(kCounterWords * sizeof(unsigned)));

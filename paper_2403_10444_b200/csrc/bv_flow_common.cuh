@@ -206,6 +206,15 @@ static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl
     atomicAdd(&fl.counters[kCtrBlocks], 1u);      // (CTAs leave when every block is finished)
 }
 
+// With diagnostic outputs every position is computed in full.
+__device__ __forceinline__ bool f_all_positions(const Params& prm) {
+    return prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
+}
+// Is the token of position gamma drawn from the first sweep of the last target row (bv_flow.cu)?
+__device__ __forceinline__ bool f_draws_in_sweep1(const Params& prm, int nch) {
+    return !f_all_positions(prm) && nch <= 8;
+}
+
 // ---- which positions get a second sweep (one thread each) ----
 // Is position i the selected one, given p_i and (for 0 < i < gamma) S_i?  Position 0 is what
 // remains when no other is selected.  (Eq. "pacc_block": h_gamma = p_gamma, h_i = S_i / (S_i + 1 - p_i).)
@@ -305,7 +314,7 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
     __threadfence();
     const bool all_positions = prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
     unsigned nskip = 0;
-    bool folded = false;
+    bool folded = false, top_done = false;
     unsigned c = ld_volatile(&fl.chain[b]);
     while (c <= static_cast<unsigned>(g)) {
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
@@ -346,6 +355,18 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
         // is the sample from P_gamma drawn.  Position 0 is what remains when no other is selected.
         // (The margin keeps a uniform within rounding of p_c on the long path; with diagnostic
         // outputs every position is computed.)
+        if (c == static_cast<unsigned>(g) && f_draws_in_sweep1(prm, cx.nch)) {
+            // the row was swept because position gamma can be selected, and its token was drawn from
+            // that very sweep: the position is complete.  It is the highest candidate, so either it
+            // is the selected one (lower candidates are dropped) or the next lower one is started.
+            __threadfence();
+            atomicExch(&fl.rel[ci], kRelSkip);
+            nskip += f_after_position(prm, fl, b, g);
+            top_done = true;
+            ++c;
+            folded = true;
+            continue;
+        }
         bool need = all_positions || c == 0;
         if (!need) need = static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + c - 1]) <= p_c * (1.0 + 1e-6);
         if (!need) {
@@ -361,7 +382,7 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
         ++c;
         folded = true;
     }
-    if (folded && c == static_cast<unsigned>(g) + 1u && !all_positions) f_release_next(fl, b, g, g + 1);
+    if (folded && !top_done && c == static_cast<unsigned>(g) + 1u && !all_positions) f_release_next(fl, b, g, g + 1);
     *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
     __threadfence();
     atomicExch(&fl.lock[b], 0u);
