@@ -229,8 +229,11 @@ static __device__ bool f_position_selected(const Params& prm, const FlowScratch&
     }
     return h > 0.0 && static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + i - 1]) <= h;
 }
-// The selected position is the highest candidate that passes its test, so the candidates are
-// swept from the top, one at a time: start the highest one on hold below `below`.
+// A position on hold changes state exactly once, whoever gets there first (positions of one block
+// may complete side by side once several candidates are swept at a time): true if this call did it.
+static __device__ bool f_leave_hold(const FlowScratch& fl, size_t ci, unsigned to) {
+    return atomicCAS(&fl.rel[ci], kRelHold, to) == kRelHold;
+}
 static __device__ void f_start_second_sweep(const FlowScratch& fl, size_t ci) {
     atomicExch(&fl.rel[ci], kRelSweep);
     // the row joins the queue from which every CTA draws pieces; the entry itself says when it is
@@ -239,30 +242,39 @@ static __device__ void f_start_second_sweep(const FlowScratch& fl, size_t ci) {
     const unsigned slot = atomicAdd(&fl.counters[kCtrQueued], 1u);
     atomicExch(&fl.s2q[slot], static_cast<unsigned>(ci) + 1u);
 }
-static __device__ void f_release_next(const FlowScratch& fl, int b, int g, int below) {
+// The selected position is the highest candidate that passes its test, so the candidates are
+// swept from the top, one at a time: start the highest one on hold below `below`.  Once the
+// first-sweep tickets have run out the GPU is emptying and a block's chain of candidates, one
+// after the other, would only prolong the launch: then all of them are started at once (a lower
+// one that turns out not to be needed costs bandwidth nobody else wants).
+static __device__ void f_release_next(const Params& prm, const FlowScratch& fl, int b, int below) {
+    const int g = prm.gamma;
+    const bool all = ld_volatile(&fl.counters[kCtrTicket]) >= static_cast<unsigned>(prm.B) * g * fl.nch;
     for (int c = below - 1; c >= 0; --c) {
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
-        if (ld_volatile(&fl.rel[ci]) == kRelHold) { f_start_second_sweep(fl, ci); return; }
+        if (ld_volatile(&fl.rel[ci]) != kRelHold || !f_leave_hold(fl, ci, kRelSweep)) continue;
+        f_start_second_sweep(fl, ci);
+        if (!all) return;
     }
 }
-// Position i has just been completed (S_i and its candidate token are in scratch): either it is
-// the selected one, and no lower position is wanted, or the next lower candidate is started.
-// Returns the number of positions that are complete through this call (itself included).
+// Position i has just been completed (S_i and its candidate token are in scratch).  If it passes
+// its test, tau >= i whatever the higher candidates do, and no lower position is wanted; if not,
+// the next lower candidate is started.  Returns the number of positions that are complete through
+// this call (itself included).
 static __device__ unsigned f_after_position(const Params& prm, const FlowScratch& fl, int b, int i) {
     const int g = prm.gamma;
     unsigned done = 1;
     if (f_position_selected(prm, fl, b, i)) {
         for (int c = i - 1; c >= 0; --c) {
             const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
-            if (ld_volatile(&fl.rel[ci]) != kRelHold) continue;
+            if (ld_volatile(&fl.rel[ci]) != kRelHold || !f_leave_hold(fl, ci, kRelSkip)) continue;
             if (c < g) fl.S[ci] = 0.0;
             fl.cand[ci] = -1;
-            __threadfence();
-            atomicExch(&fl.rel[ci], kRelSkip);
             ++done;
         }
+        __threadfence();
     } else {
-        f_release_next(fl, b, g, i);
+        f_release_next(prm, fl, b, i);
     }
     return done;
 }
@@ -382,7 +394,7 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
         ++c;
         folded = true;
     }
-    if (folded && !top_done && c == static_cast<unsigned>(g) + 1u && !all_positions) f_release_next(fl, b, g, g + 1);
+    if (folded && !top_done && c == static_cast<unsigned>(g) + 1u && !all_positions) f_release_next(prm, fl, b, g + 1);
     *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
     __threadfence();
     atomicExch(&fl.lock[b], 0u);
