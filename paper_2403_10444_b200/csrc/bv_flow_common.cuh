@@ -250,10 +250,14 @@ static __device__ void f_start_second_sweep(const FlowScratch& fl, size_t ci) {
 static __device__ void f_release_next(const Params& prm, const FlowScratch& fl, int b, int below) {
     const int g = prm.gamma;
     const bool all = ld_volatile(&fl.counters[kCtrTicket]) >= static_cast<unsigned>(prm.B) * g * fl.nch;
+    // (position 0, what remains when nothing else is selected, still waits for the others)
+    int started = 0;
     for (int c = below - 1; c >= 0; --c) {
+        if (c == 0 && started > 0) break;
         const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
         if (ld_volatile(&fl.rel[ci]) != kRelHold || !f_leave_hold(fl, ci, kRelSweep)) continue;
         f_start_second_sweep(fl, ci);
+        ++started;
         if (!all) return;
     }
 }
