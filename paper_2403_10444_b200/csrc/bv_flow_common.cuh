@@ -249,7 +249,13 @@ static __device__ void f_start_second_sweep(const FlowScratch& fl, size_t ci) {
 // one that turns out not to be needed costs bandwidth nobody else wants).
 static __device__ void f_release_next(const Params& prm, const FlowScratch& fl, int b, int below) {
     const int g = prm.gamma;
-    const bool all = ld_volatile(&fl.counters[kCtrTicket]) >= static_cast<unsigned>(prm.B) * g * fl.nch;
+    bool all = ld_volatile(&fl.counters[kCtrTicket]) >= static_cast<unsigned>(prm.B) * g * fl.nch;
+    if (all) {       // only a chain of three or more is worth the bandwidth of the ones not needed
+        int held = 0;
+        for (int c = below - 1; c >= 1; --c)
+            held += ld_volatile(&fl.rel[static_cast<size_t>(b) * (g + 1) + c]) == kRelHold;
+        all = held >= 3;
+    }
     // (position 0, what remains when nothing else is selected, still waits for the others)
     int started = 0;
     for (int c = below - 1; c >= 0; --c) {
