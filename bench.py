@@ -328,7 +328,7 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
 # ncu capture of this command at full size that profiles/ summarises; None for a workload or
 # kernel with no capture.
 TRAFFIC_BYTES = {
-    ("c4", "block", "verify_flow_kernel"): 2447101952,
+    ("c4", "block", "verify_flow_kernel"): 2492403456,
     ("c4", "sample", "sample_rows_kernel"): 1054102784,
 }
 
