@@ -1,19 +1,26 @@
 // Block Verification (Algorithm 2) as a dependency-driven flow of independent work items.
 //
-// A row pair (P_r, Q_r) of one drafted block is cut into NCH chunks.  Persistent CTAs
-// pull items from two sources:
+// Persistent CTAs (16 worker warps that only stream, one service warp that does everything
+// else) pull items from three sources, in this order of preference:
 //
-//   sweep-1 item (b, r, chunk)  streams the chunk of both rows from HBM and leaves the
-//       chunk's {reference, sum 2^{z k - M}} pair for each row in scratch.  The CTA that
-//       completes a row combines the chunks into the row normalisers and, holding the
-//       block's lock, advances the prefix recursion p_{r+1} = min(p_r P_r(X)/Q_r(X), 1)
-//       (Eq. "def_as") over every row that is complete, releasing their sweep-2 items.
-//   sweep-2 item (b, r, chunk)  re-reads the chunk (an L2 hit: it was streamed moments
-//       ago, and released items are taken before new sweep-1 items) and leaves
-//       sum max(p_r P_r(x) - Q_r(x), 0) per warp segment (Eq. "pacc_block").  The CTA
-//       that completes a position adds the segments to S_r, locates u * S_r, rescans that
-//       one segment in index order for the candidate Y_r (Eq. "pres-block"), and the CTA
-//       that completes the block forms h_i, selects tau and emits X^tau, Y_tau.
+//   sweep-2 piece (b, r, piece)  a piece of a row pair whose second sweep has been started:
+//       leaves sum max(p_r P_r(x) - Q_r(x), 0) per warp segment (Eq. "pacc_block").  The CTA
+//       that completes a position adds the segments to S_r, locates u * S_r, rescans that one
+//       segment in index order for the candidate Y_r (Eq. "pres-block"), and then either finds
+//       the position selected or starts the next lower candidate; the CTA that completes the
+//       block forms h_i, selects tau and emits X^tau, Y_tau.
+//   late sweep-1 chunk  of a last target row P_gamma, which is read only if position gamma can
+//       be the selected one; its sample is drawn from that one sweep.
+//   sweep-1 item (b, r < gamma, chunk)  by ticket, in row order: streams the chunk of both
+//       rows from HBM and leaves the chunk's {reference, sum 2^{z k - M}} pair for each row in
+//       scratch.  The CTA that completes a row combines the chunks into the row normalisers
+//       and, holding the block's lock, advances the prefix recursion
+//       p_{r+1} = min(p_r P_r(X)/Q_r(X), 1) (Eq. "def_as") over every row that is complete.
+//
+// A second sweep runs only where the outcome can depend on it: S_r <= p_r gives h_r <= p_r, so
+// a position with eta_r > p_r can never be selected; the others are swept from the top down
+// until one passes its test (bv_flow_common.cuh).  With diagnostic outputs every position is
+// swept.
 //
 // No CTA ever waits for another one while it holds work that others need: sweep-1 items
 // have no prerequisites, the lock is only held over a few scalar operations, and a CTA
@@ -58,10 +65,6 @@ struct FlowShared {
     float part_s[kFDesc][2][kFWarps];   // sweep 1: sums; sweep 2: [0] holds the residual totals
 };
 
-// Sweep-1 items are handed out in row order by a single ticket counter.  A CTA keeps the chunks
-// it has swept in a short list and runs the second sweep of each of them itself, as soon as the
-// chunk's row has been folded into the recursion: the re-read follows the first read as closely
-// as the dependency allows, so the rows are still in L2.
 // ---- service warp: Y ~ P_gamma from the first sweep of the last target row ----
 // The sample needs the row's normaliser and a second look at one segment only: the segment
 // {reference, sum} pairs of all chunks are in scratch, so u * Z is located among their prefix sums
@@ -264,7 +267,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     constexpr size_t ESZ = (DT == kF32) ? 4 : 2;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ FlowShared sh;
-    // Each worker thread streams its own vectors through a private ring of 16-byte slots filled
+    // Each worker thread streams its own vectors through a private ring of 16-byte cells filled
     // by cp.async, so loads run kFAhead steps ahead of the arithmetic without costing registers.
     extern __shared__ __align__(16) unsigned char dyn[];
 
