@@ -29,7 +29,7 @@
  *   uniforms[b, gamma]   drives the residual sample (tau < gamma)
  *   uniforms[b, gamma+1] drives the target sample   (tau == gamma)
  *
- * Readings taken where the paper is silent (each is listed in the design doc):
+ * Readings taken where the paper is silent:
  *   - temperature divides both models' logits before the softmax;
  *   - a position is selectable only if its acceptance weight is > 0, and
  *     h_i := 0 when S_i = 0 (the 0/0 case of Eq. "pacc_block");

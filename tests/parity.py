@@ -157,7 +157,7 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
             rel_p = float((np.abs(p[m] - ref.p[m]) / np.maximum(ref.p[m], 1e-30)).max())
             pS = ref.p[:, :-1]
             # h_i = S_i / (S_i + 1 - p_i), 1 <= i < gamma: propagate the S and p tolerances.
-            # Positions with S_i = 0 are skipped: h_i is then immaterial.
+            # Positions with S_i = 0 are skipped: there h_i := 0 by convention and decides nothing.
             g = ref.S.shape[1]
             for i in range(1, g):
                 Sr, pr, hr = ref.S[:, i], ref.p[:, i], ref.h[:, i]
@@ -202,7 +202,7 @@ def assert_parity(rep: ParityReport, check_diag=True):
     # an eta within 1e-6 of h_i: at most 1e-4 of trials may differ for that reason
     assert rep.excused_tau <= int(np.ceil(1e-4 * rep.trials)), str(rep)
     # the sampling uniform has one threshold per vocabulary entry; an fp32 CDF places each
-    # within ~1e-7, so the expected share of differing tokens grows with V (see DESIGN.md)
+    # within ~1e-7, so the expected share of differing tokens grows with V
     assert rep.excused_Y <= int(np.ceil(rep.trials * (1e-4 + 2e-7 * rep.vocab))), str(rep)
     if check_diag:
         assert rep.max_abs_lse <= 3e-6, str(rep)
