@@ -52,6 +52,9 @@ def _load():
         lib.oracle_verify.restype = ctypes.c_int
         lib.oracle_verify.argtypes = [ip, vp, vp, vp, vp, ip, ip, ip, ip, ctypes.c_double,
                                       vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_verify_lse.restype = ctypes.c_int
+        lib.oracle_verify_lse.argtypes = [ip, vp, vp, vp, vp, vp, ip, ip, ip, ip, ctypes.c_double,
+                                          vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_threads.restype = ctypes.c_int
         lib.oracle_sample_rows.restype = ctypes.c_int
         lib.oracle_sample_rows.argtypes = [vp, vp, ip, ip, ip, ctypes.c_double, vp, vp, vp]
@@ -78,7 +81,7 @@ class OracleResult:
 
 
 def verify(algo: int, target: np.ndarray, draft: np.ndarray, tokens: np.ndarray,
-           uniforms: np.ndarray, temperature: float = 1.0) -> OracleResult:
+           uniforms: np.ndarray, temperature: float = 1.0, draft_lse=None) -> OracleResult:
     """Run Algorithm 1 (algo=TOKEN_VERIFY) or Algorithm 2 (algo=BLOCK_VERIFY).
 
     target [B, gamma+1, V] and draft [B, gamma, V] share a dtype: float32,
@@ -105,7 +108,14 @@ def verify(algo: int, target: np.ndarray, draft: np.ndarray, tokens: np.ndarray,
         lse_t=np.empty((B, gamma + 1)), lse_d=np.empty((B, gamma)),
         margin_eta=np.empty((B,)), margin_smp=np.empty((B,)))
     ptr = lambda a: a.ctypes.data_as(ctypes.c_void_p)
-    rc = lib.oracle_verify(int(algo), ptr(target), ptr(draft), ptr(tokens), ptr(uniforms),
+    fn, extra = lib.oracle_verify, []
+    if draft_lse is not None:
+        # the draft rows' log-normalisers are supplied (float32 [B, gamma]) instead of computed
+        draft_lse = np.ascontiguousarray(draft_lse, dtype=np.float32)
+        if draft_lse.shape != (B, gamma):
+            raise ValueError("draft_lse must be [B, gamma]")
+        fn, extra = lib.oracle_verify_lse, [ptr(draft_lse)]
+    rc = fn(int(algo), ptr(target), ptr(draft), ptr(tokens), ptr(uniforms), *extra,
                            B, gamma, V, _DTYPE_CODE[target.dtype],
                            float(np.float32(temperature)),
                            ptr(res.out_tokens), ptr(res.out_len), ptr(res.p), ptr(res.S),

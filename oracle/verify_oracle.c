@@ -157,12 +157,30 @@ typedef struct {
     int gamma, V, dtype;
     double T;
     size_t toff, doff;  /* offset of row 0 of this sequence in tgt / drf */
+    const float *given_lse_d; /* gamma supplied draft log-normalisers, or NULL: compute them */
 } seq_t;
 
 typedef struct {
     double *p, *S, *h, *lse_t, *lse_d; /* per-sequence slices, may be NULL */
     double *margin_eta, *margin_smp;   /* one value each, may be NULL      */
 } diag_t;
+
+/*
+ * Log-normaliser of draft row r: computed from the row, or, when the caller supplies the
+ * normalisers (the drafting step has them already), the supplied value: M_s(x | c, X^r) is then
+ * exp(z_x / T - supplied).  Returns 1 on a domain error (a supplied value that is not finite).
+ */
+static int draft_lse(const seq_t *s, int r, double *out)
+{
+    if (s->given_lse_d) {
+        double v = (double)s->given_lse_d[r];
+        if (!isfinite(v))
+            return 1;
+        *out = v;
+        return 0;
+    }
+    return row_lse(s->drf, s->dtype, s->doff + (size_t)r * (size_t)s->V, s->V, s->T, out);
+}
 
 static void diag_fill_nan(const diag_t *d, int gamma)
 {
@@ -223,7 +241,7 @@ static void token_verify_one(const seq_t *s, const diag_t *d,
     for (int i = 1; i <= g; ++i) {
         /* the distributions conditioned on X^{i-1} */
         if (row_lse(s->tgt, s->dtype, s->toff + (size_t)(i - 1) * V, s->V, s->T, &lse_t) ||
-            row_lse(s->drf, s->dtype, s->doff + (size_t)(i - 1) * V, s->V, s->T, &lse_d)) {
+            draft_lse(s, i - 1, &lse_d)) {
             emit(s, -1, -1, out_tokens, out_len);
             return;
         }
@@ -255,7 +273,7 @@ static void token_verify_one(const seq_t *s, const diag_t *d,
     if (d->lse_t) d->lse_t[tau] = lse_t;
     int have_draft = tau < g;
     if (have_draft) {
-        if (row_lse(s->drf, s->dtype, s->doff + (size_t)tau * V, s->V, s->T, &lse_d)) {
+        if (draft_lse(s, tau, &lse_d)) {
             emit(s, -1, -1, out_tokens, out_len);
             return;
         }
@@ -291,7 +309,7 @@ static void block_verify_one(const seq_t *s, const diag_t *d,
     for (int r = 0; r <= g && !bad; ++r) {
         bad |= row_lse(s->tgt, s->dtype, s->toff + (size_t)r * V, s->V, s->T, &lse_t[r]);
         if (r < g)
-            bad |= row_lse(s->drf, s->dtype, s->doff + (size_t)r * V, s->V, s->T, &lse_d[r]);
+            bad |= draft_lse(s, r, &lse_d[r]);
     }
 
     /* p_0 = 1;  p_i = min{ p_{i-1} * M_b(X_i|c,X^{i-1}) / M_s(X_i|c,X^{i-1}), 1 } */
@@ -375,8 +393,8 @@ done:
  * Sequences are independent; the loop over b may run on several threads.
  * Returns 0, or 1 for an invalid argument.
  */
-int oracle_verify(int algo, const void *target, const void *draft,
-                  const int32_t *tokens, const float *uniforms,
+static int verify_impl(int algo, const void *target, const void *draft,
+                  const int32_t *tokens, const float *uniforms, const float *given_lse_d,
                   int B, int gamma, int V, int dtype, double temperature,
                   int32_t *out_tokens, int32_t *out_len,
                   double *p, double *S, double *h, double *lse_t, double *lse_d,
@@ -399,6 +417,7 @@ int oracle_verify(int algo, const void *target, const void *draft,
         s.gamma = gamma; s.V = V; s.dtype = dtype; s.T = temperature;
         s.toff = (size_t)b * (size_t)(gamma + 1) * (size_t)V;
         s.doff = (size_t)b * (size_t)gamma * (size_t)V;
+        s.given_lse_d = given_lse_d ? given_lse_d + (size_t)b * (size_t)gamma : NULL;
         diag_t d;
         d.p = p ? p + (size_t)b * (size_t)(gamma + 1) : NULL;
         d.S = S ? S + (size_t)b * (size_t)gamma : NULL;
@@ -414,6 +433,35 @@ int oracle_verify(int algo, const void *target, const void *draft,
             token_verify_one(&s, &d, ot, out_len + b);
     }
     return 0;
+}
+
+int oracle_verify(int algo, const void *target, const void *draft,
+                  const int32_t *tokens, const float *uniforms,
+                  int B, int gamma, int V, int dtype, double temperature,
+                  int32_t *out_tokens, int32_t *out_len,
+                  double *p, double *S, double *h, double *lse_t, double *lse_d,
+                  double *margin_eta, double *margin_smp)
+{
+    return verify_impl(algo, target, draft, tokens, uniforms, NULL, B, gamma, V, dtype, temperature,
+                       out_tokens, out_len, p, S, h, lse_t, lse_d, margin_eta, margin_smp);
+}
+
+/*
+ * The same with the draft rows' log-normalisers supplied, given_lse_d [B, gamma] float
+ * (ln sum_x exp(draft[b, r, x] / T), as the drafting step leaves them): the draft distributions
+ * are exp(z / T - given).  Everything else as oracle_verify.
+ */
+int oracle_verify_lse(int algo, const void *target, const void *draft,
+                      const int32_t *tokens, const float *uniforms, const float *given_lse_d,
+                      int B, int gamma, int V, int dtype, double temperature,
+                      int32_t *out_tokens, int32_t *out_len,
+                      double *p, double *S, double *h, double *lse_t, double *lse_d,
+                      double *margin_eta, double *margin_smp)
+{
+    if (!given_lse_d)
+        return 1;
+    return verify_impl(algo, target, draft, tokens, uniforms, given_lse_d, B, gamma, V, dtype,
+                       temperature, out_tokens, out_len, p, S, h, lse_t, lse_d, margin_eta, margin_smp);
 }
 
 /*

@@ -361,3 +361,43 @@ def test_draft_sampler_domain_errors():
     tok, lse, _ = oracle.sample_rows(z, np.full(3, 0.5, np.float32), 1.0)
     assert tok[0] == -1 and tok[1] == -1 and tok[2] == 2
     assert np.isnan(lse[0]) and np.isnan(lse[1]) and abs(lse[2] - np.log(5)) < 1e-15
+
+
+# ---------------- supplied draft normalisers (oracle_verify_lse) ----------------
+@pytest.mark.parametrize("algo", [oracle.BLOCK_VERIFY, oracle.TOKEN_VERIFY])
+def test_supplied_draft_normalisers(algo):
+    rng = np.random.default_rng(8)
+    B, g, V = 6, 4, 300
+    tgt = rng.normal(size=(B, g + 1, V)) * 2
+    drf = tgt[:, :g] + rng.normal(size=(B, g, V)) * 0.7
+    tok = rng.integers(0, V, size=(B, g)).astype(np.int32)
+    uni = rng.random((B, g + 2), dtype=np.float32)
+    base = oracle.verify(algo, tgt, drf, tok, uni, 0.9)
+    # (a) the normalisers the oracle computes itself, rounded to float32, change nothing beyond
+    #     that rounding (2e-6 absolute in lse, hence 2e-6 relative in Q)
+    own = logsumexp(drf / np.float32(0.9), axis=-1).astype(np.float32)
+    res = oracle.verify(algo, tgt, drf, tok, uni, 0.9, draft_lse=own)
+    m = ~np.isnan(base.lse_d)
+    assert np.array_equal(res.lse_d[m], own.astype(np.float64)[m])
+    if algo == oracle.BLOCK_VERIFY:
+        assert np.allclose(res.p, base.p, rtol=2e-5) and np.allclose(res.S, base.S, rtol=0, atol=1e-5)
+    # (b) the supplied value is really what is used: shifting row r's normaliser by d multiplies
+    #     Q_r by exp(-d), so the ratio P_r(X)/Q_r(X) grows by exp(d): written out for p_1
+    shifted = own.copy()
+    shifted[:, 0] += np.float32(0.25)
+    res2 = oracle.verify(algo, tgt, drf, tok, uni, 0.9, draft_lse=shifted)
+    if algo == oracle.BLOCK_VERIFY:
+        x = tok[:, 0]
+        lp = tgt[np.arange(B), 0, x] / np.float32(0.9) - logsumexp(tgt[:, 0] / np.float32(0.9), axis=-1)
+        lq = drf[np.arange(B), 0, x] / np.float32(0.9) - shifted[:, 0].astype(np.float64)
+        assert np.allclose(res2.p[:, 1], np.minimum(np.exp(lp - lq), 1.0), rtol=1e-12)
+        # and S_0 = sum max(P_0 - Q_0 e^{-d}, 0) with the shifted normaliser
+        P0 = np.exp(tgt[:, 0] / np.float32(0.9) - logsumexp(tgt[:, 0] / np.float32(0.9), axis=-1)[:, None])
+        Q0 = np.exp(drf[:, 0] / np.float32(0.9) - shifted[:, 0].astype(np.float64)[:, None])
+        assert np.allclose(res2.S[:, 0], np.maximum(P0 - Q0, 0).sum(-1), rtol=1e-11)
+    # (c) a supplied value that is not finite is a domain error of that sequence only
+    broken = own.copy()
+    broken[2, 1] = np.nan
+    res3 = oracle.verify(algo, tgt, drf, tok, uni, 0.9, draft_lse=broken)
+    if algo == oracle.BLOCK_VERIFY:
+        assert res3.out_len[2] == -1 and (res3.out_len[[0, 1, 3, 4, 5]] > 0).all()
