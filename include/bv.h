@@ -161,6 +161,31 @@ int bv_verify_noalloc(const void* target_logits, const void* draft_logits,
                       int32_t* out_tokens, int32_t* out_len, void* stream);
 
 /*
+ * Block Verification with the draft rows' log-normalisers supplied:
+ *   draft_lse [B, gamma] float, DEVICE: ln sum_x exp(draft_logits[b, r, x] / temperature),
+ *   as bv_sample_draft() leaves them when the drafting step runs through this library.
+ * The draft distributions of Algorithm 2 are then M_s(x | c, X^r) = exp(z_x / T - draft_lse[b, r]),
+ * and the first sweep does not read the draft rows at all: they are read only for the few positions
+ * whose residual mass S_r (Eq. "pacc_block") is needed, so a call moves about half the bytes of
+ * bv_verify().  A float normaliser carries about 2e-6 relative error into M_s; the emitted tokens
+ * keep the target model's law to that accuracy.  A draft_lse entry that is not finite is a data
+ * fault of its sequence (out_len = -1); the contents of a draft row are otherwise trusted.
+ * Only the 128-bit path exists (rows of whole 16-byte vectors on 16-byte aligned bases), else
+ * BV_ERR_UNSUPPORTED.  Other arguments, outputs and diagnostics as bv_verify / bv_verify_ex
+ * (out_lse_d returns the supplied values).
+ */
+int bv_verify_lse(const void* target_logits, const void* draft_logits,
+                  const int32_t* draft_tokens, const float* uniforms, const float* draft_lse,
+                  int B, int gamma, int V, int dtype, float temperature,
+                  int32_t* out_tokens, int32_t* out_len, void* stream);
+int bv_verify_lse_ex(const void* target_logits, const void* draft_logits,
+                     const int32_t* draft_tokens, const float* uniforms, const float* draft_lse,
+                     int B, int gamma, int V, int dtype, float temperature,
+                     int32_t* out_tokens, int32_t* out_len,
+                     float* out_p, float* out_S, float* out_h,
+                     float* out_lse_t, float* out_lse_d, void* stream);
+
+/*
  * The drafting step of Algorithm 3 ("Sample X_1, ..., X_gamma ~ M_s using autoregressive sampling,
  * keep the conditional probabilities at each step") for `rows` rows of draft logits [rows, V]:
  *   out_tokens[r] ~ softmax(logits[r, :] / temperature), drawn by inverse CDF in vocabulary-index

@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_verify_noalloc", "bv_sample_draft", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "bv_sample_draft", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -55,6 +55,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     for name in ("bv_verify_host", "tv_verify_host"):
         getattr(lib, name).argtypes = base
     lib.bv_sample_draft.argtypes = [vp, vp, ci, ci, ci, cf, vp, vp, vp]
+    lib.bv_verify_lse.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp]
+    lib.bv_verify_lse_ex.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp, vp, vp, vp, vp, vp]
     for name in EXPORTS:
         getattr(lib, name).restype = ci
     lib.bv_status_string.restype = ctypes.c_char_p
@@ -240,3 +242,31 @@ def bv_sample_draft(logits, uniforms, temperature: float = 1.0, want_lse: bool =
                                    float(temperature), tokens.data_ptr(), lse.data_ptr() if want_lse else None,
                                    st.cuda_stream))
     return tokens, lse
+
+
+def bv_verify_lse(target_logits, draft_logits, draft_tokens, uniforms, draft_lse, temperature: float = 1.0,
+                  diagnostics: bool = False, stream=None):
+    """Block Verification with the draft rows' log-normalisers supplied (float32 CUDA tensor
+    [B, gamma], e.g. the second output of bv_sample_draft reshaped).  Returns (out_tokens, out_len)
+    or, with ``diagnostics``, (out_tokens, out_len, dict of p, S, h, lse_t, lse_d)."""
+    lib = load_library()
+    B, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms, True)
+    if (not draft_lse.is_cuda or draft_lse.dtype != torch.float32 or tuple(draft_lse.shape) != (B, gamma)
+            or not draft_lse.is_contiguous()):
+        raise ValueError("draft_lse must be a contiguous float32 CUDA tensor of [B, gamma]")
+    dev = target_logits.device
+    out_tokens = torch.empty((B, gamma + 1), dtype=torch.int32, device=dev)
+    out_len = torch.empty((B,), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        s = stream if stream is not None else torch.cuda.current_stream(dev)
+        args = [target_logits.data_ptr(), draft_logits.data_ptr(), draft_tokens.data_ptr(), uniforms.data_ptr(),
+                draft_lse.data_ptr(), B, gamma, V, _dtype_code(target_logits), float(temperature),
+                out_tokens.data_ptr(), out_len.data_ptr()]
+        if diagnostics:
+            f = lambda *shape: torch.empty(shape, dtype=torch.float32, device=dev)
+            diag = dict(p=f(B, gamma + 1), S=f(B, gamma), h=f(B, gamma + 1), lse_t=f(B, gamma + 1), lse_d=f(B, gamma))
+            args += [diag[k].data_ptr() for k in ("p", "S", "h", "lse_t", "lse_d")]
+            _check(lib.bv_verify_lse_ex(*args, s.cuda_stream))
+            return out_tokens, out_len, diag
+        _check(lib.bv_verify_lse(*args, s.cuda_stream))
+    return out_tokens, out_len

@@ -18,6 +18,7 @@ struct Params {
     const void* drf;          // [B, gamma,   V]
     const int32_t* tok;       // [B, gamma]
     const float* uni;         // [B, gamma+2]
+    const float* lse_d;       // [B, gamma] supplied draft log-normalisers ln sum exp(z/T), or null: computed
     int B, gamma, V;
     float kf;                 // log2(e) / T, rounded to float (per-element scale)
     double kd;                // log2(e) / T in double (scalar recursion)

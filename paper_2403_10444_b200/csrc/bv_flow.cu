@@ -301,10 +301,11 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             const int ch = static_cast<int>(t % cx.nch);
             const int r = static_cast<int>(t / cx.nch) % g, b = static_cast<int>(t / cx.nch) / g;
             const int ri = b * (g + 1) + r;
-            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = 1;
+            // (with supplied draft normalisers the first sweep has nothing to learn from the draft row)
+            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = prm.lse_d == nullptr;
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
-            d.rowQ = r < g ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
-                           : nullptr;
+            d.rowQ = d.have_q ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
+                              : nullptr;
             d.cp = 1.f; d.nMP = 0.f; d.nMQ = 0.f;
         };
         // Rows whose second sweep has been started stand in a queue, each cut into np pieces.  A

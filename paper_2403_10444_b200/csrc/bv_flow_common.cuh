@@ -433,6 +433,15 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
         ZP += z.ZP * static_cast<double>(ref_scale(static_cast<float>(z.MP), static_cast<float>(MP)));
         ZQ += z.ZQ * static_cast<double>(ref_scale(static_cast<float>(z.MQ), static_cast<float>(MQ)));
     }
+    if (prm.lse_d != nullptr && r < g) {
+        // the draft row's normaliser is supplied: as an integer reference at or above every scaled
+        // logit of the row plus a sum in [2^-1/2, 2^1/2]; a value that is not finite leaves the
+        // row without a reference, which marks the block as faulty below
+        const double L2 = static_cast<double>(prm.lse_d[static_cast<size_t>(b) * g + r]) * 1.4426950408889634073599246810019;
+        const bool fin = L2 > -1e300 && L2 < 1e300;
+        MQ = fin ? rint(L2) : static_cast<double>(kNoRef);
+        ZQ = fin ? exp2(L2 - MQ) : 0.0;
+    }
     f_row_publish<DT>(prm, fl, cx, b, r, MP, ZP, MQ, ZQ);
 }
 
