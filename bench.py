@@ -112,7 +112,7 @@ def time_oracle(w, algo_name: str, budget_s: float = 20.0):
     """The CPU oracle, as it stands, on a bounded sample of the workload."""
     import numpy as np
     import oracle
-    algo = oracle.BLOCK_VERIFY if algo_name == "block" else oracle.TOKEN_VERIFY
+    algo = oracle.BLOCK_VERIFY if algo_name in ("block", "block_lse") else oracle.TOKEN_VERIFY
     cores = oracle.threads()
     # one sequence first to size the sample for about budget_s of work
     probe = wl.make_inputs(wl.scaled(w, B=max(1, min(w.B, cores))), "cpu")
@@ -123,11 +123,16 @@ def time_oracle(w, algo_name: str, budget_s: float = 20.0):
             t = t.view(torch.int16).numpy().view(np.uint16); d = d.view(torch.int16).numpy().view(np.uint16)
         else:
             t = t.numpy(); d = d.numpy()
+        if algo_name == "block_lse" and "draft_lse" not in inp:      # (outside the timed part)
+            inp["draft_lse"] = torch.logsumexp(inp["draft_logits"].double() / inp["temperature"], -1).float().numpy()
         t0 = time.perf_counter()
         if algo_name == "sample":
             g = inp["draft_tokens"].shape[1]
             oracle.sample_rows(d.reshape(-1, d.shape[-1]), inp["uniforms"].numpy()[:, :g].reshape(-1).copy(),
                                inp["temperature"])
+        elif algo_name == "block_lse":
+            oracle.verify(algo, t, d, inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), inp["temperature"],
+                          draft_lse=inp["draft_lse"])
         else:
             oracle.verify(algo, t, d, inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), inp["temperature"])
         return time.perf_counter() - t0
@@ -146,7 +151,7 @@ def time_oracle(w, algo_name: str, budget_s: float = 20.0):
     dt /= reps
     return {"value": n * w.gamma / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": "first %d of %d sequences of workload %s (%s), %d passes of %.2f s" % (
-                n, w.B, w.name, "drafting step" if algo_name == "sample" else algo_name + " verify", reps, dt),
+                n, w.B, w.name, "drafting step" if algo_name == "sample" else algo_name.replace("_lse", " with supplied draft normalisers") + " verify", reps, dt),
             "seconds": dt, "sequences": n}
 
 
@@ -182,8 +187,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(wl.CONFIGS))
-    ap.add_argument("--algo", default="block", choices=["block", "token", "sample"],
-                    help="block / token verification, or the drafting step (sampling the draft rows)")
+    ap.add_argument("--algo", default="block", choices=["block", "token", "sample", "block_lse"],
+                    help="block / token verification, the drafting step (sampling the draft rows), or block "
+                         "verification with the draft normalisers that the drafting step leaves")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
@@ -215,6 +221,13 @@ def main():
         u_rows = inp["uniforms"][:, : w.gamma].contiguous().view(-1)
         fn = lambda *_: bv.bv_sample_draft(rows2d, u_rows, inp["temperature"])
         args.e2e_steps = 0          # (no host-buffer form of this entry point)
+    if args.algo == "block_lse":
+        # normalisers as the drafting step leaves them, computed once outside the timed region
+        lse = bv.bv_sample_draft(inp["draft_logits"].view(w.B * w.gamma, w.V),
+                                 inp["uniforms"][:, : w.gamma].contiguous().view(-1), inp["temperature"])[1]
+        lse = lse.view(w.B, w.gamma).contiguous()
+        fn = lambda *_: bv.bv_verify_lse(*a[:4], lse, a[4])
+        args.e2e_steps = 0
 
     def barrier():
         if dist is not None:
@@ -288,6 +301,10 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
     if args.algo == "sample":
         algo_bytes = w.B * w.gamma * w.V * esz
         kernel = "sample_rows_kernel"
+    elif args.algo == "block_lse":
+        # what must be read at least: every target row, and one draft row per block for the residual
+        algo_bytes = w.B * (w.gamma + 2) * w.V * esz
+        kernel = "verify_flow_kernel"
     elif args.algo == "block":
         # Algorithm 2 needs every row: B (2 gamma + 1) V elements
         algo_bytes = w.logit_bytes

@@ -151,7 +151,8 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
         }
         if (per_sm > 0) {
             const long long units = static_cast<long long>(row_bytes / 16);
-            int nch = bv::flow_pick_chunks(units, B, gamma, static_cast<long long>(d->sm_count) * per_sm);
+            // (with supplied draft normalisers a first-sweep item streams one row, not two)
+            int nch = bv::flow_pick_chunks(prm.lse_d ? units / 2 : units, B, gamma, static_cast<long long>(d->sm_count) * per_sm);
             if (const char* env = std::getenv("BV_FLOW_CHUNKS")) {
                 const int v = std::atoi(env);
                 if (v >= 1 && v <= bv::kFlowMaxChunks) nch = v;

@@ -192,7 +192,11 @@ __device__ __forceinline__ void f_sweep_segment(uint32_t sb, const char* rowP, c
                                                 float& oMP, float& osP, float& oMQ, float& osQ) {
     using R = Raw<DT>;
     constexpr int EPV = R::EPV;
-    constexpr uint32_t kSlot = kFThreads * 16;               // bytes between consecutive ring slots
+    constexpr uint32_t kSlot = kFThreads * 16;               // bytes between consecutive ring cells
+    // a step takes two of the thread's ring cells, or one when there is no draft row: then the
+    // loads run twice as many steps ahead, so that as many bytes are in flight
+    constexpr int kA = HAVEQ ? kFAhead : kFDepth;
+    constexpr int kC = HAVEQ ? 2 : 1;
     const int nv = w1 - w0;
     const int nsteps = (nv + 31) >> 5;
     const int nlast = nv - 32 * (nsteps - 1);                // lanes that take part in the last step
@@ -201,27 +205,27 @@ __device__ __forceinline__ void f_sweep_segment(uint32_t sb, const char* rowP, c
     // sweep 1 asks L2 to keep the rows (they are read again soon); sweep 2 marks them as done with
     // no row is needed again soon (the few second sweeps come long after the first): stream past L2
     const uint64_t pol = l2_policy_evict_first();
-    auto fetch_step = [&](int k, int j) {                    // step k goes to slots 2j, 2j+1 (j = k & 3)
+    auto fetch_step = [&](int k, int j) {                    // step k goes to cells kC j (, + 1), j = k mod kA
         if (k < nsteps) {
             const bool ok = (k + 1 < nsteps) || lane < nlast;
-            ring_fetch_hint(sb + (2 * j) * kSlot, gP + static_cast<size_t>(k) * 512, ok, R::kNegInf, pol);
-            if (HAVEQ) ring_fetch_hint(sb + (2 * j + 1) * kSlot, gQ + static_cast<size_t>(k) * 512, ok, R::kNegInf, pol);
+            ring_fetch_hint(sb + (kC * j) * kSlot, gP + static_cast<size_t>(k) * 512, ok, R::kNegInf, pol);
+            if (HAVEQ) ring_fetch_hint(sb + (kC * j + 1) * kSlot, gQ + static_cast<size_t>(k) * 512, ok, R::kNegInf, pol);
         }
         cp_async_commit();
     };
 #pragma unroll
-    for (int j = 0; j < kFAhead; ++j) fetch_step(j, j);
+    for (int j = 0; j < kA; ++j) fetch_step(j, j);
 
     float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f, acc = 0.f;
-    for (int kb = 0; kb < nsteps; kb += kFAhead) {
+    for (int kb = 0; kb < nsteps; kb += kA) {
 #pragma unroll
-        for (int j = 0; j < kFAhead; ++j) {
+        for (int j = 0; j < kA; ++j) {
             const int k = kb + j;
             if (k < nsteps) {
-                cp_async_wait<kFAhead - 1>();                // step k of both rows has landed
+                cp_async_wait<kA - 1>();                     // step k has landed
                 float vp[EPV], vq[EPV];
-                R::unpack(lds128(sb + (2 * j) * kSlot), vp);
-                if (HAVEQ) R::unpack(lds128(sb + (2 * j + 1) * kSlot), vq);
+                R::unpack(lds128(sb + (kC * j) * kSlot), vp);
+                if (HAVEQ) R::unpack(lds128(sb + (kC * j + 1) * kSlot), vq);
                 if (KIND == kSweep1) {
                     if (j == 0 && kb == 0) {                 // references from the first vector of every lane
                         MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
@@ -247,7 +251,7 @@ __device__ __forceinline__ void f_sweep_segment(uint32_t sb, const char* rowP, c
                     float t[EPV];
                     acc += f_pair_sum<EPV, HAVEQ>(vp, vq, kf, cp, nMP, nMQ, t);
                 }
-                fetch_step(k + kFAhead, j);
+                fetch_step(k + kA, j);
             }
         }
     }
