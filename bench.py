@@ -347,6 +347,7 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
 TRAFFIC_BYTES = {
     ("c4", "block", "verify_flow_kernel"): 2492403456,
     ("c4", "sample", "sample_rows_kernel"): 1054102784,
+    ("c4", "block_lse", "verify_flow_kernel"): 1438274816,
 }
 
 
