@@ -260,6 +260,20 @@ def main():
     ms_per_step = total_ms / args.steps
     value = sharding.whole_job_rate(w.B * w.gamma, ms_per_step)
 
+    # ---- for the record: the same call with every position evaluated in full (diagnostic entry) ----
+    full_ms = None
+    if args.algo == "block":
+        for _ in range(2):
+            bv.bv_verify_ex(*a)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(5):
+            bv.bv_verify_ex(*a)
+        f1.record()
+        f1.synchronize()
+        full_ms = f0.elapsed_time(f1) / 5
+    args.full_ms = full_ms
+
     # ---- end to end: host buffers through the C-ABI host entry, copies inside the timed region ----
     e2e = None
     if args.e2e_steps > 0:
@@ -324,7 +338,10 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
         "config": {"workload": w.name, "B": w.B, "gamma": w.gamma, "V": w.V, "storage": w.dtype,
                    "temperature": w.temperature, "algo": args.algo, "parallelism": "batch-sharded x%d" % world,
                    "l2": "inputs (%.2f GB per step) exceed L2" % (w.logit_bytes / 1e9),
-                   "mean_emitted_len": mean_len},
+                   "mean_emitted_len": mean_len,
+                   # Algorithm 2's residual masses are evaluated only for positions that can be the selected
+                   # one (h_i <= p_i), with identical outputs; the time with all of them evaluated:
+                   "all_positions_ms_per_step": getattr(args, "full_ms", None)},
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": launches,
