@@ -73,6 +73,15 @@ MUTATIONS = [
     ("normaliser without the maximum added back",
      "*lse_out = m + log(s);",
      "*lse_out = log(s);"),
+    ("supplied draft normaliser ignored",
+     "    if (s->given_lse_d) {\n        double v = (double)s->given_lse_d[r];",
+     "    if (0 && s->given_lse_d) {\n        double v = (double)s->given_lse_d[r];"),
+    ("supplied draft normaliser of the wrong row",
+     "double v = (double)s->given_lse_d[r];",
+     "double v = (double)s->given_lse_d[r > 0 ? r - 1 : r];"),
+    ("drafting step samples with the verification's other uniform convention (token after)",
+     "1.0, (double)uniforms[r], &W, &m);",
+     "1.0, 1.0 - (double)uniforms[r], &W, &m);"),
     ("token verification without the min with 1",
      "double h = ratio < 1.0 ? ratio : 1.0;       /* h_i^token = min(ratio, 1) */",
      "double h = ratio;"),
@@ -105,6 +114,11 @@ def _compile(text, tmp_path, tag):
     lib.oracle_verify.restype = ctypes.c_int
     lib.oracle_verify.argtypes = [ip, vp, vp, vp, vp, ip, ip, ip, ip, ctypes.c_double,
                                   vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.oracle_verify_lse.restype = ctypes.c_int
+    lib.oracle_verify_lse.argtypes = [ip, vp, vp, vp, vp, vp, ip, ip, ip, ip, ctypes.c_double,
+                                      vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.oracle_sample_rows.restype = ctypes.c_int
+    lib.oracle_sample_rows.argtypes = [vp, vp, ip, ip, ip, ctypes.c_double, vp, vp, vp]
     lib.oracle_threads.restype = ctypes.c_int
     return lib
 
@@ -132,6 +146,8 @@ def _pins():
     yield lambda: pins.test_gamma1_bit_identical_outputs()
     yield lambda: pins.test_normalisers_reduce_to_scipy_logsumexp(np.float32)
     yield lambda: pins.test_lossless_by_brute_force_over_blocks_and_uniforms(oracle.BLOCK_VERIFY, "block")
+    yield lambda: pins.test_supplied_draft_normalisers(oracle.BLOCK_VERIFY)
+    yield lambda: pins.test_draft_sampler_frequencies_are_the_softmax()
 
 
 def _caught():
