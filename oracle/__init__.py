@@ -1,7 +1,8 @@
 """TEST INFRASTRUCTURE -- not part of the product path.
 
-Loader for the fp64 CPU oracle of Token Verification (Algorithm 1) and Block
-Verification (Algorithm 2) of arXiv 2403.10444, written in plain C in
+Loader for the fp64 CPU oracle of Token Verification (Algorithm 1), Block
+Verification (Algorithm 2) and Greedy Block Verification (Algorithm 4, one
+iteration) of arXiv 2403.10444, written in plain C in
 ``verify_oracle.c``.  Only tests, the smoke check and the benchmark's
 CPU-baseline leg may import this package; the CUDA library never does, and
 this package never imports the CUDA library.
@@ -25,6 +26,7 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 
 TOKEN_VERIFY = 0
 BLOCK_VERIFY = 1
+GREEDY_BLOCK_VERIFY = 2
 
 _DTYPE_CODE = {np.dtype(np.float32): 0, np.dtype(np.uint16): 1, np.dtype(np.float64): 2}
 
@@ -82,7 +84,9 @@ class OracleResult:
 
 def verify(algo: int, target: np.ndarray, draft: np.ndarray, tokens: np.ndarray,
            uniforms: np.ndarray, temperature: float = 1.0, draft_lse=None) -> OracleResult:
-    """Run Algorithm 1 (algo=TOKEN_VERIFY) or Algorithm 2 (algo=BLOCK_VERIFY).
+    """Run Algorithm 1 (algo=TOKEN_VERIFY), Algorithm 2 (algo=BLOCK_VERIFY) or
+    Algorithm 4 (algo=GREEDY_BLOCK_VERIFY: p holds the unclipped products, S the numerator
+    sums and h the printed ratios, which may exceed 1 or be +inf).
 
     target [B, gamma+1, V] and draft [B, gamma, V] share a dtype: float32,
     float64, or uint16 holding bf16 bit patterns.  tokens [B, gamma] int32,
@@ -128,6 +132,10 @@ def verify(algo: int, target: np.ndarray, draft: np.ndarray, tokens: np.ndarray,
 
 def block_verify(*a, **k) -> OracleResult:
     return verify(BLOCK_VERIFY, *a, **k)
+
+
+def greedy_block_verify(*a, **k) -> OracleResult:
+    return verify(GREEDY_BLOCK_VERIFY, *a, **k)
 
 
 def token_verify(*a, **k) -> OracleResult:

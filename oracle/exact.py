@@ -1,7 +1,8 @@
 """TEST INFRASTRUCTURE -- not part of the product path.
 
-Exact laws of Token Verification (Algorithm 1) and Block Verification
-(Algorithm 2) of arXiv 2403.10444 on tiny vocabularies, with the algorithm's
+Exact laws of Token Verification (Algorithm 1), Block Verification
+(Algorithm 2) and Greedy Block Verification (Algorithm 4, with the distribution
+modification of Algorithm 5) of arXiv 2403.10444 on tiny vocabularies, with the algorithm's
 own randomness (eta_1..eta_gamma and the draw of Y) integrated out
 analytically.  Works in any exact or floating number type: pass probabilities
 as ``fractions.Fraction`` for exact rational results.
@@ -53,6 +54,38 @@ def block_quantities(P: Model, Q: Model, block: Tuple[int, ...]):
         h.append(S[i] / (S[i] + 1 - p[i]) if S[i] > 0 else 0)
     h.append(p[g])
     return p, S, h
+
+
+def greedy_quantities(P: Model, Q: Model, block: Tuple[int, ...]):
+    """Algorithm 4 for one drafted block: the unclipped products
+    pt_i = pt_{i-1} M_b(X_i|.)/M_s(X_i|.), the two sums of its "Set h_i" line
+    (num_i = sum_x max(pt_i M_b - M_s, 0), den_i = sum_x max(M_s - pt_i M_b, 0)) and the
+    probabilities min(h_i, 1) with which position i passes its test (h_gamma = pt_gamma;
+    0 when num_i = 0, the reading taken for an empty residual).
+
+    Returns (pt[0..gamma], num[0..gamma-1], den[0..gamma-1], a[0..gamma]) with a[0] = 1.
+    """
+    g = len(block)
+    pt = [1]
+    for i in range(1, g + 1):
+        ctx = block[: i - 1]
+        x = block[i - 1]
+        pt.append(pt[i - 1] * P(ctx)[x] / Q(ctx)[x])
+    num, den = [], []
+    for i in range(g):
+        Pi, Qi = P(block[:i]), Q(block[:i])
+        num.append(sum(max(pt[i] * a - b, 0) for a, b in zip(Pi, Qi)))
+        den.append(sum(max(b - pt[i] * a, 0) for a, b in zip(Pi, Qi)))
+    acc = [1]
+    for i in range(1, g):
+        if num[i] == 0:
+            acc.append(0)
+        elif den[i] == 0 or num[i] >= den[i]:
+            acc.append(1)
+        else:
+            acc.append(num[i] / den[i])
+    acc.append(pt[g] if pt[g] < 1 else 1)
+    return pt, num, den, acc
 
 
 def token_quantities(P: Model, Q: Model, block: Tuple[int, ...]):
@@ -118,6 +151,11 @@ def verify_law(P: Model, Q: Model, V: int, gamma: int, algo: str):
         if algo == "block":
             p, _, h = block_quantities(P, Q, block)
             tl = tau_law_block(h)
+        elif algo == "greedy":
+            # tau = the last position whose test passes, as in Algorithm 2; the residual of
+            # Eq. "pres_greedy" is Eq. "pres-block" with the unclipped product
+            p, _, _, acc = greedy_quantities(P, Q, block)
+            tl = tau_law_block(acc)
         else:
             h = token_quantities(P, Q, block)
             tl = tau_law_token(h)
@@ -146,6 +184,47 @@ def output_law(P: Model, Q: Model, V: int, gamma: int, algo: str, ell: int):
                 if pz != 0:
                     key = head + z
                     law[key] = law.get(key, 0) + pr * pz
+    return law
+
+
+def modified_model(P: Model, Q: Model, head: Tuple[int, ...], n_mod: int) -> Model:
+    """Algorithm 5 (distribution modification) after Algorithm 4 returned ``head`` = (X^tau, Y):
+    for the next n_mod = gamma - tau - 1 positions the next-token law is proportional to
+    max(M_b(c, head, x^i) - M_s(c, head, x^i), 0) in the JOINT probabilities (Eq. "model_new");
+    after that it is M_b again.  Returns a model over continuations of ``head``."""
+
+    def M(pre: Tuple[int, ...]):
+        if len(pre) >= n_mod:
+            return P(head + pre)
+        seq = head + pre
+        Pn, Qn = P(seq), Q(seq)
+        jp, jq = joint(P, seq), joint(Q, seq)
+        w = [max(jp * a - jq * b, 0) for a, b in zip(Pn, Qn)]
+        tot = sum(w)
+        if tot == 0:  # a prefix the modified model itself cannot produce
+            return [0 for _ in w]
+        return [x / tot for x in w]
+
+    return M
+
+
+def output_law_greedy(P: Model, Q: Model, V: int, gamma: int, ell: int, modify: bool = True):
+    """Law of the first ell <= gamma tokens of (X^tau, Y, Z) for Algorithm 4, where Z follows the
+    modified model of Algorithm 5 (modify=True; Lemma "greedy_block_identical" says the result is
+    M_b^ell) or plain M_b (modify=False; the paper shows this breaks the guarantee)."""
+    law: Dict[Tuple[int, ...], object] = {}
+    for (block, i, y), pr in verify_law(P, Q, V, gamma, "greedy").items():
+        head = block[:i] + (y,)
+        if len(head) >= ell:
+            key = head[:ell]
+            law[key] = law.get(key, 0) + pr
+            continue
+        M = modified_model(P, Q, head, gamma - i - 1) if modify else (lambda pre: P(head + pre))
+        for z in _blocks(V, ell - len(head)):
+            pz = joint(M, z)
+            if pz != 0:
+                key = head + z
+                law[key] = law.get(key, 0) + pr * pz
     return law
 
 

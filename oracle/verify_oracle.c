@@ -8,6 +8,9 @@
  *   - Block Verification  (Algorithm 2, prefix recursion Eq. "def_as",
  *                          residual distribution Eq. "pres-block",
  *                          acceptance weights Eq. "pacc_block")
+ *   - Greedy Block Verification (Algorithm 4, residual Eq. "pres_greedy"): one
+ *                          iteration only; the distribution modification that must
+ *                          follow it (Algorithm 5) needs the models and is not here
  *
  * It follows the algorithms step by step in the paper's order and notation,
  * with no blocking, fusion or reordering.  It shares no code with the CUDA
@@ -38,6 +41,9 @@
  *     k with positive weight;
  *   - a residual whose total mass is exactly 0 (P_tau == Q_tau bit for bit, a
  *     probability-zero event) falls back to sampling P_tau with the same uniform;
+ *   - Algorithm 4: its last test is taken as eta_gamma <= pt_gamma like every other test
+ *     (it is printed with "<"; the two differ on a set of measure zero); a test whose
+ *     denominator sum is 0 passes; a position whose numerator sum is 0 is not selectable;
  *   - NaN / +inf logits in a row that is used, an all -inf row, a drafted token
  *     outside [0, V) or one whose draft logit is -inf are per-sequence domain
  *     errors: out_len = -1 and out_tokens = -1.
@@ -48,7 +54,7 @@
 #include <string.h>
 
 enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F64 = 2 };
-enum { ORACLE_TOKEN_VERIFY = 0, ORACLE_BLOCK_VERIFY = 1 };
+enum { ORACLE_TOKEN_VERIFY = 0, ORACLE_BLOCK_VERIFY = 1, ORACLE_GREEDY_BLOCK_VERIFY = 2 };
 
 /* One logit, widened exactly to double. */
 static double logit_at(const void *base, int dtype, size_t idx)
@@ -380,9 +386,117 @@ done:
     free(lse_t); free(lse_d); free(p); free(S); free(h);
 }
 
+/* ---------------- Algorithm 4: Greedy Block Verification ---------------- */
+/*
+ * Diagnostics: p receives the unclipped products pt_0..pt_gamma, S the numerator sums
+ * sum_x max(pt_i P_i - Q_i, 0) (i = 0..gamma-1), h the ratios h_i as printed (they may
+ * exceed 1, and are +inf when the denominator sum is 0), with h_0 := 1 and h_gamma := pt_gamma.
+ */
+static void greedy_block_verify_one(const seq_t *s, const diag_t *d,
+                                    int32_t *out_tokens, int32_t *out_len)
+{
+    const int g = s->gamma;
+    const size_t V = (size_t)s->V;
+    diag_fill_nan(d, g);
+
+    double *lse_t = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *lse_d = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *pt = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *num = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *h = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    int bad = 0;
+
+    for (int r = 0; r <= g && !bad; ++r) {
+        bad |= row_lse(s->tgt, s->dtype, s->toff + (size_t)r * V, s->V, s->T, &lse_t[r]);
+        if (r < g)
+            bad |= draft_lse(s, r, &lse_d[r]);
+    }
+    if (bad) {
+        emit(s, -1, -1, out_tokens, out_len);
+        goto done;
+    }
+
+    int tau = 0;
+    pt[0] = 1.0;
+    h[0] = 1.0;
+    /* position 0 has no test; its numerator sum is the mass of the residual at tau = 0 */
+    {
+        double acc = 0.0;
+        for (int x = 0; x < s->V; ++x)
+            acc += weight_at(s->tgt, s->toff, lse_t[0], s->drf, s->doff, lse_d[0], 1,
+                             s->dtype, x, s->T, 1.0);
+        num[0] = acc;
+    }
+    for (int i = 1; i <= g - 1; ++i) {
+        /* pt_i = pt_{i-1} * M_b(X_i | c, X^{i-1}) / M_s(X_i | c, X^{i-1}): no minimum */
+        double lr;
+        if (log_ratio(s, i, lse_t[i - 1], lse_d[i - 1], &lr)) {
+            bad = 1;
+            break;
+        }
+        pt[i] = pt[i - 1] * exp(lr);
+        /* h_i = sum_x max{pt_i M_b(x) - M_s(x), 0} / sum_x max{M_s(x) - pt_i M_b(x), 0} */
+        double a = 0.0, c = 0.0;
+        for (int x = 0; x < s->V; ++x) {
+            double P = prob_at(s->tgt, s->dtype, s->toff + (size_t)i * V, x, s->T, lse_t[i]);
+            double Q = prob_at(s->drf, s->dtype, s->doff + (size_t)i * V, x, s->T, lse_d[i]);
+            double w = pt[i] * P - Q;
+            if (w > 0.0)
+                a += w;
+            else
+                c += -w;
+        }
+        num[i] = a;
+        h[i] = c > 0.0 ? a / c : (a > 0.0 ? INFINITY : 0.0);
+        if (a > 0.0 && (double)s->u[i - 1] <= h[i])
+            tau = i;
+    }
+    if (!bad) {
+        double lr;
+        if (log_ratio(s, g, lse_t[g - 1], lse_d[g - 1], &lr))
+            bad = 1;
+        else
+            pt[g] = pt[g - 1] * exp(lr);
+    }
+    if (bad) {
+        emit(s, -1, -1, out_tokens, out_len);
+        goto done;
+    }
+    h[g] = pt[g];
+    if ((double)s->u[g - 1] <= pt[g])
+        tau = g;
+
+    {
+        /* tests at i >= tau decide the outcome; a test passes with probability min(h_i, 1) */
+        double m_eta = INFINITY;
+        for (int i = (tau > 0 ? tau : 1); i <= g; ++i) {
+            double gap = fabs((double)s->u[i - 1] - (h[i] < 1.0 ? h[i] : 1.0));
+            if (gap < m_eta) m_eta = gap;
+        }
+        int have_draft = tau < g;
+        double u = (double)s->u[have_draft ? g : g + 1];
+        double W, m_smp;
+        int Y = sample_index_order(s->tgt, s->toff + (size_t)tau * V, lse_t[tau],
+                                   s->drf, s->doff + (size_t)tau * V, lse_d[tau],
+                                   have_draft, s->dtype, s->V, s->T, pt[tau], u, &W, &m_smp);
+        if (d->margin_eta) *d->margin_eta = m_eta;
+        if (d->margin_smp) *d->margin_smp = m_smp;
+        emit(s, tau, Y, out_tokens, out_len);
+    }
+    for (int i = 0; i <= g; ++i) {
+        if (d->p) d->p[i] = pt[i];
+        if (d->h) d->h[i] = h[i];
+        if (d->lse_t) d->lse_t[i] = lse_t[i];
+        if (i < g && d->S) d->S[i] = num[i];
+        if (i < g && d->lse_d) d->lse_d[i] = lse_d[i];
+    }
+done:
+    free(lse_t); free(lse_d); free(pt); free(num); free(h);
+}
+
 /*
  * Batch entry.  All pointers are host pointers.
- *   algo: 0 = Token Verification, 1 = Block Verification
+ *   algo: 0 = Token Verification, 1 = Block Verification, 2 = Greedy Block Verification
  *   target [B, gamma+1, V], draft [B, gamma, V] in dtype (0 f32, 1 bf16 bits, 2 f64)
  *   tokens [B, gamma] int32, uniforms [B, gamma+2] f32
  *   out_tokens [B, gamma+1], out_len [B]
@@ -404,7 +518,7 @@ static int verify_impl(int algo, const void *target, const void *draft,
         return 1;
     if (B < 0 || gamma < 1 || V < 1 || !(temperature > 0.0) || !isfinite(temperature))
         return 1;
-    if (dtype < 0 || dtype > 2 || (algo != 0 && algo != 1))
+    if (dtype < 0 || dtype > 2 || algo < 0 || algo > 2)
         return 1;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 1)
@@ -429,6 +543,8 @@ static int verify_impl(int algo, const void *target, const void *draft,
         int32_t *ot = out_tokens + (size_t)b * (size_t)(gamma + 1);
         if (algo == ORACLE_BLOCK_VERIFY)
             block_verify_one(&s, &d, ot, out_len + b);
+        else if (algo == ORACLE_GREEDY_BLOCK_VERIFY)
+            greedy_block_verify_one(&s, &d, ot, out_len + b);
         else
             token_verify_one(&s, &d, ot, out_len + b);
     }

@@ -62,14 +62,14 @@ def all_blocks(V, gamma):
 
 def read_golden(path):
     """Parse tests/golden/toy_example.txt into a dict of tokens per key."""
-    out = {"bv": {}}
+    out = {"bv": {}, "gv": {}}
     with open(path) as f:
         for line in f:
             line = line.split("#")[0].split()
             if not line:
                 continue
-            if line[0] == "bv":
-                out["bv"][line[1]] = line[2:]
+            if line[0] in ("bv", "gv"):
+                out[line[0]][line[1]] = line[2:]
             else:
                 out[line[0]] = line[1:]
     return out

@@ -15,6 +15,7 @@ import pytest
 
 import oracle
 import test_oracle_c as pins
+import test_oracle_greedy as gpins
 
 SRC = open(os.path.join(os.path.dirname(oracle.__file__), "verify_oracle.c")).read()
 
@@ -82,6 +83,21 @@ MUTATIONS = [
     ("drafting step samples with the verification's other uniform convention (token after)",
      "1.0, (double)uniforms[r], &W, &m);",
      "1.0, 1.0 - (double)uniforms[r], &W, &m);"),
+    ("greedy block verification clips its running product",
+     "pt[i] = pt[i - 1] * exp(lr);",
+     "pt[i] = pt[i - 1] * exp(lr) < 1.0 ? pt[i - 1] * exp(lr) : 1.0;"),
+    ("greedy block verification: denominator sum gathers the wrong side",
+     "            else\n                c += -w;",
+     "            else\n                c += Q;"),
+    ("greedy block verification: h_i upside down",
+     "h[i] = c > 0.0 ? a / c : (a > 0.0 ? INFINITY : 0.0);",
+     "h[i] = a > 0.0 ? c / a : 0.0;"),
+    ("greedy block verification: last test against the clipped weight of Algorithm 2's form",
+     "    if ((double)s->u[g - 1] <= pt[g])\n        tau = g;",
+     "    if ((double)s->u[g - 1] <= pt[g] / (1.0 + pt[g]))\n        tau = g;"),
+    ("greedy block verification: residual with a product clipped at one",
+     "have_draft, s->dtype, s->V, s->T, pt[tau], u, &W, &m_smp);",
+     "have_draft, s->dtype, s->V, s->T, pt[tau] < 1.0 ? pt[tau] : 1.0, u, &W, &m_smp);"),
     ("token verification without the min with 1",
      "double h = ratio < 1.0 ? ratio : 1.0;       /* h_i^token = min(ratio, 1) */",
      "double h = ratio;"),
@@ -148,6 +164,11 @@ def _pins():
     yield lambda: pins.test_lossless_by_brute_force_over_blocks_and_uniforms(oracle.BLOCK_VERIFY, "block")
     yield lambda: pins.test_supplied_draft_normalisers(oracle.BLOCK_VERIFY)
     yield lambda: pins.test_draft_sampler_frequencies_are_the_softmax()
+    yield lambda: gpins.test_c_oracle_toy_example_through_uniform_grid()
+    yield lambda: gpins.test_c_oracle_intermediates_match_exact(0)
+    yield lambda: gpins.test_c_oracle_intermediates_match_exact(1)
+    yield lambda: gpins.test_c_oracle_law_by_brute_force_over_blocks_and_uniforms()
+    yield lambda: gpins.test_c_oracle_sample_follows_the_residual_with_the_unclipped_product()
 
 
 def _caught():
