@@ -8,7 +8,7 @@ workload is B=256, gamma=8, V=256000, bf16 (2.2 GB of logits, far larger than
 L2, so nothing is served from cache between steps).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload c1|c2|c3|c4] [--algo block|token]
+                    [--workload c1|c2|c3|c4] [--algo block|token|sample|block_lse|greedy]
 
 Prints one JSON line.  With N > 1 (launched by torch.distributed.run) every rank
 verifies its own batch of the same shape (weak scaling, no collective on the
@@ -112,7 +112,8 @@ def time_oracle(w, algo_name: str, budget_s: float = 20.0):
     """The CPU oracle, as it stands, on a bounded sample of the workload."""
     import numpy as np
     import oracle
-    algo = oracle.BLOCK_VERIFY if algo_name in ("block", "block_lse") else oracle.TOKEN_VERIFY
+    algo = {"block": oracle.BLOCK_VERIFY, "block_lse": oracle.BLOCK_VERIFY,
+            "greedy": oracle.GREEDY_BLOCK_VERIFY}.get(algo_name, oracle.TOKEN_VERIFY)
     cores = oracle.threads()
     # one sequence first to size the sample for about budget_s of work
     probe = wl.make_inputs(wl.scaled(w, B=max(1, min(w.B, cores))), "cpu")
@@ -187,9 +188,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(wl.CONFIGS))
-    ap.add_argument("--algo", default="block", choices=["block", "token", "sample", "block_lse"],
-                    help="block / token verification, the drafting step (sampling the draft rows), or block "
-                         "verification with the draft normalisers that the drafting step leaves")
+    ap.add_argument("--algo", default="block", choices=["block", "token", "sample", "block_lse", "greedy"],
+                    help="block / token verification, the drafting step (sampling the draft rows), block "
+                         "verification with the draft normalisers that the drafting step leaves, or one "
+                         "iteration of greedy block verification (Algorithm 4)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
@@ -228,6 +230,9 @@ def main():
         lse = lse.view(w.B, w.gamma).contiguous()
         fn = lambda *_: bv.bv_verify_lse(*a[:4], lse, a[4])
         args.e2e_steps = 0
+    if args.algo == "greedy":
+        fn = bv.gbv_verify
+        args.e2e_steps = 0          # (no host-buffer form of this entry point)
 
     def barrier():
         if dist is not None:
@@ -319,8 +324,8 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
         # what must be read at least: every target row, and one draft row per block for the residual
         algo_bytes = w.B * (w.gamma + 2) * w.V * esz
         kernel = "verify_flow_kernel"
-    elif args.algo == "block":
-        # Algorithm 2 needs every row: B (2 gamma + 1) V elements
+    elif args.algo in ("block", "greedy"):
+        # Algorithms 2 and 4 need every row: B (2 gamma + 1) V elements
         algo_bytes = w.logit_bytes
         kernel = "verify_flow_kernel"
     else:

@@ -186,6 +186,37 @@ int bv_verify_lse_ex(const void* target_logits, const void* draft_logits,
                      float* out_lse_t, float* out_lse_d, void* stream);
 
 /*
+ * Greedy Block Verification, one iteration: Algorithm 4.  The running product is not clipped,
+ *   pt_0 = 1,  pt_i = pt_{i-1} P_{i-1}(X_i) / Q_{i-1}(X_i);
+ * position 0 < i < gamma passes its test when eta_i <= h_i with
+ *   h_i = sum_x max(pt_i P_i(x) - Q_i(x), 0) / sum_x max(Q_i(x) - pt_i P_i(x), 0)
+ * (the second sum equals the first plus 1 - pt_i; a test with an empty first sum never passes),
+ * position gamma when eta_gamma <= pt_gamma (printed with "<"; taken as "<=" like every other
+ * test); tau is the highest position that passes (0 if none) and Y is drawn from Eq. "pres_greedy"
+ * at position tau (Eq. "pres-block" with pt_tau in place of p_tau), or from P_gamma when tau = gamma.
+ * The paper shows that the tokens after (X^tau, Y) must then be drawn from the modified model of
+ * Algorithm 5 to keep the target model's law; that step needs the models and is the caller's.
+ *
+ * Arguments, outputs, errors and uniform usage as bv_verify / bv_verify_ex; DEVICE pointers.
+ * Diagnostics: out_p holds pt_0..pt_gamma, out_S the first sums (i = 0..gamma-1), out_h the ratios
+ * h_i (h_0 := 1, h_gamma := pt_gamma); a ratio above one is only known to be above one (its
+ * denominator is a difference of nearly equal numbers) and is +inf when that denominator is not
+ * positive.  As for bv_verify, the sums are evaluated only for positions that can be selected
+ * (eta_i <= pt_i) unless diagnostics are asked for.  Only the 128-bit path exists (rows of whole
+ * 16-byte vectors on 16-byte aligned bases), else BV_ERR_UNSUPPORTED.
+ */
+int gbv_verify(const void* target_logits, const void* draft_logits,
+               const int32_t* draft_tokens, const float* uniforms,
+               int B, int gamma, int V, int dtype, float temperature,
+               int32_t* out_tokens, int32_t* out_len, void* stream);
+int gbv_verify_ex(const void* target_logits, const void* draft_logits,
+                  const int32_t* draft_tokens, const float* uniforms,
+                  int B, int gamma, int V, int dtype, float temperature,
+                  int32_t* out_tokens, int32_t* out_len,
+                  float* out_p, float* out_S, float* out_h,
+                  float* out_lse_t, float* out_lse_d, void* stream);
+
+/*
  * The drafting step of Algorithm 3 ("Sample X_1, ..., X_gamma ~ M_s using autoregressive sampling,
  * keep the conditional probabilities at each step") for `rows` rows of draft logits [rows, V]:
  *   out_tokens[r] ~ softmax(logits[r, :] / temperature), drawn by inverse CDF in vocabulary-index

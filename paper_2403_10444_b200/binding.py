@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "bv_sample_draft", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_sample_draft", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -48,9 +48,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib = ctypes.CDLL(p)
     vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
     base = [vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp]
-    for name in ("bv_verify", "tv_verify", "bv_verify_noalloc"):
+    for name in ("bv_verify", "tv_verify", "bv_verify_noalloc", "gbv_verify"):
         getattr(lib, name).argtypes = base + [vp]
-    for name in ("bv_verify_ex", "tv_verify_ex"):
+    for name in ("bv_verify_ex", "tv_verify_ex", "gbv_verify_ex"):
         getattr(lib, name).argtypes = base + [vp, vp, vp, vp, vp, vp]
     for name in ("bv_verify_host", "tv_verify_host"):
         getattr(lib, name).argtypes = base
@@ -168,6 +168,22 @@ def tv_verify_ex(target_logits, draft_logits, draft_tokens, uniforms, temperatur
                  stream=None):
     """tv_verify plus its intermediates (NaN where Algorithm 1 forms none)."""
     return _device_call("tv_verify_ex", target_logits, draft_logits, draft_tokens, uniforms,
+                        temperature, True, stream)
+
+
+def gbv_verify(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+               stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Greedy Block Verification, one iteration (Algorithm 4), on CUDA tensors; returns
+    (out_tokens, out_len).  Rows must be whole 16-byte vectors."""
+    return _device_call("gbv_verify", target_logits, draft_logits, draft_tokens, uniforms,
+                        temperature, False, stream)
+
+
+def gbv_verify_ex(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                  stream=None):
+    """gbv_verify plus its intermediates: p holds the unclipped products, S the numerator sums of
+    the acceptance ratios, h the ratios (above one, or +inf, where the test passes with certainty)."""
+    return _device_call("gbv_verify_ex", target_logits, draft_logits, draft_tokens, uniforms,
                         temperature, True, stream)
 
 

@@ -43,6 +43,7 @@ std::mutex g_mu;
 thread_local int t_last_launches = 0;
 thread_local int t_last_cuda_error = 0;
 thread_local const float* t_given_lse_d = nullptr;   // set by bv_verify_lse around its call of run_device
+thread_local int t_greedy = 0;                       // set by gbv_verify around its call of run_device
 
 int cuda_fail(cudaError_t e) {
     t_last_cuda_error = static_cast<int>(e);
@@ -126,6 +127,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     bv::Params prm{};
     prm.tgt = tgt; prm.drf = drf; prm.tok = tok; prm.uni = uni;
     prm.lse_d = t_given_lse_d;
+    prm.greedy = t_greedy;
     prm.B = B; prm.gamma = gamma; prm.V = V;
     const double kd = 1.4426950408889634073599246810019 / static_cast<double>(T);
     prm.kd = kd;
@@ -140,7 +142,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     const char* force = std::getenv("BV_KERNEL");   // "flow", "cluster", "resident", "stream": experiments and tests
     const bool want = force != nullptr;
     auto forced = [&](const char* name) { return want && std::strcmp(force, name) == 0; };
-    if (prm.lse_d != nullptr && !(algo == bv::kBlockVerify && vec && (!want || forced("flow")))) return BV_ERR_UNSUPPORTED;
+    if ((prm.lse_d != nullptr || prm.greedy) && !(algo == bv::kBlockVerify && vec && (!want || forced("flow")))) return BV_ERR_UNSUPPORTED;
 
     // Block Verification on 16-byte rows: the flow of independent work items
     if (algo == bv::kBlockVerify && vec && (!want || forced("flow"))) {
@@ -197,7 +199,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
         }
     }
 
-    if (prm.lse_d != nullptr) return BV_ERR_UNSUPPORTED;   // (the flow kernel could not be launched)
+    if (prm.lse_d != nullptr || prm.greedy) return BV_ERR_UNSUPPORTED;   // (the flow kernel could not be launched)
 
     if (algo == bv::kBlockVerify && vec && forced("resident")) {
         const long long units = static_cast<long long>(row_bytes / 16);
@@ -352,6 +354,25 @@ int bv_verify_lse_ex(const void* tgt, const void* drf, const int32_t* tok, const
     const int rc = run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, out_p, out_S,
                               out_h, out_lse_t, out_lse_d, static_cast<cudaStream_t>(stream));
     t_given_lse_d = nullptr;
+    return rc;
+}
+
+int gbv_verify(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+               int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
+    t_greedy = 1;
+    const int rc = run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, nullptr, nullptr,
+                              nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+    t_greedy = 0;
+    return rc;
+}
+
+int gbv_verify_ex(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+                  int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p, float* out_S,
+                  float* out_h, float* out_lse_t, float* out_lse_d, void* stream) {
+    t_greedy = 1;
+    const int rc = run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, out_p, out_S,
+                              out_h, out_lse_t, out_lse_d, static_cast<cudaStream_t>(stream));
+    t_greedy = 0;
     return rc;
 }
 

@@ -32,6 +32,7 @@ struct Params {
     unsigned int* ticket;     // [2]: next sequence index, clusters that have finished
     int* status;              // set to 1 if a bounded device-side wait gave up
     int nclusters;            // clusters in the grid
+    int greedy;               // flow kernel: Greedy Block Verification (Algorithm 4) instead of Algorithm 2
 };
 
 __device__ __forceinline__ float ex2(float x) {

@@ -158,6 +158,18 @@ __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int 
     return found;
 }
 
+// Acceptance weight of position 0 < i < gamma from p_i and S_i: Eq. "pacc_block",
+// h_i = S_i / (S_i + 1 - p_i), and 0 for an empty residual.  Algorithm 4 prints its h_i as
+// sum_x max(pt_i P_i - Q_i, 0) / sum_x max(Q_i - pt_i P_i, 0); both rows sum to one, so the second
+// sum is the first plus 1 - pt_i and the same expression serves, with the unclipped product pt_i:
+// for pt_i >= 1 the denominator is at most S_i (the test passes whatever the uniform), and a
+// denominator that is not positive gives +inf.
+__device__ __forceinline__ double f_weight(double pi, double Si) {
+    if (!(Si > 0.0)) return 0.0;
+    const double den = Si + 1.0 - pi;
+    return den > 0.0 ? Si / den : INFINITY;
+}
+
 // ---- the end of a block (one thread): Eq. "pacc_block", selection of tau, output ----
 static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl, int b) {
     const int g = prm.gamma;
@@ -175,7 +187,7 @@ static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl
         for (int i = g; i >= 1; --i) {
             const double pi = __ldcg(&p[i]);
             double h = pi;
-            if (i < g) { const double Si = __ldcg(&S[i]); h = Si > 0.0 ? Si / (Si + 1.0 - pi) : 0.0; }
+            if (i < g) h = f_weight(pi, __ldcg(&S[i]));
             if (h > 0.0 && static_cast<double>(u[i - 1]) <= h) { tau = i; break; }
         }
     }
@@ -193,7 +205,7 @@ static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl
             const size_t o1 = static_cast<size_t>(b) * (g + 1) + i, o0 = static_cast<size_t>(b) * g + i;
             const double pi = __ldcg(&p[i]);
             const double Si = i < g ? __ldcg(&S[i]) : 0.0;
-            double h = (i == 0) ? 1.0 : (i == g ? pi : (Si > 0.0 ? Si / (Si + 1.0 - pi) : 0.0));
+            double h = (i == 0) ? 1.0 : (i == g ? pi : f_weight(pi, Si));
             const RowZ z = load_rowz(&fl.rowZ[static_cast<size_t>(b) * (g + 1) + i]);
             if (prm.out_p) prm.out_p[o1] = static_cast<float>(pi);
             if (prm.out_h) prm.out_h[o1] = static_cast<float>(h);
@@ -223,10 +235,7 @@ static __device__ bool f_position_selected(const Params& prm, const FlowScratch&
     if (i == 0) return true;
     const double pi = __ldcg(&fl.pchain[static_cast<size_t>(b) * (g + 2) + i]);
     double h = pi;
-    if (i < g) {
-        const double Si = __ldcg(&fl.S[static_cast<size_t>(b) * (g + 1) + i]);
-        h = Si > 0.0 ? Si / (Si + 1.0 - pi) : 0.0;
-    }
+    if (i < g) h = f_weight(pi, __ldcg(&fl.S[static_cast<size_t>(b) * (g + 1) + i]));
     return h > 0.0 && static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + i - 1]) <= h;
 }
 // A position on hold changes state exactly once, whoever gets there first (positions of one block
@@ -366,7 +375,9 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
         if (c == 0) p[0] = 1.0;
         float cs = 1.f;
         if (c < static_cast<unsigned>(g)) {
-            p[c + 1] = fmin(p_c * __ldcg(&fl.ratio[ci]), 1.0);
+            // Eq. "def_as" clips the running product at one; Algorithm 4 ("Set pt_i") does not
+            const double next = p_c * __ldcg(&fl.ratio[ci]);
+            p[c + 1] = prm.greedy ? next : fmin(next, 1.0);
             cs = static_cast<float>(p_c * __ldcg(&fl.zratio[ci]));
         }
         fl.cscale[ci] = cs;
@@ -376,7 +387,9 @@ __device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const Fl
         // its candidate.  Position gamma is selected iff eta_gamma <= h_gamma = p_gamma, and only then
         // is the sample from P_gamma drawn.  Position 0 is what remains when no other is selected.
         // (The margin keeps a uniform within rounding of p_c on the long path; with diagnostic
-        // outputs every position is computed.)
+        // outputs every position is computed.)  The unclipped product of Algorithm 4 obeys the same
+        // bound while it is at most one; above one the position passes its test whatever the
+        // uniform, and the comparison below makes it a candidate.
         if (c == static_cast<unsigned>(g) && f_draws_in_sweep1(prm, cx.nch)) {
             // the row was swept because position gamma can be selected, and its token was drawn from
             // that very sweep: the position is complete.  It is the highest candidate, so either it

@@ -10,6 +10,8 @@ Tolerances, from the arithmetic of the CUDA path (fp32 per element, fp64 combina
     1e-5 S_i + 1e-7 p_i, because S is then the small difference of sums whose own
     fp32 rounding is 6e-8 p_i; where the oracle has S_i = 0 the CUDA value must be
     <= 1e-7 p_i (and exactly 0 when the two rows are bit-identical);
+  - Greedy Block Verification (Algorithm 4): the same bounds with the unclipped product in place
+    of p_i; where that product is one or more the acceptance ratio is only required to be >= 1;
   - tau and Y: bit-exact, except for trials in which a uniform lies within 1e-6 of
     the threshold it is compared with: a differing tau needs an eta_i within 1e-6 of
     h_i (oracle margin); a differing Y needs the sampling uniform within 1e-6 of the
@@ -48,7 +50,9 @@ def run_cuda(algo: int, inp, diagnostics=True):
     import paper_2403_10444_b200 as bv
     d = to_device(inp)
     fn = {(oracle.BLOCK_VERIFY, True): bv.bv_verify_ex, (oracle.TOKEN_VERIFY, True): bv.tv_verify_ex,
-          (oracle.BLOCK_VERIFY, False): bv.bv_verify, (oracle.TOKEN_VERIFY, False): bv.tv_verify}[(algo, diagnostics)]
+          (oracle.BLOCK_VERIFY, False): bv.bv_verify, (oracle.TOKEN_VERIFY, False): bv.tv_verify,
+          (oracle.GREEDY_BLOCK_VERIFY, True): bv.gbv_verify_ex,
+          (oracle.GREEDY_BLOCK_VERIFY, False): bv.gbv_verify}[(algo, diagnostics)]
     out = fn(d["target_logits"], d["draft_logits"], d["draft_tokens"], d["uniforms"], d["temperature"])
     torch.cuda.synchronize()
     return out
@@ -94,7 +98,7 @@ def token_is_valid(algo, ref, inp_np, b, y) -> bool:
     T = float(np.float32(T))
     P = np.exp(_widen(tgt[b, tau]) / T - ref.lse_t[b, tau])
     if tau < g:
-        p = ref.p[b, tau] if algo == oracle.BLOCK_VERIFY else 1.0
+        p = ref.p[b, tau] if algo != oracle.TOKEN_VERIFY else 1.0   # (the unclipped product for Algorithm 4)
         w = np.maximum(p * P - np.exp(_widen(drf[b, tau]) / T - ref.lse_d[b, tau]), 0.0)
         if not w.sum() > 0:
             w = P
@@ -152,7 +156,7 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
             assert not np.isnan(got[m]).any(), "CUDA path left a log-normaliser unset"
             if m.any():
                 abs_lse = max(abs_lse, float(np.abs(got[m] - want[m]).max()))
-        if algo == oracle.BLOCK_VERIFY:
+        if algo != oracle.TOKEN_VERIFY:
             m = rows[:, None] & ~np.isnan(ref.p)
             rel_p = float((np.abs(p[m] - ref.p[m]) / np.maximum(ref.p[m], 1e-30)).max())
             pS = ref.p[:, :-1]
@@ -162,6 +166,12 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
             for i in range(1, g):
                 Sr, pr, hr = ref.S[:, i], ref.p[:, i], ref.h[:, i]
                 mm = rows & (Sr > 0)
+                if algo == oracle.GREEDY_BLOCK_VERIFY:
+                    # Algorithm 4's ratio with an unclipped product of one or more is at least one:
+                    # the test passes whatever the uniform, and that is all the value says
+                    sure = mm & (pr >= 1.0)
+                    assert np.all(h[sure, i] >= 1.0), "a position with pt_i >= 1 must pass its test"
+                    mm = mm & (pr < 1.0)
                 if mm.any():
                     den = (Sr[mm] + 1.0 - pr[mm]) ** 2
                     tol = 1e-5 * hr[mm] + ((1.0 - pr[mm]) * 1e-7 * pr[mm] + Sr[mm] * 2e-7 * pr[mm]) / den + 1e-7

@@ -21,7 +21,7 @@ def lib():
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "bv.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b((?:bv|tv)_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b((?:bv|tv|gbv)_[a-z_]+)\s*\(", text)))
 
 
 def test_every_declared_symbol_is_exported(lib):
@@ -49,7 +49,7 @@ def test_bad_arguments_are_rejected_without_a_device(lib):
         return getattr(lib, fn)(tgt, drf, tok, uni, a["B"], a["gamma"], a["V"], a["dtype"],
                                 ctypes.c_float(a["T"]), ot, ol, None)
 
-    for fn in ("bv_verify", "tv_verify"):
+    for fn in ("bv_verify", "tv_verify", "gbv_verify"):
         assert call(fn, tgt=None) == -1
         assert call(fn, ol=None) == -1
         assert call(fn, B=-1) == -1
