@@ -23,7 +23,10 @@
  * Eq. "output_block_distribution"), Lemma 3 (Pr(tau >= i | X^i) = p_i), the
  * expected-length ordering of Theorem 2, the gamma = 1 coincidence of the two
  * procedures, scipy's logsumexp for the normalisers, and explicit cumulative
- * sums for the sampler.
+ * sums for the sampler.  Algorithm 4 (tests/test_oracle_greedy.py): the paper's
+ * account of the same example (12/9 accepted tokens, the 1/3 counter-example),
+ * Lemma "block-accept", Theorem "greedy_one_iter" and Lemma
+ * "greedy_block_identical" by enumeration in exact rationals.
  *
  * Notation (0-based storage rows, 1-based tokens):
  *   P_r = softmax(target_logits[b, r, :] / T),  r = 0..gamma    (M_b(. | c, X^r))

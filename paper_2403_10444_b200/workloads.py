@@ -103,3 +103,32 @@ def make_inputs(w: Workload, device="cpu") -> Dict[str, torch.Tensor]:
         uni[b] = torch.rand((g + 2,), generator=gen, device=dev, dtype=torch.float32)
     return dict(target_logits=tgt, draft_logits=drf, draft_tokens=tok, uniforms=uni,
                 temperature=float(w.temperature))
+
+
+def markov_models(V: int, dtype: str, seed: int, target_sigma: float = 2.0, draft_sigma: float = 1.0,
+                  zipf: float = 0.0, device="cpu"):
+    """Synthetic context-dependent models for the decoding loop: next-token logits depend on the last
+    token only.  Returns (target_table, draft_table), each [V, V] in the storage dtype, row t = the
+    logits after token t; the draft rows are the fp32 target rows plus iid Gaussian noise, drawn and
+    rounded like the verification workloads above."""
+    dev = torch.device(device)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    t = torch.randn((V, V), generator=gen, device=dev, dtype=torch.float32) * target_sigma
+    if zipf:
+        perm = torch.rand((V, V), generator=gen, device=dev).argsort(dim=1)
+        t = t - zipf * torch.log(torch.arange(1, V + 1, dtype=torch.float32, device=dev))[perm]
+    d = t + torch.randn((V, V), generator=gen, device=dev, dtype=torch.float32) * draft_sigma
+    td = torch.float32 if dtype == "f32" else torch.bfloat16
+    return t.to(td), d.to(td)
+
+
+def loop_uniforms(iterations: int, B: int, gamma: int, seed: int, device="cpu"):
+    """The uniforms one run of the decoding loop consumes: u_draft [iterations, gamma, B] (one per
+    drafted token) and u_verify [iterations, B, gamma+2] (the verification's), float32 in [0, 1)."""
+    dev = torch.device(device)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    u_draft = torch.rand((iterations, gamma, B), generator=gen, device=dev, dtype=torch.float32)
+    u_verify = torch.rand((iterations, B, gamma + 2), generator=gen, device=dev, dtype=torch.float32)
+    return u_draft, u_verify
