@@ -367,10 +367,10 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
 # ncu capture of this command at full size that profiles/ summarises; None for a workload or
 # kernel with no capture.
 TRAFFIC_BYTES = {
-    ("c4", "block", "verify_flow_kernel"): 2484684032,
-    ("c4", "greedy", "verify_flow_kernel"): 2491745024,
+    ("c4", "block", "verify_flow_kernel"): 2481445632,
+    ("c4", "greedy", "verify_flow_kernel"): 2479917824,
+    ("c4", "block_lse", "verify_flow_kernel"): 1442580480,
     ("c4", "sample", "sample_rows_kernel"): 1054102784,
-    ("c4", "block_lse", "verify_flow_kernel"): 1438274816,
 }
 
 
