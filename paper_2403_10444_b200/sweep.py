@@ -8,7 +8,8 @@ is timed with CUDA events around single calls after three warm-up calls; between
 larger than L2 is overwritten whenever the cell's logits would fit into L2 twice over, so no
 cell is served from cache.  Reported per cell: median milliseconds per call, verifications/s
 (B gamma per call), the bytes of all logits divided by the time as a fraction of the HBM copy
-bandwidth, and the mean number of accepted tokens tau.  Small cells are bound by launch
+bandwidth, the mean number of accepted tokens tau and, for Block Verification, the expectation of tau
+over the uniforms given the drafted blocks (from the acceptance weights the library returns).  Small cells are bound by launch
 latency and by the chain of dependent rows, not by bandwidth.
 """
 from __future__ import annotations
@@ -55,7 +56,19 @@ def time_cell(w: wl.Workload, algo: str, calls: int, flush: torch.Tensor):
         ms.append(e0.elapsed_time(e1))
     med = statistics.median(ms)
     tau = float((out[1].float() - 1).mean().item())
-    return {"B": w.B, "gamma": w.gamma, "sigma": w.draft_sigma, "algo": algo, "ms": med, "ms_min": min(ms),
+    # For Block Verification the acceptance weights h_i that the library returns give the expectation
+    # of tau over the uniforms, Pr(tau = i) = h_i prod_{j > i} (1 - h_j), which is far less noisy than
+    # the single draw above when B is small.
+    exp_tau = None
+    if algo == "block":
+        h = bv.bv_verify_ex(*a)[2]["h"].double().clamp(0.0, 1.0)
+        tail = torch.ones_like(h[:, 0])
+        e = torch.zeros_like(tail)
+        for i in range(w.gamma, 0, -1):
+            e = e + i * h[:, i] * tail
+            tail = tail * (1.0 - h[:, i])
+        exp_tau = float(e.mean().item())
+    return {"B": w.B, "gamma": w.gamma, "sigma": w.draft_sigma, "algo": algo, "ms": med, "ms_min": min(ms), "expected_tau": exp_tau,
             "verifications_per_s": w.B * w.gamma / (med * 1e-3),
             "frac_hbm": w.logit_bytes / (med * 1e-3) / 1e9 / hbm_peak_gbs(), "mean_tau": tau,
             "flushed": need_flush}
@@ -83,11 +96,12 @@ def main():
                     if not args.markdown:
                         print(json.dumps(rows[-1]), flush=True)
     if args.markdown:
-        print("| B | gamma | sigma | algo | ms / call (median) | verifications/s | logits bytes / time, of HBM copy peak | mean tau |")
-        print("|---|---|---|---|---|---|---|---|")
+        print("| B | gamma | sigma | algo | ms / call (median) | verifications/s | logits bytes / time, of HBM copy peak | mean tau | E[tau] given the blocks |")
+        print("|---|---|---|---|---|---|---|---|---|")
         for r in rows:
-            print("| %d | %d | %g | %s | %.4f | %.3g | %.3f | %.2f |" % (
-                r["B"], r["gamma"], r["sigma"], r["algo"], r["ms"], r["verifications_per_s"], r["frac_hbm"], r["mean_tau"]))
+            print("| %d | %d | %g | %s | %.4f | %.3g | %.3f | %.2f | %s |" % (
+                r["B"], r["gamma"], r["sigma"], r["algo"], r["ms"], r["verifications_per_s"], r["frac_hbm"], r["mean_tau"],
+                "%.2f" % r["expected_tau"] if r["expected_tau"] is not None else "-"))
 
 
 if __name__ == "__main__":
