@@ -58,7 +58,7 @@ def block_quantities(P: Model, Q: Model, block: Tuple[int, ...]):
 
 def greedy_quantities(P: Model, Q: Model, block: Tuple[int, ...]):
     """Algorithm 4 for one drafted block: the unclipped products
-    pt_i = pt_{i-1} M_b(X_i|.)/M_s(X_i|.), the two sums of its "Set h_i" line
+    pt_i = pt_{i-1} M_b(X_i|.)/M_s(X_i|.), the two sums of its step "Set h_i"
     (num_i = sum_x max(pt_i M_b - M_s, 0), den_i = sum_x max(M_s - pt_i M_b, 0)) and the
     probabilities min(h_i, 1) with which position i passes its test (h_gamma = pt_gamma;
     0 when num_i = 0, the reading taken for an empty residual).

@@ -5,7 +5,7 @@ behaviour, 12/9 accepted tokens, the 1/3 counter-example), Lemma "block-accept"
 (Pr(X^l = x^l, tau >= l) = min(M_b(x^l), M_s(x^l))), Theorem "greedy_one_iter" (expected length =
 sum of those minima, never below Block Verification's), Lemma "greedy_block_identical" (with the
 distribution modification of Algorithm 5 the output is distributed as the target model), the
-identity between the two sums of the "Set h_i" line, and the gamma = 1 coincidence.
+identity between the two sums of the step "Set h_i", and the gamma = 1 coincidence.
 """
 import itertools
 import os
