@@ -204,6 +204,9 @@ int bv_verify_lse_ex(const void* target_logits, const void* draft_logits,
  * positive.  As for bv_verify, the sums are evaluated only for positions that can be selected
  * (eta_i <= pt_i) unless diagnostics are asked for.  Only the 128-bit path exists (rows of whole
  * 16-byte vectors on 16-byte aligned bases), else BV_ERR_UNSUPPORTED.
+ * The product pt_i is carried in double and handed to the sweeps scaled as a float; a product
+ * beyond about 1e38 is outside the supported range (under the draft model E[pt_i] <= 1, so by
+ * Markov's inequality that has probability below 1e-38).
  */
 int gbv_verify(const void* target_logits, const void* draft_logits,
                const int32_t* draft_tokens, const float* uniforms,
