@@ -153,19 +153,24 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
         }
         if (per_sm > 0) {
             const long long units = static_cast<long long>(row_bytes / 16);
-            // (with supplied draft normalisers a first-sweep item streams one row, not two)
-            int nch = bv::flow_pick_chunks(prm.lse_d ? units / 2 : units, B, gamma, static_cast<long long>(d->sm_count) * per_sm);
+            long long nctas = static_cast<long long>(d->sm_count) * per_sm;
+            if (const char* env = std::getenv("BV_FLOW_CTAS")) {
+                const long long v = std::atoll(env);
+                if (v >= 1 && v < nctas) nctas = v;
+            }
+            int chunks = 0, pieces = 0;
             if (const char* env = std::getenv("BV_FLOW_CHUNKS")) {
                 const int v = std::atoi(env);
-                if (v >= 1 && v <= bv::kFlowMaxChunks) nch = v;
+                if (v >= 1 && v <= bv::kFlowMaxChunks) chunks = v;
             }
-            size_t zero_bytes = 0;
-            int np = bv::flow_pick_pieces(units);
             if (const char* env = std::getenv("BV_FLOW_PIECES")) {
                 const int v = std::atoi(env);
-                if (v >= 1 && v <= bv::kFlowMaxChunks) np = v;
+                if (v >= 1 && v <= 8) pieces = v;
             }
-            const size_t need = bv::flow_scratch_bytes(B, gamma, nch, np, &zero_bytes);
+            // (with supplied draft normalisers a first-sweep item streams one row, not two)
+            const bv::FlowPlan plan = bv::flow_plan(units, B, gamma, nctas, prm.lse_d == nullptr, chunks, pieces);
+            size_t zero_bytes = 0;
+            const size_t need = bv::flow_scratch_bytes(B, gamma, plan, &zero_bytes);
             const int slot = static_cast<int>(d->flow_calls++ % 4);
             if (d->flow_bytes[slot] < need) {
                 if (d->flow_ws[slot]) cudaFree(d->flow_ws[slot]);
@@ -176,19 +181,18 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
                 d->flow_bytes[slot] = need;
             }
             bv::FlowScratch fl;
-            bv::flow_scratch_layout(d->flow_ws[slot], B, gamma, nch, np, &fl);
+            bv::flow_scratch_layout(d->flow_ws[slot], B, gamma, plan, &fl);
             if (const char* env = std::getenv("BV_FLOW_DEPTH")) {
                 const int v = std::atoi(env);
-                if (v >= 2 && v <= 3) fl.depth = v;
+                if (v >= 2 && v <= 6) fl.depth = v;
+            }
+            if (const char* env = std::getenv("BV_FLOW_STRETCH")) {
+                const int v = std::atoi(env);
+                if (v >= 256) fl.stretch = v;
             }
             cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
             if (e != cudaSuccess) return cuda_fail(e);
-            long long items = static_cast<long long>(B) * (gamma + 1) * nch;
-            long long nctas = static_cast<long long>(d->sm_count) * per_sm;
-            if (const char* env = std::getenv("BV_FLOW_CTAS")) {
-                const long long v = std::atoll(env);
-                if (v >= 1 && v < nctas) nctas = v;
-            }
+            long long items = static_cast<long long>(fl.tier_t[fl.ntier]);
             if (nctas > items) nctas = items;
             prm.ticket = nullptr;
             prm.nclusters = 0;

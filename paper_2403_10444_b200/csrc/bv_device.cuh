@@ -171,8 +171,9 @@ __device__ __forceinline__ void mbar_arrive_expect(uint32_t bar, uint32_t bytes)
 }
 // Wait for the phase with the given parity.  Each attempt lets the hardware suspend the
 // thread for up to about 2 us; the number of attempts is bounded (a few seconds in all),
-// after which the wait gives up, records the fact in *status and returns, so that a
-// protocol error cannot hang the GPU.
+// after which the wait gives up, records the fact in *status and returns false, so that a
+// protocol error cannot hang the GPU.  A caller that gets false must not touch what the
+// barrier guards: it leaves its loop and returns.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
     uint32_t ok;
     asm volatile(
@@ -182,13 +183,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uin
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, uint32_t limit = 1u << 20) {
     for (uint32_t spins = 0; !mbar_try_wait(bar, parity, 2000u); ++spins) {
-        if (spins > (1u << 20)) {
+        if (spins > limit) {
             if (status) atomicExch(status, 1);
-            return;
+            return false;
         }
     }
+    return true;
 }
 // The same wait without a suspend-time hint: the thread polls and resumes as soon as the phase
 // completes (a hinted wait was seen to resume late).  Bounded like mbar_wait.
@@ -201,13 +203,26 @@ __device__ __forceinline__ bool mbar_try_wait_now(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ void mbar_wait_now(uint32_t bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait_now(uint32_t bar, uint32_t parity, int* status, uint32_t limit = 1u << 24) {
     for (uint32_t spins = 0; !mbar_try_wait_now(bar, parity); ++spins) {
-        if (spins > (1u << 24)) {
+        if (spins > limit) {
             if (status) atomicExch(status, 1);
-            return;
+            return false;
         }
     }
+    return true;
+}
+// The wait of a warp that has nothing else to do and whose wake-up may be a little late: between
+// polls it sleeps, so that it takes no issue slots from the warps that stream.  Bounded like the others.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, int* status, uint32_t ns, uint32_t limit = 1u << 22) {
+    for (uint32_t spins = 0; !mbar_try_wait_now(bar, parity); ++spins) {
+        if (spins > limit) {
+            if (status) atomicExch(status, 1);
+            return false;
+        }
+        __nanosleep(ns);
+    }
+    return true;
 }
 // 16 or 4 bytes into another CTA's shared memory; the bytes are counted by that CTA's barrier
 __device__ __forceinline__ void send_v4(uint32_t raddr, uint32_t rbar, float a, float b, float c, float d) {

@@ -29,31 +29,51 @@
 
 namespace bv {
 
-constexpr int kFThreads = 512;
+constexpr int kFThreads = 448;
 constexpr int kFWarps = kFThreads / 32;
 
-// vectors [w0, w1) of a row that worker `warp` takes of part `ch` out of `nparts`
+// vectors [u0, u1) of `units` that part `ch` out of `nparts` covers
+__device__ __forceinline__ void item_range(int units, int nparts, int ch, int& u0, int& u1) {
+    u0 = static_cast<int>(static_cast<long long>(units) * ch / nparts);
+    u1 = static_cast<int>(static_cast<long long>(units) * (ch + 1) / nparts);
+}
+// Vectors [w0, w1) of the part [u0, u1) that worker `warp` takes (a part is far below 2^27 vectors).
+// The shares are cut to the vector, not to whole ring steps of 32 vectors: with every warp's stream
+// aligned to 512 bytes the kernel was measured 9 % slower (the streams of a CTA then advance through
+// the same memory channels together), which costs more than the short last step of each share.
+__device__ __forceinline__ void warp_range(int u0, int u1, int warp, int& w0, int& w1) {
+    const unsigned n = static_cast<unsigned>(u1 - u0);
+    w0 = u0 + static_cast<int>(n * static_cast<unsigned>(warp) / kFWarps);
+    w1 = u0 + static_cast<int>(n * static_cast<unsigned>(warp + 1) / kFWarps);
+}
 __device__ __forceinline__ void chunk_range(const FlowCtx& cx, int nparts, int ch, int warp, int& w0, int& w1) {
-    const int u0 = static_cast<int>(static_cast<long long>(cx.units) * ch / nparts);
-    const int u1 = static_cast<int>(static_cast<long long>(cx.units) * (ch + 1) / nparts);
-    w0 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * warp / kFWarps);
-    w1 = u0 + static_cast<int>(static_cast<long long>(u1 - u0) * (warp + 1) / kFWarps);
+    int u0, u1;
+    item_range(cx.units, nparts, ch, u0, u1);
+    warp_range(u0, u1, warp, w0, w1);
 }
 
 
-// ring slots per worker thread: three (P, Q) steps of lookahead.  Measured at B = 256, gamma = 8,
-// V = 256000 bf16: 4 slots 0.485 ms, 6 slots 0.471 ms, 8 slots 0.482 ms, 12 slots 0.505 ms; with 32
-// streaming warps per SM the latency is hidden by the other warps, and more bytes in flight only
-// crowd the memory system.
-constexpr int kFDepth = 6;
-constexpr int kFAhead = kFDepth / 2;
-constexpr int kFDesc = 3;      // items in flight per CTA: one being swept, two queued behind it
-constexpr int kFAllThreads = kFThreads + 32;   // 16 worker warps + 1 service warp
+// Ring of a worker thread: kFSlots steps of lookahead, each of two 16-byte cells (A, B).  A step of
+// an item with a draft row holds one vector of P and the same vector of Q; without a draft row it
+// holds two consecutive vectors of P.  The ring is not drained between items: while a warp works
+// through the last steps of one item the loads of the next one are already in flight.
+constexpr int kFSlots = 3;
+constexpr int kFDepth = 2 * kFSlots;
+constexpr int kFDesc = 8;      // descriptors a CTA can hold: being swept, queued behind, or waiting for their post warp
+constexpr int kFPost = 3;      // post warps: what follows the sweep of item n is done by post warp n mod kFPost
+constexpr int kFAllThreads = kFThreads + 32 * (1 + kFPost);   // worker warps + the publisher + the post warps
 
-// One work item as the service warp hands it to the workers.
+// A first-sweep chunk is handed to the workers in stretches (same row, consecutive vectors): the
+// workers carry their sums from stretch to stretch and leave them after the last one, nothing is
+// asked of global memory in between, and a piece of a second sweep, for which a block is waiting,
+// can be slipped in after any stretch.
+enum : int { kPartFirst = 1, kPartLast = 2 };
+// One work item as the publisher hands it to the workers.
 struct FlowDesc {
     int kind;                   // kExit, kSweep1, kSweep2
     int ri, ch;                 // row index b (gamma+1) + r, chunk
+    int u0, u1;                 // vectors [u0, u1) of the row: the chunk, or one stretch of it
+    int part;                   // kPartFirst: the chunk starts here; kPartLast: it ends here
     int have_q;
     const char* rowP;
     const char* rowQ;
@@ -67,6 +87,13 @@ struct FlowShared {
     unsigned long long done[kFDesc];    // all 16 worker warps have left their partials of desc[i]
     float part_M[kFDesc][2][kFWarps];   // sweep 1: references of P and Q per worker warp
     float part_s[kFDesc][2][kFWarps];   // sweep 1: sums; sweep 2: [0] holds the residual totals
+    // a finished item is moved here by its post warp, so that its descriptor slot is free again
+    // before anything is asked of global memory
+    unsigned long long freeb[kFDesc];   // the post warp has moved the item of desc[i] out
+    FlowDesc sdesc[kFPost];
+    float stage_M[kFPost][2][kFWarps];
+    float stage_s[kFPost][2][kFWarps];
+    unsigned posted;                    // items whose post-processing is complete
 };
 
 // ---- service warp: Y ~ P_gamma from the first sweep of the last target row ----
@@ -76,7 +103,7 @@ struct FlowShared {
 template <int DT>
 __device__ void f_draw_from_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, int lane) {
     const int g = cx.g, b = ri / (g + 1);
-    const int nseg = cx.nch * kFWarps;                       // <= 128: four per lane
+    const int nseg = fl.nch_late * kFWarps;                  // <= 128: four per lane
     const float* pairs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
     float m[4], w[4];
 #pragma unroll
@@ -120,7 +147,7 @@ __device__ void f_draw_from_sweep1(const Params& prm, const FlowScratch& fl, con
         const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
         const float before = __shfl_sync(0xffffffffu, bef, src);
         int s0, s1;
-        chunk_range(cx, cx.nch, sel / kFWarps, sel % kFWarps, s0, s1);
+        chunk_range(cx, fl.nch_late, sel / kFWarps, sel % kFWarps, s0, s1);
         const char* rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
         found = f_rescan<DT>(rowP, nullptr, s0, s1, lane, cx.kf, 1.f, -Mrow, 0.f, t - before);
     }
@@ -131,141 +158,114 @@ __device__ void f_draw_from_sweep1(const Params& prm, const FlowScratch& fl, con
     __syncwarp();
 }
 
-// ---- service warp: what follows the sweep of one item ----
+// ---- service warp: what follows the sweep of an item, in three steps, so that several finished
+// items can share one fence and have their counters bumped side by side:
+//   store     the item's result goes to scratch;
+//   (one __threadfence for all of them, then one atomic per item, each by a lane of its own)
+//   complete  for the item that was the last of its row or position. ----
 template <int DT>
-__device__ void f_after_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int slot,
+__device__ void f_store_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int j,
                                int ri, int ch, int lane) {
-    // combine the 16 worker warps of this chunk in fp64
-    const float mP = lane < kFWarps ? sh.part_M[slot][0][lane] : kNoRef;
-    const float mQ = lane < kFWarps ? sh.part_M[slot][1][lane] : kNoRef;
+    // combine the worker warps of this chunk in fp64
+    const float mP = lane < kFWarps ? sh.stage_M[j][0][lane] : kNoRef;
+    const float mQ = lane < kFWarps ? sh.stage_M[j][1][lane] : kNoRef;
     const float MPc = warp_max(mP), MQc = warp_max(mQ);
-    double zP = lane < kFWarps ? static_cast<double>(sh.part_s[slot][0][lane]) * ref_scale(mP, MPc) : 0.0;
-    double zQ = lane < kFWarps ? static_cast<double>(sh.part_s[slot][1][lane]) * ref_scale(mQ, MQc) : 0.0;
+    double zP = lane < kFWarps ? static_cast<double>(sh.stage_s[j][0][lane]) * ref_scale(mP, MPc) : 0.0;
+    double zQ = lane < kFWarps ? static_cast<double>(sh.stage_s[j][1][lane]) * ref_scale(mQ, MQc) : 0.0;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) { zP += shfl_xor_d(zP, off); zQ += shfl_xor_d(zQ, off); }
     // A last target row is swept for one purpose only: the sample from P_gamma.  Its warps' pairs
-    // {reference, sum} are kept, so that the token can be drawn from this one sweep (below).
-    const bool draw = ri % (cx.g + 1) == cx.g && f_draws_in_sweep1(prm, cx.nch);
-    if (draw) {
+    // {reference, sum} are kept, so that the token can be drawn from this one sweep.
+    if (ri % (cx.g + 1) == cx.g && f_draws_in_sweep1(prm, fl.nch_late)) {
         float* pairs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs + static_cast<size_t>(ch) * kFWarps * 2;
-        if (lane < kFWarps) { pairs[2 * lane] = mP; pairs[2 * lane + 1] = sh.part_s[slot][0][lane]; }
-        __threadfence();
-        __syncwarp();
+        if (lane < kFWarps) { pairs[2 * lane] = mP; pairs[2 * lane + 1] = sh.stage_s[j][0][lane]; }
     }
-    int last = 0;
     if (lane == 0) {
         RowZ z; z.MP = MPc; z.ZP = zP; z.MQ = MQc; z.ZQ = zQ;
         fl.part[static_cast<size_t>(ri) * cx.nch + ch] = z;
-        __threadfence();
-        last = atomicAdd(&fl.row_cnt[ri], 1u) == static_cast<unsigned>(cx.nch) - 1u;
     }
-    last = __shfl_sync(0xffffffffu, last, 0);
-    if (!last) return;
+}
+template <int DT>
+__device__ void f_complete_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, int lane) {
     __threadfence();
-    if (draw) f_draw_from_sweep1<DT>(prm, fl, cx, ri, lane);
-    if (lane == 0) f_row_complete<DT>(prm, fl, cx, ri / (cx.g + 1), ri % (cx.g + 1));
-    __syncwarp();
+    const int g = cx.g, b = ri / (g + 1), r = ri % (g + 1);
+    f_row_complete<DT>(prm, fl, cx, b, r, lane);
+    if (r < g) {
+        // the warp that publishes the last of a block's rows 0 .. gamma-1 folds the block
+        unsigned n = 0;
+        if (lane == 0) n = atomicAdd(&fl.rows_in[b], 1u);
+        n = __shfl_sync(0xffffffffu, n, 0);
+        if (n == static_cast<unsigned>(g) - 1u) f_fold_block<DT>(prm, fl, cx, b, lane);
+    } else if (f_draws_in_sweep1(prm, fl.nch_late)) {
+        // The last target row was swept because position gamma can be selected, and its token is
+        // drawn from that very sweep: the position is complete.  It is the highest candidate, so
+        // either it is the selected one (lower candidates are dropped) or the next lower one is started.
+        f_draw_from_sweep1<DT>(prm, fl, cx, ri, lane);
+        if (lane == 0) {
+            atomicExch(&fl.rel[ri], kRelSkip);
+            const unsigned done = f_after_position(prm, fl, b, g);
+            if (atomicAdd(&fl.cand_cnt[b], done) + done == static_cast<unsigned>(g) + 1u) {
+                __threadfence();
+                f_finalize_block(prm, fl, b);
+            }
+        }
+        __syncwarp();
+    } else {
+        // with diagnostics the sample from P_gamma comes from a second sweep of the row, like any other
+        if (lane == 0) f_start_second_sweep(fl, static_cast<size_t>(ri));
+        __syncwarp();
+    }
 }
 
-template <int DT>
-__device__ void f_after_sweep2(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int slot,
-                               const FlowDesc& d, int lane) {
-    const int ri = d.ri;
-    const int np = fl.np;
-    const int nseg = np * kFWarps;
+__device__ __forceinline__ void f_store_sweep2(const FlowScratch& fl, FlowShared& sh, int j, int ri, int ch, int lane) {
     float* segs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
-    if (lane < kFWarps) segs[d.ch * kFWarps + lane] = sh.part_s[slot][0][lane];
-    __threadfence();
-    __syncwarp();
-    int last = 0;
-    if (lane == 0) last = atomicAdd(&fl.s2_cnt[ri], 1u) == static_cast<unsigned>(np) - 1u;
-    last = __shfl_sync(0xffffffffu, last, 0);
-    if (!last) return;
-
-    f_position_complete<DT>(prm, fl, cx, ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, nseg, segs, lane,
+    if (lane < kFWarps) segs[ch * kFWarps + lane] = sh.stage_s[j][0][lane];
+}
+template <int DT>
+__device__ void f_complete_sweep2(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, const FlowDesc& d, int lane) {
+    const int np = fl.np;
+    const float* segs = fl.seg_tot + static_cast<size_t>(d.ri) * fl.segs;
+    f_position_complete<DT>(prm, fl, cx, d.ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, np * kFWarps, segs, lane,
                             [&](int sel, int& s0, int& s1) { chunk_range(cx, np, sel / kFWarps, sel % kFWarps, s0, s1); });
 }
 
-// ---- worker warps: one warp's segment of one item ----
-// The segment's vectors go through the thread's private ring, kFAhead steps ahead of the
-// arithmetic.  A step is one vector per lane of each row; the last step may be partial, and
-// lanes past the end then find -inf logits in their slots.
-template <int DT, bool HAVEQ, int KIND>
-__device__ __forceinline__ void f_sweep_segment(uint32_t sb, const char* rowP, const char* rowQ, int w0, int w1,
-                                                int lane, float kf, float cp, float nMP, float nMQ,
-                                                float& oMP, float& osP, float& oMQ, float& osQ) {
-    using R = Raw<DT>;
-    constexpr int EPV = R::EPV;
-    constexpr uint32_t kSlot = kFThreads * 16;               // bytes between consecutive ring cells
-    // a step takes two of the thread's ring cells, or one when there is no draft row: then the
-    // loads run twice as many steps ahead, so that as many bytes are in flight
-    constexpr int kA = HAVEQ ? kFAhead : kFDepth;
-    constexpr int kC = HAVEQ ? 2 : 1;
-    const int nv = w1 - w0;
-    const int nsteps = (nv + 31) >> 5;
-    const int nlast = nv - 32 * (nsteps - 1);                // lanes that take part in the last step
-    const char* gP = rowP + static_cast<size_t>(w0 + lane) * 16;
-    const char* gQ = HAVEQ ? rowQ + static_cast<size_t>(w0 + lane) * 16 : gP;
-    // sweep 1 asks L2 to keep the rows (they are read again soon); sweep 2 marks them as done with
-    // no row is needed again soon (the few second sweeps come long after the first): stream past L2
-    const uint64_t pol = l2_policy_evict_first();
-    auto fetch_step = [&](int k, int j) {                    // step k goes to cells kC j (, + 1), j = k mod kA
-        if (k < nsteps) {
-            const bool ok = (k + 1 < nsteps) || lane < nlast;
-            ring_fetch_hint(sb + (kC * j) * kSlot, gP + static_cast<size_t>(k) * 512, ok, R::kNegInf, pol);
-            if (HAVEQ) ring_fetch_hint(sb + (kC * j + 1) * kSlot, gQ + static_cast<size_t>(k) * 512, ok, R::kNegInf, pol);
+// ---- worker warps: the arithmetic of one ring step ----
+// First sweep, one vector of each row: running sums of 2^{z k - M} against the warp's integer
+// references, which are raised when a vector's terms show a logit above them.
+template <int EPV>
+__device__ __forceinline__ void f_step_sweep1_pair(const float (&vp)[EPV], const float (&vq)[EPV], float kf,
+                                                   float& MPw, float& sP, float& MQw, float& sQ) {
+    float vsP = f_exp_sum<EPV>(vp, kf, -MPw);
+    float vsQ = f_exp_sum<EPV>(vq, kf, -MQw);
+    if (__any_sync(0xffffffffu, fmaxf(vsP, vsQ) > kRaiseBound)) {   // a logit above a reference
+        if (__any_sync(0xffffffffu, vsP > kRaiseBound)) {
+            const float y = rintf(warp_max(vec_max<EPV>(vp)) * kf);
+            if (y > MPw) { sP *= ref_scale(MPw, y); MPw = y; }
+            vsP = f_exp_sum<EPV>(vp, kf, -MPw);
         }
-        cp_async_commit();
-    };
-#pragma unroll
-    for (int j = 0; j < kA; ++j) fetch_step(j, j);
-
-    float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f, acc = 0.f;
-    for (int kb = 0; kb < nsteps; kb += kA) {
-#pragma unroll
-        for (int j = 0; j < kA; ++j) {
-            const int k = kb + j;
-            if (k < nsteps) {
-                cp_async_wait<kA - 1>();                     // step k has landed
-                float vp[EPV], vq[EPV];
-                R::unpack(lds128(sb + (kC * j) * kSlot), vp);
-                if (HAVEQ) R::unpack(lds128(sb + (kC * j + 1) * kSlot), vq);
-                if (KIND == kSweep1) {
-                    if (j == 0 && kb == 0) {                 // references from the first vector of every lane
-                        MPw = fmaxf(rintf(warp_max(vec_max<EPV>(vp)) * kf), kNoRef);
-                        if (HAVEQ) MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vq)) * kf), kNoRef);
-                    }
-                    float vsP = f_exp_sum<EPV>(vp, kf, -MPw);
-                    float vsQ = HAVEQ ? f_exp_sum<EPV>(vq, kf, -MQw) : 0.f;
-                    if (__any_sync(0xffffffffu, fmaxf(vsP, vsQ) > kRaiseBound)) {   // a logit above a reference
-                        if (__any_sync(0xffffffffu, vsP > kRaiseBound)) {
-                            const float y = rintf(warp_max(vec_max<EPV>(vp)) * kf);
-                            if (y > MPw) { sP *= ref_scale(MPw, y); MPw = y; }
-                            vsP = f_exp_sum<EPV>(vp, kf, -MPw);
-                        }
-                        if (HAVEQ && __any_sync(0xffffffffu, vsQ > kRaiseBound)) {
-                            const float y = rintf(warp_max(vec_max<EPV>(vq)) * kf);
-                            if (y > MQw) { sQ *= ref_scale(MQw, y); MQw = y; }
-                            vsQ = f_exp_sum<EPV>(vq, kf, -MQw);
-                        }
-                    }
-                    sP += vsP;
-                    sQ += vsQ;
-                } else {
-                    float t[EPV];
-                    acc += f_pair_sum<EPV, HAVEQ>(vp, vq, kf, cp, nMP, nMQ, t);
-                }
-                fetch_step(k + kA, j);
-            }
+        if (__any_sync(0xffffffffu, vsQ > kRaiseBound)) {
+            const float y = rintf(warp_max(vec_max<EPV>(vq)) * kf);
+            if (y > MQw) { sQ *= ref_scale(MQw, y); MQw = y; }
+            vsQ = f_exp_sum<EPV>(vq, kf, -MQw);
         }
     }
-    cp_async_wait<0>();
-    if (KIND == kSweep1) {
-        oMP = MPw; osP = warp_sum(sP);
-        oMQ = MQw; osQ = HAVEQ ? warp_sum(sQ) : 0.f;
-    } else {
-        osP = warp_sum(acc);
+    sP += vsP;
+    sQ += vsQ;
+}
+// First sweep, two consecutive vectors of one row.
+template <int EPV>
+__device__ __forceinline__ void f_step_sweep1_single(const float (&va)[EPV], const float (&vb)[EPV], float kf,
+                                                     float& MPw, float& sP) {
+    float vsA = f_exp_sum<EPV>(va, kf, -MPw);
+    float vsB = f_exp_sum<EPV>(vb, kf, -MPw);
+    if (__any_sync(0xffffffffu, fmaxf(vsA, vsB) > kRaiseBound)) {
+        const float y = rintf(warp_max(fmaxf(vec_max<EPV>(va), vec_max<EPV>(vb))) * kf);
+        if (y > MPw) { sP *= ref_scale(MPw, y); MPw = y; }
+        vsA = f_exp_sum<EPV>(va, kf, -MPw);
+        vsB = f_exp_sum<EPV>(vb, kf, -MPw);
     }
+    sP += vsA;
+    sP += vsB;
 }
 
 template <int DT>
@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ FlowShared sh;
     // Each worker thread streams its own vectors through a private ring of 16-byte cells filled
-    // by cp.async, so loads run kFAhead steps ahead of the arithmetic without costing registers.
+    // by cp.async, so loads run kFSlots steps ahead of the arithmetic without costing registers.
     extern __shared__ __align__(16) unsigned char dyn[];
 
     FlowCtx cx;
@@ -287,30 +287,98 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
 
     if (tid == 0) {
         for (int i = 0; i < kFDesc; ++i) {
+            sh.desc[i].kind = kExit;      // what a wait that gives up would find
             mbar_init(smem_u32(&sh.full[i]), 1);
             mbar_init(smem_u32(&sh.done[i]), kFWarps);
+            mbar_init(smem_u32(&sh.freeb[i]), 1);
         }
+        sh.posted = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
+    if (warp > kFWarps) {
+        // =============================== post warps ===============================
+        // What follows the sweep of item n is done by post warp n mod kFPost: the item's partials and
+        // descriptor are moved to the warp's staging area (the slot is free again), the result goes
+        // to scratch, and the row's or position's counter tells whether this item was its last one.
+        // Every step here is a round trip to global memory of a few microseconds on a busy GPU; three
+        // warps working on different items keep up with items of a few microseconds each.
+        const int k = warp - kFWarps - 1;
+        for (int n = k;; n += kFPost) {
+            const int slot = n % kFDesc;
+            const uint32_t par = static_cast<uint32_t>(n / kFDesc) & 1u;
+            if (!mbar_wait_relaxed(smem_u32(&sh.full[slot]), par, prm.status, 200)) break;
+            if (sh.desc[slot].kind == kExit) break;
+            if (!mbar_wait_relaxed(smem_u32(&sh.done[slot]), par, prm.status, 200)) break;
+            if (!(sh.desc[slot].part & kPartLast)) {         // a stretch inside a chunk: the workers carry on
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(smem_u32(&sh.freeb[slot])); atomicAdd(&sh.posted, 1u); }
+                continue;
+            }
+            if (lane == 0) sh.sdesc[k] = sh.desc[slot];
+            if (lane < kFWarps) {
+                sh.stage_M[k][0][lane] = sh.part_M[slot][0][lane]; sh.stage_M[k][1][lane] = sh.part_M[slot][1][lane];
+                sh.stage_s[k][0][lane] = sh.part_s[slot][0][lane]; sh.stage_s[k][1][lane] = sh.part_s[slot][1][lane];
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh.freeb[slot]));
+            const FlowDesc d = sh.sdesc[k];
+            if (d.kind == kSweep1) f_store_sweep1<DT>(prm, fl, cx, sh, k, d.ri, d.ch, lane);
+            else f_store_sweep2(fl, sh, k, d.ri, d.ch, lane);
+            __threadfence();
+            __syncwarp();
+            int last = 0;
+            if (lane == 0) {
+                if (d.kind == kSweep1) last = atomicAdd(&fl.row_cnt[d.ri], 1u) == static_cast<unsigned>(f_nch_row(fl, d.ri / (g + 1), d.ri % (g + 1), g)) - 1u;
+                else last = atomicAdd(&fl.s2_cnt[d.ri], 1u) == static_cast<unsigned>(fl.np) - 1u;
+            }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last) {
+                if (d.kind == kSweep1) f_complete_sweep1<DT>(prm, fl, cx, d.ri, lane);
+                else f_complete_sweep2<DT>(prm, fl, cx, d, lane);
+            }
+            __syncwarp();
+            if (lane == 0) atomicAdd(&sh.posted, 1u);
+        }
+        return;
+    }
     if (warp == kFWarps) {
-        // =============================== service warp ===============================
-        // takes tickets, waits for what a sweep-2 item needs, hands descriptors to the workers,
-        // and does everything that follows a sweep, so that the workers never stop streaming
+        // =============================== publisher ===============================
+        // takes tickets, waits for what a sweep-2 item needs and hands descriptors to the workers.
+        // What it asks of global memory is arranged so that the round trips overlap: the four queue
+        // counters are read after every descriptor for the next one, and tickets of first-sweep items
+        // are drawn ahead of their use.
         // tickets cover the rows that every block needs: target and draft rows 0 .. gamma-1
-        const unsigned total_s1 = static_cast<unsigned>(cx.B) * g * cx.nch;
-        // the next sweep-1 item, or kExit when all have been handed out; never blocks
-        auto take = [&](FlowDesc& d) {
-            unsigned t = 0;
-            if (lane == 0) t = atomicAdd(&fl.counters[kCtrTicket], 1u);
-            t = __shfl_sync(0xffffffffu, t, 0);
-            if (t >= total_s1) { d.kind = kExit; return; }
-            const int ch = static_cast<int>(t % cx.nch);
-            const int r = static_cast<int>(t / cx.nch) % g, b = static_cast<int>(t / cx.nch) / g;
+        const unsigned total_s1 = fl.tier_t[fl.ntier];
+        // Tickets are drawn several at a time (one atomic) and ahead of their use, so that the round
+        // trip is over by the time a descriptor slot is free.
+        unsigned tk_raw = 0, tk_lo = 0;   // (lane 0) answer of the last draw; next ticket on hand (all lanes)
+        int tk_cnt = 0;                   // tickets on hand
+        bool tk_pending = false;          // tk_raw has not been looked at yet
+        auto draw_tickets = [&](int k) {
+            if (lane == 0) tk_raw = atomicAdd(&fl.counters[kCtrTicket], static_cast<unsigned>(k));
+            tk_cnt = k;
+            tk_pending = true;
+        };
+        auto next_ticket = [&]() -> unsigned {
+            if (tk_pending) { tk_lo = __shfl_sync(0xffffffffu, tk_raw, 0); tk_pending = false; }
+            --tk_cnt;
+            return tk_lo++;
+        };
+        // the first-sweep item of ticket t
+        auto sweep1_desc = [&](unsigned t, FlowDesc& d) {
+            int k = 0;
+#pragma unroll
+            for (int j = 1; j < kFlowTiers; ++j) if (j < fl.ntier && t >= fl.tier_t[j]) k = j;
+            const unsigned local = t - fl.tier_t[k];
+            const int nch = fl.tier_n[k];
+            const int ch = static_cast<int>(local % nch);
+            const int r = static_cast<int>(local / nch) % g, b = fl.tier_b[k] + static_cast<int>(local / nch) / g;
             const int ri = b * (g + 1) + r;
             // (with supplied draft normalisers the first sweep has nothing to learn from the draft row)
-            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = prm.lse_d == nullptr;
+            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = prm.lse_d == nullptr; d.part = kPartFirst | kPartLast;
+            item_range(cx.units, nch, ch, d.u0, d.u1);
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
             d.rowQ = d.have_q ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
                               : nullptr;
@@ -319,28 +387,35 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         // Rows whose second sweep has been started stand in a queue, each cut into np pieces.  A
         // piece is claimed by a ticket from the queue's head counter, drawn only while the head is
         // seen behind the tail; a ticket that still runs ahead of the tail (several CTAs drew at
-        // once) is kept until its row arrives.  -1: no piece right now.
+        // once, or the counters were read a while ago) is kept until its row arrives.  -1: no piece
+        // right now.  Last target rows whose first sweep has been asked for stand in a queue of their
+        // own, cut into chunks.
+        unsigned seen_rows = 0, seen_pieces = 0, seen_late = 0, seen_chunks = 0;   // (lane 0) the counters as last read
+        auto poll = [&]() {
+            if (lane == 0) {
+                seen_rows = ld_volatile(&fl.counters[kCtrQueued]);
+                seen_pieces = ld_volatile(&fl.counters[kCtrPieces]);
+                seen_late = ld_volatile(&fl.counters[kCtrLateQueued]);
+                seen_chunks = ld_volatile(&fl.counters[kCtrLateChunks]);
+            }
+        };
         int held = -1, held_late = -1;    // (lane 0) tickets drawn and not yet used
-        auto claim = [&](int queued, int taken, int per_row, int& hold) -> int {
+        auto claim = [&](unsigned rows, unsigned taken_seen, int taken, int per_row, int& hold) -> int {
             int t = -1;
             if (lane == 0) {
-                const unsigned avail = ld_volatile(&fl.counters[queued]) * static_cast<unsigned>(per_row);
-                if (hold < 0 && ld_volatile(&fl.counters[taken]) < avail)
-                    hold = static_cast<int>(atomicAdd(&fl.counters[taken], 1u));
+                const unsigned avail = rows * static_cast<unsigned>(per_row);
+                if (hold < 0 && taken_seen < avail) hold = static_cast<int>(atomicAdd(&fl.counters[taken], 1u));
                 if (hold >= 0 && static_cast<unsigned>(hold) < avail) { t = hold; hold = -1; }
             }
             return __shfl_sync(0xffffffffu, t, 0);
         };
-        auto take_piece = [&]() -> int { return claim(kCtrQueued, kCtrPieces, fl.np, held); };
-        // likewise the chunks of last target rows whose first sweep has been asked for
-        auto late_desc = [&](FlowDesc& d) -> bool {
-            const int t = claim(kCtrLateQueued, kCtrLateChunks, cx.nch, held_late);
-            if (t < 0) return false;
+        auto late_desc = [&](int t, FlowDesc& d) -> bool {
             unsigned e = 0;
-            for (unsigned spins = 0; (e = ld_volatile(&fl.lq[t / cx.nch])) == 0u; ++spins)
+            for (unsigned spins = 0; (e = ld_volatile(&fl.lq[t / fl.nch_late])) == 0u; ++spins)
                 if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
             const int ri = static_cast<int>(e - 1u);
-            d.kind = kSweep1; d.ri = ri; d.ch = t % cx.nch; d.have_q = 0;
+            d.kind = kSweep1; d.ri = ri; d.ch = t % fl.nch_late; d.have_q = 0; d.part = kPartFirst | kPartLast;
+            item_range(cx.units, fl.nch_late, d.ch, d.u0, d.u1);
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
             d.rowQ = nullptr;
             d.cp = 1.f; d.nMP = 0.f; d.nMQ = 0.f;
@@ -352,7 +427,8 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
             const int ri = static_cast<int>(e - 1u);
             const int r = ri % (g + 1), b = ri / (g + 1);
-            d.kind = kSweep2; d.ri = ri; d.ch = t % fl.np; d.have_q = r < g;
+            d.kind = kSweep2; d.ri = ri; d.ch = t % fl.np; d.have_q = r < g; d.part = kPartFirst | kPartLast;
+            item_range(cx.units, fl.np, d.ch, d.u0, d.u1);
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
             d.rowQ = r < g ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
                            : nullptr;
@@ -367,99 +443,222 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             if (lane == 0) { sh.desc[q % kFDesc] = d; mbar_arrive(smem_u32(&sh.full[q % kFDesc])); }
             __syncwarp();
         };
-        int q = 0, n = 0, qexit = -1;     // items published / post-processed; index of the exit descriptor
+        int q = 0;                        // items published
+        FlowDesc open;                    // the first-sweep chunk being handed out stretch by stretch
+        open.kind = kExit;
+        int open_n = 0, open_s = 0, open_u0 = 0, open_u1 = 0;   // its stretches, how many are out, its vectors
+        bool tail = false;                // the tickets are about to run out
         bool exhausted = false;           // the ticket counter has run past the last item
+        bool failed = false;
+        int depth = fl.depth;             // descriptors published and not yet swept, at most
         unsigned idle = 0;
+        draw_tickets(1);
+        poll();
         for (;;) {
-            // 1. publish what can be published (a slot is free once its previous item is post-processed)
-            while (qexit < 0 && q - n < fl.depth) {
-                FlowDesc d;
-                // (a) a piece of a row that waits for its second sweep: they are few and others wait for them
-                const int t = take_piece();
-                if (t >= 0) {
-                    if (!piece_desc(t, d)) { exhausted = true; break; }
-                    publish(d, q);
-                    ++q;
-                    continue;
+            // the slot must be free (its previous item moved out by its post warp), and at most `depth`
+            // published items may still be with the workers
+            if (q >= kFDesc && !mbar_wait_relaxed(smem_u32(&sh.freeb[q % kFDesc]), static_cast<uint32_t>(q / kFDesc - 1) & 1u, prm.status, 100)) { failed = true; break; }
+            if (q >= depth && !mbar_wait_relaxed(smem_u32(&sh.done[(q - depth) % kFDesc]), static_cast<uint32_t>((q - depth) / kFDesc) & 1u, prm.status, 100)) { failed = true; break; }
+            FlowDesc d;
+            d.kind = kExit;
+            // (a) a piece of a row that waits for its second sweep: they are few and others wait for them
+            int t = claim(seen_rows, seen_pieces, kCtrPieces, fl.np, held);
+            if (t >= 0) {
+                if (!piece_desc(t, d)) { failed = true; break; }
+                if (lane == 0) ++seen_pieces;
+            } else if (open_s == open_n && (t = claim(seen_late, seen_chunks, kCtrLateChunks, fl.nch_late, held_late)) >= 0) {
+                // (b) a chunk of a last target row that turned out to be wanted (a first sweep as well: it
+                // waits until the open chunk is handed out, whose sums the workers are carrying)
+                if (!late_desc(t, d)) { failed = true; break; }
+                if (lane == 0) ++seen_chunks;
+            } else if (open_s < open_n || !exhausted) {
+                // (c) the next stretch of the open first-sweep chunk, or a new chunk by the ticket drawn ahead
+                if (open_s == open_n) {
+                    if (tk_cnt == 0) draw_tickets(1);
+                    const unsigned t1 = next_ticket();
+                    if (t1 >= total_s1) { exhausted = true; tk_cnt = 0; continue; }
+                    sweep1_desc(t1, open);
+                    open_u0 = open.u0; open_u1 = open.u1;
+                    open_n = (open_u1 - open_u0 + fl.stretch - 1) / fl.stretch;
+                    if (open_n < 1) open_n = 1;
+                    open_s = 0;
+                    // Towards the end of the tickets a CTA no longer claims a chunk ahead of its needs:
+                    // a CTA that has run dry could start it at once.
+                    tail = t1 + gridDim.x >= total_s1;
                 }
-                // (b) a chunk of a last target row that turned out to be wanted
-                if (late_desc(d)) {
-                    publish(d, q);
-                    ++q;
-                    continue;
-                }
-                // (c) a new sweep-1 item
-                if (!exhausted) {
-                    take(d);
-                    if (d.kind == kExit) { exhausted = true; continue; }
-                    publish(d, q);
-                    ++q;
-                    continue;
-                }
-                // (d) nothing to start: leave once every block is finished
-                if (q == n && ld_volatile(&fl.counters[kCtrBlocks]) >= static_cast<unsigned>(cx.B)) {
-                    d.kind = kExit; publish(d, q); qexit = q; ++q;
-                }
-                break;
+                d = open;
+                item_range(open_u1 - open_u0, open_n, open_s, d.u0, d.u1);
+                d.u0 += open_u0; d.u1 += open_u0;
+                d.part = (open_s == 0 ? kPartFirst : 0) | (open_s == open_n - 1 ? kPartLast : 0);
+                ++open_s;
+                // the next ticket is drawn when this chunk is nearly handed out: its round trip is over by
+                // the time it is needed, and no chunk is claimed long before it can be started
+                if (!tail && tk_cnt == 0 && open_n - open_s <= 1) draw_tickets(1);
             }
-            // 2. the oldest item in flight: wait for the workers, then do what follows its sweep
-            const int in_flight_end = qexit >= 0 ? qexit : q;
-            if (n < in_flight_end) {
-                const int slot = n % kFDesc;
-                const FlowDesc d = sh.desc[slot];
-                mbar_wait_now(smem_u32(&sh.done[slot]), static_cast<uint32_t>(n / kFDesc) & 1u, prm.status);
-                if (d.kind == kSweep1) {
-                    f_after_sweep1<DT>(prm, fl, cx, sh, slot, d.ri, d.ch, lane);
-                } else {
-                    f_after_sweep2<DT>(prm, fl, cx, sh, slot, d, lane);
-                }
-                ++n;
+            if (d.kind != kExit) {
+                publish(d, q);
+                ++q;
+                poll();                   // (answers arrive while the workers sweep)
                 idle = 0;
                 continue;
             }
-            if (qexit >= 0) break;
-            // 3. nothing in flight and the next item waits for a row that another CTA completes
-            // (all idle CTAs look at the same counters: wait long enough not to crowd those who work)
+            // (d) nothing to start: leave once every block is finished and every item post-processed
+            if (*reinterpret_cast<volatile unsigned*>(&sh.posted) == static_cast<unsigned>(q) &&
+                ld_volatile(&fl.counters[kCtrBlocks]) >= static_cast<unsigned>(cx.B)) break;
+            // the next item waits for a row that another CTA completes (all idle CTAs look at the same
+            // counters: wait long enough not to crowd those who work)
             __nanosleep(idle < 4 ? 500 : 2000);
-            if (++idle > (1u << 21)) { if (prm.status) atomicExch(prm.status, 1); break; }
+            poll();
+            if (++idle > (1u << 21)) { if (prm.status) atomicExch(prm.status, 1); failed = true; break; }
         }
-        if (qexit < 0) {      // gave up: release the workers
+        // release the workers and the post warps: one exit descriptor for each post warp to find
+        // (on the regular way out every slot is free; after a wait that gave up nothing is relied on)
+        for (int j = 0; j < kFPost; ++j) {
             FlowDesc d; d.kind = kExit;
-            publish(d, q);
+            publish(d, q + j);
         }
         return;
     }
 
     // =============================== worker warps ===============================
-    const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;   // this thread's ring slot 0
-    for (int n = 0;; ++n) {
-        const int slot = n % kFDesc;
-        const uint32_t parity = static_cast<uint32_t>(n / kFDesc) & 1u;
-        mbar_wait_now(smem_u32(&sh.full[slot]), parity, prm.status);
-        const int kind = sh.desc[slot].kind;
-        if (kind == kExit) break;
-        const bool have_q = sh.desc[slot].have_q != 0;
-        const char* rowP = sh.desc[slot].rowP;
-        const char* rowQ = sh.desc[slot].rowQ;
+    // A warp sees the CTA's items as one stream of ring steps.  The consume side does the arithmetic
+    // of the oldest step in flight and then refills that very ring slot from the issue cursor, which
+    // runs kFSlots steps ahead and moves on to the next item as soon as it has asked for the last
+    // vector of the current one, provided the next descriptor is already there.  So the ring is not
+    // drained between items; it is only when the issue cursor finds no descriptor (or the exit
+    // descriptor) that it stops for good, and the consume side restarts it with a fresh prologue once
+    // it reaches an item whose loads have not been started.  Every ring step commits exactly one
+    // copy group (an empty one when nothing was asked for), so "all but the kFSlots - 1 newest groups
+    // are complete" always means that the slot about to be consumed has landed.
+    constexpr uint32_t kCell = kFThreads * 16;               // bytes between consecutive ring cells of a thread
+    const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;   // this thread's ring cell 0
+    const uint32_t ring_end = sb + kFDepth * kCell;
+    // no row is needed again soon (the few second sweeps come long after the first): stream past L2
+    const uint64_t pol = l2_policy_evict_first();
+    const char* iA = nullptr;         // issue cursor: this lane's next vector for cell A and for cell B
+    const char* iB = nullptr;
+    int i_rem = 0;                    // vectors of the current segment not yet asked for
+    int i_adv = 32;                   // vectors a step covers: 32 of each row, or 64 of the one row
+    int n_i = 0;                      // items the issue cursor has started
+    bool i_stalled = false;
+    uint32_t rp = sb;                 // ring slot to consume next, and to refill right afterwards
+
+    auto issue_load = [&](int slot) {
         int w0, w1;
-        chunk_range(cx, kind == kSweep1 ? cx.nch : fl.np, sh.desc[slot].ch, warp, w0, w1);
-        float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
+        warp_range(sh.desc[slot].u0, sh.desc[slot].u1, warp, w0, w1);
+        const bool single = sh.desc[slot].have_q == 0;
+        i_rem = w1 - w0;
+        i_adv = single ? 64 : 32;
+        iA = sh.desc[slot].rowP + static_cast<size_t>(w0 + lane) * 16;
+        iB = single ? iA + 512 : sh.desc[slot].rowQ + static_cast<size_t>(w0 + lane) * 16;
+    };
+    // one ring step of the issue cursor into the slot at `slot_addr`
+    auto issue_step = [&](uint32_t slot_addr) {
+        if (i_rem <= 0 && !i_stalled) {
+            for (;;) {                                       // the next item with something for this warp
+                const int slot = n_i % kFDesc;
+                if (!mbar_try_wait_now(smem_u32(&sh.full[slot]), static_cast<uint32_t>(n_i / kFDesc) & 1u) ||
+                    sh.desc[slot].kind == kExit) { i_stalled = true; break; }
+                issue_load(slot);
+                ++n_i;
+                if (i_rem > 0) break;
+            }
+        }
+        if (i_rem > 0) {
+            ring_fetch_hint(slot_addr, iA, lane < i_rem, R::kNegInf, pol);
+            ring_fetch_hint(slot_addr + kCell, iB, lane + (i_adv - 32) < i_rem, R::kNegInf, pol);
+            i_rem -= i_adv;
+            iA += static_cast<size_t>(i_adv) * 16;
+            iB += static_cast<size_t>(i_adv) * 16;
+        }
+        cp_async_commit();
+    };
+    float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
+    bool first = true;
+    for (int n_c = 0;; ++n_c) {
+        const int slot = n_c % kFDesc;
+        if (n_i == n_c) {
+            // the loads of this item have not been started: the ring is empty
+            if (!mbar_wait_now(smem_u32(&sh.full[slot]), static_cast<uint32_t>(n_c / kFDesc) & 1u, prm.status)) break;
+            if (sh.desc[slot].kind == kExit) break;
+            i_stalled = false;
+            issue_load(slot);
+            n_i = n_c + 1;
+            uint32_t a = rp;
+#pragma unroll
+            for (int j = 0; j < kFSlots; ++j) {
+                issue_step(a);
+                a += 2 * kCell;
+                if (a == ring_end) a = sb;
+            }
+        }
+        const int kind = sh.desc[slot].kind;
+        const bool have_q = sh.desc[slot].have_q != 0;
+        const int part = sh.desc[slot].part;
+        int w0, w1;
+        warp_range(sh.desc[slot].u0, sh.desc[slot].u1, warp, w0, w1);
+        int c_left = have_q ? (w1 - w0 + 31) >> 5 : (w1 - w0 + 63) >> 6;
+        // the sums of a first-sweep chunk run from its first stretch to its last, whatever comes in between
+        if (kind == kSweep1 && (part & kPartFirst)) { MPw = kNoRef; sP = 0.f; MQw = kNoRef; sQ = 0.f; first = true; }
+        float acc2 = 0.f;                 // a piece of a second sweep
+        // the steps of this item; the oldest step in flight is always the next one of this item
+        auto run_steps = [&](auto&& body) {
+            for (; c_left > 0; --c_left) {
+                cp_async_wait<kFSlots - 1>();
+                float va[EPV], vb[EPV];
+                R::unpack(lds128(rp), va);
+                R::unpack(lds128(rp + kCell), vb);
+                body(va, vb);
+                issue_step(rp);
+                rp += 2 * kCell;
+                if (rp == ring_end) rp = sb;
+            }
+        };
         if (kind == kSweep1) {
-            if (have_q) f_sweep_segment<DT, true, kSweep1>(sb, rowP, rowQ, w0, w1, lane, kf, 1.f, 0.f, 0.f, MPw, sP, MQw, sQ);
-            else        f_sweep_segment<DT, false, kSweep1>(sb, rowP, rowQ, w0, w1, lane, kf, 1.f, 0.f, 0.f, MPw, sP, MQw, sQ);
-            if (lane == 0) {
-                sh.part_M[slot][0][warp] = MPw; sh.part_s[slot][0][warp] = sP;
-                sh.part_M[slot][1][warp] = MQw; sh.part_s[slot][1][warp] = sQ;
+            if (have_q) {
+                run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
+                    if (first) {                             // references from the first vector of every lane
+                        MPw = fmaxf(rintf(warp_max(vec_max<EPV>(va)) * kf), kNoRef);
+                        MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vb)) * kf), kNoRef);
+                        first = false;
+                    }
+                    f_step_sweep1_pair<EPV>(va, vb, kf, MPw, sP, MQw, sQ);
+                });
+            } else {
+                run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
+                    if (first) { MPw = fmaxf(rintf(warp_max(fmaxf(vec_max<EPV>(va), vec_max<EPV>(vb))) * kf), kNoRef); first = false; }
+                    f_step_sweep1_single<EPV>(va, vb, kf, MPw, sP);
+                });
+            }
+            if (part & kPartLast) {
+                const float tP = warp_sum(sP);
+                const float tQ = have_q ? warp_sum(sQ) : 0.f;
+                if (lane == 0) {
+                    sh.part_M[slot][0][warp] = MPw; sh.part_s[slot][0][warp] = tP;
+                    sh.part_M[slot][1][warp] = MQw; sh.part_s[slot][1][warp] = tQ;
+                }
             }
         } else {
             const float cp = sh.desc[slot].cp, nMP = sh.desc[slot].nMP, nMQ = sh.desc[slot].nMQ;
-            if (have_q) f_sweep_segment<DT, true, kSweep2>(sb, rowP, rowQ, w0, w1, lane, kf, cp, nMP, nMQ, MPw, sP, MQw, sQ);
-            else        f_sweep_segment<DT, false, kSweep2>(sb, rowP, rowQ, w0, w1, lane, kf, cp, nMP, nMQ, MPw, sP, MQw, sQ);
-            if (lane == 0) sh.part_s[slot][0][warp] = sP;
+            if (have_q) {
+                run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
+                    float t[EPV];
+                    acc2 += f_pair_sum<EPV, true>(va, vb, kf, cp, nMP, nMQ, t);
+                });
+            } else {
+                run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
+                    float t[EPV];
+                    acc2 += f_pair_sum<EPV, false>(va, va, kf, cp, nMP, nMQ, t);
+                    acc2 += f_pair_sum<EPV, false>(vb, vb, kf, cp, nMP, nMQ, t);
+                });
+            }
+            const float tP = warp_sum(acc2);
+            if (lane == 0) sh.part_s[slot][0][warp] = tP;
         }
         if (lane == 0) mbar_arrive(smem_u32(&sh.done[slot]));   // releases this warp's partials and the descriptor
         __syncwarp();
     }
+    cp_async_wait<0>();
 }
 
 // ---------------------------------------------------------------------------
@@ -467,24 +666,24 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
 // ---------------------------------------------------------------------------
 static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 // floats of seg_tot per row: the sweep-2 totals (np pieces of kFWarps segments) or, for a last
-// target row, the sweep-1 {reference, sum} pairs (nch chunks of kFWarps segments)
-static size_t flow_seg_stride(int nch, int np) {
-    const size_t a = static_cast<size_t>(np) * kFWarps, b = static_cast<size_t>(nch) * kFWarps * 2;
+// target row, the sweep-1 {reference, sum} pairs (nch_late chunks of kFWarps segments)
+static size_t flow_seg_stride(const FlowPlan& plan) {
+    const size_t a = static_cast<size_t>(plan.np) * kFWarps, b = static_cast<size_t>(plan.nch_late) * kFWarps * 2;
     return a > b ? a : b;
 }
 
-size_t flow_scratch_bytes(int B, int gamma, int nch, int np, size_t* zero_bytes) {
+size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_bytes) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
-    const size_t segs = flow_seg_stride(nch, np);
+    const size_t segs = flow_seg_stride(plan);
     size_t z = 0;
     z += up256(kCounterWords * sizeof(unsigned));   // counters
-    z += 3 * up256(rows * sizeof(unsigned));        // row_cnt, row_done, s2_cnt
-    z += 4 * up256(static_cast<size_t>(B) * sizeof(unsigned));   // cand_cnt, chain, lock, bad
+    z += 2 * up256(rows * sizeof(unsigned));        // row_cnt, s2_cnt
+    z += 3 * up256(static_cast<size_t>(B) * sizeof(unsigned));   // cand_cnt, rows_in, bad
     z += 2 * up256(rows * sizeof(unsigned));        // rel, s2q
     z += up256(static_cast<size_t>(B) * sizeof(unsigned));       // lq
     if (zero_bytes) *zero_bytes = z;
     size_t n = z;
-    n += up256(rows * nch * sizeof(RowZ));          // part
+    n += up256(rows * plan.nch_max() * sizeof(RowZ));   // part
     n += up256(rows * sizeof(RowZ));                // rowZ
     n += up256(static_cast<size_t>(B) * (gamma + 2) * sizeof(double));   // pchain
     n += up256(rows * sizeof(float));               // cscale
@@ -495,18 +694,17 @@ size_t flow_scratch_bytes(int B, int gamma, int nch, int np, size_t* zero_bytes)
     return n;
 }
 
-void flow_scratch_layout(void* base, int B, int gamma, int nch, int np, FlowScratch* fl) {
+void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, FlowScratch* fl) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
-    const size_t segs = flow_seg_stride(nch, np);
+    const size_t segs = flow_seg_stride(plan);
+    const int nch = plan.nch_max();
     char* p = static_cast<char*>(base);
     auto take = [&](size_t bytes) { char* q = p; p += up256(bytes); return q; };
     fl->counters = reinterpret_cast<unsigned*>(take(kCounterWords * sizeof(unsigned)));
     fl->row_cnt = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
-    fl->row_done = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->s2_cnt = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->cand_cnt = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
-    fl->chain = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
-    fl->lock = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
+    fl->rows_in = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->bad = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->rel = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->s2q = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
@@ -520,33 +718,81 @@ void flow_scratch_layout(void* base, int B, int gamma, int nch, int np, FlowScra
     fl->seg_tot = reinterpret_cast<float*>(take(rows * segs * sizeof(float)));
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
+    fl->ntier = plan.ntier;
+    unsigned t = 0;
+    for (int k = 0; k <= kFlowTiers; ++k) { fl->tier_b[k] = B; fl->tier_t[k] = 0; }
+    for (int k = 0; k < kFlowTiers; ++k) fl->tier_n[k] = 1;
+    for (int k = 0; k < plan.ntier; ++k) {
+        fl->tier_b[k] = plan.tier_b[k];
+        fl->tier_n[k] = plan.tier_n[k];
+        fl->tier_t[k] = t;
+        t += static_cast<unsigned>(plan.tier_b[k + 1] - plan.tier_b[k]) * gamma * plan.tier_n[k];
+    }
+    for (int k = plan.ntier; k <= kFlowTiers; ++k) fl->tier_t[k] = t;
+    fl->tier_b[plan.ntier] = B;
     fl->nch = nch;
-    fl->np = np;
-    fl->depth = kFDesc;
+    fl->nch_late = plan.nch_late;
+    fl->np = plan.np;
+    fl->depth = 3;
+    fl->stretch = 1 << 30;
     fl->segs = static_cast<int>(segs);
 }
 
-// Pieces per row in the second sweep.  Only the few rows that may hold the selected position are
-// swept again, and the candidates of a block are swept one after the other, so their rows are cut
-// finer than in the first sweep: more CTAs share a row and the chain of a block gets shorter.  A
-// piece keeps at least 2048 vectors.
-int flow_pick_pieces(long long units) {
+// How a launch is cut into work items.
+//   First sweep: an item should be large next to what it costs to hand it out and account for it
+//   (a microsecond or two), so most rows are cut into chunks of about 16000 vectors (256 KB per row),
+//   finer while the batch alone cannot give every CTA a few items.  The last blocks of the launch
+//   are cut finer and finer (twice the chunks each time the items left would no longer fill the CTAs
+//   two and a half times over), so that the CTAs run out of first-sweep work at nearly the same time.
+//   A chunk keeps at least 2048 vectors.
+//   Second sweep, and the first sweep of a last target row that turns out to be wanted: only few rows
+//   are concerned and a block's candidates are swept one after the other, so these rows are cut into
+//   pieces of about 4000 vectors that many CTAs share.
+FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces) {
+    FlowPlan pl{};
     long long np = units / 4000;
     if (np < 1) np = 1;
     if (np > 8) np = 8;
-    return static_cast<int>(np);
-}
-
-// Chunks per row.  An item should be large next to what it costs to hand it out (about
-// 16000 vectors, 256 KB, per row), yet there should be a few items per CTA to balance the
-// load, as long as a chunk keeps at least 2048 vectors.
-int flow_pick_chunks(long long units, int B, int gamma, long long nctas) {
-    long long nch = (units + 8000) / 16000;
+    pl.np = pieces > 0 ? pieces : static_cast<int>(np);
+    pl.nch_late = static_cast<int>(np);
+    const long long row_units = pair_items ? units : units / 2;   // (a single-row item streams half as much)
+    long long nch = (row_units + 8000) / 16000;
     if (nch < 1) nch = 1;
     if (nch > 8) nch = 8;
-    const long long rows = static_cast<long long>(B) * (gamma + 1);
-    while (nch < 8 && rows * nch < 4 * nctas && units / (nch + 1) >= 2048) ++nch;
-    return static_cast<int>(nch);
+    const long long rows = static_cast<long long>(B) * gamma;
+    while (nch < 8 && rows * nch < 4 * nctas && row_units / (nch + 1) >= 2048) ++nch;
+    pl.ntier = 1;
+    pl.tier_b[0] = 0;
+    pl.tier_n[0] = static_cast<int>(nch);
+    pl.tier_b[1] = B;
+    if (chunks > 0) {
+        pl.tier_n[0] = chunks;
+        if (chunks > pl.nch_late && chunks <= 8) pl.nch_late = chunks;
+        return pl;
+    }
+    // finer tiers for the last blocks
+    long long cur = nch;
+    int b0 = 0;
+    while (pl.ntier < kFlowTiers) {
+        const long long next = cur * 2;
+        if (next > kFlowMaxChunks || row_units / next < 2048) break;
+        // the tier of `cur` chunks ends where the items left (at that chunk count) fall below 2.5 nctas
+        const long long left_blocks = (5 * nctas / 2 + gamma * cur - 1) / (gamma * cur);
+        int split = B - static_cast<int>(left_blocks < B ? left_blocks : B);
+        if (split <= b0) {               // this tier would be empty: start finer right away
+            pl.tier_n[pl.ntier - 1] = static_cast<int>(next);
+            cur = next;
+            continue;
+        }
+        if (split >= B) break;
+        pl.tier_b[pl.ntier] = split;
+        pl.tier_n[pl.ntier] = static_cast<int>(next);
+        ++pl.ntier;
+        pl.tier_b[pl.ntier] = B;
+        b0 = split;
+        cur = next;
+    }
+    return pl;
 }
 
 using FKernelFn = void (*)(const Params, const FlowScratch);

@@ -101,6 +101,17 @@ __device__ __forceinline__ RowZ load_rowz(const RowZ* p) {
     return z;
 }
 
+// chunks per row of block b in the first sweep (rows 0 .. gamma-1), and of row r of block b in general
+__device__ __forceinline__ int f_nch_block(const FlowScratch& fl, int b) {
+    int n = fl.tier_n[0];
+#pragma unroll
+    for (int k = 1; k < kFlowTiers; ++k) if (k < fl.ntier && b >= fl.tier_b[k]) n = fl.tier_n[k];
+    return n;
+}
+__device__ __forceinline__ int f_nch_row(const FlowScratch& fl, int b, int r, int g) {
+    return r == g ? fl.nch_late : f_nch_block(fl, b);
+}
+
 struct FlowCtx {
     int g, V, B, nch, units;
     size_t row_bytes;
@@ -114,41 +125,57 @@ template <int DT>
 __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int lane, float kf, float cp,
                         float nMP, float nMQ, float tw) {
     constexpr int EPV = Raw<DT>::EPV;
+    constexpr int kAhead = 4;                                // runs of 32 vectors whose loads are in flight together
     float run = 0.f;
     int found = -1, last_pos = -1;
-    for (int base = w0; base < w1 && found < 0; base += 32) {
-        const int i = base + lane;
-        float vp[EPV], vq[EPV], tt[EPV];
-        f_load_tail<DT>(rowP, i, w1, vp);
-        f_load_tail<DT>(rowQ, i, w1, vq);
-        const float ls = rowQ ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, tt)
-                              : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, tt);
+    for (int base0 = w0; base0 < w1 && found < 0; base0 += 32 * kAhead) {
+        // the loads of kAhead runs are issued before the first is looked at: the walk is a chain of
+        // dependent steps, and a load's latency is what each step would otherwise wait for
+        uint4 rp[kAhead], rq[kAhead];
 #pragma unroll
-        for (int e = 0; e < EPV; ++e) if (tt[e] > 0.f) last_pos = i * EPV + e;
-        float incw = ls;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const float o = __shfl_up_sync(0xffffffffu, incw, off);
-            if (lane >= off) incw += o;
+        for (int a = 0; a < kAhead; ++a) {
+            const int i = base0 + 32 * a + lane;
+            const bool ok = i < w1;
+            rp[a] = ok ? ld_stream_v4(rowP + static_cast<size_t>(i) * 16) : make_uint4(Raw<DT>::kNegInf, Raw<DT>::kNegInf, Raw<DT>::kNegInf, Raw<DT>::kNegInf);
+            rq[a] = (ok && rowQ) ? ld_stream_v4(rowQ + static_cast<size_t>(i) * 16) : make_uint4(Raw<DT>::kNegInf, Raw<DT>::kNegInf, Raw<DT>::kNegInf, Raw<DT>::kNegInf);
         }
-        const unsigned bal = __ballot_sync(0xffffffffu, run + incw > tw && ls > 0.f);
-        if (bal) {
-            const int src = __ffs(bal) - 1;
-            int f = -1;
-            if (lane == src) {
-                float cum = run + incw - ls;
-                int lp = -1;
 #pragma unroll
-                for (int e = 0; e < EPV; ++e) {
-                    cum += tt[e];
-                    if (tt[e] > 0.f) lp = i * EPV + e;
-                    if (f < 0 && cum > tw && tt[e] > 0.f) f = i * EPV + e;
-                }
-                if (f < 0) f = lp;
+        for (int a = 0; a < kAhead; ++a) {
+            const int base = base0 + 32 * a;
+            if (base >= w1 || found >= 0) break;
+            const int i = base + lane;
+            float vp[EPV], vq[EPV], tt[EPV];
+            Raw<DT>::unpack(rp[a], vp);
+            Raw<DT>::unpack(rq[a], vq);
+            const float ls = rowQ ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, tt)
+                                  : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, tt);
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) if (tt[e] > 0.f) last_pos = i * EPV + e;
+            float incw = ls;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float o = __shfl_up_sync(0xffffffffu, incw, off);
+                if (lane >= off) incw += o;
             }
-            found = __shfl_sync(0xffffffffu, f, src);
+            const unsigned bal = __ballot_sync(0xffffffffu, run + incw > tw && ls > 0.f);
+            if (bal) {
+                const int src = __ffs(bal) - 1;
+                int f = -1;
+                if (lane == src) {
+                    float cum = run + incw - ls;
+                    int lp = -1;
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) {
+                        cum += tt[e];
+                        if (tt[e] > 0.f) lp = i * EPV + e;
+                        if (f < 0 && cum > tw && tt[e] > 0.f) f = i * EPV + e;
+                    }
+                    if (f < 0) f = lp;
+                }
+                found = __shfl_sync(0xffffffffu, f, src);
+            }
+            run += __shfl_sync(0xffffffffu, incw, 31);
         }
-        run += __shfl_sync(0xffffffffu, incw, 31);
     }
     if (found < 0) {
 #pragma unroll
@@ -223,8 +250,8 @@ __device__ __forceinline__ bool f_all_positions(const Params& prm) {
     return prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
 }
 // Is the token of position gamma drawn from the first sweep of the last target row (bv_flow.cu)?
-__device__ __forceinline__ bool f_draws_in_sweep1(const Params& prm, int nch) {
-    return !f_all_positions(prm) && nch <= 8;
+__device__ __forceinline__ bool f_draws_in_sweep1(const Params& prm, int nch_late) {
+    return !f_all_positions(prm) && nch_late <= 8;
 }
 
 // ---- which positions get a second sweep (one thread each) ----
@@ -258,7 +285,7 @@ static __device__ void f_start_second_sweep(const FlowScratch& fl, size_t ci) {
 // one that turns out not to be needed costs bandwidth nobody else wants).
 static __device__ void f_release_next(const Params& prm, const FlowScratch& fl, int b, int below) {
     const int g = prm.gamma;
-    bool all = ld_volatile(&fl.counters[kCtrTicket]) >= static_cast<unsigned>(prm.B) * g * fl.nch;
+    bool all = ld_volatile(&fl.counters[kCtrTicket]) >= fl.tier_t[fl.ntier];
     if (all) {       // only a chain of three or more is worth the bandwidth of the ones not needed
         int held = 0;
         for (int c = below - 1; c >= 1; --c)
@@ -298,164 +325,172 @@ static __device__ unsigned f_after_position(const Params& prm, const FlowScratch
     return done;
 }
 
-// ---- a row is complete (one thread): its normalisers are published, then the recursion
-// advances over every complete row of the block ----
-template <int DT>
-__device__ void f_row_publish(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int r,
-                              double MP, double ZP, double MQ, double ZQ) {
-    const int g = cx.g;
-    const size_t rowi = static_cast<size_t>(b) * (g + 1) + r;
-    RowZ out; out.MP = MP; out.ZP = ZP; out.MQ = MQ; out.ZQ = ZQ;
-    fl.rowZ[rowi] = out;
-    const bool have_q = r < g;
-    // the row's maximum is finite iff its reference is; Z is NaN / inf iff the row holds a NaN / overflowed
-    if (!(MP > kNoRef && MP < INFINITY) || !(ZP < INFINITY)) atomicOr(&fl.bad[b], 1u);
-    if (have_q && (!(MQ > kNoRef && MQ < INFINITY) || !(ZQ < INFINITY))) atomicOr(&fl.bad[b], 1u);
-    // everything the recursion needs from this row, computed before the lock is taken:
-    // ratio = P_r(X_{r+1}) / Q_r(X_{r+1}) from the two logits of the drafted token, and Z_Q / Z_P
-    if (have_q) {
-        double ratio = 0.0;
-        const int x = prm.tok[static_cast<size_t>(b) * g + r];
-        if (x < 0 || x >= cx.V) {
-            atomicOr(&fl.bad[b], 1u);
-        } else {
-            const char* rowP = static_cast<const char*>(prm.tgt) + rowi * cx.row_bytes;
-            const char* rowQ = static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes;
-            const double zq = load_logit<DT>(rowQ, x), zp = load_logit<DT>(rowP, x);
-            if (zq == -INFINITY) atomicOr(&fl.bad[b], 1u);
-            else ratio = exp2((zp - zq) * cx.kd - (MP - MQ)) * (ZQ / ZP);
-        }
-        fl.ratio[rowi] = ratio;
-        fl.zratio[rowi] = ZQ / ZP;
-    }
-    __threadfence();
-    atomicExch(&fl.row_done[rowi], 1u);
-
-    // Fold every complete row, in order, into p_{c+1} = min(p_c ratio_c, 1) and release its
-    // sweep-2 items.  The critical section is a few loads and stores per row.
-    double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
-    for (unsigned spins = 0;; ++spins) {
-        if (atomicCAS(&fl.lock[b], 0u, 1u) == 0u) break;
-        // the holder may have looked at this row before it was marked: wait for it to let go,
-        // unless the recursion has already moved past this row
-        if (ld_volatile(&fl.chain[b]) > static_cast<unsigned>(r)) return;
-        __nanosleep(32);
-        if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return; }
-    }
-    __threadfence();
-    const bool all_positions = prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
-    unsigned nskip = 0;
-    bool folded = false, top_done = false;
-    unsigned c = ld_volatile(&fl.chain[b]);
-    while (c <= static_cast<unsigned>(g)) {
-        const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
-        if (ld_volatile(&fl.row_done[ci]) == 0u) {
-            // The last target row is read only on demand: P_gamma matters only if position gamma is
-            // the selected one, i.e. if eta_gamma <= p_gamma, which is known at this point.  Its first
-            // sweep is asked for now (the row joins a queue of its own), or the position is closed.
-            if (c == static_cast<unsigned>(g) && ld_volatile(&fl.rel[ci]) == 0u) {
-                const double p_g = __ldcg(&p[g]);
-                if (all_positions || static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + g - 1]) <= p_g * (1.0 + 1e-6)) {
-                    atomicExch(&fl.rel[ci], kRelLate);
-                    const unsigned slot = atomicAdd(&fl.counters[kCtrLateQueued], 1u);
-                    atomicExch(&fl.lq[slot], static_cast<unsigned>(ci) + 1u);
-                } else {
-                    fl.cand[ci] = -1;
-                    ++nskip;
-                    __threadfence();
-                    atomicExch(&fl.rel[ci], kRelSkip);
-                    ++c;
-                    folded = true;
-                    continue;
-                }
-            }
-            break;
-        }
-        const double p_c = (c == 0) ? 1.0 : __ldcg(&p[c]);
-        if (c == 0) p[0] = 1.0;
-        float cs = 1.f;
-        if (c < static_cast<unsigned>(g)) {
-            // Eq. "def_as" clips the running product at one; Algorithm 4 ("Set pt_i") does not
-            const double next = p_c * __ldcg(&fl.ratio[ci]);
-            p[c + 1] = prm.greedy ? next : fmin(next, 1.0);
-            cs = static_cast<float>(p_c * __ldcg(&fl.zratio[ci]));
-        }
-        fl.cscale[ci] = cs;
-        // Does anything depend on this position's second sweep?  S_c <= p_c (the residual mass of
-        // Eq. "pacc_block" is at most p_c sum_x P_c(x)), hence h_c <= p_c: a position whose
-        // uniform lies above p_c can never be the selected one, and nobody will ask for its S_c or
-        // its candidate.  Position gamma is selected iff eta_gamma <= h_gamma = p_gamma, and only then
-        // is the sample from P_gamma drawn.  Position 0 is what remains when no other is selected.
-        // (The margin keeps a uniform within rounding of p_c on the long path; with diagnostic
-        // outputs every position is computed.)  The unclipped product of Algorithm 4 obeys the same
-        // bound while it is at most one; above one the position passes its test whatever the
-        // uniform, and the comparison below makes it a candidate.
-        if (c == static_cast<unsigned>(g) && f_draws_in_sweep1(prm, cx.nch)) {
-            // the row was swept because position gamma can be selected, and its token was drawn from
-            // that very sweep: the position is complete.  It is the highest candidate, so either it
-            // is the selected one (lower candidates are dropped) or the next lower one is started.
-            __threadfence();
-            atomicExch(&fl.rel[ci], kRelSkip);
-            nskip += f_after_position(prm, fl, b, g);
-            top_done = true;
-            ++c;
-            folded = true;
-            continue;
-        }
-        bool need = all_positions || c == 0;
-        if (!need) need = static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + c - 1]) <= p_c * (1.0 + 1e-6);
-        if (!need) {
-            if (c < static_cast<unsigned>(g)) fl.S[ci] = 0.0;
-            fl.cand[ci] = -1;
-            ++nskip;
-        }
-        __threadfence();                       // p, cscale are visible ...
-        // ... before the row's sweep-2 items may start.  Candidates wait (on hold) until the whole
-        // block is folded and every higher candidate has been rejected.
-        if (need && all_positions) f_start_second_sweep(fl, ci);
-        else atomicExch(&fl.rel[ci], need ? kRelHold : kRelSkip);
-        ++c;
-        folded = true;
-    }
-    if (folded && !top_done && c == static_cast<unsigned>(g) + 1u && !all_positions) f_release_next(prm, fl, b, g + 1);
-    *reinterpret_cast<volatile unsigned*>(&fl.chain[b]) = c;
-    __threadfence();
-    atomicExch(&fl.lock[b], 0u);
-    // skipped positions count as complete; the last position to complete finishes the block
-    if (nskip > 0 && atomicAdd(&fl.cand_cnt[b], nskip) + nskip == static_cast<unsigned>(g) + 1u) {
-        __threadfence();
-        f_finalize_block(prm, fl, b);
-    }
+// ---- second sweeps of a block that has just been folded: the positions in `mask` (bit c =
+// position c; mask_hi: position c + 32) are started together; they take consecutive places in the
+// queue from which every CTA draws pieces (one warp) ----
+static __device__ void f_queue_rows(const FlowScratch& fl, int b, int g, unsigned mask, unsigned mask_hi, int lane) {
+    const int n_lo = __popc(mask), n = n_lo + __popc(mask_hi);
+    if (n == 0) return;
+    unsigned slot = 0;
+    if (lane == 0) slot = atomicAdd(&fl.counters[kCtrQueued], static_cast<unsigned>(n));
+    slot = __shfl_sync(0xffffffffu, slot, 0);
+    // the entry itself says when it is written (the queue starts at zero)
+    if (mask >> lane & 1u)
+        atomicExch(&fl.s2q[slot + __popc(mask & ((1u << lane) - 1u))], static_cast<unsigned>(b * (g + 1) + lane) + 1u);
+    if (mask_hi >> lane & 1u)
+        atomicExch(&fl.s2q[slot + n_lo + __popc(mask_hi & ((1u << lane) - 1u))], static_cast<unsigned>(b * (g + 1) + lane + 32) + 1u);
 }
 
-
-// ---- a row is complete: combine its chunks (one thread, fp64), then publish ----
+// ---- all rows 0 .. gamma-1 of a block have their normalisers: the prefix recursion
+// p_{c+1} = min(p_c ratio_c, 1) (Eq. "def_as"; Algorithm 4 does not clip), what becomes of every
+// position's second sweep, and the start of the first ones (one warp; lanes c and c + 32 speak for
+// positions c and c + 32) ----
 template <int DT>
-__device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int r) {
+__device__ void f_fold_block(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int lane) {
+    const int g = cx.g;
+    const bool all_positions = f_all_positions(prm);
+    __threadfence();
+    const size_t row0 = static_cast<size_t>(b) * (g + 1);
+    const float* u = prm.uni + static_cast<size_t>(b) * (g + 2);
+    // everything this warp needs from global memory, asked for in one go
+    double rat[2], zr[2];
+    float eta[2];                         // the uniform that position c is tested with: eta_c = uniforms[c - 1]
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int c = lane + 32 * h;
+        rat[h] = c < g ? __ldcg(&fl.ratio[row0 + c]) : 1.0;
+        zr[h] = c < g ? __ldcg(&fl.zratio[row0 + c]) : 1.0;
+        eta[h] = (c >= 1 && c < g) ? u[c - 1] : 0.f;
+    }
+    const float eta_g = u[g - 1];
+    const bool tail = ld_volatile(&fl.counters[kCtrTicket]) >= fl.tier_t[fl.ntier];
+    // the recursion, by every lane alike; a lane keeps the p of its own positions
+    double pc = 1.0, mine[2] = {1.0, 1.0};
+    for (int c = 0; c < g; ++c) {
+        if ((c & 31) == lane) mine[c >> 5] = pc;
+        const double r = shfl_d(c < 32 ? rat[0] : rat[1], c & 31);
+        const double next = pc * r;
+        pc = prm.greedy ? next : fmin(next, 1.0);
+    }
+    const double p_g = pc;
+    // Does anything depend on a position's second sweep?  S_c <= p_c (the residual mass of
+    // Eq. "pacc_block" is at most p_c sum_x P_c(x)), hence h_c <= p_c: a position whose uniform
+    // lies above p_c can never be the selected one, and nobody will ask for its S_c or its
+    // candidate.  Position gamma is selected iff eta_gamma <= h_gamma = p_gamma, and only then is the
+    // last target row read and the sample from P_gamma drawn.  Position 0 is what remains when no other
+    // is selected.  (The margin keeps a uniform within rounding of p_c on the long path; with
+    // diagnostic outputs every position is computed.)  The unclipped product of Algorithm 4 obeys
+    // the same bound while it is at most one; above one the position passes its test whatever the
+    // uniform, and the comparison below makes it a candidate.
+    double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
+    bool need[2] = {false, false};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int c = lane + 32 * h;
+        if (c < g) {
+            const size_t ci = row0 + c;
+            p[c] = mine[h];
+            need[h] = all_positions || c == 0 || static_cast<double>(eta[h]) <= mine[h] * (1.0 + 1e-6);
+            fl.cscale[ci] = static_cast<float>(mine[h] * zr[h]);
+            if (!need[h]) { fl.S[ci] = 0.0; fl.cand[ci] = -1; }
+        }
+    }
+    const bool last_row_wanted = all_positions || static_cast<double>(eta_g) <= p_g * (1.0 + 1e-6);
+    if (lane == 0) {
+        p[g] = p_g;
+        if (!last_row_wanted) fl.cand[row0 + g] = -1;
+    }
+    const unsigned m_lo = __ballot_sync(0xffffffffu, need[0]), m_hi = __ballot_sync(0xffffffffu, need[1]);
+    // Which second sweeps start now.  With diagnostics: all of them.  Otherwise the selected position
+    // is the highest candidate that passes its test, so the candidates are swept from the top, one
+    // at a time: position gamma first if it is one (its row joins the queue of last target rows),
+    // else the highest candidate below; position 0 only when it is alone.  Once the first-sweep
+    // tickets have run out the GPU is emptying and a block's chain of candidates, one after the
+    // other, would only prolong the launch: then all of them are started at once (a lower one that
+    // turns out not to be needed costs bandwidth nobody else wants).
+    unsigned s_lo = 0, s_hi = 0;
+    if (all_positions) { s_lo = m_lo; s_hi = m_hi; }
+    else if (!last_row_wanted) {
+        const unsigned c_lo = m_lo & ~1u;                    // candidates other than position 0
+        if ((c_lo | m_hi) == 0u) s_lo = 1u;
+        else if (tail && __popc(c_lo) + __popc(m_hi) >= 2) { s_lo = c_lo; s_hi = m_hi; }
+        else if (m_hi) s_hi = 1u << (31 - __clz(m_hi));
+        else s_lo = 1u << (31 - __clz(c_lo));
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int c = lane + 32 * h;
+        if (c < g) {
+            const bool started = ((h ? s_hi : s_lo) >> lane & 1u) != 0u;
+            fl.rel[row0 + c] = started ? kRelSweep : (need[h] ? kRelHold : kRelSkip);
+        }
+    }
+    if (lane == 0) fl.rel[row0 + g] = last_row_wanted ? kRelLate : kRelSkip;
+    __threadfence();
+    __syncwarp();
+    f_queue_rows(fl, b, g, s_lo, s_hi, lane);
+    if (lane == 0) {
+        if (last_row_wanted) {            // the last target row joins the queue of its kind
+            const unsigned slot = atomicAdd(&fl.counters[kCtrLateQueued], 1u);
+            atomicExch(&fl.lq[slot], static_cast<unsigned>(row0 + g) + 1u);
+        }
+        // skipped positions count as complete (position 0 never is, so the block cannot end here)
+        const unsigned nskip = static_cast<unsigned>(g - __popc(m_lo) - __popc(m_hi)) + (last_row_wanted ? 0u : 1u);
+        if (nskip > 0) atomicAdd(&fl.cand_cnt[b], nskip);
+    }
+    __syncwarp();
+}
+
+// ---- a row is complete (one warp): its chunks are combined (fp64) and its normalisers
+// published, for r < gamma with the ratio P_r(X_{r+1}) / Q_r(X_{r+1}) of the drafted token ----
+template <int DT>
+__device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int r, int lane) {
     const int g = cx.g;
     const size_t rowi = static_cast<size_t>(b) * (g + 1) + r;
-    // row reference = max of the chunk references
-    double MP = kNoRef, MQ = kNoRef;
-    for (int ch = 0; ch < cx.nch; ++ch) {
-        const RowZ z = load_rowz(&fl.part[rowi * cx.nch + ch]);
-        MP = fmax(MP, z.MP); MQ = fmax(MQ, z.MQ);
+    const int nch = f_nch_row(fl, b, r, g);
+    const bool have_q = r < g;
+    // loads in flight together: the chunks' sums, the drafted token
+    RowZ z; z.MP = kNoRef; z.ZP = 0.0; z.MQ = kNoRef; z.ZQ = 0.0;
+    if (lane < nch) z = load_rowz(&fl.part[rowi * cx.nch + lane]);
+    int x = (lane == 31 && have_q) ? prm.tok[static_cast<size_t>(b) * g + r] : 0;
+    x = __shfl_sync(0xffffffffu, x, 31);
+    const bool xok = have_q && x >= 0 && x < cx.V;
+    const char* rowP = static_cast<const char*>(prm.tgt) + rowi * cx.row_bytes;
+    const char* rowQ = static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + (have_q ? r : 0)) * cx.row_bytes;
+    double zl = 0.0;                      // the two logits of the drafted token (lanes 0 and 1)
+    if (xok && lane < 2) zl = load_logit<DT>(lane == 0 ? rowP : rowQ, x);
+    // row reference = max of the chunk references (integers, exact as floats), then the scaled sums
+    const float MPf = warp_max(static_cast<float>(z.MP)), MQf = warp_max(static_cast<float>(z.MQ));
+    double ZP = z.ZP * static_cast<double>(ref_scale(static_cast<float>(z.MP), MPf));
+    double ZQ = z.ZQ * static_cast<double>(ref_scale(static_cast<float>(z.MQ), MQf));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) { ZP += shfl_xor_d(ZP, off); ZQ += shfl_xor_d(ZQ, off); }
+    const double zp = shfl_d(zl, 0), zq = shfl_d(zl, 1);
+    if (lane == 0) {
+        double MP = MPf, MQ = MQf;
+        if (prm.lse_d != nullptr && have_q) {
+            // the draft row's normaliser is supplied: as an integer reference at or above every scaled
+            // logit of the row plus a sum in [2^-1/2, 2^1/2]; a value that is not finite leaves the
+            // row without a reference, which marks the block as faulty below
+            const double L2 = static_cast<double>(prm.lse_d[static_cast<size_t>(b) * g + r]) * 1.4426950408889634073599246810019;
+            const bool fin = L2 > -1e300 && L2 < 1e300;
+            MQ = fin ? rint(L2) : static_cast<double>(kNoRef);
+            ZQ = fin ? exp2(L2 - MQ) : 0.0;
+        }
+        RowZ out; out.MP = MP; out.ZP = ZP; out.MQ = MQ; out.ZQ = ZQ;
+        fl.rowZ[rowi] = out;
+        // the row's maximum is finite iff its reference is; Z is NaN / inf iff the row holds a NaN / overflowed
+        bool bad = !(MP > kNoRef && MP < INFINITY) || !(ZP < INFINITY);
+        if (have_q) {
+            bad = bad || !(MQ > kNoRef && MQ < INFINITY) || !(ZQ < INFINITY) || !xok || zq == -INFINITY;
+            // ratio = P_r(X_{r+1}) / Q_r(X_{r+1}) from the two logits of the drafted token
+            fl.ratio[rowi] = bad ? 0.0 : exp2((zp - zq) * cx.kd - (MP - MQ)) * (ZQ / ZP);
+            fl.zratio[rowi] = ZQ / ZP;
+        }
+        if (bad) atomicOr(&fl.bad[b], 1u);
     }
-    double ZP = 0.0, ZQ = 0.0;
-    for (int ch = 0; ch < cx.nch; ++ch) {
-        const RowZ z = load_rowz(&fl.part[rowi * cx.nch + ch]);
-        ZP += z.ZP * static_cast<double>(ref_scale(static_cast<float>(z.MP), static_cast<float>(MP)));
-        ZQ += z.ZQ * static_cast<double>(ref_scale(static_cast<float>(z.MQ), static_cast<float>(MQ)));
-    }
-    if (prm.lse_d != nullptr && r < g) {
-        // the draft row's normaliser is supplied: as an integer reference at or above every scaled
-        // logit of the row plus a sum in [2^-1/2, 2^1/2]; a value that is not finite leaves the
-        // row without a reference, which marks the block as faulty below
-        const double L2 = static_cast<double>(prm.lse_d[static_cast<size_t>(b) * g + r]) * 1.4426950408889634073599246810019;
-        const bool fin = L2 > -1e300 && L2 < 1e300;
-        MQ = fin ? rint(L2) : static_cast<double>(kNoRef);
-        ZQ = fin ? exp2(L2 - MQ) : 0.0;
-    }
-    f_row_publish<DT>(prm, fl, cx, b, r, MP, ZP, MQ, ZQ);
+    __threadfence();
+    __syncwarp();
 }
 
 // ---- a position is complete (one warp): S_r from the segment totals, and the candidate Y_r.

@@ -24,17 +24,16 @@ cudaError_t launch_cluster(const Params& prm, int algo, int dtype, int cluster, 
 // counters in a scratch area of flow_scratch_bytes(); its first *zero_bytes must be zero
 // when the kernel starts.
 struct RowZ { double MP, ZP, MQ, ZQ; };   // row (or chunk) references and sums of 2^{z k - M}
+constexpr int kFlowTiers = 4;
 struct FlowScratch {
     unsigned* counters;   // ticket counter of the sweep-1 items, rows queued for their second sweep, pieces of
                           // queued rows handed out, blocks finished (one 128-byte line each)
     unsigned* row_cnt;    // [B (gamma+1)] sweep-1 chunks finished per row
-    unsigned* row_done;   // [B (gamma+1)] row normalisers published
     unsigned* s2_cnt;     // [B (gamma+1)] sweep-2 chunks finished per position
     unsigned* cand_cnt;   // [B] positions with a candidate
-    unsigned* chain;      // [B] rows folded into the recursion
-    unsigned* lock;       // [B]
+    unsigned* rows_in;    // [B] rows 0 .. gamma-1 whose normalisers are published
     unsigned* bad;        // [B] data fault seen
-    unsigned* rel;        // [B (gamma+1)] row folded into the recursion, and what becomes of its second sweep
+    unsigned* rel;        // [B (gamma+1)] what becomes of the position's second sweep (0 until the block is folded)
     unsigned* s2q;        // [B (gamma+1)] queue of rows whose second sweep has been started (row index + 1)
     unsigned* lq;         // [B] queue of last target rows whose first sweep has been asked for (row index + 1)
     RowZ* part;           // [B (gamma+1) nch]
@@ -46,17 +45,35 @@ struct FlowScratch {
     float* seg_tot;       // [B (gamma+1) segs]
     double* S;            // [B (gamma+1)]
     int* cand;            // [B (gamma+1)]
-    int nch;              // chunks per row in the first sweep (1 .. kFlowMaxChunks)
+    // Chunks per row in the first sweep, by block: blocks tier_b[k] .. tier_b[k+1]-1 are cut into
+    // tier_n[k] chunks per row and own the tickets tier_t[k] .. tier_t[k+1]-1.  The last blocks of a
+    // launch are cut finer, so that the CTAs run out of first-sweep work at nearly the same time.
+    int ntier;
+    int tier_b[kFlowTiers + 1];
+    unsigned tier_t[kFlowTiers + 1];
+    int tier_n[kFlowTiers];
+    int nch;              // the largest chunk count of any row (stride of `part`)
+    int nch_late;         // chunks of a last target row, whose first sweep is asked for on demand
     int np;               // pieces per row in the second sweep (1 .. kFlowMaxChunks)
-    int depth;            // flow kernel: descriptors a CTA may have published and not yet post-processed (2 or 3)
+    int depth;            // flow kernel: descriptors a CTA may have handed to its workers and not yet seen swept
+    int stretch;          // vectors per row of one stretch of a first-sweep chunk
     int segs;             // residual totals kept per row
 };
 constexpr int kFlowMaxChunks = 32;
-size_t flow_scratch_bytes(int B, int gamma, int nch, int np, size_t* zero_bytes);
-void flow_scratch_layout(void* base, int B, int gamma, int nch, int np, FlowScratch* fl);
-int flow_pick_pieces(long long units);
+// How a launch is cut into work items: filled by flow_plan, completed by flow_scratch_layout.
+struct FlowPlan {
+    int ntier;
+    int tier_b[kFlowTiers + 1];
+    int tier_n[kFlowTiers];
+    int nch_late, np;
+    int nch_max() const { int m = nch_late; for (int k = 0; k < ntier; ++k) m = tier_n[k] > m ? tier_n[k] : m; return m; }
+};
+// units: 16-byte vectors per row; pair_items: false when the first sweep streams one row per item
+// (supplied draft normalisers); chunks / pieces > 0 force one chunk count for every block / the piece count.
+FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces);
+size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_bytes);
+void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, FlowScratch* fl);
 int flow_max_ctas_per_sm(int dtype);
-int flow_pick_chunks(long long units, int B, int gamma, long long nctas);
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream);
 
 

@@ -83,10 +83,9 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
 
     // same chunking rule as bv_verify, so both entry points take identical arithmetic paths
     const long long units = static_cast<long long>(row_bytes / 16);
-    const int nch = bv::flow_pick_chunks(units, B, gamma, static_cast<long long>(d.sm_count) * per_sm);
+    const bv::FlowPlan plan = bv::flow_plan(units, B, gamma, static_cast<long long>(d.sm_count) * per_sm, true, 0, 0);
     size_t zero_bytes = 0;
-    const int np = bv::flow_pick_pieces(units);
-    const size_t need = bv::flow_scratch_bytes(B, gamma, nch, np, &zero_bytes) + 256;   // + the status word
+    const size_t need = bv::flow_scratch_bytes(B, gamma, plan, &zero_bytes) + 256;   // + the status word
     if (need > kScratchBytes) return BV_ERR_TOO_LARGE;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -97,7 +96,7 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     if (cudaMemsetAsync(status_word, 0, 256, s) != cudaSuccess) { cudaGetLastError(); return BV_ERR_CUDA; }
 
     bv::FlowScratch fl;
-    bv::flow_scratch_layout(d.scratch, B, gamma, nch, np, &fl);
+    bv::flow_scratch_layout(d.scratch, B, gamma, plan, &fl);
     bv::Params prm{};
     prm.tgt = tgt; prm.drf = drf; prm.tok = tok; prm.uni = uni;
     prm.B = B; prm.gamma = gamma; prm.V = V;
@@ -106,7 +105,7 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     prm.kf = static_cast<float>(kd);
     prm.out_tokens = ot; prm.out_len = ol;
     prm.status = reinterpret_cast<int*>(status_word);
-    long long items = static_cast<long long>(B) * (gamma + 1) * nch;
+    long long items = static_cast<long long>(fl.tier_t[fl.ntier]);
     long long nctas = static_cast<long long>(d.sm_count) * per_sm;
     if (nctas > items) nctas = items;
     if (bv::launch_flow(prm, fl, dtype, static_cast<int>(nctas), s) != cudaSuccess) return BV_ERR_CUDA;
