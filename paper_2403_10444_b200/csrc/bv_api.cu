@@ -186,13 +186,9 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
                 const int v = std::atoi(env);
                 if (v >= 2 && v <= 6) fl.depth = v;
             }
-            if (const char* env = std::getenv("BV_FLOW_STRETCH")) {
-                const int v = std::atoi(env);
-                if (v >= 256) fl.stretch = v;
-            }
             cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
             if (e != cudaSuccess) return cuda_fail(e);
-            long long items = static_cast<long long>(fl.tier_t[fl.ntier]);
+            long long items = static_cast<long long>(fl.total_s1);
             if (nctas > items) nctas = items;
             prm.ticket = nullptr;
             prm.nclusters = 0;

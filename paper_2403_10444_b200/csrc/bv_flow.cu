@@ -63,17 +63,11 @@ constexpr int kFDesc = 8;      // descriptors a CTA can hold: being swept, queue
 constexpr int kFPost = 3;      // post warps: what follows the sweep of item n is done by post warp n mod kFPost
 constexpr int kFAllThreads = kFThreads + 32 * (1 + kFPost);   // worker warps + the publisher + the post warps
 
-// A first-sweep chunk is handed to the workers in stretches (same row, consecutive vectors): the
-// workers carry their sums from stretch to stretch and leave them after the last one, nothing is
-// asked of global memory in between, and a piece of a second sweep, for which a block is waiting,
-// can be slipped in after any stretch.
-enum : int { kPartFirst = 1, kPartLast = 2 };
 // One work item as the publisher hands it to the workers.
 struct FlowDesc {
     int kind;                   // kExit, kSweep1, kSweep2
     int ri, ch;                 // row index b (gamma+1) + r, chunk
-    int u0, u1;                 // vectors [u0, u1) of the row: the chunk, or one stretch of it
-    int part;                   // kPartFirst: the chunk starts here; kPartLast: it ends here
+    int u0, u1;                 // the chunk's vectors [u0, u1) of the row
     int have_q;
     const char* rowP;
     const char* rowQ;
@@ -182,7 +176,7 @@ __device__ void f_store_sweep1(const Params& prm, const FlowScratch& fl, const F
     }
     if (lane == 0) {
         RowZ z; z.MP = MPc; z.ZP = zP; z.MQ = MQc; z.ZQ = zQ;
-        fl.part[static_cast<size_t>(ri) * cx.nch + ch] = z;
+        fl.part[static_cast<size_t>(ri) * fl.part_stride + ch] = z;
     }
 }
 template <int DT>
@@ -201,18 +195,15 @@ __device__ void f_complete_sweep1(const Params& prm, const FlowScratch& fl, cons
         // drawn from that very sweep: the position is complete.  It is the highest candidate, so
         // either it is the selected one (lower candidates are dropped) or the next lower one is started.
         f_draw_from_sweep1<DT>(prm, fl, cx, ri, lane);
-        if (lane == 0) {
-            atomicExch(&fl.rel[ri], kRelSkip);
-            const unsigned done = f_after_position(prm, fl, b, g);
-            if (atomicAdd(&fl.cand_cnt[b], done) + done == static_cast<unsigned>(g) + 1u) {
-                __threadfence();
-                f_finalize_block(prm, fl, b);
-            }
-        }
-        __syncwarp();
+        f_position_done(prm, fl, b, g, lane);
     } else {
         // with diagnostics the sample from P_gamma comes from a second sweep of the row, like any other
-        if (lane == 0) f_start_second_sweep(fl, static_cast<size_t>(ri));
+        if (lane == 0) {
+            atomicExch(&fl.rel[ri], kRelSweep);
+            __threadfence();
+            const unsigned slot = atomicAdd(&fl.counters[kCtrQueued], 1u);
+            atomicExch(&fl.s2q[slot], static_cast<unsigned>(ri) + 1u);
+        }
         __syncwarp();
     }
 }
@@ -280,7 +271,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     extern __shared__ __align__(16) unsigned char dyn[];
 
     FlowCtx cx;
-    cx.g = prm.gamma; cx.V = prm.V; cx.B = prm.B; cx.nch = fl.nch; cx.units = prm.V / EPV;
+    cx.g = prm.gamma; cx.V = prm.V; cx.B = prm.B; cx.units = prm.V / EPV;
     cx.row_bytes = static_cast<size_t>(prm.V) * ESZ; cx.kf = prm.kf; cx.kd = prm.kd;
     const int g = cx.g;
     const float kf = cx.kf;
@@ -311,11 +302,6 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             if (!mbar_wait_relaxed(smem_u32(&sh.full[slot]), par, prm.status, 200)) break;
             if (sh.desc[slot].kind == kExit) break;
             if (!mbar_wait_relaxed(smem_u32(&sh.done[slot]), par, prm.status, 200)) break;
-            if (!(sh.desc[slot].part & kPartLast)) {         // a stretch inside a chunk: the workers carry on
-                __syncwarp();
-                if (lane == 0) { mbar_arrive(smem_u32(&sh.freeb[slot])); atomicAdd(&sh.posted, 1u); }
-                continue;
-            }
             if (lane == 0) sh.sdesc[k] = sh.desc[slot];
             if (lane < kFWarps) {
                 sh.stage_M[k][0][lane] = sh.part_M[slot][0][lane]; sh.stage_M[k][1][lane] = sh.part_M[slot][1][lane];
@@ -330,7 +316,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             __syncwarp();
             int last = 0;
             if (lane == 0) {
-                if (d.kind == kSweep1) last = atomicAdd(&fl.row_cnt[d.ri], 1u) == static_cast<unsigned>(f_nch_row(fl, d.ri / (g + 1), d.ri % (g + 1), g)) - 1u;
+                if (d.kind == kSweep1) last = atomicAdd(&fl.row_cnt[d.ri], 1u) == static_cast<unsigned>(f_nch_row(fl, d.ri % (g + 1), g)) - 1u;
                 else last = atomicAdd(&fl.s2_cnt[d.ri], 1u) == static_cast<unsigned>(fl.np) - 1u;
             }
             last = __shfl_sync(0xffffffffu, last, 0);
@@ -350,7 +336,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         // counters are read after every descriptor for the next one, and tickets of first-sweep items
         // are drawn ahead of their use.
         // tickets cover the rows that every block needs: target and draft rows 0 .. gamma-1
-        const unsigned total_s1 = fl.tier_t[fl.ntier];
+        const unsigned total_s1 = fl.total_s1;
         // Tickets are drawn several at a time (one atomic) and ahead of their use, so that the round
         // trip is over by the time a descriptor slot is free.
         unsigned tk_raw = 0, tk_lo = 0;   // (lane 0) answer of the last draw; next ticket on hand (all lanes)
@@ -368,16 +354,12 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         };
         // the first-sweep item of ticket t
         auto sweep1_desc = [&](unsigned t, FlowDesc& d) {
-            int k = 0;
-#pragma unroll
-            for (int j = 1; j < kFlowTiers; ++j) if (j < fl.ntier && t >= fl.tier_t[j]) k = j;
-            const unsigned local = t - fl.tier_t[k];
-            const int nch = fl.tier_n[k];
-            const int ch = static_cast<int>(local % nch);
-            const int r = static_cast<int>(local / nch) % g, b = fl.tier_b[k] + static_cast<int>(local / nch) / g;
+            const int nch = fl.nch;
+            const int ch = static_cast<int>(t % nch);
+            const int r = static_cast<int>(t / nch) % g, b = static_cast<int>(t / nch) / g;
             const int ri = b * (g + 1) + r;
             // (with supplied draft normalisers the first sweep has nothing to learn from the draft row)
-            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = prm.lse_d == nullptr; d.part = kPartFirst | kPartLast;
+            d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = prm.lse_d == nullptr;
             item_range(cx.units, nch, ch, d.u0, d.u1);
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
             d.rowQ = d.have_q ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
@@ -414,7 +396,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             for (unsigned spins = 0; (e = ld_volatile(&fl.lq[t / fl.nch_late])) == 0u; ++spins)
                 if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
             const int ri = static_cast<int>(e - 1u);
-            d.kind = kSweep1; d.ri = ri; d.ch = t % fl.nch_late; d.have_q = 0; d.part = kPartFirst | kPartLast;
+            d.kind = kSweep1; d.ri = ri; d.ch = t % fl.nch_late; d.have_q = 0;
             item_range(cx.units, fl.nch_late, d.ch, d.u0, d.u1);
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
             d.rowQ = nullptr;
@@ -427,7 +409,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
             const int ri = static_cast<int>(e - 1u);
             const int r = ri % (g + 1), b = ri / (g + 1);
-            d.kind = kSweep2; d.ri = ri; d.ch = t % fl.np; d.have_q = r < g; d.part = kPartFirst | kPartLast;
+            d.kind = kSweep2; d.ri = ri; d.ch = t % fl.np; d.have_q = r < g;
             item_range(cx.units, fl.np, d.ch, d.u0, d.u1);
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
             d.rowQ = r < g ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes
@@ -444,9 +426,6 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             __syncwarp();
         };
         int q = 0;                        // items published
-        FlowDesc open;                    // the first-sweep chunk being handed out stretch by stretch
-        open.kind = kExit;
-        int open_n = 0, open_s = 0, open_u0 = 0, open_u1 = 0;   // its stretches, how many are out, its vectors
         bool tail = false;                // the tickets are about to run out
         bool exhausted = false;           // the ticket counter has run past the last item
         bool failed = false;
@@ -466,34 +445,20 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             if (t >= 0) {
                 if (!piece_desc(t, d)) { failed = true; break; }
                 if (lane == 0) ++seen_pieces;
-            } else if (open_s == open_n && (t = claim(seen_late, seen_chunks, kCtrLateChunks, fl.nch_late, held_late)) >= 0) {
-                // (b) a chunk of a last target row that turned out to be wanted (a first sweep as well: it
-                // waits until the open chunk is handed out, whose sums the workers are carrying)
+            } else if ((t = claim(seen_late, seen_chunks, kCtrLateChunks, fl.nch_late, held_late)) >= 0) {
+                // (b) a chunk of a last target row that turned out to be wanted
                 if (!late_desc(t, d)) { failed = true; break; }
                 if (lane == 0) ++seen_chunks;
-            } else if (open_s < open_n || !exhausted) {
-                // (c) the next stretch of the open first-sweep chunk, or a new chunk by the ticket drawn ahead
-                if (open_s == open_n) {
-                    if (tk_cnt == 0) draw_tickets(1);
-                    const unsigned t1 = next_ticket();
-                    if (t1 >= total_s1) { exhausted = true; tk_cnt = 0; continue; }
-                    sweep1_desc(t1, open);
-                    open_u0 = open.u0; open_u1 = open.u1;
-                    open_n = (open_u1 - open_u0 + fl.stretch - 1) / fl.stretch;
-                    if (open_n < 1) open_n = 1;
-                    open_s = 0;
-                    // Towards the end of the tickets a CTA no longer claims a chunk ahead of its needs:
-                    // a CTA that has run dry could start it at once.
-                    tail = t1 + gridDim.x >= total_s1;
-                }
-                d = open;
-                item_range(open_u1 - open_u0, open_n, open_s, d.u0, d.u1);
-                d.u0 += open_u0; d.u1 += open_u0;
-                d.part = (open_s == 0 ? kPartFirst : 0) | (open_s == open_n - 1 ? kPartLast : 0);
-                ++open_s;
-                // the next ticket is drawn when this chunk is nearly handed out: its round trip is over by
-                // the time it is needed, and no chunk is claimed long before it can be started
-                if (!tail && tk_cnt == 0 && open_n - open_s <= 1) draw_tickets(1);
+            } else if (!exhausted) {
+                // (c) a new first-sweep chunk, by the ticket drawn ahead
+                if (tk_cnt == 0) draw_tickets(1);
+                const unsigned t1 = next_ticket();
+                if (t1 >= total_s1) { exhausted = true; tk_cnt = 0; continue; }
+                sweep1_desc(t1, d);
+                // Towards the end of the tickets a CTA no longer claims a chunk ahead of its needs:
+                // a CTA that has run dry could start it at once.
+                tail = t1 + gridDim.x >= total_s1;
+                if (!tail) draw_tickets(1);
             }
             if (d.kind != kExit) {
                 publish(d, q);
@@ -573,8 +538,6 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         }
         cp_async_commit();
     };
-    float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
-    bool first = true;
     for (int n_c = 0;; ++n_c) {
         const int slot = n_c % kFDesc;
         if (n_i == n_c) {
@@ -594,13 +557,11 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         }
         const int kind = sh.desc[slot].kind;
         const bool have_q = sh.desc[slot].have_q != 0;
-        const int part = sh.desc[slot].part;
         int w0, w1;
         warp_range(sh.desc[slot].u0, sh.desc[slot].u1, warp, w0, w1);
         int c_left = have_q ? (w1 - w0 + 31) >> 5 : (w1 - w0 + 63) >> 6;
-        // the sums of a first-sweep chunk run from its first stretch to its last, whatever comes in between
-        if (kind == kSweep1 && (part & kPartFirst)) { MPw = kNoRef; sP = 0.f; MQw = kNoRef; sQ = 0.f; first = true; }
-        float acc2 = 0.f;                 // a piece of a second sweep
+        float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
+        bool first = true;
         // the steps of this item; the oldest step in flight is always the next one of this item
         auto run_steps = [&](auto&& body) {
             for (; c_left > 0; --c_left) {
@@ -630,29 +591,27 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                     f_step_sweep1_single<EPV>(va, vb, kf, MPw, sP);
                 });
             }
-            if (part & kPartLast) {
-                const float tP = warp_sum(sP);
-                const float tQ = have_q ? warp_sum(sQ) : 0.f;
-                if (lane == 0) {
-                    sh.part_M[slot][0][warp] = MPw; sh.part_s[slot][0][warp] = tP;
-                    sh.part_M[slot][1][warp] = MQw; sh.part_s[slot][1][warp] = tQ;
-                }
+            const float tP = warp_sum(sP);
+            const float tQ = have_q ? warp_sum(sQ) : 0.f;
+            if (lane == 0) {
+                sh.part_M[slot][0][warp] = MPw; sh.part_s[slot][0][warp] = tP;
+                sh.part_M[slot][1][warp] = MQw; sh.part_s[slot][1][warp] = tQ;
             }
         } else {
             const float cp = sh.desc[slot].cp, nMP = sh.desc[slot].nMP, nMQ = sh.desc[slot].nMQ;
             if (have_q) {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
                     float t[EPV];
-                    acc2 += f_pair_sum<EPV, true>(va, vb, kf, cp, nMP, nMQ, t);
+                    sP += f_pair_sum<EPV, true>(va, vb, kf, cp, nMP, nMQ, t);
                 });
             } else {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
                     float t[EPV];
-                    acc2 += f_pair_sum<EPV, false>(va, va, kf, cp, nMP, nMQ, t);
-                    acc2 += f_pair_sum<EPV, false>(vb, vb, kf, cp, nMP, nMQ, t);
+                    sP += f_pair_sum<EPV, false>(va, va, kf, cp, nMP, nMQ, t);
+                    sP += f_pair_sum<EPV, false>(vb, vb, kf, cp, nMP, nMQ, t);
                 });
             }
-            const float tP = warp_sum(acc2);
+            const float tP = warp_sum(sP);
             if (lane == 0) sh.part_s[slot][0][warp] = tP;
         }
         if (lane == 0) mbar_arrive(smem_u32(&sh.done[slot]));   // releases this warp's partials and the descriptor
@@ -683,7 +642,7 @@ size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_b
     z += up256(static_cast<size_t>(B) * sizeof(unsigned));       // lq
     if (zero_bytes) *zero_bytes = z;
     size_t n = z;
-    n += up256(rows * plan.nch_max() * sizeof(RowZ));   // part
+    n += up256(rows * plan.part_stride() * sizeof(RowZ));   // part
     n += up256(rows * sizeof(RowZ));                // rowZ
     n += up256(static_cast<size_t>(B) * (gamma + 2) * sizeof(double));   // pchain
     n += up256(rows * sizeof(float));               // cscale
@@ -697,7 +656,6 @@ size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_b
 void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, FlowScratch* fl) {
     const size_t rows = static_cast<size_t>(B) * (gamma + 1);
     const size_t segs = flow_seg_stride(plan);
-    const int nch = plan.nch_max();
     char* p = static_cast<char*>(base);
     auto take = [&](size_t bytes) { char* q = p; p += up256(bytes); return q; };
     fl->counters = reinterpret_cast<unsigned*>(take(kCounterWords * sizeof(unsigned)));
@@ -709,7 +667,7 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->rel = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->s2q = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->lq = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
-    fl->part = reinterpret_cast<RowZ*>(take(rows * nch * sizeof(RowZ)));
+    fl->part = reinterpret_cast<RowZ*>(take(rows * plan.part_stride() * sizeof(RowZ)));
     fl->rowZ = reinterpret_cast<RowZ*>(take(rows * sizeof(RowZ)));
     fl->pchain = reinterpret_cast<double*>(take(static_cast<size_t>(B) * (gamma + 2) * sizeof(double)));
     fl->cscale = reinterpret_cast<float*>(take(rows * sizeof(float)));
@@ -718,33 +676,20 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->seg_tot = reinterpret_cast<float*>(take(rows * segs * sizeof(float)));
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
-    fl->ntier = plan.ntier;
-    unsigned t = 0;
-    for (int k = 0; k <= kFlowTiers; ++k) { fl->tier_b[k] = B; fl->tier_t[k] = 0; }
-    for (int k = 0; k < kFlowTiers; ++k) fl->tier_n[k] = 1;
-    for (int k = 0; k < plan.ntier; ++k) {
-        fl->tier_b[k] = plan.tier_b[k];
-        fl->tier_n[k] = plan.tier_n[k];
-        fl->tier_t[k] = t;
-        t += static_cast<unsigned>(plan.tier_b[k + 1] - plan.tier_b[k]) * gamma * plan.tier_n[k];
-    }
-    for (int k = plan.ntier; k <= kFlowTiers; ++k) fl->tier_t[k] = t;
-    fl->tier_b[plan.ntier] = B;
-    fl->nch = nch;
+    fl->nch = plan.nch;
+    fl->part_stride = plan.part_stride();
+    fl->total_s1 = static_cast<unsigned>(B) * gamma * plan.nch;
     fl->nch_late = plan.nch_late;
     fl->np = plan.np;
     fl->depth = 3;
-    fl->stretch = 1 << 30;
     fl->segs = static_cast<int>(segs);
 }
 
 // How a launch is cut into work items.
 //   First sweep: an item should be large next to what it costs to hand it out and account for it
-//   (a microsecond or two), so most rows are cut into chunks of about 16000 vectors (256 KB per row),
-//   finer while the batch alone cannot give every CTA a few items.  The last blocks of the launch
-//   are cut finer and finer (twice the chunks each time the items left would no longer fill the CTAs
-//   two and a half times over), so that the CTAs run out of first-sweep work at nearly the same time.
-//   A chunk keeps at least 2048 vectors.
+//   (about a microsecond, and half a ring step per warp at its end), so rows are cut into chunks of
+//   about 16000 vectors (256 KB per row), finer while the batch alone cannot give every CTA a few
+//   items.  A chunk keeps at least 2048 vectors.
 //   Second sweep, and the first sweep of a last target row that turns out to be wanted: only few rows
 //   are concerned and a block's candidates are swept one after the other, so these rows are cut into
 //   pieces of about 4000 vectors that many CTAs share.
@@ -761,37 +706,8 @@ FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair
     if (nch > 8) nch = 8;
     const long long rows = static_cast<long long>(B) * gamma;
     while (nch < 8 && rows * nch < 4 * nctas && row_units / (nch + 1) >= 2048) ++nch;
-    pl.ntier = 1;
-    pl.tier_b[0] = 0;
-    pl.tier_n[0] = static_cast<int>(nch);
-    pl.tier_b[1] = B;
-    if (chunks > 0) {
-        pl.tier_n[0] = chunks;
-        if (chunks > pl.nch_late && chunks <= 8) pl.nch_late = chunks;
-        return pl;
-    }
-    // finer tiers for the last blocks
-    long long cur = nch;
-    int b0 = 0;
-    while (pl.ntier < kFlowTiers) {
-        const long long next = cur * 2;
-        if (next > kFlowMaxChunks || row_units / next < 2048) break;
-        // the tier of `cur` chunks ends where the items left (at that chunk count) fall below 2.5 nctas
-        const long long left_blocks = (5 * nctas / 2 + gamma * cur - 1) / (gamma * cur);
-        int split = B - static_cast<int>(left_blocks < B ? left_blocks : B);
-        if (split <= b0) {               // this tier would be empty: start finer right away
-            pl.tier_n[pl.ntier - 1] = static_cast<int>(next);
-            cur = next;
-            continue;
-        }
-        if (split >= B) break;
-        pl.tier_b[pl.ntier] = split;
-        pl.tier_n[pl.ntier] = static_cast<int>(next);
-        ++pl.ntier;
-        pl.tier_b[pl.ntier] = B;
-        b0 = split;
-        cur = next;
-    }
+    pl.nch = chunks > 0 ? chunks : static_cast<int>(nch);
+    if (chunks > pl.nch_late && chunks <= 8) pl.nch_late = chunks;
     return pl;
 }
 

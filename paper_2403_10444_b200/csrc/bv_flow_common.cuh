@@ -101,19 +101,11 @@ __device__ __forceinline__ RowZ load_rowz(const RowZ* p) {
     return z;
 }
 
-// chunks per row of block b in the first sweep (rows 0 .. gamma-1), and of row r of block b in general
-__device__ __forceinline__ int f_nch_block(const FlowScratch& fl, int b) {
-    int n = fl.tier_n[0];
-#pragma unroll
-    for (int k = 1; k < kFlowTiers; ++k) if (k < fl.ntier && b >= fl.tier_b[k]) n = fl.tier_n[k];
-    return n;
-}
-__device__ __forceinline__ int f_nch_row(const FlowScratch& fl, int b, int r, int g) {
-    return r == g ? fl.nch_late : f_nch_block(fl, b);
-}
+// chunks of row r of a block in its first sweep
+__device__ __forceinline__ int f_nch_row(const FlowScratch& fl, int r, int g) { return r == g ? fl.nch_late : fl.nch; }
 
 struct FlowCtx {
-    int g, V, B, nch, units;
+    int g, V, B, units;
     size_t row_bytes;
     float kf;
     double kd;
@@ -197,137 +189,93 @@ __device__ __forceinline__ double f_weight(double pi, double Si) {
     return den > 0.0 ? Si / den : INFINITY;
 }
 
-// ---- the end of a block (one thread): Eq. "pacc_block", selection of tau, output ----
-static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl, int b) {
+// With diagnostic outputs every position is computed in full.
+__device__ __forceinline__ bool f_all_positions(const Params& prm) {
+    return prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
+}
+
+// ---- the end of a block (one warp; lanes i and i + 32 speak for positions i and i + 32, position
+// gamma is handled by every lane alike): Eq. "pacc_block", selection of tau, output ----
+static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl, int b, int lane) {
     const int g = prm.gamma;
+    __threadfence();
     int32_t* ot = prm.out_tokens + static_cast<size_t>(b) * (g + 1);
     const int32_t* X = prm.tok + static_cast<size_t>(b) * g;
     const float* u = prm.uni + static_cast<size_t>(b) * (g + 2);
     const double* p = fl.pchain + static_cast<size_t>(b) * (g + 2);
     const double* S = fl.S + static_cast<size_t>(b) * (g + 1);
     const int* cand = fl.cand + static_cast<size_t>(b) * (g + 1);
+    // everything asked for in one go
+    double pi[2], Si[2];
+    float eta[2];
+    int cd[2], xi[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int i = lane + 32 * h;
+        const bool in = i < g;
+        pi[h] = in ? __ldcg(&p[i]) : 0.0;
+        Si[h] = in ? __ldcg(&S[i]) : 0.0;
+        cd[h] = in ? __ldcg(&cand[i]) : -1;
+        eta[h] = (in && i >= 1) ? u[i - 1] : 2.f;
+        xi[h] = in ? X[i] : -1;
+    }
+    const double p_g = __ldcg(&p[g]);
+    const int cand_g = __ldcg(&cand[g]);
+    const float eta_g = u[g - 1];
     const bool bad = ld_volatile(&fl.bad[b]) != 0;
-    int tau = -1;
-    if (!bad) {
-        tau = 0;
-        // h_gamma = p_gamma; h_i = S_i / (S_i + 1 - p_i); tau = max{i : eta_i <= h_i}
-        for (int i = g; i >= 1; --i) {
-            const double pi = __ldcg(&p[i]);
-            double h = pi;
-            if (i < g) h = f_weight(pi, __ldcg(&S[i]));
-            if (h > 0.0 && static_cast<double>(u[i - 1]) <= h) { tau = i; break; }
-        }
+    // h_gamma = p_gamma; h_i = S_i / (S_i + 1 - p_i); tau = max{i >= 1 : h_i > 0 and eta_i <= h_i}, else 0
+    double hw[2];
+    bool pass[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int i = lane + 32 * h;
+        hw[h] = i == 0 ? 1.0 : f_weight(pi[h], Si[h]);
+        pass[h] = i >= 1 && i < g && hw[h] > 0.0 && static_cast<double>(eta[h]) <= hw[h];
     }
-    for (int i = 0; i <= g; ++i) ot[i] = -1;
-    if (tau >= 0) {
-        for (int i = 0; i < tau; ++i) ot[i] = X[i];
-        ot[tau] = __ldcg(&cand[tau]);
-        prm.out_len[b] = tau + 1;
-    } else {
-        prm.out_len[b] = -1;
+    const unsigned m_lo = __ballot_sync(0xffffffffu, pass[0]), m_hi = __ballot_sync(0xffffffffu, pass[1]);
+    int tau = 0;
+    if (p_g > 0.0 && static_cast<double>(eta_g) <= p_g) tau = g;
+    else if (m_hi) tau = 32 + 31 - __clz(m_hi);
+    else if (m_lo) tau = 31 - __clz(m_lo);
+    if (bad) tau = -1;
+    int y = cand_g;                       // the candidate of position tau
+    if (tau >= 0 && tau < g) y = __shfl_sync(0xffffffffu, tau < 32 ? cd[0] : cd[1], tau & 31);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int i = lane + 32 * h;
+        if (i < g) ot[i] = i < tau ? xi[h] : (i == tau ? y : -1);
     }
-    if (prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d) {
+    if (lane == 0) {
+        ot[g] = tau == g ? y : -1;
+        prm.out_len[b] = tau >= 0 ? tau + 1 : -1;
+    }
+    if (f_all_positions(prm)) {
         const double ln2 = 0.693147180559945309417232;
-        for (int i = 0; i <= g; ++i) {
+        for (int i = lane; i <= g; i += 32) {
             const size_t o1 = static_cast<size_t>(b) * (g + 1) + i, o0 = static_cast<size_t>(b) * g + i;
-            const double pi = __ldcg(&p[i]);
-            const double Si = i < g ? __ldcg(&S[i]) : 0.0;
-            double h = (i == 0) ? 1.0 : (i == g ? pi : f_weight(pi, Si));
+            const double pv = i == g ? p_g : (i < 32 ? pi[0] : pi[1]);
+            const double Sv = i == g ? 0.0 : (i < 32 ? Si[0] : Si[1]);
+            const double h = (i == 0) ? 1.0 : (i == g ? pv : f_weight(pv, Sv));
             const RowZ z = load_rowz(&fl.rowZ[static_cast<size_t>(b) * (g + 1) + i]);
-            if (prm.out_p) prm.out_p[o1] = static_cast<float>(pi);
+            if (prm.out_p) prm.out_p[o1] = static_cast<float>(pv);
             if (prm.out_h) prm.out_h[o1] = static_cast<float>(h);
             if (prm.out_lse_t) prm.out_lse_t[o1] = static_cast<float>((static_cast<double>(z.MP) + log2(z.ZP)) * ln2);
-            if (i < g && prm.out_S) prm.out_S[o0] = static_cast<float>(Si);
+            if (i < g && prm.out_S) prm.out_S[o0] = static_cast<float>(Sv);
             if (i < g && prm.out_lse_d) prm.out_lse_d[o0] = static_cast<float>((static_cast<double>(z.MQ) + log2(z.ZQ)) * ln2);
         }
     }
     __threadfence();
-    atomicAdd(&fl.counters[kCtrBlocks], 1u);      // (CTAs leave when every block is finished)
+    __syncwarp();
+    if (lane == 0) atomicAdd(&fl.counters[kCtrBlocks], 1u);      // (CTAs leave when every block is finished)
 }
 
-// With diagnostic outputs every position is computed in full.
-__device__ __forceinline__ bool f_all_positions(const Params& prm) {
-    return prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
-}
 // Is the token of position gamma drawn from the first sweep of the last target row (bv_flow.cu)?
 __device__ __forceinline__ bool f_draws_in_sweep1(const Params& prm, int nch_late) {
     return !f_all_positions(prm) && nch_late <= 8;
 }
 
-// ---- which positions get a second sweep (one thread each) ----
-// Is position i the selected one, given p_i and (for 0 < i < gamma) S_i?  Position 0 is what
-// remains when no other is selected.  (Eq. "pacc_block": h_gamma = p_gamma, h_i = S_i / (S_i + 1 - p_i).)
-static __device__ bool f_position_selected(const Params& prm, const FlowScratch& fl, int b, int i) {
-    const int g = prm.gamma;
-    if (i == 0) return true;
-    const double pi = __ldcg(&fl.pchain[static_cast<size_t>(b) * (g + 2) + i]);
-    double h = pi;
-    if (i < g) h = f_weight(pi, __ldcg(&fl.S[static_cast<size_t>(b) * (g + 1) + i]));
-    return h > 0.0 && static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + i - 1]) <= h;
-}
-// A position on hold changes state exactly once, whoever gets there first (positions of one block
-// may complete side by side once several candidates are swept at a time): true if this call did it.
-static __device__ bool f_leave_hold(const FlowScratch& fl, size_t ci, unsigned to) {
-    return atomicCAS(&fl.rel[ci], kRelHold, to) == kRelHold;
-}
-static __device__ void f_start_second_sweep(const FlowScratch& fl, size_t ci) {
-    atomicExch(&fl.rel[ci], kRelSweep);
-    // the row joins the queue from which every CTA draws pieces; the entry itself says when it is
-    // written (the queue starts at zero), so the order of the two stores does not matter
-    __threadfence();
-    const unsigned slot = atomicAdd(&fl.counters[kCtrQueued], 1u);
-    atomicExch(&fl.s2q[slot], static_cast<unsigned>(ci) + 1u);
-}
-// The selected position is the highest candidate that passes its test, so the candidates are
-// swept from the top, one at a time: start the highest one on hold below `below`.  Once the
-// first-sweep tickets have run out the GPU is emptying and a block's chain of candidates, one
-// after the other, would only prolong the launch: then all of them are started at once (a lower
-// one that turns out not to be needed costs bandwidth nobody else wants).
-static __device__ void f_release_next(const Params& prm, const FlowScratch& fl, int b, int below) {
-    const int g = prm.gamma;
-    bool all = ld_volatile(&fl.counters[kCtrTicket]) >= fl.tier_t[fl.ntier];
-    if (all) {       // only a chain of three or more is worth the bandwidth of the ones not needed
-        int held = 0;
-        for (int c = below - 1; c >= 1; --c)
-            held += ld_volatile(&fl.rel[static_cast<size_t>(b) * (g + 1) + c]) == kRelHold;
-        all = held >= 3;
-    }
-    // (position 0, what remains when nothing else is selected, still waits for the others)
-    int started = 0;
-    for (int c = below - 1; c >= 0; --c) {
-        if (c == 0 && started > 0) break;
-        const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
-        if (ld_volatile(&fl.rel[ci]) != kRelHold || !f_leave_hold(fl, ci, kRelSweep)) continue;
-        f_start_second_sweep(fl, ci);
-        ++started;
-        if (!all) return;
-    }
-}
-// Position i has just been completed (S_i and its candidate token are in scratch).  If it passes
-// its test, tau >= i whatever the higher candidates do, and no lower position is wanted; if not,
-// the next lower candidate is started.  Returns the number of positions that are complete through
-// this call (itself included).
-static __device__ unsigned f_after_position(const Params& prm, const FlowScratch& fl, int b, int i) {
-    const int g = prm.gamma;
-    unsigned done = 1;
-    if (f_position_selected(prm, fl, b, i)) {
-        for (int c = i - 1; c >= 0; --c) {
-            const size_t ci = static_cast<size_t>(b) * (g + 1) + c;
-            if (ld_volatile(&fl.rel[ci]) != kRelHold || !f_leave_hold(fl, ci, kRelSkip)) continue;
-            if (c < g) fl.S[ci] = 0.0;
-            fl.cand[ci] = -1;
-            ++done;
-        }
-        __threadfence();
-    } else {
-        f_release_next(prm, fl, b, i);
-    }
-    return done;
-}
-
-// ---- second sweeps of a block that has just been folded: the positions in `mask` (bit c =
-// position c; mask_hi: position c + 32) are started together; they take consecutive places in the
-// queue from which every CTA draws pieces (one warp) ----
+// ---- second sweeps that start together: the positions in `mask` (bit c = position c; mask_hi:
+// position c + 32) take consecutive places in the queue from which every CTA draws pieces (one warp) ----
 static __device__ void f_queue_rows(const FlowScratch& fl, int b, int g, unsigned mask, unsigned mask_hi, int lane) {
     const int n_lo = __popc(mask), n = n_lo + __popc(mask_hi);
     if (n == 0) return;
@@ -339,6 +287,67 @@ static __device__ void f_queue_rows(const FlowScratch& fl, int b, int g, unsigne
         atomicExch(&fl.s2q[slot + __popc(mask & ((1u << lane) - 1u))], static_cast<unsigned>(b * (g + 1) + lane) + 1u);
     if (mask_hi >> lane & 1u)
         atomicExch(&fl.s2q[slot + n_lo + __popc(mask_hi & ((1u << lane) - 1u))], static_cast<unsigned>(b * (g + 1) + lane + 32) + 1u);
+}
+
+// Which of the candidates on hold (bit c = position c < 32, hold_hi: c + 32) are swept next.  The
+// selected position is the highest candidate that passes its test, so the candidates are swept from
+// the top, one at a time; position 0, what remains when no other is selected, only when it is alone.
+// Once the first-sweep tickets have run out the GPU is emptying and a block's chain of candidates,
+// one after the other, would only prolong the launch: then all of them are started at once (a lower
+// one that turns out not to be needed costs bandwidth nobody else wants).
+__device__ __forceinline__ void f_pick_next(unsigned hold_lo, unsigned hold_hi, bool tail, unsigned& s_lo, unsigned& s_hi) {
+    s_lo = 0; s_hi = 0;
+    const unsigned c_lo = hold_lo & ~1u;                     // candidates other than position 0
+    if ((c_lo | hold_hi) == 0u) s_lo = hold_lo & 1u;
+    else if (tail && __popc(c_lo) + __popc(hold_hi) >= 2) { s_lo = c_lo; s_hi = hold_hi; }
+    else if (hold_hi) s_hi = 1u << (31 - __clz(hold_hi));
+    else s_lo = 1u << (31 - __clz(c_lo));
+}
+
+// ---- position i of a block is complete: S_i and its candidate token are in scratch (one warp).
+// Without diagnostics: if it passes its test, tau >= i whatever the higher candidates do, and no lower
+// position is wanted; if not, the next lower candidate is started.  A position on hold changes
+// state exactly once, whoever gets there first (positions of one block may complete side by side
+// once several candidates are swept at a time).  The warp that completes a block's last position
+// ends the block. ----
+static __device__ void f_position_done(const Params& prm, const FlowScratch& fl, int b, int i, int lane) {
+    const int g = prm.gamma;
+    const size_t row0 = static_cast<size_t>(b) * (g + 1);
+    unsigned done = 1;
+    if (!f_all_positions(prm)) {
+        __threadfence();
+        // everything asked for in one go
+        unsigned rl[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int c = lane + 32 * h;
+            rl[h] = c < i && c < g ? ld_volatile(&fl.rel[row0 + c]) : 0u;
+        }
+        const double p_i = __ldcg(&fl.pchain[static_cast<size_t>(b) * (g + 2) + i]);
+        const double S_i = i < g ? __ldcg(&fl.S[row0 + i]) : 0.0;
+        const float eta_i = i >= 1 ? prm.uni[static_cast<size_t>(b) * (g + 2) + i - 1] : 0.f;
+        const bool tail = ld_volatile(&fl.counters[kCtrTicket]) >= fl.total_s1;
+        const double hw = i == g ? p_i : f_weight(p_i, S_i);
+        const bool selected = i == 0 || (hw > 0.0 && static_cast<double>(eta_i) <= hw);
+        const unsigned hold_lo = __ballot_sync(0xffffffffu, rl[0] == kRelHold), hold_hi = __ballot_sync(0xffffffffu, rl[1] == kRelHold);
+        unsigned s_lo = hold_lo, s_hi = hold_hi;             // selected: every lower candidate is dropped
+        if (!selected) f_pick_next(hold_lo, hold_hi, tail, s_lo, s_hi);
+        bool won[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int c = lane + 32 * h;
+            won[h] = ((h ? s_hi : s_lo) >> lane & 1u) && atomicCAS(&fl.rel[row0 + c], kRelHold, selected ? kRelSkip : kRelSweep) == kRelHold;
+            if (won[h] && selected) { fl.S[row0 + c] = 0.0; fl.cand[row0 + c] = -1; }
+        }
+        const unsigned w_lo = __ballot_sync(0xffffffffu, won[0]), w_hi = __ballot_sync(0xffffffffu, won[1]);
+        if (selected) done += static_cast<unsigned>(__popc(w_lo) + __popc(w_hi));
+        else { __threadfence(); f_queue_rows(fl, b, g, w_lo, w_hi, lane); }
+    }
+    __threadfence();
+    unsigned n = 0;
+    if (lane == 0) n = atomicAdd(&fl.cand_cnt[b], done);
+    n = __shfl_sync(0xffffffffu, n, 0);
+    if (n + done == static_cast<unsigned>(g) + 1u) f_finalize_block(prm, fl, b, lane);
 }
 
 // ---- all rows 0 .. gamma-1 of a block have their normalisers: the prefix recursion
@@ -363,7 +372,7 @@ __device__ void f_fold_block(const Params& prm, const FlowScratch& fl, const Flo
         eta[h] = (c >= 1 && c < g) ? u[c - 1] : 0.f;
     }
     const float eta_g = u[g - 1];
-    const bool tail = ld_volatile(&fl.counters[kCtrTicket]) >= fl.tier_t[fl.ntier];
+    const bool tail = ld_volatile(&fl.counters[kCtrTicket]) >= fl.total_s1;
     // the recursion, by every lane alike; a lane keeps the p of its own positions
     double pc = 1.0, mine[2] = {1.0, 1.0};
     for (int c = 0; c < g; ++c) {
@@ -410,13 +419,7 @@ __device__ void f_fold_block(const Params& prm, const FlowScratch& fl, const Flo
     // turns out not to be needed costs bandwidth nobody else wants).
     unsigned s_lo = 0, s_hi = 0;
     if (all_positions) { s_lo = m_lo; s_hi = m_hi; }
-    else if (!last_row_wanted) {
-        const unsigned c_lo = m_lo & ~1u;                    // candidates other than position 0
-        if ((c_lo | m_hi) == 0u) s_lo = 1u;
-        else if (tail && __popc(c_lo) + __popc(m_hi) >= 2) { s_lo = c_lo; s_hi = m_hi; }
-        else if (m_hi) s_hi = 1u << (31 - __clz(m_hi));
-        else s_lo = 1u << (31 - __clz(c_lo));
-    }
+    else if (!last_row_wanted) f_pick_next(m_lo, m_hi, tail, s_lo, s_hi);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int c = lane + 32 * h;
@@ -447,11 +450,11 @@ template <int DT>
 __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int r, int lane) {
     const int g = cx.g;
     const size_t rowi = static_cast<size_t>(b) * (g + 1) + r;
-    const int nch = f_nch_row(fl, b, r, g);
+    const int nch = f_nch_row(fl, r, g);
     const bool have_q = r < g;
     // loads in flight together: the chunks' sums, the drafted token
     RowZ z; z.MP = kNoRef; z.ZP = 0.0; z.MQ = kNoRef; z.ZQ = 0.0;
-    if (lane < nch) z = load_rowz(&fl.part[rowi * cx.nch + lane]);
+    if (lane < nch) z = load_rowz(&fl.part[rowi * fl.part_stride + lane]);
     int x = (lane == 31 && have_q) ? prm.tok[static_cast<size_t>(b) * g + r] : 0;
     x = __shfl_sync(0xffffffffu, x, 31);
     const bool xok = have_q && x >= 0 && x < cx.V;
@@ -494,89 +497,61 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
 }
 
 // ---- a position is complete (one warp): S_r from the segment totals, and the candidate Y_r.
-// `segs` holds the nseg totals of the row's segments in index order; range(s, v0, v1) gives the
-// vectors [v0, v1) of segment s. ----
+// `segs` holds the nseg <= 128 totals of the row's segments in index order (four per lane);
+// range(s, v0, v1) gives the vectors [v0, v1) of segment s. ----
 template <int DT, class RangeFn>
 __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, bool have_q,
                                     const char* rowP, const char* rowQ, float cp, float nMP, float nMQ,
                                     int nseg, const float* segs, int lane, RangeFn range) {
     constexpr int EPV = Raw<DT>::EPV;
     const int g = cx.g, r = ri % (g + 1), b = ri / (g + 1);
-    // ---------------- the position is complete: S_r and the candidate Y_r ----------------
     __threadfence();
+    // everything asked for in one go: the uniform, the segment totals, the draft row's normaliser
     const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
-    // Segment totals in index order, 128 at a time (4 per lane); `carry` is the fp32 running total
-    // of the groups before.  First pass: S_r in fp64 and the fp32 total; second pass: the segment
-    // that holds the sample, found with the very same fp32 prefix sums.
-    const int ngrp = (nseg + 127) >> 7;
-    double sd = 0.0;
-    float total = 0.f;
-    for (int grp = 0; grp < ngrp; ++grp) {
-        float w[4];
+    float w[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int i = 128 * grp + 4 * lane + j;
-            w[j] = i < nseg ? __ldcg(&segs[i]) : 0.f;
-        }
-        sd += (static_cast<double>(w[0]) + static_cast<double>(w[1])) +
-              (static_cast<double>(w[2]) + static_cast<double>(w[3]));
-        float inc = ((w[0] + w[1]) + w[2]) + w[3];
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const float o = __shfl_up_sync(0xffffffffu, inc, off);
-            if (lane >= off) inc += o;
-        }
-        total += __shfl_sync(0xffffffffu, inc, 31);
+    for (int j = 0; j < 4; ++j) {
+        const int i = 4 * lane + j;
+        w[j] = i < nseg ? __ldcg(&segs[i]) : 0.f;
     }
+    const double ZQ = have_q ? __ldcg(&fl.rowZ[ri].ZQ) : 1.0;
+    // S_r in fp64; the segment that holds the sample by fp32 prefix sums in index order
+    double sd = (static_cast<double>(w[0]) + static_cast<double>(w[1])) + (static_cast<double>(w[2]) + static_cast<double>(w[3]));
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
-    if (lane == 0 && have_q) fl.S[ri] = sd / __ldcg(&fl.rowZ[ri].ZQ);
+    if (lane == 0 && have_q) fl.S[ri] = sd / ZQ;
+    const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
+    float inc = l4;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float o = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += o;
+    }
+    const float total = __shfl_sync(0xffffffffu, inc, 31);
     int found = -1;
     if (total > 0.f) {
         const float t = uf * total;
-        float carry = 0.f;
-        int sel = -1, last_nz = -1;
-        float before = 0.f, last_before = 0.f;
-        for (int grp = 0; grp < ngrp && sel < 0; ++grp) {
-            float w[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int i = 128 * grp + 4 * lane + j;
-                w[j] = i < nseg ? __ldcg(&segs[i]) : 0.f;
-            }
-            const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
-            float inc = l4;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const float o = __shfl_up_sync(0xffffffffu, inc, off);
-                if (lane >= off) inc += o;
-            }
-            float exc = __shfl_up_sync(0xffffffffu, inc, 1);
-            if (lane == 0) exc = 0.f;
-            const float p0 = carry + exc, p1 = carry + (exc + l1), p2 = carry + (exc + l2);
-            const float p3 = carry + (exc + l3), p4 = carry + (exc + l4);
-            // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
-            const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
-            const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
-            const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
-            const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
-            if (hit) {
-                const int src = __ffs(hit) - 1;
-                int e = 3; float bef = p3;
-                if (h1) { e = 0; bef = p0; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
-                sel = __shfl_sync(0xffffffffu, 128 * grp + 4 * lane + e, src);
-                before = __shfl_sync(0xffffffffu, bef, src);
-            } else if (nz) {
-                const int src = 31 - __clz(nz);
-                int e = 0; float bef = p0;
-                if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
-                else if (w[1] > 0.f) { e = 1; bef = p1; }
-                last_nz = __shfl_sync(0xffffffffu, 128 * grp + 4 * lane + e, src);
-                last_before = __shfl_sync(0xffffffffu, bef, src);
-            }
-            carry += __shfl_sync(0xffffffffu, inc, 31);
+        float exc = __shfl_up_sync(0xffffffffu, inc, 1);
+        if (lane == 0) exc = 0.f;
+        const float p0 = exc, p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+        // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
+        const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
+        const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
+        const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
+        const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
+        int e = 3, src;
+        float bef = p3;
+        if (hit) {
+            src = __ffs(hit) - 1;
+            if (h1) { e = 0; bef = p0; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
+        } else {
+            src = 31 - __clz(nz);
+            e = 0; bef = p0;
+            if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
+            else if (w[1] > 0.f) { e = 1; bef = p1; }
         }
-        if (sel < 0) { sel = last_nz; before = last_before; }
+        const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
+        const float before = __shfl_sync(0xffffffffu, bef, src);
         int s0, s1;
         range(sel, s0, s1);
         found = f_rescan<DT>(rowP, rowQ, s0, s1, lane, cx.kf, cp, nMP, nMQ, t - before);
@@ -592,17 +567,9 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
         tot = warp_sum(tot);
         found = f_rescan<DT>(rowP, nullptr, 0, cx.units, lane, cx.kf, 1.f, nMP, nMQ, uf * tot);
     }
-    if (lane == 0) {
-        fl.cand[ri] = found;
-        __threadfence();
-        const bool all_positions = prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d;
-        const unsigned done = all_positions ? 1u : f_after_position(prm, fl, b, r);
-        if (atomicAdd(&fl.cand_cnt[b], done) + done == static_cast<unsigned>(g) + 1u) {
-            __threadfence();
-            f_finalize_block(prm, fl, b);
-        }
-    }
+    if (lane == 0) fl.cand[ri] = found;
     __syncwarp();
+    f_position_done(prm, fl, b, r, lane);
 }
 
 }  // namespace bv

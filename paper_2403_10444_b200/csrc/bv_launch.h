@@ -24,7 +24,6 @@ cudaError_t launch_cluster(const Params& prm, int algo, int dtype, int cluster, 
 // counters in a scratch area of flow_scratch_bytes(); its first *zero_bytes must be zero
 // when the kernel starts.
 struct RowZ { double MP, ZP, MQ, ZQ; };   // row (or chunk) references and sums of 2^{z k - M}
-constexpr int kFlowTiers = 4;
 struct FlowScratch {
     unsigned* counters;   // ticket counter of the sweep-1 items, rows queued for their second sweep, pieces of
                           // queued rows handed out, blocks finished (one 128-byte line each)
@@ -36,7 +35,7 @@ struct FlowScratch {
     unsigned* rel;        // [B (gamma+1)] what becomes of the position's second sweep (0 until the block is folded)
     unsigned* s2q;        // [B (gamma+1)] queue of rows whose second sweep has been started (row index + 1)
     unsigned* lq;         // [B] queue of last target rows whose first sweep has been asked for (row index + 1)
-    RowZ* part;           // [B (gamma+1) nch]
+    RowZ* part;           // [B (gamma+1) part_stride]
     RowZ* rowZ;           // [B (gamma+1)]
     double* pchain;       // [B (gamma+2)]
     float* cscale;        // [B (gamma+1)] p_r Z_Q / Z_P
@@ -45,31 +44,23 @@ struct FlowScratch {
     float* seg_tot;       // [B (gamma+1) segs]
     double* S;            // [B (gamma+1)]
     int* cand;            // [B (gamma+1)]
-    // Chunks per row in the first sweep, by block: blocks tier_b[k] .. tier_b[k+1]-1 are cut into
-    // tier_n[k] chunks per row and own the tickets tier_t[k] .. tier_t[k+1]-1.  The last blocks of a
-    // launch are cut finer, so that the CTAs run out of first-sweep work at nearly the same time.
-    int ntier;
-    int tier_b[kFlowTiers + 1];
-    unsigned tier_t[kFlowTiers + 1];
-    int tier_n[kFlowTiers];
-    int nch;              // the largest chunk count of any row (stride of `part`)
+    int nch;              // chunks per row in the first sweep of rows 0 .. gamma-1 (1 .. kFlowMaxChunks)
+    int part_stride;      // chunk results kept per row: max(nch, nch_late)
     int nch_late;         // chunks of a last target row, whose first sweep is asked for on demand
     int np;               // pieces per row in the second sweep (1 .. kFlowMaxChunks)
+    unsigned total_s1;    // first-sweep tickets: B gamma nch
     int depth;            // flow kernel: descriptors a CTA may have handed to its workers and not yet seen swept
-    int stretch;          // vectors per row of one stretch of a first-sweep chunk
     int segs;             // residual totals kept per row
 };
 constexpr int kFlowMaxChunks = 32;
-// How a launch is cut into work items: filled by flow_plan, completed by flow_scratch_layout.
+// How a launch is cut into work items (flow_plan): chunks per row in the first sweep, chunks of a
+// last target row (swept on demand), pieces per row in the second sweep.
 struct FlowPlan {
-    int ntier;
-    int tier_b[kFlowTiers + 1];
-    int tier_n[kFlowTiers];
-    int nch_late, np;
-    int nch_max() const { int m = nch_late; for (int k = 0; k < ntier; ++k) m = tier_n[k] > m ? tier_n[k] : m; return m; }
+    int nch, nch_late, np;
+    int part_stride() const { return nch > nch_late ? nch : nch_late; }
 };
 // units: 16-byte vectors per row; pair_items: false when the first sweep streams one row per item
-// (supplied draft normalisers); chunks / pieces > 0 force one chunk count for every block / the piece count.
+// (supplied draft normalisers); chunks / pieces > 0 force the chunk count / the piece count.
 FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces);
 size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_bytes);
 void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, FlowScratch* fl);

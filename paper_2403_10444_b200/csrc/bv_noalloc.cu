@@ -105,7 +105,7 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     prm.kf = static_cast<float>(kd);
     prm.out_tokens = ot; prm.out_len = ol;
     prm.status = reinterpret_cast<int*>(status_word);
-    long long items = static_cast<long long>(fl.tier_t[fl.ntier]);
+    long long items = static_cast<long long>(fl.total_s1);
     long long nctas = static_cast<long long>(d.sm_count) * per_sm;
     if (nctas > items) nctas = items;
     if (bv::launch_flow(prm, fl, dtype, static_cast<int>(nctas), s) != cudaSuccess) return BV_ERR_CUDA;
