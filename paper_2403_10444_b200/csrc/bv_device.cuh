@@ -324,6 +324,10 @@ __device__ __forceinline__ void ring_fetch_hint(uint32_t saddr, const void* src,
         "@!p st.shared.v4.b32 [%0], {%3, %3, %3, %3};\n\t}"
         ::"r"(saddr), "l"(src), "r"(static_cast<int>(pred)), "r"(fill), "l"(pol) : "memory");
 }
+// 16-byte asynchronous copy with an L2 policy, shared-space destination address
+__device__ __forceinline__ void cp_async16_hint(uint32_t saddr, const void* gmem, uint64_t pol) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(saddr), "l"(gmem), "l"(pol) : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t saddr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr) : "memory");

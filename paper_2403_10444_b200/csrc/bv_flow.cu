@@ -504,6 +504,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     const char* iB = nullptr;
     int i_rem = 0;                    // vectors of the current segment not yet asked for
     int i_adv = 32;                   // vectors a step covers: 32 of each row, or 64 of the one row
+    uint32_t i_adv16 = 512;           // the same in bytes
     int n_i = 0;                      // items the issue cursor has started
     bool i_stalled = false;
     uint32_t rp = sb;                 // ring slot to consume next, and to refill right afterwards
@@ -514,11 +515,21 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         const bool single = sh.desc[slot].have_q == 0;
         i_rem = w1 - w0;
         i_adv = single ? 64 : 32;
+        i_adv16 = single ? 1024u : 512u;
         iA = sh.desc[slot].rowP + static_cast<size_t>(w0 + lane) * 16;
         iB = single ? iA + 512 : sh.desc[slot].rowQ + static_cast<size_t>(w0 + lane) * 16;
     };
     // one ring step of the issue cursor into the slot at `slot_addr`
     auto issue_step = [&](uint32_t slot_addr) {
+        if (i_rem >= i_adv) {                                // a full step: every lane has its two vectors
+            cp_async16_hint(slot_addr, iA, pol);
+            cp_async16_hint(slot_addr + kCell, iB, pol);
+            cp_async_commit();
+            i_rem -= i_adv;
+            iA += i_adv16;
+            iB += i_adv16;
+            return;
+        }
         if (i_rem <= 0 && !i_stalled) {
             for (;;) {                                       // the next item with something for this warp
                 const int slot = n_i % kFDesc;
@@ -529,12 +540,17 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 if (i_rem > 0) break;
             }
         }
-        if (i_rem > 0) {
+        if (i_rem >= i_adv) {
+            cp_async16_hint(slot_addr, iA, pol);
+            cp_async16_hint(slot_addr + kCell, iB, pol);
+        } else if (i_rem > 0) {                              // the short last step of a segment
             ring_fetch_hint(slot_addr, iA, lane < i_rem, R::kNegInf, pol);
             ring_fetch_hint(slot_addr + kCell, iB, lane + (i_adv - 32) < i_rem, R::kNegInf, pol);
+        }
+        if (i_rem > 0) {
             i_rem -= i_adv;
-            iA += static_cast<size_t>(i_adv) * 16;
-            iB += static_cast<size_t>(i_adv) * 16;
+            iA += i_adv16;
+            iB += i_adv16;
         }
         cp_async_commit();
     };
@@ -561,7 +577,6 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         warp_range(sh.desc[slot].u0, sh.desc[slot].u1, warp, w0, w1);
         int c_left = have_q ? (w1 - w0 + 31) >> 5 : (w1 - w0 + 63) >> 6;
         float MPw = kNoRef, sP = 0.f, MQw = kNoRef, sQ = 0.f;
-        bool first = true;
         // the steps of this item; the oldest step in flight is always the next one of this item
         auto run_steps = [&](auto&& body) {
             for (; c_left > 0; --c_left) {
@@ -576,18 +591,24 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             }
         };
         if (kind == kSweep1) {
+            if (c_left > 0) {                                // references from the first vector of every lane
+                cp_async_wait<kFSlots - 1>();
+                float va[EPV], vb[EPV];
+                R::unpack(lds128(rp), va);
+                R::unpack(lds128(rp + kCell), vb);
+                if (have_q) {
+                    MPw = fmaxf(rintf(warp_max(vec_max<EPV>(va)) * kf), kNoRef);
+                    MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vb)) * kf), kNoRef);
+                } else {
+                    MPw = fmaxf(rintf(warp_max(fmaxf(vec_max<EPV>(va), vec_max<EPV>(vb))) * kf), kNoRef);
+                }
+            }
             if (have_q) {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
-                    if (first) {                             // references from the first vector of every lane
-                        MPw = fmaxf(rintf(warp_max(vec_max<EPV>(va)) * kf), kNoRef);
-                        MQw = fmaxf(rintf(warp_max(vec_max<EPV>(vb)) * kf), kNoRef);
-                        first = false;
-                    }
                     f_step_sweep1_pair<EPV>(va, vb, kf, MPw, sP, MQw, sQ);
                 });
             } else {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
-                    if (first) { MPw = fmaxf(rintf(warp_max(fmaxf(vec_max<EPV>(va), vec_max<EPV>(vb))) * kf), kNoRef); first = false; }
                     f_step_sweep1_single<EPV>(va, vb, kf, MPw, sP);
                 });
             }
