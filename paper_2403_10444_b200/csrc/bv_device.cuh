@@ -240,10 +240,12 @@ template <> struct Raw<kBF16> {
     static constexpr int EPV = 8;
     static constexpr uint32_t kNegInf = 0xff80ff80u;
     static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[8]) {
-        v[0] = __uint_as_float(r.x << 16); v[1] = __uint_as_float(r.x & 0xffff0000u);
-        v[2] = __uint_as_float(r.y << 16); v[3] = __uint_as_float(r.y & 0xffff0000u);
-        v[4] = __uint_as_float(r.z << 16); v[5] = __uint_as_float(r.z & 0xffff0000u);
-        v[6] = __uint_as_float(r.w << 16); v[7] = __uint_as_float(r.w & 0xffff0000u);
+        // (the low half by a byte permute: like the mask of the high half it runs on the integer
+        // pipe, where a shift would share the pipe of the multiply-adds)
+        v[0] = __uint_as_float(__byte_perm(r.x, 0, 0x1044)); v[1] = __uint_as_float(r.x & 0xffff0000u);
+        v[2] = __uint_as_float(__byte_perm(r.y, 0, 0x1044)); v[3] = __uint_as_float(r.y & 0xffff0000u);
+        v[4] = __uint_as_float(__byte_perm(r.z, 0, 0x1044)); v[5] = __uint_as_float(r.z & 0xffff0000u);
+        v[6] = __uint_as_float(__byte_perm(r.w, 0, 0x1044)); v[7] = __uint_as_float(r.w & 0xffff0000u);
     }
 };
 template <> struct Raw<kF32> {

@@ -472,7 +472,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 ld_volatile(&fl.counters[kCtrBlocks]) >= static_cast<unsigned>(cx.B)) break;
             // the next item waits for a row that another CTA completes (all idle CTAs look at the same
             // counters: wait long enough not to crowd those who work)
-            __nanosleep(idle < 4 ? 500 : 2000);
+            __nanosleep(exhausted || idle < 4 ? 500 : 2000);
             poll();
             if (++idle > (1u << 21)) { if (prm.status) atomicExch(prm.status, 1); failed = true; break; }
         }
@@ -716,11 +716,11 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
 //   pieces of about 4000 vectors that many CTAs share.
 FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces) {
     FlowPlan pl{};
-    long long np = units / 4000;
+    long long np = units / 3500;
     if (np < 1) np = 1;
-    if (np > 8) np = 8;
+    if (np > 128 / kFWarps) np = 128 / kFWarps;             // (a position's segment totals are looked at four per lane)
     pl.np = pieces > 0 ? pieces : static_cast<int>(np);
-    pl.nch_late = static_cast<int>(np);
+    pl.nch_late = static_cast<int>(np > 8 ? 8 : np);
     const long long row_units = pair_items ? units : units / 2;   // (a single-row item streams half as much)
     long long nch = (row_units + 8000) / 16000;
     if (nch < 1) nch = 1;

@@ -291,15 +291,14 @@ static __device__ void f_queue_rows(const FlowScratch& fl, int b, int g, unsigne
 
 // Which of the candidates on hold (bit c = position c < 32, hold_hi: c + 32) are swept next.  The
 // selected position is the highest candidate that passes its test, so the candidates are swept from
-// the top, one at a time; position 0, what remains when no other is selected, only when it is alone.
-// Once the first-sweep tickets have run out the GPU is emptying and a block's chain of candidates,
-// one after the other, would only prolong the launch: then all of them are started at once (a lower
-// one that turns out not to be needed costs bandwidth nobody else wants).
+// the top, one at a time; position 0, what remains when no other is selected, last.  Once the
+// first-sweep tickets have run out the GPU is emptying and a block's chain of candidates, one after
+// the other, would only prolong the launch: then all of them are started at once, position 0
+// included (one that turns out not to be needed costs bandwidth nobody else wants).
 __device__ __forceinline__ void f_pick_next(unsigned hold_lo, unsigned hold_hi, bool tail, unsigned& s_lo, unsigned& s_hi) {
     s_lo = 0; s_hi = 0;
     const unsigned c_lo = hold_lo & ~1u;                     // candidates other than position 0
-    if ((c_lo | hold_hi) == 0u) s_lo = hold_lo & 1u;
-    else if (tail && __popc(c_lo) + __popc(hold_hi) >= 2) { s_lo = c_lo; s_hi = hold_hi; }
+    if (tail || (c_lo | hold_hi) == 0u) { s_lo = hold_lo; s_hi = hold_hi; }
     else if (hold_hi) s_hi = 1u << (31 - __clz(hold_hi));
     else s_lo = 1u << (31 - __clz(c_lo));
 }
