@@ -29,6 +29,7 @@ struct DeviceState {
     // do not share counters (more than kFlowSlots overlapping calls on one device would)
     void* flow_ws[4] = {};
     size_t flow_bytes[4] = {};
+    size_t flow_clean[4] = {};        // leading bytes of each area known to be zero between calls
     unsigned long long flow_calls = 0;
     int flow_ctas_per_sm[2] = {};
     // staging for the host-buffer entry points
@@ -176,6 +177,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
                 if (d->flow_ws[slot]) cudaFree(d->flow_ws[slot]);
                 d->flow_ws[slot] = nullptr;
                 d->flow_bytes[slot] = 0;
+                d->flow_clean[slot] = 0;
                 cudaError_t e = cudaMalloc(&d->flow_ws[slot], need);
                 if (e != cudaSuccess) return cuda_fail(e);
                 d->flow_bytes[slot] = need;
@@ -186,8 +188,14 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
                 const int v = std::atoi(env);
                 if (v >= 2 && v <= 6) fl.depth = v;
             }
-            cudaError_t e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
-            if (e != cudaSuccess) return cuda_fail(e);
+            // The kernel leaves its counters and flags at zero when it ends, so they are cleared here only
+            // when the area is new or a larger problem needs more of them than the last launch left clean.
+            cudaError_t e = cudaSuccess;
+            if (d->flow_clean[slot] < zero_bytes) {
+                e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
+                if (e != cudaSuccess) return cuda_fail(e);
+            }
+            d->flow_clean[slot] = zero_bytes;
             long long items = static_cast<long long>(fl.total_s1);
             if (nctas > items) nctas = items;
             prm.ticket = nullptr;

@@ -482,6 +482,30 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             FlowDesc d; d.kind = kExit;
             publish(d, q + j);
         }
+        // The counters and flags must be zero when the next launch starts.  Every block is finished,
+        // so nobody needs the flags any more: each CTA clears its share of them on its way out.  The
+        // global counters are still read by CTAs that have yet to see that all blocks are finished;
+        // the last CTA to leave clears those (and everything, if a wait gave up somewhere and the
+        // others may have written after their shares were cleared).
+        {
+            unsigned* z = fl.counters;
+            const unsigned words = fl.zero_words - kCounterWords;
+            const unsigned per = (words + gridDim.x - 1) / gridDim.x;
+            const unsigned w0 = kCounterWords + blockIdx.x * per;
+            const unsigned w1 = min(w0 + per, fl.zero_words);
+            for (unsigned i = w0 + lane; i < w1; i += 32) z[i] = 0u;
+            __threadfence();
+            __syncwarp();
+            unsigned left = 0;
+            if (lane == 0) left = atomicAdd(&fl.counters[kCtrExited], 1u);
+            left = __shfl_sync(0xffffffffu, left, 0);
+            if (left == gridDim.x - 1) {
+                __threadfence();
+                if (prm.status && *reinterpret_cast<volatile int*>(prm.status) != 0)
+                    for (unsigned i = kCounterWords + lane; i < fl.zero_words; i += 32) z[i] = 0u;
+                for (unsigned i = lane; i < kCounterWords; i += 32) z[i] = 0u;
+            }
+        }
         return;
     }
 
@@ -703,6 +727,9 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->nch_late = plan.nch_late;
     fl->np = plan.np;
     fl->depth = 3;
+    size_t zb = 0;
+    flow_scratch_bytes(B, gamma, plan, &zb);
+    fl->zero_words = static_cast<unsigned>(zb / sizeof(unsigned));
     fl->segs = static_cast<int>(segs);
 }
 

@@ -15,8 +15,9 @@ enum : int { kExit = 0, kSweep1 = 1, kSweep2 = 2 };
 // Global counters, one per 128-byte line so that polling one does not slow the others down:
 // the sweep-1 ticket counter, rows queued for their second sweep, pieces of queued rows handed
 // out, blocks finished, last target rows queued for their first sweep, chunks of those handed out.
-constexpr int kCounterWords = 192;
-enum : int { kCtrTicket = 0, kCtrQueued = 32, kCtrPieces = 64, kCtrBlocks = 96, kCtrLateQueued = 128, kCtrLateChunks = 160 };
+// (and the number of CTAs that have left, by which the last one knows itself)
+constexpr int kCounterWords = 224;
+enum : int { kCtrTicket = 0, kCtrQueued = 32, kCtrPieces = 64, kCtrBlocks = 96, kCtrLateQueued = 128, kCtrLateChunks = 160, kCtrExited = 192 };
 // rel[row]: 0 = not folded yet, then whether the row's second sweep is wanted
 enum : unsigned { kRelSweep = 1u, kRelSkip = 2u, kRelHold = 3u, kRelLate = 4u };   // hold: wanted only if every higher
 // candidate is rejected; late: the last target row, whose first sweep has only now been asked for
@@ -418,7 +419,7 @@ __device__ void f_fold_block(const Params& prm, const FlowScratch& fl, const Flo
     // turns out not to be needed costs bandwidth nobody else wants).
     unsigned s_lo = 0, s_hi = 0;
     if (all_positions) { s_lo = m_lo; s_hi = m_hi; }
-    else if (!last_row_wanted) f_pick_next(m_lo, m_hi, tail, s_lo, s_hi);
+    else if (tail || !last_row_wanted) f_pick_next(m_lo, m_hi, tail, s_lo, s_hi);   // (emptying GPU: alongside the last target row)
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int c = lane + 32 * h;

@@ -22,7 +22,7 @@ cudaError_t launch_cluster(const Params& prm, int algo, int dtype, int cluster, 
 
 // Flow kernel (Block Verification, 128-bit path): independent work items with dependency
 // counters in a scratch area of flow_scratch_bytes(); its first *zero_bytes must be zero
-// when the kernel starts.
+// when the kernel starts, and the kernel leaves them zero when it ends.
 struct RowZ { double MP, ZP, MQ, ZQ; };   // row (or chunk) references and sums of 2^{z k - M}
 struct FlowScratch {
     unsigned* counters;   // ticket counter of the sweep-1 items, rows queued for their second sweep, pieces of
@@ -49,6 +49,7 @@ struct FlowScratch {
     int nch_late;         // chunks of a last target row, whose first sweep is asked for on demand
     int np;               // pieces per row in the second sweep (1 .. kFlowMaxChunks)
     unsigned total_s1;    // first-sweep tickets: B gamma nch
+    unsigned zero_words;  // 32-bit words at the start of the scratch area (from `counters` on) that start and end at zero
     int depth;            // flow kernel: descriptors a CTA may have handed to its workers and not yet seen swept
     int segs;             // residual totals kept per row
 };
