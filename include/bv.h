@@ -23,6 +23,12 @@
  * Ownership: the caller owns every buffer; inputs are never written.  The
  * device entry points enqueue work on `stream` and return without
  * synchronising; buffers must stay valid until that work has completed.
+ * The library keeps one workspace per stream (up to 32 streams per device, the
+ * least recently used one is recycled beyond that): calls on one stream run in
+ * order and share it, calls on different streams never do.  A workspace is
+ * obtained and grown with cudaMallocAsync / cudaFreeAsync on that stream, so a
+ * first or larger call allocates but does not synchronise the device; the
+ * memory is returned by bv_release().  B = 0 is accepted and does nothing.
  *
  * Errors: every entry point returns BV_OK (0) or a negative bv_status; nothing
  * is launched when an argument is rejected.  Data faults are per sequence: a
@@ -45,8 +51,9 @@ typedef enum bv_status {
                                  unknown dtype, pointer not aligned to its element size */
     BV_ERR_UNSUPPORTED = -2,  /* gamma > BV_MAX_GAMMA, or no sm_100 device              */
     BV_ERR_CUDA = -3,         /* a CUDA runtime call failed; see bv_last_cuda_error()   */
-    BV_ERR_TIMEOUT = -4,      /* a bounded device-side wait gave up (reported by the
-                                 host-buffer entry points, which synchronise)           */
+    BV_ERR_TIMEOUT = -4,      /* a bounded device-side wait gave up: reported by the
+                                 host-buffer entry points and by bv_stream_status(),
+                                 which synchronise; outputs of that call are invalid   */
     BV_ERR_TOO_LARGE = -5     /* bv_verify_noalloc: B, gamma, V need more scratch than
                                  BV_NOALLOC_SCRATCH_BYTES                               */
 } bv_status;
@@ -153,7 +160,9 @@ int tv_verify_host(const void* target_logits, const void* draft_logits,
  *     device; make that first call before any stream capture begins;
  *   - every call on a device uses the same array, which keeps the previous call's contents
  *     (the entry point clears the part that must start at zero, on `stream`).  Two calls
- *     that overlap on the GPU, on different streams, race on it: order them yourself.
+ *     that overlap on the GPU, on different streams, race on it: order them yourself;
+ *   - a device-side wait that gives up is not reported (bv_stream_status() does not see this
+ *     entry point's calls); the outputs of such a call are left unwritten.
  */
 int bv_verify_noalloc(const void* target_logits, const void* draft_logits,
                       const int32_t* draft_tokens, const float* uniforms,
@@ -220,8 +229,8 @@ int gbv_verify_ex(const void* target_logits, const void* draft_logits,
                   float* out_lse_t, float* out_lse_d, void* stream);
 
 /*
- * The drafting step of Algorithm 3 ("Sample X_1, ..., X_gamma ~ M_s using autoregressive sampling,
- * keep the conditional probabilities at each step") for `rows` rows of draft logits [rows, V]:
+ * The drafting step of Algorithm 3 (its first step: one token per draft distribution, the
+ * distribution's normaliser kept for the verification) for `rows` rows of draft logits [rows, V]:
  *   out_tokens[r] ~ softmax(logits[r, :] / temperature), drawn by inverse CDF in vocabulary-index
  *                   order with uniforms[r] in [0, 1): min{k : C_k > u W} over the running sums C_k of
  *                   the weights, the convention of the verification samples;
@@ -234,7 +243,31 @@ int gbv_verify_ex(const void* target_logits, const void* draft_logits,
 int bv_sample_draft(const void* logits, const float* uniforms, int rows, int V, int dtype,
                     float temperature, int32_t* out_tokens, float* out_lse, void* stream);
 
-/* Frees the library's cached device buffers on the current device. */
+/*
+ * Waits for `stream` and reports whether a device-side wait of any call enqueued on it since the
+ * last query gave up: BV_ERR_TIMEOUT (the outputs of those calls are not to be used; the library's
+ * state is intact and later calls work) or BV_OK.  Every device-side wait of this library is
+ * bounded, so a protocol error ends a kernel instead of hanging the GPU; this call is how a user
+ * of the device entry points learns of it.  The host-buffer entry points do the same themselves.
+ */
+int bv_stream_status(void* stream);
+
+/*
+ * Tuning and test options, process-wide, read by every later call (0 restores the default choice):
+ *   "kernel"        1 flow, 2 cluster, 3 element-wise streaming kernel for Block Verification
+ *   "cluster"       cluster width of the cluster / streaming kernels (1, 2, 4, 8)
+ *   "max_clusters"  cap on the clusters those kernels launch
+ *   "flow_chunks", "flow_pieces", "flow_ctas", "flow_depth"   work-item shape of the flow kernel
+ *   "wait_limit"    polls after which a bounded device-side wait gives up (tests)
+ *   "never_signal"  tests: the flow kernel's workers never report an item as swept, so its waits
+ *                   run out and the call ends with BV_ERR_TIMEOUT
+ * Their first values come from the environment variables BV_KERNEL (flow / cluster / stream),
+ * BV_CLUSTER, BV_MAX_CLUSTERS, BV_FLOW_CHUNKS, BV_FLOW_PIECES, BV_FLOW_CTAS, BV_FLOW_DEPTH, read once.
+ * Returns BV_ERR_INVALID_ARG for an unknown name.
+ */
+int bv_set_option(const char* name, int value);
+
+/* Frees the library's cached device buffers on the current device (waits for the device). */
 int bv_release(void);
 
 /* Number of kernel launches the last device-path call on this thread enqueued. */

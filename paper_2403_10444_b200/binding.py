@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_sample_draft", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_sample_draft", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -59,6 +59,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.bv_verify_lse_ex.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp, vp, vp, vp, vp, vp]
     for name in EXPORTS:
         getattr(lib, name).restype = ci
+    lib.bv_stream_status.argtypes = [vp]
+    lib.bv_set_option.argtypes = [ctypes.c_char_p, ci]
     lib.bv_status_string.restype = ctypes.c_char_p
     lib.bv_status_string.argtypes = [ci]
     if path is None:
@@ -80,6 +82,17 @@ def bv_last_launch_count() -> int:
 
 def bv_release() -> None:
     _check(load_library().bv_release())
+
+
+def bv_set_option(name: str, value: int) -> None:
+    """Process-wide tuning / test option of the library (see include/bv.h); 0 restores the default."""
+    _check(load_library().bv_set_option(name.encode(), int(value)))
+
+
+def bv_stream_status(stream=None) -> int:
+    """Waits for the stream and returns 0, or -4 if a device-side wait of a call on it gave up."""
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(load_library().bv_stream_status(ctypes.c_void_p(s.cuda_stream)))
 
 
 def _check(status: int) -> None:

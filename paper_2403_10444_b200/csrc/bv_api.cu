@@ -1,4 +1,4 @@
-// C-ABI layer: argument checks, per-device workspace, launch-shape selection and
+// C-ABI layer: argument checks, per-device and per-stream workspace, launch-shape selection and
 // the host-buffer entry points.  Declarations and contracts are in include/bv.h.
 #include <cuda_runtime.h>
 
@@ -14,7 +14,53 @@
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr int kTicketSlots = 64;  // concurrent calls on one device each need their own slot
+constexpr int kTicketSlots = 64;  // concurrent calls of the cluster kernels on one device each need their own slot
+constexpr int kStreamSlots = 32;  // streams per device that keep a workspace of their own
+
+// Tuning and test options (bv_set_option); their first values come from the environment, read once.
+struct Options {
+    int kernel = 0;        // 0: chosen by shape; 1 flow, 2 cluster, 3 stream
+    int cluster = 0;       // cluster width of the cluster / stream kernels (1, 2, 4, 8); 0: chosen by shape
+    int max_clusters = 0;  // cap on the clusters launched; 0: none
+    int flow_chunks = 0, flow_pieces = 0, flow_ctas = 0, flow_depth = 0;   // 0: chosen by shape
+    int wait_limit = 0;    // polls after which a bounded device-side wait gives up; 0: the built-in limits
+    int never_signal = 0;  // test switch: the flow kernel's workers never report an item as swept
+};
+Options g_opt;
+std::once_flag g_opt_once;
+
+int env_int(const char* name) {
+    const char* v = std::getenv(name);
+    return v ? std::atoi(v) : 0;
+}
+int kernel_code(const char* v) {
+    if (!v) return 0;
+    if (!std::strcmp(v, "flow")) return 1;
+    if (!std::strcmp(v, "cluster")) return 2;
+    if (!std::strcmp(v, "stream")) return 3;
+    return 0;
+}
+void load_env_options() {
+    g_opt.kernel = kernel_code(std::getenv("BV_KERNEL"));
+    g_opt.cluster = env_int("BV_CLUSTER");
+    g_opt.max_clusters = env_int("BV_MAX_CLUSTERS");
+    g_opt.flow_chunks = env_int("BV_FLOW_CHUNKS");
+    g_opt.flow_pieces = env_int("BV_FLOW_PIECES");
+    g_opt.flow_ctas = env_int("BV_FLOW_CTAS");
+    g_opt.flow_depth = env_int("BV_FLOW_DEPTH");
+}
+
+// The workspace a stream's calls share.  Calls on one stream run one after the other, and the flow
+// kernel leaves its counters at zero, so one area per stream serves any number of calls in flight;
+// it grows with cudaMallocAsync / cudaFreeAsync on that stream, which do not synchronise the device.
+struct StreamSlot {
+    cudaStream_t stream = nullptr;
+    bool used = false;
+    void* ws = nullptr;        // [status word, 256 bytes][flow scratch]
+    size_t bytes = 0;
+    size_t clean = 0;          // leading bytes of the flow scratch known to be zero between calls
+    unsigned long long stamp = 0;
+};
 
 struct DeviceState {
     bool ready = false;
@@ -23,14 +69,9 @@ struct DeviceState {
     unsigned int* tickets = nullptr;  // [kTicketSlots][2], zero when idle
     unsigned long long calls = 0;
     int max_clusters[2][2][2][bv::kMaxCluster + 1] = {};  // [algo][dtype][vec][cluster], 0 = not asked yet
-    int res_clusters[2][9][bv::kMaxCluster + 1] = {};     // resident kernel: [dtype][nk][cluster]
     int clu_clusters[2][2][bv::kMaxCluster + 1] = {};     // cluster kernel: [algo][dtype][cluster]
-    // scratch of the flow kernel: a small ring, so that calls in flight on different streams
-    // do not share counters (more than kFlowSlots overlapping calls on one device would)
-    void* flow_ws[4] = {};
-    size_t flow_bytes[4] = {};
-    size_t flow_clean[4] = {};        // leading bytes of each area known to be zero between calls
-    unsigned long long flow_calls = 0;
+    StreamSlot slots[kStreamSlots];
+    unsigned long long clock = 0;
     int flow_ctas_per_sm[2] = {};
     // staging for the host-buffer entry points
     void* stage = nullptr;
@@ -43,14 +84,8 @@ std::mutex g_mu;
 
 thread_local int t_last_launches = 0;
 thread_local int t_last_cuda_error = 0;
-thread_local const float* t_given_lse_d = nullptr;   // set by bv_verify_lse around its call of run_device
-thread_local int t_greedy = 0;                       // set by gbv_verify around its call of run_device
 
-int cuda_fail(cudaError_t e) {
-    t_last_cuda_error = static_cast<int>(e);
-    cudaGetLastError();
-    return BV_ERR_CUDA;
-}
+int cuda_fail(cudaError_t e) { return bv::note_cuda_error(e); }
 
 // Per-device set-up on first use: device attributes and the ticket slots.
 int device_state(DeviceState** out) {
@@ -65,10 +100,9 @@ int device_state(DeviceState** out) {
         if ((e = cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
             return cuda_fail(e);
         if (d.cc_major < 10) return BV_ERR_UNSUPPORTED;
-        // ticket slots, then one status word that a kernel sets if a bounded wait gives up
-        if ((e = cudaMalloc(&d.tickets, sizeof(unsigned int) * (2 * kTicketSlots + 1))) != cudaSuccess)
+        if ((e = cudaMalloc(&d.tickets, sizeof(unsigned int) * 2 * kTicketSlots)) != cudaSuccess)
             return cuda_fail(e);
-        if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned int) * (2 * kTicketSlots + 1))) != cudaSuccess)
+        if ((e = cudaMemset(d.tickets, 0, sizeof(unsigned int) * 2 * kTicketSlots)) != cudaSuccess)
             return cuda_fail(e);
         d.ready = true;
     }
@@ -76,29 +110,43 @@ int device_state(DeviceState** out) {
     return BV_OK;
 }
 
-bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
-
-int check_args(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
-               int V, int dtype, float T, const int32_t* ot, const int32_t* ol) {
-    if (!tgt || !drf || !tok || !uni || !ot || !ol) return BV_ERR_INVALID_ARG;
-    if (B < 0 || gamma < 1 || V < 1) return BV_ERR_INVALID_ARG;
-    if (!(T > 0.f) || !std::isfinite(T)) return BV_ERR_INVALID_ARG;
-    if (dtype != BV_DTYPE_F32 && dtype != BV_DTYPE_BF16) return BV_ERR_INVALID_ARG;
-    const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
-    if (!aligned(tgt, esz) || !aligned(drf, esz) || !aligned(tok, 4) || !aligned(uni, 4) ||
-        !aligned(ot, 4) || !aligned(ol, 4))
-        return BV_ERR_INVALID_ARG;
-    if (gamma > BV_MAX_GAMMA) return BV_ERR_UNSUPPORTED;
+// The workspace of `stream` with room for `need` bytes of flow scratch behind its status word.
+// A stream seen for the first time takes a free entry, or the one used longest ago (whose area is
+// freed in its own stream's order).
+int stream_slot(DeviceState& d, cudaStream_t stream, size_t need, StreamSlot** out) {
+    StreamSlot* s = nullptr;
+    StreamSlot* victim = nullptr;
+    for (StreamSlot& c : d.slots) {
+        if (c.used && c.stream == stream) { s = &c; break; }
+        if (!victim || (victim->used && (!c.used || c.stamp < victim->stamp))) victim = &c;
+    }
+    cudaError_t e;
+    if (!s) {
+        s = victim;
+        if (s->used && s->ws && (e = cudaFreeAsync(s->ws, s->stream)) != cudaSuccess) return cuda_fail(e);
+        *s = StreamSlot{};
+        s->used = true;
+        s->stream = stream;
+    }
+    s->stamp = ++d.clock;
+    const size_t total = 256 + need;
+    if (s->bytes < total) {
+        if (s->ws && (e = cudaFreeAsync(s->ws, stream)) != cudaSuccess) return cuda_fail(e);
+        s->ws = nullptr; s->bytes = 0; s->clean = 0;
+        if ((e = cudaMallocAsync(&s->ws, total, stream)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemsetAsync(s->ws, 0, 256, stream)) != cudaSuccess) return cuda_fail(e);   // the status word
+        s->bytes = total;
+    }
+    *out = s;
     return BV_OK;
 }
 
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
 // Cluster width for the streaming kernel: wide enough that a CTA's slice of a row
 // is at most 64 KB, widened further while the batch alone cannot fill the SMs.
-int pick_cluster(const DeviceState& d, int B, size_t row_bytes) {
-    if (const char* env = std::getenv("BV_CLUSTER")) {
-        int c = std::atoi(env);
-        if (c == 1 || c == 2 || c == 4 || c == 8) return c;
-    }
+int pick_cluster(const DeviceState& d, const Options& opt, int B, size_t row_bytes) {
+    if (opt.cluster == 1 || opt.cluster == 2 || opt.cluster == 4 || opt.cluster == 8) return opt.cluster;
     int c = 1;
     while (c < bv::kMaxCluster && row_bytes / c > (64u << 10)) c *= 2;
     while (c < bv::kMaxCluster && static_cast<long long>(B) * c < d.sm_count && row_bytes / (2 * c) >= (8u << 10))
@@ -109,15 +157,23 @@ int pick_cluster(const DeviceState& d, int B, size_t row_bytes) {
     return c;
 }
 
+struct Extra {              // what only some entry points pass
+    const float* lse_d = nullptr;   // supplied draft log-normalisers (bv_verify_lse)
+    int greedy = 0;                 // Algorithm 4 instead of Algorithm 2 (gbv_verify)
+    float* out_p = nullptr; float* out_S = nullptr; float* out_h = nullptr;
+    float* out_lse_t = nullptr; float* out_lse_d = nullptr;
+};
+
 int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
-               int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p, float* out_S,
-               float* out_h, float* out_lse_t, float* out_lse_d, cudaStream_t stream) {
+               int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, const Extra& ex, cudaStream_t stream) {
     t_last_launches = 0;
-    int rc = check_args(tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
+    int rc = bv::check_verify_args(tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
     if (rc != BV_OK) return rc;
     if (B == 0) return BV_OK;
+    std::call_once(g_opt_once, load_env_options);
 
     std::lock_guard<std::mutex> lock(g_mu);
+    const Options opt = g_opt;
     DeviceState* d = nullptr;
     if ((rc = device_state(&d)) != BV_OK) return rc;
 
@@ -127,26 +183,23 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
 
     bv::Params prm{};
     prm.tgt = tgt; prm.drf = drf; prm.tok = tok; prm.uni = uni;
-    prm.lse_d = t_given_lse_d;
-    prm.greedy = t_greedy;
+    prm.lse_d = ex.lse_d;
+    prm.greedy = ex.greedy;
     prm.B = B; prm.gamma = gamma; prm.V = V;
     const double kd = 1.4426950408889634073599246810019 / static_cast<double>(T);
     prm.kd = kd;
     prm.kf = static_cast<float>(kd);
     prm.out_tokens = ot; prm.out_len = ol;
-    prm.out_p = out_p; prm.out_S = out_S; prm.out_h = out_h;
-    prm.out_lse_t = out_lse_t; prm.out_lse_d = out_lse_d;
-    prm.status = reinterpret_cast<int*>(d->tickets + 2 * kTicketSlots);
+    prm.out_p = ex.out_p; prm.out_S = ex.out_S; prm.out_h = ex.out_h;
+    prm.out_lse_t = ex.out_lse_t; prm.out_lse_d = ex.out_lse_d;
+    prm.wait_limit = opt.wait_limit > 0 ? static_cast<unsigned>(opt.wait_limit) : 0u;
+    prm.never_signal = opt.never_signal;
 
-    // Block Verification on 16-byte rows: the kernel that keeps each row pair on chip,
-    // when some cluster width lets a thread hold its share (at most 8 vectors per row).
-    const char* force = std::getenv("BV_KERNEL");   // "flow", "cluster", "resident", "stream": experiments and tests
-    const bool want = force != nullptr;
-    auto forced = [&](const char* name) { return want && std::strcmp(force, name) == 0; };
-    if ((prm.lse_d != nullptr || prm.greedy) && !(algo == bv::kBlockVerify && vec && (!want || forced("flow")))) return BV_ERR_UNSUPPORTED;
+    const bool flow_ok = algo == bv::kBlockVerify && vec && (opt.kernel == 0 || opt.kernel == 1);
+    if ((prm.lse_d != nullptr || prm.greedy) && !flow_ok) return BV_ERR_UNSUPPORTED;
 
     // Block Verification on 16-byte rows: the flow of independent work items
-    if (algo == bv::kBlockVerify && vec && (!want || forced("flow"))) {
+    if (flow_ok) {
         int& per_sm = d->flow_ctas_per_sm[dtype];
         if (per_sm == 0) {
             per_sm = bv::flow_max_ctas_per_sm(dtype);
@@ -155,51 +208,32 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
         if (per_sm > 0) {
             const long long units = static_cast<long long>(row_bytes / 16);
             long long nctas = static_cast<long long>(d->sm_count) * per_sm;
-            if (const char* env = std::getenv("BV_FLOW_CTAS")) {
-                const long long v = std::atoll(env);
-                if (v >= 1 && v < nctas) nctas = v;
-            }
-            int chunks = 0, pieces = 0;
-            if (const char* env = std::getenv("BV_FLOW_CHUNKS")) {
-                const int v = std::atoi(env);
-                if (v >= 1 && v <= bv::kFlowMaxChunks) chunks = v;
-            }
-            if (const char* env = std::getenv("BV_FLOW_PIECES")) {
-                const int v = std::atoi(env);
-                if (v >= 1 && v <= 8) pieces = v;
-            }
+            if (opt.flow_ctas >= 1 && opt.flow_ctas < nctas) nctas = opt.flow_ctas;
+            const int chunks = (opt.flow_chunks >= 1 && opt.flow_chunks <= bv::kFlowMaxChunks) ? opt.flow_chunks : 0;
+            const int pieces = (opt.flow_pieces >= 1 && opt.flow_pieces <= 8) ? opt.flow_pieces : 0;
             // (with supplied draft normalisers a first-sweep item streams one row, not two)
             const bv::FlowPlan plan = bv::flow_plan(units, B, gamma, nctas, prm.lse_d == nullptr, chunks, pieces);
             size_t zero_bytes = 0;
             const size_t need = bv::flow_scratch_bytes(B, gamma, plan, &zero_bytes);
-            const int slot = static_cast<int>(d->flow_calls++ % 4);
-            if (d->flow_bytes[slot] < need) {
-                if (d->flow_ws[slot]) cudaFree(d->flow_ws[slot]);
-                d->flow_ws[slot] = nullptr;
-                d->flow_bytes[slot] = 0;
-                d->flow_clean[slot] = 0;
-                cudaError_t e = cudaMalloc(&d->flow_ws[slot], need);
-                if (e != cudaSuccess) return cuda_fail(e);
-                d->flow_bytes[slot] = need;
-            }
+            StreamSlot* slot = nullptr;
+            if ((rc = stream_slot(*d, stream, need, &slot)) != BV_OK) return rc;
+            char* scratch = static_cast<char*>(slot->ws) + 256;
             bv::FlowScratch fl;
-            bv::flow_scratch_layout(d->flow_ws[slot], B, gamma, plan, &fl);
-            if (const char* env = std::getenv("BV_FLOW_DEPTH")) {
-                const int v = std::atoi(env);
-                if (v >= 2 && v <= 6) fl.depth = v;
-            }
+            bv::flow_scratch_layout(scratch, B, gamma, plan, &fl);
+            if (opt.flow_depth >= 2 && opt.flow_depth <= 6) fl.depth = opt.flow_depth;
             // The kernel leaves its counters and flags at zero when it ends, so they are cleared here only
             // when the area is new or a larger problem needs more of them than the last launch left clean.
             cudaError_t e = cudaSuccess;
-            if (d->flow_clean[slot] < zero_bytes) {
-                e = cudaMemsetAsync(d->flow_ws[slot], 0, zero_bytes, stream);
+            if (slot->clean < zero_bytes) {
+                e = cudaMemsetAsync(scratch, 0, zero_bytes, stream);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
-            d->flow_clean[slot] = zero_bytes;
+            slot->clean = zero_bytes;
             long long items = static_cast<long long>(fl.total_s1);
             if (nctas > items) nctas = items;
             prm.ticket = nullptr;
             prm.nclusters = 0;
+            prm.status = static_cast<int*>(slot->ws);
             e = bv::launch_flow(prm, fl, dtype, static_cast<int>(nctas), stream);
             if (e != cudaSuccess) return cuda_fail(e);
             t_last_launches = 1;
@@ -209,39 +243,12 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
 
     if (prm.lse_d != nullptr || prm.greedy) return BV_ERR_UNSUPPORTED;   // (the flow kernel could not be launched)
 
-    if (algo == bv::kBlockVerify && vec && forced("resident")) {
-        const long long units = static_cast<long long>(row_bytes / 16);
-        int best_c = 0, best_nk = 0, best_n = 0;
-        long long best_sms = -1;
-        const char* ec = std::getenv("BV_RES_CLUSTER");
-        for (int c = bv::kMaxCluster; c >= 1; c /= 2) {
-            if (ec && std::atoi(ec) != c) continue;
-            const long long per_warp = ((units + c - 1) / c + 15) / 16;
-            int nk = 0;
-            for (int cand : {2, 4, 8}) if (per_warp <= 32LL * cand) { nk = cand; break; }
-            if (!nk) continue;
-            int& cached = d->res_clusters[dtype][nk][c];
-            if (cached == 0) {
-                cached = bv::resident_max_clusters(dtype, nk, c);
-                if (cached <= 0) cached = -1;
-            }
-            if (cached < 0) continue;
-            const int n = B < cached ? B : cached;
-            const long long sms = static_cast<long long>(n) * c;
-            if (sms >= best_sms) { best_sms = sms; best_c = c; best_nk = nk; best_n = n; }
-        }
-        if (best_c) {
-            prm.ticket = nullptr;
-            prm.nclusters = best_n;
-            cudaError_t e = bv::launch_resident(prm, dtype, best_nk, best_c, best_n, stream);
-            if (e != cudaSuccess) return cuda_fail(e);
-            t_last_launches = 1;
-            return BV_OK;
-        }
-    }
+    StreamSlot* slot = nullptr;
+    if ((rc = stream_slot(*d, stream, 0, &slot)) != BV_OK) return rc;
+    prm.status = static_cast<int*>(slot->ws);
 
-    int cluster = pick_cluster(*d, B, row_bytes);
-    if (vec && !forced("stream")) {
+    int cluster = pick_cluster(*d, opt, B, row_bytes);
+    if (vec && opt.kernel != 3) {
         int& cc = d->clu_clusters[algo][dtype][cluster];
         if (cc == 0) {
             cc = bv::cluster_max_clusters(algo, dtype, cluster);
@@ -249,10 +256,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
         }
         if (cc > 0) {
             int n = B < cc ? B : cc;
-            if (const char* env = std::getenv("BV_MAX_CLUSTERS")) {
-                const int cap = std::atoi(env);
-                if (cap > 0 && cap < n) n = cap;
-            }
+            if (opt.max_clusters > 0 && opt.max_clusters < n) n = opt.max_clusters;
             prm.ticket = d->tickets + 2 * (d->calls++ % kTicketSlots);
             prm.nclusters = n;
             cudaError_t e = bv::launch_cluster(prm, algo, dtype, cluster, n, stream);
@@ -278,11 +282,34 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     return BV_OK;
 }
 
+// Reads and clears the status word of `stream`'s workspace; waits for the stream.
+int take_stream_status(cudaStream_t stream) {
+    int* word = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        DeviceState* d = nullptr;
+        const int rc = device_state(&d);
+        if (rc != BV_OK) return rc;
+        for (StreamSlot& c : d->slots)
+            if (c.used && c.stream == stream) word = static_cast<int*>(c.ws);
+    }
+    cudaError_t e;
+    if (!word) {
+        if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(e);
+        return BV_OK;
+    }
+    int status = 0;
+    if ((e = cudaMemcpyAsync(&status, word, sizeof(int), cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemsetAsync(word, 0, sizeof(int), stream)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(e);
+    return status ? BV_ERR_TIMEOUT : BV_OK;
+}
+
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
              int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol) {
-    int rc = check_args(tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
+    int rc = bv::check_verify_args(tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
     if (rc != BV_OK) return rc;
     if (B == 0) return BV_OK;
     const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
@@ -296,7 +323,6 @@ int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, con
 
     char* base = nullptr;
     cudaStream_t s = nullptr;
-    int* status_word = nullptr;
     {
         std::lock_guard<std::mutex> lock(g_mu);
         DeviceState* d = nullptr;
@@ -304,6 +330,7 @@ int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, con
         cudaError_t e;
         if (!d->stream && (e = cudaStreamCreateWithFlags(&d->stream, cudaStreamNonBlocking)) != cudaSuccess)
             return cuda_fail(e);
+        // (this entry point waits for its result anyway, so its staging buffer grows with plain cudaMalloc)
         if (d->stage_bytes < total) {
             if (d->stage) cudaFree(d->stage);
             d->stage = nullptr;
@@ -313,7 +340,6 @@ int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, con
         }
         base = static_cast<char*>(d->stage);
         s = d->stream;
-        status_word = reinterpret_cast<int*>(d->tickets + 2 * kTicketSlots);
     }
     cudaError_t e;
     if ((e = cudaMemcpyAsync(base + o_t, tgt, n_t, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
@@ -322,86 +348,104 @@ int run_host(int algo, const void* tgt, const void* drf, const int32_t* tok, con
     if ((e = cudaMemcpyAsync(base + o_uni, uni, n_uni, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
     rc = run_device(algo, base + o_t, base + o_d, reinterpret_cast<const int32_t*>(base + o_tok),
                     reinterpret_cast<const float*>(base + o_uni), B, gamma, V, dtype, T,
-                    reinterpret_cast<int32_t*>(base + o_ot), reinterpret_cast<int32_t*>(base + o_ol),
-                    nullptr, nullptr, nullptr, nullptr, nullptr, s);
+                    reinterpret_cast<int32_t*>(base + o_ot), reinterpret_cast<int32_t*>(base + o_ol), Extra{}, s);
     if (rc != BV_OK) return rc;
     if ((e = cudaMemcpyAsync(ot, base + o_ot, n_ot, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaMemcpyAsync(ol, base + o_ol, n_ol, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
-    int status = 0;
-    if ((e = cudaMemcpyAsync(&status, status_word, sizeof(int), cudaMemcpyDeviceToHost, s)) != cudaSuccess)
-        return cuda_fail(e);
-    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
-    return status ? BV_ERR_TIMEOUT : BV_OK;
+    return take_stream_status(s);
+}
+
+Extra diagnostics(float* out_p, float* out_S, float* out_h, float* out_lse_t, float* out_lse_d) {
+    Extra ex;
+    ex.out_p = out_p; ex.out_S = out_S; ex.out_h = out_h; ex.out_lse_t = out_lse_t; ex.out_lse_d = out_lse_d;
+    return ex;
 }
 
 }  // namespace
+
+namespace bv {
+
+int note_cuda_error(cudaError_t e) {
+    t_last_cuda_error = static_cast<int>(e);
+    cudaGetLastError();
+    return BV_ERR_CUDA;
+}
+void note_launches(int n) { t_last_launches = n; }
+
+int check_verify_args(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+                      int V, int dtype, float T, const int32_t* ot, const int32_t* ol) {
+    if (!tgt || !drf || !tok || !uni || !ot || !ol) return BV_ERR_INVALID_ARG;
+    if (B < 0 || gamma < 1 || V < 1) return BV_ERR_INVALID_ARG;
+    if (!(T > 0.f) || !std::isfinite(T)) return BV_ERR_INVALID_ARG;
+    if (dtype != BV_DTYPE_F32 && dtype != BV_DTYPE_BF16) return BV_ERR_INVALID_ARG;
+    const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
+    if (!aligned(tgt, esz) || !aligned(drf, esz) || !aligned(tok, 4) || !aligned(uni, 4) ||
+        !aligned(ot, 4) || !aligned(ol, 4))
+        return BV_ERR_INVALID_ARG;
+    if (gamma > BV_MAX_GAMMA) return BV_ERR_UNSUPPORTED;
+    return BV_OK;
+}
+
+}  // namespace bv
 
 extern "C" {
 
 int bv_verify(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
               int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
-    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, nullptr, nullptr,
-                      nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, Extra{},
+                      static_cast<cudaStream_t>(stream));
 }
 
 int bv_verify_lse(const void* tgt, const void* drf, const int32_t* tok, const float* uni, const float* draft_lse,
                   int B, int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
     if (!draft_lse) return BV_ERR_INVALID_ARG;
-    t_given_lse_d = draft_lse;
-    const int rc = run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, nullptr, nullptr,
-                              nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
-    t_given_lse_d = nullptr;
-    return rc;
+    Extra ex;
+    ex.lse_d = draft_lse;
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, ex, static_cast<cudaStream_t>(stream));
 }
 
 int bv_verify_lse_ex(const void* tgt, const void* drf, const int32_t* tok, const float* uni, const float* draft_lse,
                      int B, int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p,
                      float* out_S, float* out_h, float* out_lse_t, float* out_lse_d, void* stream) {
     if (!draft_lse) return BV_ERR_INVALID_ARG;
-    t_given_lse_d = draft_lse;
-    const int rc = run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, out_p, out_S,
-                              out_h, out_lse_t, out_lse_d, static_cast<cudaStream_t>(stream));
-    t_given_lse_d = nullptr;
-    return rc;
+    Extra ex = diagnostics(out_p, out_S, out_h, out_lse_t, out_lse_d);
+    ex.lse_d = draft_lse;
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, ex, static_cast<cudaStream_t>(stream));
 }
 
 int gbv_verify(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
                int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
-    t_greedy = 1;
-    const int rc = run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, nullptr, nullptr,
-                              nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
-    t_greedy = 0;
-    return rc;
+    Extra ex;
+    ex.greedy = 1;
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, ex, static_cast<cudaStream_t>(stream));
 }
 
 int gbv_verify_ex(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
                   int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p, float* out_S,
                   float* out_h, float* out_lse_t, float* out_lse_d, void* stream) {
-    t_greedy = 1;
-    const int rc = run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, out_p, out_S,
-                              out_h, out_lse_t, out_lse_d, static_cast<cudaStream_t>(stream));
-    t_greedy = 0;
-    return rc;
+    Extra ex = diagnostics(out_p, out_S, out_h, out_lse_t, out_lse_d);
+    ex.greedy = 1;
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, ex, static_cast<cudaStream_t>(stream));
 }
 
 int tv_verify(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
               int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
-    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, nullptr, nullptr,
-                      nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, Extra{},
+                      static_cast<cudaStream_t>(stream));
 }
 
 int bv_verify_ex(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
                  int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p, float* out_S,
                  float* out_h, float* out_lse_t, float* out_lse_d, void* stream) {
-    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, out_p, out_S,
-                      out_h, out_lse_t, out_lse_d, static_cast<cudaStream_t>(stream));
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol,
+                      diagnostics(out_p, out_S, out_h, out_lse_t, out_lse_d), static_cast<cudaStream_t>(stream));
 }
 
 int tv_verify_ex(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
                  int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p, float* out_S,
                  float* out_h, float* out_lse_t, float* out_lse_d, void* stream) {
-    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, out_p, out_S,
-                      out_h, out_lse_t, out_lse_d, static_cast<cudaStream_t>(stream));
+    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol,
+                      diagnostics(out_p, out_S, out_h, out_lse_t, out_lse_d), static_cast<cudaStream_t>(stream));
 }
 
 int bv_verify_host(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
@@ -414,6 +458,25 @@ int tv_verify_host(const void* tgt, const void* drf, const int32_t* tok, const f
     return run_host(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
 }
 
+int bv_stream_status(void* stream) { return take_stream_status(static_cast<cudaStream_t>(stream)); }
+
+int bv_set_option(const char* name, int value) {
+    if (!name) return BV_ERR_INVALID_ARG;
+    std::call_once(g_opt_once, load_env_options);
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!std::strcmp(name, "kernel")) g_opt.kernel = value;
+    else if (!std::strcmp(name, "cluster")) g_opt.cluster = value;
+    else if (!std::strcmp(name, "max_clusters")) g_opt.max_clusters = value;
+    else if (!std::strcmp(name, "flow_chunks")) g_opt.flow_chunks = value;
+    else if (!std::strcmp(name, "flow_pieces")) g_opt.flow_pieces = value;
+    else if (!std::strcmp(name, "flow_ctas")) g_opt.flow_ctas = value;
+    else if (!std::strcmp(name, "flow_depth")) g_opt.flow_depth = value;
+    else if (!std::strcmp(name, "wait_limit")) g_opt.wait_limit = value;
+    else if (!std::strcmp(name, "never_signal")) g_opt.never_signal = value;
+    else return BV_ERR_INVALID_ARG;
+    return BV_OK;
+}
+
 int bv_release(void) {
     std::lock_guard<std::mutex> lock(g_mu);
     int dev = 0;
@@ -424,7 +487,7 @@ int bv_release(void) {
     if ((e = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(e);
     if (d.stage) cudaFree(d.stage);
     if (d.tickets) cudaFree(d.tickets);
-    for (void* w : d.flow_ws) if (w) cudaFree(w);
+    for (StreamSlot& c : d.slots) if (c.used && c.ws) cudaFree(c.ws);
     if (d.stream) cudaStreamDestroy(d.stream);
     d = DeviceState{};
     return BV_OK;
@@ -445,6 +508,6 @@ const char* bv_status_string(int status) {
     }
 }
 
-int bv_version(void) { return 100; }
+int bv_version(void) { return 200; }
 
 }  // extern "C"

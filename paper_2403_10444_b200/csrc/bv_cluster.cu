@@ -142,6 +142,7 @@ __global__ void __launch_bounds__(kCThreads, 2) verify_cluster_kernel(const Para
     const uint32_t bytes_ms = static_cast<uint32_t>(C) * kCWarps * 16u;
     const uint32_t bytes_seg = static_cast<uint32_t>(C) * kCWarps * 4u;
     uint32_t ph_ms = 0, ph_seg = 0, ph_cand = 0, ph_b = 0;
+    if (tid == 0) sh.b_next = -1;
     cluster.sync();   // barriers and exchange arrays are ready everywhere before any message
 
     for (;;) {
@@ -153,9 +154,11 @@ __global__ void __launch_bounds__(kCThreads, 2) verify_cluster_kernel(const Para
             for (int c = 0; c < C; ++c)
                 send_b32(map_to_rank(smem_u32(&sh.b_next), c), map_to_rank(smem_u32(&sh.bar_b), c), nb);
         }
-        mbar_wait(smem_u32(&sh.bar_b), ph_b, status);
+        // (a wait that gives up leaves sh.b_next at -1: the CTA goes to the final barrier without
+        // ever using a block index that nobody sent)
+        const bool told = mbar_wait(smem_u32(&sh.bar_b), ph_b, status);
         ph_b ^= 1u;
-        const int b = sh.b_next;
+        const int b = told ? sh.b_next : -1;
         if (b < 0) break;
 
         if (tid <= g) {

@@ -270,6 +270,9 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     // by cp.async, so loads run kFSlots steps ahead of the arithmetic without costing registers.
     extern __shared__ __align__(16) unsigned char dyn[];
 
+    // polls after which a bounded wait gives up
+    const uint32_t lim_spin = prm.wait_limit ? prm.wait_limit : (1u << 24);
+    const uint32_t lim_nap = prm.wait_limit ? prm.wait_limit : (1u << 22);
     FlowCtx cx;
     cx.g = prm.gamma; cx.V = prm.V; cx.B = prm.B; cx.units = prm.V / EPV;
     cx.row_bytes = static_cast<size_t>(prm.V) * ESZ; cx.kf = prm.kf; cx.kd = prm.kd;
@@ -299,9 +302,9 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         for (int n = k;; n += kFPost) {
             const int slot = n % kFDesc;
             const uint32_t par = static_cast<uint32_t>(n / kFDesc) & 1u;
-            if (!mbar_wait_relaxed(smem_u32(&sh.full[slot]), par, prm.status, 200)) break;
+            if (!mbar_wait_relaxed(smem_u32(&sh.full[slot]), par, prm.status, 200, lim_nap)) break;
             if (sh.desc[slot].kind == kExit) break;
-            if (!mbar_wait_relaxed(smem_u32(&sh.done[slot]), par, prm.status, 200)) break;
+            if (!mbar_wait_relaxed(smem_u32(&sh.done[slot]), par, prm.status, 200, lim_nap)) break;
             if (lane == 0) sh.sdesc[k] = sh.desc[slot];
             if (lane < kFWarps) {
                 sh.stage_M[k][0][lane] = sh.part_M[slot][0][lane]; sh.stage_M[k][1][lane] = sh.part_M[slot][1][lane];
@@ -394,7 +397,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         auto late_desc = [&](int t, FlowDesc& d) -> bool {
             unsigned e = 0;
             for (unsigned spins = 0; (e = ld_volatile(&fl.lq[t / fl.nch_late])) == 0u; ++spins)
-                if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
+                if (spins > lim_nap) { if (prm.status) atomicExch(prm.status, 1); return false; }
             const int ri = static_cast<int>(e - 1u);
             d.kind = kSweep1; d.ri = ri; d.ch = t % fl.nch_late; d.have_q = 0;
             item_range(cx.units, fl.nch_late, d.ch, d.u0, d.u1);
@@ -406,7 +409,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         auto piece_desc = [&](int t, FlowDesc& d) -> bool {
             unsigned e = 0;
             for (unsigned spins = 0; (e = ld_volatile(&fl.s2q[t / fl.np])) == 0u; ++spins)   // the entry follows the tail at once
-                if (spins > (1u << 22)) { if (prm.status) atomicExch(prm.status, 1); return false; }
+                if (spins > lim_nap) { if (prm.status) atomicExch(prm.status, 1); return false; }
             const int ri = static_cast<int>(e - 1u);
             const int r = ri % (g + 1), b = ri / (g + 1);
             d.kind = kSweep2; d.ri = ri; d.ch = t % fl.np; d.have_q = r < g;
@@ -436,8 +439,8 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         for (;;) {
             // the slot must be free (its previous item moved out by its post warp), and at most `depth`
             // published items may still be with the workers
-            if (q >= kFDesc && !mbar_wait_relaxed(smem_u32(&sh.freeb[q % kFDesc]), static_cast<uint32_t>(q / kFDesc - 1) & 1u, prm.status, 100)) { failed = true; break; }
-            if (q >= depth && !mbar_wait_relaxed(smem_u32(&sh.done[(q - depth) % kFDesc]), static_cast<uint32_t>((q - depth) / kFDesc) & 1u, prm.status, 100)) { failed = true; break; }
+            if (q >= kFDesc && !mbar_wait_relaxed(smem_u32(&sh.freeb[q % kFDesc]), static_cast<uint32_t>(q / kFDesc - 1) & 1u, prm.status, 100, lim_nap)) { failed = true; break; }
+            if (q >= depth && !mbar_wait_relaxed(smem_u32(&sh.done[(q - depth) % kFDesc]), static_cast<uint32_t>((q - depth) / kFDesc) & 1u, prm.status, 100, lim_nap)) { failed = true; break; }
             FlowDesc d;
             d.kind = kExit;
             // (a) a piece of a row that waits for its second sweep: they are few and others wait for them
@@ -474,7 +477,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             // counters: wait long enough not to crowd those who work)
             __nanosleep(exhausted || idle < 4 ? 500 : 2000);
             poll();
-            if (++idle > (1u << 21)) { if (prm.status) atomicExch(prm.status, 1); failed = true; break; }
+            if (++idle > (lim_nap >> 1)) { if (prm.status) atomicExch(prm.status, 1); failed = true; break; }
         }
         // release the workers and the post warps: one exit descriptor for each post warp to find
         // (on the regular way out every slot is free; after a wait that gave up nothing is relied on)
@@ -582,7 +585,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         const int slot = n_c % kFDesc;
         if (n_i == n_c) {
             // the loads of this item have not been started: the ring is empty
-            if (!mbar_wait_now(smem_u32(&sh.full[slot]), static_cast<uint32_t>(n_c / kFDesc) & 1u, prm.status)) break;
+            if (!mbar_wait_now(smem_u32(&sh.full[slot]), static_cast<uint32_t>(n_c / kFDesc) & 1u, prm.status, lim_spin)) break;
             if (sh.desc[slot].kind == kExit) break;
             i_stalled = false;
             issue_load(slot);
@@ -659,7 +662,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             const float tP = warp_sum(sP);
             if (lane == 0) sh.part_s[slot][0][warp] = tP;
         }
-        if (lane == 0) mbar_arrive(smem_u32(&sh.done[slot]));   // releases this warp's partials and the descriptor
+        if (lane == 0 && !prm.never_signal) mbar_arrive(smem_u32(&sh.done[slot]));   // releases this warp's partials and the descriptor
         __syncwarp();
     }
     cp_async_wait<0>();

@@ -7,6 +7,13 @@
 
 namespace bv {
 
+// Shared by the files that hold entry points: argument checks of the verification calls, the
+// thread's record of the last failing CUDA call (returns BV_ERR_CUDA) and of the launches of its last call.
+int check_verify_args(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+                      int V, int dtype, float T, const int32_t* ot, const int32_t* ol);
+int note_cuda_error(cudaError_t e);
+void note_launches(int n);
+
 // Most clusters of `cluster` CTAs of the streaming kernel that can be resident at once
 // on the current device (0 if that cluster size cannot be scheduled).
 int stream_max_clusters(int algo, int dtype, bool vec, int cluster);
@@ -68,12 +75,5 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
 int flow_max_ctas_per_sm(int dtype);
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream);
 
-
-// Resident kernel (Block Verification only, 128-bit path): a thread holds up to `nk`
-// vectors per row, nk in {2, 4, 8}.
-int resident_vectors_per_cta(int nk);
-int resident_max_clusters(int dtype, int nk, int cluster);
-cudaError_t launch_resident(const Params& prm, int dtype, int nk, int cluster, int nclusters,
-                            cudaStream_t stream);
 
 }  // namespace bv

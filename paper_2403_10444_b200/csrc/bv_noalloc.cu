@@ -39,37 +39,31 @@ bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p
 
 extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
                                  int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
-    if (!tgt || !drf || !tok || !uni || !ot || !ol) return BV_ERR_INVALID_ARG;
-    if (B < 0 || gamma < 1 || V < 1) return BV_ERR_INVALID_ARG;
-    if (!(T > 0.f) || !std::isfinite(T)) return BV_ERR_INVALID_ARG;
-    if (dtype != BV_DTYPE_F32 && dtype != BV_DTYPE_BF16) return BV_ERR_INVALID_ARG;
-    if (gamma > BV_MAX_GAMMA) return BV_ERR_UNSUPPORTED;
+    bv::note_launches(0);
+    const int rc = bv::check_verify_args(tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
+    if (rc != BV_OK) return rc;
     const size_t esz = dtype == BV_DTYPE_F32 ? 4 : 2;
     const size_t row_bytes = static_cast<size_t>(V) * esz;
     // only the 128-bit path exists here: rows of whole 16-byte vectors on 16-byte aligned bases
     if (row_bytes % 16 != 0 || !aligned_to(tgt, 16) || !aligned_to(drf, 16)) return BV_ERR_UNSUPPORTED;
-    if (!aligned_to(tok, 4) || !aligned_to(uni, 4) || !aligned_to(ot, 4) || !aligned_to(ol, 4))
-        return BV_ERR_INVALID_ARG;
     if (B == 0) return BV_OK;
 
     std::lock_guard<std::mutex> lock(g_na_mu);
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BV_ERR_CUDA;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return bv::note_cuda_error(e);
+    if (dev < 0 || dev >= kMaxDevices) return BV_ERR_UNSUPPORTED;
     NoAllocDevice& d = g_na[dev];
     if (!d.ready) {
         // Set-up, once per device with that device current.  In host code the array's name only
         // stands for the symbol; the address a kernel can use comes from the runtime.
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
-            cudaGetLastError();
-            return BV_ERR_CUDA;
-        }
+        if ((e = cudaGetSymbolAddress(&p, g_noalloc_scratch)) != cudaSuccess) return bv::note_cuda_error(e);
+        if (p == nullptr) return BV_ERR_UNSUPPORTED;
         int major = 0;
-        if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
-            cudaGetLastError();
-            return BV_ERR_CUDA;
-        }
+        if ((e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
+            return bv::note_cuda_error(e);
         if (major < 10) return BV_ERR_UNSUPPORTED;
         d.scratch = static_cast<unsigned char*>(p);
         d.ready = true;
@@ -91,9 +85,9 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // The array keeps what the previous call left: counters, locks and the ready list must
     // start at zero, and so does the status word at the very end of the used part.
-    if (cudaMemsetAsync(d.scratch, 0, zero_bytes, s) != cudaSuccess) { cudaGetLastError(); return BV_ERR_CUDA; }
+    if ((e = cudaMemsetAsync(d.scratch, 0, zero_bytes, s)) != cudaSuccess) return bv::note_cuda_error(e);
     unsigned char* status_word = d.scratch + (need - 256);
-    if (cudaMemsetAsync(status_word, 0, 256, s) != cudaSuccess) { cudaGetLastError(); return BV_ERR_CUDA; }
+    if ((e = cudaMemsetAsync(status_word, 0, 256, s)) != cudaSuccess) return bv::note_cuda_error(e);
 
     bv::FlowScratch fl;
     bv::flow_scratch_layout(d.scratch, B, gamma, plan, &fl);
@@ -108,6 +102,7 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     long long items = static_cast<long long>(fl.total_s1);
     long long nctas = static_cast<long long>(d.sm_count) * per_sm;
     if (nctas > items) nctas = items;
-    if (bv::launch_flow(prm, fl, dtype, static_cast<int>(nctas), s) != cudaSuccess) return BV_ERR_CUDA;
+    if ((e = bv::launch_flow(prm, fl, dtype, static_cast<int>(nctas), s)) != cudaSuccess) return bv::note_cuda_error(e);
+    bv::note_launches(1);
     return BV_OK;
 }

@@ -143,7 +143,6 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
 }  // namespace bv
 
 namespace {
-thread_local int t_sample_cuda_error = 0;
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) % 16) == 0; }
 }  // namespace
 
@@ -155,11 +154,12 @@ extern "C" int bv_sample_draft(const void* logits, const float* uniforms, int ro
     if (dtype != BV_DTYPE_F32 && dtype != BV_DTYPE_BF16) return BV_ERR_INVALID_ARG;
     const size_t row_bytes = static_cast<size_t>(V) * (dtype == BV_DTYPE_F32 ? 4 : 2);
     if (row_bytes % 16 != 0 || !aligned16(logits)) return BV_ERR_UNSUPPORTED;
+    bv::note_launches(0);
     if (rows == 0) return BV_OK;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) { t_sample_cuda_error = static_cast<int>(e); return BV_ERR_CUDA; }
+    if (e != cudaSuccess) return bv::note_cuda_error(e);
     const int grid = rows < 2 * sms ? rows : 2 * sms;
     const float kf = static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -168,6 +168,7 @@ extern "C" int bv_sample_draft(const void* logits, const float* uniforms, int ro
     else
         bv::sample_rows_kernel<bv::kBF16><<<grid, bv::kSAllThreads, 0, st>>>(static_cast<const char*>(logits), uniforms, rows, V, kf, out_tokens, out_lse);
     e = cudaGetLastError();
-    if (e != cudaSuccess) { t_sample_cuda_error = static_cast<int>(e); return BV_ERR_CUDA; }
+    if (e != cudaSuccess) return bv::note_cuda_error(e);
+    bv::note_launches(1);
     return BV_OK;
 }

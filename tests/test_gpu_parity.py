@@ -13,6 +13,7 @@ from parity import run_oracle, run_cuda, compare, assert_parity
 pytestmark = pytest.mark.gpu
 
 ALGOS = [oracle.BLOCK_VERIFY, oracle.TOKEN_VERIFY]
+KERNELS = {"flow": 1, "cluster": 2, "stream": 3}     # values of the library's "kernel" option
 
 
 def parity_case(inp, algo, check_diag=True):
@@ -61,27 +62,27 @@ def test_ragged_vocabularies(V, dtype, algo):
 
 @pytest.mark.parametrize("algo", ALGOS)
 @pytest.mark.parametrize("cluster", [1, 2, 4, 8])
-def test_every_cluster_width(cluster, algo, monkeypatch):
-    monkeypatch.setenv("BV_CLUSTER", str(cluster))
-    monkeypatch.setenv("BV_KERNEL", "cluster")
+def test_every_cluster_width(cluster, algo, bv_options):
+    bv_options("cluster", cluster)
+    bv_options("kernel", KERNELS["cluster"])
     parity_case(random_inputs(19, 4, 24000, "bf16", seed=cluster, T=0.8), algo)
     parity_case(random_inputs(7, 3, 5000, "f32", seed=cluster + 10), algo)
 
 
-@pytest.mark.parametrize("kernel", ["flow", "cluster", "resident", "stream"])
-def test_every_block_verification_kernel(kernel, monkeypatch):
+@pytest.mark.parametrize("kernel", ["flow", "cluster", "stream"])
+def test_every_block_verification_kernel(kernel, bv_options):
     # the library has several kernels for Algorithm 2; each must match the oracle
-    monkeypatch.setenv("BV_KERNEL", kernel)
+    bv_options("kernel", KERNELS[kernel])
     parity_case(random_inputs(40, 5, 24000, "bf16", seed=77, T=0.8), oracle.BLOCK_VERIFY)
     parity_case(random_inputs(9, 3, 4096, "f32", seed=78), oracle.BLOCK_VERIFY)
     parity_case(wl.make_inputs(wl.scaled(wl.CONFIGS["c4"], B=6), "cuda"), oracle.BLOCK_VERIFY)
 
 
 @pytest.mark.parametrize("chunks", [1, 3, 8])
-def test_flow_chunk_counts(chunks, monkeypatch):
-    monkeypatch.setenv("BV_FLOW_CHUNKS", str(chunks))
+def test_flow_chunk_counts(chunks, bv_options):
+    bv_options("flow_chunks", chunks)
     parity_case(random_inputs(21, 4, 16384, "bf16", seed=chunks), oracle.BLOCK_VERIFY)
-    monkeypatch.setenv("BV_FLOW_CTAS", "3")     # far fewer CTAs than items
+    bv_options("flow_ctas", 3)     # far fewer CTAs than items
     parity_case(random_inputs(21, 4, 16384, "bf16", seed=chunks + 1), oracle.BLOCK_VERIFY)
 
 

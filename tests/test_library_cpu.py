@@ -68,3 +68,9 @@ def test_bad_arguments_are_rejected_without_a_device(lib):
 def test_missing_library_fails_loudly(tmp_path):
     with pytest.raises(RuntimeError):
         bv.load_library(str(tmp_path / "nope.so"))
+
+
+def test_options_are_checked_by_name(lib):
+    assert lib.bv_set_option(b"flow_chunks", 0) == 0
+    assert lib.bv_set_option(b"no_such_option", 1) == -1
+    assert lib.bv_set_option(None, 1) == -1

@@ -17,8 +17,10 @@ import ctypes
 import pytest
 import torch
 
+import oracle
 import paper_2403_10444_b200 as bv
 from paper_2403_10444_b200 import workloads as wl
+from parity import run_oracle, compare, assert_parity
 
 pytestmark = pytest.mark.gpu
 
@@ -58,6 +60,9 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point():
         # which is the tolerance the other GPU tests use for tau and the emitted token
         assert torch.equal(ol, want_len)
         assert torch.equal(ot, want_tokens)
+        # and against the CPU oracle, by the rules of the other parity tests
+        ref = run_oracle(oracle.BLOCK_VERIFY, inp)
+        assert_parity(compare(oracle.BLOCK_VERIFY, ref, ot, ol, None, inp), False)
 
 
 def test_problem_beyond_the_fixed_scratch_is_refused():
