@@ -195,10 +195,11 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     prm.wait_limit = opt.wait_limit > 0 ? static_cast<unsigned>(opt.wait_limit) : 0u;
     prm.never_signal = opt.never_signal;
 
-    const bool flow_ok = algo == bv::kBlockVerify && vec && (opt.kernel == 0 || opt.kernel == 1);
+    prm.algo = algo;
+    const bool flow_ok = vec && (opt.kernel == 0 || opt.kernel == 1);
     if ((prm.lse_d != nullptr || prm.greedy) && !flow_ok) return BV_ERR_UNSUPPORTED;
 
-    // Block Verification on 16-byte rows: the flow of independent work items
+    // 16-byte rows: the flow of independent work items (both algorithms)
     if (flow_ok) {
         int& per_sm = d->flow_ctas_per_sm[dtype];
         if (per_sm == 0) {
@@ -212,7 +213,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             const int chunks = (opt.flow_chunks >= 1 && opt.flow_chunks <= bv::kFlowMaxChunks) ? opt.flow_chunks : 0;
             const int pieces = (opt.flow_pieces >= 1 && opt.flow_pieces <= 8) ? opt.flow_pieces : 0;
             // (with supplied draft normalisers a first-sweep item streams one row, not two)
-            const bv::FlowPlan plan = bv::flow_plan(units, B, gamma, nctas, prm.lse_d == nullptr, chunks, pieces);
+            const bv::FlowPlan plan = bv::flow_plan(units, B, gamma, nctas, prm.lse_d == nullptr, chunks, pieces, algo == bv::kTokenVerify);
             size_t zero_bytes = 0;
             const size_t need = bv::flow_scratch_bytes(B, gamma, plan, &zero_bytes);
             StreamSlot* slot = nullptr;

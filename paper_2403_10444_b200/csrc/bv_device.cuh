@@ -33,6 +33,7 @@ struct Params {
     int* status;              // set to 1 if a bounded device-side wait gave up
     int nclusters;            // clusters in the grid
     int greedy;               // flow kernel: Greedy Block Verification (Algorithm 4) instead of Algorithm 2
+    int algo;                 // flow kernel: kBlockVerify (Algorithms 2, 4) or kTokenVerify (Algorithm 1)
     unsigned wait_limit;      // flow kernel: polls after which a bounded wait gives up (0: the built-in limits)
     int never_signal;         // flow kernel, test switch: workers never report an item as swept, so the waits run out
 };

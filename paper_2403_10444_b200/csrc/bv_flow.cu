@@ -184,6 +184,21 @@ __device__ void f_complete_sweep1(const Params& prm, const FlowScratch& fl, cons
     __threadfence();
     const int g = cx.g, b = ri / (g + 1), r = ri % (g + 1);
     f_row_complete<DT>(prm, fl, cx, b, r, lane);
+    if (fl.tv) {
+        if (r < g) { f_tv_row_done<DT>(prm, fl, cx, b, r, lane); return; }
+        // the last target row of a block whose tests have all passed: Y ~ P_gamma
+        if (f_draws_in_sweep1(prm, fl.nch_late)) {
+            f_draw_from_sweep1<DT>(prm, fl, cx, ri, lane);
+            f_tv_finalize(prm, fl, b, g, lane);
+        } else {
+            if (lane == 0) {
+                const unsigned slot = atomicAdd(&fl.counters[kCtrQueued], 1u);
+                atomicExch(&fl.s2q[slot], static_cast<unsigned>(ri) + 1u);
+            }
+            __syncwarp();
+        }
+        return;
+    }
     if (r < g) {
         // the warp that publishes the last of a block's rows 0 .. gamma-1 folds the block
         unsigned n = 0;
@@ -359,7 +374,10 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         auto sweep1_desc = [&](unsigned t, FlowDesc& d) {
             const int nch = fl.nch;
             const int ch = static_cast<int>(t % nch);
-            const int r = static_cast<int>(t / nch) % g, b = static_cast<int>(t / nch) / g;
+            // Block Verification goes block by block (a block's rows are wanted together); Algorithm 1
+            // row by row over all blocks (a block's next row matters only if the one before passed)
+            const int r = fl.tv ? static_cast<int>(t / nch) / cx.B : static_cast<int>(t / nch) % g;
+            const int b = fl.tv ? static_cast<int>(t / nch) % cx.B : static_cast<int>(t / nch) / g;
             const int ri = b * (g + 1) + r;
             // (with supplied draft normalisers the first sweep has nothing to learn from the draft row)
             d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = prm.lse_d == nullptr;
@@ -399,10 +417,12 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             for (unsigned spins = 0; (e = ld_volatile(&fl.lq[t / fl.nch_late])) == 0u; ++spins)
                 if (spins > lim_nap) { if (prm.status) atomicExch(prm.status, 1); return false; }
             const int ri = static_cast<int>(e - 1u);
-            d.kind = kSweep1; d.ri = ri; d.ch = t % fl.nch_late; d.have_q = 0;
+            const int r = ri % (g + 1), b = ri / (g + 1);
+            // (a last target row, or a row pair that Algorithm 1 asks for once the tests before it have passed)
+            d.kind = kSweep1; d.ri = ri; d.ch = t % fl.nch_late; d.have_q = r < g && prm.lse_d == nullptr;
             item_range(cx.units, fl.nch_late, d.ch, d.u0, d.u1);
             d.rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
-            d.rowQ = nullptr;
+            d.rowQ = d.have_q ? static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes : nullptr;
             d.cp = 1.f; d.nMP = 0.f; d.nMQ = 0.f;
             return true;
         };
@@ -687,7 +707,11 @@ size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_b
     z += 2 * up256(rows * sizeof(unsigned));        // row_cnt, s2_cnt
     z += 3 * up256(static_cast<size_t>(B) * sizeof(unsigned));   // cand_cnt, rows_in, bad
     z += 2 * up256(rows * sizeof(unsigned));        // rel, s2q
-    z += up256(static_cast<size_t>(B) * sizeof(unsigned));       // lq
+    z += up256(rows * sizeof(unsigned));            // lq
+    if (plan.tv_spec > 0) {
+        z += 3 * up256(static_cast<size_t>(B) * sizeof(unsigned long long));   // tv_acc, tv_done, tv_badrows
+        z += 2 * up256(static_cast<size_t>(B) * sizeof(unsigned));             // tv_front, tv_decided
+    }
     if (zero_bytes) *zero_bytes = z;
     size_t n = z;
     n += up256(rows * plan.part_stride() * sizeof(RowZ));   // part
@@ -698,6 +722,7 @@ size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_b
     n += up256(rows * segs * sizeof(float));        // seg_tot
     n += up256(rows * sizeof(double));              // S
     n += up256(rows * sizeof(int));                 // cand
+    n += up256(static_cast<size_t>(B) * sizeof(int));   // tv_tau
     return n;
 }
 
@@ -714,7 +739,19 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->bad = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
     fl->rel = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
     fl->s2q = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
-    fl->lq = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
+    fl->lq = reinterpret_cast<unsigned*>(take(rows * sizeof(unsigned)));
+    fl->tv = plan.tv_spec > 0;
+    fl->tv_spec = plan.tv_spec;
+    fl->tv_ahead = plan.tv_ahead;
+    fl->tv_acc = fl->tv_done = fl->tv_badrows = nullptr;
+    fl->tv_front = fl->tv_decided = nullptr;
+    if (plan.tv_spec > 0) {
+        fl->tv_acc = reinterpret_cast<unsigned long long*>(take(static_cast<size_t>(B) * sizeof(unsigned long long)));
+        fl->tv_done = reinterpret_cast<unsigned long long*>(take(static_cast<size_t>(B) * sizeof(unsigned long long)));
+        fl->tv_badrows = reinterpret_cast<unsigned long long*>(take(static_cast<size_t>(B) * sizeof(unsigned long long)));
+        fl->tv_front = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
+        fl->tv_decided = reinterpret_cast<unsigned*>(take(static_cast<size_t>(B) * sizeof(unsigned)));
+    }
     fl->part = reinterpret_cast<RowZ*>(take(rows * plan.part_stride() * sizeof(RowZ)));
     fl->rowZ = reinterpret_cast<RowZ*>(take(rows * sizeof(RowZ)));
     fl->pchain = reinterpret_cast<double*>(take(static_cast<size_t>(B) * (gamma + 2) * sizeof(double)));
@@ -724,9 +761,10 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->seg_tot = reinterpret_cast<float*>(take(rows * segs * sizeof(float)));
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
+    fl->tv_tau = reinterpret_cast<int*>(take(static_cast<size_t>(B) * sizeof(int)));
     fl->nch = plan.nch;
     fl->part_stride = plan.part_stride();
-    fl->total_s1 = static_cast<unsigned>(B) * gamma * plan.nch;
+    fl->total_s1 = static_cast<unsigned>(B) * (plan.tv_spec > 0 ? plan.tv_spec : gamma) * plan.nch;
     fl->nch_late = plan.nch_late;
     fl->np = plan.np;
     fl->depth = 3;
@@ -744,7 +782,7 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
 //   Second sweep, and the first sweep of a last target row that turns out to be wanted: only few rows
 //   are concerned and a block's candidates are swept one after the other, so these rows are cut into
 //   pieces of about 4000 vectors that many CTAs share.
-FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces) {
+FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces, bool token_verify) {
     FlowPlan pl{};
     long long np = units / 3500;
     if (np < 1) np = 1;
@@ -755,10 +793,29 @@ FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair
     long long nch = (row_units + 8000) / 16000;
     if (nch < 1) nch = 1;
     if (nch > 8) nch = 8;
-    const long long rows = static_cast<long long>(B) * gamma;
+    // (Algorithm 1 starts with one row of every block, or a few: that is what has to fill the GPU)
+    const long long rows = static_cast<long long>(B) * (token_verify ? 1 : gamma);
     while (nch < 8 && rows * nch < 4 * nctas && row_units / (nch + 1) >= 2048) ++nch;
     pl.nch = chunks > 0 ? chunks : static_cast<int>(nch);
     if (chunks > pl.nch_late && chunks <= 8) pl.nch_late = chunks;
+    // Algorithm 1.  Where one row pair of every block is more than about 100 MB (17 us of streaming, what a
+    // dependent row costs in latency), rows are read strictly on demand: one row of every block from the
+    // start, the next only when the test before it has passed, so nothing beyond the first rejection is
+    // read.  Smaller batches leave the GPU idle while a block waits for its next row: there, as many rows
+    // from the start as it takes to give every CTA an item (at least two), and once all of those have
+    // passed, which marks a draft that is mostly accepted, all the remaining rows at once.
+    pl.tv_spec = 0;
+    pl.tv_ahead = 1;
+    if (token_verify) {
+        pl.tv_spec = 1;
+        const long long pair_bytes = units * 32;
+        if (static_cast<long long>(B) * pair_bytes <= 100000000LL) {
+            long long k = (nctas + static_cast<long long>(B) * pl.nch - 1) / (static_cast<long long>(B) * pl.nch);
+            if (k < 2) k = 2;
+            pl.tv_spec = static_cast<int>(k > gamma ? gamma : k);
+            pl.tv_ahead = gamma;
+        }
+    }
     return pl;
 }
 

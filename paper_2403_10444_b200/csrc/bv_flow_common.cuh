@@ -103,7 +103,11 @@ __device__ __forceinline__ RowZ load_rowz(const RowZ* p) {
 }
 
 // chunks of row r of a block in its first sweep
-__device__ __forceinline__ int f_nch_row(const FlowScratch& fl, int r, int g) { return r == g ? fl.nch_late : fl.nch; }
+// (rows whose first sweep is asked for on demand - a last target row, a row of Algorithm 1 beyond the
+// ones swept from the start - are cut into nch_late chunks)
+__device__ __forceinline__ int f_nch_row(const FlowScratch& fl, int r, int g) {
+    return (r == g || (fl.tv && r >= fl.tv_spec)) ? fl.nch_late : fl.nch;
+}
 
 struct FlowCtx {
     int g, V, B, units;
@@ -350,6 +354,112 @@ static __device__ void f_position_done(const Params& prm, const FlowScratch& fl,
     if (n + done == static_cast<unsigned>(g) + 1u) f_finalize_block(prm, fl, b, lane);
 }
 
+// ================= Token Verification (Algorithm 1) on the same work items =================
+// Row r feeds one acceptance test, eta_{r+1} <= min(P_r(X_{r+1}) / Q_r(X_{r+1}), 1), which needs that
+// row's normalisers only; tau is the number of tests that pass before the first one that fails, and
+// Y is drawn from Eq. "pres-token" at position tau (one second sweep of that row pair with p = 1), or
+// from P_gamma.  Rows 0 .. tv_spec-1 of every block are swept from the start; a further row is
+// asked for when every test before it has passed, so no row beyond the first rejection is read
+// unless it was among the first ones.
+
+// ---- the end of a block of Algorithm 1 (one warp): X_1 .. X_tau, Y, diagnostics ----
+static __device__ void f_tv_finalize(const Params& prm, const FlowScratch& fl, int b, int tau, int lane) {
+    const int g = prm.gamma;
+    __threadfence();
+    const size_t row0 = static_cast<size_t>(b) * (g + 1);
+    int32_t* ot = prm.out_tokens + static_cast<size_t>(b) * (g + 1);
+    const int32_t* X = prm.tok + static_cast<size_t>(b) * g;
+    const int y = __ldcg(&fl.cand[row0 + tau]);
+    const unsigned long long badrows = *reinterpret_cast<const volatile unsigned long long*>(&fl.tv_badrows[b]);
+    const int last_pair = tau < g ? tau : g - 1;             // row pairs 0 .. last_pair were needed
+    bool bad = (badrows & (last_pair >= 63 ? ~0ull : ((2ull << last_pair) - 1ull))) != 0ull;
+    if (tau == g && ld_volatile(&fl.bad[b]) != 0u) bad = true;
+    for (int i = lane; i <= g; i += 32) ot[i] = bad ? -1 : (i < tau ? X[i] : (i == tau ? y : -1));
+    if (lane == 0) prm.out_len[b] = bad ? -1 : tau + 1;
+    if (f_all_positions(prm)) {
+        const double ln2 = 0.693147180559945309417232;
+        const float nanf_ = __int_as_float(0x7fc00000);
+        for (int i = lane; i <= g; i += 32) {
+            const size_t o1 = row0 + i, o0 = static_cast<size_t>(b) * g + i;
+            const bool read_t = i <= tau, read_d = i <= last_pair;
+            const RowZ z = load_rowz(&fl.rowZ[row0 + i]);
+            // h_i = min(ratio_i, 1) for the tests made: i = 1 .. min(tau + 1, gamma)
+            float h = nanf_;
+            if (i == 0) h = 1.f;
+            else if (i <= tau + 1 && i <= g) h = static_cast<float>(fmin(__ldcg(&fl.ratio[row0 + i - 1]), 1.0));
+            if (prm.out_p) prm.out_p[o1] = nanf_;
+            if (prm.out_h) prm.out_h[o1] = h;
+            if (prm.out_lse_t) prm.out_lse_t[o1] = read_t ? static_cast<float>((static_cast<double>(z.MP) + log2(z.ZP)) * ln2) : nanf_;
+            if (i < g && prm.out_S) prm.out_S[o0] = i == tau ? static_cast<float>(__ldcg(&fl.S[row0 + i])) : nanf_;
+            if (i < g && prm.out_lse_d) prm.out_lse_d[o0] = read_d ? static_cast<float>((static_cast<double>(z.MQ) + log2(z.ZQ)) * ln2) : nanf_;
+        }
+    }
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) atomicAdd(&fl.counters[kCtrBlocks], 1u);
+}
+
+// ---- row r of a block of Algorithm 1 is complete, its normalisers and ratio published (one warp) ----
+template <int DT>
+__device__ void f_tv_row_done(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int r, int lane) {
+    const int g = cx.g;
+    const size_t row0 = static_cast<size_t>(b) * (g + 1);
+    if (lane == 0 && r < g) {
+        const double ratio = __ldcg(&fl.ratio[row0 + r]);     // 0 for a row with a data fault: the test fails
+        const double h = fmin(ratio, 1.0);
+        const bool pass = h > 0.0 && static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + r]) <= h;
+        // the verdict first, then the fact that it is in: whoever sees the second sees the first
+        if (pass) atomicOr(&fl.tv_acc[b], 1ull << r);
+        __threadfence();
+        atomicOr(&fl.tv_done[b], 1ull << r);
+        __threadfence();
+        const unsigned long long a = *reinterpret_cast<const volatile unsigned long long*>(&fl.tv_acc[b]);
+        const unsigned long long dn = *reinterpret_cast<const volatile unsigned long long*>(&fl.tv_done[b]);
+        int f = a == ~0ull ? 64 : __ffsll(static_cast<long long>(~a)) - 1;   // tests 1 .. f have passed
+        if (f > g) f = g;
+        if (f == g || (dn >> f & 1ull)) {
+            // tau = f: every test has passed, or test f + 1 has been made and failed.  The warp whose
+            // update completes the picture sees it; several may, one acts.
+            if (atomicCAS(&fl.tv_decided[b], 0u, 1u) == 0u) {
+                fl.tv_tau[b] = f;
+                if (f == g) {             // Y ~ P_gamma: the last target row is asked for
+                    const unsigned slot = atomicAdd(&fl.counters[kCtrLateQueued], 1u);
+                    atomicExch(&fl.lq[slot], static_cast<unsigned>(row0 + g) + 1u);
+                } else {                  // Y from Eq. "pres-token": one second sweep of row pair f with p = 1
+                    fl.cscale[row0 + f] = static_cast<float>(__ldcg(&fl.zratio[row0 + f]));
+                    __threadfence();
+                    const unsigned slot = atomicAdd(&fl.counters[kCtrQueued], 1u);
+                    atomicExch(&fl.s2q[slot], static_cast<unsigned>(row0 + f) + 1u);
+                }
+            }
+        } else {
+            // Every test before row f has passed.  Once that includes all the rows swept from the start,
+            // rows up to f + tv_ahead - 1 are asked for, those of them that have not been yet (tv_ahead
+            // is 1 when one row of every block fills the GPU, so that nothing beyond the first rejection
+            // is read; all the rest for small batches, whose chain of dependent rows would otherwise
+            // leave most of the GPU idle).
+            // (a block that has passed two tests or more is likely to pass more, and such blocks are few
+            // unless the draft is good: it asks for as many rows again as it has passed, which halves
+            // the chain of its dependent rows at the price of at most as many rows read in vain)
+            const int ahead = fl.tv_ahead > f ? fl.tv_ahead : (f >= 2 ? f : 1);
+            int want = f >= fl.tv_spec ? f + ahead : 0;       // (rows from the start that are still out: nothing yet)
+            if (want > g) want = g;
+            want -= fl.tv_spec;
+            for (int tries = 0; tries < 64 && want > 0; ++tries) {
+                const unsigned have = ld_volatile(&fl.tv_front[b]);
+                if (have >= static_cast<unsigned>(want)) break;
+                if (atomicCAS(&fl.tv_front[b], have, static_cast<unsigned>(want)) != have) continue;
+                const unsigned n = static_cast<unsigned>(want) - have;
+                const unsigned slot = atomicAdd(&fl.counters[kCtrLateQueued], n);
+                for (unsigned j = 0; j < n; ++j)
+                    atomicExch(&fl.lq[slot + j], static_cast<unsigned>(row0 + fl.tv_spec + have + j) + 1u);
+                break;
+            }
+        }
+    }
+    __syncwarp();
+}
+
 // ---- all rows 0 .. gamma-1 of a block have their normalisers: the prefix recursion
 // p_{c+1} = min(p_c ratio_c, 1) (Eq. "def_as"; Algorithm 4 does not clip), what becomes of every
 // position's second sweep, and the start of the first ones (one warp; lanes c and c + 32 speak for
@@ -490,7 +600,11 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
             fl.ratio[rowi] = bad ? 0.0 : exp2((zp - zq) * cx.kd - (MP - MQ)) * (ZQ / ZP);
             fl.zratio[rowi] = ZQ / ZP;
         }
-        if (bad) atomicOr(&fl.bad[b], 1u);
+        if (bad) {
+            // (Algorithm 1 reads rows 0 .. tau only: a fault counts if its row is among them)
+            if (fl.tv && have_q) atomicOr(&fl.tv_badrows[b], 1ull << r);
+            else atomicOr(&fl.bad[b], 1u);
+        }
     }
     __threadfence();
     __syncwarp();
@@ -555,8 +669,9 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
         int s0, s1;
         range(sel, s0, s1);
         found = f_rescan<DT>(rowP, rowQ, s0, s1, lane, cx.kf, cp, nMP, nMQ, t - before);
-    } else if (have_q && r == 0 && total == 0.f) {
-        // empty residual at position 0 (P_0 and Q_0 coincide bit for bit): sample P_0 with the same
+    } else if (have_q && (r == 0 || fl.tv) && total == 0.f) {
+        // empty residual where it can be selected - position 0, or the stopping position of
+        // Algorithm 1 - (P_r and Q_r coincide bit for bit): sample P_r with the same
         // uniform.  Two plain passes over the whole row by this warp: rare, so speed does not matter.
         float tot = 0.f;
         for (int base2 = 0; base2 < cx.units; base2 += 32) {
@@ -569,7 +684,8 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
     }
     if (lane == 0) fl.cand[ri] = found;
     __syncwarp();
-    f_position_done(prm, fl, b, r, lane);
+    if (fl.tv) f_tv_finalize(prm, fl, b, r, lane);
+    else f_position_done(prm, fl, b, r, lane);
 }
 
 }  // namespace bv

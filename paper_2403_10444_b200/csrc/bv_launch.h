@@ -38,7 +38,19 @@ struct FlowScratch {
     unsigned* s2_cnt;     // [B (gamma+1)] sweep-2 chunks finished per position
     unsigned* cand_cnt;   // [B] positions with a candidate
     unsigned* rows_in;    // [B] rows 0 .. gamma-1 whose normalisers are published
-    unsigned* bad;        // [B] data fault seen
+    unsigned* bad;        // [B] data fault seen (Token Verification: in the last target row)
+    // Token Verification (Algorithm 1): bit r of tv_done = the acceptance test that row r feeds has been made, of
+    // tv_acc = it passed, of tv_badrows = row r holds a data fault; tv_front = rows beyond the first tv_spec
+    // whose first sweep has been asked for; tv_decided = tau is known; tv_tau = tau
+    unsigned long long* tv_acc;
+    unsigned long long* tv_done;
+    unsigned long long* tv_badrows;
+    unsigned* tv_front;
+    unsigned* tv_decided;
+    int* tv_tau;
+    int tv;               // the launch runs Algorithm 1
+    int tv_spec;          // rows 0 .. tv_spec-1 of every block are swept from the start, the others once all before them passed
+    int tv_ahead;         // rows asked for beyond the last test that passed (1: none is read in vain)
     unsigned* rel;        // [B (gamma+1)] what becomes of the position's second sweep (0 until the block is folded)
     unsigned* s2q;        // [B (gamma+1)] queue of rows whose second sweep has been started (row index + 1)
     unsigned* lq;         // [B] queue of last target rows whose first sweep has been asked for (row index + 1)
@@ -65,11 +77,13 @@ constexpr int kFlowMaxChunks = 32;
 // last target row (swept on demand), pieces per row in the second sweep.
 struct FlowPlan {
     int nch, nch_late, np;
+    int tv_spec;          // Token Verification: rows of every block swept from the start (0: Block Verification)
+    int tv_ahead;         // Token Verification: rows asked for beyond the last test that passed
     int part_stride() const { return nch > nch_late ? nch : nch_late; }
 };
 // units: 16-byte vectors per row; pair_items: false when the first sweep streams one row per item
 // (supplied draft normalisers); chunks / pieces > 0 force the chunk count / the piece count.
-FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces);
+FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces, bool token_verify = false);
 size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_bytes);
 void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, FlowScratch* fl);
 int flow_max_ctas_per_sm(int dtype);

@@ -98,6 +98,7 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     prm.kd = kd;
     prm.kf = static_cast<float>(kd);
     prm.out_tokens = ot; prm.out_len = ol;
+    prm.algo = bv::kBlockVerify;
     prm.status = reinterpret_cast<int*>(status_word);
     long long items = static_cast<long long>(fl.total_s1);
     long long nctas = static_cast<long long>(d.sm_count) * per_sm;
