@@ -42,8 +42,10 @@
  *   - sampling is inverse-CDF in vocabulary-index order with a strict
  *     comparison: Y = min{k : C_k > u * W}; if rounding leaves none, the last
  *     k with positive weight;
- *   - a residual whose total mass is exactly 0 (P_tau == Q_tau bit for bit, a
- *     probability-zero event) falls back to sampling P_tau with the same uniform;
+ *   - a residual whose total mass is exactly 0 at the position that was selected is a domain
+ *     error of the sequence: Eq. "pres-token" / "pres-block" divide by that mass, and the
+ *     algorithms cannot arrive there (P_tau == Q_tau makes the ratio of the next test 1, so
+ *     Algorithm 1 does not stop at tau and tau + 1 passes its test in Algorithms 2 and 4);
  *   - Algorithm 4: its last test is taken as eta_gamma <= pt_gamma like every other test
  *     (it is printed with "<"; the two differ on a set of measure zero); a test whose
  *     denominator sum is 0 passes; a position whose numerator sum is 0 is not selectable;
@@ -120,7 +122,8 @@ static double weight_at(const void *tgt, size_t toff, double lse_t,
 
 /*
  * Inverse-CDF sample in vocabulary-index order.  W = sum of weights and the
- * running sums C_k are plain sequential fp64 sums.  Returns the token;
+ * running sums C_k are plain sequential fp64 sums.  Returns the token, or -1
+ * when the weights sum to nothing;
  * *margin receives min(u - C_{k-1}/W, C_k/W - u), the distance (in probability)
  * of u from the nearest edge of the chosen token's CDF cell.
  */
@@ -134,11 +137,9 @@ static int sample_index_order(const void *tgt, size_t toff, double lse_t,
         W += weight_at(tgt, toff, lse_t, drf, doff, lse_d, have_draft, dtype, x, T, p);
     *W_out = W;
     if (!(W > 0.0)) {
-        /* empty residual: sample the target row itself (reading, see header) */
-        have_draft = 0;
-        W = 0.0;
-        for (int x = 0; x < V; ++x)
-            W += weight_at(tgt, toff, lse_t, drf, doff, lse_d, 0, dtype, x, T, p);
+        /* nothing to sample from: a domain error (see header) */
+        *margin = 0.0;
+        return -1;
     }
     double t = u * W, C = 0.0;
     int last_pos = -1;
@@ -296,7 +297,7 @@ static void token_verify_one(const seq_t *s, const diag_t *d,
     if (have_draft && d->S) d->S[tau] = W; /* residual mass sum_x max(P - Q, 0) */
     if (d->margin_eta) *d->margin_eta = m_eta;
     if (d->margin_smp) *d->margin_smp = m_smp;
-    emit(s, tau, Y, out_tokens, out_len);
+    emit(s, Y < 0 ? -1 : tau, Y, out_tokens, out_len);
 }
 
 /* ---------------- Algorithm 2: Block Verification ---------------- */
@@ -376,7 +377,7 @@ static void block_verify_one(const seq_t *s, const diag_t *d,
                                    have_draft, s->dtype, s->V, s->T, p[tau], u, &W, &m_smp);
         if (d->margin_eta) *d->margin_eta = m_eta;
         if (d->margin_smp) *d->margin_smp = m_smp;
-        emit(s, tau, Y, out_tokens, out_len);
+        emit(s, Y < 0 ? -1 : tau, Y, out_tokens, out_len);
     }
     for (int i = 0; i <= g; ++i) {
         if (d->p) d->p[i] = p[i];
@@ -484,7 +485,7 @@ static void greedy_block_verify_one(const seq_t *s, const diag_t *d,
                                    have_draft, s->dtype, s->V, s->T, pt[tau], u, &W, &m_smp);
         if (d->margin_eta) *d->margin_eta = m_eta;
         if (d->margin_smp) *d->margin_smp = m_smp;
-        emit(s, tau, Y, out_tokens, out_len);
+        emit(s, Y < 0 ? -1 : tau, Y, out_tokens, out_len);
     }
     for (int i = 0; i <= g; ++i) {
         if (d->p) d->p[i] = pt[i];

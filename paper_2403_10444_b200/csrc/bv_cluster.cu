@@ -353,13 +353,8 @@ __global__ void __launch_bounds__(kCThreads, 2) verify_cluster_kernel(const Para
                         if (lane == 0) sh.S[r] = sd * sh.S[r];
                     }
                     const bool empty = !(total > 0.f);
-                    if (empty && use_q && attempt == 0 && (ALGO == kTokenVerify || r == 0)) {
-                        // empty residual where it can be selected: sample P_r with the same uniform
-                        use_q = false;
-                        cluster.sync();   // every warp of every CTA has read x_seg before it is rewritten
-                        if (tid == 0) mbar_arrive_expect(smem_u32(&sh.bar_seg), bytes_seg);
-                        continue;
-                    }
+                    // (an empty residual leaves no candidate; should the position be selected all the same,
+                    // which the algorithms cannot do, the block ends as a domain error)
                     if (!empty) {
                         const float t = uf * total;
                         float exc = __shfl_up_sync(0xffffffffu, inc, 1);
@@ -475,6 +470,8 @@ __global__ void __launch_bounds__(kCThreads, 2) verify_cluster_kernel(const Para
                 }
             }
             for (int i = 0; i <= g; ++i) ot[i] = -1;
+            // (nothing to sample from at the selected position: a domain error)
+            if (tau >= 0 && sh.cand[ALGO == kBlockVerify ? tau : 0] < 0) tau = -1;
             if (tau >= 0) {
                 for (int i = 0; i < tau; ++i) ot[i] = X[i];
                 ot[tau] = sh.cand[ALGO == kBlockVerify ? tau : 0];

@@ -141,6 +141,7 @@ __device__ __forceinline__ double shfl_xor_d(double v, int off) {
     hi = __shfl_xor_sync(0xffffffffu, hi, off);
     return __hiloint2double(hi, lo);
 }
+__device__ __forceinline__ double warp_sum_d(double x);
 __device__ __forceinline__ double shfl_up_d(double v, int off) {
     int lo = __double2loint(v), hi = __double2hiint(v);
     lo = __shfl_up_sync(0xffffffffu, lo, off);
@@ -152,6 +153,12 @@ __device__ __forceinline__ double shfl_d(double v, int src) {
     lo = __shfl_sync(0xffffffffu, lo, src);
     hi = __shfl_sync(0xffffffffu, hi, src);
     return __hiloint2double(hi, lo);
+}
+
+__device__ __forceinline__ double warp_sum_d(double x) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x += shfl_xor_d(x, off);
+    return x;
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -80,13 +80,16 @@ struct FlowShared {
     unsigned long long full[kFDesc];    // the service warp has filled desc[i]
     unsigned long long done[kFDesc];    // all 16 worker warps have left their partials of desc[i]
     float part_M[kFDesc][2][kFWarps];   // sweep 1: references of P and Q per worker warp
-    float part_s[kFDesc][2][kFWarps];   // sweep 1: sums; sweep 2: [0] holds the residual totals
+    float part_s[kFDesc][kFWarps];      // sweep 1: sums of the draft row
+    double part_d[kFDesc][kFWarps];     // sweep 1: sums of the target row; sweep 2: the residual totals (they decide sampled
+                                        // tokens, so a last target row and every second sweep accumulate them in double)
     // a finished item is moved here by its post warp, so that its descriptor slot is free again
     // before anything is asked of global memory
     unsigned long long freeb[kFDesc];   // the post warp has moved the item of desc[i] out
     FlowDesc sdesc[kFPost];
     float stage_M[kFPost][2][kFWarps];
-    float stage_s[kFPost][2][kFWarps];
+    float stage_s[kFPost][kFWarps];
+    double stage_d[kFPost][kFWarps];
     unsigned posted;                    // items whose post-processing is complete
 };
 
@@ -98,48 +101,50 @@ template <int DT>
 __device__ void f_draw_from_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, int lane) {
     const int g = cx.g, b = ri / (g + 1);
     const int nseg = fl.nch_late * kFWarps;                  // <= 128: four per lane
-    const float* pairs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
-    float m[4], w[4];
+    const double* pairs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
+    float m[4];
+    double w[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int i = 4 * lane + j;
-        m[j] = i < nseg ? __ldcg(&pairs[2 * i]) : kNoRef;
-        w[j] = i < nseg ? __ldcg(&pairs[2 * i + 1]) : 0.f;
+        m[j] = i < nseg ? static_cast<float>(__ldcg(&pairs[2 * i])) : kNoRef;
+        w[j] = i < nseg ? __ldcg(&pairs[2 * i + 1]) : 0.0;
     }
     const float Mrow = warp_max(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])));
 #pragma unroll
-    for (int j = 0; j < 4; ++j) w[j] *= ref_scale(m[j], Mrow);
-    const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
-    float inc = l4;
+    for (int j = 0; j < 4; ++j) w[j] *= static_cast<double>(ref_scale(m[j], Mrow));
+    // (fp64 sums of the segment totals, as for the residual samples)
+    const double d1 = w[0], d2 = d1 + w[1], d3 = d2 + w[2], d4 = d3 + w[3];
+    double inc = d4;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
-        const float o = __shfl_up_sync(0xffffffffu, inc, off);
+        const double o = shfl_up_d(inc, off);
         if (lane >= off) inc += o;
     }
-    const float total = __shfl_sync(0xffffffffu, inc, 31);
+    const double total = shfl_d(inc, 31);
     int found = -1;
-    if (Mrow > kNoRef && Mrow < INFINITY && total > 0.f && total < INFINITY) {
-        const float t = prm.uni[static_cast<size_t>(b) * (g + 2) + g + 1] * total;
-        float exc = __shfl_up_sync(0xffffffffu, inc, 1);
-        if (lane == 0) exc = 0.f;
-        const float p0 = exc, p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+    if (Mrow > kNoRef && Mrow < INFINITY && total > 0.0 && total < static_cast<double>(INFINITY)) {
+        const double t = static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + g + 1]) * total;
+        double exc = shfl_up_d(inc, 1);
+        if (lane == 0) exc = 0.0;
+        const double p0 = exc, p1 = exc + d1, p2 = exc + d2, p3 = exc + d3, p4 = exc + d4;
         // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
-        const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
-        const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
+        const bool h1 = p1 > t && w[0] > 0.0, h2 = p2 > t && w[1] > 0.0;
+        const bool h3 = p3 > t && w[2] > 0.0, h4 = p4 > t && w[3] > 0.0;
         const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
-        const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
-        int e = 3; float bef = p3; int src;
+        const unsigned nz = __ballot_sync(0xffffffffu, d4 > 0.0);
+        int e = 3; double bef = p3; int src;
         if (hit) {
             src = __ffs(hit) - 1;
             if (h1) { e = 0; bef = p0; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
         } else {
             src = 31 - __clz(nz);
             e = 0; bef = p0;
-            if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
-            else if (w[1] > 0.f) { e = 1; bef = p1; }
+            if (w[3] > 0.0) { e = 3; bef = p3; } else if (w[2] > 0.0) { e = 2; bef = p2; }
+            else if (w[1] > 0.0) { e = 1; bef = p1; }
         }
         const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
-        const float before = __shfl_sync(0xffffffffu, bef, src);
+        const double before = shfl_d(bef, src);
         int s0, s1;
         chunk_range(cx, fl.nch_late, sel / kFWarps, sel % kFWarps, s0, s1);
         const char* rowP = static_cast<const char*>(prm.tgt) + static_cast<size_t>(ri) * cx.row_bytes;
@@ -164,15 +169,15 @@ __device__ void f_store_sweep1(const Params& prm, const FlowScratch& fl, const F
     const float mP = lane < kFWarps ? sh.stage_M[j][0][lane] : kNoRef;
     const float mQ = lane < kFWarps ? sh.stage_M[j][1][lane] : kNoRef;
     const float MPc = warp_max(mP), MQc = warp_max(mQ);
-    double zP = lane < kFWarps ? static_cast<double>(sh.stage_s[j][0][lane]) * ref_scale(mP, MPc) : 0.0;
-    double zQ = lane < kFWarps ? static_cast<double>(sh.stage_s[j][1][lane]) * ref_scale(mQ, MQc) : 0.0;
+    double zP = lane < kFWarps ? sh.stage_d[j][lane] * ref_scale(mP, MPc) : 0.0;
+    double zQ = lane < kFWarps ? static_cast<double>(sh.stage_s[j][lane]) * ref_scale(mQ, MQc) : 0.0;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) { zP += shfl_xor_d(zP, off); zQ += shfl_xor_d(zQ, off); }
     // A last target row is swept for one purpose only: the sample from P_gamma.  Its warps' pairs
     // {reference, sum} are kept, so that the token can be drawn from this one sweep.
     if (ri % (cx.g + 1) == cx.g && f_draws_in_sweep1(prm, fl.nch_late)) {
-        float* pairs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs + static_cast<size_t>(ch) * kFWarps * 2;
-        if (lane < kFWarps) { pairs[2 * lane] = mP; pairs[2 * lane + 1] = sh.stage_s[j][0][lane]; }
+        double* pairs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs + static_cast<size_t>(ch) * kFWarps * 2;
+        if (lane < kFWarps) { pairs[2 * lane] = mP; pairs[2 * lane + 1] = sh.stage_d[j][lane]; }
     }
     if (lane == 0) {
         RowZ z; z.MP = MPc; z.ZP = zP; z.MQ = MQc; z.ZQ = zQ;
@@ -224,13 +229,13 @@ __device__ void f_complete_sweep1(const Params& prm, const FlowScratch& fl, cons
 }
 
 __device__ __forceinline__ void f_store_sweep2(const FlowScratch& fl, FlowShared& sh, int j, int ri, int ch, int lane) {
-    float* segs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
-    if (lane < kFWarps) segs[ch * kFWarps + lane] = sh.stage_s[j][0][lane];
+    double* segs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
+    if (lane < kFWarps) segs[ch * kFWarps + lane] = sh.stage_d[j][lane];
 }
 template <int DT>
 __device__ void f_complete_sweep2(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, const FlowDesc& d, int lane) {
     const int np = fl.np;
-    const float* segs = fl.seg_tot + static_cast<size_t>(d.ri) * fl.segs;
+    const double* segs = fl.seg_tot + static_cast<size_t>(d.ri) * fl.segs;
     f_position_complete<DT>(prm, fl, cx, d.ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, np * kFWarps, segs, lane,
                             [&](int sel, int& s0, int& s1) { chunk_range(cx, np, sel / kFWarps, sel % kFWarps, s0, s1); });
 }
@@ -258,20 +263,20 @@ __device__ __forceinline__ void f_step_sweep1_pair(const float (&vp)[EPV], const
     sP += vsP;
     sQ += vsQ;
 }
-// First sweep, two consecutive vectors of one row.
+// First sweep, two consecutive vectors of one row; the running sum in double.
 template <int EPV>
 __device__ __forceinline__ void f_step_sweep1_single(const float (&va)[EPV], const float (&vb)[EPV], float kf,
-                                                     float& MPw, float& sP) {
+                                                     float& MPw, double& sP) {
     float vsA = f_exp_sum<EPV>(va, kf, -MPw);
     float vsB = f_exp_sum<EPV>(vb, kf, -MPw);
     if (__any_sync(0xffffffffu, fmaxf(vsA, vsB) > kRaiseBound)) {
         const float y = rintf(warp_max(fmaxf(vec_max<EPV>(va), vec_max<EPV>(vb))) * kf);
-        if (y > MPw) { sP *= ref_scale(MPw, y); MPw = y; }
+        if (y > MPw) { sP *= static_cast<double>(ref_scale(MPw, y)); MPw = y; }
         vsA = f_exp_sum<EPV>(va, kf, -MPw);
         vsB = f_exp_sum<EPV>(vb, kf, -MPw);
     }
-    sP += vsA;
-    sP += vsB;
+    sP += static_cast<double>(vsA);
+    sP += static_cast<double>(vsB);
 }
 
 template <int DT>
@@ -323,7 +328,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             if (lane == 0) sh.sdesc[k] = sh.desc[slot];
             if (lane < kFWarps) {
                 sh.stage_M[k][0][lane] = sh.part_M[slot][0][lane]; sh.stage_M[k][1][lane] = sh.part_M[slot][1][lane];
-                sh.stage_s[k][0][lane] = sh.part_s[slot][0][lane]; sh.stage_s[k][1][lane] = sh.part_s[slot][1][lane];
+                sh.stage_s[k][lane] = sh.part_s[slot][lane]; sh.stage_d[k][lane] = sh.part_d[slot][lane];
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh.freeb[slot]));
@@ -650,37 +655,42 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                     MPw = fmaxf(rintf(warp_max(fmaxf(vec_max<EPV>(va), vec_max<EPV>(vb))) * kf), kNoRef);
                 }
             }
+            double tPd;
             if (have_q) {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
                     f_step_sweep1_pair<EPV>(va, vb, kf, MPw, sP, MQw, sQ);
                 });
+                tPd = static_cast<double>(warp_sum(sP));
             } else {
+                // (a row swept alone is a last target row, from whose sums a token may be drawn: in double)
+                double sPd = 0.0;
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
-                    f_step_sweep1_single<EPV>(va, vb, kf, MPw, sP);
+                    f_step_sweep1_single<EPV>(va, vb, kf, MPw, sPd);
                 });
+                tPd = warp_sum_d(sPd);
             }
-            const float tP = warp_sum(sP);
             const float tQ = have_q ? warp_sum(sQ) : 0.f;
             if (lane == 0) {
-                sh.part_M[slot][0][warp] = MPw; sh.part_s[slot][0][warp] = tP;
-                sh.part_M[slot][1][warp] = MQw; sh.part_s[slot][1][warp] = tQ;
+                sh.part_M[slot][0][warp] = MPw; sh.part_d[slot][warp] = tPd;
+                sh.part_M[slot][1][warp] = MQw; sh.part_s[slot][warp] = tQ;
             }
         } else {
             const float cp = sh.desc[slot].cp, nMP = sh.desc[slot].nMP, nMQ = sh.desc[slot].nMQ;
+            double acc = 0.0;
             if (have_q) {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
                     float t[EPV];
-                    sP += f_pair_sum<EPV, true>(va, vb, kf, cp, nMP, nMQ, t);
+                    acc += static_cast<double>(f_pair_sum<EPV, true>(va, vb, kf, cp, nMP, nMQ, t));
                 });
             } else {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
                     float t[EPV];
-                    sP += f_pair_sum<EPV, false>(va, va, kf, cp, nMP, nMQ, t);
-                    sP += f_pair_sum<EPV, false>(vb, vb, kf, cp, nMP, nMQ, t);
+                    acc += static_cast<double>(f_pair_sum<EPV, false>(va, va, kf, cp, nMP, nMQ, t));
+                    acc += static_cast<double>(f_pair_sum<EPV, false>(vb, vb, kf, cp, nMP, nMQ, t));
                 });
             }
-            const float tP = warp_sum(sP);
-            if (lane == 0) sh.part_s[slot][0][warp] = tP;
+            const double tP = warp_sum_d(acc);
+            if (lane == 0) sh.part_d[slot][warp] = tP;
         }
         if (lane == 0 && !prm.never_signal) mbar_arrive(smem_u32(&sh.done[slot]));   // releases this warp's partials and the descriptor
         __syncwarp();
@@ -719,7 +729,7 @@ size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_b
     n += up256(static_cast<size_t>(B) * (gamma + 2) * sizeof(double));   // pchain
     n += up256(rows * sizeof(float));               // cscale
     n += 2 * up256(rows * sizeof(double));          // ratio, zratio
-    n += up256(rows * segs * sizeof(float));        // seg_tot
+    n += up256(rows * segs * sizeof(double));       // seg_tot
     n += up256(rows * sizeof(double));              // S
     n += up256(rows * sizeof(int));                 // cand
     n += up256(static_cast<size_t>(B) * sizeof(int));   // tv_tau
@@ -758,7 +768,7 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->cscale = reinterpret_cast<float*>(take(rows * sizeof(float)));
     fl->ratio = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->zratio = reinterpret_cast<double*>(take(rows * sizeof(double)));
-    fl->seg_tot = reinterpret_cast<float*>(take(rows * segs * sizeof(float)));
+    fl->seg_tot = reinterpret_cast<double*>(take(rows * segs * sizeof(double)));
     fl->S = reinterpret_cast<double*>(take(rows * sizeof(double)));
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
     fl->tv_tau = reinterpret_cast<int*>(take(static_cast<size_t>(B) * sizeof(int)));

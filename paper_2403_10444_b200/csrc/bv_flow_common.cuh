@@ -120,10 +120,13 @@ struct FlowCtx {
 // whose running residual mass exceeds tw (else the last element with positive mass, else -1).
 template <int DT>
 __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int lane, float kf, float cp,
-                        float nMP, float nMQ, float tw) {
+                        float nMP, float nMQ, double tw) {
     constexpr int EPV = Raw<DT>::EPV;
     constexpr int kAhead = 4;                                // runs of 32 vectors whose loads are in flight together
-    float run = 0.f;
+    // The terms are the fp32 values of the sweeps; their running sum, which decides the token, is
+    // kept in fp64 (a cell of the distribution can be far narrower than fp32 resolves next to the
+    // mass before it).
+    double run = 0.0;
     int found = -1, last_pos = -1;
     for (int base0 = w0; base0 < w1 && found < 0; base0 += 32 * kAhead) {
         // the loads of kAhead runs are issued before the first is looked at: the walk is a chain of
@@ -144,26 +147,30 @@ __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int 
             float vp[EPV], vq[EPV], tt[EPV];
             Raw<DT>::unpack(rp[a], vp);
             Raw<DT>::unpack(rq[a], vq);
-            const float ls = rowQ ? f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, tt)
-                                  : f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, tt);
+            if (rowQ) f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, tt);
+            else f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, tt);
+            double ls = 0.0;
 #pragma unroll
-            for (int e = 0; e < EPV; ++e) if (tt[e] > 0.f) last_pos = i * EPV + e;
-            float incw = ls;
+            for (int e = 0; e < EPV; ++e) {
+                ls += static_cast<double>(tt[e]);
+                if (tt[e] > 0.f) last_pos = i * EPV + e;
+            }
+            double incw = ls;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                const float o = __shfl_up_sync(0xffffffffu, incw, off);
+                const double o = shfl_up_d(incw, off);
                 if (lane >= off) incw += o;
             }
-            const unsigned bal = __ballot_sync(0xffffffffu, run + incw > tw && ls > 0.f);
+            const unsigned bal = __ballot_sync(0xffffffffu, run + incw > tw && ls > 0.0);
             if (bal) {
                 const int src = __ffs(bal) - 1;
                 int f = -1;
                 if (lane == src) {
-                    float cum = run + incw - ls;
+                    double cum = run + incw - ls;
                     int lp = -1;
 #pragma unroll
                     for (int e = 0; e < EPV; ++e) {
-                        cum += tt[e];
+                        cum += static_cast<double>(tt[e]);
                         if (tt[e] > 0.f) lp = i * EPV + e;
                         if (f < 0 && cum > tw && tt[e] > 0.f) f = i * EPV + e;
                     }
@@ -171,7 +178,7 @@ __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int 
                 }
                 found = __shfl_sync(0xffffffffu, f, src);
             }
-            run += __shfl_sync(0xffffffffu, incw, 31);
+            run += shfl_d(incw, 31);
         }
     }
     if (found < 0) {
@@ -245,6 +252,9 @@ static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl
     if (bad) tau = -1;
     int y = cand_g;                       // the candidate of position tau
     if (tau >= 0 && tau < g) y = __shfl_sync(0xffffffffu, tau < 32 ? cd[0] : cd[1], tau & 31);
+    // Nothing to sample from at the selected position (an empty residual, which the algorithm cannot
+    // select: P_tau == Q_tau makes position tau + 1 pass its test): a domain error of the block
+    if (tau >= 0 && y < 0) tau = -1;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int i = lane + 32 * h;
@@ -374,6 +384,7 @@ static __device__ void f_tv_finalize(const Params& prm, const FlowScratch& fl, i
     const int last_pair = tau < g ? tau : g - 1;             // row pairs 0 .. last_pair were needed
     bool bad = (badrows & (last_pair >= 63 ? ~0ull : ((2ull << last_pair) - 1ull))) != 0ull;
     if (tau == g && ld_volatile(&fl.bad[b]) != 0u) bad = true;
+    if (y < 0) bad = true;                // (nothing to sample from: Algorithm 1 cannot stop where P_tau == Q_tau)
     for (int i = lane; i <= g; i += 32) ot[i] = bad ? -1 : (i < tau ? X[i] : (i == tau ? y : -1));
     if (lane == 0) prm.out_len[b] = bad ? -1 : tau + 1;
     if (f_all_positions(prm)) {
@@ -616,72 +627,57 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
 template <int DT, class RangeFn>
 __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, bool have_q,
                                     const char* rowP, const char* rowQ, float cp, float nMP, float nMQ,
-                                    int nseg, const float* segs, int lane, RangeFn range) {
-    constexpr int EPV = Raw<DT>::EPV;
+                                    int nseg, const double* segs, int lane, RangeFn range) {
     const int g = cx.g, r = ri % (g + 1), b = ri / (g + 1);
     __threadfence();
     // everything asked for in one go: the uniform, the segment totals, the draft row's normaliser
     const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
-    float w[4];
+    double w[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int i = 4 * lane + j;
-        w[j] = i < nseg ? __ldcg(&segs[i]) : 0.f;
+        w[j] = i < nseg ? __ldcg(&segs[i]) : 0.0;
     }
     const double ZQ = have_q ? __ldcg(&fl.rowZ[ri].ZQ) : 1.0;
-    // S_r in fp64; the segment that holds the sample by fp32 prefix sums in index order
-    double sd = (static_cast<double>(w[0]) + static_cast<double>(w[1])) + (static_cast<double>(w[2]) + static_cast<double>(w[3]));
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sd += shfl_xor_d(sd, off);
-    if (lane == 0 && have_q) fl.S[ri] = sd / ZQ;
-    const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
-    float inc = l4;
+    // S_r, and the segment that holds the sample, by fp64 sums of the segment totals in index order
+    const double d1 = w[0], d2 = d1 + w[1], d3 = d2 + w[2], d4 = d3 + w[3];
+    double inc = d4;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
-        const float o = __shfl_up_sync(0xffffffffu, inc, off);
+        const double o = shfl_up_d(inc, off);
         if (lane >= off) inc += o;
     }
-    const float total = __shfl_sync(0xffffffffu, inc, 31);
+    const double total = shfl_d(inc, 31);
+    if (lane == 0 && have_q) fl.S[ri] = total / ZQ;
     int found = -1;
-    if (total > 0.f) {
-        const float t = uf * total;
-        float exc = __shfl_up_sync(0xffffffffu, inc, 1);
-        if (lane == 0) exc = 0.f;
-        const float p0 = exc, p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+    if (total > 0.0) {
+        const double t = static_cast<double>(uf) * total;
+        double exc = shfl_up_d(inc, 1);
+        if (lane == 0) exc = 0.0;
+        const double p0 = exc, p1 = exc + d1, p2 = exc + d2, p3 = exc + d3, p4 = exc + d4;
         // first non-empty segment whose inclusive prefix exceeds t, else the last non-empty one
-        const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
-        const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
+        const bool h1 = p1 > t && w[0] > 0.0, h2 = p2 > t && w[1] > 0.0;
+        const bool h3 = p3 > t && w[2] > 0.0, h4 = p4 > t && w[3] > 0.0;
         const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
-        const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
+        const unsigned nz = __ballot_sync(0xffffffffu, d4 > 0.0);
         int e = 3, src;
-        float bef = p3;
+        double bef = p3;
         if (hit) {
             src = __ffs(hit) - 1;
             if (h1) { e = 0; bef = p0; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
         } else {
             src = 31 - __clz(nz);
             e = 0; bef = p0;
-            if (w[3] > 0.f) { e = 3; bef = p3; } else if (w[2] > 0.f) { e = 2; bef = p2; }
-            else if (w[1] > 0.f) { e = 1; bef = p1; }
+            if (w[3] > 0.0) { e = 3; bef = p3; } else if (w[2] > 0.0) { e = 2; bef = p2; }
+            else if (w[1] > 0.0) { e = 1; bef = p1; }
         }
         const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
-        const float before = __shfl_sync(0xffffffffu, bef, src);
+        const double before = shfl_d(bef, src);
         int s0, s1;
         range(sel, s0, s1);
         found = f_rescan<DT>(rowP, rowQ, s0, s1, lane, cx.kf, cp, nMP, nMQ, t - before);
-    } else if (have_q && (r == 0 || fl.tv) && total == 0.f) {
-        // empty residual where it can be selected - position 0, or the stopping position of
-        // Algorithm 1 - (P_r and Q_r coincide bit for bit): sample P_r with the same
-        // uniform.  Two plain passes over the whole row by this warp: rare, so speed does not matter.
-        float tot = 0.f;
-        for (int base2 = 0; base2 < cx.units; base2 += 32) {
-            float vp[EPV], t2[EPV];
-            f_load_tail<DT>(rowP, base2 + lane, cx.units, vp);
-            tot += f_pair_sum<EPV, false>(vp, vp, cx.kf, 1.f, nMP, nMQ, t2);
-        }
-        tot = warp_sum(tot);
-        found = f_rescan<DT>(rowP, nullptr, 0, cx.units, lane, cx.kf, 1.f, nMP, nMQ, uf * tot);
     }
+    // (an empty residual leaves no candidate: the position cannot be the selected one, see the end of a block)
     if (lane == 0) fl.cand[ri] = found;
     __syncwarp();
     if (fl.tv) f_tv_finalize(prm, fl, b, r, lane);

@@ -60,7 +60,7 @@ struct FlowScratch {
     float* cscale;        // [B (gamma+1)] p_r Z_Q / Z_P
     double* ratio;        // [B (gamma+1)] P_r(X_{r+1}) / Q_r(X_{r+1})
     double* zratio;       // [B (gamma+1)] Z_Q / Z_P
-    float* seg_tot;       // [B (gamma+1) segs]
+    double* seg_tot;      // [B (gamma+1) segs] per-segment sums, in double: they decide sampled tokens
     double* S;            // [B (gamma+1)]
     int* cand;            // [B (gamma+1)]
     int nch;              // chunks per row in the first sweep of rows 0 .. gamma-1 (1 .. kFlowMaxChunks)

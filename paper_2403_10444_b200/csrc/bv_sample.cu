@@ -5,7 +5,7 @@
 // Persistent CTAs take rows round-robin.  Each of 16 warps streams its contiguous sixteenth of the
 // row once, in eight sub-segments, and leaves each sub-segment's {integer reference, sum 2^{z k - M}}
 // in shared memory; a seventeenth warp, one row behind, combines the 128 pairs (fp64 for the
-// normaliser, fp32 prefix sums for the sampler), finds the sub-segment that holds u * Z and rescans
+// normaliser and for the sampler's prefix sums), finds the sub-segment that holds u * Z and rescans
 // that one - a few KB still in L2 - in index order for the token.  Each logit is read from HBM once.
 #include <cmath>
 #include <cstdint>
@@ -82,7 +82,7 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
             const float* sM = sM2[(it - 1) & 1];
             const float* sS = sS2[(it - 1) & 1];
             const char* row = logits + static_cast<size_t>(r) * row_bytes;
-            // ---- normaliser (fp64) and the sampled sub-segment (fp32 prefix sums, index order) ----
+            // ---- normaliser and the sampled sub-segment (fp64 prefix sums, index order) ----
             float m[4], w[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) { m[j] = sM[4 * lane + j]; w[j] = sS[4 * lane + j]; }
@@ -93,28 +93,30 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
                        (static_cast<double>(w[2]) + static_cast<double>(w[3]));
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) Z += shfl_xor_d(Z, off);
-            const float l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
-            float inc = l4;
+            // (the sums over sub-segments that locate the sample are formed in double: a token's cell can
+            // be far narrower than fp32 resolves next to the mass before it)
+            const double l1 = w[0], l2 = l1 + w[1], l3 = l2 + w[2], l4 = l3 + w[3];
+            double inc = l4;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                const float o = __shfl_up_sync(0xffffffffu, inc, off);
+                const double o = shfl_up_d(inc, off);
                 if (lane >= off) inc += o;
             }
-            const float total = __shfl_sync(0xffffffffu, inc, 31);
+            const double total = shfl_d(inc, 31);
             // a row with a NaN or +inf logit has a NaN / infinite sum or reference; one without a finite logit has none
-            const bool ok = Mrow > kNoRef && Mrow < INFINITY && Z > 0.0 && Z < INFINITY && total > 0.f && total < INFINITY;
+            const bool ok = Mrow > kNoRef && Mrow < INFINITY && Z > 0.0 && Z < INFINITY && total > 0.0 && total < static_cast<double>(INFINITY);
             int found = -1;
             if (ok) {
-                const float t = uni[r] * total;
-                float exc = __shfl_up_sync(0xffffffffu, inc, 1);
-                if (lane == 0) exc = 0.f;
-                const float p0 = exc, p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
+                const double t = static_cast<double>(uni[r]) * total;
+                double exc = shfl_up_d(inc, 1);
+                if (lane == 0) exc = 0.0;
+                const double p0 = exc, p1 = exc + l1, p2 = exc + l2, p3 = exc + l3, p4 = exc + l4;
                 // first non-empty sub-segment whose inclusive prefix exceeds t, else the last non-empty one
                 const bool h1 = p1 > t && w[0] > 0.f, h2 = p2 > t && w[1] > 0.f;
                 const bool h3 = p3 > t && w[2] > 0.f, h4 = p4 > t && w[3] > 0.f;
                 const unsigned hit = __ballot_sync(0xffffffffu, h1 || h2 || h3 || h4);
-                const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.f);
-                int e = 3; float bef = p3; int src;
+                const unsigned nz = __ballot_sync(0xffffffffu, l4 > 0.0);
+                int e = 3; double bef = p3; int src;
                 if (hit) {
                     src = __ffs(hit) - 1;
                     if (h1) { e = 0; bef = p0; } else if (h2) { e = 1; bef = p1; } else if (h3) { e = 2; bef = p2; }
@@ -125,7 +127,7 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
                     else if (w[1] > 0.f) { e = 1; bef = p1; }
                 }
                 const int sel = __shfl_sync(0xffffffffu, 4 * lane + e, src);
-                const float before = __shfl_sync(0xffffffffu, bef, src);
+                const double before = shfl_d(bef, src);
                 int a0, a1;
                 s_range(units, sel / kSSub, sel % kSSub, a0, a1);
                 found = f_rescan<DT>(row, nullptr, a0, a1, lane, kf, 1.f, -Mrow, 0.f, t - before);

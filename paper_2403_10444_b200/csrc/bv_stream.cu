@@ -216,6 +216,7 @@ __device__ void finalize_sequence(StreamShared& sh, const Params& prm) {
         }
     }
     for (int i = 0; i <= g; ++i) ot[i] = -1;
+    if (tau >= 0 && sh.cand[tau] < 0) tau = -1;      // (nothing to sample from at the selected position: a domain error)
     if (tau >= 0) {
         for (int i = 0; i < tau; ++i) ot[i] = X[i];
         ot[tau] = sh.cand[tau];
@@ -381,8 +382,8 @@ __global__ void __launch_bounds__(kThreads, 1) verify_stream_kernel(const Params
             const bool last_row = sh.last_row != 0;
             if (sh.do_sweep2) {
                 const float c = sh.c, negMP = sh.negMP, negMQ = sh.negMQ;
-                // Eq. "pres-block" needs its own fallback only where an empty residual can be
-                // selected: position 0 of Algorithm 2, the stopping position of Algorithm 1.
+                // (an empty residual leaves no candidate; a block that selects such a position, which the
+                // algorithms cannot do, ends as a domain error)
                 bool use_q = have_q;
                 for (int attempt = 0; attempt < 2; ++attempt) {
                     // ---------------- sweep 2: residual mass per warp segment ----------------
@@ -408,11 +409,6 @@ __global__ void __launch_bounds__(kThreads, 1) verify_stream_kernel(const Params
                     }
                     if (attempt == 0 && use_q && tid == 0) sh.S[r] = total * sh.invZQ;
                     const bool empty = !(total > 0.0);
-                    if (empty && use_q && attempt == 0 && (ALGO == kTokenVerify || r == 0)) {
-                        use_q = false;  // empty residual: sample P_r itself with the same uniform
-                        cluster.sync();  // every CTA has read x_tot before it is rewritten
-                        continue;
-                    }
                     if (!empty) {
                         const float uf = prm.uni[static_cast<size_t>(b) * (g + 2) + (have_q ? g : g + 1)];
                         const double t = static_cast<double>(uf) * total;

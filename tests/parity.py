@@ -6,20 +6,32 @@ Tolerances, from the arithmetic of the CUDA path (fp32 per element, fp64 combina
     fp32 ulp is 1.9e-6);
   - p_i: 1e-5 relative; h_i: 1e-5 h_i + 1e-7 plus the S and p tolerances propagated through
     h = S / (S + 1 - p);
-  - S_i: 1e-5 relative literally where S_i >= 1e-2 p_i; below that the bound is
-    1e-5 S_i + 1e-7 p_i, because S is then the small difference of sums whose own
-    fp32 rounding is 6e-8 p_i; where the oracle has S_i = 0 the CUDA value must be
-    <= 1e-7 p_i (and exactly 0 when the two rows are bit-identical);
+  - S_i: 1e-5 relative literally where S_i >= 2.4e-2 p_i (= 2^-22 / 1e-5, where the bound that
+    follows guarantees it); below that the bound is 1e-5 S_i + 2^-22 p_i: every term of S_i is a
+    difference p_i P_i(x) - Q_i(x) of two exponentials, each evaluated by ex2.approx.ftz.f32,
+    whose documented error bound is 2^-22 relative, and the terms that count add up to at most
+    p_i (measured over the whole sweep: at most 1.7e-7 p_i, 3e-8 p_i rms, unbiased); where the oracle has S_i = 0 the CUDA value must be
+    <= 2^-22 p_i (and exactly 0 when the two rows are bit-identical); the largest value seen
+    there is part of the report;
   - Greedy Block Verification (Algorithm 4): the same bounds with the unclipped product in place
     of p_i; where that product is one or more the acceptance ratio is only required to be >= 1;
   - tau and Y: bit-exact, except for trials in which a uniform lies within 1e-6 of
     the threshold it is compared with: a differing tau needs an eta_i within 1e-6 of
     h_i (oracle margin); a differing Y needs the sampling uniform within 1e-6 of the
-    CDF cell of the CUDA token (recomputed here in fp64).  Both are counted.
+    CDF cell of the CUDA token (recomputed here in fp64).  Both are counted.  Differing taus
+    must stay within 1e-4 of the trials (rounded up).  For Y the bound is
+    trials (1e-4 + 2e-8 V): the kernels form every sum that decides a token in double, but each
+    weight is an ex2.approx.ftz.f32 value with up to 2^-22 relative error, which displaces the
+    CDF by a few 1e-9, and a uniform that close to one of the V cell edges changes cell: about
+    1e-8 V of all trials (measured over the sweep at V = 152064: 3 of 2500 distinct trials).
+
+Every report can be appended, as one JSON line, to the file named by BV_PARITY_LOG.
 """
 from __future__ import annotations
 
-from dataclasses import dataclass
+import json
+import os
+from dataclasses import dataclass, asdict
 
 import numpy as np
 import torch
@@ -27,6 +39,7 @@ import torch
 import oracle
 
 NEAR = 1e-6
+S_FLOOR = 2.0 ** -22      # error bound of one ex2.approx.ftz.f32, relative: what S_i / p_i cannot be trusted below
 
 
 def to_numpy_logits(t: torch.Tensor) -> np.ndarray:
@@ -67,16 +80,17 @@ class ParityReport:
     excused_Y: int             # same tau, Y differs, and u is within 1e-6 of the CUDA token's CDF cell
     hard_mismatches: int       # differs with no such excuse
     max_rel_S: float
-    max_rel_S_conditioned: float  # over positions with S >= 1e-2 p
+    max_rel_S_conditioned: float  # over positions with S >= 2.4e-2 p
     S_floor_violations: int
     max_h_err_over_tol: float
     max_rel_p: float
     max_abs_lse: float
     vocab: int = 0
+    max_S_at_zero: float = 0.0   # largest CUDA S_i / p_i where the oracle's S_i is exactly 0
 
     def __str__(self):
         return ("trials=%d near=%d mismatch=%d excused_tau=%d excused_Y=%d hard=%d relS=%.2e "
-                "relS(S>=.01p)=%.2e floorviol=%d h_err/tol=%.2f relp=%.2e abslse=%.2e" % (
+                "relS(S>=.024p)=%.2e floorviol=%d h_err/tol=%.2f relp=%.2e abslse=%.2e" % (
                     self.trials, self.near_threshold, self.mismatches, self.excused_tau,
                     self.excused_Y, self.hard_mismatches, self.max_rel_S,
                     self.max_rel_S_conditioned, self.S_floor_violations,
@@ -141,7 +155,7 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
                 excused_Y += 1
             else:
                 hard += 1
-    rel_S = rel_Sc = h_over = rel_p = abs_lse = 0.0
+    rel_S = rel_Sc = h_over = rel_p = abs_lse = S_at_zero = 0.0
     floor_viol = 0
     V = 0
     if diag is not None:
@@ -174,7 +188,7 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
                     mm = mm & (pr < 1.0)
                 if mm.any():
                     den = (Sr[mm] + 1.0 - pr[mm]) ** 2
-                    tol = 1e-5 * hr[mm] + ((1.0 - pr[mm]) * 1e-7 * pr[mm] + Sr[mm] * 2e-7 * pr[mm]) / den + 1e-7
+                    tol = 1e-5 * hr[mm] + ((1.0 - pr[mm]) * S_FLOOR * pr[mm] + Sr[mm] * 2e-7 * pr[mm]) / den + 1e-7
                     h_over = max(h_over, float((np.abs(h[mm, i] - hr[mm]) / tol).max()))
             mm = rows
             if mm.any():
@@ -191,32 +205,41 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
         zero = m & (ref.S == 0)
         # an exactly empty residual: the CUDA value may differ from 0 only by the rounding
         # floor (it is exactly 0 for bit-identical rows, see test_draft_equals_target)
-        assert np.all(S[zero] <= 3e-7 * pS[zero]), "CUDA S must vanish where the oracle's does"
+        assert np.all(S[zero] <= S_FLOOR * pS[zero]), "CUDA S must vanish where the oracle's does"
+        S_at_zero = float((S[zero] / np.maximum(pS[zero], 1e-300)).max()) if zero.any() else 0.0
         pos = m & (ref.S > 0)
         if pos.any():
             err = np.abs(S[pos] - ref.S[pos])
             rel = err / ref.S[pos]
             rel_S = float(rel.max())
-            cond = ref.S[pos] >= 1e-2 * pS[pos]
+            cond = ref.S[pos] >= (S_FLOOR / 1e-5) * pS[pos]
             if cond.any():
                 rel_Sc = float(rel[cond].max())
-            floor_viol = int((err > 1e-5 * ref.S[pos] + 1e-7 * pS[pos]).sum())
+            floor_viol = int((err > 1e-5 * ref.S[pos] + S_FLOOR * pS[pos]).sum())
     if inp is not None:
         V = int(inp["target_logits"].shape[-1])
     return ParityReport(B, int(near.sum()), int(mism.sum()), excused_tau, excused_Y, hard, rel_S,
-                        rel_Sc, floor_viol, h_over, rel_p, abs_lse, V)
+                        rel_Sc, floor_viol, h_over, rel_p, abs_lse, V, S_at_zero)
 
 
 def assert_parity(rep: ParityReport, check_diag=True):
     assert rep.hard_mismatches == 0, str(rep)
     # an eta within 1e-6 of h_i: at most 1e-4 of trials may differ for that reason
     assert rep.excused_tau <= int(np.ceil(1e-4 * rep.trials)), str(rep)
-    # the sampling uniform has one threshold per vocabulary entry; an fp32 CDF places each
-    # within ~1e-7, so the expected share of differing tokens grows with V
-    assert rep.excused_Y <= int(np.ceil(rep.trials * (1e-4 + 2e-7 * rep.vocab))), str(rep)
+    # a sampling uniform within 1e-6 of an edge of the emitted token's CDF cell: the share of such
+    # trials that the exponentials' own error can move across an edge grows with the number of edges
+    assert rep.excused_Y <= int(np.ceil(rep.trials * (1e-4 + 2e-8 * rep.vocab))), str(rep)
     if check_diag:
         assert rep.max_abs_lse <= 3e-6, str(rep)
         assert rep.max_rel_p <= 1e-5, str(rep)
         assert rep.max_h_err_over_tol <= 1.0, str(rep)
         assert rep.max_rel_S_conditioned <= 1e-5, str(rep)
         assert rep.S_floor_violations == 0, str(rep)
+
+
+def record(rep: ParityReport, label: str):
+    """Appends the report to the file named by BV_PARITY_LOG (one JSON line), if that is set."""
+    path = os.environ.get("BV_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps(dict(case=label, **asdict(rep))) + "\n")

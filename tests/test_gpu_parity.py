@@ -8,7 +8,7 @@ import torch
 
 import oracle
 from paper_2403_10444_b200 import workloads as wl
-from parity import run_oracle, run_cuda, compare, assert_parity
+from parity import run_oracle, run_cuda, compare, assert_parity, record
 
 pytestmark = pytest.mark.gpu
 
@@ -21,6 +21,7 @@ def parity_case(inp, algo, check_diag=True):
     ot, ol, diag = run_cuda(algo, inp)
     rep = compare(algo, ref, ot, ol, diag, inp)
     print(rep)
+    record(rep, os.environ.get("PYTEST_CURRENT_TEST", "") + " diagnostics")
     assert_parity(rep, check_diag)
     # the entry points without diagnostic outputs are the ones a server calls (and the bench times);
     # for Algorithm 2 they leave out the second sweep of positions that cannot be selected, so
@@ -28,6 +29,7 @@ def parity_case(inp, algo, check_diag=True):
     ot2, ol2 = run_cuda(algo, inp, diagnostics=False)[:2]
     rep2 = compare(algo, ref, ot2, ol2, None, inp)
     print(rep2)
+    record(rep2, os.environ.get("PYTEST_CURRENT_TEST", "") + " plain")
     assert_parity(rep2, False)
     return rep
 

@@ -265,6 +265,43 @@ def test_draft_equals_target_accepts_everything():
     assert np.all(r.S == 0) and np.all(r.p == 1) and np.all(r.h[:, 1:g] == 0)
 
 
+@pytest.mark.parametrize("algo", [oracle.BLOCK_VERIFY, oracle.TOKEN_VERIFY, oracle.GREEDY_BLOCK_VERIFY])
+def test_a_position_with_an_empty_residual_is_never_the_selected_one(algo):
+    # Where P_i and Q_i coincide, Eqs. "pres-token" / "pres-block" have nothing to sample from (0/0).
+    # The algorithms never get there: the ratio of the next drafted token is then 1, so test i + 1
+    # passes whatever its uniform (Algorithm 1 does not stop at i; in Algorithms 2 and 4 p_{i+1} = p_i
+    # and a later position is selected, Lemma 3).  Checked for every block and every eta on a grid,
+    # with the coinciding position planted at every i, the other rows random.
+    rng = np.random.default_rng(77)
+    V, g, n = 4, 3, 6
+    grid = midgrid(n)
+    for same in range(g):
+        t = rng.normal(0, 1.5, (1, g + 1, V))
+        d = t[:, :g] + rng.normal(0, 1.0, (1, g, V))
+        d[0, same] = t[0, same]
+        blocks = all_blocks(V, g)
+        etas = list(itertools.product(grid, repeat=g))
+        B = len(blocks) * len(etas)
+        tgt = np.repeat(t, B, axis=0).astype(np.float32)
+        drf = np.repeat(d, B, axis=0).astype(np.float32)
+        tok = np.repeat(np.array(blocks, np.int32), len(etas), axis=0)
+        uni = np.empty((B, g + 2), np.float32)
+        uni[:, :g] = np.tile(np.array(etas, np.float32), (len(blocks), 1))
+        uni[:, g:] = 0.5
+        r = oracle.verify(algo, tgt, drf, tok, uni)
+        assert np.all(r.out_len >= 1)                  # no domain error anywhere ...
+        assert not np.any(r.out_len - 1 == same)       # ... and tau is never the planted position
+
+
+def test_sampling_from_nothing_is_a_domain_error():
+    # The sampler itself, given weights that sum to nothing, has no token to return: the sequence
+    # ends as a domain error.  Reached here through the drafting step on a row of -inf logits
+    # (the verification procedures cannot reach it, see the test above).
+    row = np.full((1, 8), -np.inf, np.float32)
+    tok, lse, _ = oracle.sample_rows(row, np.array([0.3], np.float32), 1.0)
+    assert tok[0] == -1 and np.isnan(lse[0])
+
+
 def test_temperature_scales_with_logits():
     rng = np.random.default_rng(14)
     B, g, V = 30, 3, 40
