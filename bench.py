@@ -108,75 +108,93 @@ def dist_setup(n_gpus: int):
     return 0, 1, 0, None
 
 
-def time_oracle(w, algo_name: str, budget_s: float = 20.0):
-    """The CPU oracle, as it stands, on a bounded sample of the workload."""
-    import numpy as np
-    import oracle
-    algo = {"block": oracle.BLOCK_VERIFY, "block_lse": oracle.BLOCK_VERIFY,
-            "greedy": oracle.GREEDY_BLOCK_VERIFY}.get(algo_name, oracle.TOKEN_VERIFY)
-    cores = oracle.threads()
-    # one sequence first to size the sample for about budget_s of work
-    probe = wl.make_inputs(wl.scaled(w, B=max(1, min(w.B, cores))), "cpu")
+class OracleRun:
+    """The CPU oracle, as it stands, on a bounded sample of the workload.
 
-    def run(inp):
-        t = inp["target_logits"]; d = inp["draft_logits"]
+    The sample (the first n sequences, n sized from one probe pass so that a pass over it takes about
+    ``pass_s`` seconds) is generated once; every call of :meth:`one_pass` verifies it again.
+    """
+
+    def __init__(self, w, algo_name: str, pass_s: float):
+        import oracle
+        self.oracle, self.w, self.algo_name = oracle, w, algo_name
+        self.algo = {"block": oracle.BLOCK_VERIFY, "block_lse": oracle.BLOCK_VERIFY,
+                     "greedy": oracle.GREEDY_BLOCK_VERIFY}.get(algo_name, oracle.TOKEN_VERIFY)
+        self.cores = oracle.threads()
+        probe = self._prepare(wl.make_inputs(wl.scaled(w, B=max(1, min(w.B, self.cores))), "cpu"))
+        per_seq = self._run(probe) / probe["B"]
+        n = int(max(1, min(w.B, pass_s / max(per_seq, 1e-9))))
+        self.n = max(min(n, w.B), min(w.B, self.cores))
+        self.sample = probe if self.n == probe["B"] else self._prepare(wl.make_inputs(wl.scaled(w, B=self.n), "cpu"))
+
+    def _prepare(self, inp):
+        import numpy as np
+        t, d = inp["target_logits"], inp["draft_logits"]
         if t.dtype == torch.bfloat16:
             t = t.view(torch.int16).numpy().view(np.uint16); d = d.view(torch.int16).numpy().view(np.uint16)
         else:
             t = t.numpy(); d = d.numpy()
-        if algo_name == "block_lse" and "draft_lse" not in inp:      # (outside the timed part)
-            inp["draft_lse"] = torch.logsumexp(inp["draft_logits"].double() / inp["temperature"], -1).float().numpy()
+        g = inp["draft_tokens"].shape[1]
+        p = {"t": t, "d": d, "x": inp["draft_tokens"].numpy(), "u": inp["uniforms"].numpy(),
+             "T": inp["temperature"], "B": inp["draft_tokens"].shape[0]}
+        if self.algo_name == "block_lse":
+            p["lse"] = torch.logsumexp(inp["draft_logits"].double() / inp["temperature"], -1).float().numpy()
+        if self.algo_name == "sample":
+            p["rows"] = d.reshape(-1, d.shape[-1])
+            p["u_rows"] = p["u"][:, :g].reshape(-1).copy()
+        return p
+
+    def _run(self, p) -> float:
+        o = self.oracle
         t0 = time.perf_counter()
-        if algo_name == "sample":
-            g = inp["draft_tokens"].shape[1]
-            oracle.sample_rows(d.reshape(-1, d.shape[-1]), inp["uniforms"].numpy()[:, :g].reshape(-1).copy(),
-                               inp["temperature"])
-        elif algo_name == "block_lse":
-            oracle.verify(algo, t, d, inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), inp["temperature"],
-                          draft_lse=inp["draft_lse"])
+        if self.algo_name == "sample":
+            o.sample_rows(p["rows"], p["u_rows"], p["T"])
+        elif self.algo_name == "block_lse":
+            o.verify(self.algo, p["t"], p["d"], p["x"], p["u"], p["T"], draft_lse=p["lse"])
         else:
-            oracle.verify(algo, t, d, inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), inp["temperature"])
+            o.verify(self.algo, p["t"], p["d"], p["x"], p["u"], p["T"])
         return time.perf_counter() - t0
 
-    t_probe = run(probe)
-    per_seq = t_probe / probe["draft_tokens"].shape[0]
-    n = int(max(1, min(w.B, budget_s / max(per_seq, 1e-9))))
-    n = max(min(n, w.B), min(w.B, cores))
-    sample = wl.make_inputs(wl.scaled(w, B=n), "cpu")
-    # the oracle goes through a whole workload in about a second on a many-core host: repeat the
-    # sample until about half the budget is spent, so that the figure is not one noisy second
+    def one_pass(self) -> float:
+        """Seconds the oracle takes for the sample."""
+        return self._run(self.sample)
+
+    def describe(self, passes: int, seconds: float) -> str:
+        what = "drafting step" if self.algo_name == "sample" else \
+            self.algo_name.replace("_lse", " with supplied draft normalisers") + " verify"
+        return "first %d of %d sequences of workload %s (%s), %d passes of %.2f s" % (
+            self.n, self.w.B, self.w.name, what, passes, seconds)
+
+
+def time_oracle(w, algo_name: str, budget_s: float = 20.0):
+    """cpu_baseline record: the oracle goes through a whole workload in about a second on a many-core
+    host, so the sample is repeated until about half the budget is spent (not one noisy second)."""
+    run = OracleRun(w, algo_name, budget_s)
     dt, reps = 0.0, 0
     while reps == 0 or (dt < 0.5 * budget_s and reps < 64):
-        dt += run(sample)
+        dt += run.one_pass()
         reps += 1
     dt /= reps
-    return {"value": n * w.gamma / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "first %d of %d sequences of workload %s (%s), %d passes of %.2f s" % (
-                n, w.B, w.name, "drafting step" if algo_name == "sample" else algo_name.replace("_lse", " with supplied draft normalisers") + " verify", reps, dt),
-            "seconds": dt, "sequences": n}
+    return {"value": run.n * w.gamma / dt, "unit": UNIT, "cores": run.cores, "kind": "oracle",
+            "sample": run.describe(reps, dt)}
 
 
 def reference_arm(args, w):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    """The oracle on the host cores, one pass over its bounded sample per step; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
         return
     steps, warmup = args.steps, args.warmup
-    budget = max(2.0, min(20.0, 120.0 / max(1, steps + warmup)))
-    times, last = [], None
-    for i in range(warmup + steps):
-        last = time_oracle(w, args.algo, budget_s=budget)
-        if i >= warmup:
-            times.append(last["seconds"])
-    n = last["sequences"]
+    run = OracleRun(w, args.algo, max(0.5, min(10.0, 120.0 / max(1, steps + warmup))))
+    times = [run.one_pass() for _ in range(warmup + steps)][warmup:]
     ms = 1e3 * sum(times) / len(times)
-    value = n * w.gamma / (ms * 1e-3)
+    value = run.n * w.gamma / (ms * 1e-3)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "gamma": w.gamma, "V": w.V, "storage": w.dtype,
-                       "algo": args.algo, "step": "%d sequences per step (bounded sample)" % n},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
-                             "sample": last["sample"]},
+                       "algo": args.algo, "step": "%d sequences per step (bounded sample)" % run.n},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": run.cores, "kind": "oracle",
+                             "sample": run.describe(steps, ms * 1e-3)},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -201,6 +219,9 @@ def main():
     if args.batch > 0:
         w = wl.scaled(w, B=args.batch, name="%s_B%d" % (w.name, args.batch))
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain program: become the launcher of one rank per GPU (each rank runs this file again)
+        sys.exit(sharding.launch_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
     if args.impl == "reference":
         reference_arm(args, w)
         return
@@ -278,6 +299,20 @@ def main():
         f1.synchronize()
         full_ms = f0.elapsed_time(f1) / 5
     args.full_ms = full_ms
+    # ---- Algorithm 1 on the same batch (the baseline the paper compares with), same timing rules ----
+    args.token = None
+    if args.algo == "block":
+        n_tok = max(3, min(args.steps, 10))
+        for _ in range(3):
+            tok_out = bv.tv_verify(*a)
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(n_tok):
+            tok_out = bv.tv_verify(*a)
+        t1.record()
+        t1.synchronize()
+        tok_ms = sharding.max_over_ranks(t0.elapsed_time(t1) / n_tok, dev)
+        args.token = (tok_ms, n_tok, tok_out)
 
     # ---- end to end: host buffers through the C-ABI host entry, copies inside the timed region ----
     e2e = None
@@ -312,6 +347,14 @@ def end_to_end(args, w, inp, out, bv, barrier, dist, dev, world):
             "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps}
 
 
+def token_bytes(w, out_len) -> int:
+    """Algorithm 1 stops at the first rejection: a sequence that emits n tokens needs the row pairs
+    0 .. min(n, gamma) - 1 and, when all gamma tokens were accepted, target row gamma."""
+    n = out_len.long().clamp(min=0)
+    rows = 2 * n.clamp(max=w.gamma) + (n == w.gamma + 1).long()
+    return int(rows.sum().item()) * w.V * (4 if w.dtype == "f32" else 2)
+
+
 def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches, out, dist):
     peak, peak_src = measured_peak()
     k_ms = statistics.mean(kernel_ms)
@@ -329,12 +372,8 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
         algo_bytes = w.logit_bytes
         kernel = "verify_flow_kernel"
     else:
-        # Algorithm 1 stops at the first rejection: a sequence that emits n tokens needs the row
-        # pairs 0 .. min(n, gamma) - 1 and, when all gamma tokens were accepted, target row gamma
-        n = out[1].long().clamp(min=0)
-        rows = 2 * n.clamp(max=w.gamma) + (n == w.gamma + 1).long()
-        algo_bytes = int(rows.sum().item()) * w.V * esz
-        kernel = "verify_cluster_kernel"
+        algo_bytes = token_bytes(w, out[1])
+        kernel = "verify_flow_kernel"
     achieved = algo_bytes / (k_ms * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -356,8 +395,21 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
                      "algorithmic_bytes": algo_bytes, "frac_of_8TBps": achieved / 8000.0},
         "sequences_per_s": world * w.B / (ms_per_step * 1e-3),
     }
+    if getattr(args, "token", None):
+        tok_ms, n_tok, tok_out = args.token
+        tb = token_bytes(w, tok_out[1])
+        rejected = int((tok_out[1] <= w.gamma).sum().item())
+        line["token"] = {
+            "algo": "token (Algorithm 1), same batch, same kernel machinery", "ms_per_step": tok_ms, "steps": n_tok,
+            "value": world * w.B * w.gamma / (tok_ms * 1e-3), "unit": UNIT,
+            "mean_emitted_len": float(tok_out[1].float().mean().item()),
+            # bytes Algorithm 1 needs when nothing is read twice; the kernel reads the row pair at the
+            # stopping position a second time for the residual sample
+            "algorithmic_bytes": tb, "achieved": tb / (tok_ms * 1e-3) / 1e9, "frac": tb / (tok_ms * 1e-3) / 1e9 / peak,
+            "second_sweep_bytes": rejected * 2 * w.V * esz,
+            "block_over_token_time": ms_per_step / tok_ms}
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = {k: v for k, v in time_oracle(w, args.algo).items() if k not in ("seconds", "sequences")}
+        line["cpu_baseline"] = time_oracle(w, args.algo)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -367,10 +419,6 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
 # ncu capture of this command at full size that profiles/ summarises; None for a workload or
 # kernel with no capture.
 TRAFFIC_BYTES = {
-    ("c4", "block", "verify_flow_kernel"): 2481445632,
-    ("c4", "greedy", "verify_flow_kernel"): 2479917824,
-    ("c4", "block_lse", "verify_flow_kernel"): 1442580480,
-    ("c4", "sample", "sample_rows_kernel"): 1054102784,
 }
 
 

@@ -90,3 +90,24 @@ def whole_job_rate(units_per_rank: int, ms_per_step: float, group=None) -> float
     """Units all ranks processed per second given the (already maximal) step time."""
     _, ws = world(group)
     return ws * units_per_rank / (ms_per_step * 1e-3)
+
+
+def rank_command(script: str, argv, n_ranks: int, port: Optional[int] = None):
+    """The command that starts ``n_ranks`` processes of ``script argv`` on this node, one per GPU,
+    through ``torch.distributed.run`` with the rendezvous on 127.0.0.1."""
+    import socket
+    import sys
+    if n_ranks < 1:
+        raise ValueError("n_ranks must be at least 1")
+    if port is None:
+        with socket.socket() as s:          # a port that is free now
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n_ranks),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), script, *argv]
+
+
+def launch_ranks(script: str, argv, n_ranks: int, port: Optional[int] = None, env=None) -> int:
+    """Run :func:`rank_command` to its end and return its exit status (non-zero if any rank failed)."""
+    import subprocess
+    return subprocess.call(rank_command(script, argv, n_ranks, port), env=env)

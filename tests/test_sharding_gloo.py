@@ -100,3 +100,32 @@ def test_two_gloo_ranks_reproduce_the_unsharded_result(B):
     for rank, res, slow, rate in got:
         assert slow == 11.0                      # the maximum over the two ranks
         assert rate == 2 * 100 / 2e-3            # whole-job units per second
+
+
+def test_rank_command_is_the_documented_launch():
+    cmd = sharding.rank_command("bench.py", ["--gpus", "4", "--steps", "2"], 4, port=29517)
+    assert cmd[1:] == ["-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "4", "--master-addr",
+                       "127.0.0.1", "--master-port", "29517", "bench.py", "--gpus", "4", "--steps", "2"]
+    with pytest.raises(ValueError):
+        sharding.rank_command("bench.py", [], 0)
+
+
+def test_bench_starts_its_own_ranks_when_not_under_a_launcher():
+    """`bench.py --gpus 2` run as a plain program starts two ranks of itself; shown on the CPU with the
+    reference arm (the oracle), where rank 0 alone works and prints the one line."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--workload", "c1", "--steps", "2", "--warmup", "1"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                  # rank 0 alone reports
+    line = lines[0]
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["steps"] == 2
+    assert line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
