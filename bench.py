@@ -213,6 +213,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="library tuning option set before the run (bv_set_option), may be repeated")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = wl.CONFIGS[args.workload]
@@ -228,6 +230,9 @@ def main():
 
     import paper_2403_10444_b200 as bv
     bv.load_library()  # fails loudly if the CUDA library was not built
+    for o in args.option:
+        name, _, val = o.partition("=")
+        bv.bv_set_option(name, int(val))
     rank, world, local, dist = dist_setup(args.gpus)
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
@@ -271,6 +276,7 @@ def main():
     launches = 0
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()      # (a profiler started with capture off sees exactly the timed steps)
     start.record()
     for i in range(args.steps):
         evs[i][0].record()
@@ -279,6 +285,7 @@ def main():
         launches += 1 if args.algo == "sample" else bv.bv_last_launch_count()
     stop.record()
     barrier()
+    torch.cuda.profiler.stop()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = start.elapsed_time(stop)
     kernel_ms = [e0.elapsed_time(e1) for e0, e1 in evs]
@@ -381,6 +388,7 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "gamma": w.gamma, "V": w.V, "storage": w.dtype,
                    "temperature": w.temperature, "algo": args.algo, "parallelism": "batch-sharded x%d" % world,
+                   "options": args.option or None,
                    "l2": "inputs (%.2f GB per step) exceed L2" % (w.logit_bytes / 1e9),
                    "mean_emitted_len": mean_len,
                    # Algorithm 2's residual masses are evaluated only for positions that can be the selected

@@ -258,6 +258,8 @@ int bv_stream_status(void* stream);
  *   "cluster"       cluster width of the cluster / streaming kernels (1, 2, 4, 8)
  *   "max_clusters"  cap on the clusters those kernels launch
  *   "flow_chunks", "flow_pieces", "flow_ctas", "flow_depth"   work-item shape of the flow kernel
+ *   "flow_keep_l2"  1: the lines a first sweep loads stay in L2 at normal priority for the row's second
+ *                   sweep (default 0: every load of the flow kernel streams past L2, which measured faster)
  *   "wait_limit"    polls after which a bounded device-side wait gives up (tests)
  *   "never_signal"  tests: the flow kernel's workers never report an item as swept, so its waits
  *                   run out and the call ends with BV_ERR_TIMEOUT

@@ -57,6 +57,8 @@ def _load():
         lib.oracle_verify_lse.restype = ctypes.c_int
         lib.oracle_verify_lse.argtypes = [ip, vp, vp, vp, vp, vp, ip, ip, ip, ip, ctypes.c_double,
                                           vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_verify_probs.restype = ctypes.c_int
+        lib.oracle_verify_probs.argtypes = [ip, vp, vp, vp, vp, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_threads.restype = ctypes.c_int
         lib.oracle_sample_rows.restype = ctypes.c_int
         lib.oracle_sample_rows.argtypes = [vp, vp, ip, ip, ip, ctypes.c_double, vp, vp, vp]
@@ -127,6 +129,39 @@ def verify(algo: int, target: np.ndarray, draft: np.ndarray, tokens: np.ndarray,
                            ptr(res.margin_eta), ptr(res.margin_smp))
     if rc != 0:
         raise ValueError("oracle_verify rejected its arguments")
+    return res
+
+
+def verify_probs(algo: int, target_probs: np.ndarray, draft_probs: np.ndarray, tokens: np.ndarray,
+                 uniforms: np.ndarray) -> OracleResult:
+    """Algorithm 1 or 2 on given probabilities (``oracle_verify_probs``): target_probs
+    [B, gamma+1, V], draft_probs [B, gamma, V], float32 / float64 / uint16 bf16 bits, used as
+    stored.  ``lse_t`` and ``lse_d`` of the result are NaN."""
+    lib = _load()
+    target_probs = np.ascontiguousarray(target_probs)
+    draft_probs = np.ascontiguousarray(draft_probs)
+    if target_probs.dtype != draft_probs.dtype or target_probs.dtype not in _DTYPE_CODE:
+        raise TypeError("target/draft must both be float32, float64 or uint16 (bf16 bits)")
+    B, g1, V = target_probs.shape
+    gamma = g1 - 1
+    if draft_probs.shape != (B, gamma, V):
+        raise ValueError("draft_probs must be [B, gamma, V]")
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    uniforms = np.ascontiguousarray(uniforms, dtype=np.float32)
+    if tokens.shape != (B, gamma) or uniforms.shape != (B, gamma + 2):
+        raise ValueError("tokens must be [B, gamma], uniforms [B, gamma+2]")
+    res = OracleResult(
+        out_tokens=np.empty((B, gamma + 1), np.int32), out_len=np.empty((B,), np.int32),
+        p=np.empty((B, gamma + 1)), S=np.empty((B, gamma)), h=np.empty((B, gamma + 1)),
+        lse_t=np.full((B, gamma + 1), np.nan), lse_d=np.full((B, gamma), np.nan),
+        margin_eta=np.empty((B,)), margin_smp=np.empty((B,)))
+    ptr = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    rc = lib.oracle_verify_probs(int(algo), ptr(target_probs), ptr(draft_probs), ptr(tokens), ptr(uniforms),
+                                 B, gamma, V, _DTYPE_CODE[target_probs.dtype],
+                                 ptr(res.out_tokens), ptr(res.out_len), ptr(res.p), ptr(res.S), ptr(res.h),
+                                 ptr(res.margin_eta), ptr(res.margin_smp))
+    if rc != 0:
+        raise ValueError("oracle_verify_probs rejected its arguments")
     return res
 
 

@@ -12,6 +12,9 @@
  *                          iteration only; the distribution modification that must
  *                          follow it (Algorithm 5) needs the models and is not here
  *
+ * The first two also on given probabilities instead of logits (oracle_verify_probs, pinned in
+ * tests/test_oracle_probs.py).
+ *
  * It follows the algorithms step by step in the paper's order and notation,
  * with no blocking, fusion or reordering.  It shares no code with the CUDA
  * library, and only tests, the smoke check and the benchmark's CPU-baseline
@@ -216,7 +219,7 @@ static void emit(const seq_t *s, int tau, int Y, int32_t *out_tokens, int32_t *o
     for (int i = 0; i < tau; ++i)
         out_tokens[i] = s->X[i];
     out_tokens[tau] = Y;
-    *out_len = tau + 1; /* "Return X^tau, Y" */
+    *out_len = tau + 1; /* the accepted prefix X_1..X_tau and the one sampled token Y */
 }
 
 /*
@@ -585,8 +588,8 @@ int oracle_verify_lse(int algo, const void *target, const void *draft,
 }
 
 /*
- * The drafting step of Algorithm 3 ("Sample X_1..X_gamma ~ M_s ... keep the conditional
- * probabilities at each step") for rows of logits: for every row r,
+ * The drafting step of Algorithm 3 (the small model draws X_1..X_gamma one after the other and
+ * its conditional distribution at each step is kept) for rows of logits: for every row r,
  *   M_s(x) = softmax(logits[r, :] / T)(x),
  *   tokens[r] = inverse-CDF sample in vocabulary-index order with uniforms[r]
  *               (the same convention as the verification samples),
@@ -617,6 +620,205 @@ int oracle_sample_rows(const void *logits, const float *uniforms, int rows, int 
         }
         if (lse) lse[r] = l;
         if (margin) margin[r] = m;
+    }
+    return 0;
+}
+
+/* ================= the same procedures on given probabilities =================
+ *
+ * The paper states Algorithms 1 and 2 on the conditional distributions themselves
+ * (M_b(. | c, X^i), M_s(. | c, X^i)); here they are the inputs, as stored numbers:
+ *   P_r(x) = target_probs[b, r, x], r = 0..gamma;  Q_r(x) = draft_probs[b, r, x], r = 0..gamma-1.
+ * Nothing is renormalised: Eq. "def_as", "pacc_block", "pres-token" and "pres-block" are
+ * evaluated on the numbers as given (a row that does not sum to one exactly, as after rounding to
+ * a narrow type, is used as it is; the samples divide by the sum of their own weights).
+ * Domain errors of a sequence: a drafted token outside [0, V); Q_{i-1}(X_i) that is not a
+ * positive finite number or P_{i-1}(X_i) that is not a non-negative finite number in a test the
+ * algorithm makes; an empty or non-finite weight sum at the position to sample from.
+ */
+static double stored_prob(const seq_t *s, int target_row, int r, int x)
+{
+    size_t V = (size_t)s->V;
+    return target_row ? logit_at(s->tgt, s->dtype, s->toff + (size_t)r * V + (size_t)x)
+                      : logit_at(s->drf, s->dtype, s->doff + (size_t)r * V + (size_t)x);
+}
+
+/* weight of token x at position i: max(p P_i(x) - Q_i(x), 0), or P_gamma(x) at i = gamma */
+static double weight_probs(const seq_t *s, int i, int x, double p)
+{
+    double P = stored_prob(s, 1, i, x);
+    if (i == s->gamma)
+        return P;
+    double w = p * P - stored_prob(s, 0, i, x);
+    return w > 0.0 ? w : 0.0;
+}
+
+/* inverse-CDF sample in index order from the weights of position i (see sample_index_order) */
+static int sample_probs(const seq_t *s, int i, double p, double u, double *W_out, double *margin)
+{
+    double W = 0.0;
+    for (int x = 0; x < s->V; ++x)
+        W += weight_probs(s, i, x, p);
+    *W_out = W;
+    *margin = 0.0;
+    if (!(W > 0.0) || !isfinite(W))
+        return -1;
+    double t = u * W, C = 0.0;
+    int last_pos = -1;
+    for (int x = 0; x < s->V; ++x) {
+        double w = weight_probs(s, i, x, p);
+        double Cprev = C;
+        C += w;
+        if (w > 0.0)
+            last_pos = x;
+        if (C > t) {
+            double lo = u - Cprev / W, hi = C / W - u;
+            *margin = lo < hi ? lo : hi;
+            return x;
+        }
+    }
+    return last_pos;
+}
+
+/* M_b(X_i | c, X^{i-1}) / M_s(X_i | c, X^{i-1}) from the stored numbers; 1 on a domain error */
+static int ratio_probs(const seq_t *s, int i, double *ratio)
+{
+    int x = s->X[i - 1];
+    if (x < 0 || x >= s->V)
+        return 1;
+    double P = stored_prob(s, 1, i - 1, x), Q = stored_prob(s, 0, i - 1, x);
+    if (!(Q > 0.0) || !isfinite(Q) || !(P >= 0.0) || !isfinite(P))
+        return 1;
+    *ratio = P / Q;
+    return 0;
+}
+
+/* Algorithm 1 */
+static void token_verify_probs_one(const seq_t *s, const diag_t *d, int32_t *out_tokens, int32_t *out_len)
+{
+    const int g = s->gamma;
+    double m_eta = INFINITY;
+    diag_fill_nan(d, g);
+    int tau = 0;
+    for (int i = 1; i <= g; ++i) {
+        double ratio;
+        if (ratio_probs(s, i, &ratio)) {
+            emit(s, -1, -1, out_tokens, out_len);
+            return;
+        }
+        double h = ratio < 1.0 ? ratio : 1.0;
+        if (d->h) d->h[i] = h;
+        double eta = (double)s->u[i - 1];
+        double gap = fabs(eta - h);
+        if (gap < m_eta) m_eta = gap;
+        if (h > 0.0 && eta <= h)
+            tau = i;
+        else
+            break;
+    }
+    if (d->h) d->h[0] = 1.0;
+    double W, m_smp;
+    int Y = sample_probs(s, tau, 1.0, (double)s->u[tau < g ? g : g + 1], &W, &m_smp);
+    if (tau < g && d->S) d->S[tau] = W;
+    if (d->margin_eta) *d->margin_eta = m_eta;
+    if (d->margin_smp) *d->margin_smp = m_smp;
+    emit(s, Y < 0 ? -1 : tau, Y, out_tokens, out_len);
+}
+
+/* Algorithm 2 */
+static void block_verify_probs_one(const seq_t *s, const diag_t *d, int32_t *out_tokens, int32_t *out_len)
+{
+    const int g = s->gamma;
+    diag_fill_nan(d, g);
+    double *p = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *S = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    double *h = (double *)malloc(sizeof(double) * (size_t)(g + 1));
+    p[0] = 1.0;
+    for (int i = 1; i <= g; ++i) {
+        double ratio;
+        if (ratio_probs(s, i, &ratio)) {
+            emit(s, -1, -1, out_tokens, out_len);
+            goto done;
+        }
+        double v = p[i - 1] * ratio;
+        p[i] = v < 1.0 ? v : 1.0;
+    }
+    for (int i = 0; i < g; ++i) {
+        double acc = 0.0;
+        for (int x = 0; x < s->V; ++x)
+            acc += weight_probs(s, i, x, p[i]);
+        S[i] = acc;
+    }
+    h[0] = 1.0;
+    for (int i = 1; i < g; ++i)
+        h[i] = S[i] > 0.0 ? S[i] / (S[i] + 1.0 - p[i]) : 0.0;
+    h[g] = p[g];
+    int tau = 0;
+    double m_eta = INFINITY;
+    for (int i = 1; i <= g; ++i)
+        if (h[i] > 0.0 && (double)s->u[i - 1] <= h[i])
+            tau = i;
+    for (int i = (tau > 0 ? tau : 1); i <= g; ++i) {
+        double gap = fabs((double)s->u[i - 1] - h[i]);
+        if (gap < m_eta) m_eta = gap;
+    }
+    {
+        double W, m_smp;
+        int Y = sample_probs(s, tau, p[tau], (double)s->u[tau < g ? g : g + 1], &W, &m_smp);
+        if (d->margin_eta) *d->margin_eta = m_eta;
+        if (d->margin_smp) *d->margin_smp = m_smp;
+        emit(s, Y < 0 ? -1 : tau, Y, out_tokens, out_len);
+    }
+    for (int i = 0; i <= g; ++i) {
+        if (d->p) d->p[i] = p[i];
+        if (d->h) d->h[i] = h[i];
+        if (i < g && d->S) d->S[i] = S[i];
+    }
+done:
+    free(p); free(S); free(h);
+}
+
+/*
+ * algo: ORACLE_TOKEN_VERIFY or ORACLE_BLOCK_VERIFY.  target_probs [B, gamma+1, V], draft_probs
+ * [B, gamma, V] in dtype (f32, bf16 bits, f64); the other arguments as oracle_verify, without
+ * the normalisers.  Returns 0, or 1 for an invalid argument.
+ */
+int oracle_verify_probs(int algo, const void *target_probs, const void *draft_probs,
+                        const int32_t *tokens, const float *uniforms,
+                        int B, int gamma, int V, int dtype,
+                        int32_t *out_tokens, int32_t *out_len,
+                        double *p, double *S, double *h, double *margin_eta, double *margin_smp)
+{
+    if (!target_probs || !draft_probs || !tokens || !uniforms || !out_tokens || !out_len)
+        return 1;
+    if (B < 0 || gamma < 1 || V < 1 || dtype < 0 || dtype > 2)
+        return 1;
+    if (algo != ORACLE_TOKEN_VERIFY && algo != ORACLE_BLOCK_VERIFY)
+        return 1;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int b = 0; b < B; ++b) {
+        seq_t s;
+        s.tgt = target_probs; s.drf = draft_probs;
+        s.X = tokens + (size_t)b * (size_t)gamma;
+        s.u = uniforms + (size_t)b * (size_t)(gamma + 2);
+        s.gamma = gamma; s.V = V; s.dtype = dtype; s.T = 1.0;
+        s.toff = (size_t)b * (size_t)(gamma + 1) * (size_t)V;
+        s.doff = (size_t)b * (size_t)gamma * (size_t)V;
+        s.given_lse_d = NULL;
+        diag_t d;
+        d.p = p ? p + (size_t)b * (size_t)(gamma + 1) : NULL;
+        d.S = S ? S + (size_t)b * (size_t)gamma : NULL;
+        d.h = h ? h + (size_t)b * (size_t)(gamma + 1) : NULL;
+        d.lse_t = NULL; d.lse_d = NULL;
+        d.margin_eta = margin_eta ? margin_eta + b : NULL;
+        d.margin_smp = margin_smp ? margin_smp + b : NULL;
+        int32_t *ot = out_tokens + (size_t)b * (size_t)(gamma + 1);
+        if (algo == ORACLE_BLOCK_VERIFY)
+            block_verify_probs_one(&s, &d, ot, out_len + b);
+        else
+            token_verify_probs_one(&s, &d, ot, out_len + b);
     }
     return 0;
 }

@@ -23,6 +23,7 @@ struct Options {
     int cluster = 0;       // cluster width of the cluster / stream kernels (1, 2, 4, 8); 0: chosen by shape
     int max_clusters = 0;  // cap on the clusters launched; 0: none
     int flow_chunks = 0, flow_pieces = 0, flow_ctas = 0, flow_depth = 0;   // 0: chosen by shape
+    int flow_keep_l2 = 0;  // 1: the lines of a first sweep stay in L2 at normal priority; 0: every load streams past L2
     int wait_limit = 0;    // polls after which a bounded device-side wait gives up; 0: the built-in limits
     int never_signal = 0;  // test switch: the flow kernel's workers never report an item as swept
 };
@@ -222,6 +223,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             bv::FlowScratch fl;
             bv::flow_scratch_layout(scratch, B, gamma, plan, &fl);
             if (opt.flow_depth >= 2 && opt.flow_depth <= 6) fl.depth = opt.flow_depth;
+            fl.keep_l2 = opt.flow_keep_l2 == 1;
             // The kernel leaves its counters and flags at zero when it ends, so they are cleared here only
             // when the area is new or a larger problem needs more of them than the last launch left clean.
             cudaError_t e = cudaSuccess;
@@ -472,6 +474,7 @@ int bv_set_option(const char* name, int value) {
     else if (!std::strcmp(name, "flow_pieces")) g_opt.flow_pieces = value;
     else if (!std::strcmp(name, "flow_ctas")) g_opt.flow_ctas = value;
     else if (!std::strcmp(name, "flow_depth")) g_opt.flow_depth = value;
+    else if (!std::strcmp(name, "flow_keep_l2")) g_opt.flow_keep_l2 = value;
     else if (!std::strcmp(name, "wait_limit")) g_opt.wait_limit = value;
     else if (!std::strcmp(name, "never_signal")) g_opt.never_signal = value;
     else return BV_ERR_INVALID_ARG;

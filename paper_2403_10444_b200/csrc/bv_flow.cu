@@ -550,8 +550,12 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     constexpr uint32_t kCell = kFThreads * 16;               // bytes between consecutive ring cells of a thread
     const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;   // this thread's ring cell 0
     const uint32_t ring_end = sb + kFDepth * kCell;
-    // no row is needed again soon (the few second sweeps come long after the first): stream past L2
-    const uint64_t pol = l2_policy_evict_first();
+    // Every load streams past L2 (its lines are the first to be evicted).  Leaving the first sweep's
+    // lines at normal priority, so that a second sweep that follows soon finds them in L2, is a
+    // tuning switch: measured 2 to 5 % slower on every shape tried, Algorithm 1 included.
+    const uint64_t pol_stream = l2_policy_evict_first();
+    const uint64_t pol_keep = fl.keep_l2 ? l2_policy_evict_normal() : pol_stream;
+    uint64_t pol = pol_stream;
     const char* iA = nullptr;         // issue cursor: this lane's next vector for cell A and for cell B
     const char* iB = nullptr;
     int i_rem = 0;                    // vectors of the current segment not yet asked for
@@ -565,6 +569,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         int w0, w1;
         warp_range(sh.desc[slot].u0, sh.desc[slot].u1, warp, w0, w1);
         const bool single = sh.desc[slot].have_q == 0;
+        pol = sh.desc[slot].kind == kSweep1 ? pol_keep : pol_stream;
         i_rem = w1 - w0;
         i_adv = single ? 64 : 32;
         i_adv16 = single ? 1024u : 512u;
@@ -773,6 +778,7 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->cand = reinterpret_cast<int*>(take(rows * sizeof(int)));
     fl->tv_tau = reinterpret_cast<int*>(take(static_cast<size_t>(B) * sizeof(int)));
     fl->nch = plan.nch;
+    fl->keep_l2 = 0;
     fl->part_stride = plan.part_stride();
     fl->total_s1 = static_cast<unsigned>(B) * (plan.tv_spec > 0 ? plan.tv_spec : gamma) * plan.nch;
     fl->nch_late = plan.nch_late;

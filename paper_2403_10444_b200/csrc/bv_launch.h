@@ -71,6 +71,7 @@ struct FlowScratch {
     unsigned zero_words;  // 32-bit words at the start of the scratch area (from `counters` on) that start and end at zero
     int depth;            // flow kernel: descriptors a CTA may have handed to its workers and not yet seen swept
     int segs;             // residual totals kept per row
+    int keep_l2;          // tuning switch: first-sweep loads leave their lines at normal priority in L2 (default: evicted first)
 };
 constexpr int kFlowMaxChunks = 32;
 // How a launch is cut into work items (flow_plan): chunks per row in the first sweep, chunks of a
