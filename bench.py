@@ -118,8 +118,9 @@ class OracleRun:
     def __init__(self, w, algo_name: str, pass_s: float):
         import oracle
         self.oracle, self.w, self.algo_name = oracle, w, algo_name
-        self.algo = {"block": oracle.BLOCK_VERIFY, "block_lse": oracle.BLOCK_VERIFY,
+        self.algo = {"block": oracle.BLOCK_VERIFY, "block_lse": oracle.BLOCK_VERIFY, "block_probs": oracle.BLOCK_VERIFY,
                      "greedy": oracle.GREEDY_BLOCK_VERIFY}.get(algo_name, oracle.TOKEN_VERIFY)
+        self.probs = algo_name.endswith("_probs")
         self.cores = oracle.threads()
         probe = self._prepare(wl.make_inputs(wl.scaled(w, B=max(1, min(w.B, self.cores))), "cpu"))
         per_seq = self._run(probe) / probe["B"]
@@ -130,6 +131,9 @@ class OracleRun:
     def _prepare(self, inp):
         import numpy as np
         t, d = inp["target_logits"], inp["draft_logits"]
+        if self.probs:      # (the distributions handed over as probabilities in the storage type, as on the GPU)
+            t = torch.softmax(t.float() / inp["temperature"], -1).to(t.dtype)
+            d = torch.softmax(d.float() / inp["temperature"], -1).to(d.dtype)
         if t.dtype == torch.bfloat16:
             t = t.view(torch.int16).numpy().view(np.uint16); d = d.view(torch.int16).numpy().view(np.uint16)
         else:
@@ -149,6 +153,8 @@ class OracleRun:
         t0 = time.perf_counter()
         if self.algo_name == "sample":
             o.sample_rows(p["rows"], p["u_rows"], p["T"])
+        elif self.probs:
+            o.verify_probs(self.algo, p["t"], p["d"], p["x"], p["u"])
         elif self.algo_name == "block_lse":
             o.verify(self.algo, p["t"], p["d"], p["x"], p["u"], p["T"], draft_lse=p["lse"])
         else:
@@ -161,7 +167,7 @@ class OracleRun:
 
     def describe(self, passes: int, seconds: float) -> str:
         what = "drafting step" if self.algo_name == "sample" else \
-            self.algo_name.replace("_lse", " with supplied draft normalisers") + " verify"
+            self.algo_name.replace("_lse", " with supplied draft normalisers").replace("_probs", " on probabilities") + " verify"
         return "first %d of %d sequences of workload %s (%s), %d passes of %.2f s" % (
             self.n, self.w.B, self.w.name, what, passes, seconds)
 
@@ -206,10 +212,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(wl.CONFIGS))
-    ap.add_argument("--algo", default="block", choices=["block", "token", "sample", "block_lse", "greedy"],
+    ap.add_argument("--algo", default="block", choices=["block", "token", "sample", "block_lse", "greedy", "block_probs", "token_probs"],
                     help="block / token verification, the drafting step (sampling the draft rows), block "
                          "verification with the draft normalisers that the drafting step leaves, or one "
-                         "iteration of greedy block verification (Algorithm 4)")
+                         "iteration of greedy block verification (Algorithm 4); block_probs / token_probs: the "
+                         "two verifications on the workload's distributions given as probabilities")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
@@ -259,6 +266,15 @@ def main():
     if args.algo == "greedy":
         fn = bv.gbv_verify
         args.e2e_steps = 0          # (no host-buffer form of this entry point)
+    if args.algo in ("block_probs", "token_probs"):
+        # the same distributions, handed over as probabilities in the storage type (formed outside the timed region)
+        pt = torch.empty_like(inp["target_logits"]); pd = torch.empty_like(inp["draft_logits"])
+        for b0 in range(0, w.B, 16):
+            pt[b0:b0 + 16] = torch.softmax(inp["target_logits"][b0:b0 + 16].float() / inp["temperature"], -1).to(pt.dtype)
+            pd[b0:b0 + 16] = torch.softmax(inp["draft_logits"][b0:b0 + 16].float() / inp["temperature"], -1).to(pd.dtype)
+        pfn = bv.bv_verify_probs if args.algo == "block_probs" else bv.tv_verify_probs
+        fn = lambda *_: pfn(pt, pd, a[2], a[3])
+        args.e2e_steps = 0
 
     def barrier():
         if dist is not None:
@@ -373,6 +389,12 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
     elif args.algo == "block_lse":
         # what must be read at least: every target row, and one draft row per block for the residual
         algo_bytes = w.B * (w.gamma + 2) * w.V * esz
+        kernel = "verify_flow_kernel"
+    elif args.algo in ("block_probs", "token_probs"):
+        # given probabilities, what must be read is the row pair at the selected position (or the last
+        # target row) of every sequence, besides the 2 gamma entries of its drafted tokens
+        n = out[1].long().clamp(min=0)
+        algo_bytes = int((2 * (n <= w.gamma).long() + (n == w.gamma + 1).long()).sum().item()) * w.V * esz
         kernel = "verify_flow_kernel"
     elif args.algo in ("block", "greedy"):
         # Algorithms 2 and 4 need every row: B (2 gamma + 1) V elements

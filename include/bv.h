@@ -229,6 +229,34 @@ int gbv_verify_ex(const void* target_logits, const void* draft_logits,
                   float* out_lse_t, float* out_lse_d, void* stream);
 
 /*
+ * Algorithms 2 and 1 on given probabilities, the form in which the paper states them (Algorithm 1,
+ * Algorithm 2: the conditional distributions M_b(. | c, X^i), M_s(. | c, X^i) are the inputs):
+ *   target_probs [B, gamma+1, V], draft_probs [B, gamma, V] in `dtype`, device pointers, 16-byte
+ *   aligned, rows of a multiple of 16 bytes (else BV_ERR_UNSUPPORTED); the other arguments as bv_verify.
+ * The numbers are used as stored: Eq. "def_as", "pacc_block", "pres-block" / "pres-token" are
+ * evaluated on them without renormalising (the samples divide by the sum of their own weights), and
+ * no temperature applies.  Only the rows the algorithm needs are read: the 2 gamma entries of the
+ * drafted tokens, the row pairs of the positions that can be the selected one (Algorithm 2: those
+ * with eta_i <= p_i, from the top down; Algorithm 1: the one at tau), or row gamma of the target.
+ * A sequence with a drafted token outside [0, V), with Q_{i-1}(X_i) not a positive finite number or
+ * P_{i-1}(X_i) not a non-negative finite number (Algorithm 1: in a test it makes), or with an empty
+ * or non-finite weight sum where it must sample, gets out_len = -1 and out_tokens = -1; entries the
+ * algorithm does not read are not validated.
+ * out_p [B, gamma+1], out_S [B, gamma], out_h [B, gamma+1]: optional diagnostics as in bv_verify_ex /
+ * tv_verify_ex (each may be null; with any of them Algorithm 2 evaluates every position).
+ */
+int bv_verify_probs(const void* target_probs, const void* draft_probs,
+                    const int32_t* draft_tokens, const float* uniforms,
+                    int B, int gamma, int V, int dtype,
+                    int32_t* out_tokens, int32_t* out_len,
+                    float* out_p, float* out_S, float* out_h, void* stream);
+int tv_verify_probs(const void* target_probs, const void* draft_probs,
+                    const int32_t* draft_tokens, const float* uniforms,
+                    int B, int gamma, int V, int dtype,
+                    int32_t* out_tokens, int32_t* out_len,
+                    float* out_p, float* out_S, float* out_h, void* stream);
+
+/*
  * The drafting step of Algorithm 3 (its first step: one token per draft distribution, the
  * distribution's normaliser kept for the verification) for `rows` rows of draft logits [rows, V]:
  *   out_tokens[r] ~ softmax(logits[r, :] / temperature), drawn by inverse CDF in vocabulary-index

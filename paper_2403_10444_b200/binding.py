@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_sample_draft", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_verify_probs", "tv_verify_probs", "bv_sample_draft", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -55,6 +55,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     for name in ("bv_verify_host", "tv_verify_host"):
         getattr(lib, name).argtypes = base
     lib.bv_sample_draft.argtypes = [vp, vp, ci, ci, ci, cf, vp, vp, vp]
+    for name in ("bv_verify_probs", "tv_verify_probs"):
+        getattr(lib, name).argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp]
     lib.bv_verify_lse.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp]
     lib.bv_verify_lse_ex.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp, vp, vp, vp, vp, vp]
     for name in EXPORTS:
@@ -198,6 +200,37 @@ def gbv_verify_ex(target_logits, draft_logits, draft_tokens, uniforms, temperatu
     the acceptance ratios, h the ratios (above one, or +inf, where the test passes with certainty)."""
     return _device_call("gbv_verify_ex", target_logits, draft_logits, draft_tokens, uniforms,
                         temperature, True, stream)
+
+
+def _probs_call(name: str, target_probs, draft_probs, tokens, uniforms, diagnostics: bool, stream):
+    lib = load_library()
+    B, gamma, V = _shapes(target_probs, draft_probs, tokens, uniforms, True)
+    dev = target_probs.device
+    out_tokens = torch.empty((B, gamma + 1), dtype=torch.int32, device=dev)
+    out_len = torch.empty((B,), dtype=torch.int32, device=dev)
+    diag, ptrs = None, [None, None, None]
+    if diagnostics:
+        f = lambda *shape: torch.empty(shape, dtype=torch.float32, device=dev)
+        diag = dict(p=f(B, gamma + 1), S=f(B, gamma), h=f(B, gamma + 1))
+        ptrs = [diag[k].data_ptr() for k in ("p", "S", "h")]
+    with torch.cuda.device(dev):
+        s = stream if stream is not None else torch.cuda.current_stream(dev)
+        _check(getattr(lib, name)(target_probs.data_ptr(), draft_probs.data_ptr(), tokens.data_ptr(),
+                                  uniforms.data_ptr(), B, gamma, V, _dtype_code(target_probs),
+                                  out_tokens.data_ptr(), out_len.data_ptr(), *ptrs, s.cuda_stream))
+    return (out_tokens, out_len, diag) if diagnostics else (out_tokens, out_len)
+
+
+def bv_verify_probs(target_probs, draft_probs, draft_tokens, uniforms, diagnostics: bool = False, stream=None):
+    """Block Verification (Algorithm 2) on given probabilities [B, gamma+1, V] / [B, gamma, V] (CUDA,
+    float32 or bfloat16, used as stored); returns (out_tokens, out_len) and, with ``diagnostics``,
+    dict(p, S, h)."""
+    return _probs_call("bv_verify_probs", target_probs, draft_probs, draft_tokens, uniforms, diagnostics, stream)
+
+
+def tv_verify_probs(target_probs, draft_probs, draft_tokens, uniforms, diagnostics: bool = False, stream=None):
+    """Token Verification (Algorithm 1) on given probabilities; see bv_verify_probs."""
+    return _probs_call("tv_verify_probs", target_probs, draft_probs, draft_tokens, uniforms, diagnostics, stream)
 
 
 def bv_verify_noalloc(target_logits, draft_logits, draft_tokens, uniforms, out_tokens, out_len,

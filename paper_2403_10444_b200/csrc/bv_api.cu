@@ -161,6 +161,7 @@ int pick_cluster(const DeviceState& d, const Options& opt, int B, size_t row_byt
 struct Extra {              // what only some entry points pass
     const float* lse_d = nullptr;   // supplied draft log-normalisers (bv_verify_lse)
     int greedy = 0;                 // Algorithm 4 instead of Algorithm 2 (gbv_verify)
+    int probs = 0;                  // the rows hold probabilities, not logits (bv_verify_probs, tv_verify_probs)
     float* out_p = nullptr; float* out_S = nullptr; float* out_h = nullptr;
     float* out_lse_t = nullptr; float* out_lse_d = nullptr;
 };
@@ -186,6 +187,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     prm.tgt = tgt; prm.drf = drf; prm.tok = tok; prm.uni = uni;
     prm.lse_d = ex.lse_d;
     prm.greedy = ex.greedy;
+    prm.probs = ex.probs;
     prm.B = B; prm.gamma = gamma; prm.V = V;
     const double kd = 1.4426950408889634073599246810019 / static_cast<double>(T);
     prm.kd = kd;
@@ -198,7 +200,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
 
     prm.algo = algo;
     const bool flow_ok = vec && (opt.kernel == 0 || opt.kernel == 1);
-    if ((prm.lse_d != nullptr || prm.greedy) && !flow_ok) return BV_ERR_UNSUPPORTED;
+    if ((prm.lse_d != nullptr || prm.greedy || prm.probs) && !flow_ok) return BV_ERR_UNSUPPORTED;
 
     // 16-byte rows: the flow of independent work items (both algorithms)
     if (flow_ok) {
@@ -214,7 +216,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             const int chunks = (opt.flow_chunks >= 1 && opt.flow_chunks <= bv::kFlowMaxChunks) ? opt.flow_chunks : 0;
             const int pieces = (opt.flow_pieces >= 1 && opt.flow_pieces <= 8) ? opt.flow_pieces : 0;
             // (with supplied draft normalisers a first-sweep item streams one row, not two)
-            const bv::FlowPlan plan = bv::flow_plan(units, B, gamma, nctas, prm.lse_d == nullptr, chunks, pieces, algo == bv::kTokenVerify);
+            const bv::FlowPlan plan = bv::flow_plan(units, B, gamma, nctas, prm.lse_d == nullptr, chunks, pieces, algo == bv::kTokenVerify, prm.probs != 0);
             size_t zero_bytes = 0;
             const size_t need = bv::flow_scratch_bytes(B, gamma, plan, &zero_bytes);
             StreamSlot* slot = nullptr;
@@ -232,7 +234,8 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
                 if (e != cudaSuccess) return cuda_fail(e);
             }
             slot->clean = zero_bytes;
-            long long items = static_cast<long long>(fl.total_s1);
+            // (given probabilities the items are the pieces of the positions swept: at most all of them)
+            long long items = prm.probs ? static_cast<long long>(B) * (gamma + 1) * fl.np : static_cast<long long>(fl.total_s1);
             if (nctas > items) nctas = items;
             prm.ticket = nullptr;
             prm.nclusters = 0;
@@ -244,7 +247,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
         }
     }
 
-    if (prm.lse_d != nullptr || prm.greedy) return BV_ERR_UNSUPPORTED;   // (the flow kernel could not be launched)
+    if (prm.lse_d != nullptr || prm.greedy || prm.probs) return BV_ERR_UNSUPPORTED;   // (the flow kernel could not be launched)
 
     StreamSlot* slot = nullptr;
     if ((rc = stream_slot(*d, stream, 0, &slot)) != BV_OK) return rc;
@@ -414,6 +417,20 @@ int bv_verify_lse_ex(const void* tgt, const void* drf, const int32_t* tok, const
     Extra ex = diagnostics(out_p, out_S, out_h, out_lse_t, out_lse_d);
     ex.lse_d = draft_lse;
     return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, ex, static_cast<cudaStream_t>(stream));
+}
+
+int bv_verify_probs(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+                    int V, int dtype, int32_t* ot, int32_t* ol, float* out_p, float* out_S, float* out_h, void* stream) {
+    Extra ex = diagnostics(out_p, out_S, out_h, nullptr, nullptr);
+    ex.probs = 1;
+    return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, 1.f, ot, ol, ex, static_cast<cudaStream_t>(stream));
+}
+
+int tv_verify_probs(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
+                    int V, int dtype, int32_t* ot, int32_t* ol, float* out_p, float* out_S, float* out_h, void* stream) {
+    Extra ex = diagnostics(out_p, out_S, out_h, nullptr, nullptr);
+    ex.probs = 1;
+    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, 1.f, ot, ol, ex, static_cast<cudaStream_t>(stream));
 }
 
 int gbv_verify(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,

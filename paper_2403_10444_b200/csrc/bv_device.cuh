@@ -36,6 +36,7 @@ struct Params {
     int algo;                 // flow kernel: kBlockVerify (Algorithms 2, 4) or kTokenVerify (Algorithm 1)
     unsigned wait_limit;      // flow kernel: polls after which a bounded wait gives up (0: the built-in limits)
     int never_signal;         // flow kernel, test switch: workers never report an item as swept, so the waits run out
+    int probs;                // flow kernel: tgt / drf hold probabilities, used as stored, instead of logits
 };
 
 __device__ __forceinline__ float ex2(float x) {

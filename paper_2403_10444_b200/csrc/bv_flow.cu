@@ -232,11 +232,11 @@ __device__ __forceinline__ void f_store_sweep2(const FlowScratch& fl, FlowShared
     double* segs = fl.seg_tot + static_cast<size_t>(ri) * fl.segs;
     if (lane < kFWarps) segs[ch * kFWarps + lane] = sh.stage_d[j][lane];
 }
-template <int DT>
+template <int DT, bool PROBS>
 __device__ void f_complete_sweep2(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, const FlowDesc& d, int lane) {
     const int np = fl.np;
     const double* segs = fl.seg_tot + static_cast<size_t>(d.ri) * fl.segs;
-    f_position_complete<DT>(prm, fl, cx, d.ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, np * kFWarps, segs, lane,
+    f_position_complete<DT, PROBS>(prm, fl, cx, d.ri, d.have_q != 0, d.rowP, d.rowQ, d.cp, d.nMP, d.nMQ, np * kFWarps, segs, lane,
                             [&](int sel, int& s0, int& s1) { chunk_range(cx, np, sel / kFWarps, sel % kFWarps, s0, s1); });
 }
 
@@ -279,7 +279,10 @@ __device__ __forceinline__ void f_step_sweep1_single(const float (&va)[EPV], con
     sP += static_cast<double>(vsB);
 }
 
-template <int DT>
+// PROBS: the rows hold probabilities (used as stored) instead of logits: no row has a first sweep,
+// the blocks are folded by the post warps when the launch starts, and the residual terms are formed
+// from the stored numbers.
+template <int DT, bool PROBS>
 __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Params prm, const FlowScratch fl) {
     using R = Raw<DT>;
     constexpr int EPV = R::EPV;
@@ -319,6 +322,11 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         // Every step here is a round trip to global memory of a few microseconds on a busy GPU; three
         // warps working on different items keep up with items of a few microseconds each.
         const int k = warp - kFWarps - 1;
+        if (PROBS) {
+            // every block's ratios are read off its rows and the block is folded (Algorithm 1: decided)
+            for (int b = static_cast<int>(blockIdx.x) * kFPost + k; b < cx.B; b += static_cast<int>(gridDim.x) * kFPost)
+                f_probs_start<DT>(prm, fl, cx, b, lane);
+        }
         for (int n = k;; n += kFPost) {
             const int slot = n % kFDesc;
             const uint32_t par = static_cast<uint32_t>(n / kFDesc) & 1u;
@@ -333,19 +341,19 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh.freeb[slot]));
             const FlowDesc d = sh.sdesc[k];
-            if (d.kind == kSweep1) f_store_sweep1<DT>(prm, fl, cx, sh, k, d.ri, d.ch, lane);
+            if (!PROBS && d.kind == kSweep1) f_store_sweep1<DT>(prm, fl, cx, sh, k, d.ri, d.ch, lane);
             else f_store_sweep2(fl, sh, k, d.ri, d.ch, lane);
             __threadfence();
             __syncwarp();
             int last = 0;
             if (lane == 0) {
-                if (d.kind == kSweep1) last = atomicAdd(&fl.row_cnt[d.ri], 1u) == static_cast<unsigned>(f_nch_row(fl, d.ri % (g + 1), g)) - 1u;
+                if (!PROBS && d.kind == kSweep1) last = atomicAdd(&fl.row_cnt[d.ri], 1u) == static_cast<unsigned>(f_nch_row(fl, d.ri % (g + 1), g)) - 1u;
                 else last = atomicAdd(&fl.s2_cnt[d.ri], 1u) == static_cast<unsigned>(fl.np) - 1u;
             }
             last = __shfl_sync(0xffffffffu, last, 0);
             if (last) {
-                if (d.kind == kSweep1) f_complete_sweep1<DT>(prm, fl, cx, d.ri, lane);
-                else f_complete_sweep2<DT>(prm, fl, cx, d, lane);
+                if (!PROBS && d.kind == kSweep1) f_complete_sweep1<DT>(prm, fl, cx, d.ri, lane);
+                else f_complete_sweep2<DT, PROBS>(prm, fl, cx, d, lane);
             }
             __syncwarp();
             if (lane == 0) atomicAdd(&sh.posted, 1u);
@@ -548,6 +556,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
     // copy group (an empty one when nothing was asked for), so "all but the kFSlots - 1 newest groups
     // are complete" always means that the slot about to be consumed has landed.
     constexpr uint32_t kCell = kFThreads * 16;               // bytes between consecutive ring cells of a thread
+    constexpr uint32_t kPad = PROBS ? 0u : R::kNegInf;       // what a lane beyond the end of a segment finds: no weight
     const uint32_t sb = smem_u32(dyn) + static_cast<uint32_t>(tid) * 16u;   // this thread's ring cell 0
     const uint32_t ring_end = sb + kFDepth * kCell;
     // Every load streams past L2 (its lines are the first to be evicted).  Leaving the first sweep's
@@ -601,8 +610,8 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             cp_async16_hint(slot_addr, iA, pol);
             cp_async16_hint(slot_addr + kCell, iB, pol);
         } else if (i_rem > 0) {                              // the short last step of a segment
-            ring_fetch_hint(slot_addr, iA, lane < i_rem, R::kNegInf, pol);
-            ring_fetch_hint(slot_addr + kCell, iB, lane + (i_adv - 32) < i_rem, R::kNegInf, pol);
+            ring_fetch_hint(slot_addr, iA, lane < i_rem, kPad, pol);
+            ring_fetch_hint(slot_addr + kCell, iB, lane + (i_adv - 32) < i_rem, kPad, pol);
         }
         if (i_rem > 0) {
             i_rem -= i_adv;
@@ -647,7 +656,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
                 if (rp == ring_end) rp = sb;
             }
         };
-        if (kind == kSweep1) {
+        if (!PROBS && kind == kSweep1) {
             if (c_left > 0) {                                // references from the first vector of every lane
                 cp_async_wait<kFSlots - 1>();
                 float va[EPV], vb[EPV];
@@ -685,13 +694,13 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             if (have_q) {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
                     float t[EPV];
-                    acc += static_cast<double>(f_pair_sum<EPV, true>(va, vb, kf, cp, nMP, nMQ, t));
+                    acc += static_cast<double>(f_pair_sum<EPV, true, PROBS>(va, vb, kf, cp, nMP, nMQ, t));
                 });
             } else {
                 run_steps([&](const float (&va)[EPV], const float (&vb)[EPV]) {
                     float t[EPV];
-                    acc += static_cast<double>(f_pair_sum<EPV, false>(va, va, kf, cp, nMP, nMQ, t));
-                    acc += static_cast<double>(f_pair_sum<EPV, false>(vb, vb, kf, cp, nMP, nMQ, t));
+                    acc += static_cast<double>(f_pair_sum<EPV, false, PROBS>(va, va, kf, cp, nMP, nMQ, t));
+                    acc += static_cast<double>(f_pair_sum<EPV, false, PROBS>(vb, vb, kf, cp, nMP, nMQ, t));
                 });
             }
             const double tP = warp_sum_d(acc);
@@ -780,7 +789,8 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->nch = plan.nch;
     fl->keep_l2 = 0;
     fl->part_stride = plan.part_stride();
-    fl->total_s1 = static_cast<unsigned>(B) * (plan.tv_spec > 0 ? plan.tv_spec : gamma) * plan.nch;
+    fl->total_s1 = plan.probs ? 0u : static_cast<unsigned>(B) * (plan.tv_spec > 0 ? plan.tv_spec : gamma) * plan.nch;
+    fl->tail_mode = plan.tail_mode;
     fl->nch_late = plan.nch_late;
     fl->np = plan.np;
     fl->depth = 3;
@@ -798,8 +808,9 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
 //   Second sweep, and the first sweep of a last target row that turns out to be wanted: only few rows
 //   are concerned and a block's candidates are swept one after the other, so these rows are cut into
 //   pieces of about 4000 vectors that many CTAs share.
-FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces, bool token_verify) {
+FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces, bool token_verify, bool probs) {
     FlowPlan pl{};
+    pl.probs = probs;
     long long np = units / 3500;
     if (np < 1) np = 1;
     if (np > 128 / kFWarps) np = 128 / kFWarps;             // (a position's segment totals are looked at four per lane)
@@ -820,6 +831,11 @@ FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair
     // read.  Smaller batches leave the GPU idle while a block waits for its next row: there, as many rows
     // from the start as it takes to give every CTA an item (at least two), and once all of those have
     // passed, which marks a draft that is mostly accepted, all the remaining rows at once.
+    // Given probabilities nothing is swept before a block's candidates are known.  A batch whose
+    // highest candidates alone give every CTA a few pieces sweeps them from the top down, one at a
+    // time (the fewest bytes); a smaller one starts all of a block's candidates at once.
+    pl.tail_mode = 0;
+    if (probs) pl.tail_mode = static_cast<long long>(B) * pl.np >= 2 * nctas ? 2 : 1;
     pl.tv_spec = 0;
     pl.tv_ahead = 1;
     if (token_verify) {
@@ -836,8 +852,9 @@ FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair
 }
 
 using FKernelFn = void (*)(const Params, const FlowScratch);
-static FKernelFn pick_flow(int dtype) {
-    return dtype == kF32 ? verify_flow_kernel<kF32> : verify_flow_kernel<kBF16>;
+static FKernelFn pick_flow(int dtype, bool probs) {
+    if (probs) return dtype == kF32 ? verify_flow_kernel<kF32, true> : verify_flow_kernel<kBF16, true>;
+    return dtype == kF32 ? verify_flow_kernel<kF32, false> : verify_flow_kernel<kBF16, false>;
 }
 
 static constexpr size_t kFlowSmem = sizeof(uint4) * kFDepth * kFThreads;
@@ -846,12 +863,15 @@ int flow_threads() { return kFAllThreads; }
 
 int flow_max_ctas_per_sm(int dtype) {
     int n = 0;
-    if (cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_flow(dtype)),
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kFlowSmem)) != cudaSuccess) {
-        cudaGetLastError();
-        return 0;
+    for (int probs = 0; probs < 2; ++probs) {
+        if (cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_flow(dtype, probs != 0)),
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kFlowSmem)) != cudaSuccess) {
+            cudaGetLastError();
+            return 0;
+        }
     }
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_flow(dtype), kFAllThreads, kFlowSmem) != cudaSuccess) {
+    // (the variant on logits is the larger program: its occupancy serves both)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_flow(dtype, false), kFAllThreads, kFlowSmem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -860,7 +880,7 @@ int flow_max_ctas_per_sm(int dtype) {
 
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl_in, int dtype, int nctas, cudaStream_t stream) {
     const FlowScratch& fl = fl_in;
-    pick_flow(dtype)<<<nctas, kFAllThreads, kFlowSmem, stream>>>(prm, fl);
+    pick_flow(dtype, prm.probs != 0)<<<nctas, kFAllThreads, kFlowSmem, stream>>>(prm, fl);
     return cudaGetLastError();
 }
 

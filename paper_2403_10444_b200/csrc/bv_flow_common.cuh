@@ -59,13 +59,19 @@ template <int EPV> __device__ __forceinline__ void f_accumulate(const float (&v)
     }
     s += vs;
 }
-// residual terms t_e = max(cp 2^{zP k - MP} - 2^{zQ k - MQ}, 0) and their sum; HAVEQ = false: t_e = cp 2^{zP k - MP}
-template <int EPV, bool HAVEQ>
+// residual terms t_e = max(cp 2^{zP k - MP} - 2^{zQ k - MQ}, 0) and their sum; HAVEQ = false: t_e = cp 2^{zP k - MP}.
+// PROBS: the rows hold probabilities, t_e = max(cp P_e - Q_e, 0) resp. cp P_e.
+template <int EPV, bool HAVEQ, bool PROBS = false>
 __device__ __forceinline__ float f_pair_sum(const float (&vp)[EPV], const float (&vq)[EPV], float kf, float cp,
                                             float nMP, float nMQ, float (&t)[EPV]) {
     float a[EPV], q[EPV];
-    f_exps<EPV>(vp, kf, nMP, a);
-    if (HAVEQ) f_exps<EPV>(vq, kf, nMQ, q);
+    if (PROBS) {
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) { a[e] = vp[e]; q[e] = vq[e]; }
+    } else {
+        f_exps<EPV>(vp, kf, nMP, a);
+        if (HAVEQ) f_exps<EPV>(vq, kf, nMQ, q);
+    }
     const float2 cc = f2(cp, cp), ncc = f2(-cp, -cp);
 #pragma unroll
     for (int e = 0; e < EPV; e += 2) {
@@ -118,10 +124,11 @@ struct FlowCtx {
 
 // One warp walks segment [w0, w1) of a row pair in index order and returns the first element
 // whose running residual mass exceeds tw (else the last element with positive mass, else -1).
-template <int DT>
+template <int DT, bool PROBS = false>
 __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int lane, float kf, float cp,
                         float nMP, float nMQ, double tw) {
     constexpr int EPV = Raw<DT>::EPV;
+    constexpr uint32_t kPad = PROBS ? 0u : Raw<DT>::kNegInf;   // an element beyond the segment weighs nothing
     constexpr int kAhead = 4;                                // runs of 32 vectors whose loads are in flight together
     // The terms are the fp32 values of the sweeps; their running sum, which decides the token, is
     // kept in fp64 (a cell of the distribution can be far narrower than fp32 resolves next to the
@@ -136,8 +143,8 @@ __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int 
         for (int a = 0; a < kAhead; ++a) {
             const int i = base0 + 32 * a + lane;
             const bool ok = i < w1;
-            rp[a] = ok ? ld_stream_v4(rowP + static_cast<size_t>(i) * 16) : make_uint4(Raw<DT>::kNegInf, Raw<DT>::kNegInf, Raw<DT>::kNegInf, Raw<DT>::kNegInf);
-            rq[a] = (ok && rowQ) ? ld_stream_v4(rowQ + static_cast<size_t>(i) * 16) : make_uint4(Raw<DT>::kNegInf, Raw<DT>::kNegInf, Raw<DT>::kNegInf, Raw<DT>::kNegInf);
+            rp[a] = ok ? ld_stream_v4(rowP + static_cast<size_t>(i) * 16) : make_uint4(kPad, kPad, kPad, kPad);
+            rq[a] = (ok && rowQ) ? ld_stream_v4(rowQ + static_cast<size_t>(i) * 16) : make_uint4(kPad, kPad, kPad, kPad);
         }
 #pragma unroll
         for (int a = 0; a < kAhead; ++a) {
@@ -147,8 +154,8 @@ __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int 
             float vp[EPV], vq[EPV], tt[EPV];
             Raw<DT>::unpack(rp[a], vp);
             Raw<DT>::unpack(rq[a], vq);
-            if (rowQ) f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, tt);
-            else f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, tt);
+            if (rowQ) f_pair_sum<EPV, true, PROBS>(vp, vq, kf, cp, nMP, nMQ, tt);
+            else f_pair_sum<EPV, false, PROBS>(vp, vq, kf, cp, nMP, nMQ, tt);
             double ls = 0.0;
 #pragma unroll
             for (int e = 0; e < EPV; ++e) {
@@ -284,6 +291,13 @@ static __device__ void f_finalize_block(const Params& prm, const FlowScratch& fl
     if (lane == 0) atomicAdd(&fl.counters[kCtrBlocks], 1u);      // (CTAs leave when every block is finished)
 }
 
+// Is the GPU emptying (the first-sweep tickets have run out), so that a block's candidates are all
+// started at once?  A launch on probabilities has no first sweep; it says which way it wants it.
+__device__ __forceinline__ bool f_tail(const FlowScratch& fl) {
+    if (fl.tail_mode) return fl.tail_mode == 1;
+    return ld_volatile(&fl.counters[kCtrTicket]) >= fl.total_s1;
+}
+
 // Is the token of position gamma drawn from the first sweep of the last target row (bv_flow.cu)?
 __device__ __forceinline__ bool f_draws_in_sweep1(const Params& prm, int nch_late) {
     return !f_all_positions(prm) && nch_late <= 8;
@@ -340,7 +354,7 @@ static __device__ void f_position_done(const Params& prm, const FlowScratch& fl,
         const double p_i = __ldcg(&fl.pchain[static_cast<size_t>(b) * (g + 2) + i]);
         const double S_i = i < g ? __ldcg(&fl.S[row0 + i]) : 0.0;
         const float eta_i = i >= 1 ? prm.uni[static_cast<size_t>(b) * (g + 2) + i - 1] : 0.f;
-        const bool tail = ld_volatile(&fl.counters[kCtrTicket]) >= fl.total_s1;
+        const bool tail = f_tail(fl);
         const double hw = i == g ? p_i : f_weight(p_i, S_i);
         const bool selected = i == 0 || (hw > 0.0 && static_cast<double>(eta_i) <= hw);
         const unsigned hold_lo = __ballot_sync(0xffffffffu, rl[0] == kRelHold), hold_hi = __ballot_sync(0xffffffffu, rl[1] == kRelHold);
@@ -493,7 +507,7 @@ __device__ void f_fold_block(const Params& prm, const FlowScratch& fl, const Flo
         eta[h] = (c >= 1 && c < g) ? u[c - 1] : 0.f;
     }
     const float eta_g = u[g - 1];
-    const bool tail = ld_volatile(&fl.counters[kCtrTicket]) >= fl.total_s1;
+    const bool tail = f_tail(fl);
     // the recursion, by every lane alike; a lane keeps the p of its own positions
     double pc = 1.0, mine[2] = {1.0, 1.0};
     for (int c = 0; c < g; ++c) {
@@ -549,12 +563,16 @@ __device__ void f_fold_block(const Params& prm, const FlowScratch& fl, const Flo
             fl.rel[row0 + c] = started ? kRelSweep : (need[h] ? kRelHold : kRelSkip);
         }
     }
-    if (lane == 0) fl.rel[row0 + g] = last_row_wanted ? kRelLate : kRelSkip;
+    if (lane == 0) fl.rel[row0 + g] = last_row_wanted ? (prm.probs ? kRelSweep : kRelLate) : kRelSkip;
     __threadfence();
     __syncwarp();
     f_queue_rows(fl, b, g, s_lo, s_hi, lane);
     if (lane == 0) {
-        if (last_row_wanted) {            // the last target row joins the queue of its kind
+        if (last_row_wanted && prm.probs) {
+            // (given probabilities there is no normaliser to learn: P_gamma is swept once, as a position like the others)
+            const unsigned slot = atomicAdd(&fl.counters[kCtrQueued], 1u);
+            atomicExch(&fl.s2q[slot], static_cast<unsigned>(row0 + g) + 1u);
+        } else if (last_row_wanted) {     // the last target row joins the queue of its kind
             const unsigned slot = atomicAdd(&fl.counters[kCtrLateQueued], 1u);
             atomicExch(&fl.lq[slot], static_cast<unsigned>(row0 + g) + 1u);
         }
@@ -621,10 +639,69 @@ __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const F
     __syncwarp();
 }
 
+// ---- a launch on given probabilities (one warp per block, at the start of the launch): the ratios
+// P_r(X_{r+1}) / Q_r(X_{r+1}) are read off the rows, no row needs a first sweep.  Algorithm 2: the block is
+// folded at once.  Algorithm 1: tau is known at once, and the one position to sample from is queued. ----
+template <int DT>
+__device__ void f_probs_start(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int lane) {
+    const int g = cx.g;
+    const size_t row0 = static_cast<size_t>(b) * (g + 1);
+    bool okrow[2] = {true, true};
+    double rat[2] = {0.0, 0.0};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int r = lane + 32 * h;
+        if (r < g) {
+            const int x = prm.tok[static_cast<size_t>(b) * g + r];
+            bool ok = x >= 0 && x < cx.V;
+            double P = 0.0, Q = 1.0;
+            if (ok) {
+                P = load_logit<DT>(static_cast<const char*>(prm.tgt) + (row0 + r) * cx.row_bytes, x);
+                Q = load_logit<DT>(static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + r) * cx.row_bytes, x);
+                ok = Q > 0.0 && Q < static_cast<double>(INFINITY) && P >= 0.0 && P < static_cast<double>(INFINITY);
+            }
+            okrow[h] = ok;
+            rat[h] = ok ? P / Q : 0.0;
+            fl.ratio[row0 + r] = rat[h];
+            fl.zratio[row0 + r] = 1.0;
+        }
+        if (r <= g) { RowZ z; z.MP = 0.0; z.ZP = 1.0; z.MQ = 0.0; z.ZQ = 1.0; fl.rowZ[row0 + r] = z; }
+    }
+    const unsigned bad_lo = __ballot_sync(0xffffffffu, !okrow[0]), bad_hi = __ballot_sync(0xffffffffu, !okrow[1]);
+    if (!fl.tv) {
+        if (lane == 0 && (bad_lo | bad_hi)) atomicOr(&fl.bad[b], 1u);
+        __threadfence();
+        __syncwarp();
+        f_fold_block<DT>(prm, fl, cx, b, lane);
+        return;
+    }
+    // Algorithm 1: tests 1 .. gamma in order, test r + 1 on row r; tau = the number passed before the first failure
+    bool pass[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int r = lane + 32 * h;
+        const double hw = fmin(rat[h], 1.0);
+        pass[h] = r >= g || (hw > 0.0 && static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + r]) <= hw);
+    }
+    const unsigned f_lo = __ballot_sync(0xffffffffu, !pass[0]), f_hi = __ballot_sync(0xffffffffu, !pass[1]);
+    const int tau = f_lo ? __ffs(f_lo) - 1 : (f_hi ? 32 + __ffs(f_hi) - 1 : g);
+    if (lane == 0) {
+        // (a fault counts if its row is among the ones Algorithm 1 reads: rows 0 .. min(tau, gamma - 1))
+        const unsigned long long badrows = static_cast<unsigned long long>(bad_lo) | (static_cast<unsigned long long>(bad_hi) << 32);
+        if (badrows) atomicOr(&fl.tv_badrows[b], badrows);
+        fl.tv_tau[b] = tau;
+        fl.cscale[row0 + tau] = 1.f;
+        __threadfence();
+        const unsigned slot = atomicAdd(&fl.counters[kCtrQueued], 1u);
+        atomicExch(&fl.s2q[slot], static_cast<unsigned>(row0 + tau) + 1u);
+    }
+    __syncwarp();
+}
+
 // ---- a position is complete (one warp): S_r from the segment totals, and the candidate Y_r.
 // `segs` holds the nseg <= 128 totals of the row's segments in index order (four per lane);
 // range(s, v0, v1) gives the vectors [v0, v1) of segment s. ----
-template <int DT, class RangeFn>
+template <int DT, bool PROBS = false, class RangeFn>
 __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int ri, bool have_q,
                                     const char* rowP, const char* rowQ, float cp, float nMP, float nMQ,
                                     int nseg, const double* segs, int lane, RangeFn range) {
@@ -650,7 +727,7 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
     const double total = shfl_d(inc, 31);
     if (lane == 0 && have_q) fl.S[ri] = total / ZQ;
     int found = -1;
-    if (total > 0.0) {
+    if (total > 0.0 && total < static_cast<double>(INFINITY)) {
         const double t = static_cast<double>(uf) * total;
         double exc = shfl_up_d(inc, 1);
         if (lane == 0) exc = 0.0;
@@ -675,7 +752,7 @@ __device__ void f_position_complete(const Params& prm, const FlowScratch& fl, co
         const double before = shfl_d(bef, src);
         int s0, s1;
         range(sel, s0, s1);
-        found = f_rescan<DT>(rowP, rowQ, s0, s1, lane, cx.kf, cp, nMP, nMQ, t - before);
+        found = f_rescan<DT, PROBS>(rowP, rowQ, s0, s1, lane, cx.kf, cp, nMP, nMQ, t - before);
     }
     // (an empty residual leaves no candidate: the position cannot be the selected one, see the end of a block)
     if (lane == 0) fl.cand[ri] = found;

@@ -71,6 +71,8 @@ struct FlowScratch {
     unsigned zero_words;  // 32-bit words at the start of the scratch area (from `counters` on) that start and end at zero
     int depth;            // flow kernel: descriptors a CTA may have handed to its workers and not yet seen swept
     int segs;             // residual totals kept per row
+    int tail_mode;        // 0: a block's candidates are started all at once when the first-sweep tickets have run out;
+                          // 1: always (a launch without first sweeps that would not fill the GPU); 2: never
     int keep_l2;          // tuning switch: first-sweep loads leave their lines at normal priority in L2 (default: evicted first)
 };
 constexpr int kFlowMaxChunks = 32;
@@ -80,11 +82,13 @@ struct FlowPlan {
     int nch, nch_late, np;
     int tv_spec;          // Token Verification: rows of every block swept from the start (0: Block Verification)
     int tv_ahead;         // Token Verification: rows asked for beyond the last test that passed
+    bool probs;           // the rows hold probabilities: no first sweep
+    int tail_mode;        // see FlowScratch
     int part_stride() const { return nch > nch_late ? nch : nch_late; }
 };
 // units: 16-byte vectors per row; pair_items: false when the first sweep streams one row per item
 // (supplied draft normalisers); chunks / pieces > 0 force the chunk count / the piece count.
-FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces, bool token_verify = false);
+FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair_items, int chunks, int pieces, bool token_verify = false, bool probs = false);
 size_t flow_scratch_bytes(int B, int gamma, const FlowPlan& plan, size_t* zero_bytes);
 void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, FlowScratch* fl);
 int flow_max_ctas_per_sm(int dtype);

@@ -103,17 +103,19 @@ def _widen(row: np.ndarray) -> np.ndarray:
     return row.astype(np.float64)
 
 
-def token_is_valid(algo, ref, inp_np, b, y) -> bool:
+def token_is_valid(algo, ref, inp_np, b, y, probs=False) -> bool:
     """Is token y within 1e-6 (in probability) of the CDF cell the sampling uniform falls in,
-    under the oracle's normalisers and p for sequence b?  (fp64, index order.)"""
+    under the oracle's normalisers and p for sequence b?  (fp64, index order.)  ``probs``: the
+    rows hold probabilities, used as stored."""
     tgt, drf, uni, T = inp_np
     g = drf.shape[1]
     tau = int(ref.out_len[b]) - 1
     T = float(np.float32(T))
-    P = np.exp(_widen(tgt[b, tau]) / T - ref.lse_t[b, tau])
+    P = _widen(tgt[b, tau]) if probs else np.exp(_widen(tgt[b, tau]) / T - ref.lse_t[b, tau])
     if tau < g:
         p = ref.p[b, tau] if algo != oracle.TOKEN_VERIFY else 1.0   # (the unclipped product for Algorithm 4)
-        w = np.maximum(p * P - np.exp(_widen(drf[b, tau]) / T - ref.lse_d[b, tau]), 0.0)
+        Q = _widen(drf[b, tau]) if probs else np.exp(_widen(drf[b, tau]) / T - ref.lse_d[b, tau])
+        w = np.maximum(p * P - Q, 0.0)
         if not w.sum() > 0:
             w = P
         u = float(uni[b, g])
@@ -127,7 +129,7 @@ def token_is_valid(algo, ref, inp_np, b, y) -> bool:
     return lo - NEAR <= u <= hi + NEAR
 
 
-def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=None, inp=None) -> ParityReport:
+def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=None, inp=None, probs=False) -> ParityReport:
     ot = out_tokens.cpu().numpy()
     ol = out_len.cpu().numpy()
     B = ol.shape[0]
@@ -151,7 +153,7 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
             if inp is not None and inp_np is None:
                 inp_np = (to_numpy_logits(inp["target_logits"]), to_numpy_logits(inp["draft_logits"]),
                           inp["uniforms"].cpu().numpy(), inp["temperature"])
-            if prefix_same and inp_np is not None and token_is_valid(algo, ref, inp_np, b, int(ot[b, tau])):
+            if prefix_same and inp_np is not None and token_is_valid(algo, ref, inp_np, b, int(ot[b, tau]), probs):
                 excused_Y += 1
             else:
                 hard += 1
@@ -162,10 +164,11 @@ def compare(algo: int, ref: "oracle.OracleResult", out_tokens, out_len, diag=Non
         S = diag["S"].cpu().numpy().astype(np.float64)
         h = diag["h"].cpu().numpy().astype(np.float64)
         p = diag["p"].cpu().numpy().astype(np.float64)
-        lt = diag["lse_t"].cpu().numpy().astype(np.float64)
-        ld = diag["lse_d"].cpu().numpy().astype(np.float64)
         rows = ok_rows
-        for got, want in ((lt, ref.lse_t), (ld, ref.lse_d)):
+        # (the entry points on probabilities form no normalisers)
+        pairs = [] if "lse_t" not in diag else [(diag["lse_t"].cpu().numpy().astype(np.float64), ref.lse_t),
+                                                (diag["lse_d"].cpu().numpy().astype(np.float64), ref.lse_d)]
+        for got, want in pairs:
             m = rows[:, None] & ~np.isnan(want)
             assert not np.isnan(got[m]).any(), "CUDA path left a log-normaliser unset"
             if m.any():
