@@ -32,14 +32,21 @@ ALGOS = ("block_lse", "block", "token")
 
 def run(target_table: torch.Tensor, draft_table: torch.Tensor, first_tokens: torch.Tensor,
         u_draft: torch.Tensor, u_verify: torch.Tensor, gamma: int, temperature: float = 1.0,
-        algo: str = "block_lse") -> Dict[str, torch.Tensor]:
+        algo: str = "block_lse", graph: bool = False) -> Dict[str, torch.Tensor]:
     """Run ``u_draft.shape[0]`` iterations of Algorithm 3 for ``first_tokens.shape[0]`` sequences.
 
-    target_table, draft_table: CUDA [V, V] float32 or bfloat16 (row t = logits after token t);
-    first_tokens: CUDA int32 [B], the last token of each context; u_draft [N, gamma, B] and
-    u_verify [N, B, gamma+2]: CUDA float32 uniforms.  Returns ``tokens`` int32 [B, N (gamma+1)]
-    (generated tokens, then -1), ``lengths`` int64 [B], ``tau`` int32 [N, B] (accepted draft tokens
-    per iteration) and ``drafted`` int32 [N, B, gamma].
+    target_table, draft_table: CUDA [V, V] float32 or bfloat16 (row t = logits after token t; -inf
+    entries, as a top-k / top-p mask leaves them, are allowed); first_tokens: CUDA int32 [B], the
+    last token of each context; u_draft [N, gamma, B] and u_verify [N, B, gamma+2]: CUDA float32
+    uniforms.  Returns ``tokens`` int32 [B, N (gamma+1)] (generated tokens, then -1), ``lengths``
+    int64 [B], ``tau`` int32 [N, B] (accepted draft tokens per iteration) and ``drafted`` int32
+    [N, B, gamma].
+
+    Every step of an iteration has fixed shapes and runs on the device without a host round trip
+    (the iteration number lives in a device counter), so with ``graph=True`` one iteration is
+    captured in a CUDA graph and replayed: the 5 gamma + 12 launches of an iteration then cost one
+    graph launch instead of one driver call each.  Data faults are looked for once, after the last
+    iteration.
     """
     if algo not in ALGOS:
         raise ValueError("algo must be one of %s" % (ALGOS,))
@@ -51,44 +58,72 @@ def run(target_table: torch.Tensor, draft_table: torch.Tensor, first_tokens: tor
         raise ValueError("u_draft must be [N, gamma, B] and u_verify [N, B, gamma+2]")
     dev = target_table.device
     width = N * (gamma + 1)
-    seq = torch.full((B, width), -1, dtype=torch.int32, device=dev)
+    # state of the loop, updated in place (column `width` of seq takes what is not kept)
+    seq = torch.full((B, width + 1), -1, dtype=torch.int32, device=dev)
     pos = torch.zeros((B,), dtype=torch.int64, device=dev)
     taus = torch.empty((N, B), dtype=torch.int32, device=dev)
     drafted = torch.empty((N, B, gamma), dtype=torch.int32, device=dev)
-    cur = first_tokens.to(torch.int64)
+    cur = first_tokens.to(torch.int64).clone()
+    it = torch.zeros((1,), dtype=torch.int64, device=dev)          # the iteration number, on the device
+    fault = torch.zeros((1,), dtype=torch.int32, device=dev)
     draft_logits = torch.empty((B, gamma, V), dtype=draft_table.dtype, device=dev)
+    target_logits = torch.empty((B, gamma + 1, V), dtype=target_table.dtype, device=dev)
     lse = torch.empty((B, gamma), dtype=torch.float32, device=dev)
+    toks = torch.empty((B, gamma), dtype=torch.int32, device=dev)
     col = torch.arange(gamma + 1, device=dev)
-    for n in range(N):
+    trash = torch.full((1,), width, dtype=torch.int64, device=dev)
+
+    def iteration():
+        ud = u_draft.index_select(0, it)[0]                        # [gamma, B]
+        uv = u_verify.index_select(0, it)[0]                       # [B, gamma+2]
         # drafting step: X_1..X_gamma ~ M_s autoregressively, keeping the conditional rows
         last = cur
         for i in range(gamma):
             rows = draft_table.index_select(0, last)
-            tok, row_lse = bv.bv_sample_draft(rows, u_draft[n, i].contiguous(), temperature)
+            tok, row_lse = bv.bv_sample_draft(rows, ud[i], temperature)
             draft_logits[:, i] = rows
             lse[:, i] = row_lse
-            drafted[n, :, i] = tok
+            toks[:, i] = tok
             last = tok.to(torch.int64)
         # the large model's conditional rows along the drafted path, gamma + 1 of them
-        path = torch.cat([cur[:, None], drafted[n].to(torch.int64)], dim=1)
-        target_logits = target_table.index_select(0, path.reshape(-1)).view(B, gamma + 1, V)
-        toks = drafted[n].contiguous()
+        path = torch.cat([cur[:, None], toks.to(torch.int64)], dim=1)
+        torch.index_select(target_table, 0, path.reshape(-1), out=target_logits.view(B * (gamma + 1), V))
         if algo == "block_lse":
-            out, out_len = bv.bv_verify_lse(target_logits, draft_logits, toks, u_verify[n], lse, temperature)
+            out, out_len = bv.bv_verify_lse(target_logits, draft_logits, toks, uv, lse, temperature)
         elif algo == "block":
-            out, out_len = bv.bv_verify(target_logits, draft_logits, toks, u_verify[n], temperature)
+            out, out_len = bv.bv_verify(target_logits, draft_logits, toks, uv, temperature)
         else:
-            out, out_len = bv.tv_verify(target_logits, draft_logits, toks, u_verify[n], temperature)
-        if bool((out_len < 1).any()):
-            raise RuntimeError("a sequence reported a data fault (out_len = -1)")
-        n_out = out_len.to(torch.int64)
+            out, out_len = bv.tv_verify(target_logits, draft_logits, toks, uv, temperature)
+        fault.add_((out_len < 1).any().to(torch.int32))
+        n_out = out_len.to(torch.int64).clamp_(min=1)
         keep = col[None, :] < n_out[:, None]
-        flat = (torch.arange(B, device=dev)[:, None] * width + pos[:, None] + col[None, :])[keep]
-        seq.view(-1)[flat] = out[keep]
-        cur = out.gather(1, (n_out - 1)[:, None]).squeeze(1).to(torch.int64)
-        pos = pos + n_out
-        taus[n] = out_len - 1
-    return dict(tokens=seq, lengths=pos, tau=taus, drafted=drafted)
+        seq.scatter_(1, torch.where(keep, pos[:, None] + col[None, :], trash), out)
+        cur.copy_(out.gather(1, (n_out - 1)[:, None]).squeeze(1))
+        pos.add_(n_out)
+        taus.index_copy_(0, it, (out_len - 1)[None, :])
+        drafted.index_copy_(0, it, toks[None])
+        it.add_(1)
+
+    if graph and N > 1:
+        # the first iteration runs eagerly on the side stream (the library sizes its workspace for
+        # that stream, torch its caches); the second is captured, and replayed for the rest
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream(dev))
+        with torch.cuda.stream(side):
+            iteration()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            iteration()
+        # (capturing has not run anything: replay it for iterations 1 .. N-1)
+        torch.cuda.current_stream(dev).wait_stream(side)
+        for _ in range(N - 1):
+            g.replay()
+    else:
+        for _ in range(N):
+            iteration()
+    if int(fault.item()) != 0:
+        raise RuntimeError("a sequence reported a data fault (out_len = -1)")
+    return dict(tokens=seq[:, :width].contiguous(), lengths=pos, tau=taus, drafted=drafted)
 
 
 def block_efficiency(result) -> float:
@@ -105,22 +140,26 @@ def main():
     ap.add_argument("--draft-sigma", type=float, default=1.0)
     ap.add_argument("--temperature", type=float, default=1.0)
     ap.add_argument("--seed", type=int, default=7)
+    ap.add_argument("--top-p", type=float, default=0.0, help="mask both models' rows to their top-p nucleus")
+    ap.add_argument("--graph", action="store_true", help="replay one captured iteration as a CUDA graph")
     args = ap.parse_args()
     bv.load_library()
     tt, dt = wl.markov_models(args.V, "bf16", args.seed, 2.0, args.draft_sigma, 1.1, "cuda")
+    if args.top_p > 0:
+        tt, dt = wl.top_p_mask(tt, args.top_p, args.temperature), wl.top_p_mask(dt, args.top_p, args.temperature)
     first = torch.zeros((args.B,), dtype=torch.int32, device="cuda")
     for gamma in [int(x) for x in args.gammas.split(",")]:
         ud, uv = wl.loop_uniforms(args.iterations, args.B, gamma, args.seed + gamma, "cuda")
         for algo in ALGOS:
-            run(tt, dt, first, ud[:2], uv[:2], gamma, args.temperature, algo)       # warm-up
+            run(tt, dt, first, ud[:2], uv[:2], gamma, args.temperature, algo, args.graph)       # warm-up
             torch.cuda.synchronize()
             t0 = time.perf_counter()
-            res = run(tt, dt, first, ud, uv, gamma, args.temperature, algo)
+            res = run(tt, dt, first, ud, uv, gamma, args.temperature, algo, args.graph)
             torch.cuda.synchronize()
             dt_s = time.perf_counter() - t0
             print(json.dumps({"V": args.V, "B": args.B, "gamma": gamma, "algo": algo,
                               "iterations": args.iterations, "draft_sigma": args.draft_sigma,
-                              "temperature": args.temperature,
+                              "temperature": args.temperature, "top_p": args.top_p or None, "graph": args.graph,
                               "block_efficiency": round(block_efficiency(res), 4),
                               "tokens": int(res["lengths"].sum().item()),
                               "ms_per_iteration": round(dt_s / args.iterations * 1e3, 3),

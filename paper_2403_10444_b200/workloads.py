@@ -123,6 +123,19 @@ def markov_models(V: int, dtype: str, seed: int, target_sigma: float = 2.0, draf
     return t.to(td), d.to(td)
 
 
+def top_p_mask(table: torch.Tensor, top_p: float, temperature: float = 1.0) -> torch.Tensor:
+    """Nucleus masking of every row of a [V, V] table of logits: the tokens of a row are kept in
+    order of decreasing probability under softmax(row / temperature) until their mass reaches
+    ``top_p`` (the token that crosses it included), the others are set to -inf.  Same dtype."""
+    z = table.float() / temperature
+    order = z.argsort(dim=1, descending=True)
+    prob = torch.softmax(z, dim=1).gather(1, order)
+    before = prob.cumsum(dim=1) - prob                    # mass of the tokens ahead of each one
+    drop_sorted = before >= top_p
+    drop = torch.zeros_like(drop_sorted).scatter_(1, order, drop_sorted)
+    return table.masked_fill(drop, float("-inf"))
+
+
 def loop_uniforms(iterations: int, B: int, gamma: int, seed: int, device="cpu"):
     """The uniforms one run of the decoding loop consumes: u_draft [iterations, gamma, B] (one per
     drafted token) and u_verify [iterations, B, gamma+2] (the verification's), float32 in [0, 1)."""

@@ -124,3 +124,37 @@ def test_block_verification_generates_more_per_iteration():
     first = torch.zeros(B, dtype=torch.int32, device="cuda")
     be = {a: specdec.block_efficiency(specdec.run(tt, dt, first, ud, uv, gamma, 1.0, a)) for a in specdec.ALGOS}
     assert be["block"] > be["token"] and be["block_lse"] > be["token"]
+
+
+@pytest.mark.parametrize("algo", ["block_lse", "token"])
+def test_graph_replay_generates_the_same_tokens(algo):
+    V, B, N, gamma = 4096, 48, 9, 5
+    tt, dt = wl.markov_models(V, "bf16", 41, 2.0, 1.0, 1.1, "cuda")
+    ud, uv = wl.loop_uniforms(N, B, gamma, 42, "cuda")
+    first = torch.arange(B, dtype=torch.int32, device="cuda")
+    a = specdec.run(tt, dt, first, ud, uv, gamma, 0.9, algo)
+    b = specdec.run(tt, dt, first, ud, uv, gamma, 0.9, algo, graph=True)
+    for k in ("tokens", "lengths", "tau", "drafted"):
+        assert torch.equal(a[k], b[k]), k
+
+
+@pytest.mark.parametrize("algo,oalgo", [("block", oracle.BLOCK_VERIFY), ("token", oracle.TOKEN_VERIFY)])
+def test_nucleus_masked_rows_through_the_loop(algo, oalgo):
+    # top-p masked rows (-inf outside each row's nucleus, the two models' nuclei differ): tokens the
+    # target model excludes are never emitted, and the loop still equals the oracle's
+    V, B, gamma, N, T = 1024, 10, 4, 5, 0.8
+    tt, dt = wl.markov_models(V, "f32", 51, 2.0, 1.0, 1.1, "cpu")
+    tt, dt = wl.top_p_mask(tt, 0.9, T), wl.top_p_mask(dt, 0.9, T)
+    assert 0.02 < torch.isfinite(tt).float().mean() < 0.9
+    first = torch.arange(B, dtype=torch.int32)
+    ud, uv = wl.loop_uniforms(N, B, gamma, 52, "cpu")
+    want = oracle_loop(tt, dt, first, ud, uv, gamma, T, oalgo, False)
+    res = specdec.run(tt.cuda(), dt.cuda(), first.cuda(), ud.cuda(), uv.cuda(), gamma, T, algo)
+    toks, lens = res["tokens"].cpu().numpy(), res["lengths"].cpu().numpy()
+    for b in range(B):
+        got = list(toks[b, : lens[b]])
+        assert got == want[b], b
+        prev = int(first[b])
+        for x in got:
+            assert torch.isfinite(tt[prev, x]), "a token outside the target model's nucleus was emitted"
+            prev = x
