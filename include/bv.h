@@ -282,7 +282,10 @@ int bv_stream_status(void* stream);
 
 /*
  * Tuning and test options, process-wide, read by every later call (0 restores the default choice):
- *   "kernel"        1 flow, 2 cluster, 3 element-wise streaming kernel for Block Verification
+ *   "kernel"        1 flow, 2 cluster, 3 element-wise streaming kernel, 4 small-batch kernel (for the shapes
+ *                   each admits; the default picks the small-batch kernel for up to 32 sequences whose
+ *                   logits are few enough to make the launch a matter of latency, else the flow kernel)
+ *   "small_bytes"   logit megabytes up to which the small-batch kernel is the default
  *   "cluster"       cluster width of the cluster / streaming kernels (1, 2, 4, 8)
  *   "max_clusters"  cap on the clusters those kernels launch
  *   "flow_chunks", "flow_pieces", "flow_ctas", "flow_depth"   work-item shape of the flow kernel
@@ -291,7 +294,7 @@ int bv_stream_status(void* stream);
  *   "wait_limit"    polls after which a bounded device-side wait gives up (tests)
  *   "never_signal"  tests: the flow kernel's workers never report an item as swept, so its waits
  *                   run out and the call ends with BV_ERR_TIMEOUT
- * Their first values come from the environment variables BV_KERNEL (flow / cluster / stream),
+ * Their first values come from the environment variables BV_KERNEL (flow / cluster / stream / small),
  * BV_CLUSTER, BV_MAX_CLUSTERS, BV_FLOW_CHUNKS, BV_FLOW_PIECES, BV_FLOW_CTAS, BV_FLOW_DEPTH, read once.
  * Returns BV_ERR_INVALID_ARG for an unknown name.
  */

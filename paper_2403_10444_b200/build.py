@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libbv_b200.so")
-SOURCES = ["bv_api.cu", "bv_stream.cu", "bv_cluster.cu", "bv_flow.cu", "bv_noalloc.cu", "bv_sample.cu"]
+SOURCES = ["bv_api.cu", "bv_stream.cu", "bv_cluster.cu", "bv_flow.cu", "bv_small.cu", "bv_noalloc.cu", "bv_sample.cu"]
 HEADERS = ["bv_device.cuh", "bv_launch.h", "bv_flow_common.cuh", os.path.join("..", "..", "include", "bv.h")]
 
 NVCC_FLAGS = [

@@ -15,11 +15,16 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 constexpr int kTicketSlots = 64;  // concurrent calls of the cluster kernels on one device each need their own slot
+// Logit bytes up to which the small-batch kernel is the default (measured against the flow kernel at
+// V = 152064, B <= 32: Algorithm 2 gains up to about 90 MB at low and high acceptance alike, Algorithm 1,
+// whose one residual sweep per sequence is cheap, up to about 160 MB)
+constexpr long long kSmallBytes[2] = {160LL << 20, 90LL << 20};   // [algo]
 constexpr int kStreamSlots = 32;  // streams per device that keep a workspace of their own
 
 // Tuning and test options (bv_set_option); their first values come from the environment, read once.
 struct Options {
-    int kernel = 0;        // 0: chosen by shape; 1 flow, 2 cluster, 3 stream
+    int kernel = 0;        // 0: chosen by shape; 1 flow, 2 cluster, 3 stream, 4 small-batch
+    int small_bytes = 0;   // logit bytes (in MB) up to which the small-batch kernel is chosen; 0: the built-in limit
     int cluster = 0;       // cluster width of the cluster / stream kernels (1, 2, 4, 8); 0: chosen by shape
     int max_clusters = 0;  // cap on the clusters launched; 0: none
     int flow_chunks = 0, flow_pieces = 0, flow_ctas = 0, flow_depth = 0;   // 0: chosen by shape
@@ -39,6 +44,7 @@ int kernel_code(const char* v) {
     if (!std::strcmp(v, "flow")) return 1;
     if (!std::strcmp(v, "cluster")) return 2;
     if (!std::strcmp(v, "stream")) return 3;
+    if (!std::strcmp(v, "small")) return 4;
     return 0;
 }
 void load_env_options() {
@@ -74,6 +80,7 @@ struct DeviceState {
     StreamSlot slots[kStreamSlots];
     unsigned long long clock = 0;
     int flow_ctas_per_sm[2] = {};
+    int small_ctas[2] = {};            // small-batch kernel: CTAs of a launch per dtype (0: not asked yet)
     // staging for the host-buffer entry points
     void* stage = nullptr;
     size_t stage_bytes = 0;
@@ -201,6 +208,36 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     prm.algo = algo;
     const bool flow_ok = vec && (opt.kernel == 0 || opt.kernel == 1);
     if ((prm.lse_d != nullptr || prm.greedy || prm.probs) && !flow_ok) return BV_ERR_UNSUPPORTED;
+
+    // A few sequences whose logits fit in L2: the launch is a matter of latency, and the kernel with two
+    // grid-wide barriers instead of queues takes half the time of the flow kernel or less.
+    const long long logit_bytes = static_cast<long long>(B) * (2 * gamma + 1) * static_cast<long long>(row_bytes);
+    const long long small_limit = opt.small_bytes > 0 ? static_cast<long long>(opt.small_bytes) << 20 : kSmallBytes[algo == bv::kBlockVerify ? 1 : 0];
+    if (vec && !prm.lse_d && !prm.greedy && !prm.probs && bv::small_fits(B, gamma) &&
+        (opt.kernel == 4 || (opt.kernel == 0 && logit_bytes <= small_limit))) {
+        int& nc = d->small_ctas[dtype];
+        if (nc == 0) {
+            nc = bv::small_max_ctas(dtype, d->sm_count);
+            if (nc <= 0) nc = -1;
+        }
+        if (nc > 0) {
+            const bv::SmallPlan plan = bv::small_plan(static_cast<long long>(row_bytes / 16), B, gamma, nc);
+            StreamSlot* slot = nullptr;
+            if ((rc = stream_slot(*d, stream, bv::small_scratch_bytes(B, gamma, plan), &slot)) != BV_OK) return rc;
+            slot->clean = 0;                // (the area the flow kernel expects to find zero is written here)
+            bv::SmallScratch sc;
+            // the barrier words share the 256-byte block of the status word: zero since it was allocated
+            bv::small_scratch_layout(static_cast<char*>(slot->ws) + 256, reinterpret_cast<unsigned*>(static_cast<char*>(slot->ws) + 128),
+                                     B, gamma, plan, &sc);
+            prm.ticket = nullptr;
+            prm.nclusters = 0;
+            prm.status = static_cast<int*>(slot->ws);
+            cudaError_t e = bv::launch_small(prm, sc, dtype, nc, stream);
+            if (e != cudaSuccess) return cuda_fail(e);
+            t_last_launches = 1;
+            return BV_OK;
+        }
+    }
 
     // 16-byte rows: the flow of independent work items (both algorithms)
     if (flow_ok) {
@@ -485,6 +522,7 @@ int bv_set_option(const char* name, int value) {
     std::call_once(g_opt_once, load_env_options);
     std::lock_guard<std::mutex> lock(g_mu);
     if (!std::strcmp(name, "kernel")) g_opt.kernel = value;
+    else if (!std::strcmp(name, "small_bytes")) g_opt.small_bytes = value;
     else if (!std::strcmp(name, "cluster")) g_opt.cluster = value;
     else if (!std::strcmp(name, "max_clusters")) g_opt.max_clusters = value;
     else if (!std::strcmp(name, "flow_chunks")) g_opt.flow_chunks = value;

@@ -94,5 +94,21 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
 int flow_max_ctas_per_sm(int dtype);
 cudaError_t launch_flow(const Params& prm, const FlowScratch& fl, int dtype, int nctas, cudaStream_t stream);
 
+// Small-batch kernel (bv_small.cu): a cooperative launch of one CTA per SM with two grid-wide barriers.
+constexpr int kSmallMaxB = 32;        // sequences
+constexpr int kSmallMaxChunks = 32;   // chunks per row in its first phase
+struct SmallScratch {
+    unsigned* barrier;    // [0]: arrivals at the grid barriers, [16]: CTAs that have left; both zero between launches
+    double2* part;        // [B (2 gamma + 1)][nch] {reference, sum} of every chunk
+    double* seg;          // [B (gamma + 1)][np * 16] per-segment sums of the residual terms
+    int nch, np;
+};
+struct SmallPlan { int nch, np; };
+bool small_fits(int B, int gamma);
+SmallPlan small_plan(long long units, int B, int gamma, int nctas);
+size_t small_scratch_bytes(int B, int gamma, const SmallPlan& pl);
+void small_scratch_layout(void* base, unsigned* barrier, int B, int gamma, const SmallPlan& pl, SmallScratch* sc);
+int small_max_ctas(int dtype, int sm_count);
+cudaError_t launch_small(const Params& prm, const SmallScratch& sc, int dtype, int nctas, cudaStream_t stream);
 
 }  // namespace bv

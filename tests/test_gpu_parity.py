@@ -13,7 +13,7 @@ from parity import run_oracle, run_cuda, compare, assert_parity, record
 pytestmark = pytest.mark.gpu
 
 ALGOS = [oracle.BLOCK_VERIFY, oracle.TOKEN_VERIFY]
-KERNELS = {"flow": 1, "cluster": 2, "stream": 3}     # values of the library's "kernel" option
+KERNELS = {"flow": 1, "cluster": 2, "stream": 3, "small": 4}     # values of the library's "kernel" option
 
 
 def parity_case(inp, algo, check_diag=True):
@@ -71,17 +71,19 @@ def test_every_cluster_width(cluster, algo, bv_options):
     parity_case(random_inputs(7, 3, 5000, "f32", seed=cluster + 10), algo)
 
 
-@pytest.mark.parametrize("kernel", ["flow", "cluster", "stream"])
-def test_every_block_verification_kernel(kernel, bv_options):
-    # the library has several kernels for Algorithm 2; each must match the oracle
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("kernel", ["flow", "cluster", "stream", "small"])
+def test_every_kernel(kernel, algo, bv_options):
+    # the library has several kernels for each algorithm; each must match the oracle
     bv_options("kernel", KERNELS[kernel])
-    parity_case(random_inputs(40, 5, 24000, "bf16", seed=77, T=0.8), oracle.BLOCK_VERIFY)
-    parity_case(random_inputs(9, 3, 4096, "f32", seed=78), oracle.BLOCK_VERIFY)
-    parity_case(wl.make_inputs(wl.scaled(wl.CONFIGS["c4"], B=6), "cuda"), oracle.BLOCK_VERIFY)
+    parity_case(random_inputs(32 if kernel == "small" else 40, 5, 24000, "bf16", seed=77, T=0.8), algo)
+    parity_case(random_inputs(9, 3, 4096, "f32", seed=78), algo)
+    parity_case(wl.make_inputs(wl.scaled(wl.CONFIGS["c4"], B=6), "cuda"), algo)
 
 
 @pytest.mark.parametrize("chunks", [1, 3, 8])
 def test_flow_chunk_counts(chunks, bv_options):
+    bv_options("kernel", KERNELS["flow"])
     bv_options("flow_chunks", chunks)
     parity_case(random_inputs(21, 4, 16384, "bf16", seed=chunks), oracle.BLOCK_VERIFY)
     bv_options("flow_ctas", 3)     # far fewer CTAs than items
@@ -93,16 +95,32 @@ def test_more_sequences_than_resident_clusters(algo):
     parity_case(random_inputs(700, 3, 512, "f32", seed=3), algo)
 
 
+@pytest.mark.parametrize("kernel", ["flow", "small"])
 @pytest.mark.parametrize("algo", ALGOS)
 @pytest.mark.parametrize("gamma", [1, 16, 64])
-def test_block_lengths(gamma, algo):
+def test_block_lengths(gamma, algo, kernel, bv_options):
+    bv_options("kernel", KERNELS[kernel])
     parity_case(random_inputs(6, gamma, 2048, "bf16", seed=gamma, sigma_d=0.3), algo)
 
 
+@pytest.mark.parametrize("kernel", ["flow", "small"])
 @pytest.mark.parametrize("T", [0.2, 0.6, 1.0, 2.5])
-def test_temperatures(T):
+def test_temperatures(T, kernel, bv_options):
+    bv_options("kernel", KERNELS[kernel])
     for algo in ALGOS:
         parity_case(random_inputs(12, 4, 8192, "f32", seed=5, T=T), algo)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("B,gamma,V,dtype", [(1, 8, 152064, "bf16"), (16, 8, 152064, "bf16"), (2, 2, 1024, "f32"),
+                                             (32, 15, 4096, "bf16"), (5, 33, 640, "f32"), (3, 1, 8, "bf16"), (8, 60, 2048, "bf16")])
+def test_small_batch_kernel(B, gamma, V, dtype, algo, bv_options):
+    # the kernel of the latency regime, forced for every shape it admits (chunks and pieces of every count)
+    bv_options("kernel", KERNELS["small"])
+    parity_case(random_inputs(B, gamma, V, dtype, seed=B + gamma, T=0.9, sigma_d=0.4), algo)
+    bv_options("kernel", 0)
+    bv_options("small_bytes", 1)       # ... and the default choice with the small-batch kernel all but switched off
+    parity_case(random_inputs(B, gamma, V, dtype, seed=B + gamma + 1, T=0.9, sigma_d=0.4), algo)
 
 
 def test_gamma1_block_equals_token_bitwise():
@@ -112,7 +130,9 @@ def test_gamma1_block_equals_token_bitwise():
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
 
 
-def test_draft_equals_target():
+@pytest.mark.parametrize("kernel", ["flow", "small"])
+def test_draft_equals_target(kernel, bv_options):
+    bv_options("kernel", KERNELS[kernel])
     inp = random_inputs(16, 6, 4096, "bf16", seed=22)
     inp["draft_logits"] = inp["target_logits"][:, :6].clone()
     for algo in ALGOS:
@@ -124,7 +144,9 @@ def test_draft_equals_target():
     assert torch.all(diag["S"] == 0) and torch.all(diag["p"] == 1)
 
 
-def test_masked_logits_and_domain_errors():
+@pytest.mark.parametrize("kernel", ["flow", "small"])
+def test_masked_logits_and_domain_errors(kernel, bv_options):
+    bv_options("kernel", KERNELS[kernel])
     inp = random_inputs(8, 3, 640, "f32", seed=23)
     t, d, tok = inp["target_logits"], inp["draft_logits"], inp["draft_tokens"]
     # top-k style masking: legal

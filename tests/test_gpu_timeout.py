@@ -21,8 +21,10 @@ def _tiny(seed):
     return wl.make_inputs(wl.Workload("to", 3, 2, 4096, "bf16", 1.0, seed, 2.0, 0.0, 0, 0.0, 1.0), "cpu")
 
 
-def test_wait_that_runs_out_is_reported_and_the_next_call_works(bv_options):
+@pytest.mark.parametrize("kernel", [1, 4])      # the flow kernel; the small-batch kernel (a CTA stays away from its grid barrier)
+def test_wait_that_runs_out_is_reported_and_the_next_call_works(kernel, bv_options):
     inp = _tiny(5)
+    bv_options("kernel", kernel)
     pinned = {k: (v.pin_memory() if torch.is_tensor(v) else v) for k, v in inp.items()}
     dev = {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in inp.items()}
     args = lambda d: (d["target_logits"], d["draft_logits"], d["draft_tokens"], d["uniforms"], d["temperature"])
