@@ -16,8 +16,15 @@ import pytest
 import oracle
 import test_oracle_c as pins
 import test_oracle_greedy as gpins
+import test_oracle_probs as ppins
 
 SRC = open(os.path.join(os.path.dirname(oracle.__file__), "verify_oracle.c")).read()
+# the procedures on given probabilities follow the ones on logits in the file and repeat some of
+# their lines: a mutation is planted in one part only
+PROBS_MARK = "/* ================= the same procedures on given probabilities"
+assert SRC.count(PROBS_MARK) == 1
+HEAD, TAIL = SRC.split(PROBS_MARK)
+TAIL = PROBS_MARK + TAIL
 
 # (name, text in the oracle, what replaces it)
 MUTATIONS = [
@@ -108,7 +115,7 @@ def _find_selection_mutations():
     """Mutations of the parts of the file not quoted above are located by search, so that the
     test fails loudly (rather than silently testing nothing) if the oracle's text changes."""
     extra = []
-    if "acc += weight_at(s->tgt, s->toff + (size_t)i * V, lse_t[i]," in SRC:
+    if "acc += weight_at(s->tgt, s->toff + (size_t)i * V, lse_t[i]," in HEAD:
         extra.append(("S_i from the rows of position i+1",
                       "acc += weight_at(s->tgt, s->toff + (size_t)i * V, lse_t[i],\n"
                       "                             s->drf, s->doff + (size_t)i * V, lse_d[i], 1,",
@@ -135,6 +142,8 @@ def _compile(text, tmp_path, tag):
                                       vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.oracle_sample_rows.restype = ctypes.c_int
     lib.oracle_sample_rows.argtypes = [vp, vp, ip, ip, ip, ctypes.c_double, vp, vp, vp]
+    lib.oracle_verify_probs.restype = ctypes.c_int
+    lib.oracle_verify_probs.argtypes = [ip, vp, vp, vp, vp, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp]
     lib.oracle_threads.restype = ctypes.c_int
     return lib
 
@@ -171,8 +180,19 @@ def _pins():
     yield lambda: gpins.test_c_oracle_sample_follows_the_residual_with_the_unclipped_product()
 
 
-def _caught():
-    for pin in _pins():
+def _probs_pins():
+    """The pins of the procedures on given probabilities."""
+    yield lambda: ppins.test_worked_example_accepted_lengths()
+    yield lambda: ppins.test_intermediates_equal_the_exact_rationals(3, 2, 0)
+    yield lambda: ppins.test_intermediates_equal_the_exact_rationals(4, 3, 1)
+    yield lambda: ppins.test_sampled_token_follows_the_explicit_cumulative_sums("block")
+    yield lambda: ppins.test_sampled_token_follows_the_explicit_cumulative_sums("token")
+    yield lambda: ppins.test_output_law_is_the_target_law("block")
+    yield lambda: ppins.test_agrees_with_the_logit_procedures_on_log_probabilities("token")
+
+
+def _caught(pin_set=_pins):
+    for pin in pin_set():
         try:
             pin()
         except AssertionError:
@@ -183,11 +203,40 @@ def _caught():
 def test_the_pins_pass_on_the_real_oracle_compiled_the_same_way(tmp_path):
     with _installed(_compile(SRC, tmp_path, "clean")):
         assert not _caught()
+        assert not _caught(_probs_pins)
 
 
 @pytest.mark.parametrize("idx", range(len(MUTATIONS)))
 def test_a_planted_mistake_is_caught(idx, tmp_path):
     name, old, new = MUTATIONS[idx]
-    assert SRC.count(old) == 1, "the oracle's text changed: update the mutation '%s'" % name
-    with _installed(_compile(SRC.replace(old, new), tmp_path, "m%d" % idx)):
+    assert HEAD.count(old) == 1, "the oracle's text changed: update the mutation '%s'" % name
+    with _installed(_compile(HEAD.replace(old, new) + TAIL, tmp_path, "m%d" % idx)):
         assert _caught(), "no pin noticed: " + name
+
+
+# the same kinds of mistake in the procedures on given probabilities
+PROBS_MUTATIONS = [
+    ("ratio upside down", "*ratio = P / Q;", "*ratio = Q / P;"),
+    ("ratio from the row of position i", "double P = stored_prob(s, 1, i - 1, x), Q = stored_prob(s, 0, i - 1, x);",
+     "double P = stored_prob(s, 1, i < s->gamma ? i : i - 1, x), Q = stored_prob(s, 0, i < s->gamma ? i : i - 1, x);"),
+    ("p_i not clipped at 1", "p[i] = v < 1.0 ? v : 1.0;", "p[i] = v;"),
+    ("p_i forgets p_{i-1}", "double v = p[i - 1] * ratio;", "double v = ratio;"),
+    ("h_i without the 1 - p_i term", "h[i] = S[i] > 0.0 ? S[i] / (S[i] + 1.0 - p[i]) : 0.0;",
+     "h[i] = S[i] > 0.0 ? S[i] / (S[i] + 1.0) : 0.0;"),
+    ("residual with the two models swapped", "double w = p * P - stored_prob(s, 0, i, x);",
+     "double w = stored_prob(s, 0, i, x) - p * P;"),
+    ("residual forgets p_i", "double w = p * P - stored_prob(s, 0, i, x);", "double w = P - stored_prob(s, 0, i, x);"),
+    ("token verification keeps going after a rejection", "            tau = i;\n        else\n            break;",
+     "            tau = i;\n        else\n            continue;"),
+    ("token verification without the min with 1", "double h = ratio < 1.0 ? ratio : 1.0;", "double h = ratio;"),
+    ("block verification samples with p of the wrong position", "int Y = sample_probs(s, tau, p[tau],",
+     "int Y = sample_probs(s, tau, p[tau > 0 ? tau - 1 : tau],"),
+]
+
+
+@pytest.mark.parametrize("idx", range(len(PROBS_MUTATIONS)))
+def test_a_planted_mistake_in_the_probability_procedures_is_caught(idx, tmp_path):
+    name, old, new = PROBS_MUTATIONS[idx]
+    assert TAIL.count(old) == 1, "the oracle's text changed: update the mutation '%s'" % name
+    with _installed(_compile(HEAD + TAIL.replace(old, new), tmp_path, "p%d" % idx)):
+        assert _caught(_probs_pins), "no pin noticed: " + name
