@@ -299,6 +299,7 @@ def main():
         out = fn(*a)
         evs[i][1].record()
         launches += 1 if args.algo == "sample" else bv.bv_last_launch_count()
+    args.kernel_code = bv.bv_last_kernel()
     stop.record()
     barrier()
     torch.cuda.profiler.stop()
@@ -403,6 +404,9 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
     else:
         algo_bytes = token_bytes(w, out[1])
         kernel = "verify_flow_kernel"
+    if args.algo != "sample":      # (the library says which of its verification kernels the shape got)
+        kernel = {1: "verify_flow_kernel", 2: "verify_cluster_kernel", 3: "verify_stream_kernel",
+                  4: "verify_small_kernel"}.get(getattr(args, "kernel_code", 0), kernel)
     achieved = algo_bytes / (k_ms * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -449,6 +453,13 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
 # ncu capture of this command at full size that profiles/ summarises; None for a workload or
 # kernel with no capture.
 TRAFFIC_BYTES = {
+    ("c4", "block", "verify_flow_kernel"): 2568772352,
+    ("c4", "token", "verify_flow_kernel"): 825143808,
+    ("c4", "greedy", "verify_flow_kernel"): 2579974656,
+    ("c4", "block_lse", "verify_flow_kernel"): 1521103360,
+    ("c4", "sample", "sample_rows_kernel"): 1055976192,
+    ("c4", "block_probs", "verify_flow_kernel"): 350806016,
+    ("c4", "token_probs", "verify_flow_kernel"): 264784384,
 }
 
 

@@ -305,6 +305,9 @@ int bv_release(void);
 
 /* Number of kernel launches the last device-path call on this thread enqueued. */
 int bv_last_launch_count(void);
+/* Which kernel the last bv_verify / tv_verify (or _ex, _lse, _probs, gbv_, _host) call on this thread launched, in the
+ * codes of the "kernel" option: 1 flow, 2 cluster, 3 element-wise streaming, 4 small-batch; 0 if it launched none. */
+int bv_last_kernel(void);
 /* cudaError_t value of the last failing runtime call on this thread (0 if none). */
 int bv_last_cuda_error(void);
 /* Static description of a bv_status value. */

@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_verify_probs", "tv_verify_probs", "bv_sample_draft", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_verify_probs", "tv_verify_probs", "bv_sample_draft", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_kernel", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -80,6 +80,12 @@ def bv_version() -> int:
 
 def bv_last_launch_count() -> int:
     return int(load_library().bv_last_launch_count())
+
+
+def bv_last_kernel() -> int:
+    """Code of the kernel the last verification call on this thread launched (1 flow, 2 cluster,
+    3 element-wise streaming, 4 small-batch)."""
+    return int(load_library().bv_last_kernel())
 
 
 def bv_release() -> None:

@@ -91,6 +91,7 @@ DeviceState g_dev[kMaxDevices];
 std::mutex g_mu;
 
 thread_local int t_last_launches = 0;
+thread_local int t_last_kernel = 0;     // which kernel the last verification call on this thread launched (the "kernel" option's codes)
 thread_local int t_last_cuda_error = 0;
 
 int cuda_fail(cudaError_t e) { return bv::note_cuda_error(e); }
@@ -176,6 +177,7 @@ struct Extra {              // what only some entry points pass
 int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B,
                int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, const Extra& ex, cudaStream_t stream) {
     t_last_launches = 0;
+    t_last_kernel = 0;
     int rc = bv::check_verify_args(tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol);
     if (rc != BV_OK) return rc;
     if (B == 0) return BV_OK;
@@ -234,7 +236,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             prm.status = static_cast<int*>(slot->ws);
             cudaError_t e = bv::launch_small(prm, sc, dtype, nc, stream);
             if (e != cudaSuccess) return cuda_fail(e);
-            t_last_launches = 1;
+            t_last_launches = 1; t_last_kernel = 4;
             return BV_OK;
         }
     }
@@ -279,7 +281,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             prm.status = static_cast<int*>(slot->ws);
             e = bv::launch_flow(prm, fl, dtype, static_cast<int>(nctas), stream);
             if (e != cudaSuccess) return cuda_fail(e);
-            t_last_launches = 1;
+            t_last_launches = 1; t_last_kernel = 1;
             return BV_OK;
         }
     }
@@ -304,7 +306,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             prm.nclusters = n;
             cudaError_t e = bv::launch_cluster(prm, algo, dtype, cluster, n, stream);
             if (e != cudaSuccess) return cuda_fail(e);
-            t_last_launches = 1;
+            t_last_launches = 1; t_last_kernel = 2;
             return BV_OK;
         }
     }
@@ -321,7 +323,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
 
     cudaError_t e = bv::launch_stream(prm, algo, dtype, vec, cluster, nclusters, stream);
     if (e != cudaSuccess) return cuda_fail(e);
-    t_last_launches = 1;
+    t_last_launches = 1; t_last_kernel = 3;
     return BV_OK;
 }
 
@@ -553,6 +555,7 @@ int bv_release(void) {
 }
 
 int bv_last_launch_count(void) { return t_last_launches; }
+int bv_last_kernel(void) { return t_last_kernel; }
 int bv_last_cuda_error(void) { return t_last_cuda_error; }
 
 const char* bv_status_string(int status) {
