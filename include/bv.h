@@ -60,7 +60,7 @@ typedef enum bv_status {
 
 enum { BV_DTYPE_F32 = 0, BV_DTYPE_BF16 = 1 };
 enum { BV_MAX_GAMMA = 64 };
-enum { BV_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024 };
+enum { BV_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024 };
 
 /*
  * Block Verification: Algorithm 2 with Eq. "def_as" (p_0 = 1,
@@ -147,17 +147,18 @@ int tv_verify_host(const void* target_logits, const void* draft_logits,
  * memory pool owns the whole device, code that may run under stream capture, processes
  * with allocator hooks.  Same arguments, outputs and arithmetic as bv_verify(), DEVICE
  * pointers, asynchronous on `stream`; it never calls cudaMalloc, cudaFree or any routine
- * that allocates.  Its scratch is a fixed array of BV_NOALLOC_SCRATCH_BYTES (4 MiB) inside
+ * that allocates.  Its scratch is a fixed array of BV_NOALLOC_SCRATCH_BYTES (8 MiB) inside
  * the library image, present on every GPU that loads the library until the process exits.
  *
  * Limits and rules that bv_verify() does not have:
- *   - the scratch needed grows with B (gamma+1), about 0.7 KB per logit row pair at large V
- *     (B = 256, gamma = 8, V = 256000 needs 1.5 MiB); a problem that needs more than the
+ *   - the scratch needed grows with B (gamma+1), about 2.1 KB per logit row pair at large V
+ *     (B = 256, gamma = 8, V = 256000 needs 5.0 MB); a problem that needs more than the
  *     array returns BV_ERR_TOO_LARGE and launches nothing;
  *   - rows must be whole 16-byte vectors on 16-byte aligned bases (V a multiple of 8 for
  *     bf16, of 4 for fp32), else BV_ERR_UNSUPPORTED;
- *   - the first call on each device looks the array's device address up and queries the
- *     device; make that first call before any stream capture begins;
+ *   - the first call on each device and for each dtype looks the array's device address up
+ *     and queries the device and the kernel's occupancy; make those calls before any stream
+ *     capture begins;
  *   - every call on a device uses the same array, which keeps the previous call's contents
  *     (the entry point clears the part that must start at zero, on `stream`).  Two calls
  *     that overlap on the GPU, on different streams, race on it: order them yourself;

@@ -247,7 +247,7 @@ def bv_verify_noalloc(target_logits, draft_logits, draft_tokens, uniforms, out_t
     (a memory pool that owns the device, possible stream capture, allocator hooks).  The
     caller supplies the outputs: ``out_tokens`` int32 [B, gamma+1] and ``out_len`` int32 [B],
     CUDA tensors; this wrapper creates no tensor either.  Raises BVError(status -5) when the
-    problem needs more than the library's fixed 4 MiB scratch array.
+    problem needs more than the library's fixed 8 MiB scratch array.
     """
     lib = load_library()
     B, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms, True)

@@ -3,7 +3,7 @@
 bv_verify_noalloc() is for programs that embed this library where a device allocation at
 call time is not allowed: an inference server whose memory pool owns the whole GPU, code
 that may be recording a stream capture, a process with allocator hooks.  It keeps its
-scratch in a fixed 4 MiB array inside the library, shared by all calls, which holds
+scratch in a fixed 8 MiB array inside the library, shared by all calls, which holds
 whatever the previous call left there.  So the test calls it twice in a row on different
 inputs: a second call that trips over stale counters, or a first call that only works on
 fresh memory, shows up as a difference from bv_verify().
@@ -84,3 +84,17 @@ def test_problem_beyond_the_fixed_scratch_is_refused():
                                inp["uniforms"].data_ptr(), 2, 2, 1022, 0, ctypes.c_float(1.0),
                                ot.data_ptr(), ol.data_ptr(), None)
     assert rc == -2
+
+
+def test_the_largest_benchmark_workload_fits():
+    # B = 256, gamma = 8, V = 256000 needs 5 MB of the 8 MiB array
+    lib = bv.load_library()
+    inp = wl.make_inputs(wl.CONFIGS["c4"], "cuda")
+    B, g1, _ = inp["target_logits"].shape
+    ot = torch.full((B, g1), -7, dtype=torch.int32, device="cuda")
+    ol = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    assert _call_noalloc(lib, inp, ot, ol) == 0
+    want_tokens, want_len = bv.bv_verify(inp["target_logits"], inp["draft_logits"], inp["draft_tokens"],
+                                         inp["uniforms"], inp["temperature"])
+    torch.cuda.synchronize()
+    assert torch.equal(ol, want_len) and torch.equal(ot, want_tokens)
