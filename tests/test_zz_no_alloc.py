@@ -40,7 +40,16 @@ def _call_noalloc(lib, inp, out_tokens, out_len):
                                  torch.cuda.current_stream().cuda_stream)
 
 
-def test_two_calls_in_a_row_match_the_allocating_entry_point():
+def _flow_kernel_with_default_shapes(bv_options):
+    # the entry point without allocations always runs the flow kernel with the work-item shape chosen by
+    # problem size: the call it is compared with must do the same, whatever the environment set
+    bv_options("kernel", 1)
+    for name in ("flow_chunks", "flow_pieces", "flow_ctas", "flow_depth", "flow_keep_l2"):
+        bv_options(name, 0)
+
+
+def test_two_calls_in_a_row_match_the_allocating_entry_point(bv_options):
+    _flow_kernel_with_default_shapes(bv_options)
     lib = bv.load_library()
     # the second problem is smaller and of another dtype, so leftovers of the first would matter
     cases = [_inputs(48, 6, 32768, "bf16", seed=101), _inputs(19, 3, 8192, "f32", seed=102)]
@@ -86,8 +95,9 @@ def test_problem_beyond_the_fixed_scratch_is_refused():
     assert rc == -2
 
 
-def test_the_largest_benchmark_workload_fits():
+def test_the_largest_benchmark_workload_fits(bv_options):
     # B = 256, gamma = 8, V = 256000 needs 5 MB of the 8 MiB array
+    _flow_kernel_with_default_shapes(bv_options)
     lib = bv.load_library()
     inp = wl.make_inputs(wl.CONFIGS["c4"], "cuda")
     B, g1, _ = inp["target_logits"].shape
