@@ -124,12 +124,11 @@ struct FlowCtx {
 
 // One warp walks segment [w0, w1) of a row pair in index order and returns the first element
 // whose running residual mass exceeds tw (else the last element with positive mass, else -1).
-template <int DT, bool PROBS = false>
+template <int DT, bool PROBS = false, int kAhead = 4>      // kAhead: runs of 32 vectors whose loads are in flight together
 __device__ int f_rescan(const char* rowP, const char* rowQ, int w0, int w1, int lane, float kf, float cp,
                         float nMP, float nMQ, double tw) {
     constexpr int EPV = Raw<DT>::EPV;
     constexpr uint32_t kPad = PROBS ? 0u : Raw<DT>::kNegInf;   // an element beyond the segment weighs nothing
-    constexpr int kAhead = 4;                                // runs of 32 vectors whose loads are in flight together
     // The terms are the fp32 values of the sweeps; their running sum, which decides the token, is
     // kept in fp64 (a cell of the distribution can be far narrower than fp32 resolves next to the
     // mass before it).

@@ -20,12 +20,14 @@
 
 namespace bv {
 
-constexpr int kSmThreads = 512;
+constexpr int kSmThreads = 512;       // streaming threads; one more warp fetches the scalars while they stream
 constexpr int kSmWarps = kSmThreads / 32;
+constexpr int kSmAllThreads = kSmThreads + 32;
 constexpr int kSmMaxRows = 1056;      // rows B (2 gamma + 1) whose normalisers a CTA keeps in shared memory
 constexpr int kSmMaxPos = 560;        // positions B (gamma + 1)
 constexpr int kSmInFlight = 8;        // 16-byte loads a thread has in flight in the first phase
-constexpr int kSmPairsInFlight = 4;   // pairs of them in the second
+constexpr int kSmPairsInFlight = 5;   // pairs of them in the second
+constexpr int kSmMaxUni = kSmMaxPos + kSmallMaxB;   // uniforms B (gamma + 2)
 
 struct SmallShared {
     float rowM[kSmMaxRows];
@@ -41,6 +43,10 @@ struct SmallShared {
     float wM[kSmWarps];
     float wS[kSmWarps];
     double cS[kSmMaxPos];             // third phase: S_i of this CTA's sequence
+    // fetched by the extra warp during the first phase: the logits of the drafted tokens, the uniforms
+    float zp[kSmMaxPos], zq[kSmMaxPos];
+    unsigned char xok[kSmMaxPos];
+    float u[kSmMaxUni];
 };
 
 // the grid-wide barrier: arrivals are counted up through the launch; the wait is bounded
@@ -74,7 +80,7 @@ __device__ __forceinline__ const char* small_row(const Params& prm, size_t row_b
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Params prm, const SmallScratch sc) {
+__global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Params prm, const SmallScratch sc) {
     using R = Raw<DT>;
     constexpr int EPV = R::EPV;
     constexpr size_t ESZ = (DT == kF32) ? 4 : 2;
@@ -91,6 +97,19 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
 
     // ---------------- phase 1: {reference, sum 2^{z k - M}} of every chunk of every row ----------------
     const int nch = sc.nch;
+    if (warp == kSmWarps) {
+        // nothing here depends on the first phase: the two dependent round trips (token, then its two
+        // logits) and the uniforms are over before the streaming warps are
+        for (int i = lane; i < B * g; i += 32) {
+            const int b = i / g, c = i % g;
+            const int x = prm.tok[i];
+            const bool xok = x >= 0 && x < prm.V;
+            sh.xok[b * (g + 1) + c] = xok;
+            sh.zp[b * (g + 1) + c] = xok ? static_cast<float>(load_logit<DT>(small_row(prm, row_bytes, b, c), x)) : 0.f;
+            sh.zq[b * (g + 1) + c] = xok ? static_cast<float>(load_logit<DT>(small_row(prm, row_bytes, b, g + 1 + c), x)) : 0.f;
+        }
+        for (int i = lane; i < B * (g + 2); i += 32) sh.u[i] = prm.uni[i];
+    }
     for (int item = blockIdx.x; item < nrows * nch; item += gridDim.x) {
         const int rid = item / nch, ch = item % nch;
         const char* row = small_row(prm, row_bytes, rid / rpb, rid % rpb);
@@ -98,7 +117,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
         small_seg_range(units, nch, ch, u0, u1);
         float M = kNoRef, s = 0.f;
         const uint4 ninf = make_uint4(R::kNegInf, R::kNegInf, R::kNegInf, R::kNegInf);
-        for (int base = u0; base < u1; base += kSmThreads * kSmInFlight) {
+        for (int base = u0; warp < kSmWarps && base < u1; base += kSmThreads * kSmInFlight) {
             uint4 raw[kSmInFlight];
 #pragma unroll
             for (int j = 0; j < kSmInFlight; ++j) {
@@ -115,7 +134,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
             }
         }
         s = warp_sum(s);
-        if (lane == 0) { sh.wM[warp] = M; sh.wS[warp] = s; }
+        if (lane == 0 && warp < kSmWarps) { sh.wM[warp] = M; sh.wS[warp] = s; }
         __syncthreads();
         if (warp == 0) {
             const float m = lane < kSmWarps ? sh.wM[lane] : kNoRef;
@@ -130,7 +149,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
 
     // ---------------- phase 2a: normalisers of every row, the scalar part of every sequence ----------------
     if (alive) {
-        for (int rid = tid; rid < nrows; rid += kSmThreads) {
+        for (int rid = tid; rid < nrows; rid += kSmAllThreads) {
             float M = kNoRef;
             double z[kSmallMaxChunks];
             float m[kSmallMaxChunks];
@@ -148,7 +167,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
     }
     __syncthreads();
     if (alive) {
-        for (int b = warp; b < B; b += kSmWarps) {
+        for (int b = warp; warp < kSmWarps && b < B; b += kSmWarps) {
             // lanes c and c + 32 speak for rows / positions c and c + 32
             double rat[2] = {1.0, 1.0};
             bool badrow[2] = {false, false};
@@ -159,20 +178,15 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
                 if (c < g) {
                     const float MP = sh.rowM[b * rpb + c], MQ = sh.rowM[b * rpb + g + 1 + c];
                     const double ZP = sh.rowZ[b * rpb + c], ZQ = sh.rowZ[b * rpb + g + 1 + c];
-                    const int x = prm.tok[static_cast<size_t>(b) * g + c];
-                    const bool xok = x >= 0 && x < prm.V;
-                    double zp = 0.0, zq = 0.0;
-                    if (xok) {
-                        zp = load_logit<DT>(small_row(prm, row_bytes, b, c), x);
-                        zq = load_logit<DT>(small_row(prm, row_bytes, b, g + 1 + c), x);
-                    }
+                    const bool xok = sh.xok[b * (g + 1) + c] != 0;
+                    const double zp = sh.zp[b * (g + 1) + c], zq = sh.zq[b * (g + 1) + c];
                     bool bad = !(MP > kNoRef && MP < INFINITY) || !(ZP < static_cast<double>(INFINITY)) ||
                                !(MQ > kNoRef && MQ < INFINITY) || !(ZQ < static_cast<double>(INFINITY)) || !xok || zq == -INFINITY;
                     rat[h] = bad ? 0.0 : exp2((zp - zq) * prm.kd - (static_cast<double>(MP) - static_cast<double>(MQ))) * (ZQ / ZP);
                     badrow[h] = bad;
                     sh.ratio[b * (g + 1) + c] = rat[h];
                     // the uniform that decides about this lane's row / position
-                    eta[h] = tv ? prm.uni[static_cast<size_t>(b) * (g + 2) + c] : (c >= 1 ? prm.uni[static_cast<size_t>(b) * (g + 2) + c - 1] : 0.f);
+                    eta[h] = tv ? sh.u[b * (g + 2) + c] : (c >= 1 ? sh.u[b * (g + 2) + c - 1] : 0.f);
                 }
             }
             const float MPg = sh.rowM[b * rpb + g];
@@ -227,7 +241,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
                 }
                 m_lo = __ballot_sync(0xffffffffu, need[0]);
                 m_hi = __ballot_sync(0xffffffffu, need[1]);
-                const float eta_g = prm.uni[static_cast<size_t>(b) * (g + 2) + g - 1];
+                const float eta_g = sh.u[b * (g + 2) + g - 1];
                 lastw = all_positions || static_cast<double>(eta_g) <= p_g * (1.0 + 1e-6);
                 bad = (bad_lo | bad_hi) != 0u || bad_last;
                 if (lane == 0) sh.pch[b * (g + 1) + g] = p_g;
@@ -270,9 +284,9 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
             const float cp = sh.csc[b * (g + 1) + i];
             const float nMP = -sh.rowM[b * rpb + i], nMQ = have_q ? -sh.rowM[b * rpb + g + 1 + i] : 0.f;
             int s0, s1;
-            small_seg_range(units, nseg, piece * kSmWarps + warp, s0, s1);
+            small_seg_range(units, nseg, piece * kSmWarps + (warp < kSmWarps ? warp : 0), s0, s1);
             double acc = 0.0;
-            for (int base = s0; base < s1; base += 32 * kSmPairsInFlight) {
+            for (int base = s0; warp < kSmWarps && base < s1; base += 32 * kSmPairsInFlight) {
                 uint4 rp[kSmPairsInFlight], rq[kSmPairsInFlight];
                 const uint4 ninf = make_uint4(R::kNegInf, R::kNegInf, R::kNegInf, R::kNegInf);
 #pragma unroll
@@ -291,7 +305,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
                 }
             }
             acc = warp_sum_d(acc);
-            if (lane == 0) sc.seg[(static_cast<size_t>(b) * (g + 1) + i) * nseg + piece * kSmWarps + warp] = acc;
+            if (lane == 0 && warp < kSmWarps) sc.seg[(static_cast<size_t>(b) * (g + 1) + i) * nseg + piece * kSmWarps + warp] = acc;
         }
     }
     if (alive) alive = small_grid_barrier(sc.barrier, 2u * gridDim.x, prm.status, limit, false);
@@ -300,7 +314,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
     for (int b = blockIdx.x; alive && b < B; b += gridDim.x) {
         // S_i of every candidate (a warp per position at a time)
         const unsigned m_lo = sh.mask_lo[b], m_hi = sh.mask_hi[b];
-        for (int i = warp; i < g; i += kSmWarps) {
+        for (int i = warp; i < g; i += kSmAllThreads / 32) {
             const bool cand = (i < 32 ? m_lo >> i : m_hi >> (i - 32)) & 1u;
             double tot = 0.0;
             if (cand) {
@@ -312,7 +326,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
         }
         __syncthreads();
         if (warp == 0) {
-            const float* u = prm.uni + static_cast<size_t>(b) * (g + 2);
+            const float* u = sh.u + b * (g + 2);
             int tau;
             if (tv) {
                 tau = sh.tv_tau[b];
@@ -372,7 +386,7 @@ __global__ void __launch_bounds__(kSmThreads, 1) verify_small_kernel(const Param
                 const double before = shfl_d(bef, src);
                 int s0, s1;
                 small_seg_range(units, nseg, sel, s0, s1);
-                found = f_rescan<DT>(small_row(prm, row_bytes, b, tau), have_q ? small_row(prm, row_bytes, b, g + 1 + tau) : nullptr,
+                found = f_rescan<DT, false, 5>(small_row(prm, row_bytes, b, tau), have_q ? small_row(prm, row_bytes, b, g + 1 + tau) : nullptr,
                                      s0, s1, lane, kf, sh.csc[b * (g + 1) + tau], -sh.rowM[b * rpb + tau],
                                      have_q ? -sh.rowM[b * rpb + g + 1 + tau] : 0.f, t - before);
             }
@@ -473,7 +487,7 @@ static SKernelFn pick_small(int dtype) { return dtype == kF32 ? verify_small_ker
 
 int small_max_ctas(int dtype, int sm_count) {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_small(dtype), kSmThreads, 0) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_small(dtype), kSmAllThreads, 0) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -484,7 +498,7 @@ cudaError_t launch_small(const Params& prm, const SmallScratch& sc, int dtype, i
     Params p = prm;
     SmallScratch s = sc;
     void* args[] = {&p, &s};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_small(dtype)), dim3(nctas), dim3(kSmThreads), args, 0, stream);
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_small(dtype)), dim3(nctas), dim3(kSmAllThreads), args, 0, stream);
 }
 
 }  // namespace bv
