@@ -126,9 +126,10 @@ def test_block_verification_generates_more_per_iteration():
     assert be["block"] > be["token"] and be["block_lse"] > be["token"]
 
 
-@pytest.mark.parametrize("algo", ["block_lse", "token"])
-def test_graph_replay_generates_the_same_tokens(algo):
-    V, B, N, gamma = 4096, 48, 9, 5
+@pytest.mark.parametrize("B", [48, 12])        # the flow kernel; the small-batch kernel (a cooperative launch) for block / token
+@pytest.mark.parametrize("algo", ["block_lse", "block", "token"])
+def test_graph_replay_generates_the_same_tokens(algo, B):
+    V, N, gamma = 4096, 9, 5
     tt, dt = wl.markov_models(V, "bf16", 41, 2.0, 1.0, 1.1, "cuda")
     ud, uv = wl.loop_uniforms(N, B, gamma, 42, "cuda")
     first = torch.arange(B, dtype=torch.int32, device="cuda")
