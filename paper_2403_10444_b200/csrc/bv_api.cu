@@ -215,7 +215,7 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
     // grid-wide barriers instead of queues takes half the time of the flow kernel or less.
     const long long logit_bytes = static_cast<long long>(B) * (2 * gamma + 1) * static_cast<long long>(row_bytes);
     const long long small_limit = opt.small_bytes > 0 ? static_cast<long long>(opt.small_bytes) << 20 : kSmallBytes[algo == bv::kBlockVerify ? 1 : 0];
-    if (vec && !prm.lse_d && !prm.greedy && !prm.probs && bv::small_fits(B, gamma) &&
+    if (vec && !prm.probs && bv::small_fits(B, gamma) &&
         (opt.kernel == 4 || (opt.kernel == 0 && logit_bytes <= small_limit))) {
         int& nc = d->small_ctas[dtype];
         if (nc == 0) {

@@ -1,5 +1,6 @@
-// Block Verification (Algorithm 2) and Token Verification (Algorithm 1) for batches so small that
-// a launch is a matter of latency, not of bandwidth (a few sequences: the whole input fits in L2).
+// Block Verification (Algorithm 2, also with supplied draft normalisers), Greedy Block Verification
+// (Algorithm 4) and Token Verification (Algorithm 1) for batches so small that a launch is a matter
+// of latency, not of bandwidth (a few sequences: the whole input fits in L2).
 //
 // The flow kernel hands work from CTA to CTA through queues and counters in global memory, and a
 // sequence goes through a dozen such hand-overs of a microsecond or more each.  Here all CTAs of a
@@ -112,6 +113,7 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
     }
     for (int item = blockIdx.x; item < nrows * nch; item += gridDim.x) {
         const int rid = item / nch, ch = item % nch;
+        if (prm.lse_d != nullptr && rid % rpb > g) continue;      // (a draft row whose normaliser is supplied: nothing to learn)
         const char* row = small_row(prm, row_bytes, rid / rpb, rid % rpb);
         int u0, u1;
         small_seg_range(units, nch, ch, u0, u1);
@@ -150,6 +152,15 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
     // ---------------- phase 2a: normalisers of every row, the scalar part of every sequence ----------------
     if (alive) {
         for (int rid = tid; rid < nrows; rid += kSmAllThreads) {
+            if (prm.lse_d != nullptr && rid % rpb > g) {
+                // the supplied normaliser as an integer reference at or above every scaled logit of the row
+                // plus a sum in [2^-1/2, 2^1/2]; a value that is not finite leaves the row without a reference
+                const double L2 = static_cast<double>(prm.lse_d[static_cast<size_t>(rid / rpb) * g + (rid % rpb - g - 1)]) * 1.4426950408889634073599246810019;
+                const bool fin = L2 > -1e300 && L2 < 1e300;
+                sh.rowM[rid] = fin ? static_cast<float>(rint(L2)) : kNoRef;
+                sh.rowZ[rid] = fin ? exp2(L2 - rint(L2)) : 0.0;
+                continue;
+            }
             float M = kNoRef;
             double z[kSmallMaxChunks];
             float m[kSmallMaxChunks];
