@@ -285,7 +285,8 @@ int bv_stream_status(void* stream);
  * Tuning and test options, process-wide, read by every later call (0 restores the default choice):
  *   "kernel"        1 flow, 2 cluster, 3 element-wise streaming kernel, 4 small-batch kernel (for the shapes
  *                   each admits; the default picks the small-batch kernel for up to 32 sequences whose
- *                   logits are few enough to make the launch a matter of latency, else the flow kernel)
+ *                   logits are few enough to make the launch a matter of latency - up to 16 sequences for
+ *                   the entry points on probabilities -, else the flow kernel)
  *   "small_bytes"   logit megabytes up to which the small-batch kernel is the default
  *   "cluster"       cluster width of the cluster / streaming kernels (1, 2, 4, 8)
  *   "max_clusters"  cap on the clusters those kernels launch

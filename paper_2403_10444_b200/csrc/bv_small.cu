@@ -80,10 +80,12 @@ __device__ __forceinline__ const char* small_row(const Params& prm, size_t row_b
                   : static_cast<const char*>(prm.drf) + (static_cast<size_t>(b) * g + (j - g - 1)) * row_bytes;
 }
 
-template <int DT>
+// PROBS: the rows hold probabilities, used as stored: there is no first phase (and no first barrier).
+template <int DT, bool PROBS>
 __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Params prm, const SmallScratch sc) {
     using R = Raw<DT>;
     constexpr int EPV = R::EPV;
+    constexpr uint32_t kPad = PROBS ? 0u : R::kNegInf;       // what a lane beyond the end of a segment finds: no weight
     constexpr size_t ESZ = (DT == kF32) ? 4 : 2;
     __shared__ SmallShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -111,7 +113,7 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
         }
         for (int i = lane; i < B * (g + 2); i += 32) sh.u[i] = prm.uni[i];
     }
-    for (int item = blockIdx.x; item < nrows * nch; item += gridDim.x) {
+    for (int item = blockIdx.x; !PROBS && item < nrows * nch; item += gridDim.x) {
         const int rid = item / nch, ch = item % nch;
         if (prm.lse_d != nullptr && rid % rpb > g) continue;      // (a draft row whose normaliser is supplied: nothing to learn)
         const char* row = small_row(prm, row_bytes, rid / rpb, rid % rpb);
@@ -147,11 +149,13 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
         }
         __syncthreads();
     }
-    alive = small_grid_barrier(sc.barrier, gridDim.x, prm.status, limit, prm.never_signal && blockIdx.x == 0);
+    if (PROBS) __syncthreads();
+    else alive = small_grid_barrier(sc.barrier, gridDim.x, prm.status, limit, prm.never_signal && blockIdx.x == 0);
 
     // ---------------- phase 2a: normalisers of every row, the scalar part of every sequence ----------------
     if (alive) {
         for (int rid = tid; rid < nrows; rid += kSmAllThreads) {
+            if (PROBS) { sh.rowM[rid] = 0.f; sh.rowZ[rid] = 1.0; continue; }
             if (prm.lse_d != nullptr && rid % rpb > g) {
                 // the supplied normaliser as an integer reference at or above every scaled logit of the row
                 // plus a sum in [2^-1/2, 2^1/2]; a value that is not finite leaves the row without a reference
@@ -191,9 +195,16 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
                     const double ZP = sh.rowZ[b * rpb + c], ZQ = sh.rowZ[b * rpb + g + 1 + c];
                     const bool xok = sh.xok[b * (g + 1) + c] != 0;
                     const double zp = sh.zp[b * (g + 1) + c], zq = sh.zq[b * (g + 1) + c];
-                    bool bad = !(MP > kNoRef && MP < INFINITY) || !(ZP < static_cast<double>(INFINITY)) ||
-                               !(MQ > kNoRef && MQ < INFINITY) || !(ZQ < static_cast<double>(INFINITY)) || !xok || zq == -INFINITY;
-                    rat[h] = bad ? 0.0 : exp2((zp - zq) * prm.kd - (static_cast<double>(MP) - static_cast<double>(MQ))) * (ZQ / ZP);
+                    bool bad;
+                    if (PROBS) {
+                        // the stored numbers themselves: Q must be a positive finite number, P a non-negative finite one
+                        bad = !xok || !(zq > 0.0 && zq < static_cast<double>(INFINITY)) || !(zp >= 0.0 && zp < static_cast<double>(INFINITY));
+                        rat[h] = bad ? 0.0 : zp / zq;
+                    } else {
+                        bad = !(MP > kNoRef && MP < INFINITY) || !(ZP < static_cast<double>(INFINITY)) ||
+                              !(MQ > kNoRef && MQ < INFINITY) || !(ZQ < static_cast<double>(INFINITY)) || !xok || zq == -INFINITY;
+                        rat[h] = bad ? 0.0 : exp2((zp - zq) * prm.kd - (static_cast<double>(MP) - static_cast<double>(MQ))) * (ZQ / ZP);
+                    }
                     badrow[h] = bad;
                     sh.ratio[b * (g + 1) + c] = rat[h];
                     // the uniform that decides about this lane's row / position
@@ -202,7 +213,7 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
             }
             const float MPg = sh.rowM[b * rpb + g];
             const double ZPg = sh.rowZ[b * rpb + g];
-            const bool bad_last = !(MPg > kNoRef && MPg < INFINITY) || !(ZPg < static_cast<double>(INFINITY));
+            const bool bad_last = !PROBS && (!(MPg > kNoRef && MPg < INFINITY) || !(ZPg < static_cast<double>(INFINITY)));
             const unsigned bad_lo = __ballot_sync(0xffffffffu, badrow[0]), bad_hi = __ballot_sync(0xffffffffu, badrow[1]);
             unsigned m_lo = 0, m_hi = 0;
             int lastw = 0, bad = 0, tau_tv = 0;
@@ -299,7 +310,7 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
             double acc = 0.0;
             for (int base = s0; warp < kSmWarps && base < s1; base += 32 * kSmPairsInFlight) {
                 uint4 rp[kSmPairsInFlight], rq[kSmPairsInFlight];
-                const uint4 ninf = make_uint4(R::kNegInf, R::kNegInf, R::kNegInf, R::kNegInf);
+                const uint4 ninf = make_uint4(kPad, kPad, kPad, kPad);
 #pragma unroll
                 for (int j = 0; j < kSmPairsInFlight; ++j) {
                     const int v = base + 32 * j + lane;
@@ -311,15 +322,17 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
                     float vp[EPV], vq[EPV], t[EPV];
                     R::unpack(rp[j], vp);
                     R::unpack(rq[j], vq);
-                    if (have_q) acc += static_cast<double>(f_pair_sum<EPV, true>(vp, vq, kf, cp, nMP, nMQ, t));
-                    else acc += static_cast<double>(f_pair_sum<EPV, false>(vp, vq, kf, cp, nMP, nMQ, t));
+                    if (have_q) acc += static_cast<double>(f_pair_sum<EPV, true, PROBS>(vp, vq, kf, cp, nMP, nMQ, t));
+                    else acc += static_cast<double>(f_pair_sum<EPV, false, PROBS>(vp, vq, kf, cp, nMP, nMQ, t));
                 }
             }
             acc = warp_sum_d(acc);
             if (lane == 0 && warp < kSmWarps) sc.seg[(static_cast<size_t>(b) * (g + 1) + i) * nseg + piece * kSmWarps + warp] = acc;
         }
     }
-    if (alive) alive = small_grid_barrier(sc.barrier, 2u * gridDim.x, prm.status, limit, false);
+    // (arrivals are counted up through the launch: the second barrier of a launch on logits, the only one otherwise)
+    if (alive) alive = small_grid_barrier(sc.barrier, (PROBS ? 1u : 2u) * gridDim.x, prm.status, limit,
+                                          PROBS && prm.never_signal && blockIdx.x == 0);
 
     // ---------------- phase 3: one CTA per sequence ----------------
     for (int b = blockIdx.x; alive && b < B; b += gridDim.x) {
@@ -397,7 +410,7 @@ __global__ void __launch_bounds__(kSmAllThreads, 1) verify_small_kernel(const Pa
                 const double before = shfl_d(bef, src);
                 int s0, s1;
                 small_seg_range(units, nseg, sel, s0, s1);
-                found = f_rescan<DT, false, 5>(small_row(prm, row_bytes, b, tau), have_q ? small_row(prm, row_bytes, b, g + 1 + tau) : nullptr,
+                found = f_rescan<DT, PROBS, 5>(small_row(prm, row_bytes, b, tau), have_q ? small_row(prm, row_bytes, b, g + 1 + tau) : nullptr,
                                      s0, s1, lane, kf, sh.csc[b * (g + 1) + tau], -sh.rowM[b * rpb + tau],
                                      have_q ? -sh.rowM[b * rpb + g + 1 + tau] : 0.f, t - before);
             }
@@ -494,11 +507,15 @@ void small_scratch_layout(void* base, unsigned* barrier, int B, int gamma, const
 }
 
 using SKernelFn = void (*)(const Params, const SmallScratch);
-static SKernelFn pick_small(int dtype) { return dtype == kF32 ? verify_small_kernel<kF32> : verify_small_kernel<kBF16>; }
+static SKernelFn pick_small(int dtype, bool probs) {
+    if (probs) return dtype == kF32 ? verify_small_kernel<kF32, true> : verify_small_kernel<kBF16, true>;
+    return dtype == kF32 ? verify_small_kernel<kF32, false> : verify_small_kernel<kBF16, false>;
+}
 
 int small_max_ctas(int dtype, int sm_count) {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_small(dtype), kSmAllThreads, 0) != cudaSuccess) {
+    // (the variant on logits is the larger program)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, pick_small(dtype, false), kSmAllThreads, 0) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -509,7 +526,7 @@ cudaError_t launch_small(const Params& prm, const SmallScratch& sc, int dtype, i
     Params p = prm;
     SmallScratch s = sc;
     void* args[] = {&p, &s};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_small(dtype)), dim3(nctas), dim3(kSmAllThreads), args, 0, stream);
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_small(dtype, prm.probs != 0)), dim3(nctas), dim3(kSmAllThreads), args, 0, stream);
 }
 
 }  // namespace bv

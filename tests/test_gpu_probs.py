@@ -53,11 +53,15 @@ def test_probabilities_match_the_oracle(algo, name, B, gamma):
     run_case(algo, probs_inputs(w), "probs %s B=%d gamma=%d %s" % (name, B, gamma, algo))
 
 
+@pytest.mark.parametrize("kernel", [1, 4])         # the flow kernel, the small-batch kernel
 @pytest.mark.parametrize("algo", ["block", "token"])
 @pytest.mark.parametrize("V", [8, 24, 1000, 4104, 33000])
-def test_ragged_vocabularies(algo, V):
+def test_ragged_vocabularies(algo, V, kernel, bv_options):
+    import paper_2403_10444_b200 as bv
+    bv_options("kernel", kernel)
     w = wl.scaled(wl.CONFIGS["c3"], B=17, gamma=3, V=V)
-    run_case(algo, probs_inputs(w), "probs ragged V=%d %s" % (V, algo))
+    run_case(algo, probs_inputs(w), "probs ragged V=%d %s kernel %d" % (V, algo, kernel))
+    assert bv.bv_last_kernel() == kernel
 
 
 @pytest.mark.parametrize("algo", ["block", "token"])
@@ -67,8 +71,10 @@ def test_high_acceptance_reaches_the_last_row(algo):
     assert (ref.out_len == 7).sum() > 5
 
 
+@pytest.mark.parametrize("kernel", [1, 4])
 @pytest.mark.parametrize("algo", ["block", "token"])
-def test_faults_are_per_sequence_and_rows_are_used_as_stored(algo):
+def test_faults_are_per_sequence_and_rows_are_used_as_stored(algo, kernel, bv_options):
+    bv_options("kernel", kernel)
     w = wl.scaled(wl.CONFIGS["c2"], B=6, gamma=4, V=4096)
     inp = probs_inputs(w)
     tok = inp["draft_tokens"]
@@ -91,7 +97,9 @@ def test_rows_that_are_not_whole_vectors_are_refused():
     assert e.value.status == -2
 
 
-def test_only_the_needed_rows_are_read():
+@pytest.mark.parametrize("kernel", [1, 4])
+def test_only_the_needed_rows_are_read(kernel, bv_options):
+    bv_options("kernel", kernel)
     # rows that neither algorithm reads may hold anything: here NaN everywhere except the entries of
     # the drafted tokens, in the positions that cannot be the selected one
     import paper_2403_10444_b200 as bv
