@@ -52,10 +52,13 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
         float* sS = sS2[it & 1];
         const char* row = logits + static_cast<size_t>(r) * row_bytes;
         // ---- one pass over the warp's part of the row ----
+        // (the warp's reference carries over from one sub-segment to the next: a sub-segment's pair is
+        // its sum against the reference as it stood at its end, and only the first one has to find one)
+        float M = kNoRef;
         for (int sub = 0; sub < kSSub; ++sub) {
             int a0, a1;
             s_range(units, warp, sub, a0, a1);
-            float M = kNoRef, s = 0.f;
+            float s = 0.f;
             const uint4 ninf = make_uint4(R::kNegInf, R::kNegInf, R::kNegInf, R::kNegInf);
             for (int base = a0; base < a1; base += 32 * kSInFlight) {
                 uint4 raw[kSInFlight];                // all loads of the round are issued before any is used
