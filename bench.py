@@ -464,7 +464,7 @@ TRAFFIC_BYTES = {
     ("c4", "token", "verify_flow_kernel"): 821143040,
     ("c4", "greedy", "verify_flow_kernel"): 2579974656,
     ("c4", "block_lse", "verify_flow_kernel"): 1521103360,
-    ("c4", "sample", "sample_rows_kernel"): 1056510720,
+    ("c4", "sample", "sample_rows_kernel"): 1058290944,
     ("c4", "block_probs", "verify_flow_kernel"): 350806016,
     ("c4", "token_probs", "verify_flow_kernel"): 264784384,
 }

@@ -4,7 +4,7 @@
 //
 // Persistent CTAs take rows round-robin.  Each of 16 warps streams its contiguous sixteenth of the
 // row once, in eight sub-segments, and leaves each sub-segment's {integer reference, sum 2^{z k - M}}
-// in shared memory; a seventeenth warp, one row behind, combines the 128 pairs (fp64 for the
+// in shared memory; a seventeenth warp, a row behind, combines the 128 pairs (fp64 for the
 // normaliser and for the sampler's prefix sums), finds the sub-segment that holds u * Z and rescans
 // that one - a few KB still in L2 - in index order for the token.  Each logit is read from HBM once.
 #include <cmath>
@@ -22,6 +22,16 @@ constexpr int kSAllThreads = kSThreads + 32;
 constexpr int kSSub = 8;                          // sub-segments per warp
 constexpr int kSSegs = kSWarps * kSSub;           // 128: four per lane of warp 0
 constexpr int kSInFlight = 8;                     // 16-byte loads a thread has in flight
+
+// named barriers of a CTA (hardware barriers 1 .. 15; 0 is __syncthreads): all lanes of a warp take part,
+// `threads` is the number of threads that arrive or wait at the barrier per use
+constexpr int kBarFull = 1, kBarEmpty = 3;        // ids kBarFull + buffer, kBarEmpty + buffer
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void named_bar_arrive(int id, int threads) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 
 // vectors [a0, a1) of sub-segment `sub` of warp `warp` in a row of `units` vectors
 __device__ __forceinline__ void s_range(int units, int warp, int sub, int& a0, int& a1) {
@@ -42,11 +52,18 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
     const size_t row_bytes = static_cast<size_t>(V) * ESZ;
     __shared__ float sM2[2][kSSegs], sS2[2][kSSegs];
 
-    // Iteration `it`: the streaming warps sweep the CTA's it-th row while the sampling warp draws
-    // the token of the row before from the pairs that were left for it; one barrier per row.
+    // The streaming warps sweep the CTA's rows one after the other and leave each row's pairs in one of
+    // two buffers; the sampling warp follows, a row behind or so, and draws each row's token from them.
+    // Two named barriers per buffer order the two sides, producer and consumer: "full" (the 16 streaming
+    // warps arrive when the row's pairs are written, the sampling warp waits) and "empty" (the sampling
+    // warp arrives when it has read them, the streaming warps wait before they write that buffer again,
+    // two rows later).  The streaming warps never wait for one another: there is no barrier across a row.
+    // Every wait ends: the row count is the same for all warps of the CTA, each row has exactly one
+    // arrival and one wait per side, and the streaming side waits for row `it - 2` only from row 2 on.
     const int nmine = rows > static_cast<int>(blockIdx.x) ? (rows - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
-    for (int it = 0; it <= nmine; ++it) {
-        if (warp < kSWarps && it < nmine) {
+    if (warp < kSWarps) {
+        for (int it = 0; it < nmine; ++it) {
+        if (it >= 2) named_bar_sync(kBarEmpty + (it & 1), kSAllThreads);
         const int r = blockIdx.x + it * gridDim.x;
         float* sM = sM2[it & 1];
         float* sS = sS2[it & 1];
@@ -79,11 +96,15 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
             s = warp_sum(s);
             if (lane == 0) { sM[warp * kSSub + sub] = M; sS[warp * kSSub + sub] = s; }
         }
+        __threadfence_block();
+        named_bar_arrive(kBarFull + (it & 1), kSAllThreads);
         }
-        if (warp == kSWarps && it >= 1) {
-            const int r = blockIdx.x + (it - 1) * gridDim.x;
-            const float* sM = sM2[(it - 1) & 1];
-            const float* sS = sS2[(it - 1) & 1];
+    } else {
+        for (int it = 0; it < nmine; ++it) {
+            named_bar_sync(kBarFull + (it & 1), kSAllThreads);
+            const int r = blockIdx.x + it * gridDim.x;
+            const float* sM = sM2[it & 1];
+            const float* sS = sS2[it & 1];
             const char* row = logits + static_cast<size_t>(r) * row_bytes;
             // ---- normaliser and the sampled sub-segment (fp64 prefix sums, index order) ----
             float m[4], w[4];
@@ -108,6 +129,7 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
             const double total = shfl_d(inc, 31);
             // a row with a NaN or +inf logit has a NaN / infinite sum or reference; one without a finite logit has none
             const bool ok = Mrow > kNoRef && Mrow < INFINITY && Z > 0.0 && Z < INFINITY && total > 0.0 && total < static_cast<double>(INFINITY);
+            if (it + 2 < nmine) named_bar_arrive(kBarEmpty + (it & 1), kSAllThreads);   // (the pairs are in registers; row it + 2 waits for this)
             int found = -1;
             if (ok) {
                 const double t = static_cast<double>(uni[r]) * total;
@@ -141,7 +163,6 @@ sample_rows_kernel(const char* logits, const float* uni, int rows, int V, float 
                                              : __int_as_float(0x7fc00000);
             }
         }
-        __syncthreads();      // row `it` is swept, the token of row `it - 1` is drawn
     }
 }
 
