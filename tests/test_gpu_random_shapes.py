@@ -48,3 +48,49 @@ def test_random_shapes(seed, bv_options):
                         w.B, w.gamma, w.V, w.dtype, w.temperature, w.draft_sigma, algo, name, "diagnostics" if diag else "plain"))
                     assert_parity(rep, diag), (w, algo, name, diag)
                     assert bv.bv_stream_status() == 0
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_shapes_other_entry_points(seed, bv_options):
+    """The entry points on probabilities, with supplied draft normalisers, and the drafting step."""
+    import numpy as np
+    import torch
+    import paper_2403_10444_b200 as bv
+    from parity import to_numpy_logits
+    rnd = random.Random(2000 + seed)
+    for _ in range(6):
+        w = draw(rnd)
+        inp = wl.make_inputs(w, "cpu")
+        T, g, V = w.temperature, w.gamma, w.V
+        fits_small = w.B <= 32 and w.B * (2 * g + 1) <= 1056 and w.B * (g + 1) <= 560
+        kernels = [c for n, c in KERNELS.items() if n != "small" or fits_small]
+        pin = dict(inp)
+        for k in ("target_logits", "draft_logits"):
+            pin[k] = torch.softmax(inp[k].double() / T, -1).to(inp[k].dtype).contiguous()
+        a = tuple(pin[k].cuda() for k in ("target_logits", "draft_logits", "draft_tokens", "uniforms"))
+        for algo, fn in ((oracle.BLOCK_VERIFY, bv.bv_verify_probs), (oracle.TOKEN_VERIFY, bv.tv_verify_probs)):
+            ref = oracle.verify_probs(algo, to_numpy_logits(pin["target_logits"]), to_numpy_logits(pin["draft_logits"]),
+                                      pin["draft_tokens"].numpy(), pin["uniforms"].numpy())
+            for code in kernels:
+                bv_options("kernel", code)
+                for diag in (True, False):
+                    out = fn(*a, diagnostics=diag)
+                    assert_parity(compare(algo, ref, out[0], out[1], out[2] if diag else None, pin, probs=True), diag)
+        lse = torch.logsumexp(inp["draft_logits"].double() / np.float32(T), -1).float()
+        ref = oracle.verify(oracle.BLOCK_VERIFY, to_numpy_logits(inp["target_logits"]), to_numpy_logits(inp["draft_logits"]),
+                            inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), T, draft_lse=lse.numpy())
+        d = {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in inp.items()}
+        for code in kernels:
+            bv_options("kernel", code)
+            for diag in (True, False):
+                out = bv.bv_verify_lse(d["target_logits"], d["draft_logits"], d["draft_tokens"], d["uniforms"], lse.cuda(), T,
+                                       diagnostics=diag)
+                assert_parity(compare(oracle.BLOCK_VERIFY, ref, out[0], out[1], out[2] if diag else None, inp), diag)
+        assert bv.bv_stream_status() == 0
+        rows = inp["draft_logits"].reshape(-1, V).contiguous()
+        u = inp["uniforms"][:, :g].reshape(-1).contiguous()
+        want_tok, want_lse, margin = oracle.sample_rows(to_numpy_logits(rows), u.numpy(), T)
+        tok, l = bv.bv_sample_draft(rows.cuda(), u.cuda(), T)
+        tok, l = tok.cpu().numpy(), l.cpu().numpy().astype(np.float64)
+        assert not ((tok != want_tok) & ~(margin < 1e-6)).any()
+        assert np.abs(l - want_lse).max() <= 3e-6
