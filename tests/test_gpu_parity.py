@@ -224,3 +224,28 @@ def test_skipped_second_sweeps_change_nothing(sigma_d):
         full = run_cuda(oracle.BLOCK_VERIFY, inp, diagnostics=True)
         fast = run_cuda(oracle.BLOCK_VERIFY, inp, diagnostics=False)
         assert torch.equal(full[0], fast[0]) and torch.equal(full[1], fast[1])
+
+
+def test_calls_on_several_streams_at_once():
+    # every stream has a workspace of its own: calls in flight together on different streams, of shapes
+    # that the flow kernel and the small-batch kernel serve, give what the same calls give one by one
+    import paper_2403_10444_b200 as bv
+    shapes = [(48, 5, 16384, "bf16"), (6, 4, 8192, "f32"), (80, 3, 4096, "bf16"), (2, 8, 32000, "bf16")]
+    cases = []
+    for i, (B, g, V, dt) in enumerate(shapes):
+        inp = {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in random_inputs(B, g, V, dt, seed=500 + i).items()}
+        a = (inp["target_logits"], inp["draft_logits"], inp["draft_tokens"], inp["uniforms"], inp["temperature"])
+        cases.append((a, bv.bv_verify(*a), bv.tv_verify(*a)))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in cases]
+    for rep in range(3):
+        outs = []
+        for (a, _, _), s in zip(cases, streams):
+            with torch.cuda.stream(s):
+                outs.append((bv.bv_verify(*a, stream=s), bv.tv_verify(*a, stream=s)))
+        for s in streams:
+            s.synchronize()
+            assert bv.bv_stream_status(s) == 0
+        for (a, want_b, want_t), (got_b, got_t) in zip(cases, outs):
+            assert torch.equal(got_b[0], want_b[0]) and torch.equal(got_b[1], want_b[1])
+            assert torch.equal(got_t[0], want_t[0]) and torch.equal(got_t[1], want_t[1])
