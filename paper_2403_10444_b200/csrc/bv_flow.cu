@@ -1,30 +1,34 @@
-// Block Verification (Algorithm 2) as a dependency-driven flow of independent work items.
+// Block Verification (Algorithm 2; also Algorithm 4, Algorithm 1 and the variants with supplied
+// draft normalisers or with probabilities as inputs) as a dependency-driven flow of independent work items.
 //
-// Persistent CTAs (16 worker warps that only stream, one service warp that does everything
-// else) pull items from three sources, in this order of preference:
+// Persistent CTAs of 14 worker warps that only stream, one publisher warp that finds the next items
+// and hands their descriptors to the workers, and three post warps that do what follows the sweep
+// of an item.  Items come from three sources, in this order of preference:
 //
-//   sweep-2 piece (b, r, piece)  a piece of a row pair whose second sweep has been started:
-//       leaves sum max(p_r P_r(x) - Q_r(x), 0) per warp segment (Eq. "pacc_block").  The CTA
+//   sweep-2 piece (b, r, piece)  a piece of a row pair whose second sweep has been asked for:
+//       leaves sum max(p_r P_r(x) - Q_r(x), 0) per warp segment (Eq. "pacc_block").  The warp
 //       that completes a position adds the segments to S_r, locates u * S_r, rescans that one
 //       segment in index order for the candidate Y_r (Eq. "pres-block"), and then either finds
-//       the position selected or starts the next lower candidate; the CTA that completes the
+//       the position selected or asks for the next lower candidate; the warp that completes the
 //       block forms h_i, selects tau and emits X^tau, Y_tau.
-//   late sweep-1 chunk  of a last target row P_gamma, which is read only if position gamma can
-//       be the selected one; its sample is drawn from that one sweep.
-//   sweep-1 item (b, r < gamma, chunk)  by ticket, in row order: streams the chunk of both
-//       rows from HBM and leaves the chunk's {reference, sum 2^{z k - M}} pair for each row in
-//       scratch.  The CTA that completes a row combines the chunks into the row normalisers
-//       and, holding the block's lock, advances the prefix recursion
-//       p_{r+1} = min(p_r P_r(X)/Q_r(X), 1) (Eq. "def_as") over every row that is complete.
+//   late sweep-1 chunk  of a row whose first sweep is asked for on demand: a last target row
+//       P_gamma, which is read only if position gamma can be the selected one (its sample is drawn
+//       from that one sweep); under Algorithm 1 a row whose tests before it have all passed.
+//   sweep-1 item (b, r < gamma, chunk)  by ticket: streams the chunk of both rows from HBM and
+//       leaves the chunk's {reference, sum 2^{z k - M}} pair for each row in scratch.  The warp
+//       that completes a row combines the chunks into the row normalisers; the warp that
+//       completes the last row of a block folds it: the prefix recursion
+//       p_{r+1} = min(p_r P_r(X)/Q_r(X), 1) (Eq. "def_as") and which positions are candidates.
 //
 // A second sweep runs only where the outcome can depend on it: S_r <= p_r gives h_r <= p_r, so
 // a position with eta_r > p_r can never be selected; the others are swept from the top down
 // until one passes its test (bv_flow_common.cuh).  With diagnostic outputs every position is
 // swept.
 //
-// No CTA ever waits for another one while it holds work that others need: sweep-1 items
-// have no prerequisites, the lock is only held over a few scalar operations, and a CTA
-// polls (bounded) only when nothing is left to start.  So CTAs need not be co-resident.
+// Every hand-over is a counter in global memory whose last increment elects the warp that goes on
+// (no locks).  No CTA ever waits for another one while it holds work that others need: sweep-1
+// items have no prerequisites, and a CTA polls (bounded) only when nothing is left to start.  So
+// CTAs need not be co-resident.
 #include "bv_flow_common.cuh"
 
 namespace bv {
@@ -77,8 +81,8 @@ struct FlowDesc {
 
 struct FlowShared {
     FlowDesc desc[kFDesc];
-    unsigned long long full[kFDesc];    // the service warp has filled desc[i]
-    unsigned long long done[kFDesc];    // all 16 worker warps have left their partials of desc[i]
+    unsigned long long full[kFDesc];    // the publisher has filled desc[i]
+    unsigned long long done[kFDesc];    // all worker warps have left their partials of desc[i]
     float part_M[kFDesc][2][kFWarps];   // sweep 1: references of P and Q per worker warp
     float part_s[kFDesc][kFWarps];      // sweep 1: sums of the draft row
     double part_d[kFDesc][kFWarps];     // sweep 1: sums of the target row; sweep 2: the residual totals (they decide sampled
@@ -93,7 +97,7 @@ struct FlowShared {
     unsigned posted;                    // items whose post-processing is complete
 };
 
-// ---- service warp: Y ~ P_gamma from the first sweep of the last target row ----
+// ---- post warp: Y ~ P_gamma from the first sweep of the last target row ----
 // The sample needs the row's normaliser and a second look at one segment only: the segment
 // {reference, sum} pairs of all chunks are in scratch, so u * Z is located among their prefix sums
 // (fp32, index order) and that one segment is rescanned.  No second sweep of the row.
@@ -157,7 +161,7 @@ __device__ void f_draw_from_sweep1(const Params& prm, const FlowScratch& fl, con
     __syncwarp();
 }
 
-// ---- service warp: what follows the sweep of an item, in three steps, so that several finished
+// ---- post warp: what follows the sweep of an item, in three steps, so that several finished
 // items can share one fence and have their counters bumped side by side:
 //   store     the item's result goes to scratch;
 //   (one __threadfence for all of them, then one atomic per item, each by a lane of its own)
