@@ -161,10 +161,9 @@ __device__ void f_draw_from_sweep1(const Params& prm, const FlowScratch& fl, con
     __syncwarp();
 }
 
-// ---- post warp: what follows the sweep of an item, in three steps, so that several finished
-// items can share one fence and have their counters bumped side by side:
+// ---- post warp: what follows the sweep of an item, in three steps:
 //   store     the item's result goes to scratch;
-//   (one __threadfence for all of them, then one atomic per item, each by a lane of its own)
+//   (one __threadfence, then one atomic on the counter of the item's row or position)
 //   complete  for the item that was the last of its row or position. ----
 template <int DT>
 __device__ void f_store_sweep1(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, FlowShared& sh, int j,
