@@ -83,7 +83,7 @@ extern "C" int bv_verify_noalloc(const void* tgt, const void* drf, const int32_t
     if (need > kScratchBytes) return BV_ERR_TOO_LARGE;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // The array keeps what the previous call left: counters, locks and the ready list must
+    // The array keeps what the previous call left: counters, flags and the queues must
     // start at zero, and so does the status word at the very end of the used part.
     if ((e = cudaMemsetAsync(d.scratch, 0, zero_bytes, s)) != cudaSuccess) return bv::note_cuda_error(e);
     unsigned char* status_word = d.scratch + (need - 256);
