@@ -102,13 +102,12 @@ def dist_setup(n_gpus: int):
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        # NCCL's own account of the communicator (topology, transports) goes to a file beside the other
-        # outputs of a run, not to stdout, where the one JSON line must stay alone
+        # NCCL's own account of the communicator (topology, transports) goes to a file in the system's
+        # temporary directory, not to stdout, where the one JSON line must stay alone
         if "NCCL_DEBUG" not in os.environ:
-            logdir = os.path.join(ROOT, "gpurun_out")
-            os.makedirs(logdir, exist_ok=True)
+            import tempfile
             os.environ["NCCL_DEBUG"] = "INFO"
-            os.environ.setdefault("NCCL_DEBUG_FILE", os.path.join(logdir, "nccl_%h_%p.log"))
+            os.environ.setdefault("NCCL_DEBUG_FILE", os.path.join(tempfile.gettempdir(), "bv_bench_nccl_%h_%p.log"))
         torch.cuda.set_device(local)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
         return rank, world, local, dist
