@@ -8,7 +8,7 @@ workload is B=256, gamma=8, V=256000, bf16 (2.2 GB of logits, far larger than
 L2, so nothing is served from cache between steps).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload c1|c2|c3|c4] [--algo block|token|sample|block_lse|greedy]
+                    [--workload c1|c2|c3|c4] [--algo block|token|sample|block_lse|token_lse|greedy|block_probs|token_probs]
 
 Prints one JSON line.  With N > 1 (launched by torch.distributed.run) every rank
 verifies its own batch of the same shape (weak scaling, no collective on the
@@ -147,7 +147,7 @@ class OracleRun:
         g = inp["draft_tokens"].shape[1]
         p = {"t": t, "d": d, "x": inp["draft_tokens"].numpy(), "u": inp["uniforms"].numpy(),
              "T": inp["temperature"], "B": inp["draft_tokens"].shape[0]}
-        if self.algo_name == "block_lse":
+        if self.algo_name.endswith("_lse"):
             p["lse"] = torch.logsumexp(inp["draft_logits"].double() / inp["temperature"], -1).float().numpy()
         if self.algo_name == "sample":
             p["rows"] = d.reshape(-1, d.shape[-1])
@@ -161,7 +161,7 @@ class OracleRun:
             o.sample_rows(p["rows"], p["u_rows"], p["T"])
         elif self.probs:
             o.verify_probs(self.algo, p["t"], p["d"], p["x"], p["u"])
-        elif self.algo_name == "block_lse":
+        elif self.algo_name.endswith("_lse"):
             o.verify(self.algo, p["t"], p["d"], p["x"], p["u"], p["T"], draft_lse=p["lse"])
         else:
             o.verify(self.algo, p["t"], p["d"], p["x"], p["u"], p["T"])
@@ -218,7 +218,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(wl.CONFIGS))
-    ap.add_argument("--algo", default="block", choices=["block", "token", "sample", "block_lse", "greedy", "block_probs", "token_probs"],
+    ap.add_argument("--algo", default="block", choices=["block", "token", "sample", "block_lse", "token_lse", "greedy", "block_probs", "token_probs"],
                     help="block / token verification, the drafting step (sampling the draft rows), block "
                          "verification with the draft normalisers that the drafting step leaves, or one "
                          "iteration of greedy block verification (Algorithm 4); block_probs / token_probs: the "
@@ -262,12 +262,13 @@ def main():
         u_rows = inp["uniforms"][:, : w.gamma].contiguous().view(-1)
         fn = lambda *_: bv.bv_sample_draft(rows2d, u_rows, inp["temperature"])
         args.e2e_steps = 0          # (no host-buffer form of this entry point)
-    if args.algo == "block_lse":
+    if args.algo in ("block_lse", "token_lse"):
         # normalisers as the drafting step leaves them, computed once outside the timed region
         lse = bv.bv_sample_draft(inp["draft_logits"].view(w.B * w.gamma, w.V),
                                  inp["uniforms"][:, : w.gamma].contiguous().view(-1), inp["temperature"])[1]
         lse = lse.view(w.B, w.gamma).contiguous()
-        fn = lambda *_: bv.bv_verify_lse(*a[:4], lse, a[4])
+        lfn = bv.bv_verify_lse if args.algo == "block_lse" else bv.tv_verify_lse
+        fn = lambda *_: lfn(*a[:4], lse, a[4])
         args.e2e_steps = 0
     if args.algo == "greedy":
         fn = bv.gbv_verify
@@ -396,6 +397,12 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
     elif args.algo == "block_lse":
         # what must be read at least: every target row, and one draft row per block for the residual
         algo_bytes = w.B * (w.gamma + 2) * w.V * esz
+        kernel = "verify_flow_kernel"
+    elif args.algo == "token_lse":
+        # Algorithm 1 with supplied draft normalisers: target rows 0 .. min(n, gamma) - 1 for the tests, the target
+        # row at tau (already among them unless every token was accepted) and the draft row at tau for the residual
+        n = out[1].long().clamp(min=0)
+        algo_bytes = int((n.clamp(max=w.gamma) + 1).sum().item()) * w.V * esz
         kernel = "verify_flow_kernel"
     elif args.algo in ("block_probs", "token_probs"):
         # given probabilities, what must be read is the row pair at the selected position (or the last

@@ -196,6 +196,24 @@ int bv_verify_lse_ex(const void* target_logits, const void* draft_logits,
                      float* out_lse_t, float* out_lse_d, void* stream);
 
 /*
+ * Token Verification (Algorithm 1) with the draft rows' log-normalisers supplied, as bv_verify_lse: the
+ * acceptance tests read the target rows only (the draft row of a test contributes the one logit of
+ * its drafted token), and a draft row is read in full only where the residual of Eq. "pres-token" is
+ * sampled.  Same rules as bv_verify_lse; a draft_lse entry that is not finite counts as a data fault if
+ * its row is among rows 0 .. min(tau, gamma - 1).
+ */
+int tv_verify_lse(const void* target_logits, const void* draft_logits,
+                  const int32_t* draft_tokens, const float* uniforms, const float* draft_lse,
+                  int B, int gamma, int V, int dtype, float temperature,
+                  int32_t* out_tokens, int32_t* out_len, void* stream);
+int tv_verify_lse_ex(const void* target_logits, const void* draft_logits,
+                     const int32_t* draft_tokens, const float* uniforms, const float* draft_lse,
+                     int B, int gamma, int V, int dtype, float temperature,
+                     int32_t* out_tokens, int32_t* out_len,
+                     float* out_p, float* out_S, float* out_h,
+                     float* out_lse_t, float* out_lse_d, void* stream);
+
+/*
  * Greedy Block Verification, one iteration: Algorithm 4.  The running product is not clipped,
  *   pt_0 = 1,  pt_i = pt_{i-1} P_{i-1}(X_i) / Q_{i-1}(X_i);
  * position 0 < i < gamma passes its test when eta_i <= h_i with

@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_verify_probs", "tv_verify_probs", "bv_sample_draft", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_kernel", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "tv_verify_lse", "tv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_verify_probs", "tv_verify_probs", "bv_sample_draft", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_kernel", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -57,8 +57,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.bv_sample_draft.argtypes = [vp, vp, ci, ci, ci, cf, vp, vp, vp]
     for name in ("bv_verify_probs", "tv_verify_probs"):
         getattr(lib, name).argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp]
-    lib.bv_verify_lse.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp]
-    lib.bv_verify_lse_ex.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp, vp, vp, vp, vp, vp]
+    for name in ("bv_verify_lse", "tv_verify_lse"):
+        getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp]
+        getattr(lib, name + "_ex").argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp, vp, vp, vp, vp, vp]
     for name in EXPORTS:
         getattr(lib, name).restype = ci
     lib.bv_stream_status.argtypes = [vp]
@@ -317,6 +318,18 @@ def bv_verify_lse(target_logits, draft_logits, draft_tokens, uniforms, draft_lse
     """Block Verification with the draft rows' log-normalisers supplied (float32 CUDA tensor
     [B, gamma], e.g. the second output of bv_sample_draft reshaped).  Returns (out_tokens, out_len)
     or, with ``diagnostics``, (out_tokens, out_len, dict of p, S, h, lse_t, lse_d)."""
+    return _lse_call("bv_verify_lse", target_logits, draft_logits, draft_tokens, uniforms, draft_lse, temperature,
+                     diagnostics, stream)
+
+
+def tv_verify_lse(target_logits, draft_logits, draft_tokens, uniforms, draft_lse, temperature: float = 1.0,
+                  diagnostics: bool = False, stream=None):
+    """Token Verification with the draft rows' log-normalisers supplied; see bv_verify_lse."""
+    return _lse_call("tv_verify_lse", target_logits, draft_logits, draft_tokens, uniforms, draft_lse, temperature,
+                     diagnostics, stream)
+
+
+def _lse_call(name, target_logits, draft_logits, draft_tokens, uniforms, draft_lse, temperature, diagnostics, stream):
     lib = load_library()
     B, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms, True)
     if (not draft_lse.is_cuda or draft_lse.dtype != torch.float32 or tuple(draft_lse.shape) != (B, gamma)
@@ -334,7 +347,7 @@ def bv_verify_lse(target_logits, draft_logits, draft_tokens, uniforms, draft_lse
             f = lambda *shape: torch.empty(shape, dtype=torch.float32, device=dev)
             diag = dict(p=f(B, gamma + 1), S=f(B, gamma), h=f(B, gamma + 1), lse_t=f(B, gamma + 1), lse_d=f(B, gamma))
             args += [diag[k].data_ptr() for k in ("p", "S", "h", "lse_t", "lse_d")]
-            _check(lib.bv_verify_lse_ex(*args, s.cuda_stream))
+            _check(getattr(lib, name + "_ex")(*args, s.cuda_stream))
             return out_tokens, out_len, diag
-        _check(lib.bv_verify_lse(*args, s.cuda_stream))
+        _check(getattr(lib, name)(*args, s.cuda_stream))
     return out_tokens, out_len

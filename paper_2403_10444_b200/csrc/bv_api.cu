@@ -462,6 +462,23 @@ int bv_verify_lse_ex(const void* tgt, const void* drf, const int32_t* tok, const
     return run_device(bv::kBlockVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, ex, static_cast<cudaStream_t>(stream));
 }
 
+int tv_verify_lse(const void* tgt, const void* drf, const int32_t* tok, const float* uni, const float* draft_lse,
+                  int B, int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, void* stream) {
+    if (!draft_lse) return BV_ERR_INVALID_ARG;
+    Extra ex;
+    ex.lse_d = draft_lse;
+    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, ex, static_cast<cudaStream_t>(stream));
+}
+
+int tv_verify_lse_ex(const void* tgt, const void* drf, const int32_t* tok, const float* uni, const float* draft_lse,
+                     int B, int gamma, int V, int dtype, float T, int32_t* ot, int32_t* ol, float* out_p,
+                     float* out_S, float* out_h, float* out_lse_t, float* out_lse_d, void* stream) {
+    if (!draft_lse) return BV_ERR_INVALID_ARG;
+    Extra ex = diagnostics(out_p, out_S, out_h, out_lse_t, out_lse_d);
+    ex.lse_d = draft_lse;
+    return run_device(bv::kTokenVerify, tgt, drf, tok, uni, B, gamma, V, dtype, T, ot, ol, ex, static_cast<cudaStream_t>(stream));
+}
+
 int bv_verify_probs(const void* tgt, const void* drf, const int32_t* tok, const float* uni, int B, int gamma,
                     int V, int dtype, int32_t* ot, int32_t* ol, float* out_p, float* out_S, float* out_h, void* stream) {
     Extra ex = diagnostics(out_p, out_S, out_h, nullptr, nullptr);

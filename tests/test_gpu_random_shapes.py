@@ -77,15 +77,16 @@ def test_random_shapes_other_entry_points(seed, bv_options):
                     out = fn(*a, diagnostics=diag)
                     assert_parity(compare(algo, ref, out[0], out[1], out[2] if diag else None, pin, probs=True), diag)
         lse = torch.logsumexp(inp["draft_logits"].double() / np.float32(T), -1).float()
-        ref = oracle.verify(oracle.BLOCK_VERIFY, to_numpy_logits(inp["target_logits"]), to_numpy_logits(inp["draft_logits"]),
-                            inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), T, draft_lse=lse.numpy())
         d = {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in inp.items()}
-        for code in kernels:
-            bv_options("kernel", code)
-            for diag in (True, False):
-                out = bv.bv_verify_lse(d["target_logits"], d["draft_logits"], d["draft_tokens"], d["uniforms"], lse.cuda(), T,
-                                       diagnostics=diag)
-                assert_parity(compare(oracle.BLOCK_VERIFY, ref, out[0], out[1], out[2] if diag else None, inp), diag)
+        for algo, fn in ((oracle.BLOCK_VERIFY, bv.bv_verify_lse), (oracle.TOKEN_VERIFY, bv.tv_verify_lse)):
+            ref = oracle.verify(algo, to_numpy_logits(inp["target_logits"]), to_numpy_logits(inp["draft_logits"]),
+                                inp["draft_tokens"].numpy(), inp["uniforms"].numpy(), T, draft_lse=lse.numpy())
+            for code in kernels:
+                bv_options("kernel", code)
+                for diag in (True, False):
+                    out = fn(d["target_logits"], d["draft_logits"], d["draft_tokens"], d["uniforms"], lse.cuda(), T,
+                             diagnostics=diag)
+                    assert_parity(compare(algo, ref, out[0], out[1], out[2] if diag else None, inp), diag)
         assert bv.bv_stream_status() == 0
         rows = inp["draft_logits"].reshape(-1, V).contiguous()
         u = inp["uniforms"][:, :g].reshape(-1).contiguous()
