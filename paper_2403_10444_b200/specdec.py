@@ -6,7 +6,7 @@ models whose next-token logits depend on the last token only (two [V, V] tables 
 Each iteration drafts gamma tokens autoregressively with ``bv_sample_draft`` (which also leaves every
 draft row's log-normaliser), looks up the target rows along the drafted path (the stand-in for the
 parallel scoring pass of the large model), and verifies the block with ``bv_verify_lse`` (Block
-Verification, Algorithm 2), ``bv_verify`` or ``tv_verify`` (Token Verification, Algorithm 1).  The
+Verification, Algorithm 2), ``bv_verify``, ``tv_verify`` (Token Verification, Algorithm 1) or ``tv_verify_lse``.  The
 accepted tokens and the correction token extend every sequence, whose last token is the context of the
 next iteration.  Table look-ups and the bookkeeping of sequence positions are torch indexing; sampling
 and verification run in the CUDA library.  All random numbers are inputs.
@@ -27,7 +27,7 @@ import torch
 from . import binding as bv
 from . import workloads as wl
 
-ALGOS = ("block_lse", "block", "token")
+ALGOS = ("block_lse", "block", "token", "token_lse")
 
 
 def run(target_table: torch.Tensor, draft_table: torch.Tensor, first_tokens: torch.Tensor,
@@ -90,6 +90,8 @@ def run(target_table: torch.Tensor, draft_table: torch.Tensor, first_tokens: tor
         torch.index_select(target_table, 0, path.reshape(-1), out=target_logits.view(B * (gamma + 1), V))
         if algo == "block_lse":
             out, out_len = bv.bv_verify_lse(target_logits, draft_logits, toks, uv, lse, temperature)
+        elif algo == "token_lse":
+            out, out_len = bv.tv_verify_lse(target_logits, draft_logits, toks, uv, lse, temperature)
         elif algo == "block":
             out, out_len = bv.bv_verify(target_logits, draft_logits, toks, uv, temperature)
         else:

@@ -51,7 +51,8 @@ def oracle_loop(tt, dt, first, u_draft, u_verify, gamma, T, algo, supply_lse):
 
 @pytest.mark.parametrize("algo,oalgo,lse", [("block", oracle.BLOCK_VERIFY, False),
                                             ("token", oracle.TOKEN_VERIFY, False),
-                                            ("block_lse", oracle.BLOCK_VERIFY, True)])
+                                            ("block_lse", oracle.BLOCK_VERIFY, True),
+                                            ("token_lse", oracle.TOKEN_VERIFY, True)])
 def test_loop_matches_the_oracle_loop(algo, oalgo, lse):
     V, B, gamma, N, T = 2048, 12, 4, 6, 0.9
     tt, dt = wl.markov_models(V, "bf16", 5, 2.0, 0.8, 1.1, "cpu")
