@@ -291,6 +291,22 @@ int bv_sample_draft(const void* logits, const float* uniforms, int rows, int V, 
                     float temperature, int32_t* out_tokens, float* out_lse, void* stream);
 
 /*
+ * The drafting step of Algorithm 3 as a whole for a draft model whose next-token logits depend on the
+ * last token only: draft_table [V, V] in `dtype`, DEVICE, row t = the logits after token t.  For each
+ * of B sequences, starting from first_tokens[b] (int32, DEVICE), gamma tokens are drawn one after the
+ * other, X_{i+1} from softmax(draft_table[X_i, :] / temperature) by the convention of
+ * bv_sample_draft with uniforms[i, b] (uniforms [gamma, B] float, DEVICE):
+ *   out_tokens [B, gamma] int32, out_lse [B, gamma] float (may be null): the tokens and the
+ *   log-normalisers of the rows they were drawn from, as bv_verify_lse / tv_verify_lse take them.
+ * One launch instead of gamma dependent ones.  A first token outside [0, V) or a row that cannot be
+ * sampled (see bv_sample_draft) ends that sequence's chain: its remaining tokens are -1, their
+ * normalisers NaN.  Rows must be whole 16-byte vectors on a 16-byte aligned base, else BV_ERR_UNSUPPORTED.
+ */
+int bv_draft_chain(const void* draft_table, const int32_t* first_tokens, const float* uniforms,
+                   int B, int gamma, int V, int dtype, float temperature,
+                   int32_t* out_tokens, float* out_lse, void* stream);
+
+/*
  * Waits for `stream` and reports whether a device-side wait of any call enqueued on it since the
  * last query gave up: BV_ERR_TIMEOUT (the outputs of those calls are not to be used; the library's
  * state is intact and later calls work) or BV_OK.  Every device-side wait of this library is

@@ -20,7 +20,7 @@ DTYPE_BF16 = 1
 
 # every symbol include/bv.h declares
 EXPORTS = ["bv_verify", "tv_verify", "bv_verify_ex", "tv_verify_ex", "bv_verify_host",
-           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "tv_verify_lse", "tv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_verify_probs", "tv_verify_probs", "bv_sample_draft", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_kernel", "bv_last_cuda_error",
+           "tv_verify_host", "bv_verify_noalloc", "bv_verify_lse", "bv_verify_lse_ex", "tv_verify_lse", "tv_verify_lse_ex", "gbv_verify", "gbv_verify_ex", "bv_verify_probs", "tv_verify_probs", "bv_sample_draft", "bv_draft_chain", "bv_stream_status", "bv_set_option", "bv_release", "bv_last_launch_count", "bv_last_kernel", "bv_last_cuda_error",
            "bv_status_string", "bv_version"]
 
 
@@ -55,6 +55,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     for name in ("bv_verify_host", "tv_verify_host"):
         getattr(lib, name).argtypes = base
     lib.bv_sample_draft.argtypes = [vp, vp, ci, ci, ci, cf, vp, vp, vp]
+    lib.bv_draft_chain.argtypes = [vp, vp, vp, ci, ci, ci, ci, cf, vp, vp, vp]
     for name in ("bv_verify_probs", "tv_verify_probs"):
         getattr(lib, name).argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp]
     for name in ("bv_verify_lse", "tv_verify_lse"):
@@ -310,6 +311,32 @@ def bv_sample_draft(logits, uniforms, temperature: float = 1.0, want_lse: bool =
         _check(lib.bv_sample_draft(logits.data_ptr(), uniforms.data_ptr(), rows, V, _dtype_code(logits),
                                    float(temperature), tokens.data_ptr(), lse.data_ptr() if want_lse else None,
                                    st.cuda_stream))
+    return tokens, lse
+
+
+def bv_draft_chain(draft_table, first_tokens, uniforms, temperature: float = 1.0, stream=None):
+    """The whole drafting step for a last-token table model: draft_table CUDA [V, V] float32 or bfloat16,
+    first_tokens CUDA int32 [B], uniforms CUDA float32 [gamma, B]; returns (tokens int32 [B, gamma],
+    lse float32 [B, gamma]) from one launch."""
+    lib = load_library()
+    V = draft_table.shape[0]
+    if draft_table.dim() != 2 or draft_table.shape[1] != V or not draft_table.is_cuda or not draft_table.is_contiguous():
+        raise ValueError("draft_table must be a contiguous CUDA tensor [V, V]")
+    B = first_tokens.shape[0]
+    if first_tokens.dtype != torch.int32 or not first_tokens.is_cuda or not first_tokens.is_contiguous() or first_tokens.dim() != 1:
+        raise ValueError("first_tokens must be a contiguous CUDA int32 tensor [B]")
+    if (uniforms.dim() != 2 or uniforms.shape[1] != B or uniforms.dtype != torch.float32 or not uniforms.is_cuda
+            or not uniforms.is_contiguous()):
+        raise ValueError("uniforms must be a contiguous CUDA float32 tensor [gamma, B]")
+    gamma = uniforms.shape[0]
+    dev = draft_table.device
+    tokens = torch.empty((B, gamma), dtype=torch.int32, device=dev)
+    lse = torch.empty((B, gamma), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        s = stream if stream is not None else torch.cuda.current_stream(dev)
+        _check(lib.bv_draft_chain(draft_table.data_ptr(), first_tokens.data_ptr(), uniforms.data_ptr(), B, gamma, V,
+                                  _dtype_code(draft_table), float(temperature), tokens.data_ptr(), lse.data_ptr(),
+                                  s.cuda_stream))
     return tokens, lse
 
 

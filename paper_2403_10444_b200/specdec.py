@@ -3,8 +3,8 @@ models whose next-token logits depend on the last token only (two [V, V] tables 
 
     python -m paper_2403_10444_b200.specdec [--V 32768] [--B 64] [--gammas 2,4,8] [--iterations 32]
 
-Each iteration drafts gamma tokens autoregressively with ``bv_sample_draft`` (which also leaves every
-draft row's log-normaliser), looks up the target rows along the drafted path (the stand-in for the
+Each iteration drafts gamma tokens autoregressively with ``bv_draft_chain`` (one launch; or gamma calls of
+``bv_sample_draft``), which also leaves every draft row's log-normaliser, looks up the target rows along the drafted path (the stand-in for the
 parallel scoring pass of the large model), and verifies the block with ``bv_verify_lse`` (Block
 Verification, Algorithm 2), ``bv_verify``, ``tv_verify`` (Token Verification, Algorithm 1) or ``tv_verify_lse``.  The
 accepted tokens and the correction token extend every sequence, whose last token is the context of the
@@ -32,7 +32,7 @@ ALGOS = ("block_lse", "block", "token", "token_lse")
 
 def run(target_table: torch.Tensor, draft_table: torch.Tensor, first_tokens: torch.Tensor,
         u_draft: torch.Tensor, u_verify: torch.Tensor, gamma: int, temperature: float = 1.0,
-        algo: str = "block_lse", graph: bool = False) -> Dict[str, torch.Tensor]:
+        algo: str = "block_lse", graph: bool = False, chain: bool = True) -> Dict[str, torch.Tensor]:
     """Run ``u_draft.shape[0]`` iterations of Algorithm 3 for ``first_tokens.shape[0]`` sequences.
 
     target_table, draft_table: CUDA [V, V] float32 or bfloat16 (row t = logits after token t; -inf
@@ -44,9 +44,10 @@ def run(target_table: torch.Tensor, draft_table: torch.Tensor, first_tokens: tor
 
     Every step of an iteration has fixed shapes and runs on the device without a host round trip
     (the iteration number lives in a device counter), so with ``graph=True`` one iteration is
-    captured in a CUDA graph and replayed: the 5 gamma + 12 launches of an iteration then cost one
-    graph launch instead of one driver call each.  Data faults are looked for once, after the last
-    iteration.
+    captured in a CUDA graph and replayed: the launches of an iteration then cost one graph launch
+    instead of one driver call each.  Data faults are looked for once, after the last iteration.
+    ``chain``: the gamma drafted tokens of an iteration come from one launch of ``bv_draft_chain``
+    (default) instead of gamma calls of ``bv_sample_draft`` with their look-ups and copies.
     """
     if algo not in ALGOS:
         raise ValueError("algo must be one of %s" % (ALGOS,))
@@ -77,16 +78,24 @@ def run(target_table: torch.Tensor, draft_table: torch.Tensor, first_tokens: tor
         ud = u_draft.index_select(0, it)[0]                        # [gamma, B]
         uv = u_verify.index_select(0, it)[0]                       # [B, gamma+2]
         # drafting step: X_1..X_gamma ~ M_s autoregressively, keeping the conditional rows
-        last = cur
-        for i in range(gamma):
-            rows = draft_table.index_select(0, last)
-            tok, row_lse = bv.bv_sample_draft(rows, ud[i], temperature)
-            draft_logits[:, i] = rows
-            lse[:, i] = row_lse
-            toks[:, i] = tok
-            last = tok.to(torch.int64)
+        if chain:
+            # (one launch for the whole chain; the rows it went through are gathered afterwards)
+            tok, row_lse = bv.bv_draft_chain(draft_table, cur.to(torch.int32), ud.contiguous(), temperature)
+            toks.copy_(tok)
+            lse.copy_(row_lse)
+            path = torch.cat([cur[:, None], toks.to(torch.int64)], dim=1)
+            torch.index_select(draft_table, 0, path[:, :gamma].reshape(-1), out=draft_logits.view(B * gamma, V))
+        else:
+            last = cur
+            for i in range(gamma):
+                rows = draft_table.index_select(0, last)
+                tok, row_lse = bv.bv_sample_draft(rows, ud[i], temperature)
+                draft_logits[:, i] = rows
+                lse[:, i] = row_lse
+                toks[:, i] = tok
+                last = tok.to(torch.int64)
+            path = torch.cat([cur[:, None], toks.to(torch.int64)], dim=1)
         # the large model's conditional rows along the drafted path, gamma + 1 of them
-        path = torch.cat([cur[:, None], toks.to(torch.int64)], dim=1)
         torch.index_select(target_table, 0, path.reshape(-1), out=target_logits.view(B * (gamma + 1), V))
         if algo == "block_lse":
             out, out_len = bv.bv_verify_lse(target_logits, draft_logits, toks, uv, lse, temperature)
@@ -144,6 +153,7 @@ def main():
     ap.add_argument("--seed", type=int, default=7)
     ap.add_argument("--top-p", type=float, default=0.0, help="mask both models' rows to their top-p nucleus")
     ap.add_argument("--graph", action="store_true", help="replay one captured iteration as a CUDA graph")
+    ap.add_argument("--no-chain", action="store_true", help="draft with gamma sampler calls instead of one chain launch")
     args = ap.parse_args()
     bv.load_library()
     tt, dt = wl.markov_models(args.V, "bf16", args.seed, 2.0, args.draft_sigma, 1.1, "cuda")
@@ -153,15 +163,15 @@ def main():
     for gamma in [int(x) for x in args.gammas.split(",")]:
         ud, uv = wl.loop_uniforms(args.iterations, args.B, gamma, args.seed + gamma, "cuda")
         for algo in ALGOS:
-            run(tt, dt, first, ud[:2], uv[:2], gamma, args.temperature, algo, args.graph)       # warm-up
+            run(tt, dt, first, ud[:2], uv[:2], gamma, args.temperature, algo, args.graph, not args.no_chain)       # warm-up
             torch.cuda.synchronize()
             t0 = time.perf_counter()
-            res = run(tt, dt, first, ud, uv, gamma, args.temperature, algo, args.graph)
+            res = run(tt, dt, first, ud, uv, gamma, args.temperature, algo, args.graph, not args.no_chain)
             torch.cuda.synchronize()
             dt_s = time.perf_counter() - t0
             print(json.dumps({"V": args.V, "B": args.B, "gamma": gamma, "algo": algo,
                               "iterations": args.iterations, "draft_sigma": args.draft_sigma,
-                              "temperature": args.temperature, "top_p": args.top_p or None, "graph": args.graph,
+                              "temperature": args.temperature, "top_p": args.top_p or None, "graph": args.graph, "chain": not args.no_chain,
                               "block_efficiency": round(block_efficiency(res), 4),
                               "tokens": int(res["lengths"].sum().item()),
                               "ms_per_iteration": round(dt_s / args.iterations * 1e3, 3),

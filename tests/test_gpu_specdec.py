@@ -160,3 +160,56 @@ def test_nucleus_masked_rows_through_the_loop(algo, oalgo):
         for x in got:
             assert torch.isfinite(tt[prev, x]), "a token outside the target model's nucleus was emitted"
             prev = x
+
+
+@pytest.mark.parametrize("dtype,V,B,gamma,T", [("bf16", 4096, 40, 6, 0.9), ("f32", 1024, 7, 3, 1.3), ("bf16", 32768, 300, 8, 0.8), ("f32", 8, 5, 10, 1.0)])
+def test_draft_chain_equals_the_sampler_called_step_by_step(dtype, V, B, gamma, T):
+    # one launch for the whole chain against gamma calls of bv_sample_draft with the look-ups in between
+    # (bit for bit), and against the oracle's drafting step applied step by step
+    import paper_2403_10444_b200 as bv
+    tt, dt = wl.markov_models(V, dtype, 61, 2.0, 1.0, 1.1 if V > 8 else 0.0, "cuda")
+    g = torch.Generator(device="cuda").manual_seed(62)
+    first = torch.randint(0, V, (B,), generator=g, device="cuda", dtype=torch.int32)
+    u = torch.rand((gamma, B), generator=g, device="cuda")
+    tok, lse = bv.bv_draft_chain(dt, first, u, T)
+    last = first.to(torch.int64)
+    dt_np = to_numpy_logits(dt.cpu())
+    last_np = first.cpu().numpy().astype(np.int64)
+    safe = np.ones(B, bool)
+    for i in range(gamma):
+        t_i, l_i = bv.bv_sample_draft(dt.index_select(0, last), u[i].contiguous(), T)
+        assert torch.equal(t_i, tok[:, i]) and torch.equal(l_i.view(torch.int32), lse[:, i].contiguous().view(torch.int32))
+        want, want_lse, margin = oracle.sample_rows(dt_np[last_np], u[i].cpu().numpy(), T)
+        safe &= margin > 1e-6                      # (a sequence that parts ways at a near-tie is not followed further)
+        got = tok[:, i].cpu().numpy()
+        assert (got[safe] == want[safe]).all()
+        assert np.abs(lse[:, i].cpu().numpy()[safe] - want_lse[safe]).max() < 3e-6
+        last, last_np = t_i.to(torch.int64), got.astype(np.int64)
+    assert safe.sum() >= 0.8 * B       # (a uniform within 1e-6 of an edge of its cell: about 1 % of the draws at V = 32768)
+
+
+def test_draft_chain_ends_a_sequence_at_a_token_it_cannot_follow():
+    import paper_2403_10444_b200 as bv
+    V, B, gamma = 16, 4, 5
+    dt = torch.zeros((V, V), device="cuda")
+    dt[3, :] = float("-inf")                       # nothing can follow token 3
+    dt[:, 3] += 50.0                               # ... which every other row produces almost surely
+    first = torch.tensor([0, 3, V, 5], dtype=torch.int32, device="cuda")     # sequence 2 starts outside the vocabulary
+    u = torch.full((gamma, B), 0.5, device="cuda")
+    tok, lse = bv.bv_draft_chain(dt, first, u, 1.0)
+    tok, lse = tok.cpu(), lse.cpu()
+    assert tok[0].tolist() == [3, -1, -1, -1, -1] and torch.isnan(lse[0, 1:]).all() and not torch.isnan(lse[0, 0])
+    assert tok[1].tolist() == [-1] * 5 and tok[2].tolist() == [-1] * 5 and torch.isnan(lse[1:3]).all()
+    assert tok[3].tolist() == [3, -1, -1, -1, -1]
+
+
+@pytest.mark.parametrize("algo", ["block_lse", "token"])
+def test_loop_with_and_without_the_chain_kernel_generates_the_same_tokens(algo):
+    V, B, N, gamma = 4096, 24, 7, 5
+    tt, dt = wl.markov_models(V, "bf16", 71, 2.0, 1.0, 1.1, "cuda")
+    ud, uv = wl.loop_uniforms(N, B, gamma, 72, "cuda")
+    first = torch.arange(B, dtype=torch.int32, device="cuda")
+    a = specdec.run(tt, dt, first, ud, uv, gamma, 0.9, algo, chain=True)
+    b = specdec.run(tt, dt, first, ud, uv, gamma, 0.9, algo, chain=False)
+    for k in ("tokens", "lengths", "tau", "drafted"):
+        assert torch.equal(a[k], b[k]), k
