@@ -470,7 +470,7 @@ TRAFFIC_BYTES = {
     ("c4", "token", "verify_flow_kernel"): 828606208,
     ("c4", "greedy", "verify_flow_kernel"): 2582993920,
     ("c4", "block_lse", "verify_flow_kernel"): 1511270144,
-    ("c4", "sample", "sample_rows_kernel"): 1058036736,
+    ("c4", "sample", "sample_rows_kernel"): 1058068736,
     ("c4", "block_probs", "verify_flow_kernel"): 350500352,
     ("c4", "token_probs", "verify_flow_kernel"): 265098496,
 }
