@@ -327,6 +327,9 @@ int bv_stream_status(void* stream);
  *   "flow_chunks", "flow_pieces", "flow_ctas", "flow_depth"   work-item shape of the flow kernel
  *   "flow_keep_l2"  1: the lines a first sweep loads stay in L2 at normal priority for the row's second
  *                   sweep (default 0: every load of the flow kernel streams past L2, which measured faster)
+ *   "flow_fine"     n > 0: Block Verification cuts the rows of the last n sequences of the batch into the finer
+ *                   chunks that last target rows get, so that the launch ends on short items (default 0:
+ *                   none; it helped only where most drafted tokens are accepted)
  *   "wait_limit"    polls after which a bounded device-side wait gives up (tests)
  *   "never_signal"  tests: the flow kernel's workers never report an item as swept, so its waits
  *                   run out and the call ends with BV_ERR_TIMEOUT

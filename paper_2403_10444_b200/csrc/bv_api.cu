@@ -28,6 +28,7 @@ struct Options {
     int cluster = 0;       // cluster width of the cluster / stream kernels (1, 2, 4, 8); 0: chosen by shape
     int max_clusters = 0;  // cap on the clusters launched; 0: none
     int flow_chunks = 0, flow_pieces = 0, flow_ctas = 0, flow_depth = 0;   // 0: chosen by shape
+    int flow_fine = 0;     // > 0: this many blocks at the end of the batch have their rows cut into the finer chunks
     int flow_keep_l2 = 0;  // 1: the lines of a first sweep stay in L2 at normal priority; 0: every load streams past L2
     int wait_limit = 0;    // polls after which a bounded device-side wait gives up; 0: the built-in limits
     int never_signal = 0;  // test switch: the flow kernel's workers never report an item as swept
@@ -259,7 +260,8 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             const int chunks = (opt.flow_chunks >= 1 && opt.flow_chunks <= bv::kFlowMaxChunks) ? opt.flow_chunks : 0;
             const int pieces = (opt.flow_pieces >= 1 && opt.flow_pieces <= 8) ? opt.flow_pieces : 0;
             // (with supplied draft normalisers a first-sweep item streams one row, not two)
-            const bv::FlowPlan plan = bv::flow_plan(units, B, gamma, nctas, prm.lse_d == nullptr, chunks, pieces, algo == bv::kTokenVerify, prm.probs != 0);
+            bv::FlowPlan plan = bv::flow_plan(units, B, gamma, nctas, prm.lse_d == nullptr, chunks, pieces, algo == bv::kTokenVerify, prm.probs != 0);
+            if (opt.flow_fine > 0 && algo != bv::kTokenVerify && !prm.probs && plan.nch_late > plan.nch) plan.fine_from = opt.flow_fine < B ? B - opt.flow_fine : 0;
             size_t zero_bytes = 0;
             const size_t need = bv::flow_scratch_bytes(B, gamma, plan, &zero_bytes);
             StreamSlot* slot = nullptr;
@@ -553,6 +555,7 @@ int bv_set_option(const char* name, int value) {
     else if (!std::strcmp(name, "flow_ctas")) g_opt.flow_ctas = value;
     else if (!std::strcmp(name, "flow_depth")) g_opt.flow_depth = value;
     else if (!std::strcmp(name, "flow_keep_l2")) g_opt.flow_keep_l2 = value;
+    else if (!std::strcmp(name, "flow_fine")) g_opt.flow_fine = value;
     else if (!std::strcmp(name, "wait_limit")) g_opt.wait_limit = value;
     else if (!std::strcmp(name, "never_signal")) g_opt.never_signal = value;
     else return BV_ERR_INVALID_ARG;

@@ -350,7 +350,7 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             __syncwarp();
             int last = 0;
             if (lane == 0) {
-                if (!PROBS && d.kind == kSweep1) last = atomicAdd(&fl.row_cnt[d.ri], 1u) == static_cast<unsigned>(f_nch_row(fl, d.ri % (g + 1), g)) - 1u;
+                if (!PROBS && d.kind == kSweep1) last = atomicAdd(&fl.row_cnt[d.ri], 1u) == static_cast<unsigned>(f_nch_row(fl, d.ri / (g + 1), d.ri % (g + 1), g)) - 1u;
                 else last = atomicAdd(&fl.s2_cnt[d.ri], 1u) == static_cast<unsigned>(fl.np) - 1u;
             }
             last = __shfl_sync(0xffffffffu, last, 0);
@@ -388,12 +388,16 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
         };
         // the first-sweep item of ticket t
         auto sweep1_desc = [&](unsigned t, FlowDesc& d) {
-            const int nch = fl.nch;
-            const int ch = static_cast<int>(t % nch);
+            // (the blocks from fine_from on are cut into nch_late chunks per row: Block Verification only)
+            const unsigned t_coarse = static_cast<unsigned>(fl.fine_from) * g * fl.nch;
+            const bool fine = !fl.tv && t >= t_coarse;
+            const int nch = fine ? fl.nch_late : fl.nch;
+            const unsigned tt = fine ? t - t_coarse : t;
+            const int ch = static_cast<int>(tt % nch);
             // Block Verification goes block by block (a block's rows are wanted together); Algorithm 1
             // row by row over all blocks (a block's next row matters only if the one before passed)
-            const int r = fl.tv ? static_cast<int>(t / nch) / cx.B : static_cast<int>(t / nch) % g;
-            const int b = fl.tv ? static_cast<int>(t / nch) % cx.B : static_cast<int>(t / nch) / g;
+            const int r = fl.tv ? static_cast<int>(tt / nch) / cx.B : static_cast<int>(tt / nch) % g;
+            const int b = fl.tv ? static_cast<int>(tt / nch) % cx.B : (fine ? fl.fine_from : 0) + static_cast<int>(tt / nch) / g;
             const int ri = b * (g + 1) + r;
             // (with supplied draft normalisers the first sweep has nothing to learn from the draft row)
             d.kind = kSweep1; d.ri = ri; d.ch = ch; d.have_q = prm.lse_d == nullptr;
@@ -792,7 +796,10 @@ void flow_scratch_layout(void* base, int B, int gamma, const FlowPlan& plan, Flo
     fl->nch = plan.nch;
     fl->keep_l2 = 0;
     fl->part_stride = plan.part_stride();
-    fl->total_s1 = plan.probs ? 0u : static_cast<unsigned>(B) * (plan.tv_spec > 0 ? plan.tv_spec : gamma) * plan.nch;
+    fl->fine_from = plan.fine_from;
+    fl->total_s1 = plan.probs ? 0u
+                 : plan.tv_spec > 0 ? static_cast<unsigned>(B) * plan.tv_spec * plan.nch
+                 : static_cast<unsigned>(plan.fine_from) * gamma * plan.nch + static_cast<unsigned>(B - plan.fine_from) * gamma * plan.nch_late;
     fl->tail_mode = plan.tail_mode;
     fl->nch_late = plan.nch_late;
     fl->np = plan.np;
@@ -839,6 +846,7 @@ FlowPlan flow_plan(long long units, int B, int gamma, long long nctas, bool pair
     // time (the fewest bytes); a smaller one starts all of a block's candidates at once.
     pl.tail_mode = 0;
     if (probs) pl.tail_mode = static_cast<long long>(B) * pl.np >= 2 * nctas ? 2 : 1;
+    pl.fine_from = B;
     pl.tv_spec = 0;
     pl.tv_ahead = 1;
     if (token_verify) {

@@ -111,8 +111,10 @@ __device__ __forceinline__ RowZ load_rowz(const RowZ* p) {
 // chunks of row r of a block in its first sweep
 // (rows whose first sweep is asked for on demand - a last target row, a row of Algorithm 1 beyond the
 // ones swept from the start - are cut into nch_late chunks)
-__device__ __forceinline__ int f_nch_row(const FlowScratch& fl, int r, int g) {
-    return (r == g || (fl.tv && r >= fl.tv_spec)) ? fl.nch_late : fl.nch;
+// (and so are all rows of the blocks from fine_from on, the last ones to be started: the launch ends
+// a chunk's sweep after its last ticket, so the last chunks are short ones)
+__device__ __forceinline__ int f_nch_row(const FlowScratch& fl, int b, int r, int g) {
+    return (r == g || b >= fl.fine_from || (fl.tv && r >= fl.tv_spec)) ? fl.nch_late : fl.nch;
 }
 
 struct FlowCtx {
@@ -598,7 +600,7 @@ template <int DT>
 __device__ void f_row_complete(const Params& prm, const FlowScratch& fl, const FlowCtx& cx, int b, int r, int lane) {
     const int g = cx.g;
     const size_t rowi = static_cast<size_t>(b) * (g + 1) + r;
-    const int nch = f_nch_row(fl, r, g);
+    const int nch = f_nch_row(fl, b, r, g);
     const bool have_q = r < g;
     // loads in flight together: the chunks' sums, the drafted token
     RowZ z; z.MP = kNoRef; z.ZP = 0.0; z.MQ = kNoRef; z.ZQ = 0.0;

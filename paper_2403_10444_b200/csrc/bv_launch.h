@@ -66,8 +66,9 @@ struct FlowScratch {
     int nch;              // chunks per row in the first sweep of rows 0 .. gamma-1 (1 .. kFlowMaxChunks)
     int part_stride;      // chunk results kept per row: max(nch, nch_late)
     int nch_late;         // chunks of a last target row, whose first sweep is asked for on demand
+    int fine_from;        // Block Verification: rows 0 .. gamma-1 of the blocks from this one on are cut into nch_late chunks (B: none)
     int np;               // pieces per row in the second sweep (1 .. kFlowMaxChunks)
-    unsigned total_s1;    // first-sweep tickets: B gamma nch
+    unsigned total_s1;    // first-sweep tickets: fine_from gamma nch + (B - fine_from) gamma nch_late
     unsigned zero_words;  // 32-bit words at the start of the scratch area (from `counters` on) that start and end at zero
     int depth;            // flow kernel: descriptors a CTA may have handed to its workers and not yet seen swept
     int segs;             // residual totals kept per row
@@ -84,6 +85,7 @@ struct FlowPlan {
     int tv_ahead;         // Token Verification: rows asked for beyond the last test that passed
     bool probs;           // the rows hold probabilities: no first sweep
     int tail_mode;        // see FlowScratch
+    int fine_from;        // see FlowScratch
     int part_stride() const { return nch > nch_late ? nch : nch_late; }
 };
 // units: 16-byte vectors per row; pair_items: false when the first sweep streams one row per item

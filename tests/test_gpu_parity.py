@@ -90,6 +90,16 @@ def test_flow_chunk_counts(chunks, bv_options):
     parity_case(random_inputs(21, 4, 16384, "bf16", seed=chunks + 1), oracle.BLOCK_VERIFY)
 
 
+@pytest.mark.parametrize("fine", [1, 5, 100])
+def test_flow_finer_chunks_for_the_last_sequences(fine, bv_options):
+    bv_options("kernel", KERNELS["flow"])
+    bv_options("flow_fine", fine)
+    parity_case(random_inputs(21, 4, 65536, "bf16", seed=fine), oracle.BLOCK_VERIFY)
+    parity_case(wl.make_inputs(wl.scaled(wl.CONFIGS["c4"], B=12), "cuda"), oracle.BLOCK_VERIFY)
+    bv_options("flow_ctas", 3)
+    parity_case(random_inputs(9, 6, 131072, "f32", seed=fine + 1), oracle.BLOCK_VERIFY)
+
+
 @pytest.mark.parametrize("algo", ALGOS)
 def test_more_sequences_than_resident_clusters(algo):
     parity_case(random_inputs(700, 3, 512, "f32", seed=3), algo)

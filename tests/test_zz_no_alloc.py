@@ -44,7 +44,7 @@ def _flow_kernel_with_default_shapes(bv_options):
     # the entry point without allocations always runs the flow kernel with the work-item shape chosen by
     # problem size: the call it is compared with must do the same, whatever the environment set
     bv_options("kernel", 1)
-    for name in ("flow_chunks", "flow_pieces", "flow_ctas", "flow_depth", "flow_keep_l2"):
+    for name in ("flow_chunks", "flow_pieces", "flow_ctas", "flow_depth", "flow_keep_l2", "flow_fine"):
         bv_options(name, 0)
 
 
