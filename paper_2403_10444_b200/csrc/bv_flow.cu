@@ -483,13 +483,25 @@ __global__ void __launch_bounds__(kFAllThreads, 2) verify_flow_kernel(const Para
             if (q >= depth && !mbar_wait_relaxed(smem_u32(&sh.done[(q - depth) % kFDesc]), static_cast<uint32_t>((q - depth) / kFDesc) & 1u, prm.status, 100, lim_nap)) { failed = true; break; }
             FlowDesc d;
             d.kind = kExit;
-            // (a) a piece of a row that waits for its second sweep: they are few and others wait for them
-            int t = claim(seen_rows, seen_pieces, kCtrPieces, fl.np, held);
-            if (t >= 0) {
+            // (a) a piece of a row that waits for its second sweep: they are few and others wait for them;
+            // (b) a chunk of a row whose first sweep turned out to be wanted (a last target row, or the
+            // next rows of Algorithm 1 after a test has passed).  Algorithm 1 looks at (b) first: there a
+            // second sweep ends its block and nothing waits for it, while the next row of a block that
+            // keeps accepting is what the launch waits for in the end.
+            int t = -1;
+            bool is_piece = false;
+            if (fl.tv) {
+                t = claim(seen_late, seen_chunks, kCtrLateChunks, fl.nch_late, held_late);
+                if (t < 0) { t = claim(seen_rows, seen_pieces, kCtrPieces, fl.np, held); is_piece = t >= 0; }
+            } else {
+                t = claim(seen_rows, seen_pieces, kCtrPieces, fl.np, held);
+                is_piece = t >= 0;
+                if (t < 0) t = claim(seen_late, seen_chunks, kCtrLateChunks, fl.nch_late, held_late);
+            }
+            if (t >= 0 && is_piece) {
                 if (!piece_desc(t, d)) { failed = true; break; }
                 if (lane == 0) ++seen_pieces;
-            } else if ((t = claim(seen_late, seen_chunks, kCtrLateChunks, fl.nch_late, held_late)) >= 0) {
-                // (b) a chunk of a last target row that turned out to be wanted
+            } else if (t >= 0) {
                 if (!late_desc(t, d)) { failed = true; break; }
                 if (lane == 0) ++seen_chunks;
             } else if (!exhausted) {
