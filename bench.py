@@ -466,13 +466,13 @@ def finish(args, w, world, value, ms_per_step, kernel_ms, clocks, e2e, launches,
 # ncu capture of this command at full size that profiles/ summarises; None for a workload or
 # kernel with no capture.
 TRAFFIC_BYTES = {
-    ("c4", "block", "verify_flow_kernel"): 2563923968,
-    ("c4", "token", "verify_flow_kernel"): 828606208,
-    ("c4", "greedy", "verify_flow_kernel"): 2582993920,
-    ("c4", "block_lse", "verify_flow_kernel"): 1511270144,
-    ("c4", "sample", "sample_rows_kernel"): 1058068736,
-    ("c4", "block_probs", "verify_flow_kernel"): 350500352,
-    ("c4", "token_probs", "verify_flow_kernel"): 265098496,
+    ("c4", "block", "verify_flow_kernel"): 2544254464,
+    ("c4", "token", "verify_flow_kernel"): 826027264,
+    ("c4", "greedy", "verify_flow_kernel"): 2567559424,
+    ("c4", "block_lse", "verify_flow_kernel"): 1486017536,
+    ("c4", "sample", "sample_rows_kernel"): 1058338048,
+    ("c4", "block_probs", "verify_flow_kernel"): 350525696,
+    ("c4", "token_probs", "verify_flow_kernel"): 264830208,
 }
 
 

@@ -444,7 +444,7 @@ __device__ void f_tv_row_done(const Params& prm, const FlowScratch& fl, const Fl
         const double ratio = __ldcg(&fl.ratio[row0 + r]);     // 0 for a row with a data fault: the test fails
         const double h = fmin(ratio, 1.0);
         const bool pass = h > 0.0 && static_cast<double>(prm.uni[static_cast<size_t>(b) * (g + 2) + r]) <= h;
-        // the verdict first, then the fact that it is in: whoever sees the second sees the first
+        // the decision first, then the fact that it is in: whoever sees the second sees the first
         if (pass) atomicOr(&fl.tv_acc[b], 1ull << r);
         __threadfence();
         atomicOr(&fl.tv_done[b], 1ull << r);
