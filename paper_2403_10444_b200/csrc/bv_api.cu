@@ -269,6 +269,8 @@ int run_device(int algo, const void* tgt, const void* drf, const int32_t* tok, c
             char* scratch = static_cast<char*>(slot->ws) + 256;
             bv::FlowScratch fl;
             bv::flow_scratch_layout(scratch, B, gamma, plan, &fl);
+            // (with every position swept the second sweeps are the larger half of the launch and never wait for one another: deeper measured better)
+            if (prm.out_p || prm.out_S || prm.out_h || prm.out_lse_t || prm.out_lse_d) fl.depth = 3;
             if (opt.flow_depth >= 2 && opt.flow_depth <= 6) fl.depth = opt.flow_depth;
             fl.keep_l2 = opt.flow_keep_l2 == 1;
             // The kernel leaves its counters and flags at zero when it ends, so they are cleared here only
