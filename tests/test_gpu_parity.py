@@ -101,6 +101,27 @@ def test_flow_finer_chunks_for_the_last_sequences(fine, bv_options):
 
 
 @pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("kernel", ["flow", "small", "default"])
+@pytest.mark.parametrize("dtype,V", [("f32", 1 << 21), ("bf16", (1 << 21) + 8), ("bf16", (1 << 21) + 1)])
+def test_very_large_vocabularies(dtype, V, kernel, algo, bv_options):
+    # two million logits a row: chunk, piece and segment ranges far beyond the benchmark's sizes; the odd V
+    # takes the element-wise path
+    if kernel != "default":
+        if V % 8:
+            pytest.skip("the flow and small-batch kernels take rows of whole 16-byte vectors")
+        bv_options("kernel", KERNELS[kernel])
+    parity_case(random_inputs(3, 2, V, dtype, seed=V % 97, T=0.9), algo)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_many_short_sequences(algo, bv_options):
+    # far more sequences than CTAs, rows of a few vectors: every counter and queue index of the flow kernel
+    bv_options("kernel", KERNELS["flow"])
+    parity_case(random_inputs(6000, 3, 64, "bf16", seed=5, sigma_d=0.5), algo)
+    parity_case(random_inputs(3000, 1, 16, "f32", seed=6), algo)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
 def test_more_sequences_than_resident_clusters(algo):
     parity_case(random_inputs(700, 3, 512, "f32", seed=3), algo)
 

@@ -55,11 +55,11 @@ def test_probabilities_match_the_oracle(algo, name, B, gamma):
 
 @pytest.mark.parametrize("kernel", [1, 4])         # the flow kernel, the small-batch kernel
 @pytest.mark.parametrize("algo", ["block", "token"])
-@pytest.mark.parametrize("V", [8, 24, 1000, 4104, 33000])
+@pytest.mark.parametrize("V", [8, 24, 1000, 4104, 33000, (1 << 21) + 8])
 def test_ragged_vocabularies(algo, V, kernel, bv_options):
     import paper_2403_10444_b200 as bv
     bv_options("kernel", kernel)
-    w = wl.scaled(wl.CONFIGS["c3"], B=17, gamma=3, V=V)
+    w = wl.scaled(wl.CONFIGS["c3"], B=17 if V < (1 << 20) else 3, gamma=3, V=V)
     run_case(algo, probs_inputs(w), "probs ragged V=%d %s kernel %d" % (V, algo, kernel))
     assert bv.bv_last_kernel() == kernel
 

@@ -40,7 +40,8 @@ def check(logits, uniforms, T):
 
 @pytest.mark.parametrize("rows,V,dtype,T", [(64, 256000, "bf16", 1.0), (300, 32000, "f32", 0.8),
                                             (40, 152064, "bf16", 0.8), (33, 8, "f32", 1.0),
-                                            (500, 1024, "bf16", 2.5), (7, 4104, "f32", 0.3)])
+                                            (500, 1024, "bf16", 2.5), (7, 4104, "f32", 0.3),
+                                            (5, 1 << 21, "f32", 1.0), (3, (1 << 21) + 8, "bf16", 0.7)])
 def test_sampler_matches_the_oracle(rows, V, dtype, T):
     g = torch.Generator().manual_seed(rows + V)
     z = torch.randn((rows, V), generator=g) * 3.0
