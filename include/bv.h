@@ -324,7 +324,9 @@ int bv_stream_status(void* stream);
  *   "small_bytes"   logit megabytes up to which the small-batch kernel is the default
  *   "cluster"       cluster width of the cluster / streaming kernels (1, 2, 4, 8)
  *   "max_clusters"  cap on the clusters those kernels launch
- *   "flow_chunks", "flow_pieces", "flow_ctas", "flow_depth"   work-item shape of the flow kernel
+ *   "flow_chunks", "flow_pieces", "flow_ctas", "flow_depth"   work-item shape of the flow kernel (chunks per row in
+ *                   the first sweep, pieces per row in the second, CTAs launched, descriptors a CTA hands to its
+ *                   workers ahead of the sweep: 2 for Block Verification, 3 for Algorithm 1 and with diagnostic outputs)
  *   "flow_keep_l2"  1: the lines a first sweep loads stay in L2 at normal priority for the row's second
  *                   sweep (default 0: every load of the flow kernel streams past L2, which measured faster)
  *   "flow_fine"     n > 0: Block Verification cuts the rows of the last n sequences of the batch into the finer
